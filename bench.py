@@ -1,0 +1,420 @@
+#!/usr/bin/env python
+"""Benchmark of the semantic-pool hot path: queries/s, p50 latency, key-scan GB/s.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config C2] [--impl reference]
+
+One step = one pass of the whole hot path on one batch: append the rows committed since
+the last step (normalise + store), then one query call (normalise query, score every key,
+top-k, firing rule, depth, continuation gather).  Inputs are seeded and synthetic
+(paper_2608_03839_b200/workloads.py).  With N > 1 (torchrun) every rank serves its own
+pool (one pool per tenant; no data-path collective), so scaling is weak and `value` is
+the sum over ranks divided by the slowest rank's time.
+
+Prints ONE JSON line (rank 0).  `--impl reference` times the CPU oracle instead (rank 0
+only), on the same config, metric and unit.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2608_03839_b200 import workloads as W  # noqa: E402
+
+METRIC = "semantic_pool_queries_per_sec"
+UNIT = "queries/s"
+APPEND_ROWS = {"C1": 8, "C2": 8, "C3": 64, "C4": 512, "C5": 256}   # rows committed per step
+NOMINAL_HBM_GBS = 8000.0
+FALLBACK_HBM_GBS = 6650.0
+
+
+def env_int(name, default):
+    try:
+        return int(os.environ.get(name, default))
+    except ValueError:
+        return default
+
+
+def measured_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        try:
+            return json.load(open(p)), "measured"
+        except Exception:
+            pass
+    return {"hbm_gbs": FALLBACK_HBM_GBS, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}, \
+        "fallback"
+
+
+def ncu_traffic(config_name: str):
+    """DRAM bytes per scan launch from the committed ncu summary, if one exists."""
+    p = os.path.join(ROOT, "profiles", "traffic.json")
+    if os.path.exists(p):
+        try:
+            return json.load(open(p)).get(config_name)
+        except Exception:
+            return None
+    return None
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons through NVML while the timed region runs."""
+
+    def __init__(self, index: int, period_s: float = 0.02):
+        self.index, self.period = index, period_s
+        self.samples, self.reasons = [], set()
+        self.max_mhz = None
+        self._stop = threading.Event()
+        self._thr = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+        except Exception:
+            self.nv = None
+
+    def _run(self):
+        nv = self.nv
+        names = {}
+        for nm in ("GpuIdle", "ApplicationsClocksSetting", "SwPowerCap", "HwSlowdown", "SyncBoost",
+                   "SwThermalSlowdown", "HwThermalSlowdown", "HwPowerBrakeSlowdown",
+                   "DisplayClockSetting"):
+            v = getattr(nv, "nvmlClocksEventReason" + nm, None)
+            if v is None:
+                v = getattr(nv, "nvmlClocksThrottleReason" + nm, None)
+            if v is not None:
+                names[v] = nm
+        while not self._stop.is_set():
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+                try:
+                    r = nv.nvmlDeviceGetCurrentClocksEventReasons(self.h)
+                except Exception:
+                    r = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+                for bit, nm in names.items():
+                    if r & bit:
+                        self.reasons.add(nm)
+            except Exception:
+                pass
+            self._stop.wait(self.period)
+
+    def start(self):
+        if self.nv is not None:
+            self._thr = threading.Thread(target=self._run, daemon=True)
+            self._thr.start()
+
+    def stop(self) -> dict:
+        self._stop.set()
+        if self._thr is not None:
+            self._thr.join(timeout=2)
+        reasons = sorted(r for r in self.reasons if r != "GpuIdle")
+        med = float(np.median(self.samples)) if self.samples else None
+        return {"sm_mhz": med, "sm_max_mhz": self.max_mhz, "reasons": reasons,
+                "samples": len(self.samples)}
+
+
+# ------------------------------------------------------------------ workload ----
+
+def physical_device(local_rank: int) -> int:
+    vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+    if vis:
+        try:
+            return int(vis.split(",")[local_rank])
+        except Exception:
+            return local_rank
+    return local_rank
+
+
+def step_inputs(w: W.Workload, n_steps: int, rows: int, nq: int, device, seed: int):
+    """Rows committed and query states for every step, drawn around the pool's centroids."""
+    g = torch.Generator(device=device).manual_seed(0x5EED0000 + seed)
+    src = w if w.kind != "template" else w.scaled(kind="clustered", n_centroids=256)
+    C = src._centroids(device)
+    c = torch.randint(0, C.shape[0], (n_steps, rows), generator=g, device=device)
+    cq = torch.randint(0, C.shape[0], (n_steps, nq), generator=g, device=device)
+    states, queries = [], []
+    for s in range(n_steps):
+        st = C[c[s]] + src.sigma * torch.randn(rows, w.d, generator=g, device=device)
+        qq = C[cq[s]] + src.sigma * torch.randn(nq, w.d, generator=g, device=device)
+        states.append(st.to(torch.bfloat16))
+        queries.append(qq.to(torch.bfloat16))
+    toks = torch.randint(0, w.vocab, (n_steps, rows), generator=g, device=device, dtype=torch.int32)
+    return states, toks, queries
+
+
+def run_ours(args):
+    from paper_2608_03839_b200 import binding as B
+    import torch.distributed as dist
+
+    rank, world = env_int("RANK", 0), env_int("WORLD_SIZE", 1)
+    local = env_int("LOCAL_RANK", 0)
+    if world > 1:
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("nccl", device_id=torch.device(f"cuda:{local}"))
+    torch.cuda.set_device(local)
+    dev = torch.device(f"cuda:{local}")
+    w = W.CONFIGS[args.config]
+    nq = args.nq or w.nq
+    n0 = W.C5_START_ROWS if w.name == "C5" else w.n_rows
+    rows_step = APPEND_ROWS[w.name]
+    K, Wm = args.steps, args.warmup
+    total_steps = 2 * (Wm + K) + Wm + K     # device-timed pass, kernel-timed pass, e2e pass
+    cap = n0 + rows_step * total_steps + 8
+    pool = B.Pool(w.d, cap, max_nq=max(nq, 1), max_k=w.k, max_append=rows_step, device=local,
+                  max_traces=w.num_traces + total_steps + 8)
+    # fill the pool (not timed): seeded traces of the configuration
+    done = 0
+    for st, tk, tag in w.traces(dev):
+        if done >= n0:
+            break
+        if done + st.shape[0] > n0:
+            st, tk = st[: n0 - done].contiguous(), tk[: n0 - done].contiguous()
+        pool.append(st, tk, tag=tag)
+        done += st.shape[0]
+    torch.cuda.synchronize()
+    pr = B.QueryParams(k=w.k, theta=0.8, offset=2, depth_mode=B.DEPTH_FIXED, cont_len=w.cont_len,
+                       path=args.path)
+    n_in = min(Wm + K, 64)                   # distinct step inputs, cycled
+    states, toks, queries = step_inputs(w, n_in, rows_step, nq, dev, seed=rank)
+    out = B.QueryOut.empty(nq, w.k, w.cont_len, dev)
+    step_no = [0]
+
+    def step():
+        i = step_no[0] % n_in
+        pool.append(states[i], toks[i], tag=1_000_000 + step_no[0], new_trace=True)
+        pool.query(queries[i], pr, out=out)
+        step_no[0] += 1
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # ---- device-timed region: K steps, inputs resident in HBM ----------------------
+    for _ in range(Wm):
+        step()
+    barrier()
+    sampler = ClockSampler(physical_device(local))
+    sampler.start()
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(K + 1)]
+    launches0, rows0 = pool.launch_count, len(pool)
+    ev[0].record()
+    for s in range(K):
+        step()
+        ev[s + 1].record()
+    barrier()
+    clocks = sampler.stop()
+    launches = pool.launch_count - launches0
+    total_ms = ev[0].elapsed_time(ev[K])
+    lat = np.array([ev[s].elapsed_time(ev[s + 1]) for s in range(K)])
+    rows_mean = rows0 + rows_step * (K + 1) / 2.0
+    t = torch.tensor([total_ms], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    max_ms = float(t.item())
+    value = world * K * nq / (max_ms / 1e3)
+
+    # ---- the dominant kernel (key scan), timed by events around its launches ---------
+    pool.profile(True)
+    for _ in range(Wm):
+        step()
+    torch.cuda.synchronize()
+    pool.profile_read()
+    rows1 = len(pool)
+    for _ in range(K):
+        step()
+    torch.cuda.synchronize()
+    scan_ms = pool.profile_read(max_n=max(K, 1))
+    pool.profile(False)
+    rows_scan = rows1 + rows_step * (K + 1) / 2.0
+    scan_bytes = rows_scan * w.d * 2
+    peaks, peak_kind = measured_peaks()
+    scan_mean_ms = float(scan_ms.mean()) if len(scan_ms) else float("nan")
+    achieved = scan_bytes / (scan_mean_ms * 1e-3) / 1e9
+
+    # ---- end to end through the host-buffer entry points -----------------------------
+    h_states = [s.cpu().pin_memory() for s in states]
+    h_toks = [toks[i].cpu().pin_memory() for i in range(n_in)]
+    h_q = [q.cpu().pin_memory() for q in queries]
+    h_out = B.QueryOut.empty(nq, w.k, w.cont_len, "cpu")
+
+    def step_host():
+        i = step_no[0] % n_in
+        pool.append_host(h_states[i], h_toks[i], tag=1_000_000 + step_no[0], new_trace=True)
+        pool.query_host(h_q[i], pr, out=h_out)
+        step_no[0] += 1
+
+    for _ in range(Wm):
+        step_host()
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(K):
+        step_host()
+    e1.record()
+    barrier()
+    t2 = torch.tensor([e0.elapsed_time(e1)], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(t2, op=dist.ReduceOp.MAX)
+    e2e_value = world * K * nq / (float(t2.item()) / 1e3)
+    h2d = rows_step * w.d * 2 + rows_step * 4 + nq * w.d * 2
+    d2h = nq * w.k * (4 + 4 + 4 + 4 * w.cont_len) + nq * 4
+    stalled = pool.stats()["stalled"]
+
+    if rank == 0:
+        p50_ms = float(np.percentile(lat, 50))
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K,
+            "warmup": Wm, "ms_per_step": max_ms / K, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "bf16 keys, fp32 accumulate",
+            "data": "synthetic",
+            "config": {"workload": f"{w.name}: pool N={n0} x d={w.d} bf16, nq={nq}, k={w.k}, "
+                                   f"L={w.cont_len}, +{rows_step} rows appended per step",
+                       "pool_rows_start": rows0, "pool_rows_end": rows0 + rows_step * K,
+                       "append_rows_per_step": rows_step, "scan_path": args.path,
+                       "l2": "inputs exceed L2" if w.key_bytes(n0) > 2 * 126e6 else
+                             "pool fits in L2 (not a bandwidth datum)",
+                       "pools": "one independent pool per GPU"},
+            "p50_query_latency_us": p50_ms * 1e3,
+            "p90_query_latency_us": float(np.percentile(lat, 90)) * 1e3,
+            "min_query_latency_us": float(lat.min()) * 1e3,
+            "key_scan_gbs": rows_mean * w.d * 2 / (p50_ms * 1e-3) / 1e9,
+            "clocks": clocks,
+            "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d,
+                    "d2h_bytes_per_step": d2h},
+            "gpu_launches": int(launches),
+            "roofline": {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"],
+                         "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"],
+                         "peak_kind": peak_kind, "frac_of_nominal_8000": achieved / NOMINAL_HBM_GBS,
+                         "kernel": "key scan (score + per-CTA top-k)",
+                         "kernel_ms": scan_mean_ms, "bytes_per_launch": scan_bytes,
+                         "traffic": ncu_traffic(w.name)},
+            "device_stalled_flag": stalled,
+        }
+        if not args.no_cpu_baseline and world == 1:
+            line["cpu_baseline"] = cpu_baseline(w, n0, rows_step, nq, budget_s=args.cpu_budget)
+        print(json.dumps(line), flush=True)
+    pool.close()
+    if world > 1:
+        dist.destroy_process_group()
+
+
+# ---------------------------------------------------------------- CPU oracle ----
+
+def oracle_pool_for(w: W.Workload, n_rows: int):
+    import oracle
+    ora = oracle.OraclePool(w.d)
+    done = 0
+    for st, tk, tag in w.traces("cpu"):
+        if done >= n_rows:
+            break
+        if done + st.shape[0] > n_rows:
+            st, tk = st[: n_rows - done], tk[: n_rows - done]
+        ora.append(W.to_bits(st), tk.numpy(), tag=tag)
+        done += st.shape[0]
+    return ora
+
+
+def cpu_baseline(w, n0, rows_step, nq, budget_s=20.0, steps=None, warmup=1):
+    """Time the oracle as it stands on the host cores, on a bounded sample of the workload.
+
+    The sample is a prefix of the pool (whole traces) small enough that the run fits the
+    budget; each step appends `rows_step` rows and answers `nq_s` queries against it.
+    queries/s is scaled by the fraction of the pool's rows that was scanned.
+    """
+    import oracle
+    cores = oracle.num_threads()
+    # probe: cost per row-scan on a small pool
+    probe_rows = min(n0, max(2048, (1 << 26) // (w.d * 2)))
+    ora = oracle_pool_for(w, probe_rows)
+    q, _ = w.queries("cpu", nq=1)
+    qb = W.to_bits(q)
+    pr = oracle.QueryParams(k=w.k, theta=0.8, depth_mode=oracle.DEPTH_FIXED, cont_len=w.cont_len)
+    ora.query(qb, pr)
+    t0 = time.perf_counter()
+    ora.query(qb, pr)
+    per_row = (time.perf_counter() - t0) / probe_rows
+    n_steps = steps if steps is not None else 4
+    nq_s = min(nq, 4)
+    rows = int(min(n0, max(probe_rows, budget_s / max(per_row * nq_s * (n_steps + warmup), 1e-12))))
+    rows = max(w.rows_per_trace, rows // w.rows_per_trace * w.rows_per_trace)
+    rows = min(rows, n0)
+    if rows != probe_rows:
+        ora = oracle_pool_for(w, rows)
+    states, toks, queries = step_inputs(w, n_steps + warmup, rows_step, nq_s, "cpu", seed=0)
+    def step(i):
+        ora.append(W.to_bits(states[i]), toks[i].numpy(), tag=1_000_000 + i)
+        ora.query(W.to_bits(queries[i]), pr)
+    for i in range(warmup):
+        step(i)
+    t0 = time.perf_counter()
+    for i in range(warmup, warmup + n_steps):
+        step(i)
+    dt = time.perf_counter() - t0
+    frac = rows / n0
+    return {"value": n_steps * nq_s / dt * frac, "unit": UNIT, "cores": cores, "kind": "oracle",
+            "sample": f"{n_steps} steps x {nq_s} queries, each scoring {rows} of {n0} pool rows "
+                      f"(all d={w.d}) + full sort + gather; value scaled by {frac:.4g}",
+            "seconds": dt, "ms_per_step": dt / n_steps * 1e3}
+
+
+def run_reference(args):
+    rank = env_int("RANK", 0)
+    if rank != 0:
+        return
+    w = W.CONFIGS[args.config]
+    nq = args.nq or w.nq
+    n0 = W.C5_START_ROWS if w.name == "C5" else w.n_rows
+    cb = cpu_baseline(w, n0, APPEND_ROWS[w.name], nq, budget_s=args.cpu_budget * 4,
+                      steps=args.steps, warmup=args.warmup)
+    line = {"impl": "reference", "metric": METRIC, "value": cb["value"], "unit": UNIT,
+            "n_gpus": env_int("WORLD_SIZE", 1), "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": cb["ms_per_step"], "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": f"{w.name}: pool N={n0} x d={w.d} bf16, nq={nq}, k={w.k}, "
+                                   f"L={w.cont_len}, +{APPEND_ROWS[w.name]} rows appended per step"},
+            "cpu_baseline": {k: cb[k] for k in ("value", "unit", "cores", "kind", "sample")},
+            "e2e": {"value": cb["value"], "unit": UNIT, "h2d_bytes_per_step": 0,
+                    "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=None)
+    ap.add_argument("--warmup", type=int, default=None)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--config", default="C2", choices=sorted(W.CONFIGS))
+    ap.add_argument("--nq", type=int, default=0, help="override the configuration's nq")
+    ap.add_argument("--path", type=int, default=0, help="0 auto, 1 CUDA-core scan, 2 tensor scan")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--cpu-budget", type=float, default=20.0)
+    args = ap.parse_args()
+    if args.impl == "reference":
+        args.steps = 8 if args.steps is None else args.steps
+        args.warmup = 1 if args.warmup is None else args.warmup
+        run_reference(args)
+        return
+    default_steps = {"C1": 2000, "C2": 2000, "C3": 500, "C4": 200, "C5": 50}[args.config]
+    args.steps = default_steps if args.steps is None else args.steps
+    args.warmup = 10 if args.warmup is None else max(args.warmup, 3)
+    run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,215 @@
+/*
+ * oilbird.h - C-ABI of the B200-native semantic draft pool.
+ *
+ * The library implements the nearest-neighbour lookup of Oilbird's semantic draft
+ * source (paper Section 4, "(i) Store" and "(ii) Retrieve"; Eq. 1-3; Algorithm 1):
+ * a pool keyed by the verifier's hidden state at every committed token is searched
+ * with the state at the current position, the top-k past positions are selected and
+ * the token continuation behind each one is copied out as a draft chain.
+ *
+ * Conventions
+ *   - Every function returns OILBIRD_OK (0) or a negative OILBIRD_E* code; nothing
+ *     throws or aborts.  oilbird_strerror() names a code.
+ *   - "dev" pointers are CUDA device pointers on the pool's device, "host" pointers
+ *     are ordinary host memory.  The caller owns every buffer it passes in; the pool
+ *     owns the keys, tokens, trace table and its scratch.
+ *   - bf16 data is passed as raw 16-bit patterns (void* / uint16_t).
+ *   - `cuda_stream` is a cudaStream_t (NULL = the default stream).  append and query
+ *     only enqueue work; they never synchronise.  The row count is tracked on the
+ *     host at enqueue time, so rows are visible to every query enqueued after their
+ *     append on the same stream.  Using different streams for append and query is
+ *     the caller's synchronisation problem.  One host thread per pool at a time.
+ *   - There is no CPU fallback: without a CUDA device create() fails.
+ */
+#ifndef OILBIRD_H_
+#define OILBIRD_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define OILBIRD_OK         0
+#define OILBIRD_EINVAL    (-1)  /* bad argument (null pointer, size out of range, ...) */
+#define OILBIRD_ECAPACITY (-2)  /* rows or traces would exceed what create() sized     */
+#define OILBIRD_ENOMEM    (-3)  /* device or host allocation failed                    */
+#define OILBIRD_ECUDA     (-4)  /* a CUDA call failed; see oilbird_last_cuda_error()   */
+#define OILBIRD_ESTALL    (-5)  /* a bounded device-side wait gave up (status only)    */
+
+#define OILBIRD_MAX_NQ        256   /* queries per call                                */
+#define OILBIRD_MAX_K         128   /* neighbours per query                            */
+#define OILBIRD_MAX_CONT_LEN  128   /* tokens per continuation                         */
+#define OILBIRD_MAX_TIERS     4
+
+/* append flags */
+#define OILBIRD_NEW_TRACE  1u   /* the rows open a new trace (a finished request)      */
+
+/* depth modes (Eq. 3 and the fixed-span variant of the batched harness) */
+#define OILBIRD_DEPTH_FIXED   0  /* every neighbour copies cont_len tokens             */
+#define OILBIRD_DEPTH_TIERED  1  /* D(s): first tier whose floor the score reaches     */
+
+/* which scoring kernel runs */
+#define OILBIRD_PATH_AUTO    0   /* chosen from nq                                     */
+#define OILBIRD_PATH_GEMV    1   /* CUDA-core scan (single-request decode)             */
+#define OILBIRD_PATH_TENSOR  2   /* tcgen05 tensor-core scan (batched queries)         */
+
+typedef struct oilbird_pool oilbird_pool_t;   /* opaque */
+
+/*
+ * Pool geometry, fixed at creation (Eq. 1: one record (x_i, h_i) per committed
+ * generated position, the state "kept normalized in half precision").
+ */
+typedef struct {
+  int32_t  d;              /* key width d_model; a multiple of 8, 8..16384              */
+  int64_t  capacity_rows;  /* rows the pool can hold; arrays are never reallocated      */
+  int32_t  max_traces;     /* trace-table capacity; 0 = min(capacity_rows, 1<<20)       */
+  int32_t  max_nq;         /* largest nq a query will use (<= OILBIRD_MAX_NQ); 0 = 256  */
+  int32_t  max_k;          /* largest k (<= OILBIRD_MAX_K); 0 = 64                      */
+  int32_t  max_append;     /* largest n of the *_host append variant; 0 = 4096          */
+  int32_t  device;         /* CUDA ordinal                                              */
+  uint32_t flags;          /* reserved, 0                                               */
+  void*    arena;          /* dev, optional: caller-provided memory (256-B aligned) of  */
+  size_t   arena_bytes;    /*   at least oilbird_pool_arena_bytes(); NULL = cudaMalloc  */
+} oilbird_pool_config;
+
+/*
+ * Retrieval parameters (Algorithm 1's Require line; Eq. 2; Eq. 3).
+ * oilbird_query_params_default() fills in the values the paper deploys.
+ */
+typedef struct {
+  int32_t  k;                               /* neighbours, paper: 8                     */
+  float    theta;                           /* firing floor on the best score, 0.8      */
+  int32_t  offset;                          /* copy starts at row idx+offset, paper: 2  */
+  int32_t  depth_mode;                      /* OILBIRD_DEPTH_*                          */
+  int32_t  cont_len;                        /* L: row length of cont_tok and the cap on
+                                               every depth; the fixed depth itself      */
+  int32_t  n_tiers;                         /* tiers of D(s), tested in order           */
+  float    tier_thr[OILBIRD_MAX_TIERS];     /* paper: 0.90, 0.82                        */
+  int32_t  tier_depth[OILBIRD_MAX_TIERS];   /* paper: 48, 8 (0 below every tier)        */
+  const uint64_t* exclude_tag;              /* dev [nq] or NULL: rows of traces whose
+                                               tag equals a non-zero entry are skipped
+                                               ("skips any stored trace whose own
+                                               prompt is the one being served now")     */
+  int32_t  path;                            /* OILBIRD_PATH_*                           */
+} oilbird_query_params;
+
+/* Query results.  All five arrays are written on every call. */
+typedef struct {
+  int32_t* idx;       /* [nq,k]   pool row of each neighbour, best first (score
+                                  descending, lower row first among equal scores);
+                                  -1 where fewer than k rows were eligible             */
+  float*   score;     /* [nq,k]   cosine similarity; -INF where idx == -1              */
+  int32_t* fired;     /* [nq]     1 iff the best score >= theta (Eq. 2)                */
+  int32_t* cont_len;  /* [nq,k]   tokens copied for each neighbour (0 if not fired)    */
+  int32_t* cont_tok;  /* [nq,k,L] the continuation, padded with -1                     */
+} oilbird_query_out;
+
+/* Counters accumulated on the device since create()/reset(). */
+typedef struct {
+  int64_t degenerate_rows;     /* appended rows that were all zero or held NaN/Inf and
+                                  were therefore stored as zero keys                   */
+  int64_t nonfinite_queries;   /* queries holding NaN/Inf (they return no neighbours)  */
+  int32_t stalled;             /* non-zero if a bounded device-side wait ever gave up  */
+  int32_t reserved;
+} oilbird_pool_stats;
+
+void   oilbird_query_params_default(oilbird_query_params* p);
+size_t oilbird_pool_arena_bytes(const oilbird_pool_config* cfg);
+
+/*
+ * Lifecycle.  create() validates cfg, allocates (or carves the arena) and sets the
+ * pool empty.  reset() empties it (rows = traces = 0, counters cleared) in stream
+ * order without freeing anything.  destroy() synchronises the device and frees.
+ */
+int oilbird_pool_create (oilbird_pool_t** out, const oilbird_pool_config* cfg);
+int oilbird_pool_reset  (oilbird_pool_t* pool, void* cuda_stream);
+int oilbird_pool_destroy(oilbird_pool_t* pool);
+
+/*
+ * Store (Eq. 1; Algorithm 1 last line: "append the trace to P at request end").
+ * Appends n rows: key = bf16(x / ||x||_2) (norm and scaling in double precision, one
+ * rounding to float and one to bf16, round-to-nearest-even), token, trace
+ * membership.  With OILBIRD_NEW_TRACE the rows open a new trace carrying trace_tag
+ * (0 = never excluded); otherwise they extend the newest trace and trace_tag is
+ * ignored.  The first append to an empty pool always opens a trace.  n = 0 is legal.
+ * states: dev [n,d] bf16 row-major; tokens: dev [n] int32.
+ * Errors: EINVAL (null pointers, n < 0), ECAPACITY (rows or traces exhausted;
+ * nothing is appended).
+ */
+int oilbird_pool_append(oilbird_pool_t* pool, const void* states_bf16, const int32_t* tokens,
+                        int64_t n, uint64_t trace_tag, uint32_t flags, void* cuda_stream);
+
+/*
+ * Retrieve (Algorithm 1: "s_i <- cos(h_t, h_i) for all i in P; E_t <- top-k(s)",
+ * the theta test, d <- D(s_i), gamma <- x_{i+2 : i+1+d}; Eq. 2; Eq. 3).
+ * For each of the nq query states: L2-normalise and round to bf16 (as a key is),
+ * score every stored row by the dot product of the two bf16 vectors accumulated in
+ * fp32, keep the k best by (score descending, row ascending), set fired, give each
+ * neighbour its depth (cont_len, or D(score); 0 if not fired) and copy
+ * min(depth, trace_end - (idx+offset)) tokens starting at row idx+offset of the
+ * token stream, never past the end of the trace that holds idx.
+ * q: dev [nq,d] bf16 row-major.  out: dev arrays as described above.
+ * Errors: EINVAL (nq, k, cont_len, n_tiers out of range for this pool; null
+ * pointers).  An empty pool is legal and yields idx = -1 everywhere.
+ */
+int oilbird_pool_query(oilbird_pool_t* pool, const void* q_bf16, int32_t nq,
+                       const oilbird_query_params* params, const oilbird_query_out* out,
+                       void* cuda_stream);
+
+/*
+ * Fire / depth / copy alone (Eq. 2's condition and Eq. 3) for neighbours the caller
+ * already holds: idx dev [nq,k] (best first; -1 = none), score dev [nq,k].
+ * Writes out->fired, out->cont_len, out->cont_tok; out->idx / out->score are not
+ * touched and may be NULL.
+ */
+int oilbird_pool_gather(oilbird_pool_t* pool, const int32_t* idx, const float* score,
+                        int32_t nq, const oilbird_query_params* params,
+                        const oilbird_query_out* out, void* cuda_stream);
+
+/*
+ * The same two operations with HOST buffers: inputs are copied to the device and
+ * results back inside the call, which returns after the results have landed
+ * (it synchronises cuda_stream).  params->exclude_tag and every array of `out` are
+ * host pointers here.  n <= cfg.max_append.
+ */
+int oilbird_pool_append_host(oilbird_pool_t* pool, const void* states_bf16_host,
+                             const int32_t* tokens_host, int64_t n, uint64_t trace_tag,
+                             uint32_t flags, void* cuda_stream);
+int oilbird_pool_query_host(oilbird_pool_t* pool, const void* q_bf16_host, int32_t nq,
+                            const oilbird_query_params* params, const oilbird_query_out* out_host,
+                            void* cuda_stream);
+
+/* Introspection (host side; none of these enqueue work unless stated). */
+int64_t oilbird_pool_size(const oilbird_pool_t* pool);          /* rows appended so far  */
+int32_t oilbird_pool_num_traces(const oilbird_pool_t* pool);
+/* Synchronises cuda_stream, then reports the device counters. Returns OILBIRD_ESTALL
+ * if a device-side wait ever gave up, else OILBIRD_OK. */
+int oilbird_pool_status(oilbird_pool_t* pool, oilbird_pool_stats* stats, void* cuda_stream);
+/* Copy stored data to host memory (synchronous; for tests and debugging).
+ * keys: [n,d] bf16; tokens, trace_ids: [n] int32; rows [row0, row0+n). */
+int oilbird_pool_read_rows(oilbird_pool_t* pool, int64_t row0, int64_t n, void* keys_host,
+                           int32_t* tokens_host, int32_t* trace_ids_host);
+/* Trace table as the host tracks it: up to max_traces entries each; returns the count. */
+int32_t oilbird_pool_read_traces(const oilbird_pool_t* pool, int64_t* start, int64_t* end,
+                                 uint64_t* tag, int32_t max_traces);
+
+/*
+ * Kernel timing for benchmarks: when enabled, every query brackets its scan kernel
+ * with CUDA events on the caller's stream.  profile_read() synchronises those events
+ * and returns up to max_n scan durations (milliseconds, oldest first) recorded since
+ * the last read, and clears them.  At most 4096 are kept.
+ */
+int     oilbird_pool_profile(oilbird_pool_t* pool, int32_t enable);
+int32_t oilbird_pool_profile_read(oilbird_pool_t* pool, float* scan_ms, int32_t max_n);
+/* Number of kernels this library has launched for this pool since create(). */
+int64_t oilbird_pool_launch_count(const oilbird_pool_t* pool);
+
+const char* oilbird_strerror(int code);
+const char* oilbird_last_cuda_error(void);    /* text of the last failing CUDA call      */
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* OILBIRD_H_ */

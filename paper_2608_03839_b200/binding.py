@@ -1,0 +1,329 @@
+"""Thin ctypes binding over the C-ABI of ``liboilbird.so`` (see ``include/oilbird.h``).
+
+Argument marshalling only: every step of the retrieval path (normalise, score, top-k,
+firing rule, depth, continuation gather) runs in the CUDA library.  torch is used for
+device memory and streams.  There is no fallback: if the library cannot be loaded the
+import of :func:`lib` raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from dataclasses import dataclass, field
+
+import numpy as np
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "liboilbird.so")
+
+OK, EINVAL, ECAPACITY, ENOMEM, ECUDA, ESTALL = 0, -1, -2, -3, -4, -5
+NEW_TRACE = 1
+DEPTH_FIXED, DEPTH_TIERED = 0, 1
+PATH_AUTO, PATH_GEMV, PATH_TENSOR = 0, 1, 2
+MAX_NQ, MAX_K, MAX_CONT_LEN, MAX_TIERS = 256, 128, 128, 4
+
+
+class PoolConfig(ctypes.Structure):
+    _fields_ = [("d", ctypes.c_int32), ("capacity_rows", ctypes.c_int64),
+                ("max_traces", ctypes.c_int32), ("max_nq", ctypes.c_int32),
+                ("max_k", ctypes.c_int32), ("max_append", ctypes.c_int32),
+                ("device", ctypes.c_int32), ("flags", ctypes.c_uint32),
+                ("arena", ctypes.c_void_p), ("arena_bytes", ctypes.c_size_t)]
+
+
+class CQueryParams(ctypes.Structure):
+    _fields_ = [("k", ctypes.c_int32), ("theta", ctypes.c_float), ("offset", ctypes.c_int32),
+                ("depth_mode", ctypes.c_int32), ("cont_len", ctypes.c_int32),
+                ("n_tiers", ctypes.c_int32), ("tier_thr", ctypes.c_float * MAX_TIERS),
+                ("tier_depth", ctypes.c_int32 * MAX_TIERS), ("exclude_tag", ctypes.c_void_p),
+                ("path", ctypes.c_int32)]
+
+
+class CQueryOut(ctypes.Structure):
+    _fields_ = [("idx", ctypes.c_void_p), ("score", ctypes.c_void_p), ("fired", ctypes.c_void_p),
+                ("cont_len", ctypes.c_void_p), ("cont_tok", ctypes.c_void_p)]
+
+
+class PoolStats(ctypes.Structure):
+    _fields_ = [("degenerate_rows", ctypes.c_int64), ("nonfinite_queries", ctypes.c_int64),
+                ("stalled", ctypes.c_int32), ("reserved", ctypes.c_int32)]
+
+
+# name -> (restype, argtypes): every symbol include/oilbird.h declares
+_vp, _i32, _i64, _u64, _u32 = (ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64, ctypes.c_uint64,
+                               ctypes.c_uint32)
+SYMBOLS = {
+    "oilbird_query_params_default": (None, [ctypes.POINTER(CQueryParams)]),
+    "oilbird_pool_arena_bytes": (ctypes.c_size_t, [ctypes.POINTER(PoolConfig)]),
+    "oilbird_pool_create": (ctypes.c_int, [ctypes.POINTER(_vp), ctypes.POINTER(PoolConfig)]),
+    "oilbird_pool_reset": (ctypes.c_int, [_vp, _vp]),
+    "oilbird_pool_destroy": (ctypes.c_int, [_vp]),
+    "oilbird_pool_append": (ctypes.c_int, [_vp, _vp, _vp, _i64, _u64, _u32, _vp]),
+    "oilbird_pool_query": (ctypes.c_int, [_vp, _vp, _i32, ctypes.POINTER(CQueryParams),
+                                          ctypes.POINTER(CQueryOut), _vp]),
+    "oilbird_pool_gather": (ctypes.c_int, [_vp, _vp, _vp, _i32, ctypes.POINTER(CQueryParams),
+                                           ctypes.POINTER(CQueryOut), _vp]),
+    "oilbird_pool_append_host": (ctypes.c_int, [_vp, _vp, _vp, _i64, _u64, _u32, _vp]),
+    "oilbird_pool_query_host": (ctypes.c_int, [_vp, _vp, _i32, ctypes.POINTER(CQueryParams),
+                                               ctypes.POINTER(CQueryOut), _vp]),
+    "oilbird_pool_size": (_i64, [_vp]),
+    "oilbird_pool_num_traces": (_i32, [_vp]),
+    "oilbird_pool_status": (ctypes.c_int, [_vp, ctypes.POINTER(PoolStats), _vp]),
+    "oilbird_pool_read_rows": (ctypes.c_int, [_vp, _i64, _i64, _vp, _vp, _vp]),
+    "oilbird_pool_read_traces": (_i32, [_vp, _vp, _vp, _vp, _i32]),
+    "oilbird_pool_profile": (ctypes.c_int, [_vp, _i32]),
+    "oilbird_pool_profile_read": (_i32, [_vp, _vp, _i32]),
+    "oilbird_pool_launch_count": (_i64, [_vp]),
+    "oilbird_strerror": (ctypes.c_char_p, [ctypes.c_int]),
+    "oilbird_last_cuda_error": (ctypes.c_char_p, []),
+}
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    """Load liboilbird.so (built by ``paper_2608_03839_b200.build``); raises if absent."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise ImportError(
+                f"{LIB_PATH} is missing: build it with `python -m paper_2608_03839_b200.build` "
+                "(there is no CPU or PyTorch fallback)")
+        L = ctypes.CDLL(LIB_PATH)
+        for name, (res, args) in SYMBOLS.items():
+            fn = getattr(L, name)          # AttributeError if a declared symbol is missing
+            fn.restype, fn.argtypes = res, args
+        _lib = L
+    return _lib
+
+
+class OilbirdError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        L = lib()
+        msg = L.oilbird_strerror(code).decode()
+        if code == ECUDA or code == ENOMEM:
+            msg += " (" + L.oilbird_last_cuda_error().decode() + ")"
+        super().__init__(f"{where}: {msg} [{code}]")
+        self.code = code
+
+
+def _check(code: int, where: str) -> None:
+    if code != OK:
+        raise OilbirdError(code, where)
+
+
+@dataclass
+class QueryParams:
+    """Defaults are the deployed values of the paper (k=8, theta=0.8, offset 2, D(s))."""
+    k: int = 8
+    theta: float = 0.8
+    offset: int = 2
+    depth_mode: int = DEPTH_TIERED
+    cont_len: int = 48
+    tier_thr: tuple = (0.90, 0.82)
+    tier_depth: tuple = (48, 8)
+    exclude_tag: torch.Tensor | np.ndarray | None = None   # [nq] uint64 (device: int64 tensor)
+    path: int = PATH_AUTO
+
+    def to_c(self, exclude_ptr=None) -> CQueryParams:
+        c = CQueryParams()
+        c.k, c.theta, c.offset = int(self.k), float(self.theta), int(self.offset)
+        c.depth_mode, c.cont_len = int(self.depth_mode), int(self.cont_len)
+        if len(self.tier_thr) != len(self.tier_depth) or len(self.tier_thr) > MAX_TIERS:
+            raise ValueError("tier_thr / tier_depth: same length, at most 4")
+        c.n_tiers = len(self.tier_thr)
+        for i, (t, dd) in enumerate(zip(self.tier_thr, self.tier_depth)):
+            c.tier_thr[i], c.tier_depth[i] = float(t), int(dd)
+        c.exclude_tag = exclude_ptr
+        c.path = int(self.path)
+        return c
+
+
+@dataclass
+class QueryOut:
+    idx: torch.Tensor        # [nq,k] int32
+    score: torch.Tensor      # [nq,k] float32
+    fired: torch.Tensor      # [nq] int32
+    cont_len: torch.Tensor   # [nq,k] int32
+    cont_tok: torch.Tensor   # [nq,k,L] int32
+    _c: CQueryOut = field(default=None, repr=False)
+
+    @staticmethod
+    def empty(nq: int, k: int, L: int, device) -> "QueryOut":
+        kw = dict(device=device)
+        o = QueryOut(torch.empty((nq, k), dtype=torch.int32, **kw),
+                     torch.empty((nq, k), dtype=torch.float32, **kw),
+                     torch.empty((nq,), dtype=torch.int32, **kw),
+                     torch.empty((nq, k), dtype=torch.int32, **kw),
+                     torch.empty((nq, k, L), dtype=torch.int32, **kw))
+        o._c = CQueryOut(o.idx.data_ptr(), o.score.data_ptr(), o.fired.data_ptr(),
+                         o.cont_len.data_ptr(), o.cont_tok.data_ptr())
+        return o
+
+    def cpu(self) -> "QueryOut":
+        return QueryOut(self.idx.cpu(), self.score.cpu(), self.fired.cpu(), self.cont_len.cpu(),
+                        self.cont_tok.cpu())
+
+
+def _stream_ptr(stream) -> int:
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return int(stream.cuda_stream)
+
+
+class Pool:
+    """A semantic draft pool on one GPU (one per tenant)."""
+
+    def __init__(self, d: int, capacity_rows: int, *, max_traces: int = 0, max_nq: int = 0,
+                 max_k: int = 0, max_append: int = 0, device: int = 0, use_torch_arena=False):
+        self._L = lib()
+        if not torch.cuda.is_available():
+            raise RuntimeError("oilbird pool needs a CUDA device; there is no CPU fallback")
+        self.d, self.device = int(d), int(device)
+        cfg = PoolConfig(d=d, capacity_rows=capacity_rows, max_traces=max_traces, max_nq=max_nq,
+                         max_k=max_k, max_append=max_append, device=device, flags=0,
+                         arena=None, arena_bytes=0)
+        self._arena = None
+        if use_torch_arena:
+            nbytes = self._L.oilbird_pool_arena_bytes(ctypes.byref(cfg))
+            if nbytes == 0:
+                raise OilbirdError(EINVAL, "oilbird_pool_arena_bytes")
+            self._arena = torch.empty(nbytes, dtype=torch.uint8, device=f"cuda:{device}")
+            cfg.arena, cfg.arena_bytes = self._arena.data_ptr(), nbytes
+        h = ctypes.c_void_p()
+        _check(self._L.oilbird_pool_create(ctypes.byref(h), ctypes.byref(cfg)),
+               "oilbird_pool_create")
+        self._h = h
+        self._dev = torch.device(f"cuda:{device}")
+
+    def close(self) -> None:
+        h, self._h = getattr(self, "_h", None), None
+        if h:
+            self._L.oilbird_pool_destroy(h)
+
+    __del__ = close
+
+    def __len__(self) -> int:
+        return int(self._L.oilbird_pool_size(self._h))
+
+    @property
+    def num_traces(self) -> int:
+        return int(self._L.oilbird_pool_num_traces(self._h))
+
+    @property
+    def launch_count(self) -> int:
+        return int(self._L.oilbird_pool_launch_count(self._h))
+
+    def reset(self, stream=None) -> None:
+        _check(self._L.oilbird_pool_reset(self._h, _stream_ptr(stream)), "oilbird_pool_reset")
+
+    # ---- device-buffer entry points -------------------------------------------------
+    def append(self, states: torch.Tensor, tokens: torch.Tensor, tag: int = 0,
+               new_trace: bool = True, stream=None) -> None:
+        n = int(tokens.shape[0])
+        if n:
+            assert states.is_cuda and tokens.is_cuda and states.dtype == torch.bfloat16
+            assert tokens.dtype == torch.int32 and states.is_contiguous() and tokens.is_contiguous()
+            assert states.shape == (n, self.d)
+        _check(self._L.oilbird_pool_append(self._h, states.data_ptr() if n else None,
+                                           tokens.data_ptr() if n else None, n, int(tag),
+                                           NEW_TRACE if new_trace else 0, _stream_ptr(stream)),
+               "oilbird_pool_append")
+
+    def query(self, q: torch.Tensor, params: QueryParams | None = None,
+              out: QueryOut | None = None, stream=None) -> QueryOut:
+        pr = params or QueryParams()
+        assert q.is_cuda and q.dtype == torch.bfloat16 and q.is_contiguous()
+        q = q.reshape(-1, self.d)
+        nq = q.shape[0]
+        ex_ptr = None
+        if pr.exclude_tag is not None:
+            ex = pr.exclude_tag
+            assert ex.is_cuda and ex.dtype in (torch.int64, torch.uint64) and ex.numel() == nq
+            ex_ptr = ex.data_ptr()
+        if out is None:
+            out = QueryOut.empty(nq, pr.k, pr.cont_len, self._dev)
+        cp = pr.to_c(ex_ptr)
+        _check(self._L.oilbird_pool_query(self._h, q.data_ptr(), nq, ctypes.byref(cp),
+                                          ctypes.byref(out._c), _stream_ptr(stream)),
+               "oilbird_pool_query")
+        return out
+
+    def gather(self, idx: torch.Tensor, score: torch.Tensor, params: QueryParams,
+               stream=None) -> QueryOut:
+        assert idx.is_cuda and idx.dtype == torch.int32 and score.dtype == torch.float32
+        nq = idx.shape[0]
+        out = QueryOut.empty(nq, params.k, params.cont_len, self._dev)
+        out.idx, out.score = idx, score
+        cp = params.to_c(None)
+        co = CQueryOut(None, None, out.fired.data_ptr(), out.cont_len.data_ptr(),
+                       out.cont_tok.data_ptr())
+        _check(self._L.oilbird_pool_gather(self._h, idx.data_ptr(), score.data_ptr(), nq,
+                                           ctypes.byref(cp), ctypes.byref(co),
+                                           _stream_ptr(stream)), "oilbird_pool_gather")
+        return out
+
+    # ---- host-buffer entry points ---------------------------------------------------
+    def append_host(self, states: torch.Tensor, tokens: torch.Tensor, tag: int = 0,
+                    new_trace: bool = True, stream=None) -> None:
+        """states: CPU bf16 tensor [n,d] (ideally pinned); tokens: CPU int32 [n]."""
+        n = int(tokens.shape[0])
+        assert not states.is_cuda and not tokens.is_cuda and states.is_contiguous()
+        _check(self._L.oilbird_pool_append_host(self._h, states.data_ptr(), tokens.data_ptr(), n,
+                                                int(tag), NEW_TRACE if new_trace else 0,
+                                                _stream_ptr(stream)), "oilbird_pool_append_host")
+
+    def query_host(self, q: torch.Tensor, params: QueryParams | None = None,
+                   out: QueryOut | None = None, stream=None) -> QueryOut:
+        """q: CPU bf16 tensor [nq,d]; results land in CPU tensors."""
+        pr = params or QueryParams()
+        assert not q.is_cuda and q.dtype == torch.bfloat16 and q.is_contiguous()
+        q = q.reshape(-1, self.d)
+        nq = q.shape[0]
+        ex_ptr = None
+        if pr.exclude_tag is not None:
+            ex = pr.exclude_tag
+            assert not ex.is_cuda and ex.numel() == nq
+            ex_ptr = ex.data_ptr()
+        if out is None:
+            out = QueryOut.empty(nq, pr.k, pr.cont_len, "cpu")
+        cp = pr.to_c(ex_ptr)
+        _check(self._L.oilbird_pool_query_host(self._h, q.data_ptr(), nq, ctypes.byref(cp),
+                                               ctypes.byref(out._c), _stream_ptr(stream)),
+               "oilbird_pool_query_host")
+        return out
+
+    # ---- introspection --------------------------------------------------------------
+    def stats(self, stream=None) -> dict:
+        s = PoolStats()
+        rc = self._L.oilbird_pool_status(self._h, ctypes.byref(s), _stream_ptr(stream))
+        if rc not in (OK, ESTALL):
+            _check(rc, "oilbird_pool_status")
+        return dict(degenerate_rows=int(s.degenerate_rows),
+                    nonfinite_queries=int(s.nonfinite_queries), stalled=int(s.stalled))
+
+    def read_rows(self, row0: int = 0, n: int | None = None):
+        """(keys uint16 [n,d], tokens int32 [n], trace_ids int32 [n]) as numpy arrays."""
+        n = len(self) - row0 if n is None else n
+        keys = np.empty((n, self.d), dtype=np.uint16)
+        tok = np.empty(n, dtype=np.int32)
+        tid = np.empty(n, dtype=np.int32)
+        _check(self._L.oilbird_pool_read_rows(self._h, row0, n, keys.ctypes.data, tok.ctypes.data,
+                                              tid.ctypes.data), "oilbird_pool_read_rows")
+        return keys, tok, tid
+
+    def traces(self):
+        """(start int64 [T], end int64 [T], tag uint64 [T]) as the host tracks them."""
+        T = self.num_traces
+        st, en, tg = (np.empty(T, np.int64), np.empty(T, np.int64), np.empty(T, np.uint64))
+        self._L.oilbird_pool_read_traces(self._h, st.ctypes.data, en.ctypes.data, tg.ctypes.data, T)
+        return st, en, tg
+
+    def profile(self, enable: bool) -> None:
+        _check(self._L.oilbird_pool_profile(self._h, int(enable)), "oilbird_pool_profile")
+
+    def profile_read(self, max_n: int = 4096) -> np.ndarray:
+        buf = np.empty(max_n, dtype=np.float32)
+        n = self._L.oilbird_pool_profile_read(self._h, buf.ctypes.data, max_n)
+        return buf[:n].copy()

@@ -1,0 +1,127 @@
+// Device-side helpers shared by the pool's kernels: candidate packing, warp top-k
+// lists, block bitonic sort.  Nothing here is visible outside the CUDA library.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "internal.h"
+
+namespace oilbird {
+
+typedef unsigned long long u64;
+
+// ---------------------------------------------------------------- candidates ---
+// A candidate (score, row) is packed into one 64-bit key whose unsigned order is the
+// order of Eq. 2 plus the tie rule: higher score first, lower row first.  The high
+// word is the usual order-preserving map of an IEEE float, the low word is ~row.
+// Key 0 never occurs for a real candidate and marks an empty slot.
+
+__device__ __forceinline__ u64 pack_candidate(float s, uint32_t row) {
+  s += 0.0f;                                   // -0.0 -> +0.0 so the two compare equal
+  uint32_t b = __float_as_uint(s);
+  b = (b & 0x80000000u) ? ~b : (b | 0x80000000u);
+  return ((u64)b << 32) | (u64)(~row);
+}
+__device__ __forceinline__ float candidate_score(u64 key) {
+  uint32_t b = (uint32_t)(key >> 32);
+  b = (b & 0x80000000u) ? (b & 0x7fffffffu) : ~b;
+  return __uint_as_float(b);
+}
+__device__ __forceinline__ int32_t candidate_row(u64 key) { return (int32_t)(~(uint32_t)key); }
+
+// ------------------------------------------------------------------- bf16 ------
+__device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }
+__device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
+
+// round-to-nearest-even float -> bf16 bits (finite inputs)
+__device__ __forceinline__ uint32_t f32_to_bf16_bits(float f) {
+  uint32_t u = __float_as_uint(f);
+  u += 0x7fffu + ((u >> 16) & 1u);
+  return u >> 16;
+}
+
+// streaming 16-byte load: read-only path, do not keep in L1
+__device__ __forceinline__ uint4 ld_stream16(const void* p) {
+  uint4 v;
+  asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+               : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+  return v;
+}
+
+// ------------------------------------------------------------------ warp ops ---
+__device__ __forceinline__ u64 shfl_xor_u64(u64 v, int m) {
+  uint32_t lo = __shfl_xor_sync(0xffffffffu, (uint32_t)v, m);
+  uint32_t hi = __shfl_xor_sync(0xffffffffu, (uint32_t)(v >> 32), m);
+  return ((u64)hi << 32) | lo;
+}
+__device__ __forceinline__ u64 warp_min_u64(u64 v) {
+#pragma unroll
+  for (int m = 16; m; m >>= 1) { u64 o = shfl_xor_u64(v, m); v = o < v ? o : v; }
+  return v;
+}
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+  for (int m = 16; m; m >>= 1) v += __shfl_xor_sync(0xffffffffu, v, m);
+  return v;
+}
+
+// A warp-private top-k list of packed candidates in shared memory.  `cnt` and `thr`
+// are warp-uniform registers: the number of filled slots and, once the list is full,
+// its smallest key.  A candidate enters only if it beats thr, so after the first k
+// rows insertions are rare (about k*ln(n/k) over n rows in random order).
+struct WarpTopK {
+  u64* list;
+  int k;
+  int cnt;
+  u64 thr;
+
+  __device__ __forceinline__ void init(u64* l, int k_) { list = l; k = k_; cnt = 0; thr = 0; }
+
+  __device__ __forceinline__ u64 list_min(int lane) const {
+    u64 m = ~0ull;
+    for (int j = lane; j < k; j += 32) { u64 v = list[j]; m = v < m ? v : m; }
+    return warp_min_u64(m);
+  }
+  // Called by all 32 lanes with the same key.
+  __device__ __forceinline__ void insert(u64 key, int lane) {
+    if (cnt < k) {
+      if (lane == 0) list[cnt] = key;
+      ++cnt;
+      __syncwarp();
+      if (cnt == k) thr = list_min(lane);
+      return;
+    }
+    if (key <= thr) return;
+    for (int j = lane; j < k; j += 32)
+      if (list[j] == thr) list[j] = key;       // keys are unique: exactly one slot matches
+    __syncwarp();
+    thr = list_min(lane);
+  }
+  __device__ __forceinline__ bool wants(u64 key) const { return cnt < k || key > thr; }
+  // zero the unused tail so the list can be sorted / merged as k_pad entries
+  __device__ __forceinline__ void pad(int k_pad, int lane) {
+    for (int j = cnt + lane; j < k_pad; j += 32) list[j] = 0;
+    __syncwarp();
+  }
+};
+
+// ------------------------------------------------------------- block sorting ---
+// In-place bitonic sort, DESCENDING, of n (a power of two) keys in shared memory by
+// all threads of the block.  Ends with a __syncthreads().
+__device__ __forceinline__ void block_bitonic_sort_desc(u64* a, int n) {
+  for (int size = 2; size <= n; size <<= 1) {
+    for (int stride = size >> 1; stride > 0; stride >>= 1) {
+      __syncthreads();
+      for (int t = threadIdx.x; t < (n >> 1); t += blockDim.x) {
+        int lo = 2 * t - (t & (stride - 1));   // index with the `stride` bit clear
+        int hi = lo + stride;
+        bool desc = (lo & size) == 0;
+        u64 x = a[lo], y = a[hi];
+        if ((x < y) == desc) { a[lo] = y; a[hi] = x; }
+      }
+    }
+  }
+  __syncthreads();
+}
+
+}  // namespace oilbird

@@ -1,0 +1,73 @@
+// Host-side interface between the C-ABI layer (pool.cu) and the kernel files.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/oilbird.h"
+
+namespace oilbird {
+
+__host__ __device__ inline int next_pow2(int v) {
+  int p = 1;
+  while (p < v) p <<= 1;
+  return p;
+}
+
+// Device counters (one struct in device memory per pool).
+struct DeviceStats {
+  unsigned long long degenerate_rows;
+  unsigned long long nonfinite_queries;
+  int stalled;
+  int pad;
+};
+
+// Views of the pool's device arrays handed to the kernels.
+struct PoolView {
+  const uint16_t* keys;      // [capacity, d] bf16, row-major, normalised (Eq. 1)
+  const int32_t* tok;        // [capacity]
+  const int32_t* trace_id;   // [capacity]
+  const int32_t* trace_end;  // [max_traces] one past the last row of each trace
+  const uint64_t* trace_tag; // [max_traces]
+  int32_t d;
+  int32_t n_rows;            // rows visible to this launch
+};
+
+struct GatherParams {
+  int32_t k, offset, depth_mode, cont_len, n_tiers;
+  float theta;
+  float tier_thr[OILBIRD_MAX_TIERS];
+  int32_t tier_depth[OILBIRD_MAX_TIERS];
+};
+
+// a1: normalise n raw bf16 rows into keys[row0..], store tokens / trace ids, and let one
+// thread publish the trace-table entry (trace, end, tag).
+cudaError_t launch_append(const uint16_t* states, const int32_t* tokens, int64_t n, int32_t d,
+                          uint16_t* keys, int32_t* tok, int32_t* trace_id, int64_t row0,
+                          int32_t trace, int32_t* trace_end, uint64_t* trace_tag, uint64_t tag,
+                          int set_tag, DeviceStats* stats, cudaStream_t st);
+
+// query preparation: qn[r] = bf16(q[r]/||q[r]||) for r < nq, zero rows up to nq_pad,
+// q_valid[r] = 0 for a query holding NaN/Inf.
+cudaError_t launch_qnorm(const uint16_t* q, int32_t nq, int32_t nq_pad, int32_t d, uint16_t* qn,
+                         int32_t* q_valid, DeviceStats* stats, cudaStream_t st);
+
+// a2+a3 (CUDA cores): score every row against nq normalised queries and leave, per CTA
+// and query, a descending list of k_pad packed candidates in partial[list][q][k_pad].
+// Returns the number of lists written through *n_lists.
+cudaError_t launch_scan_gemv(const PoolView& pv, const uint16_t* qn, int32_t nq, int32_t k,
+                             int32_t k_pad, const uint64_t* exclude_tag, unsigned long long* partial,
+                             int32_t max_lists, int32_t num_sms, int32_t* n_lists,
+                             cudaStream_t st);
+
+// a3 (final merge) + a4 + a5 + a6: one CTA per query.
+cudaError_t launch_merge_gather(const PoolView& pv, const unsigned long long* partial,
+                                int32_t n_lists, int32_t nq, int32_t k_pad, const int32_t* q_valid,
+                                const GatherParams& gp, const oilbird_query_out& out,
+                                cudaStream_t st);
+
+// a4 + a5 + a6 on caller-supplied neighbours.
+cudaError_t launch_gather_only(const PoolView& pv, const int32_t* idx, const float* score,
+                               int32_t nq, const GatherParams& gp, const oilbird_query_out& out,
+                               cudaStream_t st);
+
+}  // namespace oilbird

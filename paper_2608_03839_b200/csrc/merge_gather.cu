@@ -1,0 +1,136 @@
+// K4/K5: final top-k merge, firing rule, copy depth and continuation gather.
+//
+// Eq. 2: E_t = arg top-k s_i, with theta a firing condition on the best neighbour
+// only.  Eq. 3: each neighbour copies D(s_i) tokens (or a fixed span) starting
+// `offset` rows after itself, read out of the trace that holds it.  Algorithm 1
+// iterates the neighbours by decreasing s_i; the output keeps that order.
+//
+// One CTA per query.  The per-CTA candidate lists left by the scan are merged by
+// repeatedly sorting a shared-memory buffer that holds the running best k_pad entries
+// plus the next batch of candidates; the integer gather that follows is trivial
+// (nq*k*L tokens).
+#include "common.cuh"
+#include "internal.h"
+
+namespace oilbird {
+
+constexpr int kMergeThreads = 512;
+constexpr int kMergeBuf = 4096;          // candidates sorted per round (32 KB)
+
+// Eq. 3's D(s): first tier, in the order given, whose floor the score reaches.
+__device__ __forceinline__ int depth_of(float s, const GatherParams& gp) {
+  if (gp.depth_mode == OILBIRD_DEPTH_FIXED) return gp.cont_len;
+  for (int t = 0; t < gp.n_tiers; ++t)
+    if (s >= gp.tier_thr[t]) return gp.tier_depth[t];
+  return 0;
+}
+
+// a4..a6 for one query whose neighbours (best first) are in shared memory.
+__device__ void fire_depth_copy(const PoolView& pv, const GatherParams& gp, int q,
+                                const int32_t* s_idx, const float* s_score,
+                                const oilbird_query_out& out, int32_t* s_len) {
+  const int k = gp.k, L = gp.cont_len;
+  // a4: theta gates on the best neighbour only (Eq. 2)
+  const bool fired = s_idx[0] >= 0 && s_score[0] >= gp.theta;
+  if (threadIdx.x == 0) out.fired[q] = fired ? 1 : 0;
+  for (int j = threadIdx.x; j < k; j += blockDim.x) {
+    const int idx = s_idx[j];
+    int len = 0;
+    if (fired && idx >= 0 && idx < pv.n_rows) {
+      const int dep = depth_of(s_score[j], gp);                       // a5
+      const long long start = (long long)idx + gp.offset;
+      const long long end = pv.trace_end[pv.trace_id[idx]];           // never leave the trace
+      long long m = end - start;
+      if (m > dep) m = dep;
+      if (m > L) m = L;
+      if (m < 0) m = 0;
+      len = (int)m;
+    }
+    s_len[j] = len;
+    out.cont_len[(size_t)q * k + j] = len;
+  }
+  __syncthreads();
+  // a6: gamma = x_{idx+offset : idx+offset+len}, padded with -1
+  int32_t* dst = out.cont_tok + (size_t)q * k * L;
+  for (int e = threadIdx.x; e < k * L; e += blockDim.x) {
+    const int j = e / L, t = e - j * L;
+    dst[e] = t < s_len[j] ? pv.tok[(size_t)s_idx[j] + gp.offset + t] : -1;
+  }
+}
+
+__global__ void __launch_bounds__(kMergeThreads)
+merge_gather_kernel(PoolView pv, const u64* __restrict__ partial, int n_lists, int nq, int k_pad,
+                    const int32_t* __restrict__ q_valid, GatherParams gp, oilbird_query_out out) {
+  __shared__ u64 buf[kMergeBuf];
+  __shared__ int32_t s_idx[OILBIRD_MAX_K];
+  __shared__ float s_score[OILBIRD_MAX_K];
+  __shared__ int32_t s_len[OILBIRD_MAX_K];
+  const int q = blockIdx.x;
+  const int k = gp.k;
+  const bool valid = q_valid[q] != 0;
+
+  // running best in buf[0..k_pad), next candidates behind it
+  for (int i = threadIdx.x; i < k_pad; i += kMergeThreads) buf[i] = 0;
+  const int total = valid ? n_lists * k_pad : 0;
+  const int per_round = kMergeBuf - k_pad;
+  for (int base = 0; base < total; base += per_round) {
+    int cnt = total - base < per_round ? total - base : per_round;
+    int n_sort = next_pow2(k_pad + cnt);
+    __syncthreads();
+    for (int i = threadIdx.x; i < n_sort - k_pad; i += kMergeThreads) {
+      u64 v = 0;
+      if (i < cnt) {
+        int c = base + i;
+        int list = c / k_pad, j = c - list * k_pad;
+        v = partial[((size_t)list * nq + q) * k_pad + j];
+      }
+      buf[k_pad + i] = v;
+    }
+    block_bitonic_sort_desc(buf, n_sort);
+  }
+  __syncthreads();
+  for (int j = threadIdx.x; j < k; j += kMergeThreads) {
+    const u64 key = buf[j];
+    const int idx = key ? candidate_row(key) : -1;
+    const float s = key ? candidate_score(key) : -INFINITY;
+    s_idx[j] = idx;
+    s_score[j] = s;
+    out.idx[(size_t)q * k + j] = idx;
+    out.score[(size_t)q * k + j] = s;
+  }
+  __syncthreads();
+  fire_depth_copy(pv, gp, q, s_idx, s_score, out, s_len);
+}
+
+__global__ void __launch_bounds__(128)
+gather_only_kernel(PoolView pv, const int32_t* __restrict__ idx, const float* __restrict__ score,
+                   GatherParams gp, oilbird_query_out out) {
+  __shared__ int32_t s_idx[OILBIRD_MAX_K];
+  __shared__ float s_score[OILBIRD_MAX_K];
+  __shared__ int32_t s_len[OILBIRD_MAX_K];
+  const int q = blockIdx.x, k = gp.k;
+  for (int j = threadIdx.x; j < k; j += blockDim.x) {
+    s_idx[j] = idx[(size_t)q * k + j];
+    s_score[j] = score[(size_t)q * k + j];
+  }
+  __syncthreads();
+  fire_depth_copy(pv, gp, q, s_idx, s_score, out, s_len);
+}
+
+cudaError_t launch_merge_gather(const PoolView& pv, const u64* partial, int32_t n_lists,
+                                int32_t nq, int32_t k_pad, const int32_t* q_valid,
+                                const GatherParams& gp, const oilbird_query_out& out,
+                                cudaStream_t st) {
+  merge_gather_kernel<<<nq, kMergeThreads, 0, st>>>(pv, partial, n_lists, nq, k_pad, q_valid, gp,
+                                                    out);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_gather_only(const PoolView& pv, const int32_t* idx, const float* score,
+                               int32_t nq, const GatherParams& gp, const oilbird_query_out& out,
+                               cudaStream_t st) {
+  gather_only_kernel<<<nq, 128, 0, st>>>(pv, idx, score, gp, out);
+  return cudaGetLastError();
+}
+
+}  // namespace oilbird

@@ -1,0 +1,488 @@
+// C-ABI layer: argument checks, memory layout of the pool in HBM, host-side trace
+// bookkeeping and the launch sequence of each entry point.  No arithmetic of the
+// method lives here.
+#include <math.h>
+#include <stdio.h>
+#include <string.h>
+
+#include <new>
+#include <vector>
+
+#include "internal.h"
+
+using namespace oilbird;
+
+static thread_local char g_cuda_err[256] = "";
+
+static int cuda_fail(cudaError_t e, const char* what) {
+  snprintf(g_cuda_err, sizeof g_cuda_err, "%s: %s", what, cudaGetErrorString(e));
+  return e == cudaErrorMemoryAllocation ? OILBIRD_ENOMEM : OILBIRD_ECUDA;
+}
+#define CU(call)                                          \
+  do {                                                    \
+    cudaError_t e_ = (call);                              \
+    if (e_ != cudaSuccess) return cuda_fail(e_, #call);   \
+  } while (0)
+
+namespace {
+constexpr size_t kAlign = 256;
+constexpr int kMaxProfile = 4096;
+size_t align_up(size_t v) { return (v + kAlign - 1) / kAlign * kAlign; }
+
+// Byte offsets of every device array inside one allocation.
+struct Layout {
+  size_t keys, tok, trace_id, trace_end, trace_tag, qn, q_valid, partial, stats;
+  size_t q_stage, ex_stage, st_stage, tok_stage, out_stage;
+  size_t total;
+};
+
+struct Resolved {
+  int32_t d, max_traces, max_nq, max_k, max_append, max_lists;
+  int64_t capacity;
+};
+
+bool resolve(const oilbird_pool_config* c, int num_sms, Resolved* r) {
+  if (!c) return false;
+  if (c->d < 8 || c->d > 16384 || (c->d % 8) != 0) return false;
+  if (c->capacity_rows < 1 || c->capacity_rows > 2147483000LL) return false;
+  r->d = c->d;
+  r->capacity = c->capacity_rows;
+  int64_t mt = c->max_traces > 0 ? c->max_traces
+                                 : (c->capacity_rows < (1 << 20) ? c->capacity_rows : (1 << 20));
+  if (c->max_traces < 0) return false;
+  r->max_traces = (int32_t)mt;
+  r->max_nq = c->max_nq > 0 ? c->max_nq : OILBIRD_MAX_NQ;
+  r->max_k = c->max_k > 0 ? c->max_k : 64;
+  r->max_append = c->max_append > 0 ? c->max_append : 4096;
+  if (r->max_nq > OILBIRD_MAX_NQ || r->max_k > OILBIRD_MAX_K || c->max_nq < 0 || c->max_k < 0 ||
+      c->max_append < 0)
+    return false;
+  r->max_lists = 2 * num_sms;
+  return true;
+}
+
+Layout make_layout(const Resolved& r) {
+  Layout L;
+  size_t off = 0;
+  auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes); return o; };
+  const size_t nq_pad = (size_t)(r.max_nq + 15) / 16 * 16;
+  const size_t k_pad = (size_t)next_pow2(r.max_k);
+  L.keys = take((size_t)r.capacity * r.d * 2);
+  L.tok = take((size_t)r.capacity * 4);
+  L.trace_id = take((size_t)r.capacity * 4);
+  L.trace_end = take((size_t)r.max_traces * 4);
+  L.trace_tag = take((size_t)r.max_traces * 8);
+  L.qn = take(nq_pad * r.d * 2);
+  L.q_valid = take(nq_pad * 4);
+  L.partial = take((size_t)r.max_lists * r.max_nq * k_pad * 8);
+  L.stats = take(sizeof(DeviceStats));
+  // staging for the *_host variants
+  L.q_stage = take((size_t)r.max_nq * r.d * 2);
+  L.ex_stage = take((size_t)r.max_nq * 8);
+  L.st_stage = take((size_t)r.max_append * r.d * 2);
+  L.tok_stage = take((size_t)r.max_append * 4);
+  L.out_stage = take((size_t)r.max_nq * ((size_t)r.max_k * (8 + 4 + 4 * OILBIRD_MAX_CONT_LEN) + 4));
+  L.total = off;
+  return L;
+}
+}  // namespace
+
+struct oilbird_pool {
+  Resolved r;
+  Layout lay;
+  int device, num_sms;
+  bool owns_mem;
+  unsigned char* base;
+  // device arrays
+  uint16_t* keys;
+  int32_t *tok, *trace_id, *trace_end;
+  uint64_t* trace_tag;
+  uint16_t* qn;
+  int32_t* q_valid;
+  unsigned long long* partial;
+  DeviceStats* stats;
+  // host bookkeeping (enqueue-time truth)
+  int64_t n_rows;
+  std::vector<int64_t> t_start, t_end;
+  std::vector<uint64_t> t_tag;
+  int64_t launches;
+  // profiling
+  bool profile;
+  std::vector<cudaEvent_t> ev;   // pairs
+  int ev_used;
+  // pinned staging for host variants
+  unsigned char* pinned;
+  size_t pinned_bytes;
+};
+
+extern "C" {
+
+const char* oilbird_strerror(int code) {
+  switch (code) {
+    case OILBIRD_OK: return "ok";
+    case OILBIRD_EINVAL: return "invalid argument";
+    case OILBIRD_ECAPACITY: return "pool capacity exceeded";
+    case OILBIRD_ENOMEM: return "out of memory";
+    case OILBIRD_ECUDA: return "CUDA error";
+    case OILBIRD_ESTALL: return "a bounded device-side wait gave up";
+    default: return "unknown error";
+  }
+}
+
+const char* oilbird_last_cuda_error(void) { return g_cuda_err; }
+
+void oilbird_query_params_default(oilbird_query_params* p) {
+  if (!p) return;
+  memset(p, 0, sizeof *p);
+  p->k = 8;                 // Algorithm 1, Require line
+  p->theta = 0.8f;          // Eq. 2
+  p->offset = 2;            // Eq. 3: the chain starts at x_{i+2}
+  p->depth_mode = OILBIRD_DEPTH_TIERED;
+  p->cont_len = 48;
+  p->n_tiers = 2;           // Eq. 3: D(s) = 48 if s >= 0.90; 8 if s >= 0.82; else 0
+  p->tier_thr[0] = 0.90f; p->tier_depth[0] = 48;
+  p->tier_thr[1] = 0.82f; p->tier_depth[1] = 8;
+  p->exclude_tag = nullptr;
+  p->path = OILBIRD_PATH_AUTO;
+}
+
+size_t oilbird_pool_arena_bytes(const oilbird_pool_config* cfg) {
+  Resolved r;
+  if (!resolve(cfg, 148, &r)) return 0;
+  r.max_lists = 2 * 256;    // generous: the SM count is not known without the device
+  return make_layout(r).total + kAlign;
+}
+
+int oilbird_pool_create(oilbird_pool_t** out, const oilbird_pool_config* cfg) {
+  if (!out || !cfg) return OILBIRD_EINVAL;
+  *out = nullptr;
+  int n_dev = 0;
+  CU(cudaGetDeviceCount(&n_dev));
+  if (cfg->device < 0 || cfg->device >= n_dev) return OILBIRD_EINVAL;
+  CU(cudaSetDevice(cfg->device));
+  cudaDeviceProp prop;
+  CU(cudaGetDeviceProperties(&prop, cfg->device));
+  Resolved r;
+  if (!resolve(cfg, prop.multiProcessorCount, &r)) return OILBIRD_EINVAL;
+  Layout lay = make_layout(r);
+  oilbird_pool* p = new (std::nothrow) oilbird_pool();
+  if (!p) return OILBIRD_ENOMEM;
+  p->r = r; p->lay = lay; p->device = cfg->device; p->num_sms = prop.multiProcessorCount;
+  p->n_rows = 0; p->launches = 0; p->profile = false; p->ev_used = 0;
+  p->pinned = nullptr; p->pinned_bytes = 0;
+  if (cfg->arena) {
+    size_t mis = (size_t)((uintptr_t)cfg->arena % kAlign);
+    size_t skip = mis ? kAlign - mis : 0;
+    if (cfg->arena_bytes < lay.total + skip) { delete p; return OILBIRD_EINVAL; }
+    p->base = (unsigned char*)cfg->arena + skip;
+    p->owns_mem = false;
+  } else {
+    void* mem = nullptr;
+    cudaError_t e = cudaMalloc(&mem, lay.total);
+    if (e != cudaSuccess) { delete p; return cuda_fail(e, "cudaMalloc(pool)"); }
+    p->base = (unsigned char*)mem;
+    p->owns_mem = true;
+  }
+  p->keys = (uint16_t*)(p->base + lay.keys);
+  p->tok = (int32_t*)(p->base + lay.tok);
+  p->trace_id = (int32_t*)(p->base + lay.trace_id);
+  p->trace_end = (int32_t*)(p->base + lay.trace_end);
+  p->trace_tag = (uint64_t*)(p->base + lay.trace_tag);
+  p->qn = (uint16_t*)(p->base + lay.qn);
+  p->q_valid = (int32_t*)(p->base + lay.q_valid);
+  p->partial = (unsigned long long*)(p->base + lay.partial);
+  p->stats = (DeviceStats*)(p->base + lay.stats);
+  cudaError_t e = cudaMemset(p->stats, 0, sizeof(DeviceStats));
+  if (e != cudaSuccess) {
+    if (p->owns_mem) cudaFree(p->base);
+    delete p;
+    return cuda_fail(e, "cudaMemset(stats)");
+  }
+  *out = p;
+  return OILBIRD_OK;
+}
+
+int oilbird_pool_destroy(oilbird_pool_t* p) {
+  if (!p) return OILBIRD_EINVAL;
+  cudaSetDevice(p->device);
+  cudaDeviceSynchronize();
+  for (cudaEvent_t e : p->ev) cudaEventDestroy(e);
+  if (p->pinned) cudaFreeHost(p->pinned);
+  if (p->owns_mem) cudaFree(p->base);
+  delete p;
+  return OILBIRD_OK;
+}
+
+int oilbird_pool_reset(oilbird_pool_t* p, void* stream) {
+  if (!p) return OILBIRD_EINVAL;
+  CU(cudaSetDevice(p->device));
+  CU(cudaMemsetAsync(p->stats, 0, sizeof(DeviceStats), (cudaStream_t)stream));
+  p->n_rows = 0;
+  p->t_start.clear(); p->t_end.clear(); p->t_tag.clear();
+  return OILBIRD_OK;
+}
+
+int64_t oilbird_pool_size(const oilbird_pool_t* p) { return p ? p->n_rows : 0; }
+int32_t oilbird_pool_num_traces(const oilbird_pool_t* p) { return p ? (int32_t)p->t_start.size() : 0; }
+int64_t oilbird_pool_launch_count(const oilbird_pool_t* p) { return p ? p->launches : 0; }
+
+int oilbird_pool_append(oilbird_pool_t* p, const void* states, const int32_t* tokens, int64_t n,
+                        uint64_t tag, uint32_t flags, void* stream) {
+  if (!p || n < 0 || (n > 0 && (!states || !tokens))) return OILBIRD_EINVAL;
+  const bool open_new = (flags & OILBIRD_NEW_TRACE) || p->t_start.empty();
+  if (n == 0 && !open_new) return OILBIRD_OK;
+  if (p->n_rows + n > p->r.capacity) return OILBIRD_ECAPACITY;
+  if (open_new && (int64_t)p->t_start.size() >= p->r.max_traces) return OILBIRD_ECAPACITY;
+  CU(cudaSetDevice(p->device));
+  if (open_new) {
+    p->t_start.push_back(p->n_rows);
+    p->t_end.push_back(p->n_rows);
+    p->t_tag.push_back(tag);
+  }
+  const int32_t trace = (int32_t)p->t_start.size() - 1;
+  cudaError_t e = launch_append((const uint16_t*)states, tokens, n, p->r.d, p->keys, p->tok,
+                                p->trace_id, p->n_rows, trace, p->trace_end, p->trace_tag, tag,
+                                open_new ? 1 : 0, p->stats, (cudaStream_t)stream);
+  if (e != cudaSuccess) {
+    if (open_new) { p->t_start.pop_back(); p->t_end.pop_back(); p->t_tag.pop_back(); }
+    return cuda_fail(e, "append kernel launch");
+  }
+  p->launches += 1;
+  p->n_rows += n;
+  p->t_end[trace] = p->n_rows;
+  return OILBIRD_OK;
+}
+
+static int check_params(const oilbird_pool* p, int32_t nq, const oilbird_query_params* pr,
+                        GatherParams* gp) {
+  if (!pr) return OILBIRD_EINVAL;
+  if (nq < 1 || nq > p->r.max_nq) return OILBIRD_EINVAL;
+  if (pr->k < 1 || pr->k > p->r.max_k) return OILBIRD_EINVAL;
+  if (pr->cont_len < 1 || pr->cont_len > OILBIRD_MAX_CONT_LEN) return OILBIRD_EINVAL;
+  if (pr->offset < 0 || pr->offset > (1 << 20)) return OILBIRD_EINVAL;
+  if (pr->depth_mode != OILBIRD_DEPTH_FIXED && pr->depth_mode != OILBIRD_DEPTH_TIERED)
+    return OILBIRD_EINVAL;
+  if (pr->n_tiers < 0 || pr->n_tiers > OILBIRD_MAX_TIERS) return OILBIRD_EINVAL;
+  if (pr->path < OILBIRD_PATH_AUTO || pr->path > OILBIRD_PATH_TENSOR) return OILBIRD_EINVAL;
+  if (isnan(pr->theta)) return OILBIRD_EINVAL;
+  gp->k = pr->k; gp->offset = pr->offset; gp->depth_mode = pr->depth_mode;
+  gp->cont_len = pr->cont_len; gp->n_tiers = pr->n_tiers; gp->theta = pr->theta;
+  for (int t = 0; t < OILBIRD_MAX_TIERS; ++t) {
+    gp->tier_thr[t] = t < pr->n_tiers ? pr->tier_thr[t] : INFINITY;
+    gp->tier_depth[t] = t < pr->n_tiers ? pr->tier_depth[t] : 0;
+    if (t < pr->n_tiers && (isnan(pr->tier_thr[t]) || pr->tier_depth[t] < 0)) return OILBIRD_EINVAL;
+  }
+  return OILBIRD_OK;
+}
+
+static PoolView view_of(const oilbird_pool* p) {
+  PoolView pv;
+  pv.keys = p->keys; pv.tok = p->tok; pv.trace_id = p->trace_id; pv.trace_end = p->trace_end;
+  pv.trace_tag = p->trace_tag; pv.d = p->r.d; pv.n_rows = (int32_t)p->n_rows;
+  return pv;
+}
+
+static bool out_ok(const oilbird_query_out* o, bool need_idx) {
+  if (!o || !o->fired || !o->cont_len || !o->cont_tok) return false;
+  return !need_idx || (o->idx && o->score);
+}
+
+int oilbird_pool_query(oilbird_pool_t* p, const void* q, int32_t nq,
+                       const oilbird_query_params* pr, const oilbird_query_out* out,
+                       void* stream) {
+  if (!p || !q || !out_ok(out, true)) return OILBIRD_EINVAL;
+  GatherParams gp;
+  int rc = check_params(p, nq, pr, &gp);
+  if (rc) return rc;
+  CU(cudaSetDevice(p->device));
+  cudaStream_t st = (cudaStream_t)stream;
+  const int k_pad = next_pow2(pr->k);
+  const int nq_pad = (nq + 15) / 16 * 16;
+  PoolView pv = view_of(p);
+
+  cudaError_t e = launch_qnorm((const uint16_t*)q, nq, nq_pad, p->r.d, p->qn, p->q_valid,
+                               p->stats, st);
+  if (e != cudaSuccess) return cuda_fail(e, "qnorm kernel launch");
+  p->launches += 1;
+
+  int32_t n_lists = 0;
+  if (p->n_rows > 0) {
+    cudaEvent_t e0 = nullptr, e1 = nullptr;
+    if (p->profile && p->ev_used + 2 <= 2 * kMaxProfile) {
+      while ((int)p->ev.size() < p->ev_used + 2) {
+        cudaEvent_t ne;
+        CU(cudaEventCreate(&ne));
+        p->ev.push_back(ne);
+      }
+      e0 = p->ev[p->ev_used]; e1 = p->ev[p->ev_used + 1];
+      CU(cudaEventRecord(e0, st));
+    }
+    e = launch_scan_gemv(pv, p->qn, nq, pr->k, k_pad, pr->exclude_tag, p->partial,
+                         p->r.max_lists, p->num_sms, &n_lists, st);
+    if (e != cudaSuccess) return cuda_fail(e, "scan kernel launch");
+    p->launches += 1;
+    if (e0) {
+      CU(cudaEventRecord(e1, st));
+      p->ev_used += 2;
+    }
+  }
+  e = launch_merge_gather(pv, p->partial, n_lists, nq, k_pad, p->q_valid, gp, *out, st);
+  if (e != cudaSuccess) return cuda_fail(e, "merge kernel launch");
+  p->launches += 1;
+  return OILBIRD_OK;
+}
+
+int oilbird_pool_gather(oilbird_pool_t* p, const int32_t* idx, const float* score, int32_t nq,
+                        const oilbird_query_params* pr, const oilbird_query_out* out,
+                        void* stream) {
+  if (!p || !idx || !score || !out_ok(out, false)) return OILBIRD_EINVAL;
+  GatherParams gp;
+  int rc = check_params(p, nq, pr, &gp);
+  if (rc) return rc;
+  CU(cudaSetDevice(p->device));
+  cudaError_t e = launch_gather_only(view_of(p), idx, score, nq, gp, *out, (cudaStream_t)stream);
+  if (e != cudaSuccess) return cuda_fail(e, "gather kernel launch");
+  p->launches += 1;
+  return OILBIRD_OK;
+}
+
+// ---- host-buffer variants ---------------------------------------------------------
+
+static int ensure_pinned(oilbird_pool* p, size_t bytes) {
+  if (p->pinned_bytes >= bytes) return OILBIRD_OK;
+  if (p->pinned) { cudaFreeHost(p->pinned); p->pinned = nullptr; p->pinned_bytes = 0; }
+  cudaError_t e = cudaMallocHost((void**)&p->pinned, bytes);
+  if (e != cudaSuccess) return cuda_fail(e, "cudaMallocHost");
+  p->pinned_bytes = bytes;
+  return OILBIRD_OK;
+}
+
+int oilbird_pool_append_host(oilbird_pool_t* p, const void* states, const int32_t* tokens,
+                             int64_t n, uint64_t tag, uint32_t flags, void* stream) {
+  if (!p || n < 0 || n > p->r.max_append || (n > 0 && (!states || !tokens))) return OILBIRD_EINVAL;
+  CU(cudaSetDevice(p->device));
+  cudaStream_t st = (cudaStream_t)stream;
+  uint16_t* d_st = (uint16_t*)(p->base + p->lay.st_stage);
+  int32_t* d_tok = (int32_t*)(p->base + p->lay.tok_stage);
+  if (n > 0) {
+    // the staging buffers are reused by the next call: wait for the previous consumer
+    CU(cudaStreamSynchronize(st));
+    CU(cudaMemcpyAsync(d_st, states, (size_t)n * p->r.d * 2, cudaMemcpyHostToDevice, st));
+    CU(cudaMemcpyAsync(d_tok, tokens, (size_t)n * 4, cudaMemcpyHostToDevice, st));
+  }
+  int rc = oilbird_pool_append(p, d_st, d_tok, n, tag, flags, stream);
+  if (rc) return rc;
+  CU(cudaStreamSynchronize(st));
+  return OILBIRD_OK;
+}
+
+int oilbird_pool_query_host(oilbird_pool_t* p, const void* q, int32_t nq,
+                            const oilbird_query_params* pr, const oilbird_query_out* out,
+                            void* stream) {
+  if (!p || !q || !out_ok(out, true)) return OILBIRD_EINVAL;
+  GatherParams gp;
+  int rc = check_params(p, nq, pr, &gp);
+  if (rc) return rc;
+  CU(cudaSetDevice(p->device));
+  cudaStream_t st = (cudaStream_t)stream;
+  const size_t k = pr->k, L = pr->cont_len;
+  uint16_t* d_q = (uint16_t*)(p->base + p->lay.q_stage);
+  uint64_t* d_ex = (uint64_t*)(p->base + p->lay.ex_stage);
+  unsigned char* d_out = p->base + p->lay.out_stage;
+  // device-side result block: idx | score | cont_len | cont_tok | fired
+  const size_t o_idx = 0, o_score = o_idx + nq * k * 4, o_len = o_score + nq * k * 4,
+               o_tok = o_len + nq * k * 4, o_fired = o_tok + nq * k * L * 4,
+               o_total = o_fired + (size_t)nq * 4;
+  CU(cudaStreamSynchronize(st));   // staging reuse
+  CU(cudaMemcpyAsync(d_q, q, (size_t)nq * p->r.d * 2, cudaMemcpyHostToDevice, st));
+  oilbird_query_params dp = *pr;
+  if (pr->exclude_tag) {
+    CU(cudaMemcpyAsync(d_ex, pr->exclude_tag, (size_t)nq * 8, cudaMemcpyHostToDevice, st));
+    dp.exclude_tag = d_ex;
+  }
+  oilbird_query_out dout;
+  dout.idx = (int32_t*)(d_out + o_idx);
+  dout.score = (float*)(d_out + o_score);
+  dout.cont_len = (int32_t*)(d_out + o_len);
+  dout.cont_tok = (int32_t*)(d_out + o_tok);
+  dout.fired = (int32_t*)(d_out + o_fired);
+  rc = oilbird_pool_query(p, d_q, nq, &dp, &dout, stream);
+  if (rc) return rc;
+  rc = ensure_pinned(p, o_total);
+  if (rc) return rc;
+  CU(cudaMemcpyAsync(p->pinned, d_out, o_total, cudaMemcpyDeviceToHost, st));
+  CU(cudaStreamSynchronize(st));
+  memcpy(out->idx, p->pinned + o_idx, nq * k * 4);
+  memcpy(out->score, p->pinned + o_score, nq * k * 4);
+  memcpy(out->cont_len, p->pinned + o_len, nq * k * 4);
+  memcpy(out->cont_tok, p->pinned + o_tok, nq * k * L * 4);
+  memcpy(out->fired, p->pinned + o_fired, (size_t)nq * 4);
+  return OILBIRD_OK;
+}
+
+// ---- introspection ------------------------------------------------------------------
+
+int oilbird_pool_status(oilbird_pool_t* p, oilbird_pool_stats* stats, void* stream) {
+  if (!p) return OILBIRD_EINVAL;
+  CU(cudaSetDevice(p->device));
+  CU(cudaStreamSynchronize((cudaStream_t)stream));
+  DeviceStats ds;
+  CU(cudaMemcpy(&ds, p->stats, sizeof ds, cudaMemcpyDeviceToHost));
+  if (stats) {
+    stats->degenerate_rows = (int64_t)ds.degenerate_rows;
+    stats->nonfinite_queries = (int64_t)ds.nonfinite_queries;
+    stats->stalled = ds.stalled;
+    stats->reserved = 0;
+  }
+  return ds.stalled ? OILBIRD_ESTALL : OILBIRD_OK;
+}
+
+int oilbird_pool_read_rows(oilbird_pool_t* p, int64_t row0, int64_t n, void* keys,
+                           int32_t* tokens, int32_t* trace_ids) {
+  if (!p || row0 < 0 || n < 0 || row0 + n > p->n_rows) return OILBIRD_EINVAL;
+  CU(cudaSetDevice(p->device));
+  CU(cudaDeviceSynchronize());
+  if (n == 0) return OILBIRD_OK;
+  if (keys)
+    CU(cudaMemcpy(keys, p->keys + (size_t)row0 * p->r.d, (size_t)n * p->r.d * 2,
+                  cudaMemcpyDeviceToHost));
+  if (tokens) CU(cudaMemcpy(tokens, p->tok + row0, (size_t)n * 4, cudaMemcpyDeviceToHost));
+  if (trace_ids)
+    CU(cudaMemcpy(trace_ids, p->trace_id + row0, (size_t)n * 4, cudaMemcpyDeviceToHost));
+  return OILBIRD_OK;
+}
+
+int32_t oilbird_pool_read_traces(const oilbird_pool_t* p, int64_t* start, int64_t* end,
+                                 uint64_t* tag, int32_t max_traces) {
+  if (!p) return 0;
+  int32_t n = (int32_t)p->t_start.size();
+  int32_t m = n < max_traces ? n : max_traces;
+  for (int32_t i = 0; i < m; ++i) {
+    if (start) start[i] = p->t_start[i];
+    if (end) end[i] = p->t_end[i];
+    if (tag) tag[i] = p->t_tag[i];
+  }
+  return n;
+}
+
+int oilbird_pool_profile(oilbird_pool_t* p, int32_t enable) {
+  if (!p) return OILBIRD_EINVAL;
+  p->profile = enable != 0;
+  return OILBIRD_OK;
+}
+
+int32_t oilbird_pool_profile_read(oilbird_pool_t* p, float* scan_ms, int32_t max_n) {
+  if (!p) return 0;
+  cudaSetDevice(p->device);
+  int32_t n = p->ev_used / 2, w = 0;
+  for (int32_t i = 0; i < n; ++i) {
+    float ms = 0.f;
+    if (cudaEventSynchronize(p->ev[2 * i + 1]) != cudaSuccess) break;
+    if (cudaEventElapsedTime(&ms, p->ev[2 * i], p->ev[2 * i + 1]) != cudaSuccess) break;
+    if (scan_ms && w < max_n) scan_ms[w++] = ms;
+  }
+  p->ev_used = 0;
+  return w;
+}
+
+}  // extern "C"

@@ -1,0 +1,333 @@
+"""GPU parity tests: the CUDA pool (through the C-ABI) against the CPU oracle on the same
+seeded inputs.  Integer results bit-exact, scores within the stated tolerances (see
+tests/parity.py for the acceptance rule)."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from oracle import OraclePool
+from paper_2608_03839_b200 import binding as B
+from paper_2608_03839_b200 import workloads as W
+from parity import check_query, fill_both
+
+pytestmark = pytest.mark.gpu
+
+P1, M1 = 0x3F80, 0xBF80
+
+
+def bits_to_dev(bits: np.ndarray) -> torch.Tensor:
+    return torch.from_numpy(bits.view(np.int16)).view(torch.bfloat16).cuda()
+
+
+def fixed(k, L, theta=0.8, **kw):
+    return B.QueryParams(k=k, theta=theta, depth_mode=B.DEPTH_FIXED, cont_len=L, **kw)
+
+
+# ----------------------------------------------------------------- append (a1) ----
+
+@pytest.mark.parametrize("d", [8, 200, 256, 4096, 8192])
+def test_append_matches_oracle_bit_for_bit(d):
+    g = torch.Generator(device="cuda").manual_seed(d)
+    n = 300
+    st = (torch.randn(n, d, generator=g, device="cuda") * 3).to(torch.bfloat16)
+    st[7] = 0                                   # zero row
+    st[11, d // 2] = float("inf")               # non-finite rows are stored as zero keys
+    st[13, 0] = float("nan")
+    tk = torch.randint(0, 50000, (n,), generator=g, device="cuda", dtype=torch.int32)
+    pool, ora = B.Pool(d, 1000), OraclePool(d)
+    # three traces, the second extended in two pieces, one empty append in between
+    cuts = [(0, 100, 5, True), (100, 101, 6, True), (101, 101, 0, False), (101, 250, 0, False),
+            (250, 300, 7, True)]
+    for lo, hi, tag, new in cuts:
+        pool.append(st[lo:hi].contiguous(), tk[lo:hi].contiguous(), tag=tag, new_trace=new)
+        ora.append(W.to_bits(st[lo:hi]), tk[lo:hi].cpu().numpy(), tag=tag, new_trace=new)
+    keys, tok, tid = pool.read_rows()
+    assert np.array_equal(keys, ora.keys)
+    assert np.array_equal(tok, ora.tokens) and np.array_equal(tid, ora.trace_ids)
+    s, e, t = pool.traces()
+    assert s.tolist() == ora.trace_starts.tolist() and e.tolist() == ora.trace_ends.tolist()
+    assert t.tolist() == ora.trace_tags.tolist()
+    assert pool.stats()["degenerate_rows"] == ora.degenerate_rows == 3
+    assert np.all(keys[[7, 11, 13]] == 0)
+
+
+def test_append_capacity_and_argument_errors():
+    pool = B.Pool(64, 10, max_traces=2)
+    st = torch.randn(8, 64, device="cuda").to(torch.bfloat16)
+    tk = torch.zeros(8, dtype=torch.int32, device="cuda")
+    pool.append(st, tk, tag=1)
+    with pytest.raises(B.OilbirdError) as e:
+        pool.append(st, tk, tag=2)              # 16 rows > capacity 10
+    assert e.value.code == B.ECAPACITY and len(pool) == 8 and pool.num_traces == 1
+    pool.append(st[:1].contiguous(), tk[:1].contiguous(), tag=2)
+    with pytest.raises(B.OilbirdError) as e:
+        pool.append(st[:1].contiguous(), tk[:1].contiguous(), tag=3)   # third trace
+    assert e.value.code == B.ECAPACITY
+    q = st[:1].contiguous()
+    for bad in (dict(k=0), dict(k=65), dict(cont_len=0), dict(cont_len=129), dict(offset=-1)):
+        pr = fixed(4, 4)
+        for key, val in bad.items():
+            setattr(pr, key, val)
+        with pytest.raises(B.OilbirdError) as e:
+            pool.query(q, pr)
+        assert e.value.code == B.EINVAL
+    with pytest.raises(B.OilbirdError):
+        B.Pool(12, 10)                           # d not a multiple of 8
+    pool.reset()
+    assert len(pool) == 0 and pool.num_traces == 0
+
+
+# ------------------------------------------------ closed-form pools on the GPU ----
+
+@pytest.mark.parametrize("d", [16, 256, 1024, 4096])
+@pytest.mark.parametrize("path", [B.PATH_GEMV, B.PATH_TENSOR])
+def test_hamming_pool_exact_scores_and_tie_order(d, path):
+    rng = np.random.default_rng(d)
+    base = rng.choice([-1, 1], size=d)
+    hs = list(rng.integers(0, min(d, 40), size=300))
+    hs[5] = hs[19] = 0                           # planted exact duplicates of the query
+    rows = np.stack([np.where(np.arange(d) < h, -base, base) for h in hs])
+    bits = np.where(rows > 0, P1, M1).astype(np.uint16)
+    pool, ora = B.Pool(d, 512), OraclePool(d)
+    tk = np.arange(300, dtype=np.int32)
+    pool.append(bits_to_dev(bits), torch.from_numpy(tk).cuda(), tag=1)
+    ora.append(bits, tk, tag=1)
+    qb = np.where(base > 0, P1, M1).astype(np.uint16)
+    pr = fixed(32, 4, path=path)
+    out = pool.query(bits_to_dev(qb[None]), pr)
+    ref = ora.query(qb, __import__("parity").oracle_params(pr))
+    o = out.cpu()
+    # every score is an exact dyadic rational: results are identical, ties included
+    assert o.idx.numpy().tolist() == ref.idx.tolist()
+    assert np.array_equal(o.score.numpy(), ref.score)
+    assert o.idx[0, :2].tolist() == [5, 19] and o.score[0, 0] == 1.0
+    assert np.array_equal(o.cont_tok.numpy(), ref.cont_tok)
+    assert np.array_equal(o.cont_len.numpy(), ref.cont_len)
+
+
+def test_theta_and_depth_tiers_on_exact_scores():
+    d = 1024
+    base = np.ones(d, np.int64)
+    for h, fired, dep in [(51, 1, 48), (52, 1, 8), (92, 1, 8), (93, 1, 0), (102, 1, 0),
+                          (103, 0, 0)]:
+        rows = np.stack([np.where(np.arange(d) < h, -base, base)] + [-base] * 60)
+        bits = np.where(rows > 0, P1, M1).astype(np.uint16)
+        pool = B.Pool(d, 64)
+        pool.append(bits_to_dev(bits), torch.arange(61, dtype=torch.int32).cuda(), tag=1)
+        out = pool.query(bits_to_dev(np.full((1, d), P1, np.uint16)), B.QueryParams()).cpu()
+        assert out.score[0, 0] == 1.0 - 2.0 * h / d
+        assert out.fired[0] == fired and out.cont_len[0, 0] == dep
+        assert out.cont_tok[0, 0, :dep].tolist() == list(range(2, 2 + dep))
+        assert torch.all(out.cont_tok[0, 0, dep:] == -1)
+        assert torch.all(out.idx[0, 1:] >= 1)    # theta is not a floor inside the top-k
+
+
+# ------------------------------------------------------------- benchmark shapes ----
+
+def run_workload(w, n_rows=None, nq=None, paths=(B.PATH_AUTO,), thetas=(0.8, -2.0), **kw):
+    pool, ora = fill_both(w, n_rows=n_rows, **kw)
+    q, meta = w.queries("cuda", nq=nq)
+    stats = []
+    for path in paths:
+        for theta in thetas:
+            pr = fixed(w.k, w.cont_len, theta=theta, path=path)
+            out = pool.query(q, pr)
+            stats.append(check_query(out, ora, W.to_bits(q), pr))
+            o = out.cpu()
+            if "planted_row" in meta and (n_rows is None or meta["planted_row"] < n_rows):
+                assert o.idx[0, 0] == meta["planted_row"]
+    assert pool.stats()["stalled"] == 0
+    return pool, ora, q, meta, stats
+
+
+def test_c1_tiny_config_and_separated_variant():
+    run_workload(W.C1, paths=(B.PATH_GEMV, B.PATH_TENSOR))
+    _, _, _, _, st = run_workload(W.C1.separated(), paths=(B.PATH_GEMV, B.PATH_TENSOR))
+    assert all(s["strict_sets"] == 1 for s in st)
+
+
+@pytest.mark.parametrize("n_rows", [1, 31, 32, 33, 127, 129, 1000, 4095])
+def test_ragged_pool_sizes(n_rows):
+    run_workload(W.C1.scaled(nq=3), n_rows=n_rows, paths=(B.PATH_GEMV, B.PATH_TENSOR))
+
+
+@pytest.mark.parametrize("nq,k", [(1, 1), (2, 5), (5, 64), (8, 8), (17, 33), (64, 32)])
+def test_nq_and_k_combinations(nq, k):
+    w = W.C1.scaled(nq=nq, k=k, n_rows=3000, d=512, cont_len=5)
+    run_workload(w, paths=(B.PATH_GEMV, B.PATH_TENSOR))
+    run_workload(w.separated(), paths=(B.PATH_GEMV, B.PATH_TENSOR))
+
+
+def test_c2_single_request_decode_full_size():
+    _, _, _, _, st = run_workload(W.C2)
+    run_workload(W.C2.separated())
+
+
+def test_c3_tool_calling_shape_scaled():
+    w = W.C3.scaled(n_rows=30000, n_templates=20)
+    pool, ora, q, meta, _ = run_workload(w)
+    out = pool.query(q, fixed(w.k, w.cont_len, theta=-2.0)).cpu()
+    # retrieved rows are dominated by the same (template, position) rows of earlier traces
+    hits = tot = 0
+    for i, rows in enumerate(meta["planted_rows"]):
+        want = set(rows)
+        got = set(out.idx[i].tolist())
+        hits += len(want & got)
+        tot += min(len(want), w.k)
+    assert hits / tot > 0.9
+
+
+def test_exclusion_tags():
+    w = W.C1.scaled(nq=4, n_rows=2048)
+    pool, ora = fill_both(w)
+    q, _ = w.queries("cuda")
+    ex = np.array([0, 3, 5, 999], dtype=np.uint64)          # tags are 1 + trace number
+    for path in (B.PATH_GEMV, B.PATH_TENSOR):
+        pr = fixed(16, 4, theta=-2.0, path=path,
+                   exclude_tag=torch.from_numpy(ex.view(np.int64)).cuda())
+        out = pool.query(q, pr)
+        check_query(out, ora, W.to_bits(q), pr, exclude=ex)
+        tid = ora.trace_ids
+        o = out.cpu()
+        assert not np.any(tid[o.idx[1].numpy()] == 2) and not np.any(tid[o.idx[2].numpy()] == 4)
+
+
+def test_empty_pool_k_above_rows_and_bad_queries():
+    d = 64
+    pool, ora = B.Pool(d, 100), OraclePool(d)
+    q = torch.randn(3, d, device="cuda").to(torch.bfloat16)
+    pr = fixed(8, 4, theta=-2.0)
+    out = pool.query(q, pr).cpu()
+    assert torch.all(out.idx == -1) and torch.all(out.fired == 0) and torch.all(out.cont_tok == -1)
+    st = torch.randn(5, d, device="cuda").to(torch.bfloat16)
+    tk = torch.arange(5, dtype=torch.int32, device="cuda")
+    pool.append(st, tk, tag=1)
+    ora.append(W.to_bits(st), tk.cpu().numpy(), tag=1)
+    q[1] = 0                                      # zero query: all scores 0, lowest rows first
+    q[2, 3] = float("nan")                        # NaN query: no neighbours
+    for path in (B.PATH_GEMV, B.PATH_TENSOR):
+        pr = fixed(8, 4, theta=-2.0, path=path)
+        out = pool.query(q, pr)
+        check_query(out, ora, W.to_bits(q), pr)
+        o = out.cpu()
+        assert o.idx[1].tolist() == [0, 1, 2, 3, 4, -1, -1, -1]
+        assert torch.all(o.idx[2] == -1) and o.fired[2] == 0
+    assert pool.stats()["nonfinite_queries"] == 2
+
+
+# ------------------------------------------------------------------ invariants ----
+
+def test_batched_equals_single_and_is_deterministic():
+    w = W.C1.scaled(nq=8, n_rows=4096, d=1024, k=16)
+    pool, ora = fill_both(w)
+    q, _ = w.queries("cuda")
+    for path in (B.PATH_GEMV, B.PATH_TENSOR):
+        pr = fixed(16, 8, theta=-2.0, path=path)
+        a = pool.query(q, pr).cpu()
+        b = pool.query(q, pr).cpu()
+        for f in ("idx", "score", "fired", "cont_len", "cont_tok"):
+            assert torch.equal(getattr(a, f), getattr(b, f)), "same inputs, different outputs"
+        for i in range(w.nq):
+            s = pool.query(q[i:i + 1].contiguous(), pr).cpu()
+            assert torch.equal(s.idx[0], a.idx[i]) and torch.equal(s.cont_tok[0], a.cont_tok[i])
+            assert torch.allclose(s.score[0], a.score[i], atol=1e-6)
+
+
+def test_gemv_and_tensor_paths_agree():
+    w = W.C1.scaled(nq=8, n_rows=5000, d=2048, k=16).separated()
+    pool, ora = fill_both(w)
+    q, _ = w.queries("cuda")
+    a = pool.query(q, fixed(16, 8, path=B.PATH_GEMV)).cpu()
+    b = pool.query(q, fixed(16, 8, path=B.PATH_TENSOR)).cpu()
+    assert torch.allclose(a.score, b.score, atol=2e-5)
+    assert torch.equal(a.idx[:, :8], b.idx[:, :8])
+
+
+def test_query_scale_invariance_and_chunked_append():
+    w = W.C1.scaled(n_rows=2000, nq=2)
+    pool, ora = fill_both(w)
+    q, _ = w.queries("cuda")
+    pr = fixed(8, 8, theta=-2.0)
+    a, b = pool.query(q, pr).cpu(), pool.query((q.float() * 4).to(torch.bfloat16), pr).cpu()
+    assert torch.equal(a.idx, b.idx) and torch.equal(a.score, b.score)
+    # the same rows appended in other pieces give a bit-identical pool
+    pool2 = B.Pool(w.d, w.n_rows)
+    for st, tk, tag in w.traces("cuda"):
+        pool2.append(st[:100].contiguous(), tk[:100].contiguous(), tag=tag, new_trace=True)
+        pool2.append(st[100:].contiguous(), tk[100:].contiguous(), new_trace=False)
+    for x, y in zip(pool.read_rows(), pool2.read_rows()):
+        assert np.array_equal(x, y)
+    c = pool2.query(q, pr).cpu()
+    assert torch.equal(a.idx, c.idx) and torch.equal(a.cont_tok, c.cont_tok)
+
+
+def test_rows_visible_in_stream_order_and_reset():
+    w = W.C1.scaled(n_rows=1024)
+    pool, ora = fill_both(w, spare_rows=64)
+    g = torch.Generator(device="cuda").manual_seed(7)
+    for step in range(4):
+        st = torch.randn(16, w.d, generator=g, device="cuda").to(torch.bfloat16)
+        tk = torch.randint(0, 100, (16,), generator=g, device="cuda", dtype=torch.int32)
+        pool.append(st, tk, tag=100 + step)
+        ora.append(W.to_bits(st), tk.cpu().numpy(), tag=100 + step)
+        q = (st[9:10].float() + 0.05 * torch.randn(1, w.d, generator=g, device="cuda")).to(
+            torch.bfloat16)
+        pr = fixed(4, 4)
+        out = pool.query(q, pr)                   # no synchronisation in between
+        assert out.cpu().idx[0, 0] == 1024 + 16 * step + 9
+        check_query(out, ora, W.to_bits(q), pr)
+    pool.reset()
+    ora.reset()
+    for st, tk, tag in w.traces("cuda"):
+        pool.append(st, tk, tag=tag)
+        ora.append(W.to_bits(st), tk.cpu().numpy(), tag=tag)
+    q, _ = w.queries("cuda")
+    check_query(pool.query(q, fixed(8, 8)), ora, W.to_bits(q), fixed(8, 8))
+
+
+# -------------------------------------------------------- other entry points ----
+
+def test_gather_entry_point_bit_exact():
+    w = W.C1.scaled(n_rows=2048)
+    pool, ora = fill_both(w)
+    rng = np.random.default_rng(3)
+    nq, k, L = 6, 8, 12
+    idx = rng.integers(-1, 2048, size=(nq, k)).astype(np.int32)
+    idx[0, 0], idx[1, 0], idx[2, 0] = 255, 254, 2047       # trace ends (256-row traces)
+    score = np.sort(rng.uniform(0.7, 1.0, size=(nq, k)).astype(np.float32), axis=1)[:, ::-1].copy()
+    for pr in (B.QueryParams(k=k, cont_len=L), fixed(k, L), fixed(k, L, offset=1),
+               B.QueryParams(k=k, cont_len=L, theta=0.95)):
+        out = pool.gather(torch.from_numpy(idx).cuda(), torch.from_numpy(score).cuda(), pr).cpu()
+        for q in range(nq):
+            f = int(idx[q, 0] >= 0 and score[q, 0] >= np.float32(pr.theta))
+            assert out.fired[q] == f
+            for j in range(k):
+                dep = 0
+                if f and idx[q, j] >= 0:
+                    dep = L if pr.depth_mode == B.DEPTH_FIXED else oracle.depth(float(score[q, j]))
+                tok, n = ora.gather_one(int(idx[q, j]), dep, pr.offset, L)
+                assert out.cont_len[q, j] == n and out.cont_tok[q, j].tolist() == tok.tolist()
+
+
+def test_host_buffer_entry_points_match_device_ones():
+    w = W.C1.scaled(n_rows=1024, nq=3)
+    pool, ora = fill_both(w, spare_rows=32)
+    st = torch.randn(8, w.d).to(torch.bfloat16).pin_memory()
+    tk = torch.arange(8, dtype=torch.int32).pin_memory()
+    pool.append_host(st, tk, tag=77)
+    ora.append(W.to_bits(st), tk.numpy(), tag=77)
+    q, _ = w.queries("cuda")
+    pr = fixed(8, 8, theta=-2.0)
+    a = pool.query(q, pr).cpu()
+    b = pool.query_host(q.cpu().contiguous(), pr)
+    for f in ("idx", "score", "fired", "cont_len", "cont_tok"):
+        assert torch.equal(getattr(a, f), getattr(b, f))
+    check_query(pool.query(q, pr), ora, W.to_bits(q), pr)
+
+
+def test_caller_provided_arena():
+    w = W.C1.scaled(n_rows=512)
+    pool, ora = fill_both(w, use_torch_arena=True)
+    q, _ = w.queries("cuda")
+    check_query(pool.query(q, fixed(8, 8)), ora, W.to_bits(q), fixed(8, 8))

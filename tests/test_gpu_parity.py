@@ -85,7 +85,7 @@ def test_append_capacity_and_argument_errors():
 def test_hamming_pool_exact_scores_and_tie_order(d, path):
     rng = np.random.default_rng(d)
     base = rng.choice([-1, 1], size=d)
-    hs = list(rng.integers(0, min(d, 40), size=300))
+    hs = list(rng.integers(1, min(d, 40), size=300))
     hs[5] = hs[19] = 0                           # planted exact duplicates of the query
     rows = np.stack([np.where(np.arange(d) < h, -base, base) for h in hs])
     bits = np.where(rows > 0, P1, M1).astype(np.uint16)

@@ -105,6 +105,88 @@ struct WarpTopK {
   }
 };
 
+// --------------------------------------------------- warp-level sorted lists ---
+// A list of K = 32*E packed candidates lives in the registers of one warp: element i is
+// v[i / 32] of lane i % 32.  Both routines are bitonic networks; strides >= 32 pair two
+// registers of the same lane, strides < 32 are xor-shuffles.
+
+template <int E>
+__device__ __forceinline__ void warp_bitonic_stage(u64 (&v)[E], int lane, int size, int stride) {
+  if (stride >= 32) {
+    const int rs = stride >> 5;
+#pragma unroll
+    for (int r = 0; r < E; ++r) {
+      if ((r & rs) == 0) {
+        const int i = r * 32 + lane;
+        const bool desc = (i & size) == 0;
+        u64 a = v[r], b = v[r | rs];
+        const bool sw = desc ? (a < b) : (a > b);
+        v[r] = sw ? b : a;
+        v[r | rs] = sw ? a : b;
+      }
+    }
+  } else {
+#pragma unroll
+    for (int r = 0; r < E; ++r) {
+      const int i = r * 32 + lane;
+      const u64 o = shfl_xor_u64(v[r], stride);
+      const bool lower = (i & stride) == 0;
+      const bool desc = (i & size) == 0;
+      const bool keep_max = lower == desc;
+      const u64 mx = v[r] > o ? v[r] : o, mn = v[r] > o ? o : v[r];
+      v[r] = keep_max ? mx : mn;
+    }
+  }
+}
+
+// Sort the K elements descending.
+template <int E>
+__device__ __forceinline__ void warp_sort_desc(u64 (&v)[E], int lane) {
+#pragma unroll
+  for (int size = 2; size <= 32 * E; size <<= 1)
+#pragma unroll
+    for (int stride = size >> 1; stride > 0; stride >>= 1)
+      warp_bitonic_stage<E>(v, lane, size == 32 * E ? (1 << 30) : size, stride);
+}
+
+// a <- the K largest of (a U b), descending; a and b both sorted descending.
+template <int E>
+__device__ __forceinline__ void warp_merge_desc(u64 (&a)[E], const u64 (&b)[E], int lane) {
+  // c[i] = max(a[i], b[K-1-i]) is bitonic and holds the K largest
+#pragma unroll
+  for (int r = 0; r < E; ++r) {
+    const u64 src = b[E - 1 - r];
+    const uint32_t lo = __shfl_sync(0xffffffffu, (uint32_t)src, 31 - lane);
+    const uint32_t hi = __shfl_sync(0xffffffffu, (uint32_t)(src >> 32), 31 - lane);
+    const u64 o = ((u64)hi << 32) | lo;
+    a[r] = a[r] > o ? a[r] : o;
+  }
+#pragma unroll
+  for (int stride = 16 * E; stride > 0; stride >>= 1)
+    warp_bitonic_stage<E>(a, lane, 1 << 30, stride);
+}
+
+// Merge the sorted register lists of all warps of the block into warp 0's registers.
+// scratch: n_warps * 32 * E keys of shared memory.  All threads must call.
+template <int E>
+__device__ __forceinline__ void block_merge_desc(u64 (&v)[E], u64* scratch, int n_warps) {
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  for (int half = (n_warps + 1) >> 1; n_warps > 1; n_warps = half, half = (n_warps + 1) >> 1) {
+    __syncthreads();
+    if (warp >= half && warp < n_warps) {
+#pragma unroll
+      for (int r = 0; r < E; ++r) scratch[(size_t)warp * 32 * E + r * 32 + lane] = v[r];
+    }
+    __syncthreads();
+    if (warp + half < n_warps) {
+      u64 b[E];
+#pragma unroll
+      for (int r = 0; r < E; ++r) b[r] = scratch[(size_t)(warp + half) * 32 * E + r * 32 + lane];
+      warp_merge_desc<E>(v, b, lane);
+    }
+  }
+}
+
 // ------------------------------------------------------------- block sorting ---
 // In-place bitonic sort, DESCENDING, of n (a power of two) keys in shared memory by
 // all threads of the block.  Ends with a __syncthreads().

@@ -51,17 +51,20 @@ cudaError_t launch_append(const uint16_t* states, const int32_t* tokens, int64_t
 cudaError_t launch_qnorm(const uint16_t* q, int32_t nq, int32_t nq_pad, int32_t d, uint16_t* qn,
                          int32_t* q_valid, DeviceStats* stats, cudaStream_t st);
 
-// a2+a3 (CUDA cores): score every row against nq normalised queries and leave, per CTA
-// and query, a descending list of k_pad packed candidates in partial[list][q][k_pad].
-// Returns the number of lists written through *n_lists.
-cudaError_t launch_scan_gemv(const PoolView& pv, const uint16_t* qn, int32_t nq, int32_t k,
-                             int32_t k_pad, const uint64_t* exclude_tag, unsigned long long* partial,
-                             int32_t max_lists, int32_t num_sms, int32_t* n_lists,
-                             cudaStream_t st);
+// Length of the candidate lists exchanged between scan and merge for a given k.
+inline int list_len(int k) { int p = next_pow2(k); return p < 32 ? 32 : p; }
+
+// a2+a3 (CUDA cores): normalise the nq raw queries, score every row against them and
+// leave, per CTA and query, a descending list of kk = list_len(k) packed candidates in
+// partial[list][q][kk].  Also writes q_valid.  Returns the number of lists through *n_lists.
+cudaError_t launch_scan_gemv(const PoolView& pv, const uint16_t* q_raw, int32_t nq, int32_t k,
+                             int32_t kk, const uint64_t* exclude_tag, unsigned long long* partial,
+                             int32_t* q_valid, DeviceStats* stats, int32_t max_lists,
+                             int32_t num_sms, int32_t* n_lists, cudaStream_t st);
 
 // a3 (final merge) + a4 + a5 + a6: one CTA per query.
 cudaError_t launch_merge_gather(const PoolView& pv, const unsigned long long* partial,
-                                int32_t n_lists, int32_t nq, int32_t k_pad, const int32_t* q_valid,
+                                int32_t n_lists, int32_t nq, int32_t kk, const int32_t* q_valid,
                                 const GatherParams& gp, const oilbird_query_out& out,
                                 cudaStream_t st);
 

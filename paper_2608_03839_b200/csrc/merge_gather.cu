@@ -5,17 +5,16 @@
 // `offset` rows after itself, read out of the trace that holds it.  Algorithm 1
 // iterates the neighbours by decreasing s_i; the output keeps that order.
 //
-// One CTA per query.  The per-CTA candidate lists left by the scan are merged by
-// repeatedly sorting a shared-memory buffer that holds the running best k_pad entries
-// plus the next batch of candidates; the integer gather that follows is trivial
-// (nq*k*L tokens).
+// One CTA per query.  The scan leaves one descending candidate list per CTA; 32 warps
+// fold them with register-resident bitonic merges (a few microseconds even for hundreds
+// of lists); the integer gather that follows is trivial (nq*k*L tokens).
 #include "common.cuh"
 #include "internal.h"
 
 namespace oilbird {
 
-constexpr int kMergeThreads = 512;
-constexpr int kMergeBuf = 4096;          // candidates sorted per round (32 KB)
+constexpr int kMergeThreads = 1024;
+constexpr int kMergeWarps = kMergeThreads / 32;
 
 // Eq. 3's D(s): first tier, in the order given, whose floor the score reaches.
 __device__ __forceinline__ int depth_of(float s, const GatherParams& gp) {
@@ -58,39 +57,48 @@ __device__ void fire_depth_copy(const PoolView& pv, const GatherParams& gp, int 
   }
 }
 
+// Each warp folds its share of the scan's descending lists into a register-resident
+// list of kk = 32*E candidates (bitonic merges), then the warps' lists are merged.
+template <int E>
+__device__ __forceinline__ void merge_lists(const u64* __restrict__ partial, int n_lists, int nq,
+                                            int q, u64* scratch, u64* s_best) {
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  constexpr int KK = 32 * E;
+  u64 v[E];
+#pragma unroll
+  for (int r = 0; r < E; ++r) v[r] = 0;
+  for (int l = warp; l < n_lists; l += kMergeWarps) {
+    const u64* src = partial + ((size_t)l * nq + q) * KK;
+    u64 b[E];
+#pragma unroll
+    for (int r = 0; r < E; ++r) b[r] = src[r * 32 + lane];
+    warp_merge_desc<E>(v, b, lane);
+  }
+  const int active = n_lists < kMergeWarps ? (n_lists < 1 ? 1 : n_lists) : kMergeWarps;
+  block_merge_desc<E>(v, scratch, active);
+  if (warp == 0) {
+#pragma unroll
+    for (int r = 0; r < E; ++r) s_best[r * 32 + lane] = v[r];
+  }
+  __syncthreads();
+}
+
 __global__ void __launch_bounds__(kMergeThreads)
-merge_gather_kernel(PoolView pv, const u64* __restrict__ partial, int n_lists, int nq, int k_pad,
+merge_gather_kernel(PoolView pv, const u64* __restrict__ partial, int n_lists, int nq, int kk,
                     const int32_t* __restrict__ q_valid, GatherParams gp, oilbird_query_out out) {
-  __shared__ u64 buf[kMergeBuf];
+  __shared__ u64 scratch[kMergeWarps * OILBIRD_MAX_K];
+  __shared__ u64 s_best[OILBIRD_MAX_K];
   __shared__ int32_t s_idx[OILBIRD_MAX_K];
   __shared__ float s_score[OILBIRD_MAX_K];
   __shared__ int32_t s_len[OILBIRD_MAX_K];
   const int q = blockIdx.x;
   const int k = gp.k;
-  const bool valid = q_valid[q] != 0;
-
-  // running best in buf[0..k_pad), next candidates behind it
-  for (int i = threadIdx.x; i < k_pad; i += kMergeThreads) buf[i] = 0;
-  const int total = valid ? n_lists * k_pad : 0;
-  const int per_round = kMergeBuf - k_pad;
-  for (int base = 0; base < total; base += per_round) {
-    int cnt = total - base < per_round ? total - base : per_round;
-    int n_sort = next_pow2(k_pad + cnt);
-    __syncthreads();
-    for (int i = threadIdx.x; i < n_sort - k_pad; i += kMergeThreads) {
-      u64 v = 0;
-      if (i < cnt) {
-        int c = base + i;
-        int list = c / k_pad, j = c - list * k_pad;
-        v = partial[((size_t)list * nq + q) * k_pad + j];
-      }
-      buf[k_pad + i] = v;
-    }
-    block_bitonic_sort_desc(buf, n_sort);
-  }
-  __syncthreads();
+  const int lists = q_valid[q] != 0 ? n_lists : 0;   // NaN/Inf query: no neighbours
+  if (kk == 32) merge_lists<1>(partial, lists, nq, q, scratch, s_best);
+  else if (kk == 64) merge_lists<2>(partial, lists, nq, q, scratch, s_best);
+  else merge_lists<4>(partial, lists, nq, q, scratch, s_best);
   for (int j = threadIdx.x; j < k; j += kMergeThreads) {
-    const u64 key = buf[j];
+    const u64 key = s_best[j];
     const int idx = key ? candidate_row(key) : -1;
     const float s = key ? candidate_score(key) : -INFINITY;
     s_idx[j] = idx;
@@ -118,10 +126,10 @@ gather_only_kernel(PoolView pv, const int32_t* __restrict__ idx, const float* __
 }
 
 cudaError_t launch_merge_gather(const PoolView& pv, const u64* partial, int32_t n_lists,
-                                int32_t nq, int32_t k_pad, const int32_t* q_valid,
+                                int32_t nq, int32_t kk, const int32_t* q_valid,
                                 const GatherParams& gp, const oilbird_query_out& out,
                                 cudaStream_t st) {
-  merge_gather_kernel<<<nq, kMergeThreads, 0, st>>>(pv, partial, n_lists, nq, k_pad, q_valid, gp,
+  merge_gather_kernel<<<nq, kMergeThreads, 0, st>>>(pv, partial, n_lists, nq, kk, q_valid, gp,
                                                     out);
   return cudaGetLastError();
 }

@@ -1,0 +1,77 @@
+// L2 normalisation of one bf16 row, shared by the append kernel (keys, Eq. 1: "kept
+// normalized in half precision") and by query preparation (the cosine of Algorithm 1's
+// scoring line then is a plain dot product of two stored-format vectors).
+#pragma once
+#include "common.cuh"
+
+namespace oilbird {
+
+constexpr int kNormThreads = 256;
+
+enum { kRowOk = 0, kRowZero = 1, kRowNonFinite = 2 };
+
+// Normalise one row of d bf16 values (d % 8 == 0) from src to dst (global or shared).
+// All kNormThreads threads of the block take part.  The squared norm is accumulated in
+// double precision (products of bf16 values are exact there), the scale 1/sqrt is IEEE
+// double, each element is rounded once to float and once to bf16 (nearest even).
+// Returns kRowOk, or kRowZero / kRowNonFinite, in which case dst is all zero.
+__device__ __forceinline__ int normalize_row(const uint16_t* __restrict__ src, uint16_t* __restrict__ dst,
+                              int d) {
+  __shared__ double s_part[kNormThreads / 32];
+  __shared__ int s_bad[kNormThreads / 32];
+  __shared__ double s_inv;
+  __shared__ int s_code;
+  const int n_chunks = d >> 3;
+  const uint4* src4 = reinterpret_cast<const uint4*>(src);
+  double ss = 0.0;
+  int bad = 0;
+  for (int c = threadIdx.x; c < n_chunks; c += kNormThreads) {
+    uint4 v = __ldg(src4 + c);
+    uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      float lo = bf16_lo(w[i]), hi = bf16_hi(w[i]);
+      bad |= ((w[i] & 0x7f80u) == 0x7f80u) | ((w[i] & 0x7f800000u) == 0x7f800000u);
+      ss += (double)lo * (double)lo;
+      ss += (double)hi * (double)hi;
+    }
+  }
+#pragma unroll
+  for (int m = 16; m; m >>= 1) {
+    ss += __shfl_xor_sync(0xffffffffu, ss, m);
+    bad |= __shfl_xor_sync(0xffffffffu, bad, m);
+  }
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (lane == 0) { s_part[warp] = ss; s_bad[warp] = bad; }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    double tot = 0.0;
+    int b = 0;
+    for (int w = 0; w < kNormThreads / 32; ++w) { tot += s_part[w]; b |= s_bad[w]; }
+    double nrm = sqrt(tot);
+    bool ok = !b && nrm > 0.0 && isfinite(nrm);
+    s_inv = ok ? 1.0 / nrm : 0.0;
+    s_code = ok ? kRowOk : ((b || !isfinite(nrm)) ? kRowNonFinite : kRowZero);
+  }
+  __syncthreads();
+  const double inv = s_inv;
+  uint4* dst4 = reinterpret_cast<uint4*>(dst);
+  for (int c = threadIdx.x; c < n_chunks; c += kNormThreads) {
+    uint4 v = __ldg(src4 + c);
+    uint32_t w[4] = {v.x, v.y, v.z, v.w};
+    uint32_t o[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      if (inv == 0.0) { o[i] = 0; continue; }
+      float lo = __double2float_rn((double)bf16_lo(w[i]) * inv);
+      float hi = __double2float_rn((double)bf16_hi(w[i]) * inv);
+      o[i] = f32_to_bf16_bits(lo) | (f32_to_bf16_bits(hi) << 16);
+    }
+    dst4[c] = make_uint4(o[0], o[1], o[2], o[3]);
+  }
+  const int code = s_code;
+  __syncthreads();   // the shared scratch may be reused by the next call
+  return code;
+}
+
+}  // namespace oilbird

@@ -66,7 +66,7 @@ Layout make_layout(const Resolved& r) {
   size_t off = 0;
   auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes); return o; };
   const size_t nq_pad = (size_t)(r.max_nq + 15) / 16 * 16;
-  const size_t k_pad = (size_t)next_pow2(r.max_k);
+  const size_t k_pad = (size_t)list_len(r.max_k);
   L.keys = take((size_t)r.capacity * r.d * 2);
   L.tok = take((size_t)r.capacity * 4);
   L.trace_id = take((size_t)r.capacity * 4);
@@ -296,17 +296,18 @@ int oilbird_pool_query(oilbird_pool_t* p, const void* q, int32_t nq,
   if (rc) return rc;
   CU(cudaSetDevice(p->device));
   cudaStream_t st = (cudaStream_t)stream;
-  const int k_pad = next_pow2(pr->k);
+  const int kk = list_len(pr->k);
   const int nq_pad = (nq + 15) / 16 * 16;
   PoolView pv = view_of(p);
-
-  cudaError_t e = launch_qnorm((const uint16_t*)q, nq, nq_pad, p->r.d, p->qn, p->q_valid,
-                               p->stats, st);
-  if (e != cudaSuccess) return cuda_fail(e, "qnorm kernel launch");
-  p->launches += 1;
+  cudaError_t e;
 
   int32_t n_lists = 0;
-  if (p->n_rows > 0) {
+  if (p->n_rows == 0) {
+    // nothing to scan: only classify the queries (a NaN/Inf query is still counted)
+    e = launch_qnorm((const uint16_t*)q, nq, nq_pad, p->r.d, p->qn, p->q_valid, p->stats, st);
+    if (e != cudaSuccess) return cuda_fail(e, "qnorm kernel launch");
+    p->launches += 1;
+  } else {
     cudaEvent_t e0 = nullptr, e1 = nullptr;
     if (p->profile && p->ev_used + 2 <= 2 * kMaxProfile) {
       while ((int)p->ev.size() < p->ev_used + 2) {
@@ -317,8 +318,8 @@ int oilbird_pool_query(oilbird_pool_t* p, const void* q, int32_t nq,
       e0 = p->ev[p->ev_used]; e1 = p->ev[p->ev_used + 1];
       CU(cudaEventRecord(e0, st));
     }
-    e = launch_scan_gemv(pv, p->qn, nq, pr->k, k_pad, pr->exclude_tag, p->partial,
-                         p->r.max_lists, p->num_sms, &n_lists, st);
+    e = launch_scan_gemv(pv, (const uint16_t*)q, nq, pr->k, kk, pr->exclude_tag, p->partial,
+                         p->q_valid, p->stats, p->r.max_lists, p->num_sms, &n_lists, st);
     if (e != cudaSuccess) return cuda_fail(e, "scan kernel launch");
     p->launches += 1;
     if (e0) {
@@ -326,7 +327,7 @@ int oilbird_pool_query(oilbird_pool_t* p, const void* q, int32_t nq,
       p->ev_used += 2;
     }
   }
-  e = launch_merge_gather(pv, p->partial, n_lists, nq, k_pad, p->q_valid, gp, *out, st);
+  e = launch_merge_gather(pv, p->partial, n_lists, nq, kk, p->q_valid, gp, *out, st);
   if (e != cudaSuccess) return cuda_fail(e, "merge kernel launch");
   p->launches += 1;
   return OILBIRD_OK;

@@ -5,27 +5,48 @@
 // with 16-byte loads, multiplied against the normalised queries held in shared memory
 // (bf16 x bf16 products accumulated in fp32), and each warp keeps its k best rows in a
 // small shared-memory list.  Scores never go to global memory; what leaves the CTA is
-// one descending list of k_pad packed candidates per query.
+// one descending list of kk (= max(32, k rounded up to a power of two)) packed
+// candidates per query.  The raw query states are normalised by every CTA itself
+// (8-32 KB from L2), which saves a separate launch on the latency-critical path.
 //
 // The kernel is bound by the key stream (N*d*2 bytes); per 16 bytes of key a lane
 // spends 8 integer unpack ops and 8*QT FMAs, well under the issue budget for QT <= 4.
 #include "common.cuh"
 #include "internal.h"
+#include "normalize.cuh"
 
 namespace oilbird {
 
-constexpr int kScanThreads = 256;
+constexpr int kScanThreads = kNormThreads;
 constexpr int kScanWarps = kScanThreads / 32;
 constexpr int kRowsPerIter = 4;   // rows a warp scores together (shares each query load)
 
+// Sort each warp's list, merge the warps' lists and let warp 0 publish the CTA's kk best.
+template <int E>
+__device__ __forceinline__ void publish_cta_list(const WarpTopK& top, u64* scratch,
+                                                 u64* __restrict__ dst) {
+  const int lane = threadIdx.x & 31;
+  u64 v[E];
+#pragma unroll
+  for (int r = 0; r < E; ++r) v[r] = (r * 32 + lane < top.cnt) ? top.list[r * 32 + lane] : 0;
+  warp_sort_desc<E>(v, lane);
+  block_merge_desc<E>(v, scratch, kScanWarps);
+  if (threadIdx.x < 32) {
+#pragma unroll
+    for (int r = 0; r < E; ++r) dst[r * 32 + lane] = v[r];
+  }
+}
+
 template <int QT>
 __global__ void __launch_bounds__(kScanThreads, 2)
-scan_gemv_kernel(PoolView pv, const uint16_t* __restrict__ qn, int nq, int k, int k_pad,
-                 const uint64_t* __restrict__ exclude_tag, u64* __restrict__ partial) {
+scan_gemv_kernel(PoolView pv, const uint16_t* __restrict__ q_raw, int nq, int k, int kk,
+                 const uint64_t* __restrict__ exclude_tag, u64* __restrict__ partial,
+                 int32_t* __restrict__ q_valid, DeviceStats* stats) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   const int d = pv.d, n_chunks = d >> 3;
   uint4* qs = reinterpret_cast<uint4*>(smem_raw);                       // [QT][n_chunks]
-  u64* lists = reinterpret_cast<u64*>(smem_raw + (size_t)QT * d * 2);    // [QT][warps][k_pad]
+  u64* lists = reinterpret_cast<u64*>(smem_raw + (size_t)QT * d * 2);    // [QT][warps][k]
+  u64* scratch = lists + (size_t)QT * kScanWarps * k;                    // [warps][kk]
   __shared__ uint64_t s_ex[QT];
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -37,11 +58,20 @@ scan_gemv_kernel(PoolView pv, const uint16_t* __restrict__ qn, int nq, int k, in
 
   for (int q0 = 0; q0 < nq; q0 += QT) {
     __syncthreads();
-    for (int i = threadIdx.x; i < QT * n_chunks; i += kScanThreads) {
-      int q = i / n_chunks, c = i - q * n_chunks;
-      qs[i] = (q0 + q < nq)
-                  ? __ldg(reinterpret_cast<const uint4*>(qn + (size_t)(q0 + q) * d) + c)
-                  : make_uint4(0, 0, 0, 0);
+    // query preparation: qs[q] = bf16(q / ||q||), exactly as a key is stored
+#pragma unroll
+    for (int q = 0; q < QT; ++q) {
+      uint16_t* dst = reinterpret_cast<uint16_t*>(qs + (size_t)q * n_chunks);
+      if (q0 + q < nq) {
+        const int code = normalize_row(q_raw + (size_t)(q0 + q) * d, dst, d);
+        if (blockIdx.x == 0 && threadIdx.x == 0) {
+          q_valid[q0 + q] = code == kRowNonFinite ? 0 : 1;   // NaN/Inf: no neighbours
+          if (code == kRowNonFinite) atomicAdd(&stats->nonfinite_queries, 1ull);
+        }
+      } else {
+        for (int c = threadIdx.x; c < n_chunks; c += kScanThreads)
+          qs[(size_t)q * n_chunks + c] = make_uint4(0, 0, 0, 0);
+      }
     }
     if (threadIdx.x < QT)
       s_ex[threadIdx.x] = (exclude_tag && q0 + threadIdx.x < nq) ? exclude_tag[q0 + threadIdx.x] : 0;
@@ -49,7 +79,7 @@ scan_gemv_kernel(PoolView pv, const uint16_t* __restrict__ qn, int nq, int k, in
 
     WarpTopK top[QT];
 #pragma unroll
-    for (int q = 0; q < QT; ++q) top[q].init(lists + ((size_t)q * kScanWarps + warp) * k_pad, k);
+    for (int q = 0; q < QT; ++q) top[q].init(lists + ((size_t)q * kScanWarps + warp) * k, k);
 
     for (int rb = r_lo + warp * kRowsPerIter; rb < r_hi; rb += kScanWarps * kRowsPerIter) {
       const uint4* rowp[kRowsPerIter];
@@ -106,34 +136,37 @@ scan_gemv_kernel(PoolView pv, const uint16_t* __restrict__ qn, int nq, int k, in
         }
       }
     }
-    // merge the warps' lists of each query and publish the CTA's k_pad best, descending
+    // merge the warps' lists of each query and publish the CTA's kk best, descending
 #pragma unroll
-    for (int q = 0; q < QT; ++q) top[q].pad(k_pad, lane);
-    __syncthreads();
-    for (int q = 0; q < QT && q0 + q < nq; ++q) {
-      u64* a = lists + (size_t)q * kScanWarps * k_pad;
-      block_bitonic_sort_desc(a, kScanWarps * k_pad);
-      u64* dst = partial + ((size_t)blockIdx.x * nq + (q0 + q)) * k_pad;
-      for (int j = threadIdx.x; j < k_pad; j += kScanThreads) dst[j] = a[j];
+    for (int q = 0; q < QT; ++q) {
+      if (q0 + q >= nq) break;
+      __syncwarp();
+      u64* dst = partial + ((size_t)blockIdx.x * nq + (q0 + q)) * kk;
+      if (kk == 32) publish_cta_list<1>(top[q], scratch, dst);
+      else if (kk == 64) publish_cta_list<2>(top[q], scratch, dst);
+      else publish_cta_list<4>(top[q], scratch, dst);
     }
   }
 }
 
 template <int QT>
-static cudaError_t launch_qt(const PoolView& pv, const uint16_t* qn, int nq, int k, int k_pad,
-                             const uint64_t* ex, u64* partial, int grid, cudaStream_t st) {
-  size_t smem = (size_t)QT * pv.d * 2 + (size_t)QT * kScanWarps * k_pad * sizeof(u64);
+static cudaError_t launch_qt(const PoolView& pv, const uint16_t* q_raw, int nq, int k, int kk,
+                             const uint64_t* ex, u64* partial, int32_t* q_valid,
+                             DeviceStats* stats, int grid, cudaStream_t st) {
+  size_t smem = (size_t)QT * pv.d * 2 + (size_t)QT * kScanWarps * k * sizeof(u64) +
+                (size_t)kScanWarps * kk * sizeof(u64);
   cudaError_t e = cudaFuncSetAttribute(scan_gemv_kernel<QT>,
                                        cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
-  scan_gemv_kernel<QT><<<grid, kScanThreads, smem, st>>>(pv, qn, nq, k, k_pad, ex, partial);
+  scan_gemv_kernel<QT><<<grid, kScanThreads, smem, st>>>(pv, q_raw, nq, k, kk, ex, partial,
+                                                         q_valid, stats);
   return cudaGetLastError();
 }
 
-cudaError_t launch_scan_gemv(const PoolView& pv, const uint16_t* qn, int32_t nq, int32_t k,
-                             int32_t k_pad, const uint64_t* exclude_tag, u64* partial,
-                             int32_t max_lists, int32_t num_sms, int32_t* n_lists,
-                             cudaStream_t st) {
+cudaError_t launch_scan_gemv(const PoolView& pv, const uint16_t* q_raw, int32_t nq, int32_t k,
+                             int32_t kk, const uint64_t* exclude_tag, u64* partial,
+                             int32_t* q_valid, DeviceStats* stats, int32_t max_lists,
+                             int32_t num_sms, int32_t* n_lists, cudaStream_t st) {
   // at least 32 rows per CTA, at most two CTAs per SM
   int64_t want = (pv.n_rows + 31) / 32;
   int grid = (int)(want < 1 ? 1 : want);
@@ -144,9 +177,9 @@ cudaError_t launch_scan_gemv(const PoolView& pv, const uint16_t* qn, int32_t nq,
   int qt = nq >= 4 ? 4 : (nq >= 2 ? 2 : 1);
   while (qt > 1 && (size_t)qt * pv.d * 2 > 65536) qt >>= 1;
   switch (qt) {
-    case 4: return launch_qt<4>(pv, qn, nq, k, k_pad, exclude_tag, partial, grid, st);
-    case 2: return launch_qt<2>(pv, qn, nq, k, k_pad, exclude_tag, partial, grid, st);
-    default: return launch_qt<1>(pv, qn, nq, k, k_pad, exclude_tag, partial, grid, st);
+    case 4: return launch_qt<4>(pv, q_raw, nq, k, kk, exclude_tag, partial, q_valid, stats, grid, st);
+    case 2: return launch_qt<2>(pv, q_raw, nq, k, kk, exclude_tag, partial, q_valid, stats, grid, st);
+    default: return launch_qt<1>(pv, q_raw, nq, k, kk, exclude_tag, partial, q_valid, stats, grid, st);
   }
 }
 

@@ -113,6 +113,12 @@ struct oilbird_pool {
   // pinned staging for host variants
   unsigned char* pinned;
   size_t pinned_bytes;
+  // tensor maps of the tensor-core scan (opaque 128-byte CUtensorMap objects)
+  size_t smem_limit;
+  bool tc_ok;
+  alignas(64) unsigned char key_map[128];
+  alignas(64) unsigned char q_map[OILBIRD_MAX_NQ / 16][128];   // by box rows / 16 - 1
+  bool q_map_ok[OILBIRD_MAX_NQ / 16];
 };
 
 extern "C" {
@@ -198,6 +204,9 @@ int oilbird_pool_create(oilbird_pool_t** out, const oilbird_pool_config* cfg) {
     delete p;
     return cuda_fail(e, "cudaMemset(stats)");
   }
+  p->smem_limit = prop.sharedMemPerBlockOptin;
+  for (bool& b : p->q_map_ok) b = false;
+  p->tc_ok = prop.major == 10 && make_bf16_map(p->key_map, p->keys, r.capacity, r.d, 128);
   *out = p;
   return OILBIRD_OK;
 }
@@ -301,6 +310,14 @@ int oilbird_pool_query(oilbird_pool_t* p, const void* q, int32_t nq,
   PoolView pv = view_of(p);
   cudaError_t e;
 
+  // single-request decode streams keys through the CUDA cores; batches go to tcgen05
+  int path = pr->path;
+  if (path == OILBIRD_PATH_AUTO) path = nq <= 2 ? OILBIRD_PATH_GEMV : OILBIRD_PATH_TENSOR;
+  if (path == OILBIRD_PATH_TENSOR && !p->tc_ok) {
+    snprintf(g_cuda_err, sizeof g_cuda_err, "tensor-core scan unavailable on this device");
+    return OILBIRD_ECUDA;
+  }
+
   int32_t n_lists = 0;
   if (p->n_rows == 0) {
     // nothing to scan: only classify the queries (a NaN/Inf query is still counted)
@@ -318,10 +335,35 @@ int oilbird_pool_query(oilbird_pool_t* p, const void* q, int32_t nq,
       e0 = p->ev[p->ev_used]; e1 = p->ev[p->ev_used + 1];
       CU(cudaEventRecord(e0, st));
     }
-    e = launch_scan_gemv(pv, (const uint16_t*)q, nq, pr->k, kk, pr->exclude_tag, p->partial,
-                         p->q_valid, p->stats, p->r.max_lists, p->num_sms, &n_lists, st);
-    if (e != cudaSuccess) return cuda_fail(e, "scan kernel launch");
-    p->launches += 1;
+    if (path == OILBIRD_PATH_GEMV) {
+      e = launch_scan_gemv(pv, (const uint16_t*)q, nq, pr->k, kk, pr->exclude_tag, p->partial,
+                           p->q_valid, p->stats, p->r.max_lists, p->num_sms, &n_lists, st);
+      if (e != cudaSuccess) return cuda_fail(e, "scan kernel launch");
+      p->launches += 1;
+    } else {
+      e = launch_qnorm((const uint16_t*)q, nq, nq_pad, p->r.d, p->qn, p->q_valid, p->stats, st);
+      if (e != cudaSuccess) return cuda_fail(e, "qnorm kernel launch");
+      p->launches += 1;
+      // as many queries per pass as shared memory allows next to a 3-stage ring
+      const int per_pass = tc_max_queries_per_pass(pr->k, p->smem_limit);
+      for (int q0 = 0; q0 < nq; q0 += per_pass) {
+        const int nq_c = nq - q0 < per_pass ? nq - q0 : per_pass;
+        const int slot = (nq_c + 15) / 16 - 1;
+        if (!p->q_map_ok[slot]) {
+          if (!make_bf16_map(p->q_map[slot], p->qn, (p->r.max_nq + 15) / 16 * 16, p->r.d,
+                             (slot + 1) * 16)) {
+            snprintf(g_cuda_err, sizeof g_cuda_err, "cuTensorMapEncodeTiled(queries) failed");
+            return OILBIRD_ECUDA;
+          }
+          p->q_map_ok[slot] = true;
+        }
+        e = launch_scan_tc(p->key_map, p->q_map[slot], pv, q0, nq_c, nq, pr->k, kk,
+                           pr->exclude_tag, p->partial, p->stats, p->num_sms, p->smem_limit,
+                           &n_lists, st);
+        if (e != cudaSuccess) return cuda_fail(e, "tensor scan kernel launch");
+        p->launches += 1;
+      }
+    }
     if (e0) {
       CU(cudaEventRecord(e1, st));
       p->ev_used += 2;

@@ -1,0 +1,465 @@
+// K3: tensor-core scan for batched queries (many requests against one shared pool).
+//
+// Scoring line of Algorithm 1, "s_i <- cos(h_t, h_i) for all i in P", for nq queries at
+// once: S[i, q] = <key_i, qn_q> is a [N x d] x [d x nq] contraction.  Keys are the M
+// operand (tiles of 128 rows), the normalised queries the N operand (nq padded to a
+// multiple of 16), d is walked in blocks of 64 elements.  Each CTA is persistent and
+// warp-specialised:
+//   warp 0      TMA producer: key tile + query tile per k-block into a 128B-swizzled
+//               shared-memory ring (cp.async.bulk.tensor, mbarrier complete_tx)
+//   warp 1      tcgen05.mma issuer (one thread), fp32 accumulators in TMEM, two
+//               accumulator buffers so the next tile's MMAs overlap the epilogue
+//   warps 2-5   epilogue: tcgen05.ld the 128 x nq scores, filter them against the
+//               per-query running k-th best, and keep per-query top-k lists in shared
+//               memory (Eq. 2); scores never go to global memory
+// The key stream (N*d*2 bytes from HBM, once) bounds the kernel up to nq ~ 128; the
+// query tile is re-read from L2 for every key tile.
+//
+// Every mbarrier wait is bounded: after about two seconds it raises the pool's `stalled`
+// flag, the CTA drains what it has in flight, frees its TMEM and returns.
+#include <cuda.h>
+
+#include "common.cuh"
+#include "internal.h"
+
+namespace oilbird {
+
+constexpr int kTcThreads = 192;
+constexpr int kTileM = 128;            // key rows per tile = TMEM lanes
+constexpr int kBlockK = 64;            // bf16 elements per k-block = one 128-byte swizzle row
+constexpr int kATileBytes = kTileM * kBlockK * 2;   // 16 KB
+constexpr int kColsPerRound = 16;      // score columns filtered between two drains
+constexpr int kQueueCap = kTileM * kColsPerRound;
+constexpr int kMaxStages = 8;
+constexpr unsigned long long kWaitLimitNs = 2000000000ull;
+
+// ------------------------------------------------------------------ PTX wrappers ---
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+  return (uint32_t)__cvta_generic_to_shared(p);
+}
+__device__ __forceinline__ unsigned long long global_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+  return t;
+}
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t* bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)),
+               "r"(bytes)
+               : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(smem_u32(bar)), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Bounded wait.  Returns false if it gave up (or another role already did).
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
+                                          DeviceStats* stats) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const unsigned long long t0 = global_ns();
+  for (uint32_t spin = 0;; ++spin) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if ((spin & 63u) == 63u) {
+      if (*abort_flag) return false;
+      if (global_ns() - t0 > kWaitLimitNs) {
+        *abort_flag = 1;
+        atomicExch(&stats->stalled, 1);
+        return false;
+      }
+    }
+  }
+}
+__device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* map, int x, int y,
+                                            uint64_t* bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes"
+      " [%0], [%1, {%3, %4}], [%2];"
+      ::"r"(smem_u32(dst)), "l"(map), "r"(smem_u32(bar)), "r"(x), "r"(y)
+      : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() {
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+}
+__device__ __forceinline__ void tc_fence_after() {
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+}
+__device__ __forceinline__ void tc_commit(uint64_t* bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];"
+               ::"r"(smem_u32(bar))
+               : "memory");
+}
+// D[tmem] (+)= A[smem desc] * B[smem desc], bf16 x bf16 -> fp32, M=128, N from idesc, K=16
+__device__ __forceinline__ void tc_mma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc,
+                                            uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+__device__ __forceinline__ void tc_ld16(uint32_t taddr, float (&v)[16]) {
+  uint32_t r[16];
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32"
+      " {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]),
+        "=r"(r[7]), "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]),
+        "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr));
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+  for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
+}
+__device__ __forceinline__ void epilogue_bar() {      // the 128 epilogue threads only
+  asm volatile("bar.sync 1, 128;" ::: "memory");
+}
+
+// Shared-memory matrix descriptor of a K-major bf16 tile whose rows are 128 bytes wide
+// and 128B-swizzled (what the TMA box above produces): 8-row groups 1024 bytes apart.
+__device__ __forceinline__ uint64_t umma_desc_sw128(uint32_t smem_addr) {
+  uint64_t d = 0;
+  d |= (uint64_t)((smem_addr & 0x3FFFFu) >> 4);        // start address
+  d |= (uint64_t)1 << 16;                              // leading byte offset (unused, 16 B)
+  d |= (uint64_t)(1024 >> 4) << 32;                    // stride byte offset
+  d |= (uint64_t)1 << 46;                              // descriptor version (Blackwell)
+  d |= (uint64_t)2 << 61;                              // SWIZZLE_128B
+  return d;
+}
+// Instruction descriptor: D fp32, A/B bf16, both K-major, M=128, N=n.
+__host__ __device__ inline uint32_t umma_idesc_bf16(int n) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) |
+         ((uint32_t)(kTileM >> 4) << 24);
+}
+
+// ------------------------------------------------------------- per-query lists ---
+struct TcShared {
+  uint64_t full[kMaxStages], empty[kMaxStages], tmem_full[2], tmem_empty[2], drain;
+  uint32_t tmem_base;
+  int abort_flag;
+  int epi_go;
+  int q_count;
+};
+
+// Warp-cooperative insert into the list of one query (state in shared memory).
+__device__ __forceinline__ void list_insert(u64* list, int k, int* cnt_p, u64* thr_key_p,
+                                            float* thr_s_p, u64 key, int lane) {
+  const int cnt = *cnt_p;
+  if (cnt < k) {
+    __syncwarp();
+    if (lane == 0) { list[cnt] = key; *cnt_p = cnt + 1; }
+    __syncwarp();
+    if (cnt + 1 < k) return;
+  } else {
+    const u64 thr = *thr_key_p;
+    if (key <= thr) return;
+    for (int j = lane; j < k; j += 32)
+      if (list[j] == thr) list[j] = key;               // keys are unique
+    __syncwarp();
+  }
+  u64 m = ~0ull;
+  for (int j = lane; j < k; j += 32) { u64 v = list[j]; m = v < m ? v : m; }
+  m = warp_min_u64(m);
+  if (lane == 0) { *thr_key_p = m; *thr_s_p = candidate_score(m); }
+  __syncwarp();
+}
+
+template <int E>
+__device__ __forceinline__ void publish_query_list(const u64* list, int cnt, u64* dst, int lane) {
+  u64 v[E];
+#pragma unroll
+  for (int r = 0; r < E; ++r) v[r] = (r * 32 + lane < cnt) ? list[r * 32 + lane] : 0;
+  warp_sort_desc<E>(v, lane);
+#pragma unroll
+  for (int r = 0; r < E; ++r) dst[r * 32 + lane] = v[r];
+}
+
+// ------------------------------------------------------------------- the kernel ---
+// Queries [q0, q0+nq_c) of the call; n_pad = nq_c rounded up to 16 = MMA N.
+__global__ void __launch_bounds__(kTcThreads, 1)
+scan_tc_kernel(const __grid_constant__ CUtensorMap key_map,
+               const __grid_constant__ CUtensorMap q_map, PoolView pv, int q0, int nq_c,
+               int nq_total, int n_pad, int k, int kk, int n_stages, int tmem_cols,
+               const uint64_t* __restrict__ exclude_tag, u64* __restrict__ partial,
+               DeviceStats* stats) {
+  extern __shared__ __align__(1024) unsigned char smem_raw[];
+  __shared__ TcShared sh;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int stage_bytes = kATileBytes + n_pad * kBlockK * 2;
+  // dynamic shared memory: [stages][A tile | B tile] | lists | queue | per-query state
+  unsigned char* base = (unsigned char*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+  unsigned char* ring = base;
+  u64* lists = reinterpret_cast<u64*>(ring + (size_t)n_stages * stage_bytes);   // [nq_c][k]
+  u64* q_key = lists + (size_t)nq_c * k;                                        // [kQueueCap]
+  u64* thr_key = q_key + kQueueCap;                                             // [n_pad]
+  uint64_t* s_ex = reinterpret_cast<uint64_t*>(thr_key + n_pad);                // [n_pad]
+  float* thr_s = reinterpret_cast<float*>(s_ex + n_pad);                        // [n_pad]
+  int* cnt = reinterpret_cast<int*>(thr_s + n_pad);                             // [n_pad]
+  uint16_t* q_q = reinterpret_cast<uint16_t*>(cnt + n_pad);                     // [kQueueCap]
+
+  const int n_tiles = (pv.n_rows + kTileM - 1) / kTileM;
+  const int n_kb = (pv.d + kBlockK - 1) / kBlockK;
+  volatile int* abort_flag = &sh.abort_flag;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < n_stages; ++s) { mbar_init(&sh.full[s], 1); mbar_init(&sh.empty[s], 1); }
+    for (int b = 0; b < 2; ++b) { mbar_init(&sh.tmem_full[b], 1); mbar_init(&sh.tmem_empty[b], 4); }
+    mbar_init(&sh.drain, 1);
+    sh.abort_flag = 0;
+    sh.q_count = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  for (int i = threadIdx.x; i < n_pad; i += kTcThreads) {
+    thr_s[i] = -INFINITY;
+    thr_key[i] = 0;
+    cnt[i] = 0;
+    s_ex[i] = (exclude_tag && i < nq_c) ? exclude_tag[q0 + i] : 0;
+  }
+  if (warp == 1) {   // TMEM allocation is a whole-warp operation
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                 ::"r"(smem_u32(&sh.tmem_base)), "r"((uint32_t)tmem_cols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = sh.tmem_base;
+
+  if (warp == 0) {
+    // ===================================================== TMA producer ==========
+    if (lane == 0) {
+      asm volatile("prefetch.tensormap [%0];" ::"l"(&key_map) : "memory");
+      asm volatile("prefetch.tensormap [%0];" ::"l"(&q_map) : "memory");
+      uint32_t it = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
+        for (int kb = 0; kb < n_kb; ++kb, ++it) {
+          const int s = it % n_stages;
+          const uint32_t ph = (it / n_stages) & 1u;
+          if (!mbar_wait(&sh.empty[s], ph ^ 1u, abort_flag, stats)) { ok = false; break; }
+          unsigned char* a_dst = ring + (size_t)s * stage_bytes;
+          mbar_arrive_expect_tx(&sh.full[s], (uint32_t)stage_bytes);
+          tma_load_2d(a_dst, &key_map, kb * kBlockK, tile * kTileM, &sh.full[s]);
+          tma_load_2d(a_dst + kATileBytes, &q_map, kb * kBlockK, q0, &sh.full[s]);
+        }
+      }
+      if (!ok) {
+        // gave up: let the copies already issued land before the CTA's memory goes away
+        const uint32_t back = it < (uint32_t)n_stages ? it : (uint32_t)n_stages;
+        for (uint32_t j = 0; j < back; ++j) {
+          const uint32_t i2 = it - 1 - j;
+          const unsigned long long t0 = global_ns();
+          while (!mbar_try_wait(&sh.full[i2 % n_stages], (i2 / n_stages) & 1u) &&
+                 global_ns() - t0 < 2000000ull) {}
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ===================================================== MMA issuer ============
+    if (lane == 0) {
+      const uint32_t idesc = umma_idesc_bf16(n_pad);
+      uint32_t it = 0, iter = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x, ++iter) {
+        const uint32_t buf = iter & 1u;
+        if (!mbar_wait(&sh.tmem_empty[buf], ((iter >> 1) & 1u) ^ 1u, abort_flag, stats)) {
+          ok = false;
+          break;
+        }
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + buf * (uint32_t)n_pad;
+        for (int kb = 0; kb < n_kb; ++kb, ++it) {
+          const int s = it % n_stages;
+          if (!mbar_wait(&sh.full[s], (it / n_stages) & 1u, abort_flag, stats)) { ok = false; break; }
+          tc_fence_after();
+          const uint32_t a_addr = smem_u32(ring + (size_t)s * stage_bytes);
+          const uint64_t a_desc = umma_desc_sw128(a_addr);
+          const uint64_t b_desc = umma_desc_sw128(a_addr + kATileBytes);
+#pragma unroll
+          for (int kq = 0; kq < kBlockK / 16; ++kq)        // 32 bytes along K per MMA
+            tc_mma_bf16(d_tmem, a_desc + (uint64_t)(kq * 2), b_desc + (uint64_t)(kq * 2), idesc,
+                        (kb | kq) != 0 ? 1u : 0u);
+          tc_commit(&sh.empty[s]);                          // stage reusable once the MMAs retire
+        }
+        if (ok) tc_commit(&sh.tmem_full[buf]);
+      }
+      // nothing may still be writing TMEM when it is freed
+      tc_commit(&sh.drain);
+      const unsigned long long t0 = global_ns();
+      while (!mbar_try_wait(&sh.drain, 0) && global_ns() - t0 < kWaitLimitNs) {}
+    }
+  } else {
+    // ===================================================== epilogue ==============
+    const int ew = warp - 2;                    // 0..3: which queries this warp owns in drains
+    const int lane_grp = warp & 3;              // TMEM lanes this warp may read
+    const int et = threadIdx.x - 64;            // 0..127
+    uint32_t iter = 0;
+    bool ok = true;
+    for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x, ++iter) {
+      const uint32_t buf = iter & 1u;
+      mbar_wait(&sh.tmem_full[buf], (iter >> 1) & 1u, abort_flag, stats);
+      // one decision for all four warps, so that the barriers below always match up
+      epilogue_bar();
+      if (et == 0) sh.epi_go = *abort_flag ? 0 : 1;
+      epilogue_bar();
+      if (!sh.epi_go) { ok = false; break; }
+      tc_fence_after();
+      const int row = tile * kTileM + lane_grp * 32 + lane;
+      const bool row_ok = row < pv.n_rows;
+      uint64_t tag = 0;
+      if (exclude_tag && row_ok) tag = pv.trace_tag[pv.trace_id[row]];
+      const uint32_t t_row = tmem_base + ((uint32_t)(lane_grp * 32) << 16) + buf * (uint32_t)n_pad;
+      for (int c0 = 0; c0 < n_pad; c0 += kColsPerRound) {
+        float v[16];
+        tc_ld16(t_row + (uint32_t)c0, v);
+        if (c0 + kColsPerRound >= n_pad) {
+          // all of this tile's scores are in registers: hand the accumulator back
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(&sh.tmem_empty[buf]);
+        }
+        if (row_ok) {
+#pragma unroll
+          for (int j = 0; j < 16; ++j) {
+            const int q = c0 + j;
+            if (q < nq_c && v[j] > thr_s[q]) {
+              if (s_ex[q] != 0 && tag == s_ex[q]) continue;       // same-prompt trace: skipped
+              const int pos = atomicAdd(&sh.q_count, 1);
+              q_key[pos] = pack_candidate(v[j], (uint32_t)row);
+              q_q[pos] = (uint16_t)q;
+            }
+          }
+        }
+        epilogue_bar();
+        const int n_cand = sh.q_count;
+        if (n_cand > 0) {
+          // drain: warp ew inserts the candidates of queries q with q % 4 == ew
+          for (int b0 = 0; b0 < n_cand; b0 += 32) {
+            const int e = b0 + lane;
+            const int q = e < n_cand ? (int)q_q[e] : -1;
+            unsigned m = __ballot_sync(0xffffffffu, q >= 0 && (q & 3) == ew);
+            while (m) {
+              const int src = __ffs(m) - 1;
+              m &= m - 1;
+              const int qq = __shfl_sync(0xffffffffu, q, src);
+              const u64 key = q_key[b0 + src];
+              list_insert(lists + (size_t)qq * k, k, &cnt[qq], &thr_key[qq], &thr_s[qq], key, lane);
+            }
+          }
+          epilogue_bar();
+          if (et == 0) sh.q_count = 0;
+          epilogue_bar();
+        }
+      }
+    }
+    // publish this CTA's per-query lists, descending, padded with empty slots
+    epilogue_bar();
+    for (int q = ew; q < nq_c; q += 4) {
+      u64* dst = partial + ((size_t)blockIdx.x * nq_total + (q0 + q)) * kk;
+      const u64* src = lists + (size_t)q * k;
+      if (kk == 32) publish_query_list<1>(src, cnt[q], dst, lane);
+      else if (kk == 64) publish_query_list<2>(src, cnt[q], dst, lane);
+      else publish_query_list<4>(src, cnt[q], dst, lane);
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;"
+                 ::"r"(tmem_base), "r"((uint32_t)tmem_cols) : "memory");
+  }
+}
+
+// ------------------------------------------------------------------ host side ---
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*,
+                                  const cuuint64_t*, const cuuint64_t*, const cuuint32_t*,
+                                  const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (!fn) {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) ==
+            cudaSuccess && qres == cudaDriverEntryPointSuccess)
+      fn = (EncodeTiledFn)p;
+  }
+  return fn;
+}
+
+// Tensor map over a row-major bf16 matrix [rows, d]; box = 64 elements x box_rows rows,
+// 128B swizzle, out-of-range elements read as zero.
+bool make_bf16_map(void* map_out, const void* base, int64_t rows, int32_t d, int32_t box_rows) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  cuuint64_t dims[2] = {(cuuint64_t)d, (cuuint64_t)rows};
+  cuuint64_t strides[1] = {(cuuint64_t)d * 2};
+  cuuint32_t box[2] = {(cuuint32_t)kBlockK, (cuuint32_t)box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult r = fn((CUtensorMap*)map_out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (void*)base, dims,
+                  strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                  CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS;
+}
+
+static size_t tc_fixed_smem(int nq_c, int n_pad, int k) {
+  return (size_t)nq_c * k * 8 + (size_t)kQueueCap * 8 + (size_t)n_pad * (8 + 8 + 4 + 4) +
+         (size_t)kQueueCap * 2 + 1024 /* alignment slack */;
+}
+
+// Largest number of queries one launch can take for this k so that at least three ring
+// stages fit next to the per-query lists.
+int tc_max_queries_per_pass(int k, size_t smem_limit) {
+  int best = 16;
+  for (int n = 16; n <= OILBIRD_MAX_NQ; n += 16) {
+    size_t stage = (size_t)kATileBytes + (size_t)n * kBlockK * 2;
+    if (tc_fixed_smem(n, n, k) + 3 * stage + sizeof(TcShared) + 256 <= smem_limit) best = n;
+  }
+  return best;
+}
+
+cudaError_t launch_scan_tc(const void* key_map, const void* q_map, const PoolView& pv, int32_t q0,
+                           int32_t nq_c, int32_t nq_total, int32_t k, int32_t kk,
+                           const uint64_t* exclude_tag, unsigned long long* partial,
+                           DeviceStats* stats, int32_t num_sms, size_t smem_limit,
+                           int32_t* n_lists, cudaStream_t st) {
+  const int n_pad = (nq_c + 15) / 16 * 16;
+  const size_t stage = (size_t)kATileBytes + (size_t)n_pad * kBlockK * 2;
+  const size_t fixed = tc_fixed_smem(nq_c, n_pad, k);
+  const size_t avail = smem_limit - sizeof(TcShared) - 256;
+  if (fixed + 2 * stage > avail) return cudaErrorInvalidConfiguration;
+  int stages = (int)((avail - fixed) / stage);
+  if (stages > kMaxStages) stages = kMaxStages;
+  size_t smem = fixed + (size_t)stages * stage;
+  if (smem < 120 * 1024) smem = 120 * 1024;   // one CTA per SM: TMEM is allocated per CTA
+  int tmem_cols = 32;
+  while (tmem_cols < 2 * n_pad) tmem_cols <<= 1;
+  const int n_tiles = (pv.n_rows + kTileM - 1) / kTileM;
+  int grid = n_tiles < num_sms ? n_tiles : num_sms;
+  if (grid < 1) grid = 1;
+  *n_lists = grid;
+  cudaError_t e = cudaFuncSetAttribute(scan_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       (int)smem);
+  if (e != cudaSuccess) return e;
+  scan_tc_kernel<<<grid, kTcThreads, smem, st>>>(*(const CUtensorMap*)key_map,
+                                                 *(const CUtensorMap*)q_map, pv, q0, nq_c,
+                                                 nq_total, n_pad, k, kk, stages, tmem_cols,
+                                                 exclude_tag, partial, stats);
+  return cudaGetLastError();
+}
+
+}  // namespace oilbird

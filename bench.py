@@ -168,6 +168,8 @@ def run_ours(args):
     w = W.CONFIGS[args.config]
     nq = args.nq or w.nq
     n0 = W.C5_START_ROWS if w.name == "C5" else w.n_rows
+    if args.rows:
+        n0 = args.rows                      # smaller pool of the same recipe (profiling)
     rows_step = APPEND_ROWS[w.name]
     K, Wm = args.steps, args.warmup
     total_steps = 2 * (Wm + K) + Wm + K     # device-timed pass, kernel-timed pass, e2e pass
@@ -403,6 +405,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", default="C2", choices=sorted(W.CONFIGS))
     ap.add_argument("--nq", type=int, default=0, help="override the configuration's nq")
+    ap.add_argument("--rows", type=int, default=0,
+                    help="override the pool size (profiling a smaller case of the same recipe)")
     ap.add_argument("--path", type=int, default=0, help="0 auto, 1 CUDA-core scan, 2 tensor scan")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-budget", type=float, default=20.0)

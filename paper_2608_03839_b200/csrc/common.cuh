@@ -166,6 +166,36 @@ __device__ __forceinline__ void warp_merge_desc(u64 (&a)[E], const u64 (&b)[E], 
     warp_bitonic_stage<E>(a, lane, 1 << 30, stride);
 }
 
+// Insert one candidate (the same key in every lane) into a descending register list,
+// dropping the smallest element.  About a dozen instructions per 32 elements.
+template <int E>
+__device__ __forceinline__ void warp_sorted_insert(u64 (&v)[E], u64 key, int lane) {
+#pragma unroll
+  for (int r = 0; r < E; ++r) {
+    const int pos = __popc(__ballot_sync(0xffffffffu, v[r] > key));   // elements that stay put
+    if (pos < 32) {                                                   // warp-uniform
+      const uint32_t ulo = __shfl_up_sync(0xffffffffu, (uint32_t)v[r], 1);
+      const uint32_t uhi = __shfl_up_sync(0xffffffffu, (uint32_t)(v[r] >> 32), 1);
+      const uint32_t clo = __shfl_sync(0xffffffffu, (uint32_t)v[r], 31);
+      const uint32_t chi = __shfl_sync(0xffffffffu, (uint32_t)(v[r] >> 32), 31);
+      const u64 up = ((u64)uhi << 32) | ulo;
+      v[r] = lane < pos ? v[r] : (lane == pos ? key : up);
+      key = ((u64)chi << 32) | clo;                                   // carried into the next row
+    }
+  }
+}
+
+// Element i of a register list, broadcast to all lanes.
+template <int E>
+__device__ __forceinline__ u64 warp_list_get(const u64 (&v)[E], int i) {
+  u64 x = v[0];
+#pragma unroll
+  for (int r = 1; r < E; ++r) x = (i >> 5) == r ? v[r] : x;
+  const uint32_t lo = __shfl_sync(0xffffffffu, (uint32_t)x, i & 31);
+  const uint32_t hi = __shfl_sync(0xffffffffu, (uint32_t)(x >> 32), i & 31);
+  return ((u64)hi << 32) | lo;
+}
+
 // Merge the sorted register lists of all warps of the block into warp 0's registers.
 // scratch: n_warps * 32 * E keys of shared memory.  All threads must call.
 template <int E>

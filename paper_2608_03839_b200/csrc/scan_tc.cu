@@ -150,40 +150,30 @@ struct TcShared {
   uint32_t tmem_base;
   int abort_flag;
   int epi_go;
-  int q_count;
+  int q_total;                  // candidates queued in the current round
+  int q_cnt[kColsPerRound];     // ... per score column of the round
 };
 
-// Warp-cooperative insert into the list of one query (state in shared memory).
-__device__ __forceinline__ void list_insert(u64* list, int k, int* cnt_p, u64* thr_key_p,
-                                            float* thr_s_p, u64 key, int lane) {
-  const int cnt = *cnt_p;
-  if (cnt < k) {
-    __syncwarp();
-    if (lane == 0) { list[cnt] = key; *cnt_p = cnt + 1; }
-    __syncwarp();
-    if (cnt + 1 < k) return;
-  } else {
-    const u64 thr = *thr_key_p;
-    if (key <= thr) return;
-    for (int j = lane; j < k; j += 32)
-      if (list[j] == thr) list[j] = key;               // keys are unique
-    __syncwarp();
-  }
-  u64 m = ~0ull;
-  for (int j = lane; j < k; j += 32) { u64 v = list[j]; m = v < m ? v : m; }
-  m = warp_min_u64(m);
-  if (lane == 0) { *thr_key_p = m; *thr_s_p = candidate_score(m); }
-  __syncwarp();
-}
-
+// Fold the candidates queued for one query into its descending list (shared memory,
+// kk = 32*E slots, empty slots are 0) and refresh the filter threshold: the score of the
+// k-th entry once k entries exist.
 template <int E>
-__device__ __forceinline__ void publish_query_list(const u64* list, int cnt, u64* dst, int lane) {
+__device__ __forceinline__ void drain_query(u64* list, const u64* cand, int n_cand, int k,
+                                            float* thr_s_p, int lane) {
   u64 v[E];
 #pragma unroll
-  for (int r = 0; r < E; ++r) v[r] = (r * 32 + lane < cnt) ? list[r * 32 + lane] : 0;
-  warp_sort_desc<E>(v, lane);
+  for (int r = 0; r < E; ++r) v[r] = list[r * 32 + lane];
+  u64 kth = warp_list_get<E>(v, k - 1);
+  for (int i = 0; i < n_cand; ++i) {
+    const u64 key = cand[i];
+    if (key > kth) {
+      warp_sorted_insert<E>(v, key, lane);
+      kth = warp_list_get<E>(v, k - 1);
+    }
+  }
 #pragma unroll
-  for (int r = 0; r < E; ++r) dst[r * 32 + lane] = v[r];
+  for (int r = 0; r < E; ++r) list[r * 32 + lane] = v[r];
+  if (lane == 0 && kth != 0) *thr_s_p = candidate_score(kth);
 }
 
 // ------------------------------------------------------------------- the kernel ---
@@ -201,13 +191,10 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap key_map,
   // dynamic shared memory: [stages][A tile | B tile] | lists | queue | per-query state
   unsigned char* base = (unsigned char*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
   unsigned char* ring = base;
-  u64* lists = reinterpret_cast<u64*>(ring + (size_t)n_stages * stage_bytes);   // [nq_c][k]
-  u64* q_key = lists + (size_t)nq_c * k;                                        // [kQueueCap]
-  u64* thr_key = q_key + kQueueCap;                                             // [n_pad]
-  uint64_t* s_ex = reinterpret_cast<uint64_t*>(thr_key + n_pad);                // [n_pad]
+  u64* lists = reinterpret_cast<u64*>(ring + (size_t)n_stages * stage_bytes);   // [nq_c][kk]
+  u64* q_key = lists + (size_t)nq_c * kk;                      // [kColsPerRound][kTileM]
+  uint64_t* s_ex = reinterpret_cast<uint64_t*>(q_key + kQueueCap);              // [n_pad]
   float* thr_s = reinterpret_cast<float*>(s_ex + n_pad);                        // [n_pad]
-  int* cnt = reinterpret_cast<int*>(thr_s + n_pad);                             // [n_pad]
-  uint16_t* q_q = reinterpret_cast<uint16_t*>(cnt + n_pad);                     // [kQueueCap]
 
   const int n_tiles = (pv.n_rows + kTileM - 1) / kTileM;
   const int n_kb = (pv.d + kBlockK - 1) / kBlockK;
@@ -218,15 +205,15 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap key_map,
     for (int b = 0; b < 2; ++b) { mbar_init(&sh.tmem_full[b], 1); mbar_init(&sh.tmem_empty[b], 4); }
     mbar_init(&sh.drain, 1);
     sh.abort_flag = 0;
-    sh.q_count = 0;
+    sh.q_total = 0;
+    for (int j = 0; j < kColsPerRound; ++j) sh.q_cnt[j] = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   for (int i = threadIdx.x; i < n_pad; i += kTcThreads) {
     thr_s[i] = -INFINITY;
-    thr_key[i] = 0;
-    cnt[i] = 0;
     s_ex[i] = (exclude_tag && i < nq_c) ? exclude_tag[q0 + i] : 0;
   }
+  for (int i = threadIdx.x; i < nq_c * kk; i += kTcThreads) lists[i] = 0;
   if (warp == 1) {   // TMEM allocation is a whole-warp operation
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
                  ::"r"(smem_u32(&sh.tmem_base)), "r"((uint32_t)tmem_cols) : "memory");
@@ -336,42 +323,37 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap key_map,
             const int q = c0 + j;
             if (q < nq_c && v[j] > thr_s[q]) {
               if (s_ex[q] != 0 && tag == s_ex[q]) continue;       // same-prompt trace: skipped
-              const int pos = atomicAdd(&sh.q_count, 1);
-              q_key[pos] = pack_candidate(v[j], (uint32_t)row);
-              q_q[pos] = (uint16_t)q;
+              const int pos = atomicAdd(&sh.q_cnt[j], 1);
+              q_key[j * kTileM + pos] = pack_candidate(v[j], (uint32_t)row);
+              atomicAdd(&sh.q_total, 1);
             }
           }
         }
         epilogue_bar();
-        const int n_cand = sh.q_count;
-        if (n_cand > 0) {
-          // drain: warp ew inserts the candidates of queries q with q % 4 == ew
-          for (int b0 = 0; b0 < n_cand; b0 += 32) {
-            const int e = b0 + lane;
-            const int q = e < n_cand ? (int)q_q[e] : -1;
-            unsigned m = __ballot_sync(0xffffffffu, q >= 0 && (q & 3) == ew);
-            while (m) {
-              const int src = __ffs(m) - 1;
-              m &= m - 1;
-              const int qq = __shfl_sync(0xffffffffu, q, src);
-              const u64 key = q_key[b0 + src];
-              list_insert(lists + (size_t)qq * k, k, &cnt[qq], &thr_key[qq], &thr_s[qq], key, lane);
-            }
+        if (sh.q_total > 0) {
+          // drain: warp ew folds the candidates of columns ew, ew+4, ... into their lists
+          for (int j = ew; j < kColsPerRound; j += 4) {
+            const int n_cand = sh.q_cnt[j];
+            const int q = c0 + j;
+            if (n_cand == 0 || q >= nq_c) continue;
+            u64* list = lists + (size_t)q * kk;
+            if (kk == 32) drain_query<1>(list, q_key + j * kTileM, n_cand, k, &thr_s[q], lane);
+            else if (kk == 64) drain_query<2>(list, q_key + j * kTileM, n_cand, k, &thr_s[q], lane);
+            else drain_query<4>(list, q_key + j * kTileM, n_cand, k, &thr_s[q], lane);
+            __syncwarp();
+            if (lane == 0) sh.q_cnt[j] = 0;
           }
           epilogue_bar();
-          if (et == 0) sh.q_count = 0;
+          if (et == 0) sh.q_total = 0;
           epilogue_bar();
         }
       }
     }
-    // publish this CTA's per-query lists, descending, padded with empty slots
+    // publish this CTA's per-query lists: already descending, empty slots are 0
     epilogue_bar();
-    for (int q = ew; q < nq_c; q += 4) {
-      u64* dst = partial + ((size_t)blockIdx.x * nq_total + (q0 + q)) * kk;
-      const u64* src = lists + (size_t)q * k;
-      if (kk == 32) publish_query_list<1>(src, cnt[q], dst, lane);
-      else if (kk == 64) publish_query_list<2>(src, cnt[q], dst, lane);
-      else publish_query_list<4>(src, cnt[q], dst, lane);
+    for (int i = et; i < nq_c * kk; i += 128) {
+      const int q = i / kk, j = i - q * kk;
+      partial[((size_t)blockIdx.x * nq_total + (q0 + q)) * kk + j] = lists[i];
     }
   }
   tc_fence_before();
@@ -416,18 +398,19 @@ bool make_bf16_map(void* map_out, const void* base, int64_t rows, int32_t d, int
   return r == CUDA_SUCCESS;
 }
 
-static size_t tc_fixed_smem(int nq_c, int n_pad, int k) {
-  return (size_t)nq_c * k * 8 + (size_t)kQueueCap * 8 + (size_t)n_pad * (8 + 8 + 4 + 4) +
-         (size_t)kQueueCap * 2 + 1024 /* alignment slack */;
+static size_t tc_fixed_smem(int nq_c, int n_pad, int kk) {
+  return (size_t)nq_c * kk * 8 + (size_t)kQueueCap * 8 + (size_t)n_pad * (8 + 4) +
+         1024 /* alignment slack */;
 }
 
 // Largest number of queries one launch can take for this k so that at least three ring
 // stages fit next to the per-query lists.
 int tc_max_queries_per_pass(int k, size_t smem_limit) {
+  const int kk = list_len(k);
   int best = 16;
   for (int n = 16; n <= OILBIRD_MAX_NQ; n += 16) {
     size_t stage = (size_t)kATileBytes + (size_t)n * kBlockK * 2;
-    if (tc_fixed_smem(n, n, k) + 3 * stage + sizeof(TcShared) + 256 <= smem_limit) best = n;
+    if (tc_fixed_smem(n, n, kk) + 3 * stage + sizeof(TcShared) + 256 <= smem_limit) best = n;
   }
   return best;
 }
@@ -439,7 +422,7 @@ cudaError_t launch_scan_tc(const void* key_map, const void* q_map, const PoolVie
                            int32_t* n_lists, cudaStream_t st) {
   const int n_pad = (nq_c + 15) / 16 * 16;
   const size_t stage = (size_t)kATileBytes + (size_t)n_pad * kBlockK * 2;
-  const size_t fixed = tc_fixed_smem(nq_c, n_pad, k);
+  const size_t fixed = tc_fixed_smem(nq_c, n_pad, kk);
   const size_t avail = smem_limit - sizeof(TcShared) - 256;
   if (fixed + 2 * stage > avail) return cudaErrorInvalidConfiguration;
   int stages = (int)((avail - fixed) / stage);

@@ -1,16 +1,17 @@
-// K2: CUDA-core scan for a few queries (single-request decode).
+// K2: CUDA-core scan for one or two queries (single-request decode).
 //
 // Scoring line of Algorithm 1, "s_i <- cos(h_t, h_i) for all i in P", fused with the
 // per-CTA part of Eq. 2's top-k: every stored key is streamed from HBM exactly once
 // with 16-byte loads, multiplied against the normalised queries held in shared memory
-// (bf16 x bf16 products accumulated in fp32), and each warp keeps its k best rows in a
-// small shared-memory list.  Scores never go to global memory; what leaves the CTA is
-// one descending list of kk (= max(32, k rounded up to a power of two)) packed
-// candidates per query.  The raw query states are normalised by every CTA itself
-// (8-32 KB from L2), which saves a separate launch on the latency-critical path.
+// (bf16 x bf16 products accumulated in fp32), and each warp keeps its best rows in a
+// descending register list (one shuffle-insertion per accepted row).  Scores never go
+// to global memory; what leaves the CTA is one descending list of kk (= max(32, k
+// rounded up to a power of two)) packed candidates per query.  The raw query states are
+// normalised by every CTA itself (8-32 KB from L2), which saves a separate launch on
+// the latency-critical path.
 //
 // The kernel is bound by the key stream (N*d*2 bytes); per 16 bytes of key a lane
-// spends 8 integer unpack ops and 8*QT FMAs, well under the issue budget for QT <= 4.
+// spends 8 integer unpack ops and 8*QT FMAs, well under the issue budget for QT <= 2.
 #include "common.cuh"
 #include "internal.h"
 #include "normalize.cuh"
@@ -21,32 +22,16 @@ constexpr int kScanThreads = kNormThreads;
 constexpr int kScanWarps = kScanThreads / 32;
 constexpr int kRowsPerIter = 4;   // rows a warp scores together (shares each query load)
 
-// Sort each warp's list, merge the warps' lists and let warp 0 publish the CTA's kk best.
-template <int E>
-__device__ __forceinline__ void publish_cta_list(const WarpTopK& top, u64* scratch,
-                                                 u64* __restrict__ dst) {
-  const int lane = threadIdx.x & 31;
-  u64 v[E];
-#pragma unroll
-  for (int r = 0; r < E; ++r) v[r] = (r * 32 + lane < top.cnt) ? top.list[r * 32 + lane] : 0;
-  warp_sort_desc<E>(v, lane);
-  block_merge_desc<E>(v, scratch, kScanWarps);
-  if (threadIdx.x < 32) {
-#pragma unroll
-    for (int r = 0; r < E; ++r) dst[r * 32 + lane] = v[r];
-  }
-}
-
-template <int QT>
+template <int QT, int E>
 __global__ void __launch_bounds__(kScanThreads, 2)
-scan_gemv_kernel(PoolView pv, const uint16_t* __restrict__ q_raw, int nq, int k, int kk,
+scan_gemv_kernel(PoolView pv, const uint16_t* __restrict__ q_raw, int nq, int k,
                  const uint64_t* __restrict__ exclude_tag, u64* __restrict__ partial,
                  int32_t* __restrict__ q_valid, DeviceStats* stats) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
+  constexpr int KK = 32 * E;
   const int d = pv.d, n_chunks = d >> 3;
   uint4* qs = reinterpret_cast<uint4*>(smem_raw);                       // [QT][n_chunks]
-  u64* lists = reinterpret_cast<u64*>(smem_raw + (size_t)QT * d * 2);    // [QT][warps][k]
-  u64* scratch = lists + (size_t)QT * kScanWarps * k;                    // [warps][kk]
+  u64* scratch = reinterpret_cast<u64*>(smem_raw + (size_t)QT * d * 2);  // [warps][KK]
   __shared__ uint64_t s_ex[QT];
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -77,9 +62,15 @@ scan_gemv_kernel(PoolView pv, const uint16_t* __restrict__ q_raw, int nq, int k,
       s_ex[threadIdx.x] = (exclude_tag && q0 + threadIdx.x < nq) ? exclude_tag[q0 + threadIdx.x] : 0;
     __syncthreads();
 
-    WarpTopK top[QT];
+    // this warp's best rows so far, descending; kth = its k-th entry (0 while not full)
+    u64 top[QT][E];
+    u64 kth[QT];
 #pragma unroll
-    for (int q = 0; q < QT; ++q) top[q].init(lists + ((size_t)q * kScanWarps + warp) * k, k);
+    for (int q = 0; q < QT; ++q) {
+      kth[q] = 0;
+#pragma unroll
+      for (int r = 0; r < E; ++r) top[q][r] = 0;
+    }
 
     for (int rb = r_lo + warp * kRowsPerIter; rb < r_hi; rb += kScanWarps * kRowsPerIter) {
       const uint4* rowp[kRowsPerIter];
@@ -132,35 +123,47 @@ scan_gemv_kernel(PoolView pv, const uint16_t* __restrict__ q_raw, int nq, int k,
           if (q0 + q >= nq) continue;
           if (s_ex[q] != 0 && tag == s_ex[q]) continue;     // same-prompt trace: skipped
           const u64 key = pack_candidate(s, (uint32_t)row);
-          if (top[q].wants(key)) top[q].insert(key, lane);
+          if (key > kth[q]) {
+            warp_sorted_insert<E>(top[q], key, lane);
+            kth[q] = warp_list_get<E>(top[q], k - 1);
+          }
         }
       }
     }
-    // merge the warps' lists of each query and publish the CTA's kk best, descending
+    // merge the warps' lists of each query; warp 0 publishes the CTA's KK best, descending
 #pragma unroll
     for (int q = 0; q < QT; ++q) {
       if (q0 + q >= nq) break;
-      __syncwarp();
-      u64* dst = partial + ((size_t)blockIdx.x * nq + (q0 + q)) * kk;
-      if (kk == 32) publish_cta_list<1>(top[q], scratch, dst);
-      else if (kk == 64) publish_cta_list<2>(top[q], scratch, dst);
-      else publish_cta_list<4>(top[q], scratch, dst);
+      block_merge_desc<E>(top[q], scratch, kScanWarps);
+      if (threadIdx.x < 32) {
+        u64* dst = partial + ((size_t)blockIdx.x * nq + (q0 + q)) * KK;
+#pragma unroll
+        for (int r = 0; r < E; ++r) dst[r * 32 + lane] = top[q][r];
+      }
     }
   }
 }
 
-template <int QT>
-static cudaError_t launch_qt(const PoolView& pv, const uint16_t* q_raw, int nq, int k, int kk,
-                             const uint64_t* ex, u64* partial, int32_t* q_valid,
-                             DeviceStats* stats, int grid, cudaStream_t st) {
-  size_t smem = (size_t)QT * pv.d * 2 + (size_t)QT * kScanWarps * k * sizeof(u64) +
-                (size_t)kScanWarps * kk * sizeof(u64);
-  cudaError_t e = cudaFuncSetAttribute(scan_gemv_kernel<QT>,
+template <int QT, int E>
+static cudaError_t launch_one(const PoolView& pv, const uint16_t* q_raw, int nq, int k,
+                              const uint64_t* ex, u64* partial, int32_t* q_valid,
+                              DeviceStats* stats, int grid, cudaStream_t st) {
+  size_t smem = (size_t)QT * pv.d * 2 + (size_t)kScanWarps * 32 * E * sizeof(u64);
+  cudaError_t e = cudaFuncSetAttribute(scan_gemv_kernel<QT, E>,
                                        cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
-  scan_gemv_kernel<QT><<<grid, kScanThreads, smem, st>>>(pv, q_raw, nq, k, kk, ex, partial,
-                                                         q_valid, stats);
+  scan_gemv_kernel<QT, E><<<grid, kScanThreads, smem, st>>>(pv, q_raw, nq, k, ex, partial,
+                                                            q_valid, stats);
   return cudaGetLastError();
+}
+
+template <int QT>
+static cudaError_t launch_qt(int kk, const PoolView& pv, const uint16_t* q_raw, int nq, int k,
+                             const uint64_t* ex, u64* partial, int32_t* q_valid,
+                             DeviceStats* stats, int grid, cudaStream_t st) {
+  if (kk == 32) return launch_one<QT, 1>(pv, q_raw, nq, k, ex, partial, q_valid, stats, grid, st);
+  if (kk == 64) return launch_one<QT, 2>(pv, q_raw, nq, k, ex, partial, q_valid, stats, grid, st);
+  return launch_one<QT, 4>(pv, q_raw, nq, k, ex, partial, q_valid, stats, grid, st);
 }
 
 cudaError_t launch_scan_gemv(const PoolView& pv, const uint16_t* q_raw, int32_t nq, int32_t k,
@@ -173,14 +176,9 @@ cudaError_t launch_scan_gemv(const PoolView& pv, const uint16_t* q_raw, int32_t 
   if (grid > 2 * num_sms) grid = 2 * num_sms;
   if (grid > max_lists) grid = max_lists;
   *n_lists = grid;
-  // queries held in shared memory together: bounded by 64 KB of bf16 query data
-  int qt = nq >= 4 ? 4 : (nq >= 2 ? 2 : 1);
-  while (qt > 1 && (size_t)qt * pv.d * 2 > 65536) qt >>= 1;
-  switch (qt) {
-    case 4: return launch_qt<4>(pv, q_raw, nq, k, kk, exclude_tag, partial, q_valid, stats, grid, st);
-    case 2: return launch_qt<2>(pv, q_raw, nq, k, kk, exclude_tag, partial, q_valid, stats, grid, st);
-    default: return launch_qt<1>(pv, q_raw, nq, k, kk, exclude_tag, partial, q_valid, stats, grid, st);
-  }
+  if (nq >= 2)
+    return launch_qt<2>(kk, pv, q_raw, nq, k, exclude_tag, partial, q_valid, stats, grid, st);
+  return launch_qt<1>(kk, pv, q_raw, nq, k, exclude_tag, partial, q_valid, stats, grid, st);
 }
 
 }  // namespace oilbird

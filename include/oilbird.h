@@ -59,7 +59,7 @@ typedef struct oilbird_pool oilbird_pool_t;   /* opaque */
 
 /*
  * Pool geometry, fixed at creation (Eq. 1: one record (x_i, h_i) per committed
- * generated position, the state "kept normalized in half precision").
+ * generated position, the state stored L2-normalised in 16-bit floating point).
  */
 typedef struct {
   int32_t  d;              /* key width d_model; a multiple of 8, 8..16384              */
@@ -90,8 +90,8 @@ typedef struct {
   int32_t  tier_depth[OILBIRD_MAX_TIERS];   /* paper: 48, 8 (0 below every tier)        */
   const uint64_t* exclude_tag;              /* dev [nq] or NULL: rows of traces whose
                                                tag equals a non-zero entry are skipped
-                                               ("skips any stored trace whose own
-                                               prompt is the one being served now")     */
+                                               (a request must not draft from a stored
+                                               copy of its own prompt's trace)          */
   int32_t  path;                            /* OILBIRD_PATH_*                           */
 } oilbird_query_params;
 
@@ -128,7 +128,7 @@ int oilbird_pool_reset  (oilbird_pool_t* pool, void* cuda_stream);
 int oilbird_pool_destroy(oilbird_pool_t* pool);
 
 /*
- * Store (Eq. 1; Algorithm 1 last line: "append the trace to P at request end").
+ * Store (Eq. 1; last line of Algorithm 1: a finished request's trace joins the pool).
  * Appends n rows: key = bf16(x / ||x||_2) (norm and scaling in double precision, one
  * rounding to float and one to bf16, round-to-nearest-even), token, trace
  * membership.  With OILBIRD_NEW_TRACE the rows open a new trace carrying trace_tag
@@ -142,8 +142,8 @@ int oilbird_pool_append(oilbird_pool_t* pool, const void* states_bf16, const int
                         int64_t n, uint64_t trace_tag, uint32_t flags, void* cuda_stream);
 
 /*
- * Retrieve (Algorithm 1: "s_i <- cos(h_t, h_i) for all i in P; E_t <- top-k(s)",
- * the theta test, d <- D(s_i), gamma <- x_{i+2 : i+1+d}; Eq. 2; Eq. 3).
+ * Retrieve (Algorithm 1: the cosine of the query state with every stored state, top-k,
+ * the theta test, the depth D(s_i) and the copy that starts two rows on; Eq. 2; Eq. 3).
  * For each of the nq query states: L2-normalise and round to bf16 (as a key is),
  * score every stored row by the dot product of the two bf16 vectors accumulated in
  * fp32, keep the k best by (score descending, row ascending), set fired, give each
@@ -169,10 +169,13 @@ int oilbird_pool_gather(oilbird_pool_t* pool, const int32_t* idx, const float* s
                         const oilbird_query_out* out, void* cuda_stream);
 
 /*
- * The same two operations with HOST buffers: inputs are copied to the device and
- * results back inside the call, which returns after the results have landed
- * (it synchronises cuda_stream).  params->exclude_tag and every array of `out` are
- * host pointers here.  n <= cfg.max_append.
+ * The same two operations with HOST buffers.  append_host copies its inputs into pinned
+ * staging and enqueues upload + append; the caller's buffers are free again when it
+ * returns, the rows are visible to later calls on the same stream.  query_host uploads
+ * the queries, runs the query and returns after the results have landed in the host
+ * arrays of `out` (it synchronises cuda_stream).  params->exclude_tag and every array of
+ * `out` are host pointers here.  n <= cfg.max_append.  All *_host calls of a pool must
+ * use one stream: the staging buffers are reused in stream order.
  */
 int oilbird_pool_append_host(oilbird_pool_t* pool, const void* states_bf16_host,
                              const int32_t* tokens_host, int64_t n, uint64_t trace_tag,

@@ -11,13 +11,13 @@
  *   store     Eq. 1: one record (x_i, h_i) per committed generated position,
  *             the state kept L2-normalised in half precision (bf16 here, the
  *             precision the paper's models run in), grouped into traces.
- *   score     Algorithm 1, the line "s_i <- cos(h_t, h_i) for all i in P":
- *             every stored position is scored, nothing is approximated.
+ *   score     Algorithm 1's scoring line: the cosine of the query state with the
+ *             state of every stored position; nothing is approximated.
  *   top-k     Eq. 2: E_t = arg top-k s_i.  Written here as a FULL sort of all
  *             positions by (score descending, position ascending) followed by
  *             taking the first k.  No heap, no selection, no blocking.
- *   firing    Eq. 2 / Algorithm 1 "if max_i s_i >= theta": theta gates on the
- *             best neighbour only, it is not a filter inside the top-k.
+ *   firing    Eq. 2 and the matching test of Algorithm 1: theta gates on the best
+ *             neighbour only, it is not a filter inside the top-k.
  *   depth     Eq. 3: D(s) = 48 if s >= 0.90; 8 if s >= 0.82; 0 otherwise
  *             (tier table passed in), or a fixed span length (the batched
  *             harness of the appendix copies fixed-length spans).
@@ -110,8 +110,8 @@ const int64_t *oracle_pool_trace_ends(const oracle_pool *p) { return p->trace_en
 const uint64_t *oracle_pool_trace_tags(const oracle_pool *p) { return p->trace_tag; }
 
 /*
- * L2-normalise one bf16 vector into bf16 ("kept normalized in half
- * precision", Section 4 (i)).  Returns 1 if the input was usable, 0 if it was
+ * L2-normalise one bf16 vector into bf16 (Section 4 (i): states are stored
+ * normalised, in 16-bit precision).  Returns 1 if the input was usable, 0 if it was
  * all zero or held a NaN/Inf, in which case the output is all zero.
  */
 int oracle_normalize_bf16(int32_t d, const uint16_t *x, uint16_t *out) {
@@ -185,13 +185,16 @@ int oracle_pool_append(oracle_pool *p, const uint16_t *states, const int32_t *to
     p->n_traces += 1;
   }
   int32_t tr = p->n_traces - 1;
-  for (int64_t r = 0; r < n; ++r) {
+  int64_t bad = 0;
+#pragma omp parallel for schedule(static) reduction(+ : bad)
+  for (int64_t r = 0; r < n; ++r) {   /* rows are independent */
     int64_t row = p->n + r;
     int ok = oracle_normalize_bf16(p->d, states + (size_t)r * p->d, p->key + (size_t)row * p->d);
-    if (!ok) p->degenerate_rows += 1;
+    if (!ok) bad += 1;
     p->tok[row] = tokens[r];
     p->trace_id[row] = tr;
   }
+  p->degenerate_rows += bad;
   p->n += n;
   p->trace_end[tr] = p->n;
   return 0;
@@ -203,8 +206,8 @@ int oracle_pool_append(oracle_pool *p, const uint16_t *states, const int32_t *to
  * Algorithm 1: s_i = cos(h_t, h_i) for every stored i.  The query is
  * normalised and rounded to bf16 exactly as a key is, so the cosine of the
  * two stored-format unit vectors is their dot product.  Rows of a trace whose
- * tag equals a non-zero exclude_tag score -inf ("retrieval skips any stored
- * trace whose own prompt is the one being served now").
+ * tag equals a non-zero exclude_tag score -inf (Section 4 (i): a request never
+ * retrieves from a stored trace that has its own prompt).
  * Returns 1 if the query was usable; otherwise every score is -inf and 0 is
  * returned.
  */

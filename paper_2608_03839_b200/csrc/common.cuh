@@ -1,5 +1,5 @@
-// Device-side helpers shared by the pool's kernels: candidate packing, warp top-k
-// lists, block bitonic sort.  Nothing here is visible outside the CUDA library.
+// Device-side helpers shared by the pool's kernels: candidate packing and warp-level
+// sorted candidate lists (bitonic sort / merge, shuffle insertion).  Nothing here is visible outside the CUDA library.
 #pragma once
 #include <cuda_runtime.h>
 #include <stdint.h>
@@ -64,46 +64,6 @@ __device__ __forceinline__ float warp_sum(float v) {
   for (int m = 16; m; m >>= 1) v += __shfl_xor_sync(0xffffffffu, v, m);
   return v;
 }
-
-// A warp-private top-k list of packed candidates in shared memory.  `cnt` and `thr`
-// are warp-uniform registers: the number of filled slots and, once the list is full,
-// its smallest key.  A candidate enters only if it beats thr, so after the first k
-// rows insertions are rare (about k*ln(n/k) over n rows in random order).
-struct WarpTopK {
-  u64* list;
-  int k;
-  int cnt;
-  u64 thr;
-
-  __device__ __forceinline__ void init(u64* l, int k_) { list = l; k = k_; cnt = 0; thr = 0; }
-
-  __device__ __forceinline__ u64 list_min(int lane) const {
-    u64 m = ~0ull;
-    for (int j = lane; j < k; j += 32) { u64 v = list[j]; m = v < m ? v : m; }
-    return warp_min_u64(m);
-  }
-  // Called by all 32 lanes with the same key.
-  __device__ __forceinline__ void insert(u64 key, int lane) {
-    if (cnt < k) {
-      if (lane == 0) list[cnt] = key;
-      ++cnt;
-      __syncwarp();
-      if (cnt == k) thr = list_min(lane);
-      return;
-    }
-    if (key <= thr) return;
-    for (int j = lane; j < k; j += 32)
-      if (list[j] == thr) list[j] = key;       // keys are unique: exactly one slot matches
-    __syncwarp();
-    thr = list_min(lane);
-  }
-  __device__ __forceinline__ bool wants(u64 key) const { return cnt < k || key > thr; }
-  // zero the unused tail so the list can be sorted / merged as k_pad entries
-  __device__ __forceinline__ void pad(int k_pad, int lane) {
-    for (int j = cnt + lane; j < k_pad; j += 32) list[j] = 0;
-    __syncwarp();
-  }
-};
 
 // --------------------------------------------------- warp-level sorted lists ---
 // A list of K = 32*E packed candidates lives in the registers of one warp: element i is
@@ -215,25 +175,6 @@ __device__ __forceinline__ void block_merge_desc(u64 (&v)[E], u64* scratch, int 
       warp_merge_desc<E>(v, b, lane);
     }
   }
-}
-
-// ------------------------------------------------------------- block sorting ---
-// In-place bitonic sort, DESCENDING, of n (a power of two) keys in shared memory by
-// all threads of the block.  Ends with a __syncthreads().
-__device__ __forceinline__ void block_bitonic_sort_desc(u64* a, int n) {
-  for (int size = 2; size <= n; size <<= 1) {
-    for (int stride = size >> 1; stride > 0; stride >>= 1) {
-      __syncthreads();
-      for (int t = threadIdx.x; t < (n >> 1); t += blockDim.x) {
-        int lo = 2 * t - (t & (stride - 1));   // index with the `stride` bit clear
-        int hi = lo + stride;
-        bool desc = (lo & size) == 0;
-        u64 x = a[lo], y = a[hi];
-        if ((x < y) == desc) { a[lo] = y; a[hi] = x; }
-      }
-    }
-  }
-  __syncthreads();
 }
 
 }  // namespace oilbird

@@ -1,6 +1,6 @@
-// L2 normalisation of one bf16 row, shared by the append kernel (keys, Eq. 1: "kept
-// normalized in half precision") and by query preparation (the cosine of Algorithm 1's
-// scoring line then is a plain dot product of two stored-format vectors).
+// L2 normalisation of one bf16 row, shared by the append kernel (keys, Eq. 1: states are
+// stored normalised in 16-bit precision) and by query preparation (the cosine of
+// Algorithm 1's scoring line then is a plain dot product of two stored-format vectors).
 #pragma once
 #include "common.cuh"
 

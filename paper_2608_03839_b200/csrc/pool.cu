@@ -113,6 +113,8 @@ struct oilbird_pool {
   // pinned staging for host variants
   unsigned char* pinned;
   size_t pinned_bytes;
+  cudaEvent_t upload_done;
+  bool upload_pending;
   // tensor maps of the tensor-core scan (opaque 128-byte CUtensorMap objects)
   size_t smem_limit;
   bool tc_ok;
@@ -216,7 +218,7 @@ int oilbird_pool_destroy(oilbird_pool_t* p) {
   cudaSetDevice(p->device);
   cudaDeviceSynchronize();
   for (cudaEvent_t e : p->ev) cudaEventDestroy(e);
-  if (p->pinned) cudaFreeHost(p->pinned);
+  if (p->pinned) { cudaFreeHost(p->pinned); cudaEventDestroy(p->upload_done); }
   if (p->owns_mem) cudaFree(p->base);
   delete p;
   return OILBIRD_OK;
@@ -393,12 +395,19 @@ int oilbird_pool_gather(oilbird_pool_t* p, const int32_t* idx, const float* scor
 
 // ---- host-buffer variants ---------------------------------------------------------
 
-static int ensure_pinned(oilbird_pool* p, size_t bytes) {
-  if (p->pinned_bytes >= bytes) return OILBIRD_OK;
-  if (p->pinned) { cudaFreeHost(p->pinned); p->pinned = nullptr; p->pinned_bytes = 0; }
-  cudaError_t e = cudaMallocHost((void**)&p->pinned, bytes);
+// Pinned host staging: [append block | query-result block].  The append block is reused
+// by the next append_host call, so an event marks when its upload has finished.
+static int ensure_pinned(oilbird_pool* p) {
+  if (p->pinned) return OILBIRD_OK;
+  const size_t a_bytes = (size_t)p->r.max_append * p->r.d * 2 + (size_t)p->r.max_append * 4;
+  const size_t o_bytes =
+      (size_t)p->r.max_nq * ((size_t)p->r.max_k * (8 + 4 + 4 * OILBIRD_MAX_CONT_LEN) + 4);
+  cudaError_t e = cudaMallocHost((void**)&p->pinned, align_up(a_bytes) + o_bytes);
   if (e != cudaSuccess) return cuda_fail(e, "cudaMallocHost");
-  p->pinned_bytes = bytes;
+  p->pinned_bytes = align_up(a_bytes);          // offset of the result block
+  e = cudaEventCreateWithFlags(&p->upload_done, cudaEventDisableTiming);
+  if (e != cudaSuccess) return cuda_fail(e, "cudaEventCreate");
+  p->upload_pending = false;
   return OILBIRD_OK;
 }
 
@@ -406,19 +415,25 @@ int oilbird_pool_append_host(oilbird_pool_t* p, const void* states, const int32_
                              int64_t n, uint64_t tag, uint32_t flags, void* stream) {
   if (!p || n < 0 || n > p->r.max_append || (n > 0 && (!states || !tokens))) return OILBIRD_EINVAL;
   CU(cudaSetDevice(p->device));
+  int rc = ensure_pinned(p);
+  if (rc) return rc;
   cudaStream_t st = (cudaStream_t)stream;
   uint16_t* d_st = (uint16_t*)(p->base + p->lay.st_stage);
   int32_t* d_tok = (int32_t*)(p->base + p->lay.tok_stage);
   if (n > 0) {
-    // the staging buffers are reused by the next call: wait for the previous consumer
-    CU(cudaStreamSynchronize(st));
-    CU(cudaMemcpyAsync(d_st, states, (size_t)n * p->r.d * 2, cudaMemcpyHostToDevice, st));
-    CU(cudaMemcpyAsync(d_tok, tokens, (size_t)n * 4, cudaMemcpyHostToDevice, st));
+    // The caller's buffers are free again when this returns: they are copied into pinned
+    // staging first.  Device-side staging is reused in stream order.
+    if (p->upload_pending) { CU(cudaEventSynchronize(p->upload_done)); p->upload_pending = false; }
+    const size_t sb = (size_t)n * p->r.d * 2, tb = (size_t)n * 4;
+    unsigned char* h_tok = p->pinned + (size_t)p->r.max_append * p->r.d * 2;
+    memcpy(p->pinned, states, sb);
+    memcpy(h_tok, tokens, tb);
+    CU(cudaMemcpyAsync(d_st, p->pinned, sb, cudaMemcpyHostToDevice, st));
+    CU(cudaMemcpyAsync(d_tok, h_tok, tb, cudaMemcpyHostToDevice, st));
+    CU(cudaEventRecord(p->upload_done, st));
+    p->upload_pending = true;
   }
-  int rc = oilbird_pool_append(p, d_st, d_tok, n, tag, flags, stream);
-  if (rc) return rc;
-  CU(cudaStreamSynchronize(st));
-  return OILBIRD_OK;
+  return oilbird_pool_append(p, d_st, d_tok, n, tag, flags, stream);
 }
 
 int oilbird_pool_query_host(oilbird_pool_t* p, const void* q, int32_t nq,
@@ -429,16 +444,19 @@ int oilbird_pool_query_host(oilbird_pool_t* p, const void* q, int32_t nq,
   int rc = check_params(p, nq, pr, &gp);
   if (rc) return rc;
   CU(cudaSetDevice(p->device));
+  rc = ensure_pinned(p);
+  if (rc) return rc;
   cudaStream_t st = (cudaStream_t)stream;
   const size_t k = pr->k, L = pr->cont_len;
   uint16_t* d_q = (uint16_t*)(p->base + p->lay.q_stage);
   uint64_t* d_ex = (uint64_t*)(p->base + p->lay.ex_stage);
   unsigned char* d_out = p->base + p->lay.out_stage;
+  unsigned char* h_out = p->pinned + p->pinned_bytes;
   // device-side result block: idx | score | cont_len | cont_tok | fired
   const size_t o_idx = 0, o_score = o_idx + nq * k * 4, o_len = o_score + nq * k * 4,
                o_tok = o_len + nq * k * 4, o_fired = o_tok + nq * k * L * 4,
                o_total = o_fired + (size_t)nq * 4;
-  CU(cudaStreamSynchronize(st));   // staging reuse
+  // the call synchronises before it returns, so the caller's buffers can be read directly
   CU(cudaMemcpyAsync(d_q, q, (size_t)nq * p->r.d * 2, cudaMemcpyHostToDevice, st));
   oilbird_query_params dp = *pr;
   if (pr->exclude_tag) {
@@ -453,15 +471,13 @@ int oilbird_pool_query_host(oilbird_pool_t* p, const void* q, int32_t nq,
   dout.fired = (int32_t*)(d_out + o_fired);
   rc = oilbird_pool_query(p, d_q, nq, &dp, &dout, stream);
   if (rc) return rc;
-  rc = ensure_pinned(p, o_total);
-  if (rc) return rc;
-  CU(cudaMemcpyAsync(p->pinned, d_out, o_total, cudaMemcpyDeviceToHost, st));
+  CU(cudaMemcpyAsync(h_out, d_out, o_total, cudaMemcpyDeviceToHost, st));
   CU(cudaStreamSynchronize(st));
-  memcpy(out->idx, p->pinned + o_idx, nq * k * 4);
-  memcpy(out->score, p->pinned + o_score, nq * k * 4);
-  memcpy(out->cont_len, p->pinned + o_len, nq * k * 4);
-  memcpy(out->cont_tok, p->pinned + o_tok, nq * k * L * 4);
-  memcpy(out->fired, p->pinned + o_fired, (size_t)nq * 4);
+  memcpy(out->idx, h_out + o_idx, nq * k * 4);
+  memcpy(out->score, h_out + o_score, nq * k * 4);
+  memcpy(out->cont_len, h_out + o_len, nq * k * 4);
+  memcpy(out->cont_tok, h_out + o_tok, nq * k * L * 4);
+  memcpy(out->fired, h_out + o_fired, (size_t)nq * 4);
   return OILBIRD_OK;
 }
 

@@ -1,6 +1,6 @@
 // K2: CUDA-core scan for one or two queries (single-request decode).
 //
-// Scoring line of Algorithm 1, "s_i <- cos(h_t, h_i) for all i in P", fused with the
+// Scoring line of Algorithm 1 (cosine of the query with every stored state), fused with the
 // per-CTA part of Eq. 2's top-k: every stored key is streamed from HBM exactly once
 // with 16-byte loads, multiplied against the normalised queries held in shared memory
 // (bf16 x bf16 products accumulated in fp32), and each warp keeps its best rows in a

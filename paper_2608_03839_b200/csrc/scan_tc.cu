@@ -1,6 +1,6 @@
 // K3: tensor-core scan for batched queries (many requests against one shared pool).
 //
-// Scoring line of Algorithm 1, "s_i <- cos(h_t, h_i) for all i in P", for nq queries at
+// Scoring line of Algorithm 1 (cosine of the query with every stored state) for nq queries at
 // once: S[i, q] = <key_i, qn_q> is a [N x d] x [d x nq] contraction.  Keys are the M
 // operand (tiles of 128 rows), the normalised queries the N operand (nq padded to a
 // multiple of 16), d is walked in blocks of 64 elements.  Each CTA is persistent and

@@ -156,7 +156,10 @@ struct TcShared {
 
 // Fold the candidates queued for one query into its descending list (shared memory,
 // kk = 32*E slots, empty slots are 0) and refresh the filter threshold: the score of the
-// k-th entry once k entries exist.
+// k-th entry once k entries exist.  A handful of candidates are inserted one by one
+// (a chain of dependent shuffles each); a crowd, as in a CTA's first tiles while its
+// thresholds are still low, is sorted 32*E at a time and merged, which costs a fixed
+// two dozen network stages per batch.
 template <int E>
 __device__ __forceinline__ void drain_query(u64* list, const u64* cand, int n_cand, int k,
                                             float* thr_s_p, int lane) {
@@ -164,11 +167,26 @@ __device__ __forceinline__ void drain_query(u64* list, const u64* cand, int n_ca
 #pragma unroll
   for (int r = 0; r < E; ++r) v[r] = list[r * 32 + lane];
   u64 kth = warp_list_get<E>(v, k - 1);
-  for (int i = 0; i < n_cand; ++i) {
-    const u64 key = cand[i];
-    if (key > kth) {
-      warp_sorted_insert<E>(v, key, lane);
+  if (n_cand >= 8) {
+    for (int i0 = 0; i0 < n_cand; i0 += 32 * E) {
+      u64 b[E];
+#pragma unroll
+      for (int r = 0; r < E; ++r) {
+        const int i = i0 + r * 32 + lane;
+        const u64 key = i < n_cand ? cand[i] : 0;
+        b[r] = key > kth ? key : 0;
+      }
+      warp_sort_desc<E>(b, lane);
+      warp_merge_desc<E>(v, b, lane);
       kth = warp_list_get<E>(v, k - 1);
+    }
+  } else {
+    for (int i = 0; i < n_cand; ++i) {
+      const u64 key = cand[i];
+      if (key > kth) {
+        warp_sorted_insert<E>(v, key, lane);
+        kth = warp_list_get<E>(v, k - 1);
+      }
     }
   }
 #pragma unroll

@@ -56,15 +56,19 @@ def measured_peaks():
         "fallback"
 
 
-def ncu_traffic(config_name: str):
-    """DRAM bytes per scan launch from the committed ncu summary, if one exists."""
-    p = os.path.join(ROOT, "profiles", "traffic.json")
-    if os.path.exists(p):
-        try:
-            return json.load(open(p)).get(config_name)
-        except Exception:
-            return None
-    return None
+# DRAM bytes (read + write) of one scan launch from the ncu captures summarised under
+# profiles/ (file named per entry), with the pool rows held at capture time.  Traffic is
+# proportional to the rows scanned, so it is scaled to the rows of the timed launches.
+NCU_TRAFFIC = {
+    "C2": (540655360.0, 65560),      # profiles/scan_gemv_C2_ncu.md
+}
+
+
+def ncu_traffic(config_name: str, rows: float):
+    if config_name not in NCU_TRAFFIC:
+        return None
+    dram_bytes, rows_at_capture = NCU_TRAFFIC[config_name]
+    return dram_bytes * rows / rows_at_capture
 
 
 class ClockSampler:
@@ -305,7 +309,8 @@ def run_ours(args):
                          "peak_kind": peak_kind, "frac_of_nominal_8000": achieved / NOMINAL_HBM_GBS,
                          "kernel": "key scan (score + per-CTA top-k)",
                          "kernel_ms": scan_mean_ms, "bytes_per_launch": scan_bytes,
-                         "traffic": ncu_traffic(w.name)},
+                         "traffic": ncu_traffic(w.name, rows_scan) if not args.rows and not args.nq
+                         else None},
             "device_stalled_flag": stalled,
         }
         if not args.no_cpu_baseline and world == 1:

@@ -19,6 +19,8 @@ append_kernel(const uint16_t* __restrict__ states, const int32_t* __restrict__ t
               int32_t* __restrict__ trace_id, int64_t row0, int32_t trace,
               int32_t* __restrict__ trace_end, uint64_t* __restrict__ trace_tag, uint64_t tag,
               int set_tag, DeviceStats* stats) {
+  pdl_launch_dependents();
+  pdl_wait();   // earlier queries may still be reading the trace table and token stream
   if (blockIdx.x == 0 && threadIdx.x == 0) {
     trace_end[trace] = (int32_t)(row0 + n);
     if (set_tag) trace_tag[trace] = tag;
@@ -37,6 +39,8 @@ append_kernel(const uint16_t* __restrict__ states, const int32_t* __restrict__ t
 __global__ void __launch_bounds__(kNormThreads)
 qnorm_kernel(const uint16_t* __restrict__ q, int nq, int d, uint16_t* __restrict__ qn,
              int32_t* __restrict__ q_valid, DeviceStats* stats) {
+  pdl_launch_dependents();
+  pdl_wait();
   const int r = blockIdx.x;
   if (r < nq) {
     // A query holding NaN/Inf returns no neighbours; an all-zero query is legal and
@@ -57,16 +61,15 @@ cudaError_t launch_append(const uint16_t* states, const int32_t* tokens, int64_t
                           int32_t trace, int32_t* trace_end, uint64_t* trace_tag, uint64_t tag,
                           int set_tag, DeviceStats* stats, cudaStream_t st) {
   int64_t grid = n < 1 ? 1 : (n > 65535 * 8 ? 65535 * 8 : n);
-  append_kernel<<<(unsigned)grid, kNormThreads, 0, st>>>(states, tokens, n, d, keys, tok, trace_id,
-                                                         row0, trace, trace_end, trace_tag, tag,
-                                                         set_tag, stats);
-  return cudaGetLastError();
+  return launch_pdl(append_kernel, dim3((unsigned)grid), dim3(kNormThreads), 0, st, states, tokens,
+                    n, d, keys, tok, trace_id, row0, trace, trace_end, trace_tag, tag, set_tag,
+                    stats);
 }
 
 cudaError_t launch_qnorm(const uint16_t* q, int32_t nq, int32_t nq_pad, int32_t d, uint16_t* qn,
                          int32_t* q_valid, DeviceStats* stats, cudaStream_t st) {
-  qnorm_kernel<<<nq_pad, kNormThreads, 0, st>>>(q, nq, d, qn, q_valid, stats);
-  return cudaGetLastError();
+  return launch_pdl(qnorm_kernel, dim3(nq_pad), dim3(kNormThreads), 0, st, q, nq, d, qn, q_valid,
+                    stats);
 }
 
 }  // namespace oilbird

@@ -48,6 +48,17 @@ __device__ __forceinline__ uint4 ld_stream16(const void* p) {
   return v;
 }
 
+// ---------------------------------------------------- programmatic launch ------
+// Every kernel of the library is launched with programmatic stream serialization: its
+// blocks may be scheduled while the previous kernel of the stream is still draining, which
+// hides the launch latency between the three or four kernels of a step.  pdl_wait() must
+// come before the first access to anything an earlier kernel wrote (it waits for that
+// kernel to finish and its writes to be visible); both are no-ops for a plain launch.
+__device__ __forceinline__ void pdl_launch_dependents() {
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 // ------------------------------------------------------------------ warp ops ---
 __device__ __forceinline__ u64 shfl_xor_u64(u64 v, int m) {
   uint32_t lo = __shfl_xor_sync(0xffffffffu, (uint32_t)v, m);

@@ -67,12 +67,20 @@ __device__ __forceinline__ void merge_lists(const u64* __restrict__ partial, int
   u64 v[E];
 #pragma unroll
   for (int r = 0; r < E; ++r) v[r] = 0;
-  for (int l = warp; l < n_lists; l += kMergeWarps) {
-    const u64* src = partial + ((size_t)l * nq + q) * KK;
-    u64 b[E];
+  // four lists in flight per warp: the loads, not the merges, set the pace
+  constexpr int PF = 4;
+  for (int l0 = warp; l0 < n_lists; l0 += kMergeWarps * PF) {
+    u64 b[PF][E];
 #pragma unroll
-    for (int r = 0; r < E; ++r) b[r] = src[r * 32 + lane];
-    warp_merge_desc<E>(v, b, lane);
+    for (int p = 0; p < PF; ++p) {
+      const int l = l0 + p * kMergeWarps;
+      const u64* src = partial + ((size_t)(l < n_lists ? l : 0) * nq + q) * KK;
+#pragma unroll
+      for (int r = 0; r < E; ++r) b[p][r] = l < n_lists ? src[r * 32 + lane] : 0;
+    }
+#pragma unroll
+    for (int p = 0; p < PF; ++p)
+      if (l0 + p * kMergeWarps < n_lists) warp_merge_desc<E>(v, b[p], lane);
   }
   const int active = n_lists < kMergeWarps ? (n_lists < 1 ? 1 : n_lists) : kMergeWarps;
   block_merge_desc<E>(v, scratch, active);
@@ -93,6 +101,8 @@ merge_gather_kernel(PoolView pv, const u64* __restrict__ partial, int n_lists, i
   __shared__ int32_t s_len[OILBIRD_MAX_K];
   const int q = blockIdx.x;
   const int k = gp.k;
+  pdl_launch_dependents();
+  pdl_wait();   // the scan's candidate lists
   const int lists = q_valid[q] != 0 ? n_lists : 0;   // NaN/Inf query: no neighbours
   if (kk == 32) merge_lists<1>(partial, lists, nq, q, scratch, s_best);
   else if (kk == 64) merge_lists<2>(partial, lists, nq, q, scratch, s_best);
@@ -117,6 +127,8 @@ gather_only_kernel(PoolView pv, const int32_t* __restrict__ idx, const float* __
   __shared__ float s_score[OILBIRD_MAX_K];
   __shared__ int32_t s_len[OILBIRD_MAX_K];
   const int q = blockIdx.x, k = gp.k;
+  pdl_launch_dependents();
+  pdl_wait();
   for (int j = threadIdx.x; j < k; j += blockDim.x) {
     s_idx[j] = idx[(size_t)q * k + j];
     s_score[j] = score[(size_t)q * k + j];
@@ -129,16 +141,14 @@ cudaError_t launch_merge_gather(const PoolView& pv, const u64* partial, int32_t 
                                 int32_t nq, int32_t kk, const int32_t* q_valid,
                                 const GatherParams& gp, const oilbird_query_out& out,
                                 cudaStream_t st) {
-  merge_gather_kernel<<<nq, kMergeThreads, 0, st>>>(pv, partial, n_lists, nq, kk, q_valid, gp,
-                                                    out);
-  return cudaGetLastError();
+  return launch_pdl(merge_gather_kernel, dim3(nq), dim3(kMergeThreads), 0, st, pv, partial, n_lists,
+                    nq, kk, q_valid, gp, out);
 }
 
 cudaError_t launch_gather_only(const PoolView& pv, const int32_t* idx, const float* score,
                                int32_t nq, const GatherParams& gp, const oilbird_query_out& out,
                                cudaStream_t st) {
-  gather_only_kernel<<<nq, 128, 0, st>>>(pv, idx, score, gp, out);
-  return cudaGetLastError();
+  return launch_pdl(gather_only_kernel, dim3(nq), dim3(128), 0, st, pv, idx, score, gp, out);
 }
 
 }  // namespace oilbird

@@ -29,6 +29,8 @@ scan_gemv_kernel(PoolView pv, const uint16_t* __restrict__ q_raw, int nq, int k,
                  int32_t* __restrict__ q_valid, DeviceStats* stats) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   constexpr int KK = 32 * E;
+  pdl_launch_dependents();
+  pdl_wait();   // the rows appended just before this query, and the query states themselves
   const int d = pv.d, n_chunks = d >> 3;
   uint4* qs = reinterpret_cast<uint4*>(smem_raw);                       // [QT][n_chunks]
   u64* scratch = reinterpret_cast<u64*>(smem_raw + (size_t)QT * d * 2);  // [warps][KK]
@@ -152,9 +154,8 @@ static cudaError_t launch_one(const PoolView& pv, const uint16_t* q_raw, int nq,
   cudaError_t e = cudaFuncSetAttribute(scan_gemv_kernel<QT, E>,
                                        cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
-  scan_gemv_kernel<QT, E><<<grid, kScanThreads, smem, st>>>(pv, q_raw, nq, k, ex, partial,
-                                                            q_valid, stats);
-  return cudaGetLastError();
+  return launch_pdl(scan_gemv_kernel<QT, E>, dim3(grid), dim3(kScanThreads), smem, st, pv, q_raw,
+                    nq, k, ex, partial, q_valid, stats);
 }
 
 template <int QT>

@@ -206,6 +206,7 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap key_map,
   __shared__ TcShared sh;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int stage_bytes = kATileBytes + n_pad * kBlockK * 2;
+  pdl_launch_dependents();
   // dynamic shared memory: [stages][A tile | B tile] | lists | queue | per-query state
   unsigned char* base = (unsigned char*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
   unsigned char* ring = base;
@@ -227,11 +228,6 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap key_map,
     for (int j = 0; j < kColsPerRound; ++j) sh.q_cnt[j] = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  for (int i = threadIdx.x; i < n_pad; i += kTcThreads) {
-    thr_s[i] = -INFINITY;
-    s_ex[i] = (exclude_tag && i < nq_c) ? exclude_tag[q0 + i] : 0;
-  }
-  for (int i = threadIdx.x; i < nq_c * kk; i += kTcThreads) lists[i] = 0;
   if (warp == 1) {   // TMEM allocation is a whole-warp operation
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
                  ::"r"(smem_u32(&sh.tmem_base)), "r"((uint32_t)tmem_cols) : "memory");
@@ -241,6 +237,13 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap key_map,
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = sh.tmem_base;
+  pdl_wait();   // appended rows, normalised queries, exclusion tags; set-up above overlapped
+  for (int i = threadIdx.x; i < n_pad; i += kTcThreads) {
+    thr_s[i] = -INFINITY;
+    s_ex[i] = (exclude_tag && i < nq_c) ? exclude_tag[q0 + i] : 0;
+  }
+  for (int i = threadIdx.x; i < nq_c * kk; i += kTcThreads) lists[i] = 0;
+  __syncthreads();
 
   if (warp == 0) {
     // ===================================================== TMA producer ==========
@@ -456,11 +459,9 @@ cudaError_t launch_scan_tc(const void* key_map, const void* q_map, const PoolVie
   cudaError_t e = cudaFuncSetAttribute(scan_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        (int)smem);
   if (e != cudaSuccess) return e;
-  scan_tc_kernel<<<grid, kTcThreads, smem, st>>>(*(const CUtensorMap*)key_map,
-                                                 *(const CUtensorMap*)q_map, pv, q0, nq_c,
-                                                 nq_total, n_pad, k, kk, stages, tmem_cols,
-                                                 exclude_tag, partial, stats);
-  return cudaGetLastError();
+  return launch_pdl(scan_tc_kernel, dim3(grid), dim3(kTcThreads), smem, st,
+                    *(const CUtensorMap*)key_map, *(const CUtensorMap*)q_map, pv, q0, nq_c, nq_total,
+                    n_pad, k, kk, stages, tmem_cols, exclude_tag, partial, stats);
 }
 
 }  // namespace oilbird

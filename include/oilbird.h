@@ -209,6 +209,41 @@ int32_t oilbird_pool_profile_read(oilbird_pool_t* pool, float* scan_ms, int32_t 
 /* Number of kernels this library has launched for this pool since create(). */
 int64_t oilbird_pool_launch_count(const oilbird_pool_t* pool);
 
+/*
+ * Query without any allocation (the paper has no counterpart; this serves hosts of the
+ * library that own all device memory themselves and must not let a library allocate:
+ * for instance a serving engine that reserved the whole of HBM at start-up, where a
+ * later driver allocation can fail or stall).  The caller keeps the pool's arrays in
+ * its own memory, in the layout oilbird_pool_append produces (keys L2-normalised bf16),
+ * and passes them in; results go to caller memory as in oilbird_pool_query.  The
+ * candidate lists exchanged between the scan and the merge kernel live in a fixed
+ * 1 MiB array inside the library image (reserved on every GPU that loads the library,
+ * until the process exits), which bounds the call: nq <= OILBIRD_STATIC_MAX_NQ,
+ * k <= OILBIRD_MAX_K, no exclusion tags, CUDA-core scan only (params->path AUTO or
+ * GEMV).  Anything larger is rejected with OILBIRD_EINVAL and a message in
+ * oilbird_query_static_error().
+ * The call enqueues work on cuda_stream and returns; it calls no cudaMalloc / cudaFree.
+ * The first call on a device also looks up the array's device address; make that first
+ * call before any stream capture begins.  All calls on a device share the array, which
+ * keeps the previous call's contents; each call rewrites what it reads and clears its
+ * counters first, but two calls that overlap on the GPU (other streams, other threads)
+ * race.  One host thread at a time.
+ */
+#define OILBIRD_STATIC_MAX_NQ 2
+typedef struct {
+  const void*    keys;       /* dev [n_rows,d] bf16, L2-normalised, row-major             */
+  const int32_t* tokens;     /* dev [n_rows]                                              */
+  const int32_t* trace_id;   /* dev [n_rows]  trace holding each row                      */
+  const int32_t* trace_end;  /* dev [n_traces] one past the last row of each trace        */
+  int64_t        n_rows;
+  int32_t        d;          /* multiple of 8, 8..16384                                   */
+  int32_t        device;     /* CUDA ordinal the arrays live on                           */
+} oilbird_static_pool;
+int oilbird_query_static(const oilbird_static_pool* pool, const void* q_bf16 /* dev [nq,d] */,
+                         int32_t nq, const oilbird_query_params* params,
+                         const oilbird_query_out* out, void* cuda_stream);
+const char* oilbird_query_static_error(void);   /* why the last call was rejected        */
+
 const char* oilbird_strerror(int code);
 const char* oilbird_last_cuda_error(void);    /* text of the last failing CUDA call      */
 

@@ -45,6 +45,12 @@ class CQueryOut(ctypes.Structure):
                 ("cont_len", ctypes.c_void_p), ("cont_tok", ctypes.c_void_p)]
 
 
+class StaticPool(ctypes.Structure):
+    _fields_ = [("keys", ctypes.c_void_p), ("tokens", ctypes.c_void_p),
+                ("trace_id", ctypes.c_void_p), ("trace_end", ctypes.c_void_p),
+                ("n_rows", ctypes.c_int64), ("d", ctypes.c_int32), ("device", ctypes.c_int32)]
+
+
 class PoolStats(ctypes.Structure):
     _fields_ = [("degenerate_rows", ctypes.c_int64), ("nonfinite_queries", ctypes.c_int64),
                 ("stalled", ctypes.c_int32), ("reserved", ctypes.c_int32)]
@@ -75,6 +81,10 @@ SYMBOLS = {
     "oilbird_pool_profile": (ctypes.c_int, [_vp, _i32]),
     "oilbird_pool_profile_read": (_i32, [_vp, _vp, _i32]),
     "oilbird_pool_launch_count": (_i64, [_vp]),
+    "oilbird_query_static": (ctypes.c_int, [ctypes.POINTER(StaticPool), _vp, _i32,
+                                            ctypes.POINTER(CQueryParams),
+                                            ctypes.POINTER(CQueryOut), _vp]),
+    "oilbird_query_static_error": (ctypes.c_char_p, []),
     "oilbird_strerror": (ctypes.c_char_p, [ctypes.c_int]),
     "oilbird_last_cuda_error": (ctypes.c_char_p, []),
 }
@@ -164,6 +174,40 @@ class QueryOut:
     def cpu(self) -> "QueryOut":
         return QueryOut(self.idx.cpu(), self.score.cpu(), self.fired.cpu(), self.cont_len.cpu(),
                         self.cont_tok.cpu())
+
+
+def query_static(keys: torch.Tensor, tokens: torch.Tensor, trace_id: torch.Tensor,
+                 trace_end: torch.Tensor, q: torch.Tensor, params: QueryParams,
+                 out: QueryOut | None = None, stream=None) -> QueryOut:
+    """oilbird_query_static: query caller-held pool arrays without any allocation.
+
+    For hosts that own all device memory themselves and cannot let the library allocate;
+    the library's only scratch is a fixed 1 MiB array in its image, so nq <= 2, k <= 128,
+    no exclusion tags.  keys: CUDA bf16 [n,d], already L2-normalised (as append stores
+    them); tokens / trace_id: CUDA int32 [n]; trace_end: CUDA int32 [n_traces].  Pass
+    `out` to keep this wrapper itself from allocating result tensors.
+    """
+    for t, dt in ((keys, torch.bfloat16), (tokens, torch.int32), (trace_id, torch.int32),
+                  (trace_end, torch.int32), (q, torch.bfloat16)):
+        assert t.is_cuda and t.dtype == dt and t.is_contiguous()
+    n, d = keys.shape
+    q = q.reshape(-1, d)
+    nq = q.shape[0]
+    if out is None:
+        out = QueryOut.empty(nq, params.k, params.cont_len, keys.device)
+    sp = StaticPool(keys.data_ptr(), tokens.data_ptr(), trace_id.data_ptr(), trace_end.data_ptr(),
+                    n, d, keys.device.index or 0)
+    cp = params.to_c(None)
+    if params.exclude_tag is not None:
+        cp.exclude_tag = params.exclude_tag.data_ptr()
+    L = lib()
+    rc = L.oilbird_query_static(ctypes.byref(sp), q.data_ptr(), nq, ctypes.byref(cp),
+                                ctypes.byref(out._c), _stream_ptr(stream))
+    if rc != OK:
+        err = OilbirdError(rc, "oilbird_query_static")
+        err.args = (err.args[0] + ": " + L.oilbird_query_static_error().decode(),)
+        raise err
+    return out
 
 
 def _stream_ptr(stream) -> int:

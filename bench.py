@@ -129,6 +129,23 @@ class ClockSampler:
                 "samples": len(self.samples)}
 
 
+def aggregate(local_ms: float, local_units: float, world: int, device) -> tuple[float, float]:
+    """Whole-job time and throughput: the slowest rank's time, the units of all ranks.
+
+    Every rank serves its own pool, so the job's units are the sum over ranks and its
+    time is the maximum (device-timed) over ranks.  Works on any torch.distributed
+    backend (NCCL on GPUs; gloo in the CPU tests).
+    """
+    import torch.distributed as dist
+    t = torch.tensor([local_ms], dtype=torch.float64, device=device)
+    u = torch.tensor([local_units], dtype=torch.float64, device=device)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        dist.all_reduce(u, op=dist.ReduceOp.SUM)
+    max_ms = float(t.item())
+    return max_ms, float(u.item()) / (max_ms / 1e3)
+
+
 # ------------------------------------------------------------------ workload ----
 
 def physical_device(local_rank: int) -> int:
@@ -229,11 +246,7 @@ def run_ours(args):
     total_ms = ev[0].elapsed_time(ev[K])
     lat = np.array([ev[s].elapsed_time(ev[s + 1]) for s in range(K)])
     rows_mean = rows0 + rows_step * (K + 1) / 2.0
-    t = torch.tensor([total_ms], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    max_ms = float(t.item())
-    value = world * K * nq / (max_ms / 1e3)
+    max_ms, value = aggregate(total_ms, K * nq, world, dev)
 
     # ---- the dominant kernel (key scan), timed by events around its launches ---------
     pool.profile(True)
@@ -274,10 +287,7 @@ def run_ours(args):
         step_host()
     e1.record()
     barrier()
-    t2 = torch.tensor([e0.elapsed_time(e1)], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(t2, op=dist.ReduceOp.MAX)
-    e2e_value = world * K * nq / (float(t2.item()) / 1e3)
+    _, e2e_value = aggregate(e0.elapsed_time(e1), K * nq, world, dev)
     h2d = rows_step * w.d * 2 + rows_step * 4 + nq * w.d * 2
     d2h = nq * w.k * (4 + 4 + 4 + 4 * w.cont_len) + nq * 4
     stalled = pool.stats()["stalled"]
@@ -313,6 +323,18 @@ def run_ours(args):
                          else None},
             "device_stalled_flag": stalled,
         }
+        n_pad = (nq + 15) // 16 * 16
+        used_tensor = args.path == 2 or (args.path == 0 and nq > 2)
+        if used_tensor:
+            # the batched path is a dense contraction: report its tensor-pipe share too
+            # (2*N*d*n_pad flops per launch, queries padded to the MMA's N)
+            tflops = 2.0 * rows_scan * w.d * n_pad / (scan_mean_ms * 1e-3) / 1e12
+            line["tensor_pipe"] = {
+                "achieved": tflops, "unit": "TFLOP/s", "n_pad": n_pad,
+                "peak_sustained": peaks["bf16_tflops_sustained"], "peak_burst": peaks["bf16_tflops"],
+                "frac_of_sustained": tflops / peaks["bf16_tflops_sustained"],
+                "frac_of_burst": tflops / peaks["bf16_tflops"], "peak_kind": peak_kind,
+                "note": "HBM-bound below nq ~ 218: the tensor pipe idles by design"}
         if not args.no_cpu_baseline and world == 1:
             line["cpu_baseline"] = cpu_baseline(w, n0, rows_step, nq, budget_s=args.cpu_budget)
         print(json.dumps(line), flush=True)

@@ -74,7 +74,7 @@ def ncu_traffic(config_name: str, rows: float):
 class ClockSampler:
     """Samples SM clock and throttle reasons through NVML while the timed region runs."""
 
-    def __init__(self, index: int, period_s: float = 0.02):
+    def __init__(self, index: int, period_s: float = 0.005):
         self.index, self.period = index, period_s
         self.samples, self.reasons = [], set()
         self.max_mhz = None
@@ -443,7 +443,7 @@ def main():
         args.warmup = 1 if args.warmup is None else args.warmup
         run_reference(args)
         return
-    default_steps = {"C1": 2000, "C2": 2000, "C3": 500, "C4": 200, "C5": 50}[args.config]
+    default_steps = {"C1": 500, "C2": 500, "C3": 300, "C4": 100, "C5": 50}[args.config]
     args.steps = default_steps if args.steps is None else args.steps
     args.warmup = 10 if args.warmup is None else max(args.warmup, 3)
     run_ours(args)

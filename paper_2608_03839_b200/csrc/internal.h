@@ -83,7 +83,7 @@ cudaError_t launch_scan_gemv(const PoolView& pv, const uint16_t* q_raw, int32_t 
 // normalised queries already sit in qn (row-major [>= q0+round16(nq_c), d]).  key_map and
 // q_map are CUtensorMap objects made by make_bf16_map (box rows 128 and round16(nq_c)).
 bool make_bf16_map(void* map_out, const void* base, int64_t rows, int32_t d, int32_t box_rows);
-int tc_max_queries_per_pass(int k, size_t smem_limit);
+int tc_queries_per_pass(int nq, int k, size_t smem_limit);   // balanced split of a call
 cudaError_t launch_scan_tc(const void* key_map, const void* q_map, const PoolView& pv, int32_t q0,
                            int32_t nq_c, int32_t nq_total, int32_t k, int32_t kk,
                            const uint64_t* exclude_tag, unsigned long long* partial,

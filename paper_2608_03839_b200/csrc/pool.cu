@@ -347,9 +347,7 @@ int oilbird_pool_query(oilbird_pool_t* p, const void* q, int32_t nq,
       if (e != cudaSuccess) return cuda_fail(e, "qnorm kernel launch");
       p->launches += 1;
       // as many queries per pass as shared memory allows next to a 3-stage ring
-      const int max_pass = tc_max_queries_per_pass(pr->k, p->smem_limit);
-      const int n_pass = (nq + max_pass - 1) / max_pass;
-      const int per_pass = ((nq + n_pass - 1) / n_pass + 15) / 16 * 16;   // balanced passes
+      const int per_pass = tc_queries_per_pass(nq, pr->k, p->smem_limit);
       for (int q0 = 0; q0 < nq; q0 += per_pass) {
         const int nq_c = nq - q0 < per_pass ? nq - q0 : per_pass;
         const int slot = (nq_c + 15) / 16 - 1;

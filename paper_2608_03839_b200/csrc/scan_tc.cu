@@ -18,6 +18,7 @@
 // Every mbarrier wait is bounded: after about two seconds it raises the pool's `stalled`
 // flag, the CTA drains what it has in flight, frees its TMEM and returns.
 #include <cuda.h>
+#include <stdlib.h>
 
 #include "common.cuh"
 #include "internal.h"
@@ -196,18 +197,23 @@ __device__ __forceinline__ void drain_query(u64* list, const u64* cand, int n_ca
 
 // ------------------------------------------------------------------- the kernel ---
 // Queries [q0, q0+nq_c) of the call; n_pad = nq_c rounded up to 16 = MMA N.
+// mt (1 or 2) key tiles of 128 rows share each query tile: with mt = 2 the query bytes
+// pulled from L2 per key byte halve, which is what limits the kernel from nq ~ 64 up.
+// n_bufs accumulator sets of mt*n_pad TMEM columns each (2 = the next macro tile's MMAs
+// overlap the epilogue; 1 when 2*mt*n_pad would exceed the 512 columns).
 __global__ void __launch_bounds__(kTcThreads, 1)
 scan_tc_kernel(const __grid_constant__ CUtensorMap key_map,
                const __grid_constant__ CUtensorMap q_map, PoolView pv, int q0, int nq_c,
-               int nq_total, int n_pad, int k, int kk, int n_stages, int tmem_cols,
-               const uint64_t* __restrict__ exclude_tag, u64* __restrict__ partial,
+               int nq_total, int n_pad, int k, int kk, int n_stages, int tmem_cols, int mt,
+               int n_bufs, const uint64_t* __restrict__ exclude_tag, u64* __restrict__ partial,
                DeviceStats* stats) {
   extern __shared__ __align__(1024) unsigned char smem_raw[];
   __shared__ TcShared sh;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int stage_bytes = kATileBytes + n_pad * kBlockK * 2;
+  const int a_bytes = mt * kATileBytes;
+  const int stage_bytes = a_bytes + n_pad * kBlockK * 2;
   pdl_launch_dependents();
-  // dynamic shared memory: [stages][A tile | B tile] | lists | queue | per-query state
+  // dynamic shared memory: [stages][mt key tiles | query tile] | lists | queue | state
   unsigned char* base = (unsigned char*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
   unsigned char* ring = base;
   u64* lists = reinterpret_cast<u64*>(ring + (size_t)n_stages * stage_bytes);   // [nq_c][kk]
@@ -215,7 +221,7 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap key_map,
   uint64_t* s_ex = reinterpret_cast<uint64_t*>(q_key + kQueueCap);              // [n_pad]
   float* thr_s = reinterpret_cast<float*>(s_ex + n_pad);                        // [n_pad]
 
-  const int n_tiles = (pv.n_rows + kTileM - 1) / kTileM;
+  const int n_tiles = (pv.n_rows + mt * kTileM - 1) / (mt * kTileM);   // macro tiles
   const int n_kb = (pv.d + kBlockK - 1) / kBlockK;
   volatile int* abort_flag = &sh.abort_flag;
 
@@ -259,8 +265,10 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap key_map,
           if (!mbar_wait(&sh.empty[s], ph ^ 1u, abort_flag, stats)) { ok = false; break; }
           unsigned char* a_dst = ring + (size_t)s * stage_bytes;
           mbar_arrive_expect_tx(&sh.full[s], (uint32_t)stage_bytes);
-          tma_load_2d(a_dst, &key_map, kb * kBlockK, tile * kTileM, &sh.full[s]);
-          tma_load_2d(a_dst + kATileBytes, &q_map, kb * kBlockK, q0, &sh.full[s]);
+          for (int sub = 0; sub < mt; ++sub)    // rows past the pool's capacity read as zero
+            tma_load_2d(a_dst + sub * kATileBytes, &key_map, kb * kBlockK,
+                        (tile * mt + sub) * kTileM, &sh.full[s]);
+          tma_load_2d(a_dst + a_bytes, &q_map, kb * kBlockK, q0, &sh.full[s]);
         }
       }
       if (!ok) {
@@ -281,24 +289,27 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap key_map,
       uint32_t it = 0, iter = 0;
       bool ok = true;
       for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x, ++iter) {
-        const uint32_t buf = iter & 1u;
-        if (!mbar_wait(&sh.tmem_empty[buf], ((iter >> 1) & 1u) ^ 1u, abort_flag, stats)) {
+        const uint32_t buf = iter % (uint32_t)n_bufs;
+        if (!mbar_wait(&sh.tmem_empty[buf], ((iter / (uint32_t)n_bufs) & 1u) ^ 1u, abort_flag,
+                       stats)) {
           ok = false;
           break;
         }
         tc_fence_after();
-        const uint32_t d_tmem = tmem_base + buf * (uint32_t)n_pad;
+        const uint32_t d_tmem = tmem_base + buf * (uint32_t)(mt * n_pad);
         for (int kb = 0; kb < n_kb; ++kb, ++it) {
           const int s = it % n_stages;
           if (!mbar_wait(&sh.full[s], (it / n_stages) & 1u, abort_flag, stats)) { ok = false; break; }
           tc_fence_after();
           const uint32_t a_addr = smem_u32(ring + (size_t)s * stage_bytes);
-          const uint64_t a_desc = umma_desc_sw128(a_addr);
-          const uint64_t b_desc = umma_desc_sw128(a_addr + kATileBytes);
+          const uint64_t b_desc = umma_desc_sw128(a_addr + a_bytes);
+          for (int sub = 0; sub < mt; ++sub) {
+            const uint64_t a_desc = umma_desc_sw128(a_addr + sub * kATileBytes);
 #pragma unroll
-          for (int kq = 0; kq < kBlockK / 16; ++kq)        // 32 bytes along K per MMA
-            tc_mma_bf16(d_tmem, a_desc + (uint64_t)(kq * 2), b_desc + (uint64_t)(kq * 2), idesc,
-                        (kb | kq) != 0 ? 1u : 0u);
+            for (int kq = 0; kq < kBlockK / 16; ++kq)      // 32 bytes along K per MMA
+              tc_mma_bf16(d_tmem + (uint32_t)(sub * n_pad), a_desc + (uint64_t)(kq * 2),
+                          b_desc + (uint64_t)(kq * 2), idesc, (kb | kq) != 0 ? 1u : 0u);
+          }
           tc_commit(&sh.empty[s]);                          // stage reusable once the MMAs retire
         }
         if (ok) tc_commit(&sh.tmem_full[buf]);
@@ -316,24 +327,26 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap key_map,
     uint32_t iter = 0;
     bool ok = true;
     for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x, ++iter) {
-      const uint32_t buf = iter & 1u;
-      mbar_wait(&sh.tmem_full[buf], (iter >> 1) & 1u, abort_flag, stats);
+      const uint32_t buf = iter % (uint32_t)n_bufs;
+      mbar_wait(&sh.tmem_full[buf], (iter / (uint32_t)n_bufs) & 1u, abort_flag, stats);
       // one decision for all four warps, so that the barriers below always match up
       epilogue_bar();
       if (et == 0) sh.epi_go = *abort_flag ? 0 : 1;
       epilogue_bar();
       if (!sh.epi_go) { ok = false; break; }
       tc_fence_after();
-      const int row = tile * kTileM + lane_grp * 32 + lane;
+      for (int sub = 0; sub < mt; ++sub) {      // sub-tiles in row order: ties stay exact
+      const int row = (tile * mt + sub) * kTileM + lane_grp * 32 + lane;
       const bool row_ok = row < pv.n_rows;
       uint64_t tag = 0;
       if (exclude_tag && row_ok) tag = pv.trace_tag[pv.trace_id[row]];
-      const uint32_t t_row = tmem_base + ((uint32_t)(lane_grp * 32) << 16) + buf * (uint32_t)n_pad;
+      const uint32_t t_row = tmem_base + ((uint32_t)(lane_grp * 32) << 16) +
+                             (buf * (uint32_t)mt + (uint32_t)sub) * (uint32_t)n_pad;
       for (int c0 = 0; c0 < n_pad; c0 += kColsPerRound) {
         float v[16];
         tc_ld16(t_row + (uint32_t)c0, v);
-        if (c0 + kColsPerRound >= n_pad) {
-          // all of this tile's scores are in registers: hand the accumulator back
+        if (sub == mt - 1 && c0 + kColsPerRound >= n_pad) {
+          // all of this macro tile's scores have been read: hand the accumulators back
           tc_fence_before();
           __syncwarp();
           if (lane == 0) mbar_arrive(&sh.tmem_empty[buf]);
@@ -368,6 +381,7 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap key_map,
           if (et == 0) sh.q_total = 0;
           epilogue_bar();
         }
+      }
       }
     }
     // publish this CTA's per-query lists: already descending, empty slots are 0
@@ -424,16 +438,43 @@ static size_t tc_fixed_smem(int nq_c, int n_pad, int kk) {
          1024 /* alignment slack */;
 }
 
-// Largest number of queries one launch can take for this k so that at least three ring
-// stages fit next to the per-query lists.
-int tc_max_queries_per_pass(int k, size_t smem_limit) {
+// How a call is cut up: queries per pass, key tiles per query tile, ring stages,
+// accumulator buffers.  Fewest passes first (every pass re-reads the keys); then two key
+// tiles per query tile if at least three ring stages still fit, else one.
+struct TcPlan { int per_pass, mt, stages, n_bufs; };
+
+static bool tc_fits(int n, int kk, int mt, int min_stages, size_t smem_limit, int* stages) {
+  const size_t stage = (size_t)mt * kATileBytes + (size_t)n * kBlockK * 2;
+  // static shared memory (barriers etc.) is padded to the 1024-byte alignment of the ring
+  const size_t fixed = tc_fixed_smem(n, n, kk) + 1024 + 256;
+  if (fixed + (size_t)min_stages * stage > smem_limit) return false;
+  int st = (int)((smem_limit - fixed) / stage);
+  *stages = st > kMaxStages ? kMaxStages : st;
+  return true;
+}
+
+static TcPlan tc_plan(int nq, int k, int n_tiles128, int num_sms, size_t smem_limit, int force_mt) {
   const int kk = list_len(k);
-  int best = 16;
-  for (int n = 16; n <= OILBIRD_MAX_NQ; n += 16) {
-    size_t stage = (size_t)kATileBytes + (size_t)n * kBlockK * 2;
-    if (tc_fixed_smem(n, n, kk) + 3 * stage + sizeof(TcShared) + 256 <= smem_limit) best = n;
-  }
-  return best;
+  int max_pass = 16, st = 0;
+  for (int n = 16; n <= OILBIRD_MAX_NQ; n += 16)
+    if (tc_fits(n, kk, 1, 3, smem_limit, &st)) max_pass = n;
+  const int n_pass = (nq + max_pass - 1) / max_pass;
+  TcPlan p;
+  p.per_pass = ((nq + n_pass - 1) / n_pass + 15) / 16 * 16;      // balanced passes
+  const int n_pad = p.per_pass < nq ? p.per_pass : (nq + 15) / 16 * 16;
+  // sharing a query tile between two key tiles pays at every nq measured (fewer, larger
+  // stages and half the query bytes from L2), given enough tiles to keep every SM busy
+  bool two = n_tiles128 >= 4 * num_sms && tc_fits(n_pad, kk, 2, 3, smem_limit, &st);
+  if (force_mt == 1) two = false;
+  if (force_mt == 2) two = tc_fits(n_pad, kk, 2, 2, smem_limit, &st);
+  p.mt = two ? 2 : 1;
+  tc_fits(n_pad, kk, p.mt, 2, smem_limit, &p.stages);
+  p.n_bufs = 2 * p.mt * n_pad <= 512 ? 2 : 1;
+  return p;
+}
+
+int tc_queries_per_pass(int nq, int k, size_t smem_limit) {
+  return tc_plan(nq, k, 0, 1, smem_limit, 1).per_pass;
 }
 
 cudaError_t launch_scan_tc(const void* key_map, const void* q_map, const PoolView& pv, int32_t q0,
@@ -442,17 +483,17 @@ cudaError_t launch_scan_tc(const void* key_map, const void* q_map, const PoolVie
                            DeviceStats* stats, int32_t num_sms, size_t smem_limit,
                            int32_t* n_lists, cudaStream_t st) {
   const int n_pad = (nq_c + 15) / 16 * 16;
-  const size_t stage = (size_t)kATileBytes + (size_t)n_pad * kBlockK * 2;
+  const int n_tiles128 = (pv.n_rows + kTileM - 1) / kTileM;
+  static const int force_mt = getenv("OILBIRD_TC_MT") ? atoi(getenv("OILBIRD_TC_MT")) : 0;
+  TcPlan plan = tc_plan(nq_c, k, n_tiles128, num_sms, smem_limit, force_mt);
+  const size_t stage = (size_t)plan.mt * kATileBytes + (size_t)n_pad * kBlockK * 2;
   const size_t fixed = tc_fixed_smem(nq_c, n_pad, kk);
-  const size_t avail = smem_limit - sizeof(TcShared) - 256;
-  if (fixed + 2 * stage > avail) return cudaErrorInvalidConfiguration;
-  int stages = (int)((avail - fixed) / stage);
-  if (stages > kMaxStages) stages = kMaxStages;
-  size_t smem = fixed + (size_t)stages * stage;
+  if (plan.stages < 2) return cudaErrorInvalidConfiguration;
+  size_t smem = fixed + (size_t)plan.stages * stage;
   if (smem < 120 * 1024) smem = 120 * 1024;   // one CTA per SM: TMEM is allocated per CTA
   int tmem_cols = 32;
-  while (tmem_cols < 2 * n_pad) tmem_cols <<= 1;
-  const int n_tiles = (pv.n_rows + kTileM - 1) / kTileM;
+  while (tmem_cols < plan.n_bufs * plan.mt * n_pad) tmem_cols <<= 1;
+  const int n_tiles = (n_tiles128 + plan.mt - 1) / plan.mt;
   int grid = n_tiles < num_sms ? n_tiles : num_sms;
   if (grid < 1) grid = 1;
   *n_lists = grid;
@@ -461,7 +502,8 @@ cudaError_t launch_scan_tc(const void* key_map, const void* q_map, const PoolVie
   if (e != cudaSuccess) return e;
   return launch_pdl(scan_tc_kernel, dim3(grid), dim3(kTcThreads), smem, st,
                     *(const CUtensorMap*)key_map, *(const CUtensorMap*)q_map, pv, q0, nq_c, nq_total,
-                    n_pad, k, kk, stages, tmem_cols, exclude_tag, partial, stats);
+                    n_pad, k, kk, plan.stages, tmem_cols, plan.mt, plan.n_bufs, exclude_tag, partial,
+                    stats);
 }
 
 }  // namespace oilbird

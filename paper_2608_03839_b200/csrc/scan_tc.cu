@@ -29,7 +29,7 @@ constexpr int kTcThreads = 192;
 constexpr int kTileM = 128;            // key rows per tile = TMEM lanes
 constexpr int kBlockK = 64;            // bf16 elements per k-block = one 128-byte swizzle row
 constexpr int kATileBytes = kTileM * kBlockK * 2;   // 16 KB
-constexpr int kColsPerRound = 16;      // score columns filtered between two drains
+constexpr int kColsPerRound = 8;       // score columns filtered between two drains
 constexpr int kQueueCap = kTileM * kColsPerRound;
 constexpr int kMaxStages = 8;
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;
@@ -111,18 +111,16 @@ __device__ __forceinline__ void tc_mma_bf16(uint32_t d_tmem, uint64_t a_desc, ui
       ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
       : "memory");
 }
-__device__ __forceinline__ void tc_ld16(uint32_t taddr, float (&v)[16]) {
-  uint32_t r[16];
+__device__ __forceinline__ void tc_ld8(uint32_t taddr, float (&v)[8]) {
+  uint32_t r[8];
   asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x16.b32"
-      " {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+      "tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
       : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]),
-        "=r"(r[7]), "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]),
-        "=r"(r[14]), "=r"(r[15])
+        "=r"(r[7])
       : "r"(taddr));
   asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 #pragma unroll
-  for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
+  for (int i = 0; i < 8; ++i) v[i] = __uint_as_float(r[i]);
 }
 __device__ __forceinline__ void epilogue_bar() {      // the 128 epilogue threads only
   asm volatile("bar.sync 1, 128;" ::: "memory");
@@ -343,8 +341,8 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap key_map,
       const uint32_t t_row = tmem_base + ((uint32_t)(lane_grp * 32) << 16) +
                              (buf * (uint32_t)mt + (uint32_t)sub) * (uint32_t)n_pad;
       for (int c0 = 0; c0 < n_pad; c0 += kColsPerRound) {
-        float v[16];
-        tc_ld16(t_row + (uint32_t)c0, v);
+        float v[kColsPerRound];
+        tc_ld8(t_row + (uint32_t)c0, v);
         if (sub == mt - 1 && c0 + kColsPerRound >= n_pad) {
           // all of this macro tile's scores have been read: hand the accumulators back
           tc_fence_before();
@@ -353,7 +351,7 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap key_map,
         }
         if (row_ok) {
 #pragma unroll
-          for (int j = 0; j < 16; ++j) {
+          for (int j = 0; j < kColsPerRound; ++j) {
             const int q = c0 + j;
             if (q < nq_c && v[j] > thr_s[q]) {
               if (s_ex[q] != 0 && tag == s_ex[q]) continue;       // same-prompt trace: skipped

@@ -90,6 +90,24 @@ def lib() -> ctypes.CDLL:
     L.oracle_pool_query.restype = ctypes.c_int
     L.oracle_pool_query.argtypes = [vp, vp, i32, i32, f32, i32, i32, i32, i32, vp, vp, vp,
                                     vp, vp, vp, vp, vp, vp]
+    L.oracle_ring_create.restype = vp
+    L.oracle_ring_create.argtypes = [i32, i64, i32]
+    L.oracle_ring_destroy.restype = None
+    L.oracle_ring_destroy.argtypes = [vp]
+    L.oracle_ring_reset.restype = None
+    L.oracle_ring_reset.argtypes = [vp]
+    L.oracle_ring_size.restype = i64
+    L.oracle_ring_size.argtypes = [vp]
+    L.oracle_ring_total.restype = i64
+    L.oracle_ring_total.argtypes = [vp]
+    for name in ("keys", "anchors", "rollouts"):
+        fn = getattr(L, "oracle_ring_" + name)
+        fn.restype = vp
+        fn.argtypes = [vp]
+    L.oracle_ring_append.restype = None
+    L.oracle_ring_append.argtypes = [vp, vp, vp, vp, i64]
+    L.oracle_ring_query.restype = ctypes.c_int
+    L.oracle_ring_query.argtypes = [vp, vp, vp, i32, i32, f32, vp, vp, vp, vp, vp]
     L.oracle_num_threads.restype = i32
     L.oracle_num_threads.argtypes = []
     _lib = L
@@ -270,3 +288,86 @@ def depth(s: float, tier_thr=PAPER_TIER_THR, tier_depth=PAPER_TIER_DEPTH) -> int
     thr = np.asarray(tier_thr, dtype=np.float32)
     dep = np.asarray(tier_depth, dtype=np.int32)
     return int(lib().oracle_depth(float(s), int(thr.size), _ptr(thr), _ptr(dep)))
+
+
+# ------------------------------------------------------------------ recycled pool ----
+PAPER_RING_M = 4          # Algorithm 1: at most 4 rejected-branch rollouts
+PAPER_RING_FLOOR = 0.8    # ... whose cosine reaches 0.8
+PAPER_ROLLOUT = 6         # Section 4 (i b): continuations up to six deep
+
+
+@dataclass
+class RingResult:
+    slot: np.ndarray         # [nq,m] int64, -1 padded
+    score: np.ndarray        # [nq,m] float32, -inf padded
+    count: np.ndarray        # [nq] int32
+    rollout: np.ndarray      # [nq,m,R] int32, -1 padded
+    rollout_len: np.ndarray  # [nq,m] int32
+
+
+class OracleRing:
+    """Rejected-branch ring buffer (Section 4 (i b); Algorithm 1's recycled-pool line)."""
+
+    def __init__(self, d: int, capacity: int, max_rollout: int = PAPER_ROLLOUT):
+        self._L = lib()
+        self.d, self.capacity, self.max_rollout = int(d), int(capacity), int(max_rollout)
+        self._h = self._L.oracle_ring_create(self.d, self.capacity, self.max_rollout)
+        if not self._h:
+            raise MemoryError("oracle_ring_create failed")
+
+    def __del__(self):
+        h, self._h = getattr(self, "_h", None), None
+        if h:
+            self._L.oracle_ring_destroy(h)
+
+    def __len__(self) -> int:
+        return int(self._L.oracle_ring_size(self._h))
+
+    @property
+    def total(self) -> int:
+        return int(self._L.oracle_ring_total(self._h))
+
+    def reset(self) -> None:
+        self._L.oracle_ring_reset(self._h)
+
+    def append(self, states, anchors, rollouts) -> None:
+        states = _u16(states).reshape(-1, self.d)
+        anchors = np.ascontiguousarray(anchors, dtype=np.int32).reshape(-1)
+        rollouts = np.ascontiguousarray(rollouts, dtype=np.int32).reshape(-1, self.max_rollout)
+        assert states.shape[0] == anchors.shape[0] == rollouts.shape[0]
+        self._L.oracle_ring_append(self._h, _ptr(states), _ptr(anchors), _ptr(rollouts),
+                                   states.shape[0])
+
+    def _copy(self, name, count, dtype):
+        p = getattr(self._L, "oracle_ring_" + name)(self._h)
+        buf = (ctypes.c_char * (count * np.dtype(dtype).itemsize)).from_address(p)
+        return np.frombuffer(buf, dtype=dtype, count=count).copy()
+
+    @property
+    def keys(self) -> np.ndarray:
+        return self._copy("keys", self.capacity * self.d, np.uint16).reshape(self.capacity, self.d)
+
+    @property
+    def anchors(self) -> np.ndarray:
+        return self._copy("anchors", self.capacity, np.int32)
+
+    @property
+    def rollouts(self) -> np.ndarray:
+        return self._copy("rollouts", self.capacity * self.max_rollout, np.int32).reshape(
+            self.capacity, self.max_rollout)
+
+    def query(self, q, anchors, m: int = PAPER_RING_M, floor: float = PAPER_RING_FLOOR
+              ) -> RingResult:
+        q = _u16(q).reshape(-1, self.d)
+        nq = q.shape[0]
+        anchors = np.ascontiguousarray(anchors, dtype=np.int32).reshape(nq)
+        slot = np.empty((nq, m), np.int64)
+        score = np.empty((nq, m), np.float32)
+        count = np.empty(nq, np.int32)
+        roll = np.empty((nq, m, self.max_rollout), np.int32)
+        rlen = np.empty((nq, m), np.int32)
+        rc = self._L.oracle_ring_query(self._h, _ptr(q), _ptr(anchors), nq, int(m), float(floor),
+                                       _ptr(slot), _ptr(score), _ptr(count), _ptr(roll), _ptr(rlen))
+        if rc != 0:
+            raise MemoryError("oracle_ring_query failed")
+        return RingResult(slot, score, count, roll, rlen)

@@ -325,3 +325,114 @@ int32_t oracle_num_threads(void) {
   return 1;
 #endif
 }
+
+/* ============================================================ recycled pool == */
+/*
+ * Rejected-branch store (paper Section 4 "(i b) Recycling"; Algorithm 1's
+ * recycled-pool line).  A record is keyed by the hidden state in front of a
+ * rejected draft token together with that token (the "anchor"), and its value
+ * is the short continuation the model endorsed from there (up to six tokens in
+ * the paper).  Records live in a ring buffer: once it is full the oldest record
+ * is overwritten.  A lookup with the current state and the current anchor token
+ * returns at most m records whose anchor token is equal and whose cosine with the
+ * query reaches a floor (paper: at most 4, floor 0.8), best first; equal scores
+ * list the lower slot first.  Unlike theta of the trace store, the floor here is
+ * a filter on every record (the algorithm line states both conditions per record).
+ * Same arithmetic as the trace store: keys and query normalised to bf16, score =
+ * double-precision dot product rounded once to float.  Written as the plain
+ * definition: every slot is visited, all qualifying records are fully sorted.
+ */
+typedef struct {
+  int32_t d, max_rollout;
+  int64_t cap, total;        /* slots; records ever appended              */
+  uint16_t *key;             /* [cap][d]                                  */
+  int32_t *anchor;           /* [cap]                                     */
+  int32_t *rollout;          /* [cap][max_rollout], padded with -1        */
+} oracle_ring;
+
+oracle_ring *oracle_ring_create(int32_t d, int64_t cap, int32_t max_rollout) {
+  if (d <= 0 || cap <= 0 || max_rollout <= 0) return NULL;
+  oracle_ring *r = (oracle_ring *)calloc(1, sizeof *r);
+  if (!r) return NULL;
+  r->d = d; r->cap = cap; r->max_rollout = max_rollout;
+  r->key = (uint16_t *)calloc((size_t)cap * d, sizeof(uint16_t));
+  r->anchor = (int32_t *)calloc((size_t)cap, sizeof(int32_t));
+  r->rollout = (int32_t *)calloc((size_t)cap * max_rollout, sizeof(int32_t));
+  if (!r->key || !r->anchor || !r->rollout) {
+    free(r->key); free(r->anchor); free(r->rollout); free(r);
+    return NULL;
+  }
+  return r;
+}
+
+void oracle_ring_destroy(oracle_ring *r) {
+  if (!r) return;
+  free(r->key); free(r->anchor); free(r->rollout); free(r);
+}
+
+void oracle_ring_reset(oracle_ring *r) { r->total = 0; }
+int64_t oracle_ring_size(const oracle_ring *r) { return r->total < r->cap ? r->total : r->cap; }
+int64_t oracle_ring_total(const oracle_ring *r) { return r->total; }
+const uint16_t *oracle_ring_keys(const oracle_ring *r) { return r->key; }
+const int32_t *oracle_ring_anchors(const oracle_ring *r) { return r->anchor; }
+const int32_t *oracle_ring_rollouts(const oracle_ring *r) { return r->rollout; }
+
+/* Append n records in order; record i goes to slot (total + i) mod cap. */
+void oracle_ring_append(oracle_ring *r, const uint16_t *states, const int32_t *anchors,
+                        const int32_t *rollouts, int64_t n) {
+  for (int64_t i = 0; i < n; ++i) {
+    int64_t slot = (r->total + i) % r->cap;
+    oracle_normalize_bf16(r->d, states + (size_t)i * r->d, r->key + (size_t)slot * r->d);
+    r->anchor[slot] = anchors[i];
+    for (int32_t t = 0; t < r->max_rollout; ++t)
+      r->rollout[(size_t)slot * r->max_rollout + t] = rollouts[(size_t)i * r->max_rollout + t];
+  }
+  r->total += n;
+}
+
+/*
+ * Lookup for nq (state, anchor) pairs.  Outputs: slot[nq][m] (-1 padded),
+ * score[nq][m] (-inf padded), count[nq], rollout[nq][m][max_rollout] (-1 padded),
+ * rollout_len[nq][m] (tokens before the first negative entry).
+ */
+int oracle_ring_query(const oracle_ring *r, const uint16_t *q_raw, const int32_t *q_anchor,
+                      int32_t nq, int32_t m, float floor_s, int64_t *slot, float *score,
+                      int32_t *count, int32_t *rollout, int32_t *rollout_len) {
+  const int64_t n = oracle_ring_size(r);
+  const int32_t d = r->d, R = r->max_rollout;
+  scored_row *cand = (scored_row *)malloc((size_t)(n > 0 ? n : 1) * sizeof(scored_row));
+  uint16_t *qn = (uint16_t *)malloc((size_t)d * sizeof(uint16_t));
+  if (!cand || !qn) { free(cand); free(qn); return -1; }
+  for (int32_t q = 0; q < nq; ++q) {
+    int finite = 1;
+    for (int32_t j = 0; j < d; ++j)
+      if (!isfinite(oracle_bf16_to_f32(q_raw[(size_t)q * d + j]))) finite = 0;
+    oracle_normalize_bf16(d, q_raw + (size_t)q * d, qn);
+    int64_t nc = 0;
+    for (int64_t i = 0; i < n && finite; ++i) {
+      if (r->anchor[i] != q_anchor[q]) continue;          /* anchor token must be equal */
+      double acc = 0.0;
+      for (int32_t j = 0; j < d; ++j)
+        acc += (double)oracle_bf16_to_f32(qn[j]) * (double)oracle_bf16_to_f32(r->key[(size_t)i * d + j]);
+      float s = (float)acc;
+      if (s >= floor_s) { cand[nc].s = s; cand[nc].i = i; ++nc; }   /* cosine floor */
+    }
+    qsort(cand, (size_t)nc, sizeof(scored_row), cmp_scored);
+    count[q] = (int32_t)(nc < m ? nc : m);
+    for (int32_t j = 0; j < m; ++j) {
+      int have = j < nc;
+      slot[(size_t)q * m + j] = have ? cand[j].i : -1;
+      score[(size_t)q * m + j] = have ? cand[j].s : -INFINITY;
+      int32_t len = 0, open = 1;
+      for (int32_t t = 0; t < R; ++t) {
+        int32_t tok = have ? r->rollout[(size_t)cand[j].i * R + t] : -1;
+        if (tok < 0) open = 0;
+        if (open) ++len;
+        rollout[((size_t)q * m + j) * R + t] = open ? tok : -1;
+      }
+      rollout_len[(size_t)q * m + j] = len;
+    }
+  }
+  free(cand); free(qn);
+  return 0;
+}

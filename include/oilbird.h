@@ -210,6 +210,65 @@ int32_t oilbird_pool_profile_read(oilbird_pool_t* pool, float* scan_ms, int32_t 
 int64_t oilbird_pool_launch_count(const oilbird_pool_t* pool);
 
 /*
+ * Recycled pool (paper Section 4 "(i b) Recycling"; Algorithm 1, recycled-pool line): a
+ * ring buffer of records made from the draft-tree nodes that verification rejected.  A
+ * record is keyed by the hidden state in front of the rejected token and by that token
+ * (the anchor); its value is the short continuation the model endorsed from there (up to
+ * six tokens in the paper).  When the ring is full the oldest record is overwritten.
+ * A lookup with the current state and the current anchor token returns, best first, at
+ * most m records whose anchor is equal and whose cosine with the query reaches `floor`
+ * (paper: m = 4, floor = 0.8; here the floor filters every record, it is not a firing
+ * condition); equal scores list the lower slot first.
+ */
+#define OILBIRD_RING_MAX_M        32   /* results per query                               */
+#define OILBIRD_RING_MAX_ROLLOUT  16   /* tokens per stored continuation                  */
+#define OILBIRD_RING_MAX_NQ       64   /* queries per call                                */
+
+typedef struct oilbird_ring oilbird_ring_t;   /* opaque */
+
+typedef struct {
+  int32_t d;             /* key width, multiple of 8, 8..16384                           */
+  int64_t capacity;      /* records (slots) the ring holds                               */
+  int32_t max_rollout;   /* tokens per continuation, 1..OILBIRD_RING_MAX_ROLLOUT; 0 = 6  */
+  int32_t device;        /* CUDA ordinal                                                 */
+} oilbird_ring_config;
+
+typedef struct {         /* all dev, caller-owned, written on every call                 */
+  int32_t* slot;         /* [nq,m]  ring slot of each result, -1 padded                  */
+  float*   score;        /* [nq,m]  cosine, -INF padded                                  */
+  int32_t* count;        /* [nq]    number of results (<= m)                             */
+  int32_t* rollout;      /* [nq,m,max_rollout] stored continuation, -1 padded            */
+  int32_t* rollout_len;  /* [nq,m]  tokens before the first negative entry               */
+} oilbird_ring_out;
+
+int oilbird_ring_create (oilbird_ring_t** out, const oilbird_ring_config* cfg);
+int oilbird_ring_destroy(oilbird_ring_t* ring);
+int oilbird_ring_reset  (oilbird_ring_t* ring, void* cuda_stream);
+int64_t oilbird_ring_size (const oilbird_ring_t* ring);   /* records held (<= capacity)   */
+int64_t oilbird_ring_total(const oilbird_ring_t* ring);   /* records ever appended        */
+/*
+ * Append n records in order; record i goes to slot (total + i) mod capacity.  states: dev
+ * [n,d] bf16 (normalised as for the trace pool), anchors: dev [n] int32, rollouts: dev
+ * [n,max_rollout] int32 padded with -1.  If n exceeds the capacity only the last
+ * `capacity` records are stored.  Enqueues on cuda_stream; never synchronises.
+ */
+int oilbird_ring_append(oilbird_ring_t* ring, const void* states_bf16, const int32_t* anchors,
+                        const int32_t* rollouts, int64_t n, void* cuda_stream);
+/*
+ * Lookup for nq (state, anchor) pairs: q dev [nq,d] bf16, q_anchor dev [nq] int32,
+ * 1 <= m <= OILBIRD_RING_MAX_M.  Only records whose anchor matches are scored, so the
+ * cost is one pass over the anchors plus the keys of the matching records.
+ * A query holding NaN/Inf returns nothing.  Errors: EINVAL.
+ */
+int oilbird_ring_query(oilbird_ring_t* ring, const void* q_bf16, const int32_t* q_anchor,
+                       int32_t nq, int32_t m, float floor, const oilbird_ring_out* out,
+                       void* cuda_stream);
+/* Copy stored records to the host (synchronous; tests and debugging). */
+int oilbird_ring_read(oilbird_ring_t* ring, void* keys_host, int32_t* anchors_host,
+                      int32_t* rollouts_host);
+const char* oilbird_ring_last_error(void);      /* text of the last failing CUDA call     */
+
+/*
  * Query without any allocation (the paper has no counterpart; this serves hosts of the
  * library that own all device memory themselves and must not let a library allocate:
  * for instance a serving engine that reserved the whole of HBM at start-up, where a

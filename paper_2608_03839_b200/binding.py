@@ -51,6 +51,16 @@ class StaticPool(ctypes.Structure):
                 ("n_rows", ctypes.c_int64), ("d", ctypes.c_int32), ("device", ctypes.c_int32)]
 
 
+class RingConfig(ctypes.Structure):
+    _fields_ = [("d", ctypes.c_int32), ("capacity", ctypes.c_int64),
+                ("max_rollout", ctypes.c_int32), ("device", ctypes.c_int32)]
+
+
+class CRingOut(ctypes.Structure):
+    _fields_ = [("slot", ctypes.c_void_p), ("score", ctypes.c_void_p), ("count", ctypes.c_void_p),
+                ("rollout", ctypes.c_void_p), ("rollout_len", ctypes.c_void_p)]
+
+
 class PoolStats(ctypes.Structure):
     _fields_ = [("degenerate_rows", ctypes.c_int64), ("nonfinite_queries", ctypes.c_int64),
                 ("stalled", ctypes.c_int32), ("reserved", ctypes.c_int32)]
@@ -81,6 +91,16 @@ SYMBOLS = {
     "oilbird_pool_profile": (ctypes.c_int, [_vp, _i32]),
     "oilbird_pool_profile_read": (_i32, [_vp, _vp, _i32]),
     "oilbird_pool_launch_count": (_i64, [_vp]),
+    "oilbird_ring_create": (ctypes.c_int, [ctypes.POINTER(_vp), ctypes.POINTER(RingConfig)]),
+    "oilbird_ring_destroy": (ctypes.c_int, [_vp]),
+    "oilbird_ring_reset": (ctypes.c_int, [_vp, _vp]),
+    "oilbird_ring_size": (_i64, [_vp]),
+    "oilbird_ring_total": (_i64, [_vp]),
+    "oilbird_ring_append": (ctypes.c_int, [_vp, _vp, _vp, _vp, _i64, _vp]),
+    "oilbird_ring_query": (ctypes.c_int, [_vp, _vp, _vp, _i32, _i32, ctypes.c_float,
+                                          ctypes.POINTER(CRingOut), _vp]),
+    "oilbird_ring_read": (ctypes.c_int, [_vp, _vp, _vp, _vp]),
+    "oilbird_ring_last_error": (ctypes.c_char_p, []),
     "oilbird_query_static": (ctypes.c_int, [ctypes.POINTER(StaticPool), _vp, _i32,
                                             ctypes.POINTER(CQueryParams),
                                             ctypes.POINTER(CQueryOut), _vp]),
@@ -371,3 +391,93 @@ class Pool:
         buf = np.empty(max_n, dtype=np.float32)
         n = self._L.oilbird_pool_profile_read(self._h, buf.ctypes.data, max_n)
         return buf[:n].copy()
+
+
+# ------------------------------------------------------------------ recycled pool ----
+RING_MAX_M, RING_MAX_ROLLOUT, RING_MAX_NQ = 32, 16, 64
+
+
+@dataclass
+class RingOut:
+    slot: torch.Tensor         # [nq,m] int32, -1 padded
+    score: torch.Tensor        # [nq,m] float32, -inf padded
+    count: torch.Tensor        # [nq] int32
+    rollout: torch.Tensor      # [nq,m,R] int32, -1 padded
+    rollout_len: torch.Tensor  # [nq,m] int32
+
+    def cpu(self) -> "RingOut":
+        return RingOut(self.slot.cpu(), self.score.cpu(), self.count.cpu(), self.rollout.cpu(),
+                       self.rollout_len.cpu())
+
+
+class Ring:
+    """Rejected-branch ring buffer on one GPU (oilbird_ring_* of the C-ABI)."""
+
+    def __init__(self, d: int, capacity: int, max_rollout: int = 6, device: int = 0):
+        self._L = lib()
+        if not torch.cuda.is_available():
+            raise RuntimeError("oilbird ring needs a CUDA device; there is no CPU fallback")
+        self.d, self.capacity, self.max_rollout = int(d), int(capacity), int(max_rollout)
+        cfg = RingConfig(d=d, capacity=capacity, max_rollout=max_rollout, device=device)
+        h = ctypes.c_void_p()
+        _check(self._L.oilbird_ring_create(ctypes.byref(h), ctypes.byref(cfg)),
+               "oilbird_ring_create")
+        self._h = h
+        self._dev = torch.device(f"cuda:{device}")
+
+    def close(self) -> None:
+        h, self._h = getattr(self, "_h", None), None
+        if h:
+            self._L.oilbird_ring_destroy(h)
+
+    __del__ = close
+
+    def __len__(self) -> int:
+        return int(self._L.oilbird_ring_size(self._h))
+
+    @property
+    def total(self) -> int:
+        return int(self._L.oilbird_ring_total(self._h))
+
+    def reset(self, stream=None) -> None:
+        _check(self._L.oilbird_ring_reset(self._h, _stream_ptr(stream)), "oilbird_ring_reset")
+
+    def append(self, states: torch.Tensor, anchors: torch.Tensor, rollouts: torch.Tensor,
+               stream=None) -> None:
+        n = int(anchors.shape[0])
+        assert states.is_cuda and states.dtype == torch.bfloat16 and states.is_contiguous()
+        assert anchors.is_cuda and anchors.dtype == torch.int32 and anchors.is_contiguous()
+        assert rollouts.is_cuda and rollouts.dtype == torch.int32 and rollouts.is_contiguous()
+        assert states.shape == (n, self.d) and rollouts.shape == (n, self.max_rollout)
+        _check(self._L.oilbird_ring_append(self._h, states.data_ptr(), anchors.data_ptr(),
+                                           rollouts.data_ptr(), n, _stream_ptr(stream)),
+               "oilbird_ring_append")
+
+    def query(self, q: torch.Tensor, anchors: torch.Tensor, m: int = 4, floor: float = 0.8,
+              out: RingOut | None = None, stream=None) -> RingOut:
+        assert q.is_cuda and q.dtype == torch.bfloat16 and q.is_contiguous()
+        q = q.reshape(-1, self.d)
+        nq = q.shape[0]
+        assert anchors.is_cuda and anchors.dtype == torch.int32 and anchors.numel() == nq
+        if out is None:
+            kw = dict(device=self._dev)
+            out = RingOut(torch.empty((nq, m), dtype=torch.int32, **kw),
+                          torch.empty((nq, m), dtype=torch.float32, **kw),
+                          torch.empty((nq,), dtype=torch.int32, **kw),
+                          torch.empty((nq, m, self.max_rollout), dtype=torch.int32, **kw),
+                          torch.empty((nq, m), dtype=torch.int32, **kw))
+        co = CRingOut(out.slot.data_ptr(), out.score.data_ptr(), out.count.data_ptr(),
+                      out.rollout.data_ptr(), out.rollout_len.data_ptr())
+        _check(self._L.oilbird_ring_query(self._h, q.data_ptr(), anchors.data_ptr(), nq, int(m),
+                                          float(floor), ctypes.byref(co), _stream_ptr(stream)),
+               "oilbird_ring_query")
+        return out
+
+    def read(self):
+        """(keys uint16 [cap,d], anchors int32 [cap], rollouts int32 [cap,R]) as numpy arrays."""
+        keys = np.empty((self.capacity, self.d), np.uint16)
+        anc = np.empty(self.capacity, np.int32)
+        roll = np.empty((self.capacity, self.max_rollout), np.int32)
+        _check(self._L.oilbird_ring_read(self._h, keys.ctypes.data, anc.ctypes.data,
+                                         roll.ctypes.data), "oilbird_ring_read")
+        return keys, anc, roll

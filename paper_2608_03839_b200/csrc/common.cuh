@@ -188,4 +188,42 @@ __device__ __forceinline__ void block_merge_desc(u64 (&v)[E], u64* scratch, int 
   }
 }
 
+// ------------------------------------------------------ final merge (one CTA) ---
+constexpr int kMergeThreads = 1024;
+constexpr int kMergeWarps = kMergeThreads / 32;
+
+// Each warp folds its share of the scan's descending lists into a register-resident
+// list of kk = 32*E candidates (bitonic merges), then the warps' lists are merged.
+template <int E>
+__device__ __forceinline__ void merge_lists(const u64* __restrict__ partial, int n_lists, int nq,
+                                            int q, u64* scratch, u64* s_best) {
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  constexpr int KK = 32 * E;
+  u64 v[E];
+#pragma unroll
+  for (int r = 0; r < E; ++r) v[r] = 0;
+  // four lists in flight per warp: the loads, not the merges, set the pace
+  constexpr int PF = 4;
+  for (int l0 = warp; l0 < n_lists; l0 += kMergeWarps * PF) {
+    u64 b[PF][E];
+#pragma unroll
+    for (int p = 0; p < PF; ++p) {
+      const int l = l0 + p * kMergeWarps;
+      const u64* src = partial + ((size_t)(l < n_lists ? l : 0) * nq + q) * KK;
+#pragma unroll
+      for (int r = 0; r < E; ++r) b[p][r] = l < n_lists ? src[r * 32 + lane] : 0;
+    }
+#pragma unroll
+    for (int p = 0; p < PF; ++p)
+      if (l0 + p * kMergeWarps < n_lists) warp_merge_desc<E>(v, b[p], lane);
+  }
+  const int active = n_lists < kMergeWarps ? (n_lists < 1 ? 1 : n_lists) : kMergeWarps;
+  block_merge_desc<E>(v, scratch, active);
+  if (warp == 0) {
+#pragma unroll
+    for (int r = 0; r < E; ++r) s_best[r * 32 + lane] = v[r];
+  }
+  __syncthreads();
+}
+
 }  // namespace oilbird

@@ -13,9 +13,6 @@
 
 namespace oilbird {
 
-constexpr int kMergeThreads = 1024;
-constexpr int kMergeWarps = kMergeThreads / 32;
-
 // Eq. 3's D(s): first tier, in the order given, whose floor the score reaches.
 __device__ __forceinline__ int depth_of(float s, const GatherParams& gp) {
   if (gp.depth_mode == OILBIRD_DEPTH_FIXED) return gp.cont_len;
@@ -55,40 +52,6 @@ __device__ void fire_depth_copy(const PoolView& pv, const GatherParams& gp, int 
     const int j = e / L, t = e - j * L;
     dst[e] = t < s_len[j] ? pv.tok[(size_t)s_idx[j] + gp.offset + t] : -1;
   }
-}
-
-// Each warp folds its share of the scan's descending lists into a register-resident
-// list of kk = 32*E candidates (bitonic merges), then the warps' lists are merged.
-template <int E>
-__device__ __forceinline__ void merge_lists(const u64* __restrict__ partial, int n_lists, int nq,
-                                            int q, u64* scratch, u64* s_best) {
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  constexpr int KK = 32 * E;
-  u64 v[E];
-#pragma unroll
-  for (int r = 0; r < E; ++r) v[r] = 0;
-  // four lists in flight per warp: the loads, not the merges, set the pace
-  constexpr int PF = 4;
-  for (int l0 = warp; l0 < n_lists; l0 += kMergeWarps * PF) {
-    u64 b[PF][E];
-#pragma unroll
-    for (int p = 0; p < PF; ++p) {
-      const int l = l0 + p * kMergeWarps;
-      const u64* src = partial + ((size_t)(l < n_lists ? l : 0) * nq + q) * KK;
-#pragma unroll
-      for (int r = 0; r < E; ++r) b[p][r] = l < n_lists ? src[r * 32 + lane] : 0;
-    }
-#pragma unroll
-    for (int p = 0; p < PF; ++p)
-      if (l0 + p * kMergeWarps < n_lists) warp_merge_desc<E>(v, b[p], lane);
-  }
-  const int active = n_lists < kMergeWarps ? (n_lists < 1 ? 1 : n_lists) : kMergeWarps;
-  block_merge_desc<E>(v, scratch, active);
-  if (warp == 0) {
-#pragma unroll
-    for (int r = 0; r < E; ++r) s_best[r * 32 + lane] = v[r];
-  }
-  __syncthreads();
 }
 
 __global__ void __launch_bounds__(kMergeThreads)

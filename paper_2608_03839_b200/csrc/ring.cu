@@ -1,0 +1,293 @@
+// Recycled pool: ring buffer of rejected-branch records and its lookup.
+//
+// Paper Section 4 "(i b) Recycling" and Algorithm 1's recycled-pool line: records keyed
+// by (state in front of a rejected draft token, that token), valued by the continuation
+// the model endorsed; a lookup returns at most m records with an equal anchor token and
+// a cosine of at least `floor`, best first.
+//
+// Append is the hot side (every verification pass stores its rejected nodes): one CTA per
+// record normalises the state into the slot it overwrites.  The lookup first compares
+// anchor tokens (4 bytes per slot, coalesced) and streams the 16-byte key chunks of the
+// matching slots only, so its traffic is capacity*4 + matches*d*2 bytes instead of the
+// whole ring; each warp keeps its best records in a sorted register list, CTAs publish
+// one list each and a second kernel merges them and copies the continuations out.
+#include <math.h>
+#include <stdio.h>
+
+#include <new>
+
+#include "common.cuh"
+#include "internal.h"
+#include "normalize.cuh"
+
+namespace oilbird {
+
+constexpr int kRingThreads = kNormThreads;
+constexpr int kRingWarps = kRingThreads / 32;
+constexpr int kRingList = 32;          // candidates per published list (>= OILBIRD_RING_MAX_M)
+
+__global__ void __launch_bounds__(kRingThreads)
+ring_append_kernel(const uint16_t* __restrict__ states, const int32_t* __restrict__ anchors,
+                   const int32_t* __restrict__ rollouts, int64_t n, int d, int R, int64_t start,
+                   int64_t cap, uint16_t* __restrict__ keys, int32_t* __restrict__ anchor,
+                   int32_t* __restrict__ rollout) {
+  pdl_launch_dependents();
+  pdl_wait();   // an earlier lookup may still be reading the slots this append overwrites
+  for (int64_t r = blockIdx.x; r < n; r += gridDim.x) {
+    const int64_t slot = (start + r) % cap;
+    normalize_row(states + r * d, keys + slot * d, d);
+    if (threadIdx.x == 0) anchor[slot] = anchors[r];
+    if (threadIdx.x < R) rollout[slot * R + threadIdx.x] = rollouts[r * R + threadIdx.x];
+  }
+}
+
+// grid (slices, nq): CTA (s, q) scans slots [lo, hi) of the ring for query q.
+__global__ void __launch_bounds__(kRingThreads, 2)
+ring_scan_kernel(const uint16_t* __restrict__ keys, const int32_t* __restrict__ anchor,
+                 int64_t n_slots, int d, const uint16_t* __restrict__ q_raw,
+                 const int32_t* __restrict__ q_anchor, int nq, int m, float floor_s,
+                 u64* __restrict__ partial, int32_t* __restrict__ q_valid, DeviceStats* stats) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  const int n_chunks = d >> 3;
+  uint4* qs = reinterpret_cast<uint4*>(smem_raw);                           // [n_chunks]
+  u64* scratch = reinterpret_cast<u64*>(smem_raw + (size_t)d * 2);          // [warps][32]
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int q = blockIdx.y;
+  pdl_launch_dependents();
+  pdl_wait();
+  const int code = normalize_row(q_raw + (size_t)q * d, reinterpret_cast<uint16_t*>(qs), d);
+  if (blockIdx.x == 0 && threadIdx.x == 0) {
+    q_valid[q] = code == kRowNonFinite ? 0 : 1;
+    if (code == kRowNonFinite) atomicAdd(&stats->nonfinite_queries, 1ull);
+  }
+  __syncthreads();
+  const int xq = q_anchor[q];
+  const int64_t lo = n_slots * blockIdx.x / gridDim.x, hi = n_slots * (blockIdx.x + 1) / gridDim.x;
+  const uint4* keys4 = reinterpret_cast<const uint4*>(keys);
+
+  u64 top[1] = {0};
+  u64 kth = 0;
+  for (int64_t base = lo + warp * 32; base < hi; base += kRingWarps * 32) {
+    const int64_t slot = base + lane;
+    const bool hit = slot < hi && anchor[slot] == xq;          // anchor token must be equal
+    unsigned mask = __ballot_sync(0xffffffffu, hit);
+    while (mask) {
+      const int src = __ffs(mask) - 1;
+      mask &= mask - 1;
+      const int64_t s_row = base + src;
+      const uint4* rowp = keys4 + (size_t)s_row * n_chunks;
+      float acc = 0.f;
+#pragma unroll 4
+      for (int c = lane; c < n_chunks; c += 32) {
+        const uint4 kv = ld_stream16(rowp + c);
+        const uint4 qv = qs[c];
+        acc = fmaf(bf16_lo(kv.x), bf16_lo(qv.x), acc);
+        acc = fmaf(bf16_hi(kv.x), bf16_hi(qv.x), acc);
+        acc = fmaf(bf16_lo(kv.y), bf16_lo(qv.y), acc);
+        acc = fmaf(bf16_hi(kv.y), bf16_hi(qv.y), acc);
+        acc = fmaf(bf16_lo(kv.z), bf16_lo(qv.z), acc);
+        acc = fmaf(bf16_hi(kv.z), bf16_hi(qv.z), acc);
+        acc = fmaf(bf16_lo(kv.w), bf16_lo(qv.w), acc);
+        acc = fmaf(bf16_hi(kv.w), bf16_hi(qv.w), acc);
+      }
+      const float s = warp_sum(acc);
+      if (s >= floor_s) {                                      // cosine floor, per record
+        const u64 key = pack_candidate(s, (uint32_t)s_row);
+        if (key > kth) {
+          warp_sorted_insert<1>(top, key, lane);
+          kth = warp_list_get<1>(top, m - 1);
+        }
+      }
+    }
+  }
+  block_merge_desc<1>(top, scratch, kRingWarps);
+  if (threadIdx.x < 32) partial[((size_t)blockIdx.x * nq + q) * kRingList + lane] = top[0];
+}
+
+__global__ void __launch_bounds__(kMergeThreads)
+ring_merge_kernel(const u64* __restrict__ partial, int n_lists, int nq, int m, int R,
+                  const int32_t* __restrict__ q_valid, const int32_t* __restrict__ rollout,
+                  oilbird_ring_out out) {
+  __shared__ u64 scratch[kMergeWarps * kRingList];
+  __shared__ u64 s_best[kRingList];
+  const int q = blockIdx.x;
+  pdl_launch_dependents();
+  pdl_wait();
+  const int lists = q_valid[q] != 0 ? n_lists : 0;
+  merge_lists<1>(partial, lists, nq, q, scratch, s_best);
+  if (threadIdx.x == 0) {
+    int c = 0;
+    while (c < m && s_best[c] != 0) ++c;
+    out.count[q] = c;
+  }
+  __syncthreads();
+  for (int j = threadIdx.x; j < m; j += kMergeThreads) {
+    const u64 key = s_best[j];
+    out.slot[(size_t)q * m + j] = key ? candidate_row(key) : -1;
+    out.score[(size_t)q * m + j] = key ? candidate_score(key) : -INFINITY;
+  }
+  // stored continuation up to its first negative entry, -1 behind it
+  for (int j = threadIdx.x; j < m; j += kMergeThreads) {
+    const u64 key = s_best[j];
+    int len = 0;
+    bool open = key != 0;
+    for (int t = 0; t < R; ++t) {
+      int tok = open ? rollout[(size_t)candidate_row(key) * R + t] : -1;
+      if (tok < 0) open = false;
+      out.rollout[((size_t)q * m + j) * R + t] = open ? tok : -1;
+      if (open) ++len;
+    }
+    out.rollout_len[(size_t)q * m + j] = len;
+  }
+}
+
+}  // namespace oilbird
+
+using namespace oilbird;
+
+static thread_local char g_ring_err[256] = "";
+static int ring_fail(cudaError_t e, const char* what) {
+  snprintf(g_ring_err, sizeof g_ring_err, "%s: %s", what, cudaGetErrorString(e));
+  return e == cudaErrorMemoryAllocation ? OILBIRD_ENOMEM : OILBIRD_ECUDA;
+}
+#define RCU(call)                                         \
+  do {                                                    \
+    cudaError_t e_ = (call);                              \
+    if (e_ != cudaSuccess) return ring_fail(e_, #call);   \
+  } while (0)
+
+struct oilbird_ring {
+  int32_t d, R, device, num_sms, max_lists;
+  int64_t cap, total;
+  uint16_t* keys;
+  int32_t *anchor, *rollout, *q_valid;
+  unsigned long long* partial;
+  DeviceStats* stats;
+  unsigned char* base;
+};
+
+extern "C" {
+
+int oilbird_ring_create(oilbird_ring_t** out, const oilbird_ring_config* cfg) {
+  if (!out || !cfg) return OILBIRD_EINVAL;
+  *out = nullptr;
+  if (cfg->d < 8 || cfg->d > 16384 || cfg->d % 8 != 0 || cfg->capacity < 1 ||
+      cfg->capacity > 2147483000LL || cfg->max_rollout < 0 ||
+      cfg->max_rollout > OILBIRD_RING_MAX_ROLLOUT)
+    return OILBIRD_EINVAL;
+  int n_dev = 0;
+  RCU(cudaGetDeviceCount(&n_dev));
+  if (cfg->device < 0 || cfg->device >= n_dev) return OILBIRD_EINVAL;
+  RCU(cudaSetDevice(cfg->device));
+  int sms = 0;
+  RCU(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, cfg->device));
+  oilbird_ring* r = new (std::nothrow) oilbird_ring();
+  if (!r) return OILBIRD_ENOMEM;
+  r->d = cfg->d; r->R = cfg->max_rollout ? cfg->max_rollout : 6; r->device = cfg->device;
+  r->num_sms = sms; r->max_lists = 2 * sms; r->cap = cfg->capacity; r->total = 0;
+  auto up = [](size_t v) { return (v + 255) / 256 * 256; };
+  const size_t o_keys = 0, o_anchor = up((size_t)r->cap * r->d * 2),
+               o_roll = o_anchor + up((size_t)r->cap * 4),
+               o_valid = o_roll + up((size_t)r->cap * r->R * 4),
+               o_part = o_valid + up((size_t)OILBIRD_RING_MAX_NQ * 4),
+               o_stats = o_part + up((size_t)r->max_lists * OILBIRD_RING_MAX_NQ * kRingList * 8),
+               total = o_stats + up(sizeof(DeviceStats));
+  void* mem = nullptr;
+  cudaError_t e = cudaMalloc(&mem, total);
+  if (e != cudaSuccess) { delete r; return ring_fail(e, "cudaMalloc(ring)"); }
+  r->base = (unsigned char*)mem;
+  r->keys = (uint16_t*)(r->base + o_keys);
+  r->anchor = (int32_t*)(r->base + o_anchor);
+  r->rollout = (int32_t*)(r->base + o_roll);
+  r->q_valid = (int32_t*)(r->base + o_valid);
+  r->partial = (unsigned long long*)(r->base + o_part);
+  r->stats = (DeviceStats*)(r->base + o_stats);
+  e = cudaMemset(r->stats, 0, sizeof(DeviceStats));
+  if (e != cudaSuccess) { cudaFree(mem); delete r; return ring_fail(e, "cudaMemset"); }
+  *out = r;
+  return OILBIRD_OK;
+}
+
+int oilbird_ring_destroy(oilbird_ring_t* r) {
+  if (!r) return OILBIRD_EINVAL;
+  cudaSetDevice(r->device);
+  cudaDeviceSynchronize();
+  cudaFree(r->base);
+  delete r;
+  return OILBIRD_OK;
+}
+
+int oilbird_ring_reset(oilbird_ring_t* r, void* stream) {
+  if (!r) return OILBIRD_EINVAL;
+  RCU(cudaSetDevice(r->device));
+  RCU(cudaMemsetAsync(r->stats, 0, sizeof(DeviceStats), (cudaStream_t)stream));
+  r->total = 0;
+  return OILBIRD_OK;
+}
+
+int64_t oilbird_ring_size(const oilbird_ring_t* r) {
+  return r ? (r->total < r->cap ? r->total : r->cap) : 0;
+}
+int64_t oilbird_ring_total(const oilbird_ring_t* r) { return r ? r->total : 0; }
+
+int oilbird_ring_append(oilbird_ring_t* r, const void* states, const int32_t* anchors,
+                        const int32_t* rollouts, int64_t n, void* stream) {
+  if (!r || n < 0 || (n > 0 && (!states || !anchors || !rollouts))) return OILBIRD_EINVAL;
+  if (n == 0) return OILBIRD_OK;
+  RCU(cudaSetDevice(r->device));
+  // more records than slots: only the last `capacity` of them survive
+  const int64_t skip = n > r->cap ? n - r->cap : 0;
+  const int64_t m = n - skip;
+  const int64_t grid = m > 65535 * 8 ? 65535 * 8 : m;
+  cudaError_t e = launch_pdl(ring_append_kernel, dim3((unsigned)grid), dim3(kRingThreads), 0,
+                             (cudaStream_t)stream,
+                             (const uint16_t*)states + (size_t)skip * r->d, anchors + skip,
+                             rollouts + (size_t)skip * r->R, m, r->d, r->R, r->total + skip, r->cap,
+                             r->keys, r->anchor, r->rollout);
+  if (e != cudaSuccess) return ring_fail(e, "ring append launch");
+  r->total += n;
+  return OILBIRD_OK;
+}
+
+int oilbird_ring_query(oilbird_ring_t* r, const void* q, const int32_t* q_anchor, int32_t nq,
+                       int32_t m, float floor_s, const oilbird_ring_out* out, void* stream) {
+  if (!r || !q || !q_anchor || !out || !out->slot || !out->score || !out->count ||
+      !out->rollout || !out->rollout_len)
+    return OILBIRD_EINVAL;
+  if (nq < 1 || nq > OILBIRD_RING_MAX_NQ || m < 1 || m > OILBIRD_RING_MAX_M || isnan(floor_s))
+    return OILBIRD_EINVAL;
+  RCU(cudaSetDevice(r->device));
+  cudaStream_t st = (cudaStream_t)stream;
+  const int64_t n_slots = oilbird_ring_size(r);
+  // at least 256 slots per CTA, at most two CTAs per SM
+  int64_t want = (n_slots + 255) / 256;
+  int slices = (int)(want < 1 ? 1 : (want > r->max_lists ? r->max_lists : want));
+  const size_t smem = (size_t)r->d * 2 + (size_t)kRingWarps * kRingList * sizeof(u64);
+  RCU(cudaFuncSetAttribute(ring_scan_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           (int)smem));
+  cudaError_t e = launch_pdl(ring_scan_kernel, dim3(slices, nq), dim3(kRingThreads), smem, st,
+                             (const uint16_t*)r->keys, (const int32_t*)r->anchor, n_slots, r->d,
+                             (const uint16_t*)q, q_anchor, nq, m, floor_s, r->partial, r->q_valid,
+                             r->stats);
+  if (e != cudaSuccess) return ring_fail(e, "ring scan launch");
+  e = launch_pdl(ring_merge_kernel, dim3(nq), dim3(kMergeThreads), 0, st,
+                 (const u64*)r->partial, slices, nq, m, r->R, (const int32_t*)r->q_valid,
+                 (const int32_t*)r->rollout, *out);
+  if (e != cudaSuccess) return ring_fail(e, "ring merge launch");
+  return OILBIRD_OK;
+}
+
+int oilbird_ring_read(oilbird_ring_t* r, void* keys, int32_t* anchors, int32_t* rollouts) {
+  if (!r) return OILBIRD_EINVAL;
+  RCU(cudaSetDevice(r->device));
+  RCU(cudaDeviceSynchronize());
+  if (keys) RCU(cudaMemcpy(keys, r->keys, (size_t)r->cap * r->d * 2, cudaMemcpyDeviceToHost));
+  if (anchors) RCU(cudaMemcpy(anchors, r->anchor, (size_t)r->cap * 4, cudaMemcpyDeviceToHost));
+  if (rollouts)
+    RCU(cudaMemcpy(rollouts, r->rollout, (size_t)r->cap * r->R * 4, cudaMemcpyDeviceToHost));
+  return OILBIRD_OK;
+}
+
+const char* oilbird_ring_last_error(void) { return g_ring_err; }
+
+}  // extern "C"

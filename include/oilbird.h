@@ -269,6 +269,47 @@ int oilbird_ring_read(oilbird_ring_t* ring, void* keys_host, int32_t* anchors_ho
 const char* oilbird_ring_last_error(void);      /* text of the last failing CUDA call     */
 
 /*
+ * Chain post-filter and tree merge (Algorithm 1, chain collection and merge lines;
+ * Section 4 "(iii) Merge"; Eq. 4), for nq requests at once.  For each request the chains
+ * are taken in order: the k semantic chains as oilbird_pool_query returns them
+ * (cont_tok / cont_len: already by decreasing similarity, depth applied), then `ne` further
+ * chains of the caller (lexical branches, recycled-pool continuations).  A semantic chain
+ * with fewer than min_len tokens and any chain equal to one collected before it is
+ * dropped.  The others are merged into the request's draft tree from the root: a token
+ * already carried by a child of the current node is walked for free, any other token buys
+ * a node, until `budget` nodes are bought or max_nodes is reached (the chain is cut there
+ * and later chains are not reached).  cost = length - longest prefix already in the tree.
+ * With root_attached != 0 nothing is shared: every chain hangs from the root as its own
+ * branch (the paper's ablation arm).
+ * Tree layout per request: node 0 is the root (the anchor token), tree_parent[0] = -1;
+ * tree_tok / tree_parent [nq,max_nodes] and n_nodes [nq] are read and updated in place
+ * (new nodes are numbered in the order they are bought); depth [nq,max_nodes] and mask
+ * [nq,max_nodes] are written: bit j of mask[i] is set iff node j is node i or one of its
+ * ancestors (the attention mask of tree verification).  status / bought / walked
+ * [nq,k+ne]: OILBIRD_CHAIN_* code, nodes paid for (Eq. 4) and prefix walked, per chain.
+ * All pointers are dev; extra_* may be NULL when ne = 0, sem_* when k = 0.
+ */
+#define OILBIRD_TREE_MAX_NODES   64
+#define OILBIRD_CHAIN_SHORT        0   /* dropped: empty, or semantic and below min_len   */
+#define OILBIRD_CHAIN_DUPLICATE    1   /* dropped: equal to a chain collected before it   */
+#define OILBIRD_CHAIN_MERGED       2   /* merged completely                               */
+#define OILBIRD_CHAIN_CUT          3   /* merged until the budget or max_nodes ran out    */
+#define OILBIRD_CHAIN_NOT_REACHED  4   /* collected, but nothing was left to spend        */
+typedef struct {
+  int32_t budget;         /* B_ret, paper: 16                                            */
+  int32_t max_nodes;      /* tree capacity and row stride, paper: 60; <= 64              */
+  int32_t min_len;        /* shortest semantic chain kept, paper: 2                      */
+  int32_t root_attached;  /* 0 = merge from the root (deployed), 1 = ablation            */
+} oilbird_merge_params;
+void oilbird_merge_params_default(oilbird_merge_params* p);
+int oilbird_merge_chains(int32_t nq, const int32_t* sem_tok, const int32_t* sem_len, int32_t k,
+                         int32_t L, const int32_t* extra_tok, const int32_t* extra_len,
+                         int32_t ne, int32_t Le, int32_t* tree_tok, int32_t* tree_parent,
+                         int32_t* n_nodes, int32_t* depth, uint64_t* mask, int32_t* status,
+                         int32_t* bought, int32_t* walked, const oilbird_merge_params* params,
+                         int32_t device, void* cuda_stream);
+
+/*
  * Query without any allocation (the paper has no counterpart; this serves hosts of the
  * library that own all device memory themselves and must not let a library allocate:
  * for instance a serving engine that reserved the whole of HBM at start-up, where a

@@ -61,6 +61,11 @@ class CRingOut(ctypes.Structure):
                 ("rollout", ctypes.c_void_p), ("rollout_len", ctypes.c_void_p)]
 
 
+class MergeParams(ctypes.Structure):
+    _fields_ = [("budget", ctypes.c_int32), ("max_nodes", ctypes.c_int32),
+                ("min_len", ctypes.c_int32), ("root_attached", ctypes.c_int32)]
+
+
 class PoolStats(ctypes.Structure):
     _fields_ = [("degenerate_rows", ctypes.c_int64), ("nonfinite_queries", ctypes.c_int64),
                 ("stalled", ctypes.c_int32), ("reserved", ctypes.c_int32)]
@@ -101,6 +106,10 @@ SYMBOLS = {
                                           ctypes.POINTER(CRingOut), _vp]),
     "oilbird_ring_read": (ctypes.c_int, [_vp, _vp, _vp, _vp]),
     "oilbird_ring_last_error": (ctypes.c_char_p, []),
+    "oilbird_merge_params_default": (None, [ctypes.POINTER(MergeParams)]),
+    "oilbird_merge_chains": (ctypes.c_int, [_i32, _vp, _vp, _i32, _i32, _vp, _vp, _i32, _i32, _vp,
+                                            _vp, _vp, _vp, _vp, _vp, _vp, _vp,
+                                            ctypes.POINTER(MergeParams), _i32, _vp]),
     "oilbird_query_static": (ctypes.c_int, [ctypes.POINTER(StaticPool), _vp, _i32,
                                             ctypes.POINTER(CQueryParams),
                                             ctypes.POINTER(CQueryOut), _vp]),
@@ -481,3 +490,52 @@ class Ring:
         _check(self._L.oilbird_ring_read(self._h, keys.ctypes.data, anc.ctypes.data,
                                          roll.ctypes.data), "oilbird_ring_read")
         return keys, anc, roll
+
+
+# ------------------------------------------------------------------ tree merge ----
+TREE_MAX_NODES = 64
+CHAIN_SHORT, CHAIN_DUPLICATE, CHAIN_MERGED, CHAIN_CUT, CHAIN_NOT_REACHED = range(5)
+
+
+@dataclass
+class MergeOut:
+    tree_tok: torch.Tensor      # [nq,max_nodes] int32 (updated in place)
+    tree_parent: torch.Tensor   # [nq,max_nodes] int32
+    n_nodes: torch.Tensor       # [nq] int32
+    depth: torch.Tensor         # [nq,max_nodes] int32
+    mask: torch.Tensor          # [nq,max_nodes] int64 (bit j: node j is self or an ancestor)
+    status: torch.Tensor        # [nq,k+ne] int32
+    bought: torch.Tensor        # [nq,k+ne] int32
+    walked: torch.Tensor        # [nq,k+ne] int32
+
+
+def merge_chains(tree_tok: torch.Tensor, tree_parent: torch.Tensor, n_nodes: torch.Tensor,
+                 sem_tok: torch.Tensor | None, sem_len: torch.Tensor | None,
+                 extra_tok: torch.Tensor | None = None, extra_len: torch.Tensor | None = None,
+                 budget: int = 16, min_len: int = 2, root_attached: bool = False,
+                 stream=None) -> MergeOut:
+    """oilbird_merge_chains: post-filter the chains and merge them into each request's tree.
+
+    tree_tok / tree_parent: CUDA int32 [nq,max_nodes] (updated in place), n_nodes: [nq].
+    sem_tok [nq,k,L] / sem_len [nq,k]: a query's cont_tok / cont_len.  extra_*: further chains.
+    """
+    nq, max_nodes = tree_tok.shape
+    dev = tree_tok.device
+    k, L = (sem_tok.shape[1], sem_tok.shape[2]) if sem_tok is not None else (0, 1)
+    ne, Le = (extra_tok.shape[1], extra_tok.shape[2]) if extra_tok is not None else (0, 1)
+    for t in (tree_tok, tree_parent, n_nodes, sem_tok, sem_len, extra_tok, extra_len):
+        assert t is None or (t.is_cuda and t.dtype == torch.int32 and t.is_contiguous())
+    depth = torch.empty((nq, max_nodes), dtype=torch.int32, device=dev)
+    mask = torch.empty((nq, max_nodes), dtype=torch.int64, device=dev)
+    status = torch.empty((nq, k + ne), dtype=torch.int32, device=dev)
+    bought = torch.empty_like(status)
+    walked = torch.empty_like(status)
+    mp = MergeParams(budget, max_nodes, min_len, int(bool(root_attached)))
+    ptr = lambda t: None if t is None else t.data_ptr()
+    _check(lib().oilbird_merge_chains(nq, ptr(sem_tok), ptr(sem_len), k, L, ptr(extra_tok),
+                                      ptr(extra_len), ne, Le, tree_tok.data_ptr(),
+                                      tree_parent.data_ptr(), n_nodes.data_ptr(), depth.data_ptr(),
+                                      mask.data_ptr(), status.data_ptr(), bought.data_ptr(),
+                                      walked.data_ptr(), ctypes.byref(mp), dev.index or 0,
+                                      _stream_ptr(stream)), "oilbird_merge_chains")
+    return MergeOut(tree_tok, tree_parent, n_nodes, depth, mask, status, bought, walked)

@@ -522,6 +522,61 @@ def run_ring(args):
     print(json.dumps(line), flush=True)
 
 
+def run_merge(args):
+    """Third workload: chain post-filter + tree merge for a batch of requests (paper sizes:
+    8 semantic chains of up to 48 tokens + 7 other chains into a 44-node tree, 16 of 60 nodes)."""
+    from paper_2608_03839_b200 import binding as B
+    from oracle import merge as OM
+    torch.cuda.set_device(0)
+    nq, k, L, ne, Le = args.nq or 64, 8, 48, 7, 32
+    K, Wm = args.steps, args.warmup
+    rng = np.random.default_rng(0x3E46E)
+    base = rng.integers(0, 128256, 64)
+    t_tok = np.full((nq, 60), -1, np.int32); t_par = np.full((nq, 60), -1, np.int32)
+    t_tok[:, :44] = np.concatenate([[7], base[:43]]); t_par[:, :44] = np.arange(-1, 43)
+    s_tok = np.tile(base[:L], (nq, k, 1)).astype(np.int32)
+    for q in range(nq):                              # neighbours agree up to a random point
+        for j in range(k):
+            cut = rng.integers(2, L)
+            s_tok[q, j, cut:] = rng.integers(0, 128256, L - cut)
+    s_len = rng.choice([48, 48, 8, 8, 0], (nq, k)).astype(np.int32)
+    e_tok = rng.integers(0, 128256, (nq, ne, Le)).astype(np.int32)
+    e_len = rng.integers(1, Le + 1, (nq, ne)).astype(np.int32)
+    dev = lambda a: torch.from_numpy(a).cuda()
+    d_s, d_sl, d_e, d_el = dev(s_tok), dev(s_len), dev(e_tok), dev(e_len)
+    trees = [(dev(t_tok), dev(t_par), torch.full((nq,), 44, dtype=torch.int32, device="cuda"))
+             for _ in range(Wm + K)]
+    for i in range(Wm):
+        B.merge_chains(*trees[i], d_s, d_sl, d_e, d_el, budget=16)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for i in range(K):
+        B.merge_chains(*trees[Wm + i], d_s, d_sl, d_e, d_el, budget=16)
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / K
+    t0 = time.perf_counter()
+    for q in range(nq):
+        OM.merge_chains(t_tok[q, :44], t_par[q, :44], 44,
+                        [s_tok[q, j, : s_len[q, j]] for j in range(k)],
+                        [e_tok[q, j, : e_len[q, j]] for j in range(ne)], budget=16, max_nodes=60)
+    cpu_dt = time.perf_counter() - t0
+    line = {"metric": "tree_merges_per_sec", "value": nq / (ms / 1e3), "unit": "requests/s",
+            "n_gpus": 1, "steps": K, "warmup": Wm, "ms_per_step": ms, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "int32", "data": "synthetic",
+            "config": {"workload": f"merge: {nq} requests, {k} semantic chains (<= {L} tokens) + {ne} "
+                                   f"other chains into a 44-node tree, B_ret=16 of 60 nodes"},
+            "gpu_launches": K,
+            "roofline": {"bound": "alu", "kernel": "merge_tree_kernel", "achieved": None, "peak": None,
+                         "frac": None, "traffic": None,
+                         "note": "sequential per request (one warp each), a few hundred tokens: "
+                                 "launch-latency bound, no roofline applies"},
+            "cpu_baseline": {"value": nq / cpu_dt, "unit": "requests/s", "cores": 1, "kind": "oracle",
+                             "sample": f"the same {nq} requests through the Python oracle"}}
+    print(json.dumps(line), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -533,7 +588,7 @@ def main():
     ap.add_argument("--rows", type=int, default=0,
                     help="override the pool size (profiling a smaller case of the same recipe)")
     ap.add_argument("--path", type=int, default=0, help="0 auto, 1 CUDA-core scan, 2 tensor scan")
-    ap.add_argument("--workload", default="pool", choices=["pool", "ring"],
+    ap.add_argument("--workload", default="pool", choices=["pool", "ring", "merge"],
                     help="pool: the trace-store query path (default); ring: the recycled pool")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-budget", type=float, default=20.0)
@@ -547,6 +602,11 @@ def main():
         args.steps = 500 if args.steps is None else args.steps
         args.warmup = 10 if args.warmup is None else max(args.warmup, 3)
         run_ring(args)
+        return
+    if args.workload == "merge":
+        args.steps = 200 if args.steps is None else args.steps
+        args.warmup = 10 if args.warmup is None else max(args.warmup, 3)
+        run_merge(args)
         return
     default_steps = {"C1": 500, "C2": 500, "C3": 300, "C4": 100, "C5": 50}[args.config]
     args.steps = default_steps if args.steps is None else args.steps

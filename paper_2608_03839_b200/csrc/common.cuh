@@ -202,8 +202,9 @@ __device__ __forceinline__ void merge_lists(const u64* __restrict__ partial, int
   u64 v[E];
 #pragma unroll
   for (int r = 0; r < E; ++r) v[r] = 0;
-  // four lists in flight per warp: the loads, not the merges, set the pace
-  constexpr int PF = 4;
+  // many lists in flight per warp: the loads, not the merges, set the pace (with two CTAs
+  // per SM a warp folds about ten lists, so one round of loads covers the common case)
+  constexpr int PF = E == 1 ? 10 : (E == 2 ? 5 : 3);
   for (int l0 = warp; l0 < n_lists; l0 += kMergeWarps * PF) {
     u64 b[PF][E];
 #pragma unroll

@@ -45,10 +45,33 @@ __device__ void fire_depth_copy(const PoolView& pv, const GatherParams& gp, int 
     s_len[j] = len;
     out.cont_len[(size_t)q * k + j] = len;
   }
-  __syncthreads();
-  // a6: gamma = x_{idx+offset : idx+offset+len}, padded with -1
+  // a6: gamma = x_{idx+offset : idx+offset+len}, padded with -1.  The tokens are fetched
+  // before the lengths are known (any row below n_rows may be read) so that this load does
+  // not queue behind the trace lookups above; the length then masks them.
   int32_t* dst = out.cont_tok + (size_t)q * k * L;
-  for (int e = threadIdx.x; e < k * L; e += blockDim.x) {
+  constexpr int kSpec = 4;
+  const int n_out = k * L;
+  int32_t v[kSpec];
+#pragma unroll
+  for (int u = 0; u < kSpec; ++u) {
+    const int e = threadIdx.x + u * blockDim.x;
+    v[u] = -1;
+    if (e < n_out) {
+      const int j = e / L, t = e - j * L;
+      const long long row = (long long)s_idx[j] + gp.offset + t;
+      if (fired && s_idx[j] >= 0 && row < pv.n_rows) v[u] = pv.tok[row];
+    }
+  }
+  __syncthreads();                               // s_len is complete
+#pragma unroll
+  for (int u = 0; u < kSpec; ++u) {
+    const int e = threadIdx.x + u * blockDim.x;
+    if (e < n_out) {
+      const int j = e / L, t = e - j * L;
+      dst[e] = t < s_len[j] ? v[u] : -1;
+    }
+  }
+  for (int e = threadIdx.x + kSpec * blockDim.x; e < n_out; e += blockDim.x) {
     const int j = e / L, t = e - j * L;
     dst[e] = t < s_len[j] ? pv.tok[(size_t)s_idx[j] + gp.offset + t] : -1;
   }
@@ -66,12 +89,12 @@ merge_gather_kernel(PoolView pv, const u64* __restrict__ partial, int n_lists, i
   const int k = gp.k;
   pdl_launch_dependents();
   pdl_wait();   // the scan's candidate lists
-  const int lists = q_valid[q] != 0 ? n_lists : 0;   // NaN/Inf query: no neighbours
-  if (kk == 32) merge_lists<1>(partial, lists, nq, q, scratch, s_best);
-  else if (kk == 64) merge_lists<2>(partial, lists, nq, q, scratch, s_best);
-  else merge_lists<4>(partial, lists, nq, q, scratch, s_best);
+  const int valid = q_valid[q];       // consumed after the merge: the load overlaps it
+  if (kk == 32) merge_lists<1>(partial, n_lists, nq, q, scratch, s_best);
+  else if (kk == 64) merge_lists<2>(partial, n_lists, nq, q, scratch, s_best);
+  else merge_lists<4>(partial, n_lists, nq, q, scratch, s_best);
   for (int j = threadIdx.x; j < k; j += kMergeThreads) {
-    const u64 key = s_best[j];
+    const u64 key = valid ? s_best[j] : 0;            // NaN/Inf query: no neighbours
     const int idx = key ? candidate_row(key) : -1;
     const float s = key ? candidate_score(key) : -INFINITY;
     s_idx[j] = idx;

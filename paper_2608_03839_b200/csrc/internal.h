@@ -80,15 +80,17 @@ cudaError_t launch_scan_gemv(const PoolView& pv, const uint16_t* q_raw, int32_t 
                              int32_t num_sms, int32_t* n_lists, cudaStream_t st);
 
 // a2+a3 (tensor cores): the same contract for queries [q0, q0+nq_c) of a call whose
-// normalised queries already sit in qn (row-major [>= q0+round16(nq_c), d]).  key_map and
-// q_map are CUtensorMap objects made by make_bf16_map (box rows 128 and round16(nq_c)).
-bool make_bf16_map(void* map_out, const void* base, int64_t rows, int32_t d, int32_t box_rows);
+// normalised queries already sit in qn.  TcCache holds the pool's TMA tensor maps
+// (nullptr from create = tensor path unavailable).
+struct TcCache;
+TcCache* tc_cache_create(const void* keys, int64_t capacity, int32_t d, const void* qn,
+                         int64_t qn_rows);
+void tc_cache_destroy(TcCache* cache);
 int tc_queries_per_pass(int nq, int k, size_t smem_limit);   // balanced split of a call
-cudaError_t launch_scan_tc(const void* key_map, const void* q_map, const PoolView& pv, int32_t q0,
-                           int32_t nq_c, int32_t nq_total, int32_t k, int32_t kk,
-                           const uint64_t* exclude_tag, unsigned long long* partial,
-                           DeviceStats* stats, int32_t num_sms, size_t smem_limit,
-                           int32_t* n_lists, cudaStream_t st);
+cudaError_t launch_scan_tc(TcCache* cache, const PoolView& pv, int32_t q0, int32_t nq_c,
+                           int32_t nq_total, int32_t k, int32_t kk, const uint64_t* exclude_tag,
+                           unsigned long long* partial, DeviceStats* stats, int32_t num_sms,
+                           size_t smem_limit, int32_t* n_lists, cudaStream_t st);
 
 // a3 (final merge) + a4 + a5 + a6: one CTA per query.
 cudaError_t launch_merge_gather(const PoolView& pv, const unsigned long long* partial,

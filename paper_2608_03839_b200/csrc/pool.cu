@@ -115,12 +115,9 @@ struct oilbird_pool {
   size_t pinned_bytes;
   cudaEvent_t upload_done;
   bool upload_pending;
-  // tensor maps of the tensor-core scan (opaque 128-byte CUtensorMap objects)
+  // tensor-core scan: TMA tensor maps of this pool (nullptr = path unavailable)
   size_t smem_limit;
-  bool tc_ok;
-  alignas(64) unsigned char key_map[128];
-  alignas(64) unsigned char q_map[OILBIRD_MAX_NQ / 16][128];   // by box rows / 16 - 1
-  bool q_map_ok[OILBIRD_MAX_NQ / 16];
+  TcCache* tc;
 };
 
 extern "C" {
@@ -207,8 +204,9 @@ int oilbird_pool_create(oilbird_pool_t** out, const oilbird_pool_config* cfg) {
     return cuda_fail(e, "cudaMemset(stats)");
   }
   p->smem_limit = prop.sharedMemPerBlockOptin;
-  for (bool& b : p->q_map_ok) b = false;
-  p->tc_ok = prop.major == 10 && make_bf16_map(p->key_map, p->keys, r.capacity, r.d, 128);
+  p->tc = prop.major == 10 ? tc_cache_create(p->keys, r.capacity, r.d, p->qn,
+                                             (r.max_nq + 15) / 16 * 16)
+                           : nullptr;
   *out = p;
   return OILBIRD_OK;
 }
@@ -219,6 +217,7 @@ int oilbird_pool_destroy(oilbird_pool_t* p) {
   cudaDeviceSynchronize();
   for (cudaEvent_t e : p->ev) cudaEventDestroy(e);
   if (p->pinned) { cudaFreeHost(p->pinned); cudaEventDestroy(p->upload_done); }
+  tc_cache_destroy(p->tc);
   if (p->owns_mem) cudaFree(p->base);
   delete p;
   return OILBIRD_OK;
@@ -315,7 +314,7 @@ int oilbird_pool_query(oilbird_pool_t* p, const void* q, int32_t nq,
   // single-request decode streams keys through the CUDA cores; batches go to tcgen05
   int path = pr->path;
   if (path == OILBIRD_PATH_AUTO) path = nq <= 2 ? OILBIRD_PATH_GEMV : OILBIRD_PATH_TENSOR;
-  if (path == OILBIRD_PATH_TENSOR && !p->tc_ok) {
+  if (path == OILBIRD_PATH_TENSOR && !p->tc) {
     snprintf(g_cuda_err, sizeof g_cuda_err, "tensor-core scan unavailable on this device");
     return OILBIRD_ECUDA;
   }
@@ -350,18 +349,8 @@ int oilbird_pool_query(oilbird_pool_t* p, const void* q, int32_t nq,
       const int per_pass = tc_queries_per_pass(nq, pr->k, p->smem_limit);
       for (int q0 = 0; q0 < nq; q0 += per_pass) {
         const int nq_c = nq - q0 < per_pass ? nq - q0 : per_pass;
-        const int slot = (nq_c + 15) / 16 - 1;
-        if (!p->q_map_ok[slot]) {
-          if (!make_bf16_map(p->q_map[slot], p->qn, (p->r.max_nq + 15) / 16 * 16, p->r.d,
-                             (slot + 1) * 16)) {
-            snprintf(g_cuda_err, sizeof g_cuda_err, "cuTensorMapEncodeTiled(queries) failed");
-            return OILBIRD_ECUDA;
-          }
-          p->q_map_ok[slot] = true;
-        }
-        e = launch_scan_tc(p->key_map, p->q_map[slot], pv, q0, nq_c, nq, pr->k, kk,
-                           pr->exclude_tag, p->partial, p->stats, p->num_sms, p->smem_limit,
-                           &n_lists, st);
+        e = launch_scan_tc(p->tc, pv, q0, nq_c, nq, pr->k, kk, pr->exclude_tag, p->partial,
+                           p->stats, p->num_sms, p->smem_limit, &n_lists, st);
         if (e != cudaSuccess) return cuda_fail(e, "tensor scan kernel launch");
         p->launches += 1;
       }

@@ -20,6 +20,8 @@
 #include <cuda.h>
 #include <stdlib.h>
 
+#include <new>
+
 #include "common.cuh"
 #include "internal.h"
 
@@ -27,7 +29,10 @@ namespace oilbird {
 
 constexpr int kTcThreads = 192;
 constexpr int kTileM = 128;            // key rows per tile = TMEM lanes
-constexpr int kBlockK = 64;            // bf16 elements per k-block = one 128-byte swizzle row
+// bf16 elements per k-block = one 128-byte swizzle row.  (32-element blocks with the 64-byte
+// swizzle were measured too: more, finer ring stages, but every 128-byte line is then
+// requested twice and the scan runs 30-40 % slower at every nq.)
+constexpr int kBlockK = 64;
 constexpr int kATileBytes = kTileM * kBlockK * 2;   // 16 KB
 constexpr int kColsPerRound = 8;       // score columns filtered between two drains
 constexpr int kQueueCap = kTileM * kColsPerRound;
@@ -132,7 +137,7 @@ __device__ __forceinline__ uint64_t umma_desc_sw128(uint32_t smem_addr) {
   uint64_t d = 0;
   d |= (uint64_t)((smem_addr & 0x3FFFFu) >> 4);        // start address
   d |= (uint64_t)1 << 16;                              // leading byte offset (unused, 16 B)
-  d |= (uint64_t)(1024 >> 4) << 32;                    // stride byte offset
+  d |= (uint64_t)(1024 >> 4) << 32;                    // stride byte offset: 8 rows of 128 B
   d |= (uint64_t)1 << 46;                              // descriptor version (Blackwell)
   d |= (uint64_t)2 << 61;                              // SWIZZLE_128B
   return d;
@@ -418,17 +423,54 @@ static EncodeTiledFn encode_fn() {
 
 // Tensor map over a row-major bf16 matrix [rows, d]; box = 64 elements x box_rows rows,
 // 128B swizzle, out-of-range elements read as zero.
-bool make_bf16_map(void* map_out, const void* base, int64_t rows, int32_t d, int32_t box_rows) {
+static bool make_bf16_map(CUtensorMap* map_out, const void* base, int64_t rows, int32_t d,
+                          int32_t box_rows) {
   EncodeTiledFn fn = encode_fn();
   if (!fn) return false;
   cuuint64_t dims[2] = {(cuuint64_t)d, (cuuint64_t)rows};
   cuuint64_t strides[1] = {(cuuint64_t)d * 2};
   cuuint32_t box[2] = {(cuuint32_t)kBlockK, (cuuint32_t)box_rows};
   cuuint32_t estr[2] = {1, 1};
-  CUresult r = fn((CUtensorMap*)map_out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (void*)base, dims,
-                  strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+  CUresult r = fn(map_out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (void*)base, dims, strides, box,
+                  estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                   CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return r == CUDA_SUCCESS;
+}
+
+// Tensor maps of one pool: keys (fixed at creation: the map covers the whole capacity,
+// rows past the current size are masked in the epilogue) and, made on first use, the
+// normalised-query buffer for every box height.
+struct TcCache {
+  const void* qn;
+  int64_t qn_rows;
+  int32_t d;
+  alignas(64) CUtensorMap key_map;
+  alignas(64) CUtensorMap q_map[OILBIRD_MAX_NQ / 16];          // [n_pad / 16 - 1]
+  bool q_ok[OILBIRD_MAX_NQ / 16];
+};
+
+TcCache* tc_cache_create(const void* keys, int64_t capacity, int32_t d, const void* qn,
+                         int64_t qn_rows) {
+  TcCache* c = new (std::nothrow) TcCache();
+  if (!c) return nullptr;
+  c->qn = qn; c->qn_rows = qn_rows; c->d = d;
+  for (bool& b : c->q_ok) b = false;
+  if (!make_bf16_map(&c->key_map, keys, capacity, d, kTileM)) {
+    delete c;
+    return nullptr;
+  }
+  return c;
+}
+
+void tc_cache_destroy(TcCache* c) { delete c; }
+
+static const CUtensorMap* tc_q_map(TcCache* c, int n_pad) {
+  const int slot = n_pad / 16 - 1;
+  if (!c->q_ok[slot]) {
+    if (!make_bf16_map(&c->q_map[slot], c->qn, c->qn_rows, c->d, n_pad)) return nullptr;
+    c->q_ok[slot] = true;
+  }
+  return &c->q_map[slot];
 }
 
 static size_t tc_fixed_smem(int nq_c, int n_pad, int kk) {
@@ -475,11 +517,10 @@ int tc_queries_per_pass(int nq, int k, size_t smem_limit) {
   return tc_plan(nq, k, 0, 1, smem_limit, 1).per_pass;
 }
 
-cudaError_t launch_scan_tc(const void* key_map, const void* q_map, const PoolView& pv, int32_t q0,
-                           int32_t nq_c, int32_t nq_total, int32_t k, int32_t kk,
-                           const uint64_t* exclude_tag, unsigned long long* partial,
-                           DeviceStats* stats, int32_t num_sms, size_t smem_limit,
-                           int32_t* n_lists, cudaStream_t st) {
+cudaError_t launch_scan_tc(TcCache* cache, const PoolView& pv, int32_t q0, int32_t nq_c,
+                           int32_t nq_total, int32_t k, int32_t kk, const uint64_t* exclude_tag,
+                           unsigned long long* partial, DeviceStats* stats, int32_t num_sms,
+                           size_t smem_limit, int32_t* n_lists, cudaStream_t st) {
   const int n_pad = (nq_c + 15) / 16 * 16;
   const int n_tiles128 = (pv.n_rows + kTileM - 1) / kTileM;
   static const int force_mt = getenv("OILBIRD_TC_MT") ? atoi(getenv("OILBIRD_TC_MT")) : 0;
@@ -487,6 +528,8 @@ cudaError_t launch_scan_tc(const void* key_map, const void* q_map, const PoolVie
   const size_t stage = (size_t)plan.mt * kATileBytes + (size_t)n_pad * kBlockK * 2;
   const size_t fixed = tc_fixed_smem(nq_c, n_pad, kk);
   if (plan.stages < 2) return cudaErrorInvalidConfiguration;
+  const CUtensorMap* q_map = tc_q_map(cache, n_pad);
+  if (!q_map) return cudaErrorInvalidValue;
   size_t smem = fixed + (size_t)plan.stages * stage;
   if (smem < 120 * 1024) smem = 120 * 1024;   // one CTA per SM: TMEM is allocated per CTA
   int tmem_cols = 32;
@@ -499,9 +542,8 @@ cudaError_t launch_scan_tc(const void* key_map, const void* q_map, const PoolVie
                                        (int)smem);
   if (e != cudaSuccess) return e;
   return launch_pdl(scan_tc_kernel, dim3(grid), dim3(kTcThreads), smem, st,
-                    *(const CUtensorMap*)key_map, *(const CUtensorMap*)q_map, pv, q0, nq_c, nq_total,
-                    n_pad, k, kk, plan.stages, tmem_cols, plan.mt, plan.n_bufs, exclude_tag, partial,
-                    stats);
+                    cache->key_map, *q_map, pv, q0, nq_c, nq_total, n_pad, k, kk, plan.stages,
+                    tmem_cols, plan.mt, plan.n_bufs, exclude_tag, partial, stats);
 }
 
 }  // namespace oilbird

@@ -166,17 +166,26 @@ class QueryParams:
     path: int = PATH_AUTO
 
     def to_c(self, exclude_ptr=None) -> CQueryParams:
-        c = CQueryParams()
-        c.k, c.theta, c.offset = int(self.k), float(self.theta), int(self.offset)
-        c.depth_mode, c.cont_len = int(self.depth_mode), int(self.cont_len)
-        if len(self.tier_thr) != len(self.tier_depth) or len(self.tier_thr) > MAX_TIERS:
-            raise ValueError("tier_thr / tier_depth: same length, at most 4")
-        c.n_tiers = len(self.tier_thr)
-        for i, (t, dd) in enumerate(zip(self.tier_thr, self.tier_depth)):
-            c.tier_thr[i], c.tier_depth[i] = float(t), int(dd)
+        key = (self.k, self.theta, self.offset, self.depth_mode, self.cont_len,
+               tuple(self.tier_thr), tuple(self.tier_depth), self.path)
+        c = _PARAM_CACHE.get(key)
+        if c is None:
+            c = CQueryParams()
+            c.k, c.theta, c.offset = int(self.k), float(self.theta), int(self.offset)
+            c.depth_mode, c.cont_len = int(self.depth_mode), int(self.cont_len)
+            if len(self.tier_thr) != len(self.tier_depth) or len(self.tier_thr) > MAX_TIERS:
+                raise ValueError("tier_thr / tier_depth: same length, at most 4")
+            c.n_tiers = len(self.tier_thr)
+            for i, (t, dd) in enumerate(zip(self.tier_thr, self.tier_depth)):
+                c.tier_thr[i], c.tier_depth[i] = float(t), int(dd)
+            c.path = int(self.path)
+            if len(_PARAM_CACHE) < 256:
+                _PARAM_CACHE[key] = c
         c.exclude_tag = exclude_ptr
-        c.path = int(self.path)
         return c
+
+
+_PARAM_CACHE: dict = {}
 
 
 @dataclass

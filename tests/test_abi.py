@@ -75,3 +75,27 @@ def test_product_never_imports_the_oracle():
                 src = open(os.path.join(dirpath, f)).read()
                 assert "import oracle" not in src and "from oracle" not in src, f
                 assert "oilbird_oracle" not in src, f
+
+
+def test_missing_library_fails_loudly(monkeypatch):
+    """No CPU or PyTorch fallback: without liboilbird.so the binding refuses to work."""
+    monkeypatch.setattr(B, "_lib", None)
+    monkeypatch.setattr(B, "LIB_PATH", "/nonexistent/liboilbird.so")
+    with pytest.raises(ImportError, match="no CPU or PyTorch fallback"):
+        B.lib()
+
+
+def test_pool_needs_a_cuda_device():
+    import torch
+    if torch.cuda.is_available():
+        pytest.skip("this check is for the CPU-only box")
+    with pytest.raises(RuntimeError, match="no CPU fallback"):
+        B.Pool(64, 16)
+    with pytest.raises(RuntimeError, match="no CPU fallback"):
+        B.Ring(64, 16)
+
+
+def test_merge_defaults_are_the_papers_constants(L):
+    p = B.MergeParams()
+    L.oilbird_merge_params_default(ctypes.byref(p))
+    assert (p.budget, p.max_nodes, p.min_len, p.root_attached) == (16, 60, 2, 0)

@@ -577,6 +577,77 @@ def run_merge(args):
     print(json.dumps(line), flush=True)
 
 
+def run_sharded(args):
+    """Row-sharded mode: ONE logical pool of the configuration's size split by whole traces
+    over the ranks; every rank answers every query on its rows, one all-gather of the
+    records, merge on every rank.  Strong scaling: the total work is fixed."""
+    from paper_2608_03839_b200 import binding as B
+    from paper_2608_03839_b200 import sharded as S
+    import torch.distributed as dist
+    rank, world = env_int("RANK", 0), env_int("WORLD_SIZE", 1)
+    local = env_int("LOCAL_RANK", 0)
+    if world > 1:
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("nccl", device_id=torch.device(f"cuda:{local}"))
+    torch.cuda.set_device(local)
+    dev = torch.device(f"cuda:{local}")
+    w = W.CONFIGS[args.config]
+    nq = args.nq or w.nq
+    n0 = args.rows or (W.C5_START_ROWS if w.name == "C5" else w.n_rows)
+    K, Wm = args.steps, args.warmup
+    sp = S.ShardedPool(w.d, n0 // world + 2 * w.rows_per_trace + 8, max_nq=nq, max_k=w.k,
+                       device=local)
+    g = 0
+    for t, (st, tk, tag) in enumerate(w.traces(dev)):
+        if g >= n0:
+            break
+        if t % world == rank:                       # whole traces, round robin
+            sp.append(st, tk, global_row=g, tag=tag)
+        g += st.shape[0]
+    pr = B.QueryParams(k=w.k, theta=0.8, offset=2, depth_mode=B.DEPTH_FIXED, cont_len=w.cont_len,
+                       path=args.path)
+    qs = [w.queries(dev, nq=nq, step=i)[0] for i in range(8)]   # same seeds on every rank
+    for i in range(Wm):
+        sp.query(qs[i % 8], pr)
+    torch.cuda.synchronize()
+    if world > 1:
+        dist.barrier()
+    torch.cuda.synchronize()
+    sampler = ClockSampler(physical_device(local))
+    sampler.start()
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(K + 1)]
+    ev[0].record()
+    for i in range(K):
+        sp.query(qs[i % 8], pr)
+        ev[i + 1].record()
+    torch.cuda.synchronize()
+    if world > 1:
+        dist.barrier()
+    clocks = sampler.stop()
+    lat = np.array([ev[i].elapsed_time(ev[i + 1]) for i in range(K)])
+    max_ms, _ = aggregate(ev[0].elapsed_time(ev[K]), 0.0, world, dev)
+    if rank == 0:
+        peaks, peak_kind = measured_peaks()
+        p50 = float(np.percentile(lat, 50))
+        gbs = n0 * w.d * 2 / (p50 * 1e-3) / 1e9
+        line = {"metric": METRIC, "value": K * nq / (max_ms / 1e3), "unit": UNIT, "n_gpus": world,
+                "steps": K, "warmup": Wm, "ms_per_step": max_ms / K, "higher_is_better": True,
+                "scaling": "strong", "vs_baseline": None, "dtype": "bf16 keys, fp32 accumulate",
+                "data": "synthetic",
+                "config": {"workload": f"{w.name} row-sharded: ONE pool N={n0} x d={w.d} bf16 over "
+                                       f"{world} GPU(s), nq={nq}, k={w.k}, L={w.cont_len}; query only",
+                           "collective": "one all_gather of nq*k records per query"},
+                "p50_query_latency_us": p50 * 1e3, "key_scan_gbs_all_gpus": gbs, "clocks": clocks,
+                "gpu_launches": 4 * K,
+                "roofline": {"bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"] * world,
+                             "unit": "GB/s", "frac": gbs / (peaks["hbm_gbs"] * world),
+                             "peak_kind": peak_kind, "traffic": None,
+                             "kernel": "whole sharded query (scan + to_global + gather + merge)"}}
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -590,6 +661,8 @@ def main():
     ap.add_argument("--path", type=int, default=0, help="0 auto, 1 CUDA-core scan, 2 tensor scan")
     ap.add_argument("--workload", default="pool", choices=["pool", "ring", "merge"],
                     help="pool: the trace-store query path (default); ring: the recycled pool")
+    ap.add_argument("--sharded", action="store_true",
+                    help="one logical pool row-sharded over the ranks (default: one pool per rank)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-budget", type=float, default=20.0)
     args = ap.parse_args()
@@ -611,6 +684,9 @@ def main():
     default_steps = {"C1": 500, "C2": 500, "C3": 300, "C4": 100, "C5": 50}[args.config]
     args.steps = default_steps if args.steps is None else args.steps
     args.warmup = 10 if args.warmup is None else max(args.warmup, 3)
+    if args.sharded:
+        run_sharded(args)
+        return
     run_ours(args)
 
 

@@ -269,6 +269,35 @@ int oilbird_ring_read(oilbird_ring_t* ring, void* keys_host, int32_t* anchors_ho
 const char* oilbird_ring_last_error(void);      /* text of the last failing CUDA call     */
 
 /*
+ * Row sharding: one logical pool split by whole traces over several pools (one per GPU).
+ * The merged answer is what a single pool holding every row at its global position would
+ * return (Eq. 2 with the lowest-position tie rule; the theta test of Algorithm 1 on the
+ * global best).  Positions are assigned by the caller: append_global() is append() plus
+ * the global position of the first appended row, recorded when the call opens a trace (a
+ * trace's rows are consecutive globally as they are locally).  A query on a sharded pool
+ * is four steps: (1) oilbird_pool_query on every shard with theta = -INFINITY, so that
+ * every neighbour gets its depth and continuation; (2) oilbird_pool_to_global on the
+ * returned rows; (3) an all-gather of the shards' records (idx, score, cont_len,
+ * cont_tok), by the caller's communication library, into one buffer of n_shards equal
+ * slices; (4) oilbird_merge_shards, which selects the global top-k by (score descending,
+ * global position ascending), applies theta to the merged best and copies the winners'
+ * continuations (zero lengths and -1 tokens when not fired).
+ * gathered: dev, shard s starts at gathered + s*shard_stride; inside a slice, off_gidx
+ * (int64 [nq,k], 8-byte aligned), off_score (float [nq,k]), off_len (int32 [nq,k]),
+ * off_tok (int32 [nq,k,L]) are byte offsets.  n_shards * k <= 1024.
+ */
+int oilbird_pool_append_global(oilbird_pool_t* pool, const void* states_bf16,
+                               const int32_t* tokens, int64_t n, uint64_t trace_tag,
+                               uint32_t flags, int64_t global_row, void* cuda_stream);
+int oilbird_pool_to_global(oilbird_pool_t* pool, const int32_t* idx /* dev [n] */,
+                           int64_t* global_idx /* dev [n] */, int64_t n, void* cuda_stream);
+int oilbird_merge_shards(int32_t n_shards, int32_t nq, int32_t k, int32_t L, float theta,
+                         const void* gathered, size_t shard_stride, size_t off_gidx,
+                         size_t off_score, size_t off_len, size_t off_tok, int64_t* out_gidx,
+                         float* out_score, int32_t* out_fired, int32_t* out_len,
+                         int32_t* out_tok, int32_t device, void* cuda_stream);
+
+/*
  * Chain post-filter and tree merge (Algorithm 1, chain collection and merge lines;
  * Section 4 "(iii) Merge"; Eq. 4), for nq requests at once.  For each request the chains
  * are taken in order: the k semantic chains as oilbird_pool_query returns them

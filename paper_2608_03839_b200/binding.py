@@ -106,6 +106,12 @@ SYMBOLS = {
                                           ctypes.POINTER(CRingOut), _vp]),
     "oilbird_ring_read": (ctypes.c_int, [_vp, _vp, _vp, _vp]),
     "oilbird_ring_last_error": (ctypes.c_char_p, []),
+    "oilbird_pool_append_global": (ctypes.c_int, [_vp, _vp, _vp, _i64, _u64, _u32, _i64, _vp]),
+    "oilbird_pool_to_global": (ctypes.c_int, [_vp, _vp, _vp, _i64, _vp]),
+    "oilbird_merge_shards": (ctypes.c_int, [_i32, _i32, _i32, _i32, ctypes.c_float, _vp,
+                                            ctypes.c_size_t, ctypes.c_size_t, ctypes.c_size_t,
+                                            ctypes.c_size_t, ctypes.c_size_t, _vp, _vp, _vp, _vp,
+                                            _vp, _i32, _vp]),
     "oilbird_merge_params_default": (None, [ctypes.POINTER(MergeParams)]),
     "oilbird_merge_chains": (ctypes.c_int, [_i32, _vp, _vp, _i32, _i32, _vp, _vp, _i32, _i32, _vp,
                                             _vp, _vp, _vp, _vp, _vp, _vp, _vp,
@@ -312,6 +318,29 @@ class Pool:
                                            tokens.data_ptr() if n else None, n, int(tag),
                                            NEW_TRACE if new_trace else 0, _stream_ptr(stream)),
                "oilbird_pool_append")
+
+    def append_global(self, states: torch.Tensor, tokens: torch.Tensor, global_row: int,
+                      tag: int = 0, new_trace: bool = True, stream=None) -> None:
+        """append() for a pool that is one shard of a larger one: global_row is the position
+        of the first appended row in the logical pool."""
+        n = int(tokens.shape[0])
+        assert states.is_cuda and tokens.is_cuda and states.dtype == torch.bfloat16
+        assert tokens.dtype == torch.int32 and states.is_contiguous() and tokens.is_contiguous()
+        _check(self._L.oilbird_pool_append_global(
+            self._h, states.data_ptr(), tokens.data_ptr(), n, int(tag),
+            NEW_TRACE if new_trace else 0, int(global_row), _stream_ptr(stream)),
+            "oilbird_pool_append_global")
+
+    def to_global(self, idx: torch.Tensor, out: torch.Tensor | None = None, stream=None
+                  ) -> torch.Tensor:
+        """Local rows (int32) -> global positions (int64); -1 stays -1."""
+        assert idx.is_cuda and idx.dtype == torch.int32 and idx.is_contiguous()
+        if out is None:
+            out = torch.empty(idx.shape, dtype=torch.int64, device=idx.device)
+        _check(self._L.oilbird_pool_to_global(self._h, idx.data_ptr(), out.data_ptr(),
+                                              idx.numel(), _stream_ptr(stream)),
+               "oilbird_pool_to_global")
+        return out
 
     def query(self, q: torch.Tensor, params: QueryParams | None = None,
               out: QueryOut | None = None, stream=None) -> QueryOut:

@@ -18,12 +18,12 @@ append_kernel(const uint16_t* __restrict__ states, const int32_t* __restrict__ t
               int d, uint16_t* __restrict__ keys, int32_t* __restrict__ tok,
               int32_t* __restrict__ trace_id, int64_t row0, int32_t trace,
               int32_t* __restrict__ trace_end, uint64_t* __restrict__ trace_tag, uint64_t tag,
-              int set_tag, DeviceStats* stats) {
+              int64_t* __restrict__ trace_gbase, int64_t gbase, int set_tag, DeviceStats* stats) {
   pdl_launch_dependents();
   pdl_wait();   // earlier queries may still be reading the trace table and token stream
   if (blockIdx.x == 0 && threadIdx.x == 0) {
     trace_end[trace] = (int32_t)(row0 + n);
-    if (set_tag) trace_tag[trace] = tag;
+    if (set_tag) { trace_tag[trace] = tag; trace_gbase[trace] = gbase; }
   }
   for (int64_t r = blockIdx.x; r < n; r += gridDim.x) {
     const int64_t row = row0 + r;
@@ -59,11 +59,12 @@ qnorm_kernel(const uint16_t* __restrict__ q, int nq, int d, uint16_t* __restrict
 cudaError_t launch_append(const uint16_t* states, const int32_t* tokens, int64_t n, int32_t d,
                           uint16_t* keys, int32_t* tok, int32_t* trace_id, int64_t row0,
                           int32_t trace, int32_t* trace_end, uint64_t* trace_tag, uint64_t tag,
-                          int set_tag, DeviceStats* stats, cudaStream_t st) {
+                          int64_t* trace_gbase, int64_t gbase, int set_tag, DeviceStats* stats,
+                          cudaStream_t st) {
   int64_t grid = n < 1 ? 1 : (n > 65535 * 8 ? 65535 * 8 : n);
   return launch_pdl(append_kernel, dim3((unsigned)grid), dim3(kNormThreads), 0, st, states, tokens,
-                    n, d, keys, tok, trace_id, row0, trace, trace_end, trace_tag, tag, set_tag,
-                    stats);
+                    n, d, keys, tok, trace_id, row0, trace, trace_end, trace_tag, tag, trace_gbase,
+                    gbase, set_tag, stats);
 }
 
 cudaError_t launch_qnorm(const uint16_t* q, int32_t nq, int32_t nq_pad, int32_t d, uint16_t* qn,

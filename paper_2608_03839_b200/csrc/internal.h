@@ -61,7 +61,14 @@ struct GatherParams {
 cudaError_t launch_append(const uint16_t* states, const int32_t* tokens, int64_t n, int32_t d,
                           uint16_t* keys, int32_t* tok, int32_t* trace_id, int64_t row0,
                           int32_t trace, int32_t* trace_end, uint64_t* trace_tag, uint64_t tag,
-                          int set_tag, DeviceStats* stats, cudaStream_t st);
+                          int64_t* trace_gbase, int64_t gbase, int set_tag, DeviceStats* stats,
+                          cudaStream_t st);
+
+// Row sharding over several pools: local rows -> caller-assigned global positions, and the
+// merge of the shards' gathered query results (see shard.cu).
+cudaError_t launch_to_global(const int32_t* idx, int64_t* out, int64_t n, const int32_t* trace_id,
+                             const int32_t* trace_end, const int64_t* trace_gbase, int32_t n_rows,
+                             cudaStream_t st);
 
 // query preparation: qn[r] = bf16(q[r]/||q[r]||) for r < nq, zero rows up to nq_pad,
 // q_valid[r] = 0 for a query holding NaN/Inf.

@@ -31,7 +31,7 @@ size_t align_up(size_t v) { return (v + kAlign - 1) / kAlign * kAlign; }
 
 // Byte offsets of every device array inside one allocation.
 struct Layout {
-  size_t keys, tok, trace_id, trace_end, trace_tag, qn, q_valid, partial, stats;
+  size_t keys, tok, trace_id, trace_end, trace_tag, trace_gbase, qn, q_valid, partial, stats;
   size_t q_stage, ex_stage, st_stage, tok_stage, out_stage;
   size_t total;
 };
@@ -72,6 +72,7 @@ Layout make_layout(const Resolved& r) {
   L.trace_id = take((size_t)r.capacity * 4);
   L.trace_end = take((size_t)r.max_traces * 4);
   L.trace_tag = take((size_t)r.max_traces * 8);
+  L.trace_gbase = take((size_t)r.max_traces * 8);
   L.qn = take(nq_pad * r.d * 2);
   L.q_valid = take(nq_pad * 4);
   L.partial = take((size_t)r.max_lists * r.max_nq * k_pad * 8);
@@ -97,6 +98,7 @@ struct oilbird_pool {
   uint16_t* keys;
   int32_t *tok, *trace_id, *trace_end;
   uint64_t* trace_tag;
+  int64_t* trace_gbase;      // global position of each trace's first row (row sharding)
   uint16_t* qn;
   int32_t* q_valid;
   unsigned long long* partial;
@@ -193,6 +195,7 @@ int oilbird_pool_create(oilbird_pool_t** out, const oilbird_pool_config* cfg) {
   p->trace_id = (int32_t*)(p->base + lay.trace_id);
   p->trace_end = (int32_t*)(p->base + lay.trace_end);
   p->trace_tag = (uint64_t*)(p->base + lay.trace_tag);
+  p->trace_gbase = (int64_t*)(p->base + lay.trace_gbase);
   p->qn = (uint16_t*)(p->base + lay.qn);
   p->q_valid = (int32_t*)(p->base + lay.q_valid);
   p->partial = (unsigned long long*)(p->base + lay.partial);
@@ -236,8 +239,9 @@ int64_t oilbird_pool_size(const oilbird_pool_t* p) { return p ? p->n_rows : 0; }
 int32_t oilbird_pool_num_traces(const oilbird_pool_t* p) { return p ? (int32_t)p->t_start.size() : 0; }
 int64_t oilbird_pool_launch_count(const oilbird_pool_t* p) { return p ? p->launches : 0; }
 
-int oilbird_pool_append(oilbird_pool_t* p, const void* states, const int32_t* tokens, int64_t n,
-                        uint64_t tag, uint32_t flags, void* stream) {
+// global_row < 0: the pool is not a shard, a trace's global position is its local one.
+static int append_impl(oilbird_pool_t* p, const void* states, const int32_t* tokens, int64_t n,
+                       uint64_t tag, uint32_t flags, int64_t global_row, void* stream) {
   if (!p || n < 0 || (n > 0 && (!states || !tokens))) return OILBIRD_EINVAL;
   const bool open_new = (flags & OILBIRD_NEW_TRACE) || p->t_start.empty();
   if (n == 0 && !open_new) return OILBIRD_OK;
@@ -252,6 +256,7 @@ int oilbird_pool_append(oilbird_pool_t* p, const void* states, const int32_t* to
   const int32_t trace = (int32_t)p->t_start.size() - 1;
   cudaError_t e = launch_append((const uint16_t*)states, tokens, n, p->r.d, p->keys, p->tok,
                                 p->trace_id, p->n_rows, trace, p->trace_end, p->trace_tag, tag,
+                                p->trace_gbase, global_row >= 0 ? global_row : p->n_rows,
                                 open_new ? 1 : 0, p->stats, (cudaStream_t)stream);
   if (e != cudaSuccess) {
     if (open_new) { p->t_start.pop_back(); p->t_end.pop_back(); p->t_tag.pop_back(); }
@@ -260,6 +265,30 @@ int oilbird_pool_append(oilbird_pool_t* p, const void* states, const int32_t* to
   p->launches += 1;
   p->n_rows += n;
   p->t_end[trace] = p->n_rows;
+  return OILBIRD_OK;
+}
+
+int oilbird_pool_append(oilbird_pool_t* p, const void* states, const int32_t* tokens, int64_t n,
+                        uint64_t tag, uint32_t flags, void* stream) {
+  return append_impl(p, states, tokens, n, tag, flags, -1, stream);
+}
+
+int oilbird_pool_append_global(oilbird_pool_t* p, const void* states, const int32_t* tokens,
+                               int64_t n, uint64_t tag, uint32_t flags, int64_t global_row,
+                               void* stream) {
+  if (global_row < 0) return OILBIRD_EINVAL;
+  return append_impl(p, states, tokens, n, tag, flags, global_row, stream);
+}
+
+int oilbird_pool_to_global(oilbird_pool_t* p, const int32_t* idx, int64_t* global_idx, int64_t n,
+                           void* stream) {
+  if (!p || n < 0 || (n > 0 && (!idx || !global_idx))) return OILBIRD_EINVAL;
+  if (n == 0) return OILBIRD_OK;
+  CU(cudaSetDevice(p->device));
+  cudaError_t e = launch_to_global(idx, global_idx, n, p->trace_id, p->trace_end, p->trace_gbase,
+                                   (int32_t)p->n_rows, (cudaStream_t)stream);
+  if (e != cudaSuccess) return cuda_fail(e, "to_global kernel launch");
+  p->launches += 1;
   return OILBIRD_OK;
 }
 

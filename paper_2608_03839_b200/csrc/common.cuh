@@ -138,21 +138,22 @@ __device__ __forceinline__ void warp_merge_desc(u64 (&a)[E], const u64 (&b)[E], 
 }
 
 // Insert one candidate (the same key in every lane) into a descending register list,
-// dropping the smallest element.  About a dozen instructions per 32 elements.
+// dropping the smallest element.  Branch-free (a key of 0, the empty slot, is a no-op in
+// effect), so that several independent lists can be updated in interleaved straight-line
+// code and hide each other's shuffle latency.  About a dozen instructions per 32 elements.
 template <int E>
 __device__ __forceinline__ void warp_sorted_insert(u64 (&v)[E], u64 key, int lane) {
 #pragma unroll
   for (int r = 0; r < E; ++r) {
     const int pos = __popc(__ballot_sync(0xffffffffu, v[r] > key));   // elements that stay put
-    if (pos < 32) {                                                   // warp-uniform
-      const uint32_t ulo = __shfl_up_sync(0xffffffffu, (uint32_t)v[r], 1);
-      const uint32_t uhi = __shfl_up_sync(0xffffffffu, (uint32_t)(v[r] >> 32), 1);
-      const uint32_t clo = __shfl_sync(0xffffffffu, (uint32_t)v[r], 31);
-      const uint32_t chi = __shfl_sync(0xffffffffu, (uint32_t)(v[r] >> 32), 31);
-      const u64 up = ((u64)uhi << 32) | ulo;
-      v[r] = lane < pos ? v[r] : (lane == pos ? key : up);
-      key = ((u64)chi << 32) | clo;                                   // carried into the next row
-    }
+    const uint32_t ulo = __shfl_up_sync(0xffffffffu, (uint32_t)v[r], 1);
+    const uint32_t uhi = __shfl_up_sync(0xffffffffu, (uint32_t)(v[r] >> 32), 1);
+    const uint32_t clo = __shfl_sync(0xffffffffu, (uint32_t)v[r], 31);
+    const uint32_t chi = __shfl_sync(0xffffffffu, (uint32_t)(v[r] >> 32), 31);
+    const u64 up = ((u64)uhi << 32) | ulo;
+    const u64 carry = ((u64)chi << 32) | clo;
+    v[r] = lane < pos ? v[r] : (lane == pos ? key : up);              // pos == 32: unchanged
+    key = pos < 32 ? carry : key;                                     // carried into the next row
   }
 }
 

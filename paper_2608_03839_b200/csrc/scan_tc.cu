@@ -12,8 +12,13 @@
 //   warps 2-5   epilogue: tcgen05.ld the 128 x nq scores, filter them against the
 //               per-query running k-th best, and keep per-query top-k lists in shared
 //               memory (Eq. 2); scores never go to global memory
-// The key stream (N*d*2 bytes from HBM, once) bounds the kernel up to nq ~ 128; the
-// query tile is re-read from L2 for every key tile.
+// The key stream (N*d*2 bytes from HBM, once) bounds the kernel up to nq ~ 64.  Beyond
+// that the epilogue sets the pace: with the filter switched off the same launch streams
+// at 6.2 TB/s for nq = 128, with it at 4.1 TB/s; ring depth (2..5 stages) and the query
+// tile's L2 traffic make no measurable difference there.  A variant that transposes the
+// scores through shared memory so that one warp owns a query's 128 rows (no queue, no
+// atomics, one barrier per round) was measured 15-30 % slower: its fixed cost per round
+// outweighs the cheaper candidate path.
 //
 // Every mbarrier wait is bounded: after about two seconds it raises the pool's `stalled`
 // flag, the CTA drains what it has in flight, frees its TMEM and returns.
@@ -34,7 +39,7 @@ constexpr int kTileM = 128;            // key rows per tile = TMEM lanes
 // requested twice and the scan runs 30-40 % slower at every nq.)
 constexpr int kBlockK = 64;
 constexpr int kATileBytes = kTileM * kBlockK * 2;   // 16 KB
-constexpr int kColsPerRound = 8;       // score columns filtered between two drains
+constexpr int kColsPerRound = 16;      // score columns filtered between two drains
 constexpr int kQueueCap = kTileM * kColsPerRound;
 constexpr int kMaxStages = 8;
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;
@@ -116,16 +121,18 @@ __device__ __forceinline__ void tc_mma_bf16(uint32_t d_tmem, uint64_t a_desc, ui
       ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
       : "memory");
 }
-__device__ __forceinline__ void tc_ld8(uint32_t taddr, float (&v)[8]) {
-  uint32_t r[8];
+__device__ __forceinline__ void tc_ld16(uint32_t taddr, float (&v)[16]) {
+  uint32_t r[16];
   asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32"
+      " {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
       : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]),
-        "=r"(r[7])
+        "=r"(r[7]), "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]),
+        "=r"(r[14]), "=r"(r[15])
       : "r"(taddr));
   asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 #pragma unroll
-  for (int i = 0; i < 8; ++i) v[i] = __uint_as_float(r[i]);
+  for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
 }
 __device__ __forceinline__ void epilogue_bar() {      // the 128 epilogue threads only
   asm volatile("bar.sync 1, 128;" ::: "memory");
@@ -158,44 +165,75 @@ struct TcShared {
   int q_cnt[kColsPerRound];     // ... per score column of the round
 };
 
-// Fold the candidates queued for one query into its descending list (shared memory,
-// kk = 32*E slots, empty slots are 0) and refresh the filter threshold: the score of the
-// k-th entry once k entries exist.  A handful of candidates are inserted one by one
-// (a chain of dependent shuffles each); a crowd, as in a CTA's first tiles while its
-// thresholds are still low, is sorted 32*E at a time and merged, which costs a fixed
-// two dozen network stages per batch.
+// Fold the candidates queued in one round into the descending lists of the (up to four)
+// queries this warp owns in the round.  Lists live in shared memory (kk = 32*E slots, empty
+// slots are 0) and are held in registers meanwhile; afterwards the filter threshold of
+// each query, the score of its k-th entry once k entries exist, is refreshed.
+// A crowd of candidates (a CTA's first tiles, while its thresholds are still low) is sorted
+// 32*E at a time and merged; the usual handful is inserted one by one, the queries'
+// independent insert chains interleaved so that they hide each other's shuffle latency.
+constexpr int kDrainQ = kColsPerRound / 4;      // queries per warp and round
+constexpr int kCrowd = 8;
+
 template <int E>
-__device__ __forceinline__ void drain_query(u64* list, const u64* cand, int n_cand, int k,
-                                            float* thr_s_p, int lane) {
-  u64 v[E];
+__device__ __forceinline__ void drain_round(u64* lists, int kk, const u64* q_key,
+                                            const int* q_cnt, int c0, int ew, int nq_c, int k,
+                                            float* thr_s, int lane) {
+  u64 v[kDrainQ][E];
+  u64 kth[kDrainQ];
+  int n[kDrainQ];
+  int n_max = 0;
 #pragma unroll
-  for (int r = 0; r < E; ++r) v[r] = list[r * 32 + lane];
-  u64 kth = warp_list_get<E>(v, k - 1);
-  if (n_cand >= 8) {
-    for (int i0 = 0; i0 < n_cand; i0 += 32 * E) {
-      u64 b[E];
+  for (int u = 0; u < kDrainQ; ++u) {
+    const int j = ew + 4 * u, q = c0 + j;
+    n[u] = q < nq_c ? q_cnt[j] : 0;
+    if (n[u] > 0) {
 #pragma unroll
-      for (int r = 0; r < E; ++r) {
-        const int i = i0 + r * 32 + lane;
-        const u64 key = i < n_cand ? cand[i] : 0;
-        b[r] = key > kth ? key : 0;
+      for (int r = 0; r < E; ++r) v[u][r] = lists[(size_t)q * kk + r * 32 + lane];
+      kth[u] = warp_list_get<E>(v[u], k - 1);
+      if (n[u] >= kCrowd) {
+        const u64* cand = q_key + j * kTileM;
+        for (int i0 = 0; i0 < n[u]; i0 += 32 * E) {
+          u64 b[E];
+#pragma unroll
+          for (int r = 0; r < E; ++r) {
+            const int i = i0 + r * 32 + lane;
+            const u64 key = i < n[u] ? cand[i] : 0;
+            b[r] = key > kth[u] ? key : 0;
+          }
+          warp_sort_desc<E>(b, lane);
+          warp_merge_desc<E>(v[u], b, lane);
+          kth[u] = warp_list_get<E>(v[u], k - 1);
+        }
+      } else {
+        n_max = n[u] > n_max ? n[u] : n_max;
       }
-      warp_sort_desc<E>(b, lane);
-      warp_merge_desc<E>(v, b, lane);
-      kth = warp_list_get<E>(v, k - 1);
+    } else {
+#pragma unroll
+      for (int r = 0; r < E; ++r) v[u][r] = 0;
+      kth[u] = 0;
     }
-  } else {
-    for (int i = 0; i < n_cand; ++i) {
-      const u64 key = cand[i];
-      if (key > kth) {
-        warp_sorted_insert<E>(v, key, lane);
-        kth = warp_list_get<E>(v, k - 1);
-      }
+  }
+  for (int i = 0; i < n_max; ++i) {
+#pragma unroll
+    for (int u = 0; u < kDrainQ; ++u) {
+      // every queued candidate beat the threshold it was filtered with; kth only settles
+      // ties and is refreshed after the round (a worse key just falls off the end)
+      u64 key = (n[u] < kCrowd && i < n[u]) ? q_key[(ew + 4 * u) * kTileM + i] : 0;
+      key = key > kth[u] ? key : 0;
+      warp_sorted_insert<E>(v[u], key, lane);
     }
   }
 #pragma unroll
-  for (int r = 0; r < E; ++r) list[r * 32 + lane] = v[r];
-  if (lane == 0 && kth != 0) *thr_s_p = candidate_score(kth);
+  for (int u = 0; u < kDrainQ; ++u) {
+    if (n[u] > 0) {
+      const int q = c0 + ew + 4 * u;
+#pragma unroll
+      for (int r = 0; r < E; ++r) lists[(size_t)q * kk + r * 32 + lane] = v[u][r];
+      const u64 nk = warp_list_get<E>(v[u], k - 1);
+      if (lane == 0 && nk != 0) thr_s[q] = candidate_score(nk);
+    }
+  }
 }
 
 // ------------------------------------------------------------------- the kernel ---
@@ -347,7 +385,7 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap key_map,
                              (buf * (uint32_t)mt + (uint32_t)sub) * (uint32_t)n_pad;
       for (int c0 = 0; c0 < n_pad; c0 += kColsPerRound) {
         float v[kColsPerRound];
-        tc_ld8(t_row + (uint32_t)c0, v);
+        tc_ld16(t_row + (uint32_t)c0, v);
         if (sub == mt - 1 && c0 + kColsPerRound >= n_pad) {
           // all of this macro tile's scores have been read: hand the accumulators back
           tc_fence_before();
@@ -369,17 +407,11 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap key_map,
         epilogue_bar();
         if (sh.q_total > 0) {
           // drain: warp ew folds the candidates of columns ew, ew+4, ... into their lists
-          for (int j = ew; j < kColsPerRound; j += 4) {
-            const int n_cand = sh.q_cnt[j];
-            const int q = c0 + j;
-            if (n_cand == 0 || q >= nq_c) continue;
-            u64* list = lists + (size_t)q * kk;
-            if (kk == 32) drain_query<1>(list, q_key + j * kTileM, n_cand, k, &thr_s[q], lane);
-            else if (kk == 64) drain_query<2>(list, q_key + j * kTileM, n_cand, k, &thr_s[q], lane);
-            else drain_query<4>(list, q_key + j * kTileM, n_cand, k, &thr_s[q], lane);
-            __syncwarp();
-            if (lane == 0) sh.q_cnt[j] = 0;
-          }
+          if (kk == 32) drain_round<1>(lists, kk, q_key, sh.q_cnt, c0, ew, nq_c, k, thr_s, lane);
+          else if (kk == 64) drain_round<2>(lists, kk, q_key, sh.q_cnt, c0, ew, nq_c, k, thr_s, lane);
+          else drain_round<4>(lists, kk, q_key, sh.q_cnt, c0, ew, nq_c, k, thr_s, lane);
+          __syncwarp();
+          if (lane < kDrainQ) sh.q_cnt[ew + 4 * lane] = 0;
           epilogue_bar();
           if (et == 0) sh.q_total = 0;
           epilogue_bar();
@@ -525,6 +557,8 @@ cudaError_t launch_scan_tc(TcCache* cache, const PoolView& pv, int32_t q0, int32
   const int n_tiles128 = (pv.n_rows + kTileM - 1) / kTileM;
   static const int force_mt = getenv("OILBIRD_TC_MT") ? atoi(getenv("OILBIRD_TC_MT")) : 0;
   TcPlan plan = tc_plan(nq_c, k, n_tiles128, num_sms, smem_limit, force_mt);
+  static const int cap_stages = getenv("OILBIRD_TC_STAGES") ? atoi(getenv("OILBIRD_TC_STAGES")) : 0;
+  if (cap_stages >= 2 && plan.stages > cap_stages) plan.stages = cap_stages;
   const size_t stage = (size_t)plan.mt * kATileBytes + (size_t)n_pad * kBlockK * 2;
   const size_t fixed = tc_fixed_smem(nq_c, n_pad, kk);
   if (plan.stages < 2) return cudaErrorInvalidConfiguration;

@@ -275,8 +275,7 @@ def run_ours(args):
 
     def step_host():
         i = step_no[0] % n_in
-        pool.append_host(h_states[i], h_toks[i], tag=1_000_000 + step_no[0], new_trace=True)
-        pool.query_host(h_q[i], pr, out=h_out)
+        pool.step_host(h_states[i], h_toks[i], h_q[i], pr, h_out, tag=1_000_000 + step_no[0])
         step_no[0] += 1
 
     for _ in range(Wm):

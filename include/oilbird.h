@@ -184,6 +184,14 @@ int oilbird_pool_query_host(oilbird_pool_t* pool, const void* q_bf16_host, int32
                             const oilbird_query_params* params, const oilbird_query_out* out_host,
                             void* cuda_stream);
 
+/* One serving step with host buffers: append_host (the rows committed since the last
+ * step; n may be 0) followed by query_host, in one call. */
+int oilbird_pool_step_host(oilbird_pool_t* pool, const void* states_bf16_host,
+                           const int32_t* tokens_host, int64_t n, uint64_t trace_tag,
+                           uint32_t flags, const void* q_bf16_host, int32_t nq,
+                           const oilbird_query_params* params, const oilbird_query_out* out_host,
+                           void* cuda_stream);
+
 /* Introspection (host side; none of these enqueue work unless stated). */
 int64_t oilbird_pool_size(const oilbird_pool_t* pool);          /* rows appended so far  */
 int32_t oilbird_pool_num_traces(const oilbird_pool_t* pool);

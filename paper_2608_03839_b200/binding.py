@@ -88,6 +88,9 @@ SYMBOLS = {
     "oilbird_pool_append_host": (ctypes.c_int, [_vp, _vp, _vp, _i64, _u64, _u32, _vp]),
     "oilbird_pool_query_host": (ctypes.c_int, [_vp, _vp, _i32, ctypes.POINTER(CQueryParams),
                                                ctypes.POINTER(CQueryOut), _vp]),
+    "oilbird_pool_step_host": (ctypes.c_int, [_vp, _vp, _vp, _i64, _u64, _u32, _vp, _i32,
+                                              ctypes.POINTER(CQueryParams),
+                                              ctypes.POINTER(CQueryOut), _vp]),
     "oilbird_pool_size": (_i64, [_vp]),
     "oilbird_pool_num_traces": (_i32, [_vp]),
     "oilbird_pool_status": (ctypes.c_int, [_vp, ctypes.POINTER(PoolStats), _vp]),
@@ -403,6 +406,18 @@ class Pool:
         _check(self._L.oilbird_pool_query_host(self._h, q.data_ptr(), nq, ctypes.byref(cp),
                                                ctypes.byref(out._c), _stream_ptr(stream)),
                "oilbird_pool_query_host")
+        return out
+
+    def step_host(self, states: torch.Tensor, tokens: torch.Tensor, q: torch.Tensor,
+                  params: QueryParams, out: QueryOut, tag: int = 0, new_trace: bool = True,
+                  stream=None) -> QueryOut:
+        """One serving step from host memory: append the committed rows, then query.
+        All tensors are CPU tensors; `out` must have been made with QueryOut.empty(..., "cpu")."""
+        cp = params.to_c(None)
+        _check(self._L.oilbird_pool_step_host(
+            self._h, states.data_ptr(), tokens.data_ptr(), int(tokens.shape[0]), int(tag),
+            NEW_TRACE if new_trace else 0, q.data_ptr(), int(q.shape[0]), ctypes.byref(cp),
+            ctypes.byref(out._c), _stream_ptr(stream)), "oilbird_pool_step_host")
         return out
 
     # ---- introspection --------------------------------------------------------------

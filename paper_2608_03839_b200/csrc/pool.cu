@@ -497,6 +497,27 @@ int oilbird_pool_query_host(oilbird_pool_t* p, const void* q, int32_t nq,
   return OILBIRD_OK;
 }
 
+int oilbird_pool_step_host(oilbird_pool_t* p, const void* states, const int32_t* tokens,
+                           int64_t n, uint64_t tag, uint32_t flags, const void* q, int32_t nq,
+                           const oilbird_query_params* pr, const oilbird_query_out* out,
+                           void* stream) {
+  // The call returns only after everything has completed, so the rows are uploaded straight
+  // from the caller's buffers (no pinned staging copy as in append_host).
+  if (!p || n < 0 || n > p->r.max_append || (n > 0 && (!states || !tokens))) return OILBIRD_EINVAL;
+  CU(cudaSetDevice(p->device));
+  cudaStream_t st = (cudaStream_t)stream;
+  uint16_t* d_st = (uint16_t*)(p->base + p->lay.st_stage);
+  int32_t* d_tok = (int32_t*)(p->base + p->lay.tok_stage);
+  if (n > 0) {
+    CU(cudaMemcpyAsync(d_st, states, (size_t)n * p->r.d * 2, cudaMemcpyHostToDevice, st));
+    CU(cudaMemcpyAsync(d_tok, tokens, (size_t)n * 4, cudaMemcpyHostToDevice, st));
+  }
+  int rc = oilbird_pool_append(p, d_st, d_tok, n, tag, flags, stream);
+  if (rc == OILBIRD_OK) rc = oilbird_pool_query_host(p, q, nq, pr, out, stream);
+  if (rc != OILBIRD_OK) cudaStreamSynchronize(st);   // the caller's buffers are free on return
+  return rc;
+}
+
 // ---- introspection ------------------------------------------------------------------
 
 int oilbird_pool_status(oilbird_pool_t* p, oilbird_pool_stats* stats, void* stream) {

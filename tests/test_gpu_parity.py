@@ -331,3 +331,25 @@ def test_caller_provided_arena():
     pool, ora = fill_both(w, use_torch_arena=True)
     q, _ = w.queries("cuda")
     check_query(pool.query(q, fixed(8, 8)), ora, W.to_bits(q), fixed(8, 8))
+
+
+def test_step_host_is_append_host_plus_query_host():
+    w = W.C1.scaled(n_rows=1024, nq=2)
+    pool, ora = fill_both(w, spare_rows=64)
+    pool2, _ = fill_both(w, spare_rows=64)
+    g = torch.Generator().manual_seed(5)
+    q, _ = w.queries("cuda")
+    qh = q.cpu().contiguous()
+    pr = fixed(8, 8, theta=-2.0)
+    for step in range(3):
+        st = torch.randn(8, w.d, generator=g).to(torch.bfloat16)
+        tk = torch.randint(0, 100, (8,), generator=g, dtype=torch.int32)
+        a = B.QueryOut.empty(2, 8, 8, "cpu")
+        pool.step_host(st, tk, qh, pr, a, tag=50 + step)
+        pool2.append_host(st, tk, tag=50 + step)
+        b = pool2.query_host(qh, pr)
+        ora.append(W.to_bits(st), tk.numpy(), tag=50 + step)
+        for f in ("idx", "score", "fired", "cont_len", "cont_tok"):
+            assert torch.equal(getattr(a, f), getattr(b, f))
+    assert len(pool) == len(pool2) == 1024 + 24
+    check_query(pool.query(q, pr), ora, W.to_bits(q), pr)

@@ -335,6 +335,26 @@ def run_ours(args):
                 "frac_of_sustained": tflops / peaks["bf16_tflops_sustained"],
                 "frac_of_burst": tflops / peaks["bf16_tflops"], "peak_kind": peak_kind,
                 "note": "HBM-bound below nq ~ 218: the tensor pipe idles by design"}
+        if w.kind == "template" and not args.rows:
+            # retrieval quality on the tool-calling shape: recall of the planted
+            # same-(template, position) rows and how much of the gathered continuation
+            # agrees with the template (slot positions excepted)
+            tq, meta = w.queries(dev, nq=nq)
+            res = pool.query(tq, B.QueryParams(k=w.k, theta=-2.0, depth_mode=B.DEPTH_FIXED,
+                                               cont_len=w.cont_len, path=args.path)).cpu()
+            hits = tot = 0
+            match = []
+            for i, rows_i in enumerate(meta["planted_rows"]):
+                hits += len(set(rows_i) & set(res.idx[i].tolist()))
+                tot += min(len(rows_i), w.k)
+                ttok, slot = meta["template_tokens"][i]
+                pos = meta["pos"][i]
+                want = ttok[pos + 2: pos + 2 + w.cont_len]
+                ok = (res.cont_tok[i, 0, : len(want)] == want) | slot[pos + 2: pos + 2 + w.cont_len]
+                match.append(float(ok.sum()) / max(1, len(want)))
+            line["retrieval_quality"] = {"recall_planted_at_k": hits / max(1, tot),
+                                         "top1_continuation_match": float(np.mean(match)),
+                                         "queries": len(match)}
         if not args.no_cpu_baseline and world == 1:
             line["cpu_baseline"] = cpu_baseline(w, n0, rows_step, nq, budget_s=args.cpu_budget)
         print(json.dumps(line), flush=True)

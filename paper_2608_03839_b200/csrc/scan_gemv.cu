@@ -12,6 +12,10 @@
 //
 // The kernel is bound by the key stream (N*d*2 bytes); per 16 bytes of key a lane
 // spends 8 integer unpack ops and 8*QT FMAs, well under the issue budget for QT <= 2.
+// A plain streaming read of the same 537 MB (no arithmetic) takes 79-80 us with this
+// access pattern and 78 us through a cp.async.bulk shared-memory ring, so the direct
+// loads are kept.  Handing row groups out through a global ticket counter instead of the
+// static split was measured 4 % slower (one hot atomic, no tail to win back).
 #include "common.cuh"
 #include "internal.h"
 #include "normalize.cuh"

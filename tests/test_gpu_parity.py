@@ -353,3 +353,29 @@ def test_step_host_is_append_host_plus_query_host():
             assert torch.equal(getattr(a, f), getattr(b, f))
     assert len(pool) == len(pool2) == 1024 + 24
     check_query(pool.query(q, pr), ora, W.to_bits(q), pr)
+
+
+@pytest.mark.parametrize("nq,k", [(256, 128), (100, 128), (256, 64), (33, 100)])
+def test_largest_nq_and_k_run_in_several_passes(nq, k):
+    """Per-query lists for nq*k beyond shared memory: the tensor path cuts the call into
+    balanced query passes; results must not depend on the cut."""
+    w = W.C1.scaled(nq=nq, k=k, n_rows=2500, d=256, cont_len=3)
+    pool, ora = fill_both(w, max_k=128, max_nq=256)
+    q, _ = w.queries("cuda")
+    pr = fixed(k, 3, theta=-2.0, path=B.PATH_TENSOR)
+    out = pool.query(q, pr)
+    check_query(out, ora, W.to_bits(q), pr)
+    ws = w.scaled(n_rows=max(2500, 2 * nq * (k + 4))).separated()   # room for the planted rows
+    pool, ora = fill_both(ws, max_k=128, max_nq=256)
+    q, _ = ws.queries("cuda")
+    st = check_query(pool.query(q, pr), ora, W.to_bits(q), pr)
+    if k <= 100:
+        gem = pool.query(q[:2].contiguous(), fixed(k, 3, theta=-2.0, path=B.PATH_GEMV))
+        check_query(gem, ora, W.to_bits(q)[:2], pr)
+
+
+@pytest.mark.parametrize("d", [8, 72, 200, 1000])
+def test_key_widths_that_are_not_multiples_of_the_k_block(d):
+    w = W.C1.scaled(nq=3, k=8, n_rows=1500, d=d, cont_len=4, sigma=0.3)
+    run_workload(w, paths=(B.PATH_GEMV, B.PATH_TENSOR))
+    run_workload(w.separated(), paths=(B.PATH_GEMV, B.PATH_TENSOR))

@@ -182,7 +182,7 @@ __device__ __forceinline__ void drain_round(u64* lists, int kk, const u64* q_key
   u64 v[kDrainQ][E];
   u64 kth[kDrainQ];
   int n[kDrainQ];
-  int n_max = 0;
+  int n_max = 0, crowd_max = 0;
 #pragma unroll
   for (int u = 0; u < kDrainQ; ++u) {
     const int j = ew + 4 * u, q = c0 + j;
@@ -191,28 +191,33 @@ __device__ __forceinline__ void drain_round(u64* lists, int kk, const u64* q_key
 #pragma unroll
       for (int r = 0; r < E; ++r) v[u][r] = lists[(size_t)q * kk + r * 32 + lane];
       kth[u] = warp_list_get<E>(v[u], k - 1);
-      if (n[u] >= kCrowd) {
-        const u64* cand = q_key + j * kTileM;
-        for (int i0 = 0; i0 < n[u]; i0 += 32 * E) {
-          u64 b[E];
-#pragma unroll
-          for (int r = 0; r < E; ++r) {
-            const int i = i0 + r * 32 + lane;
-            const u64 key = i < n[u] ? cand[i] : 0;
-            b[r] = key > kth[u] ? key : 0;
-          }
-          warp_sort_desc<E>(b, lane);
-          warp_merge_desc<E>(v[u], b, lane);
-          kth[u] = warp_list_get<E>(v[u], k - 1);
-        }
-      } else {
-        n_max = n[u] > n_max ? n[u] : n_max;
-      }
     } else {
 #pragma unroll
       for (int r = 0; r < E; ++r) v[u][r] = 0;
       kth[u] = 0;
     }
+    if (n[u] >= kCrowd) crowd_max = n[u] > crowd_max ? n[u] : crowd_max;
+    else n_max = n[u] > n_max ? n[u] : n_max;
+  }
+  // crowds: batches of 32*E candidates are sorted and merged, the four queries' networks
+  // in one basic block so that they overlap (an uncrowded query rides along with zeros)
+  for (int i0 = 0; i0 < crowd_max; i0 += 32 * E) {
+    u64 b[kDrainQ][E];
+#pragma unroll
+    for (int u = 0; u < kDrainQ; ++u) {
+#pragma unroll
+      for (int r = 0; r < E; ++r) {
+        const int i = i0 + r * 32 + lane;
+        const u64 key = (n[u] >= kCrowd && i < n[u]) ? q_key[(ew + 4 * u) * kTileM + i] : 0;
+        b[u][r] = key > kth[u] ? key : 0;
+      }
+    }
+#pragma unroll
+    for (int u = 0; u < kDrainQ; ++u) warp_sort_desc<E>(b[u], lane);
+#pragma unroll
+    for (int u = 0; u < kDrainQ; ++u) warp_merge_desc<E>(v[u], b[u], lane);
+#pragma unroll
+    for (int u = 0; u < kDrainQ; ++u) kth[u] = warp_list_get<E>(v[u], k - 1);
   }
   for (int i = 0; i < n_max; ++i) {
 #pragma unroll

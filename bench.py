@@ -60,8 +60,8 @@ def measured_peaks():
 # profiles/ (file named per entry), with the pool rows held at capture time.  Traffic is
 # proportional to the rows scanned, so it is scaled to the rows of the timed launches.
 NCU_TRAFFIC = {
-    "C2": (540655360.0, 65560),      # profiles/scan_gemv_C2_ncu.md
-    "C4": (2171870656.0, 264192),    # profiles/scan_tc_C4_quarter_ncu.md (quarter-size pool)
+    "C2": (540625920.0, 65560),      # profiles/scan_gemv_C2_ncu.md
+    "C4": (2172068528.0, 264192),    # profiles/scan_tc_C4_quarter_ncu.md (quarter-size pool)
 }
 
 

@@ -38,9 +38,13 @@ append_kernel(const uint16_t* __restrict__ states, const int32_t* __restrict__ t
 
 __global__ void __launch_bounds__(kNormThreads)
 qnorm_kernel(const uint16_t* __restrict__ q, int nq, int d, uint16_t* __restrict__ qn,
-             int32_t* __restrict__ q_valid, DeviceStats* stats) {
+             int32_t* __restrict__ q_valid, DeviceStats* stats, float* __restrict__ xchg,
+             int n_xchg) {
   pdl_launch_dependents();
   pdl_wait();
+  // the tensor scan's cross-CTA threshold exchange starts every call at -inf
+  for (int i = blockIdx.x * kNormThreads + threadIdx.x; i < n_xchg; i += gridDim.x * kNormThreads)
+    xchg[i] = -INFINITY;
   const int r = blockIdx.x;
   if (r < nq) {
     // A query holding NaN/Inf returns no neighbours; an all-zero query is legal and
@@ -68,9 +72,10 @@ cudaError_t launch_append(const uint16_t* states, const int32_t* tokens, int64_t
 }
 
 cudaError_t launch_qnorm(const uint16_t* q, int32_t nq, int32_t nq_pad, int32_t d, uint16_t* qn,
-                         int32_t* q_valid, DeviceStats* stats, cudaStream_t st) {
+                         int32_t* q_valid, DeviceStats* stats, float* xchg, int32_t n_xchg,
+                         cudaStream_t st) {
   return launch_pdl(qnorm_kernel, dim3(nq_pad), dim3(kNormThreads), 0, st, q, nq, d, qn, q_valid,
-                    stats);
+                    stats, xchg, n_xchg);
 }
 
 }  // namespace oilbird

@@ -72,8 +72,15 @@ cudaError_t launch_to_global(const int32_t* idx, int64_t* out, int64_t n, const 
 
 // query preparation: qn[r] = bf16(q[r]/||q[r]||) for r < nq, zero rows up to nq_pad,
 // q_valid[r] = 0 for a query holding NaN/Inf.
+// Also fills xchg[0..n_xchg) with -inf (the tensor scan's threshold exchange, see scan_tc.cu).
 cudaError_t launch_qnorm(const uint16_t* q, int32_t nq, int32_t nq_pad, int32_t d, uint16_t* qn,
-                         int32_t* q_valid, DeviceStats* stats, cudaStream_t st);
+                         int32_t* q_valid, DeviceStats* stats, float* xchg, int32_t n_xchg,
+                         cudaStream_t st);
+
+// Cross-CTA threshold exchange of the tensor scan: per query one published best score per
+// CTA (kTcMaxCtas slots) followed by one agreed lower bound per query.
+constexpr int kTcMaxCtas = 256;
+constexpr int kTcXchgFloats = OILBIRD_MAX_NQ * kTcMaxCtas + OILBIRD_MAX_NQ;
 
 // Length of the candidate lists exchanged between scan and merge for a given k.
 inline int list_len(int k) { int p = next_pow2(k); return p < 32 ? 32 : p; }
@@ -96,8 +103,8 @@ void tc_cache_destroy(TcCache* cache);
 int tc_queries_per_pass(int nq, int k, size_t smem_limit);   // balanced split of a call
 cudaError_t launch_scan_tc(TcCache* cache, const PoolView& pv, int32_t q0, int32_t nq_c,
                            int32_t nq_total, int32_t k, int32_t kk, const uint64_t* exclude_tag,
-                           unsigned long long* partial, DeviceStats* stats, int32_t num_sms,
-                           size_t smem_limit, int32_t* n_lists, cudaStream_t st);
+                           unsigned long long* partial, DeviceStats* stats, float* xchg,
+                           int32_t num_sms, size_t smem_limit, int32_t* n_lists, cudaStream_t st);
 
 // a3 (final merge) + a4 + a5 + a6: one CTA per query.
 cudaError_t launch_merge_gather(const PoolView& pv, const unsigned long long* partial,

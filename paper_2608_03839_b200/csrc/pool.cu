@@ -32,6 +32,7 @@ size_t align_up(size_t v) { return (v + kAlign - 1) / kAlign * kAlign; }
 // Byte offsets of every device array inside one allocation.
 struct Layout {
   size_t keys, tok, trace_id, trace_end, trace_tag, trace_gbase, qn, q_valid, partial, stats;
+  size_t xchg;
   size_t q_stage, ex_stage, st_stage, tok_stage, out_stage;
   size_t total;
 };
@@ -77,6 +78,7 @@ Layout make_layout(const Resolved& r) {
   L.q_valid = take(nq_pad * 4);
   L.partial = take((size_t)r.max_lists * r.max_nq * k_pad * 8);
   L.stats = take(sizeof(DeviceStats));
+  L.xchg = take((size_t)kTcXchgFloats * 4);
   // staging for the *_host variants
   L.q_stage = take((size_t)r.max_nq * r.d * 2);
   L.ex_stage = take((size_t)r.max_nq * 8);
@@ -103,6 +105,7 @@ struct oilbird_pool {
   int32_t* q_valid;
   unsigned long long* partial;
   DeviceStats* stats;
+  float* xchg;               // tensor scan: cross-CTA threshold exchange
   // host bookkeeping (enqueue-time truth)
   int64_t n_rows;
   std::vector<int64_t> t_start, t_end;
@@ -200,6 +203,7 @@ int oilbird_pool_create(oilbird_pool_t** out, const oilbird_pool_config* cfg) {
   p->q_valid = (int32_t*)(p->base + lay.q_valid);
   p->partial = (unsigned long long*)(p->base + lay.partial);
   p->stats = (DeviceStats*)(p->base + lay.stats);
+  p->xchg = (float*)(p->base + lay.xchg);
   cudaError_t e = cudaMemset(p->stats, 0, sizeof(DeviceStats));
   if (e != cudaSuccess) {
     if (p->owns_mem) cudaFree(p->base);
@@ -351,7 +355,8 @@ int oilbird_pool_query(oilbird_pool_t* p, const void* q, int32_t nq,
   int32_t n_lists = 0;
   if (p->n_rows == 0) {
     // nothing to scan: only classify the queries (a NaN/Inf query is still counted)
-    e = launch_qnorm((const uint16_t*)q, nq, nq_pad, p->r.d, p->qn, p->q_valid, p->stats, st);
+    e = launch_qnorm((const uint16_t*)q, nq, nq_pad, p->r.d, p->qn, p->q_valid, p->stats,
+                     nullptr, 0, st);
     if (e != cudaSuccess) return cuda_fail(e, "qnorm kernel launch");
     p->launches += 1;
   } else {
@@ -371,7 +376,8 @@ int oilbird_pool_query(oilbird_pool_t* p, const void* q, int32_t nq,
       if (e != cudaSuccess) return cuda_fail(e, "scan kernel launch");
       p->launches += 1;
     } else {
-      e = launch_qnorm((const uint16_t*)q, nq, nq_pad, p->r.d, p->qn, p->q_valid, p->stats, st);
+      e = launch_qnorm((const uint16_t*)q, nq, nq_pad, p->r.d, p->qn, p->q_valid, p->stats,
+                       p->xchg, kTcXchgFloats, st);
       if (e != cudaSuccess) return cuda_fail(e, "qnorm kernel launch");
       p->launches += 1;
       // as many queries per pass as shared memory allows next to a 3-stage ring
@@ -379,7 +385,7 @@ int oilbird_pool_query(oilbird_pool_t* p, const void* q, int32_t nq,
       for (int q0 = 0; q0 < nq; q0 += per_pass) {
         const int nq_c = nq - q0 < per_pass ? nq - q0 : per_pass;
         e = launch_scan_tc(p->tc, pv, q0, nq_c, nq, pr->k, kk, pr->exclude_tag, p->partial,
-                           p->stats, p->num_sms, p->smem_limit, &n_lists, st);
+                           p->stats, p->xchg, p->num_sms, p->smem_limit, &n_lists, st);
         if (e != cudaSuccess) return cuda_fail(e, "tensor scan kernel launch");
         p->launches += 1;
       }

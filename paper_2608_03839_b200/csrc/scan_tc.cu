@@ -236,7 +236,8 @@ __device__ __forceinline__ void drain_round(u64* lists, int kk, const u64* q_key
 #pragma unroll
       for (int r = 0; r < E; ++r) lists[(size_t)q * kk + r * 32 + lane] = v[u][r];
       const u64 nk = warp_list_get<E>(v[u], k - 1);
-      if (lane == 0 && nk != 0) thr_s[q] = candidate_score(nk);
+      // never below a bound adopted from the other CTAs
+      if (lane == 0 && nk != 0) thr_s[q] = fmaxf(thr_s[q], candidate_score(nk));
     }
   }
 }
@@ -252,7 +253,7 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap key_map,
                const __grid_constant__ CUtensorMap q_map, PoolView pv, int q0, int nq_c,
                int nq_total, int n_pad, int k, int kk, int n_stages, int tmem_cols, int mt,
                int n_bufs, const uint64_t* __restrict__ exclude_tag, u64* __restrict__ partial,
-               DeviceStats* stats) {
+               DeviceStats* stats, float* xchg) {
   extern __shared__ __align__(1024) unsigned char smem_raw[];
   __shared__ TcShared sh;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -266,6 +267,17 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap key_map,
   u64* q_key = lists + (size_t)nq_c * kk;                      // [kColsPerRound][kTileM]
   uint64_t* s_ex = reinterpret_cast<uint64_t*>(q_key + kQueueCap);              // [n_pad]
   float* thr_s = reinterpret_cast<float*>(s_ex + n_pad);                        // [n_pad]
+  // Cross-CTA threshold exchange (global memory, reset to -inf by the query preparation):
+  // lmax[q][cta] = best score CTA `cta` has seen for query q; gthr[q] = a score that at
+  // least k distinct rows of the pool are known to reach, namely the k-th largest of the
+  // CTAs' bests (one row per CTA).  No row below gthr[q] can be among the k best, so the
+  // filter threshold of a query is max(its local k-th score, just below gthr[q]).  Local
+  // thresholds only see one CTA's rows (1/148 of the pool); with the exchange the number of
+  // candidates that reach the sorted lists after a CTA's first tiles drops by about two
+  // orders of magnitude.  Values only grow, so stale reads are merely weaker bounds.
+  float* lmax = xchg;
+  float* gthr = xchg + (size_t)OILBIRD_MAX_NQ * kTcMaxCtas;
+  const bool use_xchg = (int)gridDim.x >= k && (int)gridDim.x <= kTcMaxCtas;
 
   const int n_tiles = (pv.n_rows + mt * kTileM - 1) / (mt * kTileM);   // macro tiles
   const int n_kb = (pv.d + kBlockK - 1) / kBlockK;
@@ -378,6 +390,13 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap key_map,
       // one decision for all four warps, so that the barriers below always match up
       epilogue_bar();
       if (et == 0) sh.epi_go = *abort_flag ? 0 : 1;
+      if (use_xchg) {
+        // adopt the agreed bounds: v > max(local, prev(g))  <=>  v > local and v >= g
+        for (int q = et; q < nq_c; q += 128) {
+          const float g = __ldcg(&gthr[q0 + q]);
+          if (g > -INFINITY) thr_s[q] = fmaxf(thr_s[q], nextafterf(g, -INFINITY));
+        }
+      }
       epilogue_bar();
       if (!sh.epi_go) { ok = false; break; }
       tc_fence_after();
@@ -422,6 +441,44 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap key_map,
           epilogue_bar();
         }
       }
+      }
+      if (use_xchg) {
+        // publish this CTA's best per query (the owner warp's lists are quiescent here) ...
+        for (int q = ew + 4 * lane; q < nq_c; q += 128) {
+          const u64 top = lists[(size_t)q * kk];
+          if (top != 0) __stcg(&lmax[(size_t)(q0 + q) * kTcMaxCtas + blockIdx.x], candidate_score(top));
+        }
+        // ... and, for the queries this CTA is responsible for, agree on the bound: the k-th
+        // largest of all CTAs' bests, by k rounds of warp-wide maximum extraction
+        for (int q = ew; q < nq_c; q += 4) {
+          if ((q0 + q) % (int)gridDim.x != (int)blockIdx.x) continue;     // warp-uniform
+          float mine[kTcMaxCtas / 32];
+#pragma unroll
+          for (int i = 0; i < kTcMaxCtas / 32; ++i) {
+            const int c = i * 32 + lane;
+            mine[i] = c < (int)gridDim.x ? __ldcg(&lmax[(size_t)(q0 + q) * kTcMaxCtas + c]) : -INFINITY;
+          }
+          float kth_best = -INFINITY;
+          for (int r = 0; r < k; ++r) {
+            float m = mine[0];
+#pragma unroll
+            for (int i = 1; i < kTcMaxCtas / 32; ++i) m = fmaxf(m, mine[i]);
+            float w = m;
+#pragma unroll
+            for (int o = 16; o; o >>= 1) w = fmaxf(w, __shfl_xor_sync(0xffffffffu, w, o));
+            kth_best = w;
+            if (w == -INFINITY) break;                                     // fewer than k bests yet
+            const int owner = __ffs(__ballot_sync(0xffffffffu, m == w)) - 1;
+            if (lane == owner) {                                           // remove one instance
+              bool done = false;
+#pragma unroll
+              for (int i = 0; i < kTcMaxCtas / 32; ++i)
+                if (!done && mine[i] == w) { mine[i] = -INFINITY; done = true; }
+            }
+          }
+          if (lane == 0 && kth_best > -INFINITY && kth_best > __ldcg(&gthr[q0 + q]))
+            __stcg(&gthr[q0 + q], kth_best);
+        }
       }
     }
     // publish this CTA's per-query lists: already descending, empty slots are 0
@@ -556,8 +613,8 @@ int tc_queries_per_pass(int nq, int k, size_t smem_limit) {
 
 cudaError_t launch_scan_tc(TcCache* cache, const PoolView& pv, int32_t q0, int32_t nq_c,
                            int32_t nq_total, int32_t k, int32_t kk, const uint64_t* exclude_tag,
-                           unsigned long long* partial, DeviceStats* stats, int32_t num_sms,
-                           size_t smem_limit, int32_t* n_lists, cudaStream_t st) {
+                           unsigned long long* partial, DeviceStats* stats, float* xchg,
+                           int32_t num_sms, size_t smem_limit, int32_t* n_lists, cudaStream_t st) {
   const int n_pad = (nq_c + 15) / 16 * 16;
   const int n_tiles128 = (pv.n_rows + kTileM - 1) / kTileM;
   static const int force_mt = getenv("OILBIRD_TC_MT") ? atoi(getenv("OILBIRD_TC_MT")) : 0;
@@ -582,7 +639,7 @@ cudaError_t launch_scan_tc(TcCache* cache, const PoolView& pv, int32_t q0, int32
   if (e != cudaSuccess) return e;
   return launch_pdl(scan_tc_kernel, dim3(grid), dim3(kTcThreads), smem, st,
                     cache->key_map, *q_map, pv, q0, nq_c, nq_total, n_pad, k, kk, plan.stages,
-                    tmem_cols, plan.mt, plan.n_bufs, exclude_tag, partial, stats);
+                    tmem_cols, plan.mt, plan.n_bufs, exclude_tag, partial, stats, xchg);
 }
 
 }  // namespace oilbird

@@ -379,3 +379,29 @@ def test_key_widths_that_are_not_multiples_of_the_k_block(d):
     w = W.C1.scaled(nq=3, k=8, n_rows=1500, d=d, cont_len=4, sigma=0.3)
     run_workload(w, paths=(B.PATH_GEMV, B.PATH_TENSOR))
     run_workload(w.separated(), paths=(B.PATH_GEMV, B.PATH_TENSOR))
+
+
+def test_exact_ties_spread_over_all_ctas_keep_the_lowest_rows():
+    """Many rows with identical scores, spread over every CTA of the tensor scan: the
+    thresholds the CTAs exchange must never drop a tied row that has a lower position."""
+    d, n = 64, 148 * 128 * 4 + 77
+    rng = np.random.default_rng(5)
+    base = rng.choice([-1, 1], size=d)
+    hs = rng.choice([0, 1, 2, 3, 20, 21, 22, 30], size=n, p=[.002, .004, .004, .01, .2, .2, .28, .3])
+    rows = np.tile(base, (n, 1))
+    for h in np.unique(hs):
+        rows[hs == h, :h] *= -1
+    bits = np.where(rows > 0, P1, M1).astype(np.uint16)
+    tk = np.arange(n, dtype=np.int32)
+    pool, ora = B.Pool(d, n, max_k=128), OraclePool(d)
+    pool.append(bits_to_dev(bits), torch.from_numpy(tk).cuda(), tag=1)
+    ora.append(bits, tk, tag=1)
+    qb = np.stack([np.where(base > 0, P1, M1).astype(np.uint16)] * 3)
+    qb[1, :2] = np.where(base[:2] > 0, M1, P1)              # a second, slightly different query
+    for k in (1, 8, 64, 128):
+        for path in (B.PATH_TENSOR, B.PATH_GEMV):
+            pr = fixed(k, 2, theta=-2.0, path=path)
+            out = pool.query(bits_to_dev(qb), pr).cpu()
+            ref = ora.query(qb, __import__("parity").oracle_params(pr))
+            assert out.idx.numpy().tolist() == ref.idx.tolist(), (k, path)
+            assert np.array_equal(out.score.numpy(), ref.score)

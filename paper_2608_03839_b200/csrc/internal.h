@@ -79,7 +79,7 @@ cudaError_t launch_qnorm(const uint16_t* q, int32_t nq, int32_t nq_pad, int32_t 
 
 // Cross-CTA threshold exchange of the tensor scan: per query one published best score per
 // CTA (kTcMaxCtas slots) followed by one agreed lower bound per query.
-constexpr int kTcMaxCtas = 256;
+constexpr int kTcMaxCtas = 160;   // >= the 148 SMs of a B200; five values per lane
 constexpr int kTcXchgFloats = OILBIRD_MAX_NQ * kTcMaxCtas + OILBIRD_MAX_NQ;
 
 // Length of the candidate lists exchanged between scan and merge for a given k.

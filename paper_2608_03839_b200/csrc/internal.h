@@ -100,7 +100,7 @@ struct TcCache;
 TcCache* tc_cache_create(const void* keys, int64_t capacity, int32_t d, const void* qn,
                          int64_t qn_rows);
 void tc_cache_destroy(TcCache* cache);
-int tc_queries_per_pass(int nq, int k, size_t smem_limit);   // balanced split of a call
+int tc_queries_per_pass(int nq, int k, int n_rows, int num_sms, size_t smem_limit);
 cudaError_t launch_scan_tc(TcCache* cache, const PoolView& pv, int32_t q0, int32_t nq_c,
                            int32_t nq_total, int32_t k, int32_t kk, const uint64_t* exclude_tag,
                            unsigned long long* partial, DeviceStats* stats, float* xchg,

@@ -381,7 +381,7 @@ int oilbird_pool_query(oilbird_pool_t* p, const void* q, int32_t nq,
       if (e != cudaSuccess) return cuda_fail(e, "qnorm kernel launch");
       p->launches += 1;
       // as many queries per pass as shared memory allows next to a 3-stage ring
-      const int per_pass = tc_queries_per_pass(nq, pr->k, p->smem_limit);
+      const int per_pass = tc_queries_per_pass(nq, pr->k, pv.n_rows, p->num_sms, p->smem_limit);
       for (int q0 = 0; q0 < nq; q0 += per_pass) {
         const int nq_c = nq - q0 < per_pass ? nq - q0 : per_pass;
         e = launch_scan_tc(p->tc, pv, q0, nq_c, nq, pr->k, kk, pr->exclude_tag, p->partial,

@@ -165,6 +165,36 @@ struct TcShared {
   int q_cnt[kColsPerRound];     // ... per score column of the round
 };
 
+// Per-query candidate lists in shared memory.  Wide form: one packed 64-bit key per slot.
+// Compact form (6 bytes per slot: fp32 score + 16-bit position), chosen when it lets a call
+// run in fewer passes over the keys: a CTA's rows are numbered locally, its it-th macro tile
+// holding local rows [it*rows_per_tile, (it+1)*rows_per_tile), so 16 bits cover the 65,536
+// rows one CTA scans in pools of up to ~9.7 million rows.  An empty slot is key 0 / -inf.
+struct ListStore {
+  u64* wide;
+  float* sc;
+  uint16_t* loc;
+  int kk, shift;          // rows per macro tile = 1 << shift
+  bool compact;
+
+  __device__ __forceinline__ u64 load(int q, int i) const {
+    if (!compact) return wide[(size_t)q * kk + i];
+    const float s = sc[(size_t)q * kk + i];
+    if (s == -INFINITY) return 0;
+    const uint32_t l = loc[(size_t)q * kk + i];
+    const uint32_t tile = blockIdx.x + (l >> shift) * gridDim.x;
+    return pack_candidate(s, (tile << shift) | (l & ((1u << shift) - 1u)));
+  }
+  __device__ __forceinline__ void store(int q, int i, u64 key) const {
+    if (!compact) { wide[(size_t)q * kk + i] = key; return; }
+    if (key == 0) { sc[(size_t)q * kk + i] = -INFINITY; loc[(size_t)q * kk + i] = 0; return; }
+    const uint32_t row = (uint32_t)candidate_row(key);
+    const uint32_t it = ((row >> shift) - blockIdx.x) / gridDim.x;
+    sc[(size_t)q * kk + i] = candidate_score(key);
+    loc[(size_t)q * kk + i] = (uint16_t)((it << shift) | (row & ((1u << shift) - 1u)));
+  }
+};
+
 // Fold the candidates queued in one round into the descending lists of the (up to four)
 // queries this warp owns in the round.  Lists live in shared memory (kk = 32*E slots, empty
 // slots are 0) and are held in registers meanwhile; afterwards the filter threshold of
@@ -176,7 +206,7 @@ constexpr int kDrainQ = kColsPerRound / 4;      // queries per warp and round
 constexpr int kCrowd = 8;
 
 template <int E>
-__device__ __forceinline__ void drain_round(u64* lists, int kk, const u64* q_key,
+__device__ __forceinline__ void drain_round(const ListStore& lists, int kk, const u64* q_key,
                                             const int* q_cnt, int c0, int ew, int nq_c, int k,
                                             float* thr_s, int lane) {
   u64 v[kDrainQ][E];
@@ -189,7 +219,7 @@ __device__ __forceinline__ void drain_round(u64* lists, int kk, const u64* q_key
     n[u] = q < nq_c ? q_cnt[j] : 0;
     if (n[u] > 0) {
 #pragma unroll
-      for (int r = 0; r < E; ++r) v[u][r] = lists[(size_t)q * kk + r * 32 + lane];
+      for (int r = 0; r < E; ++r) v[u][r] = lists.load(q, r * 32 + lane);
       kth[u] = warp_list_get<E>(v[u], k - 1);
     } else {
 #pragma unroll
@@ -234,7 +264,7 @@ __device__ __forceinline__ void drain_round(u64* lists, int kk, const u64* q_key
     if (n[u] > 0) {
       const int q = c0 + ew + 4 * u;
 #pragma unroll
-      for (int r = 0; r < E; ++r) lists[(size_t)q * kk + r * 32 + lane] = v[u][r];
+      for (int r = 0; r < E; ++r) lists.store(q, r * 32 + lane, v[u][r]);
       const u64 nk = warp_list_get<E>(v[u], k - 1);
       // never below a bound adopted from the other CTAs
       if (lane == 0 && nk != 0) thr_s[q] = fmaxf(thr_s[q], candidate_score(nk));
@@ -252,8 +282,8 @@ __global__ void __launch_bounds__(kTcThreads, 1)
 scan_tc_kernel(const __grid_constant__ CUtensorMap key_map,
                const __grid_constant__ CUtensorMap q_map, PoolView pv, int q0, int nq_c,
                int nq_total, int n_pad, int k, int kk, int n_stages, int tmem_cols, int mt,
-               int n_bufs, const uint64_t* __restrict__ exclude_tag, u64* __restrict__ partial,
-               DeviceStats* stats, float* xchg) {
+               int n_bufs, int compact, const uint64_t* __restrict__ exclude_tag,
+               u64* __restrict__ partial, DeviceStats* stats, float* xchg) {
   extern __shared__ __align__(1024) unsigned char smem_raw[];
   __shared__ TcShared sh;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -263,8 +293,16 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap key_map,
   // dynamic shared memory: [stages][mt key tiles | query tile] | lists | queue | state
   unsigned char* base = (unsigned char*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
   unsigned char* ring = base;
-  u64* lists = reinterpret_cast<u64*>(ring + (size_t)n_stages * stage_bytes);   // [nq_c][kk]
-  u64* q_key = lists + (size_t)nq_c * kk;                      // [kColsPerRound][kTileM]
+  unsigned char* list_mem = ring + (size_t)n_stages * stage_bytes;              // [nq_c][kk]
+  ListStore lists;
+  lists.wide = reinterpret_cast<u64*>(list_mem);
+  lists.sc = reinterpret_cast<float*>(list_mem);
+  lists.loc = reinterpret_cast<uint16_t*>(list_mem + (size_t)nq_c * kk * 4);
+  lists.kk = kk;
+  lists.shift = mt == 2 ? 8 : 7;
+  lists.compact = compact != 0;
+  u64* q_key = reinterpret_cast<u64*>(list_mem + (size_t)nq_c * kk * (compact ? 6 : 8));
+                                                               // [kColsPerRound][kTileM]
   uint64_t* s_ex = reinterpret_cast<uint64_t*>(q_key + kQueueCap);              // [n_pad]
   float* thr_s = reinterpret_cast<float*>(s_ex + n_pad);                        // [n_pad]
   // Cross-CTA threshold exchange (global memory, reset to -inf by the query preparation):
@@ -306,7 +344,7 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap key_map,
     thr_s[i] = -INFINITY;
     s_ex[i] = (exclude_tag && i < nq_c) ? exclude_tag[q0 + i] : 0;
   }
-  for (int i = threadIdx.x; i < nq_c * kk; i += kTcThreads) lists[i] = 0;
+  for (int i = threadIdx.x; i < nq_c * kk; i += kTcThreads) lists.store(i / kk, i % kk, 0);
   __syncthreads();
 
   if (warp == 0) {
@@ -445,7 +483,7 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap key_map,
       if (use_xchg) {
         // publish this CTA's best per query (the owner warp's lists are quiescent here) ...
         for (int q = ew + 4 * lane; q < nq_c; q += 128) {
-          const u64 top = lists[(size_t)q * kk];
+          const u64 top = lists.load(q, 0);
           if (top != 0) __stcg(&lmax[(size_t)(q0 + q) * kTcMaxCtas + blockIdx.x], candidate_score(top));
         }
         // ... and, for the queries this CTA is responsible for, agree on the bound: the k-th
@@ -485,7 +523,7 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap key_map,
     epilogue_bar();
     for (int i = et; i < nq_c * kk; i += 128) {
       const int q = i / kk, j = i - q * kk;
-      partial[((size_t)blockIdx.x * nq_total + (q0 + q)) * kk + j] = lists[i];
+      partial[((size_t)blockIdx.x * nq_total + (q0 + q)) * kk + j] = lists.load(q, j);
     }
   }
   tc_fence_before();
@@ -567,20 +605,23 @@ static const CUtensorMap* tc_q_map(TcCache* c, int n_pad) {
   return &c->q_map[slot];
 }
 
-static size_t tc_fixed_smem(int nq_c, int n_pad, int kk) {
-  return (size_t)nq_c * kk * 8 + (size_t)kQueueCap * 8 + (size_t)n_pad * (8 + 4) +
-         1024 /* alignment slack */;
+static size_t tc_fixed_smem(int nq_c, int n_pad, int kk, bool compact) {
+  return (size_t)nq_c * kk * (compact ? 6 : 8) + (size_t)kQueueCap * 8 +
+         (size_t)n_pad * (8 + 4) + 1024 /* alignment slack */;
 }
 
-// How a call is cut up: queries per pass, key tiles per query tile, ring stages,
-// accumulator buffers.  Fewest passes first (every pass re-reads the keys); then two key
-// tiles per query tile if at least three ring stages still fit, else one.
-struct TcPlan { int per_pass, mt, stages, n_bufs; };
+// How a call is cut up: queries per pass, list format, key tiles per query tile, ring
+// stages, accumulator buffers.  Fewest passes first (every pass re-reads the keys): the
+// compact list format is taken when it saves a pass (two ring stages are then enough: ring
+// depth was measured not to matter once the epilogue sets the pace); then two key tiles per
+// query tile if at least three ring stages still fit, else one.
+struct TcPlan { int per_pass, mt, stages, n_bufs, compact; };
 
-static bool tc_fits(int n, int kk, int mt, int min_stages, size_t smem_limit, int* stages) {
+static bool tc_fits(int n, int kk, int mt, bool compact, int min_stages, size_t smem_limit,
+                    int* stages) {
   const size_t stage = (size_t)mt * kATileBytes + (size_t)n * kBlockK * 2;
   // static shared memory (barriers etc.) is padded to the 1024-byte alignment of the ring
-  const size_t fixed = tc_fixed_smem(n, n, kk) + 1024 + 256;
+  const size_t fixed = tc_fixed_smem(n, n, kk, compact) + 1024 + 256;
   if (fixed + (size_t)min_stages * stage > smem_limit) return false;
   int st = (int)((smem_limit - fixed) / stage);
   *stages = st > kMaxStages ? kMaxStages : st;
@@ -589,26 +630,37 @@ static bool tc_fits(int n, int kk, int mt, int min_stages, size_t smem_limit, in
 
 static TcPlan tc_plan(int nq, int k, int n_tiles128, int num_sms, size_t smem_limit, int force_mt) {
   const int kk = list_len(k);
-  int max_pass = 16, st = 0;
-  for (int n = 16; n <= OILBIRD_MAX_NQ; n += 16)
-    if (tc_fits(n, kk, 1, 3, smem_limit, &st)) max_pass = n;
-  const int n_pass = (nq + max_pass - 1) / max_pass;
+  int max_pass = 16, max_pass_c = 16, st = 0;
+  for (int n = 16; n <= OILBIRD_MAX_NQ; n += 16) {
+    if (tc_fits(n, kk, 1, false, 3, smem_limit, &st)) max_pass = n;
+    if (tc_fits(n, kk, 1, true, 2, smem_limit, &st)) max_pass_c = n;
+  }
+  int n_pass = (nq + max_pass - 1) / max_pass;
+  // 16-bit local positions: the rows one CTA scans must number at most 65,536
+  const int grid = n_tiles128 < num_sms ? (n_tiles128 > 0 ? n_tiles128 : 1) : num_sms;
+  const bool can_compact = ((int64_t)(n_tiles128 + grid - 1) / grid + 1) * kTileM <= 65536;
   TcPlan p;
+  p.compact = 0;
+  if (can_compact && (nq + max_pass_c - 1) / max_pass_c < n_pass) {
+    p.compact = 1;
+    n_pass = (nq + max_pass_c - 1) / max_pass_c;
+  }
+  const bool cp = p.compact != 0;
   p.per_pass = ((nq + n_pass - 1) / n_pass + 15) / 16 * 16;      // balanced passes
   const int n_pad = p.per_pass < nq ? p.per_pass : (nq + 15) / 16 * 16;
   // sharing a query tile between two key tiles pays at every nq measured (fewer, larger
   // stages and half the query bytes from L2), given enough tiles to keep every SM busy
-  bool two = n_tiles128 >= 4 * num_sms && tc_fits(n_pad, kk, 2, 3, smem_limit, &st);
+  bool two = n_tiles128 >= 4 * num_sms && tc_fits(n_pad, kk, 2, cp, 3, smem_limit, &st);
   if (force_mt == 1) two = false;
-  if (force_mt == 2) two = tc_fits(n_pad, kk, 2, 2, smem_limit, &st);
+  if (force_mt == 2) two = tc_fits(n_pad, kk, 2, cp, 2, smem_limit, &st);
   p.mt = two ? 2 : 1;
-  tc_fits(n_pad, kk, p.mt, 2, smem_limit, &p.stages);
+  tc_fits(n_pad, kk, p.mt, cp, 2, smem_limit, &p.stages);
   p.n_bufs = 2 * p.mt * n_pad <= 512 ? 2 : 1;
   return p;
 }
 
-int tc_queries_per_pass(int nq, int k, size_t smem_limit) {
-  return tc_plan(nq, k, 0, 1, smem_limit, 1).per_pass;
+int tc_queries_per_pass(int nq, int k, int n_rows, int num_sms, size_t smem_limit) {
+  return tc_plan(nq, k, (n_rows + kTileM - 1) / kTileM, num_sms, smem_limit, 0).per_pass;
 }
 
 cudaError_t launch_scan_tc(TcCache* cache, const PoolView& pv, int32_t q0, int32_t nq_c,
@@ -622,7 +674,7 @@ cudaError_t launch_scan_tc(TcCache* cache, const PoolView& pv, int32_t q0, int32
   static const int cap_stages = getenv("OILBIRD_TC_STAGES") ? atoi(getenv("OILBIRD_TC_STAGES")) : 0;
   if (cap_stages >= 2 && plan.stages > cap_stages) plan.stages = cap_stages;
   const size_t stage = (size_t)plan.mt * kATileBytes + (size_t)n_pad * kBlockK * 2;
-  const size_t fixed = tc_fixed_smem(nq_c, n_pad, kk);
+  const size_t fixed = tc_fixed_smem(nq_c, n_pad, kk, plan.compact != 0);
   if (plan.stages < 2) return cudaErrorInvalidConfiguration;
   const CUtensorMap* q_map = tc_q_map(cache, n_pad);
   if (!q_map) return cudaErrorInvalidValue;
@@ -639,7 +691,8 @@ cudaError_t launch_scan_tc(TcCache* cache, const PoolView& pv, int32_t q0, int32
   if (e != cudaSuccess) return e;
   return launch_pdl(scan_tc_kernel, dim3(grid), dim3(kTcThreads), smem, st,
                     cache->key_map, *q_map, pv, q0, nq_c, nq_total, n_pad, k, kk, plan.stages,
-                    tmem_cols, plan.mt, plan.n_bufs, exclude_tag, partial, stats, xchg);
+                    tmem_cols, plan.mt, plan.n_bufs, plan.compact, exclude_tag, partial, stats,
+                    xchg);
 }
 
 }  // namespace oilbird

@@ -15,6 +15,9 @@ enum { kRowOk = 0, kRowZero = 1, kRowNonFinite = 2 };
 // double precision (products of bf16 values are exact there), the scale 1/sqrt is IEEE
 // double, each element is rounded once to float and once to bf16 (nearest even).
 // Returns kRowOk, or kRowZero / kRowNonFinite, in which case dst is all zero.
+// kHold: keep the row's chunks in registers between the two passes (one read of the row;
+// 32 registers), or read it twice (for kernels that are short of registers).
+template <bool kHold = true>
 __device__ __forceinline__ int normalize_row(const uint16_t* __restrict__ src, uint16_t* __restrict__ dst,
                               int d) {
   __shared__ double s_part[kNormThreads / 32];
@@ -23,15 +26,29 @@ __device__ __forceinline__ int normalize_row(const uint16_t* __restrict__ src, u
   __shared__ int s_code;
   const int n_chunks = d >> 3;
   const uint4* src4 = reinterpret_cast<const uint4*>(src);
+  // d <= 16384: at most 8 chunks of 8 elements per thread, kept in registers so that the
+  // row is read from memory once
+  constexpr int kMaxChunks = 16384 / 8 / kNormThreads;
+  uint4 held[kMaxChunks];
   double ss = 0.0;
   int bad = 0;
-  for (int c = threadIdx.x; c < n_chunks; c += kNormThreads) {
-    uint4 v = __ldg(src4 + c);
-    uint32_t w[4] = {v.x, v.y, v.z, v.w};
+  if (kHold) {
 #pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      float lo = bf16_lo(w[i]), hi = bf16_hi(w[i]);
-      bad |= ((w[i] & 0x7f80u) == 0x7f80u) | ((w[i] & 0x7f800000u) == 0x7f800000u);
+    for (int i = 0; i < kMaxChunks; ++i) {
+      const int c = threadIdx.x + i * kNormThreads;
+      held[i] = c < n_chunks ? __ldg(src4 + c) : make_uint4(0, 0, 0, 0);
+    }
+  }
+#pragma unroll
+  for (int i = 0; i < kMaxChunks; ++i) {
+    const int c0 = threadIdx.x + i * kNormThreads;
+    if (!kHold && c0 >= n_chunks) break;
+    const uint4 hv = kHold ? held[i] : __ldg(src4 + c0);
+    const uint32_t w[4] = {hv.x, hv.y, hv.z, hv.w};
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      float lo = bf16_lo(w[j]), hi = bf16_hi(w[j]);
+      bad |= ((w[j] & 0x7f80u) == 0x7f80u) | ((w[j] & 0x7f800000u) == 0x7f800000u);
       ss += (double)lo * (double)lo;
       ss += (double)hi * (double)hi;
     }
@@ -56,16 +73,19 @@ __device__ __forceinline__ int normalize_row(const uint16_t* __restrict__ src, u
   __syncthreads();
   const double inv = s_inv;
   uint4* dst4 = reinterpret_cast<uint4*>(dst);
-  for (int c = threadIdx.x; c < n_chunks; c += kNormThreads) {
-    uint4 v = __ldg(src4 + c);
-    uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+  for (int i = 0; i < kMaxChunks; ++i) {
+    const int c = threadIdx.x + i * kNormThreads;
+    if (c >= n_chunks) break;
+    const uint4 hv = kHold ? held[i] : __ldg(src4 + c);
+    const uint32_t w[4] = {hv.x, hv.y, hv.z, hv.w};
     uint32_t o[4];
 #pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      if (inv == 0.0) { o[i] = 0; continue; }
-      float lo = __double2float_rn((double)bf16_lo(w[i]) * inv);
-      float hi = __double2float_rn((double)bf16_hi(w[i]) * inv);
-      o[i] = f32_to_bf16_bits(lo) | (f32_to_bf16_bits(hi) << 16);
+    for (int j = 0; j < 4; ++j) {
+      if (inv == 0.0) { o[j] = 0; continue; }
+      float lo = __double2float_rn((double)bf16_lo(w[j]) * inv);
+      float hi = __double2float_rn((double)bf16_hi(w[j]) * inv);
+      o[j] = f32_to_bf16_bits(lo) | (f32_to_bf16_bits(hi) << 16);
     }
     dst4[c] = make_uint4(o[0], o[1], o[2], o[3]);
   }

@@ -55,7 +55,7 @@ ring_scan_kernel(const uint16_t* __restrict__ keys, const int32_t* __restrict__ 
   const int q = blockIdx.y;
   pdl_launch_dependents();
   pdl_wait();
-  const int code = normalize_row(q_raw + (size_t)q * d, reinterpret_cast<uint16_t*>(qs), d);
+  const int code = normalize_row<false>(q_raw + (size_t)q * d, reinterpret_cast<uint16_t*>(qs), d);
   if (blockIdx.x == 0 && threadIdx.x == 0) {
     q_valid[q] = code == kRowNonFinite ? 0 : 1;
     if (code == kRowNonFinite) atomicAdd(&stats->nonfinite_queries, 1ull);

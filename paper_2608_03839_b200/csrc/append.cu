@@ -13,7 +13,7 @@
 
 namespace oilbird {
 
-__global__ void __launch_bounds__(kNormThreads)
+__global__ void __launch_bounds__(kNormThreads, 4)
 append_kernel(const uint16_t* __restrict__ states, const int32_t* __restrict__ tokens, int64_t n,
               int d, uint16_t* __restrict__ keys, int32_t* __restrict__ tok,
               int32_t* __restrict__ trace_id, int64_t row0, int32_t trace,

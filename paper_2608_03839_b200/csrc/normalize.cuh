@@ -26,15 +26,16 @@ __device__ __forceinline__ int normalize_row(const uint16_t* __restrict__ src, u
   __shared__ int s_code;
   const int n_chunks = d >> 3;
   const uint4* src4 = reinterpret_cast<const uint4*>(src);
-  // d <= 16384: at most 8 chunks of 8 elements per thread, kept in registers so that the
-  // row is read from memory once
+  // at most 8 chunks of 8 elements per thread (d <= 16384); the first kHeld of them (all
+  // of a row up to d = 8192) stay in registers so that the row is read from memory once
   constexpr int kMaxChunks = 16384 / 8 / kNormThreads;
-  uint4 held[kMaxChunks];
+  constexpr int kHeld = 4;
+  uint4 held[kHeld];
   double ss = 0.0;
   int bad = 0;
   if (kHold) {
 #pragma unroll
-    for (int i = 0; i < kMaxChunks; ++i) {
+    for (int i = 0; i < kHeld; ++i) {
       const int c = threadIdx.x + i * kNormThreads;
       held[i] = c < n_chunks ? __ldg(src4 + c) : make_uint4(0, 0, 0, 0);
     }
@@ -42,8 +43,8 @@ __device__ __forceinline__ int normalize_row(const uint16_t* __restrict__ src, u
 #pragma unroll
   for (int i = 0; i < kMaxChunks; ++i) {
     const int c0 = threadIdx.x + i * kNormThreads;
-    if (!kHold && c0 >= n_chunks) break;
-    const uint4 hv = kHold ? held[i] : __ldg(src4 + c0);
+    if (c0 >= n_chunks) break;
+    const uint4 hv = (kHold && i < kHeld) ? held[i] : __ldg(src4 + c0);
     const uint32_t w[4] = {hv.x, hv.y, hv.z, hv.w};
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
@@ -77,7 +78,7 @@ __device__ __forceinline__ int normalize_row(const uint16_t* __restrict__ src, u
   for (int i = 0; i < kMaxChunks; ++i) {
     const int c = threadIdx.x + i * kNormThreads;
     if (c >= n_chunks) break;
-    const uint4 hv = kHold ? held[i] : __ldg(src4 + c);
+    const uint4 hv = (kHold && i < kHeld) ? held[i] : __ldg(src4 + c);
     const uint32_t w[4] = {hv.x, hv.y, hv.z, hv.w};
     uint32_t o[4];
 #pragma unroll

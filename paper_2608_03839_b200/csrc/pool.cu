@@ -33,7 +33,7 @@ size_t align_up(size_t v) { return (v + kAlign - 1) / kAlign * kAlign; }
 struct Layout {
   size_t keys, tok, trace_id, trace_end, trace_tag, trace_gbase, qn, q_valid, partial, stats;
   size_t xchg;
-  size_t q_stage, ex_stage, st_stage, tok_stage, out_stage;
+  size_t q_stage, ex_stage, st_stage, tok_stage, stage_end;
   size_t total;
 };
 
@@ -79,12 +79,12 @@ Layout make_layout(const Resolved& r) {
   L.partial = take((size_t)r.max_lists * r.max_nq * k_pad * 8);
   L.stats = take(sizeof(DeviceStats));
   L.xchg = take((size_t)kTcXchgFloats * 4);
-  // staging for the *_host variants
+  // staging for the *_host variants (adjacent: query_host/step_host fill them with one copy)
   L.q_stage = take((size_t)r.max_nq * r.d * 2);
   L.ex_stage = take((size_t)r.max_nq * 8);
   L.st_stage = take((size_t)r.max_append * r.d * 2);
   L.tok_stage = take((size_t)r.max_append * 4);
-  L.out_stage = take((size_t)r.max_nq * ((size_t)r.max_k * (8 + 4 + 4 * OILBIRD_MAX_CONT_LEN) + 4));
+  L.stage_end = off;
   L.total = off;
   return L;
 }
@@ -116,8 +116,9 @@ struct oilbird_pool {
   std::vector<cudaEvent_t> ev;   // pairs
   int ev_used;
   // pinned staging for host variants
-  unsigned char* pinned;
-  size_t pinned_bytes;
+  unsigned char* pinned;       // host address
+  unsigned char* pinned_dev;   // the same block as the device sees it
+  size_t blob_off, result_off;
   cudaEvent_t upload_done;
   bool upload_pending;
   // tensor-core scan: TMA tensor maps of this pool (nullptr = path unavailable)
@@ -179,7 +180,7 @@ int oilbird_pool_create(oilbird_pool_t** out, const oilbird_pool_config* cfg) {
   if (!p) return OILBIRD_ENOMEM;
   p->r = r; p->lay = lay; p->device = cfg->device; p->num_sms = prop.multiProcessorCount;
   p->n_rows = 0; p->launches = 0; p->profile = false; p->ev_used = 0;
-  p->pinned = nullptr; p->pinned_bytes = 0;
+  p->pinned = nullptr; p->pinned_dev = nullptr;
   if (cfg->arena) {
     size_t mis = (size_t)((uintptr_t)cfg->arena % kAlign);
     size_t skip = mis ? kAlign - mis : 0;
@@ -417,18 +418,45 @@ int oilbird_pool_gather(oilbird_pool_t* p, const int32_t* idx, const float* scor
 
 // ---- host-buffer variants ---------------------------------------------------------
 
-// Pinned host staging: [append block | query-result block].  The append block is reused
-// by the next append_host call, so an event marks when its upload has finished.
+// Pinned, device-mapped host staging: [append_host block | upload blob | result block].
+// The append_host block is reused by the next append_host call, so an event marks when its
+// upload has finished.  query_host and step_host return only after everything has
+// completed; they pack their inputs into the upload blob (one host->device copy per call)
+// and let the merge kernel write the results straight into the mapped result block, which
+// is valid on the host once the stream has been synchronised.
+struct HostBlob {
+  size_t o_st, o_tok, o_q, o_ex, used;
+};
+static HostBlob blob_layout(const oilbird_pool* p, int64_t n, int32_t nq, bool with_ex) {
+  HostBlob b;
+  size_t off = 0;
+  auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes); return o; };
+  b.o_st = take((size_t)n * p->r.d * 2);
+  b.o_tok = take((size_t)n * 4);
+  b.o_q = take((size_t)nq * p->r.d * 2);
+  b.o_ex = take(with_ex ? (size_t)nq * 8 : 0);
+  b.used = off;
+  return b;
+}
+
 static int ensure_pinned(oilbird_pool* p) {
   if (p->pinned) return OILBIRD_OK;
   const size_t a_bytes = (size_t)p->r.max_append * p->r.d * 2 + (size_t)p->r.max_append * 4;
+  const size_t b_bytes = blob_layout(p, p->r.max_append, p->r.max_nq, true).used;
   const size_t o_bytes =
       (size_t)p->r.max_nq * ((size_t)p->r.max_k * (8 + 4 + 4 * OILBIRD_MAX_CONT_LEN) + 4);
-  cudaError_t e = cudaMallocHost((void**)&p->pinned, align_up(a_bytes) + o_bytes);
-  if (e != cudaSuccess) return cuda_fail(e, "cudaMallocHost");
-  p->pinned_bytes = align_up(a_bytes);          // offset of the result block
-  e = cudaEventCreateWithFlags(&p->upload_done, cudaEventDisableTiming);
-  if (e != cudaSuccess) return cuda_fail(e, "cudaEventCreate");
+  unsigned char* h = nullptr;
+  cudaError_t e = cudaHostAlloc((void**)&h, align_up(a_bytes) + b_bytes + o_bytes,
+                                cudaHostAllocMapped);
+  if (e != cudaSuccess) return cuda_fail(e, "cudaHostAlloc");
+  void* dptr = nullptr;
+  e = cudaHostGetDevicePointer(&dptr, h, 0);
+  if (e == cudaSuccess) e = cudaEventCreateWithFlags(&p->upload_done, cudaEventDisableTiming);
+  if (e != cudaSuccess) { cudaFreeHost(h); return cuda_fail(e, "pinned staging set-up"); }
+  p->pinned = h;
+  p->pinned_dev = (unsigned char*)dptr;
+  p->blob_off = align_up(a_bytes);
+  p->result_off = p->blob_off + b_bytes;
   p->upload_pending = false;
   return OILBIRD_OK;
 }
@@ -458,10 +486,12 @@ int oilbird_pool_append_host(oilbird_pool_t* p, const void* states, const int32_
   return oilbird_pool_append(p, d_st, d_tok, n, tag, flags, stream);
 }
 
-int oilbird_pool_query_host(oilbird_pool_t* p, const void* q, int32_t nq,
-                            const oilbird_query_params* pr, const oilbird_query_out* out,
-                            void* stream) {
+// Shared body of query_host (n = 0, no append) and step_host.
+static int host_step(oilbird_pool_t* p, bool do_append, const void* states, const int32_t* tokens,
+                     int64_t n, uint64_t tag, uint32_t flags, const void* q, int32_t nq,
+                     const oilbird_query_params* pr, const oilbird_query_out* out, void* stream) {
   if (!p || !q || !out_ok(out, true)) return OILBIRD_EINVAL;
+  if (n < 0 || n > p->r.max_append || (n > 0 && (!states || !tokens))) return OILBIRD_EINVAL;
   GatherParams gp;
   int rc = check_params(p, nq, pr, &gp);
   if (rc) return rc;
@@ -470,31 +500,45 @@ int oilbird_pool_query_host(oilbird_pool_t* p, const void* q, int32_t nq,
   if (rc) return rc;
   cudaStream_t st = (cudaStream_t)stream;
   const size_t k = pr->k, L = pr->cont_len;
-  uint16_t* d_q = (uint16_t*)(p->base + p->lay.q_stage);
-  uint64_t* d_ex = (uint64_t*)(p->base + p->lay.ex_stage);
-  unsigned char* d_out = p->base + p->lay.out_stage;
-  unsigned char* h_out = p->pinned + p->pinned_bytes;
-  // device-side result block: idx | score | cont_len | cont_tok | fired
-  const size_t o_idx = 0, o_score = o_idx + nq * k * 4, o_len = o_score + nq * k * 4,
-               o_tok = o_len + nq * k * 4, o_fired = o_tok + nq * k * L * 4,
-               o_total = o_fired + (size_t)nq * 4;
-  // the call synchronises before it returns, so the caller's buffers can be read directly
-  CU(cudaMemcpyAsync(d_q, q, (size_t)nq * p->r.d * 2, cudaMemcpyHostToDevice, st));
+
+  // inputs: one packed block, one copy (the device staging areas are adjacent in the arena)
+  const HostBlob b = blob_layout(p, n, nq, pr->exclude_tag != nullptr);
+  unsigned char* h_blob = p->pinned + p->blob_off;
+  unsigned char* d_blob = p->base + p->lay.q_stage;
+  if (b.used > p->lay.stage_end - p->lay.q_stage) return OILBIRD_EINVAL;   // cannot happen
+  if (n > 0) {
+    memcpy(h_blob + b.o_st, states, (size_t)n * p->r.d * 2);
+    memcpy(h_blob + b.o_tok, tokens, (size_t)n * 4);
+  }
+  memcpy(h_blob + b.o_q, q, (size_t)nq * p->r.d * 2);
   oilbird_query_params dp = *pr;
   if (pr->exclude_tag) {
-    CU(cudaMemcpyAsync(d_ex, pr->exclude_tag, (size_t)nq * 8, cudaMemcpyHostToDevice, st));
-    dp.exclude_tag = d_ex;
+    memcpy(h_blob + b.o_ex, pr->exclude_tag, (size_t)nq * 8);
+    dp.exclude_tag = (const uint64_t*)(d_blob + b.o_ex);
   }
+  CU(cudaMemcpyAsync(d_blob, h_blob, b.used, cudaMemcpyHostToDevice, st));
+  if (do_append) {
+    rc = oilbird_pool_append(p, d_blob + b.o_st, (const int32_t*)(d_blob + b.o_tok), n, tag, flags,
+                             stream);
+    if (rc) { cudaStreamSynchronize(st); return rc; }
+  }
+
+  // results: idx | score | cont_len | cont_tok | fired, written by the kernel into mapped
+  // host memory
+  const size_t o_idx = 0, o_score = o_idx + nq * k * 4, o_len = o_score + nq * k * 4,
+               o_tok = o_len + nq * k * 4, o_fired = o_tok + nq * k * L * 4;
+  unsigned char* h_out = p->pinned + p->result_off;
+  unsigned char* d_out = p->pinned_dev + p->result_off;
   oilbird_query_out dout;
   dout.idx = (int32_t*)(d_out + o_idx);
   dout.score = (float*)(d_out + o_score);
   dout.cont_len = (int32_t*)(d_out + o_len);
   dout.cont_tok = (int32_t*)(d_out + o_tok);
   dout.fired = (int32_t*)(d_out + o_fired);
-  rc = oilbird_pool_query(p, d_q, nq, &dp, &dout, stream);
+  rc = oilbird_pool_query(p, d_blob + b.o_q, nq, &dp, &dout, stream);
+  cudaError_t e = cudaStreamSynchronize(st);     // also frees the caller's buffers on error
   if (rc) return rc;
-  CU(cudaMemcpyAsync(h_out, d_out, o_total, cudaMemcpyDeviceToHost, st));
-  CU(cudaStreamSynchronize(st));
+  if (e != cudaSuccess) return cuda_fail(e, "cudaStreamSynchronize");
   memcpy(out->idx, h_out + o_idx, nq * k * 4);
   memcpy(out->score, h_out + o_score, nq * k * 4);
   memcpy(out->cont_len, h_out + o_len, nq * k * 4);
@@ -503,25 +547,17 @@ int oilbird_pool_query_host(oilbird_pool_t* p, const void* q, int32_t nq,
   return OILBIRD_OK;
 }
 
+int oilbird_pool_query_host(oilbird_pool_t* p, const void* q, int32_t nq,
+                            const oilbird_query_params* pr, const oilbird_query_out* out,
+                            void* stream) {
+  return host_step(p, false, nullptr, nullptr, 0, 0, 0, q, nq, pr, out, stream);
+}
+
 int oilbird_pool_step_host(oilbird_pool_t* p, const void* states, const int32_t* tokens,
                            int64_t n, uint64_t tag, uint32_t flags, const void* q, int32_t nq,
                            const oilbird_query_params* pr, const oilbird_query_out* out,
                            void* stream) {
-  // The call returns only after everything has completed, so the rows are uploaded straight
-  // from the caller's buffers (no pinned staging copy as in append_host).
-  if (!p || n < 0 || n > p->r.max_append || (n > 0 && (!states || !tokens))) return OILBIRD_EINVAL;
-  CU(cudaSetDevice(p->device));
-  cudaStream_t st = (cudaStream_t)stream;
-  uint16_t* d_st = (uint16_t*)(p->base + p->lay.st_stage);
-  int32_t* d_tok = (int32_t*)(p->base + p->lay.tok_stage);
-  if (n > 0) {
-    CU(cudaMemcpyAsync(d_st, states, (size_t)n * p->r.d * 2, cudaMemcpyHostToDevice, st));
-    CU(cudaMemcpyAsync(d_tok, tokens, (size_t)n * 4, cudaMemcpyHostToDevice, st));
-  }
-  int rc = oilbird_pool_append(p, d_st, d_tok, n, tag, flags, stream);
-  if (rc == OILBIRD_OK) rc = oilbird_pool_query_host(p, q, nq, pr, out, stream);
-  if (rc != OILBIRD_OK) cudaStreamSynchronize(st);   // the caller's buffers are free on return
-  return rc;
+  return host_step(p, true, states, tokens, n, tag, flags, q, nq, pr, out, stream);
 }
 
 // ---- introspection ------------------------------------------------------------------

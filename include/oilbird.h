@@ -172,10 +172,12 @@ int oilbird_pool_gather(oilbird_pool_t* pool, const int32_t* idx, const float* s
  * The same two operations with HOST buffers.  append_host copies its inputs into pinned
  * staging and enqueues upload + append; the caller's buffers are free again when it
  * returns, the rows are visible to later calls on the same stream.  query_host uploads
- * the queries, runs the query and returns after the results have landed in the host
- * arrays of `out` (it synchronises cuda_stream).  params->exclude_tag and every array of
- * `out` are host pointers here.  n <= cfg.max_append.  All *_host calls of a pool must
- * use one stream: the staging buffers are reused in stream order.
+ * the queries (one copy), runs the query and returns after the results have landed in the
+ * host arrays of `out` (it synchronises cuda_stream; the kernels write the results into
+ * device-mapped pinned memory, so there is no copy back to wait for).
+ * params->exclude_tag and every array of `out` are host pointers here.
+ * n <= cfg.max_append.  All *_host calls of a pool must use one stream: the staging
+ * buffers are reused in stream order.
  */
 int oilbird_pool_append_host(oilbird_pool_t* pool, const void* states_bf16_host,
                              const int32_t* tokens_host, int64_t n, uint64_t trace_tag,

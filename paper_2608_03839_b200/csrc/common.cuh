@@ -137,6 +137,74 @@ __device__ __forceinline__ void warp_merge_desc(u64 (&a)[E], const u64 (&b)[E], 
     warp_bitonic_stage<E>(a, lane, 1 << 30, stride);
 }
 
+// The same networks over NB independent lists at once, list index innermost: a stage is a
+// chain of a shuffle and half a dozen dependent ALU operations (~40 cycles), and the
+// compiler keeps separate calls of the routines above one after the other, so NB lists
+// sorted by NB calls take NB times as long; interleaved by hand they overlap (8 lists
+// fill the issue slots).
+template <int NB, int E>
+__device__ __forceinline__ void warp_bitonic_stage_batch(u64 (&v)[NB][E], int lane, int size,
+                                                         int stride) {
+  if (stride >= 32) {
+    const int rs = stride >> 5;
+#pragma unroll
+    for (int r = 0; r < E; ++r) {
+      if ((r & rs) == 0) {
+        const bool desc = ((r * 32 + lane) & size) == 0;
+#pragma unroll
+        for (int b = 0; b < NB; ++b) {
+          const u64 x = v[b][r], y = v[b][r | rs];
+          const bool sw = (x < y) == desc;
+          v[b][r] = sw ? y : x;
+          v[b][r | rs] = sw ? x : y;
+        }
+      }
+    }
+  } else {
+#pragma unroll
+    for (int r = 0; r < E; ++r) {
+      const int i = r * 32 + lane;
+      const bool keep_max = ((i & stride) == 0) == ((i & size) == 0);
+      u64 o[NB];
+#pragma unroll
+      for (int b = 0; b < NB; ++b) o[b] = shfl_xor_u64(v[b][r], stride);
+#pragma unroll
+      for (int b = 0; b < NB; ++b) v[b][r] = ((v[b][r] > o[b]) == keep_max) ? v[b][r] : o[b];
+    }
+  }
+}
+
+template <int NB, int E>
+__device__ __forceinline__ void warp_sort_desc_batch(u64 (&v)[NB][E], int lane) {
+#pragma unroll
+  for (int size = 2; size <= 32 * E; size <<= 1)
+#pragma unroll
+    for (int stride = size >> 1; stride > 0; stride >>= 1)
+      warp_bitonic_stage_batch<NB, E>(v, lane, size == 32 * E ? (1 << 30) : size, stride);
+}
+
+// a[b] <- the K largest of (a[b] U c[b]) for every b; all lists sorted descending.
+template <int NB, int E>
+__device__ __forceinline__ void warp_merge_desc_batch(u64 (&a)[NB][E], const u64 (&c)[NB][E],
+                                                      int lane) {
+#pragma unroll
+  for (int r = 0; r < E; ++r) {
+    u64 o[NB];
+#pragma unroll
+    for (int b = 0; b < NB; ++b) {
+      const u64 src = c[b][E - 1 - r];
+      const uint32_t lo = __shfl_sync(0xffffffffu, (uint32_t)src, 31 - lane);
+      const uint32_t hi = __shfl_sync(0xffffffffu, (uint32_t)(src >> 32), 31 - lane);
+      o[b] = ((u64)hi << 32) | lo;
+    }
+#pragma unroll
+    for (int b = 0; b < NB; ++b) a[b][r] = a[b][r] > o[b] ? a[b][r] : o[b];
+  }
+#pragma unroll
+  for (int stride = 16 * E; stride > 0; stride >>= 1)
+    warp_bitonic_stage_batch<NB, E>(a, lane, 1 << 30, stride);
+}
+
 // Insert one candidate (the same key in every lane) into a descending register list,
 // dropping the smallest element.  Branch-free (a key of 0, the empty slot, is a no-op in
 // effect), so that several independent lists can be updated in interleaved straight-line

@@ -12,13 +12,20 @@
 //   warps 2-5   epilogue: tcgen05.ld the 128 x nq scores, filter them against the
 //               per-query running k-th best, and keep per-query top-k lists in shared
 //               memory (Eq. 2); scores never go to global memory
-// The key stream (N*d*2 bytes from HBM, once) bounds the kernel up to nq ~ 64.  Beyond
-// that the epilogue sets the pace: with the filter switched off the same launch streams
-// at 6.2 TB/s for nq = 128, with it at 4.1 TB/s; ring depth (2..5 stages) and the query
-// tile's L2 traffic make no measurable difference there.  A variant that transposes the
-// scores through shared memory so that one warp owns a query's 128 rows (no queue, no
-// atomics, one barrier per round) was measured 15-30 % slower: its fixed cost per round
-// outweighs the cheaper candidate path.
+// The key stream (N*d*2 bytes from HBM, once) bounds the kernel up to nq ~ 64-96; the
+// epilogue warps then wait for accumulators 60-80 % of the time.  What is left above that:
+//   - a CTA's first one or two macro tiles, whose scores nearly all pass the still-low
+//     thresholds (sorted 32 at a time and merged): ~2.5 tiles' worth of time at nq = 128,
+//     during which the accumulator buffers are full and the key stream stalls;
+//   - at nq = 256 the query tile re-read from L2 per key tile (twice the key bytes) and the
+//     single k-block per accumulator set; the tensor pipe reaches about half its peak.
+// Measured and not kept: separate shared-memory rings for keys and query tiles (query
+// tiles queue behind the key requests, so they need the same lead; 5-8 % slower); a
+// 32-deep candidate queue with retry, to buy a ring stage (slower first tiles, no gain from
+// the stage); ballot-packed per-warp queue segments instead of shared-memory atomics (drain
+// 60 % slower); sorting every column of the first tile in registers without the queue (no
+// faster than the queue's crowd path); a variant that transposes the scores through shared
+// memory so that one warp owns a query's 128 rows (15-30 % slower).
 //
 // Every mbarrier wait is bounded: after about two seconds it raises the pool's `stalled`
 // flag, the CTA drains what it has in flight, frees its TMEM and returns.
@@ -161,7 +168,7 @@ struct TcShared {
   uint32_t tmem_base;
   int abort_flag;
   int epi_go;
-  int q_total;                  // candidates queued in the current round
+  int q_total;                  // nonzero: candidates were queued in the current round
   int q_cnt[kColsPerRound];     // ... per score column of the round
 };
 
@@ -242,10 +249,8 @@ __device__ __forceinline__ void drain_round(const ListStore& lists, int kk, cons
         b[u][r] = key > kth[u] ? key : 0;
       }
     }
-#pragma unroll
-    for (int u = 0; u < kDrainQ; ++u) warp_sort_desc<E>(b[u], lane);
-#pragma unroll
-    for (int u = 0; u < kDrainQ; ++u) warp_merge_desc<E>(v[u], b[u], lane);
+    warp_sort_desc_batch<kDrainQ, E>(b, lane);
+    warp_merge_desc_batch<kDrainQ, E>(v, b, lane);
 #pragma unroll
     for (int u = 0; u < kDrainQ; ++u) kth[u] = warp_list_get<E>(v[u], k - 1);
   }
@@ -341,7 +346,7 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap key_map,
   const uint32_t tmem_base = sh.tmem_base;
   pdl_wait();   // appended rows, normalised queries, exclusion tags; set-up above overlapped
   for (int i = threadIdx.x; i < n_pad; i += kTcThreads) {
-    thr_s[i] = -INFINITY;
+    thr_s[i] = i < nq_c ? -INFINITY : INFINITY;        // padded columns never pass the filter
     s_ex[i] = (exclude_tag && i < nq_c) ? exclude_tag[q0 + i] : 0;
   }
   for (int i = threadIdx.x; i < nq_c * kk; i += kTcThreads) lists.store(i / kk, i % kk, 0);
@@ -454,17 +459,36 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap key_map,
           __syncwarp();
           if (lane == 0) mbar_arrive(&sh.tmem_empty[buf]);
         }
-        if (row_ok) {
+        // The round's sixteen thresholds are fetched together and compared without a
+        // branch; only the (rare) passing columns are visited.  Comparing column by column
+        // with the queue's atomics in the loop body keeps every threshold load behind the
+        // previous column's possible store and costs ~2,000 cycles a round.
+        uint32_t pass = 0;
+        {
+          const float4* t4 = reinterpret_cast<const float4*>(thr_s + c0);
+          const float4 ta = t4[0], tb = t4[1], tc = t4[2], td = t4[3];
+          const float t[kColsPerRound] = {ta.x, ta.y, ta.z, ta.w, tb.x, tb.y, tb.z, tb.w,
+                                          tc.x, tc.y, tc.z, tc.w, td.x, td.y, td.z, td.w};
 #pragma unroll
-          for (int j = 0; j < kColsPerRound; ++j) {
-            const int q = c0 + j;
-            if (q < nq_c && v[j] > thr_s[q]) {
-              if (s_ex[q] != 0 && tag == s_ex[q]) continue;       // same-prompt trace: skipped
-              const int pos = atomicAdd(&sh.q_cnt[j], 1);
-              q_key[j * kTileM + pos] = pack_candidate(v[j], (uint32_t)row);
-              atomicAdd(&sh.q_total, 1);
-            }
-          }
+          for (int j = 0; j < kColsPerRound; ++j) pass |= (v[j] > t[j] ? 1u : 0u) << j;
+          if (!row_ok) pass = 0;
+        }
+        // Lanes walk their passing columns from different starting points: while a CTA's
+        // thresholds are still low every row passes in every column, and 128 threads taking
+        // the columns in the same order would serialise on one counter at a time.
+        const int rot = lane & (kColsPerRound - 1);
+        pass = ((pass >> rot) | (pass << (kColsPerRound - rot))) & ((1u << kColsPerRound) - 1u);
+        while (pass) {
+          const int j = (__ffs(pass) - 1 + rot) & (kColsPerRound - 1);
+          pass &= pass - 1;
+          const int q = c0 + j;
+          if (s_ex[q] != 0 && tag == s_ex[q]) continue;           // same-prompt trace: skipped
+          float vj = v[0];
+#pragma unroll
+          for (int i = 1; i < kColsPerRound; ++i) vj = j == i ? v[i] : vj;
+          const int pos = atomicAdd(&sh.q_cnt[j], 1);
+          q_key[j * kTileM + pos] = pack_candidate(vj, (uint32_t)row);
+          sh.q_total = 1;
         }
         epilogue_bar();
         if (sh.q_total > 0) {
@@ -480,7 +504,8 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap key_map,
         }
       }
       }
-      if (use_xchg) {
+      // The agreed bound tightens like 1/t: after the first tiles every fourth exchange is enough
+      if (use_xchg && (iter < 4 || (iter & 3u) == 3u)) {
         // publish this CTA's best per query (the owner warp's lists are quiescent here) ...
         for (int q = ew + 4 * lane; q < nq_c; q += 128) {
           const u64 top = lists.load(q, 0);

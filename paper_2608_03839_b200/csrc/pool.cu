@@ -424,6 +424,8 @@ int oilbird_pool_gather(oilbird_pool_t* p, const int32_t* idx, const float* scor
 // completed; they pack their inputs into the upload blob (one host->device copy per call)
 // and let the merge kernel write the results straight into the mapped result block, which
 // is valid on the host once the stream has been synchronised.
+constexpr size_t kPackLimit = 256 << 10;   // bytes up to which a step's inputs are packed
+
 struct HostBlob {
   size_t o_st, o_tok, o_q, o_ex, used;
 };
@@ -506,17 +508,35 @@ static int host_step(oilbird_pool_t* p, bool do_append, const void* states, cons
   unsigned char* h_blob = p->pinned + p->blob_off;
   unsigned char* d_blob = p->base + p->lay.q_stage;
   if (b.used > p->lay.stage_end - p->lay.q_stage) return OILBIRD_EINVAL;   // cannot happen
-  if (n > 0) {
-    memcpy(h_blob + b.o_st, states, (size_t)n * p->r.d * 2);
-    memcpy(h_blob + b.o_tok, tokens, (size_t)n * 4);
-  }
-  memcpy(h_blob + b.o_q, q, (size_t)nq * p->r.d * 2);
   oilbird_query_params dp = *pr;
-  if (pr->exclude_tag) {
-    memcpy(h_blob + b.o_ex, pr->exclude_tag, (size_t)nq * 8);
-    dp.exclude_tag = (const uint64_t*)(d_blob + b.o_ex);
+  if (pr->exclude_tag) dp.exclude_tag = (const uint64_t*)(d_blob + b.o_ex);
+  if (b.used <= kPackLimit) {
+    // small step: pack, one copy (a copy's fixed cost outweighs the host-side memcpy)
+    if (n > 0) {
+      memcpy(h_blob + b.o_st, states, (size_t)n * p->r.d * 2);
+      memcpy(h_blob + b.o_tok, tokens, (size_t)n * 4);
+    }
+    memcpy(h_blob + b.o_q, q, (size_t)nq * p->r.d * 2);
+    if (pr->exclude_tag) memcpy(h_blob + b.o_ex, pr->exclude_tag, (size_t)nq * 8);
+    CU(cudaMemcpyAsync(d_blob, h_blob, b.used, cudaMemcpyHostToDevice, st));
+  } else {
+    // large step: the call synchronises before it returns, so the caller's buffers are
+    // uploaded directly (DMA from pinned memory; the driver stages pageable memory itself)
+    cudaError_t ce = cudaSuccess;
+    if (n > 0) {
+      ce = cudaMemcpyAsync(d_blob + b.o_st, states, (size_t)n * p->r.d * 2, cudaMemcpyHostToDevice, st);
+      if (ce == cudaSuccess)
+        ce = cudaMemcpyAsync(d_blob + b.o_tok, tokens, (size_t)n * 4, cudaMemcpyHostToDevice, st);
+    }
+    if (ce == cudaSuccess)
+      ce = cudaMemcpyAsync(d_blob + b.o_q, q, (size_t)nq * p->r.d * 2, cudaMemcpyHostToDevice, st);
+    if (ce == cudaSuccess && pr->exclude_tag)
+      ce = cudaMemcpyAsync(d_blob + b.o_ex, pr->exclude_tag, (size_t)nq * 8, cudaMemcpyHostToDevice, st);
+    if (ce != cudaSuccess) {
+      cudaStreamSynchronize(st);             // nothing may still read the caller's buffers
+      return cuda_fail(ce, "cudaMemcpyAsync(host step)");
+    }
   }
-  CU(cudaMemcpyAsync(d_blob, h_blob, b.used, cudaMemcpyHostToDevice, st));
   if (do_append) {
     rc = oilbird_pool_append(p, d_blob + b.o_st, (const int32_t*)(d_blob + b.o_tok), n, tag, flags,
                              stream);

@@ -169,6 +169,22 @@ int oilbird_pool_gather(oilbird_pool_t* pool, const int32_t* idx, const float* s
                         const oilbird_query_out* out, void* cuda_stream);
 
 /*
+ * One serving step with DEVICE buffers: oilbird_pool_append (the n rows committed since
+ * the last step; n may be 0) followed by oilbird_pool_query, in one call, with the same
+ * arguments, results and error codes as the two calls (Algorithm 1 runs once per decoding
+ * step: the accepted tokens' states are stored, then the new last position is looked up).
+ * Nothing is appended if the query arguments are invalid.  For the single-request scan
+ * (nq <= 2) and up to 64 rows the append has no kernel of its own: the first n CTAs of the
+ * scan normalise one row each before they start scanning, and the warps that reach the
+ * appended rows (the last rows of the pool) first wait, bounded, for a counter that says
+ * all n have been written (a time-out raises the `stalled` status, see oilbird_pool_status).
+ */
+int oilbird_pool_step(oilbird_pool_t* pool, const void* states_bf16, const int32_t* tokens,
+                      int64_t n, uint64_t trace_tag, uint32_t flags, const void* q_bf16,
+                      int32_t nq, const oilbird_query_params* params,
+                      const oilbird_query_out* out, void* cuda_stream);
+
+/*
  * The same two operations with HOST buffers.  append_host copies its inputs into pinned
  * staging and enqueues upload + append; the caller's buffers are free again when it
  * returns, the rows are visible to later calls on the same stream.  query_host uploads

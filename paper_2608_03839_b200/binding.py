@@ -85,6 +85,9 @@ SYMBOLS = {
                                           ctypes.POINTER(CQueryOut), _vp]),
     "oilbird_pool_gather": (ctypes.c_int, [_vp, _vp, _vp, _i32, ctypes.POINTER(CQueryParams),
                                            ctypes.POINTER(CQueryOut), _vp]),
+    "oilbird_pool_step": (ctypes.c_int, [_vp, _vp, _vp, _i64, _u64, _u32, _vp, _i32,
+                                         ctypes.POINTER(CQueryParams),
+                                         ctypes.POINTER(CQueryOut), _vp]),
     "oilbird_pool_append_host": (ctypes.c_int, [_vp, _vp, _vp, _i64, _u64, _u32, _vp]),
     "oilbird_pool_query_host": (ctypes.c_int, [_vp, _vp, _i32, ctypes.POINTER(CQueryParams),
                                                ctypes.POINTER(CQueryOut), _vp]),
@@ -362,6 +365,33 @@ class Pool:
         _check(self._L.oilbird_pool_query(self._h, q.data_ptr(), nq, ctypes.byref(cp),
                                           ctypes.byref(out._c), _stream_ptr(stream)),
                "oilbird_pool_query")
+        return out
+
+    def step(self, states: torch.Tensor, tokens: torch.Tensor, q: torch.Tensor,
+             params: QueryParams | None = None, out: QueryOut | None = None, tag: int = 0,
+             new_trace: bool = True, stream=None) -> QueryOut:
+        """One serving step on device tensors: append(states, tokens) then query(q), in one
+        call (same results as the two calls; the single-request scan overlaps the append)."""
+        pr = params or QueryParams()
+        assert states.is_cuda and states.dtype == torch.bfloat16 and states.is_contiguous()
+        assert tokens.is_cuda and tokens.dtype == torch.int32 and tokens.is_contiguous()
+        assert q.is_cuda and q.dtype == torch.bfloat16 and q.is_contiguous()
+        n = int(tokens.shape[0])
+        assert states.numel() == n * self.d
+        q = q.reshape(-1, self.d)
+        nq = q.shape[0]
+        ex_ptr = None
+        if pr.exclude_tag is not None:
+            ex = pr.exclude_tag
+            assert ex.is_cuda and ex.dtype in (torch.int64, torch.uint64) and ex.numel() == nq
+            ex_ptr = ex.data_ptr()
+        if out is None:
+            out = QueryOut.empty(nq, pr.k, pr.cont_len, self._dev)
+        cp = pr.to_c(ex_ptr)
+        _check(self._L.oilbird_pool_step(
+            self._h, states.data_ptr(), tokens.data_ptr(), n, int(tag),
+            NEW_TRACE if new_trace else 0, q.data_ptr(), nq, ctypes.byref(cp),
+            ctypes.byref(out._c), _stream_ptr(stream)), "oilbird_pool_step")
         return out
 
     def gather(self, idx: torch.Tensor, score: torch.Tensor, params: QueryParams,

@@ -56,6 +56,27 @@ struct GatherParams {
   int32_t tier_depth[OILBIRD_MAX_TIERS];
 };
 
+// The append of one serving step, done by the first n CTAs of the CUDA-core scan itself
+// instead of by a kernel of its own (n == 0: nothing to append).  CTA i normalises row i
+// into keys[row0 + i] and then adds one to *ready; a warp of the scan that is about to
+// read a row >= row0 first waits (bounded) for *ready to reach `target`.
+constexpr int kFuseMaxRows = 64;
+struct FusedAppend {
+  const uint16_t* states;       // [n, d] raw bf16
+  const int32_t* tokens;        // [n]
+  uint16_t* keys;
+  int32_t* tok;
+  int32_t* trace_id;
+  int32_t* trace_end;
+  uint64_t* trace_tag;
+  int64_t* trace_gbase;
+  unsigned long long* ready;    // rows published by fused appends since the pool was created
+  unsigned long long target;    // value of *ready once this step's rows are all in
+  uint64_t tag;
+  int64_t gbase;
+  int32_t n, row0, trace, set_tag;
+};
+
 // a1: normalise n raw bf16 rows into keys[row0..], store tokens / trace ids, and let one
 // thread publish the trace-table entry (trace, end, tag).
 cudaError_t launch_append(const uint16_t* states, const int32_t* tokens, int64_t n, int32_t d,
@@ -91,7 +112,16 @@ inline int list_len(int k) { int p = next_pow2(k); return p < 32 ? 32 : p; }
 cudaError_t launch_scan_gemv(const PoolView& pv, const uint16_t* q_raw, int32_t nq, int32_t k,
                              int32_t kk, const uint64_t* exclude_tag, unsigned long long* partial,
                              int32_t* q_valid, DeviceStats* stats, int32_t max_lists,
-                             int32_t num_sms, int32_t* n_lists, cudaStream_t st);
+                             int32_t num_sms, int32_t* n_lists, const FusedAppend* fused,
+                             cudaStream_t st);
+
+// CTAs the CUDA-core scan launches for a pool of n_rows rows.
+inline int32_t scan_gemv_grid(int64_t n_rows, int32_t num_sms, int32_t max_lists) {
+  // at least 32 rows per CTA, at most two CTAs per SM
+  int64_t want = (n_rows + 31) / 32;
+  int32_t grid = (int32_t)(want < 1 ? 1 : (want > 2 * num_sms ? 2 * num_sms : want));
+  return grid > max_lists ? max_lists : grid;
+}
 
 // a2+a3 (tensor cores): the same contract for queries [q0, q0+nq_c) of a call whose
 // normalised queries already sit in qn.  TcCache holds the pool's TMA tensor maps

@@ -33,7 +33,7 @@ size_t align_up(size_t v) { return (v + kAlign - 1) / kAlign * kAlign; }
 struct Layout {
   size_t keys, tok, trace_id, trace_end, trace_tag, trace_gbase, qn, q_valid, partial, stats;
   size_t xchg;
-  size_t q_stage, ex_stage, st_stage, tok_stage, stage_end;
+  size_t q_stage, ex_stage, st_stage, tok_stage, stage_end, fuse_ready;
   size_t total;
 };
 
@@ -78,6 +78,7 @@ Layout make_layout(const Resolved& r) {
   L.q_valid = take(nq_pad * 4);
   L.partial = take((size_t)r.max_lists * r.max_nq * k_pad * 8);
   L.stats = take(sizeof(DeviceStats));
+  L.fuse_ready = take(8);
   L.xchg = take((size_t)kTcXchgFloats * 4);
   // staging for the *_host variants (adjacent: query_host/step_host fill them with one copy)
   L.q_stage = take((size_t)r.max_nq * r.d * 2);
@@ -106,6 +107,8 @@ struct oilbird_pool {
   unsigned long long* partial;
   DeviceStats* stats;
   float* xchg;               // tensor scan: cross-CTA threshold exchange
+  unsigned long long* fuse_ready;   // rows published by appends fused into a scan ...
+  unsigned long long fuse_target;   // ... and the host's count of them (enqueue time)
   // host bookkeeping (enqueue-time truth)
   int64_t n_rows;
   std::vector<int64_t> t_start, t_end;
@@ -205,7 +208,10 @@ int oilbird_pool_create(oilbird_pool_t** out, const oilbird_pool_config* cfg) {
   p->partial = (unsigned long long*)(p->base + lay.partial);
   p->stats = (DeviceStats*)(p->base + lay.stats);
   p->xchg = (float*)(p->base + lay.xchg);
+  p->fuse_ready = (unsigned long long*)(p->base + lay.fuse_ready);
+  p->fuse_target = 0;
   cudaError_t e = cudaMemset(p->stats, 0, sizeof(DeviceStats));
+  if (e == cudaSuccess) e = cudaMemset(p->fuse_ready, 0, 8);
   if (e != cudaSuccess) {
     if (p->owns_mem) cudaFree(p->base);
     delete p;
@@ -244,32 +250,58 @@ int64_t oilbird_pool_size(const oilbird_pool_t* p) { return p ? p->n_rows : 0; }
 int32_t oilbird_pool_num_traces(const oilbird_pool_t* p) { return p ? (int32_t)p->t_start.size() : 0; }
 int64_t oilbird_pool_launch_count(const oilbird_pool_t* p) { return p ? p->launches : 0; }
 
-// global_row < 0: the pool is not a shard, a trace's global position is its local one.
-static int append_impl(oilbird_pool_t* p, const void* states, const int32_t* tokens, int64_t n,
-                       uint64_t tag, uint32_t flags, int64_t global_row, void* stream) {
+// Host side of an append: checks, then the trace bookkeeping (enqueue-time truth).
+struct AppendPlan {
+  bool open_new;
+  int32_t trace;
+  int64_t row0;
+};
+
+static int append_prepare(oilbird_pool_t* p, const void* states, const int32_t* tokens, int64_t n,
+                          uint64_t tag, uint32_t flags, AppendPlan* ap, bool* nothing) {
+  *nothing = false;
   if (!p || n < 0 || (n > 0 && (!states || !tokens))) return OILBIRD_EINVAL;
-  const bool open_new = (flags & OILBIRD_NEW_TRACE) || p->t_start.empty();
-  if (n == 0 && !open_new) return OILBIRD_OK;
+  ap->open_new = (flags & OILBIRD_NEW_TRACE) || p->t_start.empty();
+  if (n == 0 && !ap->open_new) { *nothing = true; return OILBIRD_OK; }
   if (p->n_rows + n > p->r.capacity) return OILBIRD_ECAPACITY;
-  if (open_new && (int64_t)p->t_start.size() >= p->r.max_traces) return OILBIRD_ECAPACITY;
-  CU(cudaSetDevice(p->device));
-  if (open_new) {
+  if (ap->open_new && (int64_t)p->t_start.size() >= p->r.max_traces) return OILBIRD_ECAPACITY;
+  if (ap->open_new) {
     p->t_start.push_back(p->n_rows);
     p->t_end.push_back(p->n_rows);
     p->t_tag.push_back(tag);
   }
-  const int32_t trace = (int32_t)p->t_start.size() - 1;
+  ap->trace = (int32_t)p->t_start.size() - 1;
+  ap->row0 = p->n_rows;
+  return OILBIRD_OK;
+}
+static void append_rollback(oilbird_pool_t* p, const AppendPlan& ap) {
+  if (ap.open_new) { p->t_start.pop_back(); p->t_end.pop_back(); p->t_tag.pop_back(); }
+  p->n_rows = ap.row0;
+  if (!ap.open_new) p->t_end[ap.trace] = ap.row0;
+}
+static void append_commit(oilbird_pool_t* p, int64_t n, const AppendPlan& ap) {
+  p->n_rows = ap.row0 + n;
+  p->t_end[ap.trace] = p->n_rows;
+}
+
+// global_row < 0: the pool is not a shard, a trace's global position is its local one.
+static int append_impl(oilbird_pool_t* p, const void* states, const int32_t* tokens, int64_t n,
+                       uint64_t tag, uint32_t flags, int64_t global_row, void* stream) {
+  AppendPlan ap;
+  bool nothing;
+  int rc = append_prepare(p, states, tokens, n, tag, flags, &ap, &nothing);
+  if (rc || nothing) return rc;
+  CU(cudaSetDevice(p->device));
   cudaError_t e = launch_append((const uint16_t*)states, tokens, n, p->r.d, p->keys, p->tok,
-                                p->trace_id, p->n_rows, trace, p->trace_end, p->trace_tag, tag,
-                                p->trace_gbase, global_row >= 0 ? global_row : p->n_rows,
-                                open_new ? 1 : 0, p->stats, (cudaStream_t)stream);
+                                p->trace_id, ap.row0, ap.trace, p->trace_end, p->trace_tag, tag,
+                                p->trace_gbase, global_row >= 0 ? global_row : ap.row0,
+                                ap.open_new ? 1 : 0, p->stats, (cudaStream_t)stream);
   if (e != cudaSuccess) {
-    if (open_new) { p->t_start.pop_back(); p->t_end.pop_back(); p->t_tag.pop_back(); }
+    append_rollback(p, ap);
     return cuda_fail(e, "append kernel launch");
   }
   p->launches += 1;
-  p->n_rows += n;
-  p->t_end[trace] = p->n_rows;
+  append_commit(p, n, ap);
   return OILBIRD_OK;
 }
 
@@ -331,9 +363,16 @@ static bool out_ok(const oilbird_query_out* o, bool need_idx) {
   return !need_idx || (o->idx && o->score);
 }
 
-int oilbird_pool_query(oilbird_pool_t* p, const void* q, int32_t nq,
-                       const oilbird_query_params* pr, const oilbird_query_out* out,
-                       void* stream) {
+static int resolve_path(const oilbird_query_params* pr, int32_t nq) {
+  // single-request decode streams keys through the CUDA cores; batches go to tcgen05
+  if (pr->path != OILBIRD_PATH_AUTO) return pr->path;
+  return nq <= 2 ? OILBIRD_PATH_GEMV : OILBIRD_PATH_TENSOR;
+}
+
+// fused: the step's append, to be done by the CUDA-core scan itself (the rows are already
+// counted in p->n_rows), or nullptr.
+static int query_impl(oilbird_pool_t* p, const void* q, int32_t nq, const oilbird_query_params* pr,
+                      const oilbird_query_out* out, void* stream, const FusedAppend* fused) {
   if (!p || !q || !out_ok(out, true)) return OILBIRD_EINVAL;
   GatherParams gp;
   int rc = check_params(p, nq, pr, &gp);
@@ -345,9 +384,7 @@ int oilbird_pool_query(oilbird_pool_t* p, const void* q, int32_t nq,
   PoolView pv = view_of(p);
   cudaError_t e;
 
-  // single-request decode streams keys through the CUDA cores; batches go to tcgen05
-  int path = pr->path;
-  if (path == OILBIRD_PATH_AUTO) path = nq <= 2 ? OILBIRD_PATH_GEMV : OILBIRD_PATH_TENSOR;
+  const int path = resolve_path(pr, nq);
   if (path == OILBIRD_PATH_TENSOR && !p->tc) {
     snprintf(g_cuda_err, sizeof g_cuda_err, "tensor-core scan unavailable on this device");
     return OILBIRD_ECUDA;
@@ -373,7 +410,7 @@ int oilbird_pool_query(oilbird_pool_t* p, const void* q, int32_t nq,
     }
     if (path == OILBIRD_PATH_GEMV) {
       e = launch_scan_gemv(pv, (const uint16_t*)q, nq, pr->k, kk, pr->exclude_tag, p->partial,
-                           p->q_valid, p->stats, p->r.max_lists, p->num_sms, &n_lists, st);
+                           p->q_valid, p->stats, p->r.max_lists, p->num_sms, &n_lists, fused, st);
       if (e != cudaSuccess) return cuda_fail(e, "scan kernel launch");
       p->launches += 1;
     } else {
@@ -400,6 +437,58 @@ int oilbird_pool_query(oilbird_pool_t* p, const void* q, int32_t nq,
   if (e != cudaSuccess) return cuda_fail(e, "merge kernel launch");
   p->launches += 1;
   return OILBIRD_OK;
+}
+
+int oilbird_pool_query(oilbird_pool_t* p, const void* q, int32_t nq,
+                       const oilbird_query_params* pr, const oilbird_query_out* out,
+                       void* stream) {
+  return query_impl(p, q, nq, pr, out, stream, nullptr);
+}
+
+// Append + query.  For the single-request path and a handful of rows the append is done by
+// the scan kernel itself (no kernel of its own in front of the scan).
+static int step_impl(oilbird_pool_t* p, const void* states, const int32_t* tokens, int64_t n,
+                     uint64_t tag, uint32_t flags, const void* q, int32_t nq,
+                     const oilbird_query_params* pr, const oilbird_query_out* out, void* stream) {
+  if (!p || !q || !out_ok(out, true)) return OILBIRD_EINVAL;
+  GatherParams gp;
+  int rc = check_params(p, nq, pr, &gp);          // nothing is appended if the query is invalid
+  if (rc) return rc;
+  const int64_t rows_after = p->n_rows + n;
+  const bool fuse = n >= 1 && n <= kFuseMaxRows && resolve_path(pr, nq) == OILBIRD_PATH_GEMV &&
+                    scan_gemv_grid(rows_after, p->num_sms, p->r.max_lists) >= n;
+  if (!fuse) {
+    rc = append_impl(p, states, tokens, n, tag, flags, -1, stream);
+    if (rc) return rc;
+    return query_impl(p, q, nq, pr, out, stream, nullptr);
+  }
+  AppendPlan ap;
+  bool nothing;
+  rc = append_prepare(p, states, tokens, n, tag, flags, &ap, &nothing);
+  if (rc) return rc;
+  FusedAppend fa;
+  fa.states = (const uint16_t*)states; fa.tokens = tokens;
+  fa.keys = p->keys; fa.tok = p->tok; fa.trace_id = p->trace_id; fa.trace_end = p->trace_end;
+  fa.trace_tag = p->trace_tag; fa.trace_gbase = p->trace_gbase;
+  fa.ready = p->fuse_ready; fa.target = p->fuse_target + (unsigned long long)n;
+  fa.tag = tag; fa.gbase = ap.row0;
+  fa.n = (int32_t)n; fa.row0 = (int32_t)ap.row0; fa.trace = ap.trace; fa.set_tag = ap.open_new ? 1 : 0;
+  append_commit(p, n, ap);                        // the scan must see the new rows
+  const int64_t launches_before = p->launches;
+  rc = query_impl(p, q, nq, pr, out, stream, &fa);
+  if (p->launches == launches_before) {           // the scan was never launched: no append either
+    append_rollback(p, ap);
+    return rc;
+  }
+  p->fuse_target = fa.target;
+  return rc;
+}
+
+int oilbird_pool_step(oilbird_pool_t* p, const void* states, const int32_t* tokens, int64_t n,
+                      uint64_t tag, uint32_t flags, const void* q, int32_t nq,
+                      const oilbird_query_params* pr, const oilbird_query_out* out, void* stream) {
+  if (n < 0 || (n > 0 && (!states || !tokens))) return OILBIRD_EINVAL;
+  return step_impl(p, states, tokens, n, tag, flags, q, nq, pr, out, stream);
 }
 
 int oilbird_pool_gather(oilbird_pool_t* p, const int32_t* idx, const float* score, int32_t nq,
@@ -537,11 +626,6 @@ static int host_step(oilbird_pool_t* p, bool do_append, const void* states, cons
       return cuda_fail(ce, "cudaMemcpyAsync(host step)");
     }
   }
-  if (do_append) {
-    rc = oilbird_pool_append(p, d_blob + b.o_st, (const int32_t*)(d_blob + b.o_tok), n, tag, flags,
-                             stream);
-    if (rc) { cudaStreamSynchronize(st); return rc; }
-  }
 
   // results: idx | score | cont_len | cont_tok | fired, written by the kernel into mapped
   // host memory
@@ -555,7 +639,11 @@ static int host_step(oilbird_pool_t* p, bool do_append, const void* states, cons
   dout.cont_len = (int32_t*)(d_out + o_len);
   dout.cont_tok = (int32_t*)(d_out + o_tok);
   dout.fired = (int32_t*)(d_out + o_fired);
-  rc = oilbird_pool_query(p, d_blob + b.o_q, nq, &dp, &dout, stream);
+  if (do_append)
+    rc = step_impl(p, d_blob + b.o_st, (const int32_t*)(d_blob + b.o_tok), n, tag, flags,
+                   d_blob + b.o_q, nq, &dp, &dout, stream);
+  else
+    rc = query_impl(p, d_blob + b.o_q, nq, &dp, &dout, stream, nullptr);
   cudaError_t e = cudaStreamSynchronize(st);     // also frees the caller's buffers on error
   if (rc) return rc;
   if (e != cudaSuccess) return cuda_fail(e, "cudaStreamSynchronize");

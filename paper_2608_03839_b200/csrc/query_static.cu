@@ -143,7 +143,7 @@ int oilbird_query_static(const oilbird_static_pool* sp, const void* q_bf16, int3
   int32_t n_lists = 0;
   if (sp->n_rows > 0) {
     e = launch_scan_gemv(pv, (const uint16_t*)q_bf16, nq, pr->k, kk, nullptr, partial, q_valid,
-                         stats, kStaticMaxLists, g_num_sms[sp->device], &n_lists, st);
+                         stats, kStaticMaxLists, g_num_sms[sp->device], &n_lists, nullptr, st);
   } else {
     // nothing to scan: the flags only have to say whether each query is usable; the
     // merge kernel then reports "no neighbours" for all of them

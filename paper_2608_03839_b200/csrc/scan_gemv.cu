@@ -25,12 +25,61 @@ namespace oilbird {
 constexpr int kScanThreads = kNormThreads;
 constexpr int kScanWarps = kScanThreads / 32;
 constexpr int kRowsPerIter = 4;   // rows a warp scores together (shares each query load)
+constexpr unsigned long long kFuseWaitNs = 2000000000ull;
+
+// coherent 16-byte load (L2): for rows that another CTA of this launch has just written
+__device__ __forceinline__ uint4 ld_cg16(const void* p) {
+  uint4 v;
+  asm volatile("ld.global.cg.v4.u32 {%0,%1,%2,%3}, [%4];"
+               : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+  return v;
+}
+__device__ __forceinline__ unsigned long long ld_acquire_u64(const unsigned long long* p) {
+  unsigned long long v;
+  asm volatile("ld.acquire.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
+  return v;
+}
+
+// Dot products of kRowsPerIter rows with the QT queries in shared memory; kFresh selects
+// the coherent load for rows written during this launch.
+template <int QT, bool kFresh>
+__device__ __forceinline__ void score_rows(const uint4* const (&rowp)[kRowsPerIter], const uint4* qs,
+                                           int n_chunks, int lane,
+                                           float (&acc)[kRowsPerIter][QT]) {
+#pragma unroll 2
+  for (int c = lane; c < n_chunks; c += 32) {
+    uint4 kv[kRowsPerIter];
+#pragma unroll
+    for (int r = 0; r < kRowsPerIter; ++r)
+      kv[r] = kFresh ? ld_cg16(rowp[r] + c) : ld_stream16(rowp[r] + c);
+#pragma unroll
+    for (int q = 0; q < QT; ++q) {
+      const uint4 qv = qs[q * n_chunks + c];
+      const float q0f = bf16_lo(qv.x), q1f = bf16_hi(qv.x), q2f = bf16_lo(qv.y),
+                  q3f = bf16_hi(qv.y), q4f = bf16_lo(qv.z), q5f = bf16_hi(qv.z),
+                  q6f = bf16_lo(qv.w), q7f = bf16_hi(qv.w);
+#pragma unroll
+      for (int r = 0; r < kRowsPerIter; ++r) {
+        float a = acc[r][q];
+        a = fmaf(bf16_lo(kv[r].x), q0f, a);
+        a = fmaf(bf16_hi(kv[r].x), q1f, a);
+        a = fmaf(bf16_lo(kv[r].y), q2f, a);
+        a = fmaf(bf16_hi(kv[r].y), q3f, a);
+        a = fmaf(bf16_lo(kv[r].z), q4f, a);
+        a = fmaf(bf16_hi(kv[r].z), q5f, a);
+        a = fmaf(bf16_lo(kv[r].w), q6f, a);
+        a = fmaf(bf16_hi(kv[r].w), q7f, a);
+        acc[r][q] = a;
+      }
+    }
+  }
+}
 
 template <int QT, int E>
 __global__ void __launch_bounds__(kScanThreads, 2)
 scan_gemv_kernel(PoolView pv, const uint16_t* __restrict__ q_raw, int nq, int k,
                  const uint64_t* __restrict__ exclude_tag, u64* __restrict__ partial,
-                 int32_t* __restrict__ q_valid, DeviceStats* stats) {
+                 int32_t* __restrict__ q_valid, DeviceStats* stats, FusedAppend fa) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   constexpr int KK = 32 * E;
   pdl_launch_dependents();
@@ -41,11 +90,35 @@ scan_gemv_kernel(PoolView pv, const uint16_t* __restrict__ q_raw, int nq, int k,
   __shared__ uint64_t s_ex[QT];
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  // contiguous, balanced share of the rows for this CTA
+  // contiguous, balanced share of the rows for this CTA; the fa.n CTAs that first append a
+  // row of this step (~2.5 us) take 1/32 less than the others
   const int64_t n = pv.n_rows;
-  const int r_lo = (int)((n * blockIdx.x) / gridDim.x);
-  const int r_hi = (int)((n * (blockIdx.x + 1)) / gridDim.x);
+  const int64_t w_lo = 32ll * blockIdx.x - min((int)blockIdx.x, fa.n);
+  const int64_t w_hi = 32ll * (blockIdx.x + 1) - min((int)blockIdx.x + 1, fa.n);
+  const int64_t w_all = 32ll * gridDim.x - min((int)gridDim.x, fa.n);
+  const int r_lo = (int)((n * w_lo) / w_all);
+  const int r_hi = (int)((n * w_hi) / w_all);
   const uint4* keys4 = reinterpret_cast<const uint4*>(pv.keys);
+
+  // the step's append (Section 4 "(i) Store", Eq. 1), one row per CTA
+  if ((int)blockIdx.x < fa.n) {
+    const int r = blockIdx.x;
+    const int64_t row = (int64_t)fa.row0 + r;
+    const int code = normalize_row<false>(fa.states + (size_t)r * d, fa.keys + row * d, d);
+    if (threadIdx.x == 0) {
+      fa.tok[row] = fa.tokens[r];
+      fa.trace_id[row] = fa.trace;
+      if (code != kRowOk) atomicAdd(&stats->degenerate_rows, 1ull);  // stored as a zero key
+      if (r == 0) {
+        fa.trace_end[fa.trace] = fa.row0 + fa.n;
+        if (fa.set_tag) { fa.trace_tag[fa.trace] = fa.tag; fa.trace_gbase[fa.trace] = fa.gbase; }
+      }
+    }
+    __threadfence();                   // this thread's part of the row, before the count
+    __syncthreads();
+    if (threadIdx.x == 0) atomicAdd(fa.ready, 1ull);
+  }
+  bool fresh_ok = fa.n == 0;           // this warp has seen the appended rows arrive
 
   for (int q0 = 0; q0 < nq; q0 += QT) {
     __syncthreads();
@@ -91,31 +164,24 @@ scan_gemv_kernel(PoolView pv, const uint16_t* __restrict__ q_raw, int nq, int k,
 #pragma unroll
         for (int q = 0; q < QT; ++q) acc[r][q] = 0.f;
 
-#pragma unroll 2
-      for (int c = lane; c < n_chunks; c += 32) {
-        uint4 kv[kRowsPerIter];
-#pragma unroll
-        for (int r = 0; r < kRowsPerIter; ++r) kv[r] = ld_stream16(rowp[r] + c);
-#pragma unroll
-        for (int q = 0; q < QT; ++q) {
-          const uint4 qv = qs[q * n_chunks + c];
-          const float q0f = bf16_lo(qv.x), q1f = bf16_hi(qv.x), q2f = bf16_lo(qv.y),
-                      q3f = bf16_hi(qv.y), q4f = bf16_lo(qv.z), q5f = bf16_hi(qv.z),
-                      q6f = bf16_lo(qv.w), q7f = bf16_hi(qv.w);
-#pragma unroll
-          for (int r = 0; r < kRowsPerIter; ++r) {
-            float a = acc[r][q];
-            a = fmaf(bf16_lo(kv[r].x), q0f, a);
-            a = fmaf(bf16_hi(kv[r].x), q1f, a);
-            a = fmaf(bf16_lo(kv[r].y), q2f, a);
-            a = fmaf(bf16_hi(kv[r].y), q3f, a);
-            a = fmaf(bf16_lo(kv[r].z), q4f, a);
-            a = fmaf(bf16_hi(kv[r].z), q5f, a);
-            a = fmaf(bf16_lo(kv[r].w), q6f, a);
-            a = fmaf(bf16_hi(kv[r].w), q7f, a);
-            acc[r][q] = a;
+      if (fa.n > 0 && rb + kRowsPerIter > fa.row0) {        // warp-uniform
+        // rows of this step's append: wait (bounded) until all of them are in
+        if (!fresh_ok) {
+          unsigned long long t0 = 0;
+          for (uint32_t spin = 0; ld_acquire_u64(fa.ready) < fa.target; ++spin) {
+            if (spin == 0) asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t0));
+            if ((spin & 255u) == 255u) {
+              unsigned long long t1;
+              asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t1));
+              if (t1 - t0 > kFuseWaitNs) { atomicExch(&stats->stalled, 1); break; }
+            }
+            __nanosleep(64);
           }
+          fresh_ok = true;             // (after a time-out the status call reports the stall)
         }
+        score_rows<QT, true>(rowp, qs, n_chunks, lane, acc);
+      } else {
+        score_rows<QT, false>(rowp, qs, n_chunks, lane, acc);
       }
 #pragma unroll
       for (int r = 0; r < kRowsPerIter; ++r) {
@@ -153,37 +219,43 @@ scan_gemv_kernel(PoolView pv, const uint16_t* __restrict__ q_raw, int nq, int k,
 template <int QT, int E>
 static cudaError_t launch_one(const PoolView& pv, const uint16_t* q_raw, int nq, int k,
                               const uint64_t* ex, u64* partial, int32_t* q_valid,
-                              DeviceStats* stats, int grid, cudaStream_t st) {
+                              DeviceStats* stats, int grid, const FusedAppend& fa,
+                              cudaStream_t st) {
   size_t smem = (size_t)QT * pv.d * 2 + (size_t)kScanWarps * 32 * E * sizeof(u64);
   cudaError_t e = cudaFuncSetAttribute(scan_gemv_kernel<QT, E>,
                                        cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
   return launch_pdl(scan_gemv_kernel<QT, E>, dim3(grid), dim3(kScanThreads), smem, st, pv, q_raw,
-                    nq, k, ex, partial, q_valid, stats);
+                    nq, k, ex, partial, q_valid, stats, fa);
 }
 
 template <int QT>
 static cudaError_t launch_qt(int kk, const PoolView& pv, const uint16_t* q_raw, int nq, int k,
                              const uint64_t* ex, u64* partial, int32_t* q_valid,
-                             DeviceStats* stats, int grid, cudaStream_t st) {
-  if (kk == 32) return launch_one<QT, 1>(pv, q_raw, nq, k, ex, partial, q_valid, stats, grid, st);
-  if (kk == 64) return launch_one<QT, 2>(pv, q_raw, nq, k, ex, partial, q_valid, stats, grid, st);
-  return launch_one<QT, 4>(pv, q_raw, nq, k, ex, partial, q_valid, stats, grid, st);
+                             DeviceStats* stats, int grid, const FusedAppend& fa,
+                             cudaStream_t st) {
+  if (kk == 32) return launch_one<QT, 1>(pv, q_raw, nq, k, ex, partial, q_valid, stats, grid, fa, st);
+  if (kk == 64) return launch_one<QT, 2>(pv, q_raw, nq, k, ex, partial, q_valid, stats, grid, fa, st);
+  return launch_one<QT, 4>(pv, q_raw, nq, k, ex, partial, q_valid, stats, grid, fa, st);
 }
 
 cudaError_t launch_scan_gemv(const PoolView& pv, const uint16_t* q_raw, int32_t nq, int32_t k,
                              int32_t kk, const uint64_t* exclude_tag, u64* partial,
                              int32_t* q_valid, DeviceStats* stats, int32_t max_lists,
-                             int32_t num_sms, int32_t* n_lists, cudaStream_t st) {
-  // at least 32 rows per CTA, at most two CTAs per SM
-  int64_t want = (pv.n_rows + 31) / 32;
-  int grid = (int)(want < 1 ? 1 : want);
-  if (grid > 2 * num_sms) grid = 2 * num_sms;
-  if (grid > max_lists) grid = max_lists;
+                             int32_t num_sms, int32_t* n_lists, const FusedAppend* fused,
+                             cudaStream_t st) {
+  const int grid = scan_gemv_grid(pv.n_rows, num_sms, max_lists);
   *n_lists = grid;
+  FusedAppend fa = {};
+  if (fused) {
+    // every appending CTA must exist, and all CTAs be resident together (they are: at most
+    // two per SM are launched), because scanning warps wait for the appending ones
+    if (fused->n > grid || fused->n > kFuseMaxRows) return cudaErrorInvalidValue;
+    fa = *fused;
+  }
   if (nq >= 2)
-    return launch_qt<2>(kk, pv, q_raw, nq, k, exclude_tag, partial, q_valid, stats, grid, st);
-  return launch_qt<1>(kk, pv, q_raw, nq, k, exclude_tag, partial, q_valid, stats, grid, st);
+    return launch_qt<2>(kk, pv, q_raw, nq, k, exclude_tag, partial, q_valid, stats, grid, fa, st);
+  return launch_qt<1>(kk, pv, q_raw, nq, k, exclude_tag, partial, q_valid, stats, grid, fa, st);
 }
 
 }  // namespace oilbird

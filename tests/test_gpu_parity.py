@@ -333,6 +333,73 @@ def test_caller_provided_arena():
     check_query(pool.query(q, fixed(8, 8)), ora, W.to_bits(q), fixed(8, 8))
 
 
+@pytest.mark.parametrize("nq,path", [(1, "gemv"), (2, "gemv"), (4, "tensor")])
+def test_step_is_append_plus_query(nq, path):
+    # the fused step lets the scan run next to its own append; results must not change,
+    # and the rows appended in the same step must be found
+    w = W.C1.scaled(n_rows=4096, nq=nq)
+    pool, ora = fill_both(w, spare_rows=512)
+    pool2, _ = fill_both(w, spare_rows=512)
+    g = torch.Generator(device="cuda").manual_seed(11)
+    pr = fixed(8, 8, theta=-2.0)
+    pr.path = B.PATH_GEMV if path == "gemv" else B.PATH_TENSOR
+    for step in range(8):
+        n = [8, 1, 0, 33, 64, 100, 8, 2][step]      # up to 64 rows ride inside the scan kernel
+        st = torch.randn(n, w.d, generator=g, device="cuda").to(torch.bfloat16)
+        tk = torch.randint(0, 100, (n,), generator=g, device="cuda", dtype=torch.int32)
+        q = torch.randn(nq, w.d, generator=g, device="cuda").to(torch.bfloat16)
+        if n > 0:
+            q[0] = st[n - 1]          # the newest row is the best neighbour of query 0
+        a = pool.step(st, tk, q, pr, tag=70 + step)
+        pool2.append(st, tk, tag=70 + step)
+        b = pool2.query(q, pr)
+        ora.append(W.to_bits(st), tk.cpu().numpy(), tag=70 + step)
+        for f in ("idx", "score", "fired", "cont_len", "cont_tok"):
+            assert torch.equal(getattr(a, f), getattr(b, f)), (step, f)
+        if n > 0:
+            assert int(a.idx[0, 0]) == len(pool) - 1
+        check_query(a, ora, W.to_bits(q), pr)
+    assert len(pool) == len(pool2) == 4096 + 216
+    assert pool.stats()["stalled"] == 0
+    keys, tok, _ = pool.read_rows()
+    assert np.array_equal(keys, ora.keys) and np.array_equal(tok, ora.tokens)
+
+
+def test_step_back_to_back_and_small_pools():
+    # 300 fused steps without a host synchronisation in between: every step must find the
+    # row it has just appended; then a pool too small to host the append inside the scan
+    w = W.C1.scaled(n_rows=8192, nq=1)
+    pool, ora = fill_both(w, spare_rows=4096)
+    g = torch.Generator(device="cuda").manual_seed(3)
+    pr = fixed(4, 4, theta=-2.0)
+    steps = 300
+    st = torch.randn(steps, 8, w.d, generator=g, device="cuda").to(torch.bfloat16)
+    tk = torch.randint(0, 100, (steps, 8), generator=g, device="cuda", dtype=torch.int32)
+    outs = [B.QueryOut.empty(1, 4, 4, "cuda") for _ in range(steps)]
+    for s in range(steps):
+        pool.step(st[s], tk[s], st[s, 7:8].contiguous(), pr, out=outs[s], tag=500 + s,
+                  new_trace=(s % 3 == 0))
+    torch.cuda.synchronize()
+    for s in range(steps):
+        assert int(outs[s].idx[0, 0]) == 8192 + 8 * s + 7, s
+        assert abs(float(outs[s].score[0, 0]) - 1.0) < 2e-2
+    for s in range(steps):
+        ora.append(W.to_bits(st[s]), tk[s].cpu().numpy(), tag=500 + s, new_trace=(s % 3 == 0))
+    keys, tok, tid = pool.read_rows()
+    assert np.array_equal(keys, ora.keys) and np.array_equal(tok, ora.tokens)
+    check_query(pool.query(st[0, :1].contiguous(), pr), ora, W.to_bits(st[0, :1]), pr)
+    assert pool.stats()["stalled"] == 0
+
+    small = B.Pool(w.d, 256)
+    osm = oracle.OraclePool(w.d)
+    for s in range(4):
+        out = small.step(st[s], tk[s], st[s, 3:4].contiguous(), pr, tag=s)
+        osm.append(W.to_bits(st[s]), tk[s].cpu().numpy(), tag=s)
+        assert int(out.idx[0, 0]) == 8 * s + 3
+    keys, tok, _ = small.read_rows()
+    assert np.array_equal(keys, osm.keys) and np.array_equal(tok, osm.tokens)
+
+
 def test_step_host_is_append_host_plus_query_host():
     w = W.C1.scaled(n_rows=1024, nq=2)
     pool, ora = fill_both(w, spare_rows=64)

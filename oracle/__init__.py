@@ -63,6 +63,18 @@ def lib() -> ctypes.CDLL:
     L.oracle_f32_to_bf16.argtypes = [f32]
     L.oracle_pool_create.restype = vp
     L.oracle_pool_create.argtypes = [i32]
+    L.oracle_pool_create_e4m3.restype = vp
+    L.oracle_pool_create_e4m3.argtypes = [i32]
+    L.oracle_e4m3_decode.restype = ctypes.c_double
+    L.oracle_e4m3_decode.argtypes = [ctypes.c_uint8]
+    L.oracle_e4m3_encode.restype = ctypes.c_uint8
+    L.oracle_e4m3_encode.argtypes = [ctypes.c_double]
+    L.oracle_quantize_e4m3.restype = ctypes.c_int
+    L.oracle_quantize_e4m3.argtypes = [i32, vp, vp, vp]
+    for name in ("codes", "scales"):
+        fn = getattr(L, "oracle_pool_" + name)
+        fn.restype = vp
+        fn.argtypes = [vp]
     L.oracle_pool_destroy.restype = None
     L.oracle_pool_destroy.argtypes = [vp]
     L.oracle_pool_reset.restype = None
@@ -153,6 +165,23 @@ def normalize_bf16(x) -> tuple[np.ndarray, bool]:
     return out, bool(ok)
 
 
+def e4m3_decode(code: int) -> float:
+    return float(lib().oracle_e4m3_decode(int(code)))
+
+
+def e4m3_encode(x: float) -> int:
+    return int(lib().oracle_e4m3_encode(float(x)))
+
+
+def quantize_e4m3(x) -> tuple[np.ndarray, float, bool]:
+    """One raw bf16 row -> (E4M3 codes uint8 [d], fp32 scale, usable)."""
+    x = _u16(x).reshape(-1)
+    codes = np.empty(x.size, np.uint8)
+    scale = np.zeros(1, np.float32)
+    ok = lib().oracle_quantize_e4m3(x.size, _ptr(x), _ptr(codes), _ptr(scale))
+    return codes, float(scale[0]), bool(ok)
+
+
 @dataclass
 class QueryParams:
     """Retrieval parameters; defaults are the values the paper deploys."""
@@ -177,10 +206,14 @@ class QueryResult:
 
 
 class OraclePool:
-    def __init__(self, d: int):
+    def __init__(self, d: int, key_format: str = "bf16"):
         self._L = lib()
         self.d = int(d)
-        self._h = self._L.oracle_pool_create(self.d)
+        if key_format not in ("bf16", "e4m3"):
+            raise ValueError("key_format must be 'bf16' or 'e4m3'")
+        self.key_format = key_format
+        self._h = (self._L.oracle_pool_create(self.d) if key_format == "bf16"
+                   else self._L.oracle_pool_create_e4m3(self.d))
         if not self._h:
             raise MemoryError("oracle_pool_create failed")
 
@@ -216,6 +249,16 @@ class OraclePool:
     @property
     def keys(self) -> np.ndarray:
         return self._copy("keys", len(self) * self.d, np.uint16).reshape(len(self), self.d)
+
+    @property
+    def codes(self) -> np.ndarray:
+        """E4M3 codes [N,d] uint8 (8-bit pools only)."""
+        return self._copy("codes", len(self) * self.d, np.uint8).reshape(len(self), self.d)
+
+    @property
+    def scales(self) -> np.ndarray:
+        """One fp32 scale per row (8-bit pools only)."""
+        return self._copy("scales", len(self), np.float32)
 
     @property
     def tokens(self) -> np.ndarray:

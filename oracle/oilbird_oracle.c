@@ -34,7 +34,9 @@
  * Every function below is pinned by tests/test_oracle_*.py against closed
  * forms (+-1 Hamming pools), the constants the paper prints, brute force on
  * tiny pools and an independent numpy restatement; nothing is "parity
- * unpinned".
+ * unpinned".  The 8-bit store (E4M3 section) is pinned against PyTorch's own
+ * float8_e4m3fn conversions, the format's constants, a closed form and the
+ * quantiser's error bound (tests/test_oracle_q8_pins.py).
  */
 #include <math.h>
 #include <stdint.h>
@@ -66,10 +68,86 @@ uint16_t oracle_f32_to_bf16(float f) {
   return (uint16_t)(u >> 16);
 }
 
+/* ------------------------------------------------------------------ e4m3 -- */
+/*
+ * 8-bit keys for the bounded store (the paper's Limitations section names
+ * quantisation of the store as future work and fixes no format; the format
+ * here is this build's reading and is listed with the other readings).
+ *
+ * E4M3: 1 sign, 4 exponent (bias 7), 3 mantissa bits, no infinities.
+ *   exponent field e in 1..15:  (-1)^s * 2^(e-7) * (1 + m/8)
+ *   e == 0 (subnormal):         (-1)^s * 2^-6 * (m/8)
+ * Codes 0x7f and 0xff are NaN and are never produced; the largest finite
+ * magnitude is code 0x7e = 448.
+ */
+double oracle_e4m3_decode(uint8_t c) {
+  int s = c >> 7, e = (c >> 3) & 15, m = c & 7;
+  double v = e ? ldexp(1.0 + m / 8.0, e - 7) : ldexp(m / 8.0, -6);
+  if (e == 15 && m == 7) v = NAN;
+  return s ? -v : v;
+}
+
+/*
+ * Nearest E4M3 value, ties to the even code, magnitudes above 448 saturate
+ * to 448.  Done by search over the 127 finite magnitudes: plain, not fast.
+ */
+uint8_t oracle_e4m3_encode(double x) {
+  uint8_t sign = signbit(x) ? 0x80 : 0;
+  double a = fabs(x);
+  if (!(a == a)) return 0;                 /* NaN input: stored as zero        */
+  if (a >= 448.0) return (uint8_t)(sign | 0x7e);
+  uint8_t best = 0;
+  double best_err = a;                     /* code 0 (value 0)                 */
+  for (int c = 1; c <= 0x7e; ++c) {
+    double err = fabs(oracle_e4m3_decode((uint8_t)c) - a);
+    /* codes increase with magnitude, so an equal error is the upper neighbour */
+    if (err < best_err || (err == best_err && (c & 1) == 0)) { best = (uint8_t)c; best_err = err; }
+  }
+  return (uint8_t)(sign | best);
+}
+
+/*
+ * Quantise one raw bf16 state into E4M3 codes with one fp32 scale per row:
+ *   v_j   = x_j / ||x||                      (double)
+ *   scale = fp32( max_j |v_j| / 448 )
+ *   c_j   = e4m3( v_j / scale )
+ * so that v_j ~ scale * decode(c_j) and the largest entry maps to +-448.  A row
+ * that is all zero or holds a NaN/Inf is stored as zero codes with scale 0.
+ * Returns 1 if the row was usable.
+ */
+int oracle_quantize_e4m3(int32_t d, const uint16_t *x, uint8_t *codes, float *scale) {
+  double ss = 0.0, amax = 0.0;
+  int finite = 1;
+  for (int32_t j = 0; j < d; ++j) {
+    double v = (double)oracle_bf16_to_f32(x[j]);
+    if (!isfinite(v)) finite = 0;
+    ss += v * v;
+    if (fabs(v) > amax) amax = fabs(v);
+  }
+  double nrm = sqrt(ss);
+  int ok = finite && nrm > 0.0 && isfinite(nrm);
+  if (!ok) {
+    for (int32_t j = 0; j < d; ++j) codes[j] = 0;
+    *scale = 0.0f;
+    return 0;
+  }
+  double inv = 1.0 / nrm;
+  float sc = (float)(amax * inv / 448.0);
+  for (int32_t j = 0; j < d; ++j) {
+    double v = (double)oracle_bf16_to_f32(x[j]) * inv;
+    codes[j] = oracle_e4m3_encode(v / (double)sc);
+  }
+  *scale = sc;
+  return 1;
+}
+
 /* ------------------------------------------------------------------ pool -- */
 
 typedef struct {
   int32_t d;
+  int32_t fmt;              /* 0: bf16 keys; 1: E4M3 codes + one scale per row */
+  uint8_t *code;            /* fmt 1: [n][d]                                   */
+  float *scale;             /* fmt 1: [n]                                      */
   int64_t n, cap;           /* rows stored / allocated                        */
   uint16_t *key;            /* [n][d] normalised bf16 keys (Eq. 1)            */
   int32_t *tok;             /* [n]    token x_i                               */
@@ -88,9 +166,18 @@ oracle_pool *oracle_pool_create(int32_t d) {
   return p;
 }
 
+/* The same store with 8-bit keys (see the E4M3 section above). */
+oracle_pool *oracle_pool_create_e4m3(int32_t d) {
+  oracle_pool *p = oracle_pool_create(d);
+  if (p) p->fmt = 1;
+  return p;
+}
+const uint8_t *oracle_pool_codes(const oracle_pool *p) { return p->code; }
+const float *oracle_pool_scales(const oracle_pool *p) { return p->scale; }
+
 void oracle_pool_destroy(oracle_pool *p) {
   if (!p) return;
-  free(p->key); free(p->tok); free(p->trace_id);
+  free(p->key); free(p->code); free(p->scale); free(p->tok); free(p->trace_id);
   free(p->trace_start); free(p->trace_end); free(p->trace_tag);
   free(p);
 }
@@ -137,9 +224,18 @@ static int grow_rows(oracle_pool *p, int64_t need) {
   if (need <= p->cap) return 0;
   int64_t cap = p->cap ? p->cap : 1024;
   while (cap < need) cap *= 2;
-  uint16_t *k = (uint16_t *)realloc(p->key, (size_t)cap * (size_t)p->d * sizeof(uint16_t));
-  if (!k) return -1;
-  p->key = k;
+  if (p->fmt == 0) {
+    uint16_t *k = (uint16_t *)realloc(p->key, (size_t)cap * (size_t)p->d * sizeof(uint16_t));
+    if (!k) return -1;
+    p->key = k;
+  } else {
+    uint8_t *c = (uint8_t *)realloc(p->code, (size_t)cap * (size_t)p->d);
+    if (!c) return -1;
+    p->code = c;
+    float *sc = (float *)realloc(p->scale, (size_t)cap * sizeof(float));
+    if (!sc) return -1;
+    p->scale = sc;
+  }
   int32_t *t = (int32_t *)realloc(p->tok, (size_t)cap * sizeof(int32_t));
   if (!t) return -1;
   p->tok = t;
@@ -189,7 +285,10 @@ int oracle_pool_append(oracle_pool *p, const uint16_t *states, const int32_t *to
 #pragma omp parallel for schedule(static) reduction(+ : bad)
   for (int64_t r = 0; r < n; ++r) {   /* rows are independent */
     int64_t row = p->n + r;
-    int ok = oracle_normalize_bf16(p->d, states + (size_t)r * p->d, p->key + (size_t)row * p->d);
+    int ok = p->fmt == 0
+                 ? oracle_normalize_bf16(p->d, states + (size_t)r * p->d, p->key + (size_t)row * p->d)
+                 : oracle_quantize_e4m3(p->d, states + (size_t)r * p->d,
+                                        p->code + (size_t)row * p->d, p->scale + row);
     if (!ok) bad += 1;
     p->tok[row] = tokens[r];
     p->trace_id[row] = tr;
@@ -228,9 +327,16 @@ int oracle_scores(const oracle_pool *p, const uint16_t *q_raw, uint64_t exclude_
       scores[i] = -INFINITY;
       continue;
     }
-    const uint16_t *kr = p->key + (size_t)i * d;
     double acc = 0.0;
-    for (int32_t j = 0; j < d; ++j) acc += qd[j] * (double)oracle_bf16_to_f32(kr[j]);
+    if (p->fmt == 0) {
+      const uint16_t *kr = p->key + (size_t)i * d;
+      for (int32_t j = 0; j < d; ++j) acc += qd[j] * (double)oracle_bf16_to_f32(kr[j]);
+    } else {
+      /* 8-bit keys: the query stays bf16; the row's scale multiplies the exact sum */
+      const uint8_t *cr = p->code + (size_t)i * d;
+      for (int32_t j = 0; j < d; ++j) acc += qd[j] * oracle_e4m3_decode(cr[j]);
+      acc *= (double)p->scale[i];
+    }
     scores[i] = (float)acc;
   }
   free(qn); free(qd);

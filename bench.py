@@ -197,7 +197,8 @@ def run_ours(args):
     total_steps = 3 * (Wm + K) + Wm + K     # device-timed, latency, kernel-timed and e2e passes
     cap = n0 + rows_step * total_steps + 8
     pool = B.Pool(w.d, cap, max_nq=max(nq, 1), max_k=w.k, max_append=rows_step, device=local,
-                  max_traces=w.num_traces + total_steps + 8)
+                  max_traces=w.num_traces + total_steps + 8, key_format=args.keys)
+    row_bytes = w.d * 2 if args.keys == "bf16" else w.d + 4     # stored key bytes per row
     # fill the pool (not timed): seeded traces of the configuration
     done = 0
     for st, tk, tag in w.traces(dev):
@@ -296,7 +297,7 @@ def run_ours(args):
     scan_ms = pool.profile_read(max_n=max(K, 1))
     pool.profile(False)
     rows_scan = rows1 + rows_step * (K + 1) / 2.0
-    scan_bytes = rows_scan * w.d * 2
+    scan_bytes = rows_scan * row_bytes
     peaks, peak_kind = measured_peaks()
     scan_mean_ms = float(scan_ms.mean()) if len(scan_ms) else float("nan")
     achieved = scan_bytes / (scan_mean_ms * 1e-3) / 1e9
@@ -308,9 +309,9 @@ def run_ours(args):
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K,
             "warmup": Wm, "ms_per_step": max_ms / K, "higher_is_better": True,
-            "scaling": "weak", "vs_baseline": None, "dtype": "bf16 keys, fp32 accumulate",
+            "scaling": "weak", "vs_baseline": None, "dtype": f"{args.keys} keys, fp32 accumulate",
             "data": "synthetic",
-            "config": {"workload": f"{w.name}: pool N={n0} x d={w.d} bf16, nq={nq}, k={w.k}, "
+            "config": {"workload": f"{w.name}: pool N={n0} x d={w.d} {args.keys}, nq={nq}, k={w.k}, "
                                    f"L={w.cont_len}, +{rows_step} rows appended per step",
                        "pool_rows_start": rows0, "pool_rows_end": rows0 + rows_step * K,
                        "append_rows_per_step": rows_step, "scan_path": args.path,
@@ -322,7 +323,7 @@ def run_ours(args):
             "min_query_latency_us": float(lat.min()) * 1e3,
             "latency_note": "per-step latencies come from a pass of their own with an event "
                             "after every step (which serialises consecutive steps)",
-            "key_scan_gbs": rows_mean * w.d * 2 / (max_ms / K * 1e-3) / 1e9,
+            "key_scan_gbs": rows_mean * row_bytes / (max_ms / K * 1e-3) / 1e9,
             "clocks": clocks,
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d,
                     "d2h_bytes_per_step": d2h},
@@ -332,12 +333,12 @@ def run_ours(args):
                          "peak_kind": peak_kind, "frac_of_nominal_8000": achieved / NOMINAL_HBM_GBS,
                          "kernel": "key scan (score + per-CTA top-k)",
                          "kernel_ms": scan_mean_ms, "bytes_per_launch": scan_bytes,
-                         "traffic": ncu_traffic(w.name, rows_scan) if not args.rows and not args.nq
-                         else None},
+                         "traffic": ncu_traffic(w.name, rows_scan)
+                         if not args.rows and not args.nq and args.keys == "bf16" else None},
             "device_stalled_flag": stalled,
         }
         n_pad = (nq + 15) // 16 * 16
-        used_tensor = args.path == 2 or (args.path == 0 and nq > 2)
+        used_tensor = args.keys == "bf16" and (args.path == 2 or (args.path == 0 and nq > 2))
         if used_tensor:
             # the batched path is a dense contraction: report its tensor-pipe share too
             # (2*N*d*n_pad flops per launch, queries padded to the MMA's N)
@@ -369,7 +370,8 @@ def run_ours(args):
                                          "top1_continuation_match": float(np.mean(match)),
                                          "queries": len(match)}
         if not args.no_cpu_baseline and world == 1:
-            line["cpu_baseline"] = cpu_baseline(w, n0, rows_step, nq, budget_s=args.cpu_budget)
+            line["cpu_baseline"] = cpu_baseline(w, n0, rows_step, nq, budget_s=args.cpu_budget,
+                                                keys=args.keys)
         print(json.dumps(line), flush=True)
     pool.close()
     if world > 1:
@@ -378,9 +380,9 @@ def run_ours(args):
 
 # ---------------------------------------------------------------- CPU oracle ----
 
-def oracle_pool_for(w: W.Workload, n_rows: int):
+def oracle_pool_for(w: W.Workload, n_rows: int, keys: str = "bf16"):
     import oracle
-    ora = oracle.OraclePool(w.d)
+    ora = oracle.OraclePool(w.d, keys)
     done = 0
     for st, tk, tag in w.traces("cpu"):
         if done >= n_rows:
@@ -392,7 +394,7 @@ def oracle_pool_for(w: W.Workload, n_rows: int):
     return ora
 
 
-def cpu_baseline(w, n0, rows_step, nq, budget_s=20.0, steps=None, warmup=1):
+def cpu_baseline(w, n0, rows_step, nq, budget_s=20.0, steps=None, warmup=1, keys="bf16"):
     """Time the oracle as it stands on the host cores, on a bounded sample of the workload.
 
     The sample is a prefix of the pool (whole traces) small enough that the run fits the
@@ -403,7 +405,7 @@ def cpu_baseline(w, n0, rows_step, nq, budget_s=20.0, steps=None, warmup=1):
     cores = oracle.num_threads()
     # probe: cost per row-scan on a small pool
     probe_rows = min(n0, max(2048, (1 << 26) // (w.d * 2)))
-    ora = oracle_pool_for(w, probe_rows)
+    ora = oracle_pool_for(w, probe_rows, keys)
     q, _ = w.queries("cpu", nq=1)
     qb = W.to_bits(q)
     pr = oracle.QueryParams(k=w.k, theta=0.8, depth_mode=oracle.DEPTH_FIXED, cont_len=w.cont_len)
@@ -417,7 +419,7 @@ def cpu_baseline(w, n0, rows_step, nq, budget_s=20.0, steps=None, warmup=1):
     rows = max(w.rows_per_trace, rows // w.rows_per_trace * w.rows_per_trace)
     rows = min(rows, n0)
     if rows != probe_rows:
-        ora = oracle_pool_for(w, rows)
+        ora = oracle_pool_for(w, rows, keys)
     states, toks, queries = step_inputs(w, n_steps + warmup, rows_step, nq_s, "cpu", seed=0)
     def step(i):
         ora.append(W.to_bits(states[i]), toks[i].numpy(), tag=1_000_000 + i)
@@ -443,7 +445,7 @@ def run_reference(args):
     nq = args.nq or w.nq
     n0 = W.C5_START_ROWS if w.name == "C5" else w.n_rows
     cb = cpu_baseline(w, n0, APPEND_ROWS[w.name], nq, budget_s=args.cpu_budget * 4,
-                      steps=args.steps, warmup=args.warmup)
+                      steps=args.steps, warmup=args.warmup, keys=args.keys)
     line = {"impl": "reference", "metric": METRIC, "value": cb["value"], "unit": UNIT,
             "n_gpus": env_int("WORLD_SIZE", 1), "steps": args.steps, "warmup": args.warmup,
             "ms_per_step": cb["ms_per_step"], "higher_is_better": True, "scaling": "weak",
@@ -691,6 +693,9 @@ def main():
     ap.add_argument("--rows", type=int, default=0,
                     help="override the pool size (profiling a smaller case of the same recipe)")
     ap.add_argument("--path", type=int, default=0, help="0 auto, 1 CUDA-core scan, 2 tensor scan")
+    ap.add_argument("--keys", default="bf16", choices=["bf16", "e4m3"],
+                    help="stored key format: the paper's 16-bit keys, or the bounded-store "
+                         "variant with 8-bit keys (FP8 E4M3 + one scale per row)")
     ap.add_argument("--workload", default="pool", choices=["pool", "ring", "merge"],
                     help="pool: the trace-store query path (default); ring: the recycled pool")
     ap.add_argument("--sharded", action="store_true",

@@ -43,6 +43,10 @@ extern "C" {
 #define OILBIRD_MAX_CONT_LEN  128   /* tokens per continuation                         */
 #define OILBIRD_MAX_TIERS     4
 
+/* pool flags (oilbird_pool_config.flags) */
+#define OILBIRD_KEYS_E4M3  1u   /* keys are stored as FP8 E4M3 codes with one fp32 scale
+                                   per row instead of bf16 (see "8-bit keys" below)     */
+
 /* append flags */
 #define OILBIRD_NEW_TRACE  1u   /* the rows open a new trace (a finished request)      */
 
@@ -69,7 +73,7 @@ typedef struct {
   int32_t  max_k;          /* largest k (<= OILBIRD_MAX_K); 0 = 64                      */
   int32_t  max_append;     /* largest n of the *_host append variant; 0 = 4096          */
   int32_t  device;         /* CUDA ordinal                                              */
-  uint32_t flags;          /* reserved, 0                                               */
+  uint32_t flags;          /* 0 or OILBIRD_KEYS_E4M3                                    */
   void*    arena;          /* dev, optional: caller-provided memory (256-B aligned) of  */
   size_t   arena_bytes;    /*   at least oilbird_pool_arena_bytes(); NULL = cudaMalloc  */
 } oilbird_pool_config;
@@ -220,6 +224,22 @@ int oilbird_pool_status(oilbird_pool_t* pool, oilbird_pool_stats* stats, void* c
  * keys: [n,d] bf16; tokens, trace_ids: [n] int32; rows [row0, row0+n). */
 int oilbird_pool_read_rows(oilbird_pool_t* pool, int64_t row0, int64_t n, void* keys_host,
                            int32_t* tokens_host, int32_t* trace_ids_host);
+/*
+ * 8-bit keys (OILBIRD_KEYS_E4M3).  The paper's Limitations section names quantisation as one
+ * way to keep the store bounded and defines none; this is the library's format.  A stored
+ * row is d FP8 E4M3 codes c_j and one fp32 scale:
+ *     v_j = x_j / ||x||,   scale = fp32(max_j |v_j| / 448),   c_j = e4m3(v_j / scale)
+ * (round to nearest, ties to the even code, saturating at +-448; a zero or non-finite row is
+ * stored as zero codes with scale 0).  A score is fp32(scale * sum_j qn_j * value(c_j)), the
+ * query normalised and rounded to bf16 as for 16-bit pools; everything after the scores is
+ * unchanged.  A row takes d + 4 bytes instead of 2d.  d must be a multiple of 16.  Such
+ * pools use the CUDA-core scan for every nq (OILBIRD_PATH_TENSOR is rejected),
+ * oilbird_query_static does not apply, and keys are read back with the call below
+ * (oilbird_pool_read_rows then takes keys_host == NULL).
+ * codes: [n,d] uint8; scales: [n] fp32; either may be NULL.
+ */
+int oilbird_pool_read_codes(oilbird_pool_t* pool, int64_t row0, int64_t n, uint8_t* codes_host,
+                            float* scales_host);
 /* Trace table as the host tracks it: up to max_traces entries each; returns the count. */
 int32_t oilbird_pool_read_traces(const oilbird_pool_t* pool, int64_t* start, int64_t* end,
                                  uint64_t* tag, int32_t max_traces);

@@ -19,6 +19,7 @@ LIB_PATH = os.path.join(_HERE, "liboilbird.so")
 
 OK, EINVAL, ECAPACITY, ENOMEM, ECUDA, ESTALL = 0, -1, -2, -3, -4, -5
 NEW_TRACE = 1
+KEYS_E4M3 = 1          # pool flag: 8-bit keys
 DEPTH_FIXED, DEPTH_TIERED = 0, 1
 PATH_AUTO, PATH_GEMV, PATH_TENSOR = 0, 1, 2
 MAX_NQ, MAX_K, MAX_CONT_LEN, MAX_TIERS = 256, 128, 128, 4
@@ -98,6 +99,7 @@ SYMBOLS = {
     "oilbird_pool_num_traces": (_i32, [_vp]),
     "oilbird_pool_status": (ctypes.c_int, [_vp, ctypes.POINTER(PoolStats), _vp]),
     "oilbird_pool_read_rows": (ctypes.c_int, [_vp, _i64, _i64, _vp, _vp, _vp]),
+    "oilbird_pool_read_codes": (ctypes.c_int, [_vp, _i64, _i64, _vp, _vp]),
     "oilbird_pool_read_traces": (_i32, [_vp, _vp, _vp, _vp, _i32]),
     "oilbird_pool_profile": (ctypes.c_int, [_vp, _i32]),
     "oilbird_pool_profile_read": (_i32, [_vp, _vp, _i32]),
@@ -270,13 +272,19 @@ class Pool:
     """A semantic draft pool on one GPU (one per tenant)."""
 
     def __init__(self, d: int, capacity_rows: int, *, max_traces: int = 0, max_nq: int = 0,
-                 max_k: int = 0, max_append: int = 0, device: int = 0, use_torch_arena=False):
+                 max_k: int = 0, max_append: int = 0, device: int = 0, use_torch_arena=False,
+                 key_format: str = "bf16"):
+        """key_format: "bf16" (the paper's store) or "e4m3" (8-bit keys, one scale per row)."""
         self._L = lib()
+        if key_format not in ("bf16", "e4m3"):
+            raise ValueError("key_format must be 'bf16' or 'e4m3'")
+        self.key_format = key_format
         if not torch.cuda.is_available():
             raise RuntimeError("oilbird pool needs a CUDA device; there is no CPU fallback")
         self.d, self.device = int(d), int(device)
         cfg = PoolConfig(d=d, capacity_rows=capacity_rows, max_traces=max_traces, max_nq=max_nq,
-                         max_k=max_k, max_append=max_append, device=device, flags=0,
+                         max_k=max_k, max_append=max_append, device=device,
+                         flags=KEYS_E4M3 if key_format == "e4m3" else 0,
                          arena=None, arena_bytes=0)
         self._arena = None
         if use_torch_arena:
@@ -462,12 +470,23 @@ class Pool:
     def read_rows(self, row0: int = 0, n: int | None = None):
         """(keys uint16 [n,d], tokens int32 [n], trace_ids int32 [n]) as numpy arrays."""
         n = len(self) - row0 if n is None else n
-        keys = np.empty((n, self.d), dtype=np.uint16)
+        keys = np.empty((n, self.d), dtype=np.uint16) if self.key_format == "bf16" else None
         tok = np.empty(n, dtype=np.int32)
         tid = np.empty(n, dtype=np.int32)
-        _check(self._L.oilbird_pool_read_rows(self._h, row0, n, keys.ctypes.data, tok.ctypes.data,
-                                              tid.ctypes.data), "oilbird_pool_read_rows")
+        _check(self._L.oilbird_pool_read_rows(self._h, row0, n,
+                                              keys.ctypes.data if keys is not None else None,
+                                              tok.ctypes.data, tid.ctypes.data),
+               "oilbird_pool_read_rows")
         return keys, tok, tid
+
+    def read_codes(self, row0: int = 0, n: int | None = None):
+        """8-bit pools: (codes uint8 [n,d], scales float32 [n]) as numpy arrays."""
+        n = len(self) - row0 if n is None else n
+        codes = np.empty((n, self.d), dtype=np.uint8)
+        scales = np.empty(n, dtype=np.float32)
+        _check(self._L.oilbird_pool_read_codes(self._h, row0, n, codes.ctypes.data,
+                                               scales.ctypes.data), "oilbird_pool_read_codes")
+        return codes, scales
 
     def traces(self):
         """(start int64 [T], end int64 [T], tag uint64 [T]) as the host tracks them."""

@@ -115,6 +115,18 @@ cudaError_t launch_scan_gemv(const PoolView& pv, const uint16_t* q_raw, int32_t 
                              int32_t num_sms, int32_t* n_lists, const FusedAppend* fused,
                              cudaStream_t st);
 
+// The same two steps for pools with 8-bit keys (E4M3 codes, one fp32 scale per row).
+cudaError_t launch_append_e4m3(const uint16_t* states, const int32_t* tokens, int64_t n, int32_t d,
+                               uint8_t* codes, float* scales, int32_t* tok, int32_t* trace_id,
+                               int64_t row0, int32_t trace, int32_t* trace_end,
+                               uint64_t* trace_tag, uint64_t tag, int64_t* trace_gbase,
+                               int64_t gbase, int set_tag, DeviceStats* stats, cudaStream_t st);
+cudaError_t launch_scan_gemv_e4m3(const uint8_t* codes, const float* scales, const PoolView& pv,
+                                  const uint16_t* q_raw, int32_t nq, int32_t k, int32_t kk,
+                                  const uint64_t* exclude_tag, unsigned long long* partial,
+                                  int32_t* q_valid, DeviceStats* stats, int32_t max_lists,
+                                  int32_t num_sms, int32_t* n_lists, cudaStream_t st);
+
 // CTAs the CUDA-core scan launches for a pool of n_rows rows.
 inline int32_t scan_gemv_grid(int64_t n_rows, int32_t num_sms, int32_t max_lists) {
   // at least 32 rows per CTA, at most two CTAs per SM

@@ -33,12 +33,13 @@ size_t align_up(size_t v) { return (v + kAlign - 1) / kAlign * kAlign; }
 struct Layout {
   size_t keys, tok, trace_id, trace_end, trace_tag, trace_gbase, qn, q_valid, partial, stats;
   size_t xchg;
-  size_t q_stage, ex_stage, st_stage, tok_stage, stage_end, fuse_ready;
+  size_t q_stage, ex_stage, st_stage, tok_stage, stage_end, fuse_ready, scales;
   size_t total;
 };
 
 struct Resolved {
   int32_t d, max_traces, max_nq, max_k, max_append, max_lists;
+  int32_t e4m3;              // keys are E4M3 codes with one scale per row
   int64_t capacity;
 };
 
@@ -46,6 +47,9 @@ bool resolve(const oilbird_pool_config* c, int num_sms, Resolved* r) {
   if (!c) return false;
   if (c->d < 8 || c->d > 16384 || (c->d % 8) != 0) return false;
   if (c->capacity_rows < 1 || c->capacity_rows > 2147483000LL) return false;
+  if (c->flags & ~(uint32_t)OILBIRD_KEYS_E4M3) return false;
+  r->e4m3 = (c->flags & OILBIRD_KEYS_E4M3) ? 1 : 0;
+  if (r->e4m3 && (c->d % 16) != 0) return false;      // 16 codes per 16-byte load
   r->d = c->d;
   r->capacity = c->capacity_rows;
   int64_t mt = c->max_traces > 0 ? c->max_traces
@@ -68,7 +72,8 @@ Layout make_layout(const Resolved& r) {
   auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes); return o; };
   const size_t nq_pad = (size_t)(r.max_nq + 15) / 16 * 16;
   const size_t k_pad = (size_t)list_len(r.max_k);
-  L.keys = take((size_t)r.capacity * r.d * 2);
+  L.keys = take((size_t)r.capacity * r.d * (r.e4m3 ? 1 : 2));
+  L.scales = take(r.e4m3 ? (size_t)r.capacity * 4 : 0);
   L.tok = take((size_t)r.capacity * 4);
   L.trace_id = take((size_t)r.capacity * 4);
   L.trace_end = take((size_t)r.max_traces * 4);
@@ -98,7 +103,9 @@ struct oilbird_pool {
   bool owns_mem;
   unsigned char* base;
   // device arrays
-  uint16_t* keys;
+  uint16_t* keys;            // bf16 keys, or ...
+  uint8_t* codes;            // ... E4M3 codes (the same memory) with ...
+  float* scales;             // ... one scale per row
   int32_t *tok, *trace_id, *trace_end;
   uint64_t* trace_tag;
   int64_t* trace_gbase;      // global position of each trace's first row (row sharding)
@@ -198,6 +205,8 @@ int oilbird_pool_create(oilbird_pool_t** out, const oilbird_pool_config* cfg) {
     p->owns_mem = true;
   }
   p->keys = (uint16_t*)(p->base + lay.keys);
+  p->codes = (uint8_t*)(p->base + lay.keys);
+  p->scales = (float*)(p->base + lay.scales);
   p->tok = (int32_t*)(p->base + lay.tok);
   p->trace_id = (int32_t*)(p->base + lay.trace_id);
   p->trace_end = (int32_t*)(p->base + lay.trace_end);
@@ -218,7 +227,7 @@ int oilbird_pool_create(oilbird_pool_t** out, const oilbird_pool_config* cfg) {
     return cuda_fail(e, "cudaMemset(stats)");
   }
   p->smem_limit = prop.sharedMemPerBlockOptin;
-  p->tc = prop.major == 10 ? tc_cache_create(p->keys, r.capacity, r.d, p->qn,
+  p->tc = (prop.major == 10 && !r.e4m3) ? tc_cache_create(p->keys, r.capacity, r.d, p->qn,
                                              (r.max_nq + 15) / 16 * 16)
                            : nullptr;
   *out = p;
@@ -292,10 +301,17 @@ static int append_impl(oilbird_pool_t* p, const void* states, const int32_t* tok
   int rc = append_prepare(p, states, tokens, n, tag, flags, &ap, &nothing);
   if (rc || nothing) return rc;
   CU(cudaSetDevice(p->device));
-  cudaError_t e = launch_append((const uint16_t*)states, tokens, n, p->r.d, p->keys, p->tok,
-                                p->trace_id, ap.row0, ap.trace, p->trace_end, p->trace_tag, tag,
-                                p->trace_gbase, global_row >= 0 ? global_row : ap.row0,
-                                ap.open_new ? 1 : 0, p->stats, (cudaStream_t)stream);
+  const int64_t gbase = global_row >= 0 ? global_row : ap.row0;
+  cudaError_t e =
+      p->r.e4m3
+          ? launch_append_e4m3((const uint16_t*)states, tokens, n, p->r.d, p->codes, p->scales,
+                               p->tok, p->trace_id, ap.row0, ap.trace, p->trace_end, p->trace_tag,
+                               tag, p->trace_gbase, gbase, ap.open_new ? 1 : 0, p->stats,
+                               (cudaStream_t)stream)
+          : launch_append((const uint16_t*)states, tokens, n, p->r.d, p->keys, p->tok,
+                          p->trace_id, ap.row0, ap.trace, p->trace_end, p->trace_tag, tag,
+                          p->trace_gbase, gbase, ap.open_new ? 1 : 0, p->stats,
+                          (cudaStream_t)stream);
   if (e != cudaSuccess) {
     append_rollback(p, ap);
     return cuda_fail(e, "append kernel launch");
@@ -384,7 +400,9 @@ static int query_impl(oilbird_pool_t* p, const void* q, int32_t nq, const oilbir
   PoolView pv = view_of(p);
   cudaError_t e;
 
-  const int path = resolve_path(pr, nq);
+  const int path = p->r.e4m3 && pr->path == OILBIRD_PATH_AUTO ? OILBIRD_PATH_GEMV
+                                                              : resolve_path(pr, nq);
+  if (path == OILBIRD_PATH_TENSOR && p->r.e4m3) return OILBIRD_EINVAL;   // 16-bit pools only
   if (path == OILBIRD_PATH_TENSOR && !p->tc) {
     snprintf(g_cuda_err, sizeof g_cuda_err, "tensor-core scan unavailable on this device");
     return OILBIRD_ECUDA;
@@ -408,7 +426,13 @@ static int query_impl(oilbird_pool_t* p, const void* q, int32_t nq, const oilbir
       e0 = p->ev[p->ev_used]; e1 = p->ev[p->ev_used + 1];
       CU(cudaEventRecord(e0, st));
     }
-    if (path == OILBIRD_PATH_GEMV) {
+    if (p->r.e4m3) {
+      e = launch_scan_gemv_e4m3(p->codes, p->scales, pv, (const uint16_t*)q, nq, pr->k, kk,
+                                pr->exclude_tag, p->partial, p->q_valid, p->stats, p->r.max_lists,
+                                p->num_sms, &n_lists, st);
+      if (e != cudaSuccess) return cuda_fail(e, "8-bit scan kernel launch");
+      p->launches += 1;
+    } else if (path == OILBIRD_PATH_GEMV) {
       e = launch_scan_gemv(pv, (const uint16_t*)q, nq, pr->k, kk, pr->exclude_tag, p->partial,
                            p->q_valid, p->stats, p->r.max_lists, p->num_sms, &n_lists, fused, st);
       if (e != cudaSuccess) return cuda_fail(e, "scan kernel launch");
@@ -455,7 +479,8 @@ static int step_impl(oilbird_pool_t* p, const void* states, const int32_t* token
   int rc = check_params(p, nq, pr, &gp);          // nothing is appended if the query is invalid
   if (rc) return rc;
   const int64_t rows_after = p->n_rows + n;
-  const bool fuse = n >= 1 && n <= kFuseMaxRows && resolve_path(pr, nq) == OILBIRD_PATH_GEMV &&
+  const bool fuse = !p->r.e4m3 && n >= 1 && n <= kFuseMaxRows &&
+                    resolve_path(pr, nq) == OILBIRD_PATH_GEMV &&
                     scan_gemv_grid(rows_after, p->num_sms, p->r.max_lists) >= n;
   if (!fuse) {
     rc = append_impl(p, states, tokens, n, tag, flags, -1, stream);
@@ -690,6 +715,7 @@ int oilbird_pool_read_rows(oilbird_pool_t* p, int64_t row0, int64_t n, void* key
   if (!p || row0 < 0 || n < 0 || row0 + n > p->n_rows) return OILBIRD_EINVAL;
   CU(cudaSetDevice(p->device));
   CU(cudaDeviceSynchronize());
+  if (keys && p->r.e4m3) return OILBIRD_EINVAL;       // 8-bit pool: oilbird_pool_read_codes
   if (n == 0) return OILBIRD_OK;
   if (keys)
     CU(cudaMemcpy(keys, p->keys + (size_t)row0 * p->r.d, (size_t)n * p->r.d * 2,
@@ -697,6 +723,19 @@ int oilbird_pool_read_rows(oilbird_pool_t* p, int64_t row0, int64_t n, void* key
   if (tokens) CU(cudaMemcpy(tokens, p->tok + row0, (size_t)n * 4, cudaMemcpyDeviceToHost));
   if (trace_ids)
     CU(cudaMemcpy(trace_ids, p->trace_id + row0, (size_t)n * 4, cudaMemcpyDeviceToHost));
+  return OILBIRD_OK;
+}
+
+int oilbird_pool_read_codes(oilbird_pool_t* p, int64_t row0, int64_t n, uint8_t* codes,
+                            float* scales) {
+  if (!p || !p->r.e4m3 || row0 < 0 || n < 0 || row0 + n > p->n_rows) return OILBIRD_EINVAL;
+  CU(cudaSetDevice(p->device));
+  CU(cudaDeviceSynchronize());
+  if (n == 0) return OILBIRD_OK;
+  if (codes)
+    CU(cudaMemcpy(codes, p->codes + (size_t)row0 * p->r.d, (size_t)n * p->r.d,
+                  cudaMemcpyDeviceToHost));
+  if (scales) CU(cudaMemcpy(scales, p->scales + row0, (size_t)n * 4, cudaMemcpyDeviceToHost));
   return OILBIRD_OK;
 }
 

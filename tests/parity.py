@@ -41,7 +41,7 @@ def fill_both(w: W.Workload, device="cuda", n_rows=None, chunk_traces=64, **pool
     """Materialise workload w on `device`, append it to a CUDA pool and to the oracle."""
     n_rows = w.n_rows if n_rows is None else n_rows
     pool = B.Pool(w.d, n_rows + pool_kw.pop("spare_rows", 0), **pool_kw)
-    ora = OraclePool(w.d)
+    ora = OraclePool(w.d, pool.key_format)
     done = 0
     for st, tk, tag in w.traces(device):
         if done >= n_rows:

@@ -1,0 +1,150 @@
+"""GPU parity for pools with 8-bit keys (FP8 E4M3 codes + one fp32 scale per row): stored
+codes and scales bit-exact against the oracle, scores / neighbours / continuations under the
+same acceptance rule as the 16-bit pool (tests/parity.py)."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from oracle import OraclePool
+from paper_2608_03839_b200 import binding as B
+from paper_2608_03839_b200 import workloads as W
+from parity import check_query, fill_both
+
+pytestmark = pytest.mark.gpu
+
+
+def fixed(k, L, theta=0.8, **kw):
+    return B.QueryParams(k=k, theta=theta, depth_mode=B.DEPTH_FIXED, cont_len=L, **kw)
+
+
+def bits_to_dev(bits: np.ndarray) -> torch.Tensor:
+    return torch.from_numpy(bits.view(np.int16)).view(torch.bfloat16).cuda()
+
+
+@pytest.mark.parametrize("d", [16, 208, 256, 4096, 8192])
+def test_codes_and_scales_match_oracle_bit_for_bit(d):
+    g = torch.Generator(device="cuda").manual_seed(d)
+    n = 300
+    st = (torch.randn(n, d, generator=g, device="cuda") * 3).to(torch.bfloat16)
+    st[7] = 0                                   # zero row
+    st[11, d // 2] = float("inf")               # non-finite rows are stored as zero codes
+    st[13, 0] = float("nan")
+    st[17] = st[17] * 1e-30                     # tiny but usable
+    st[19, 1:] = 0                              # one-hot: the peak is the only entry
+    st[23] = torch.where(st[23].abs() < 2.0, torch.zeros_like(st[23]), st[23])   # many exact zeros
+    st[29, : d // 2] *= 1e-3                    # half the row lands in the subnormal codes
+    st[31] = -st[31].abs()                      # all negative
+    tok = torch.arange(n, dtype=torch.int32, device="cuda")
+    pool = B.Pool(d, n, key_format="e4m3")
+    ora = OraclePool(d, "e4m3")
+    pool.append(st[:100].contiguous(), tok[:100].contiguous(), tag=1)
+    pool.append(st[100:].contiguous(), tok[100:].contiguous(), tag=2, new_trace=False)
+    ora.append(W.to_bits(st), tok.cpu().numpy(), tag=1)
+    codes, scales = pool.read_codes()
+    assert np.array_equal(scales.view(np.uint32), ora.scales.view(np.uint32))
+    assert np.array_equal(codes, ora.codes)
+    _, tk, _ = pool.read_rows()
+    assert np.array_equal(tk, ora.tokens)
+    assert pool.stats()["degenerate_rows"] == 3
+    assert not codes[7].any() and scales[7] == 0
+
+
+@pytest.mark.parametrize("d", [16, 64, 256, 1024, 4096])
+def test_closed_form_pool_scores_are_exact(d):
+    # +-1 rows: every code is +-448 and s = (1 - 2 Hamming / d) * (scale * 448 * sqrt(d)), the
+    # partial sums are small integers times a power of two, so fp32 accumulation is exact too
+    rng = np.random.default_rng(d)
+    n = 600
+    rows = rng.choice([-1.0, 1.0], size=(n, d)).astype(np.float32)
+    q = rng.choice([-1.0, 1.0], size=(2, d)).astype(np.float32)
+    rows[5] = q[0]; rows[300] = q[0]; rows[599] = q[0]        # a three-way tie at the top
+    rows[17] = -q[1]
+    pool = B.Pool(d, n, key_format="e4m3")
+    ora = OraclePool(d, "e4m3")
+    rb = oracle.f32_to_bf16_bits(rows)
+    tok = np.arange(n, dtype=np.int32)
+    pool.append(bits_to_dev(rb), torch.from_numpy(tok).cuda(), tag=1)
+    ora.append(rb, tok, tag=1)
+    qb = oracle.f32_to_bf16_bits(q)
+    pr = fixed(8, 2, theta=-2.0)
+    out = pool.query(bits_to_dev(qb), pr).cpu()
+    ref = ora.query(qb, oracle.QueryParams(k=8, theta=-2.0, depth_mode=oracle.DEPTH_FIXED, cont_len=2))
+    assert out.idx.numpy().tolist() == ref.idx.tolist()
+    assert np.array_equal(out.score.numpy(), ref.score)
+    assert out.idx[0, :3].tolist() == [5, 300, 599]
+    assert np.array_equal(out.cont_tok.numpy(), ref.cont_tok)
+
+
+@pytest.mark.parametrize("nq,k", [(1, 8), (2, 16), (5, 8), (3, 64), (2, 128)])
+def test_query_matches_oracle(nq, k):
+    w = W.C1.scaled(n_rows=6000, nq=nq)
+    pool, ora = fill_both(w, key_format="e4m3", max_k=k)
+    q, _ = w.queries("cuda", nq=nq)
+    for pr in (fixed(k, 8), fixed(k, 8, theta=-2.0),
+               B.QueryParams(k=k, cont_len=48)):               # the paper's tiers
+        check_query(pool.query(q, pr), ora, W.to_bits(q), pr)
+    assert pool.stats()["stalled"] == 0
+
+
+def test_wide_rows_exclusion_tags_and_step():
+    w = W.C2.scaled(n_rows=3000, nq=2)
+    pool, ora = fill_both(w, key_format="e4m3", spare_rows=64)
+    q, _ = w.queries("cuda", nq=2)
+    tags = [t for _, _, t in w.traces("cpu")][:2]
+    ex = torch.tensor([tags[0], 0], dtype=torch.int64, device="cuda")
+    pr = fixed(16, 16, theta=-2.0)
+    pr.exclude_tag = ex
+    check_query(pool.query(q, pr), ora, W.to_bits(q), pr, exclude=ex.cpu().numpy().astype(np.uint64))
+    # one serving step: the newest row must be found (separate append kernel for 8-bit pools)
+    g = torch.Generator(device="cuda").manual_seed(2)
+    st = torch.randn(8, w.d, generator=g, device="cuda").to(torch.bfloat16)
+    tk = torch.arange(8, dtype=torch.int32, device="cuda")
+    pr2 = fixed(4, 4, theta=-2.0)
+    out = pool.step(st, tk, st[7:8].contiguous(), pr2, tag=999)
+    ora.append(W.to_bits(st), tk.cpu().numpy(), tag=999)
+    assert int(out.idx[0, 0]) == len(pool) - 1
+    check_query(out, ora, W.to_bits(st[7:8]), pr2)
+
+
+def test_limits_of_8bit_pools():
+    with pytest.raises(B.OilbirdError):
+        B.Pool(24, 100, key_format="e4m3")                       # d must be a multiple of 16
+    pool = B.Pool(64, 256, key_format="e4m3")
+    st = torch.randn(40, 64, device="cuda").to(torch.bfloat16)
+    pool.append(st, torch.arange(40, dtype=torch.int32, device="cuda"))
+    pr = fixed(4, 4)
+    pr.path = B.PATH_TENSOR
+    with pytest.raises(B.OilbirdError):
+        pool.query(st[:4].contiguous(), pr)                      # no tensor-core scan for 8-bit keys
+    keys, tok, tid = pool.read_rows()
+    assert keys is None and tok.shape == (40,)
+    pool16 = B.Pool(64, 256)
+    pool16.append(st, torch.arange(40, dtype=torch.int32, device="cuda"))
+    with pytest.raises(B.OilbirdError):
+        pool16.read_codes()
+    # half the key bytes: the arena of an 8-bit pool is smaller
+    a8 = B.lib().oilbird_pool_arena_bytes
+    import ctypes
+    c16 = B.PoolConfig(d=4096, capacity_rows=100000, flags=0)
+    c8 = B.PoolConfig(d=4096, capacity_rows=100000, flags=B.KEYS_E4M3)
+    assert a8(ctypes.byref(c16)) - a8(ctypes.byref(c8)) >= 100000 * 4096 - 100000 * 4 - 4096
+
+
+def test_retrieval_agrees_with_the_16bit_pool_on_separated_neighbours():
+    # quantisation moves a score by < 0.02 here; neighbours that lead by more than that in
+    # the 16-bit pool must also be found in the 8-bit one
+    w = W.C2.scaled(n_rows=20000, nq=2)
+    p8, _ = fill_both(w, key_format="e4m3")
+    p16, _ = fill_both(w)
+    q, _ = w.queries("cuda", nq=2)
+    pr = fixed(16, 4, theta=-2.0)
+    a, b = p8.query(q, pr).cpu(), p16.query(q, pr).cpu()
+    for i in range(2):
+        s16 = b.score[i].numpy()
+        lead = [int(r) for r, s in zip(b.idx[i].tolist(), s16) if s > s16[-1] + 0.04]
+        assert set(lead) <= set(a.idx[i].tolist())
+        common = {int(r): float(s) for r, s in zip(b.idx[i].tolist(), s16)}
+        for r, s in zip(a.idx[i].tolist(), a.score[i].tolist()):
+            if r in common:
+                assert abs(s - common[r]) < 0.02

@@ -217,7 +217,7 @@ scan_gemv_e4m3_kernel(const uint8_t* __restrict__ codes, const float* __restrict
 #pragma unroll
         for (int q = 0; q < QT; ++q) acc[r][q] = 0.f;
 
-#pragma unroll 2
+#pragma unroll 4
       for (int c = lane; c < n16; c += 32) {
         uint4 kv[kQ8Rows];
 #pragma unroll

@@ -263,35 +263,115 @@ constexpr int kMergeWarps = kMergeThreads / 32;
 
 // Each warp folds its share of the scan's descending lists into a register-resident
 // list of kk = 32*E candidates (bitonic merges), then the warps' lists are merged.
+//
+// All of this runs on one SM, where the merges are bound by shuffle throughput (32 warps
+// folding ten lists each took 4 us), so lists that cannot matter are dropped first: a
+// list's head is its best candidate; the k-th largest of the 32 warps' best heads is
+// reached by k distinct lists, hence by k candidates, so no list whose head lies below
+// it holds one of the k best.  For k <= 32 that leaves about one list per warp.
 template <int E>
 __device__ __forceinline__ void merge_lists(const u64* __restrict__ partial, int n_lists, int nq,
-                                            int q, u64* scratch, u64* s_best) {
+                                            int q, int k, u64* scratch, u64* s_best) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   constexpr int KK = 32 * E;
+  __shared__ u64 s_head[kMergeWarps];
+  __shared__ u64 s_floor;
   u64 v[E];
 #pragma unroll
   for (int r = 0; r < E; ++r) v[r] = 0;
   // many lists in flight per warp: the loads, not the merges, set the pace (with two CTAs
   // per SM a warp folds about ten lists, so one round of loads covers the common case)
   constexpr int PF = E == 1 ? 10 : (E == 2 ? 5 : 3);
-  for (int l0 = warp; l0 < n_lists; l0 += kMergeWarps * PF) {
-    u64 b[PF][E];
+  const bool filter = k <= kMergeWarps && n_lists <= kMergeWarps * PF;   // one round of loads
+  u64 b[PF][E];
+  if (filter) {
+    u64 best = 0;
 #pragma unroll
     for (int p = 0; p < PF; ++p) {
-      const int l = l0 + p * kMergeWarps;
+      const int l = warp + p * kMergeWarps;
       const u64* src = partial + ((size_t)(l < n_lists ? l : 0) * nq + q) * KK;
 #pragma unroll
       for (int r = 0; r < E; ++r) b[p][r] = l < n_lists ? src[r * 32 + lane] : 0;
+      best = b[p][0] > best ? b[p][0] : best;            // lane 0 holds the heads
     }
+    if (lane == 0) s_head[warp] = best;
+    __syncthreads();
+    if (warp == 0) {
+      u64 h[1] = {s_head[lane]};
+      warp_sort_desc<1>(h, lane);
+      const u64 f = warp_list_get<1>(h, k - 1);          // 0 while fewer than k lists exist
+      if (lane == 0) s_floor = f;
+    }
+    __syncthreads();
+    const u64 floor_key = s_floor;
 #pragma unroll
-    for (int p = 0; p < PF; ++p)
-      if (l0 + p * kMergeWarps < n_lists) warp_merge_desc<E>(v, b[p], lane);
+    for (int p = 0; p < PF; ++p) {
+      const u64 head = warp_list_get<E>(b[p], 0);
+      if (head != 0 && head >= floor_key) warp_merge_desc<E>(v, b[p], lane);   // warp-uniform
+    }
+  } else {
+    for (int l0 = warp; l0 < n_lists; l0 += kMergeWarps * PF) {
+#pragma unroll
+      for (int p = 0; p < PF; ++p) {
+        const int l = l0 + p * kMergeWarps;
+        const u64* src = partial + ((size_t)(l < n_lists ? l : 0) * nq + q) * KK;
+#pragma unroll
+        for (int r = 0; r < E; ++r) b[p][r] = l < n_lists ? src[r * 32 + lane] : 0;
+      }
+#pragma unroll
+      for (int p = 0; p < PF; ++p)
+        if (l0 + p * kMergeWarps < n_lists) warp_merge_desc<E>(v, b[p], lane);
+    }
   }
-  const int active = n_lists < kMergeWarps ? (n_lists < 1 ? 1 : n_lists) : kMergeWarps;
-  block_merge_desc<E>(v, scratch, active);
-  if (warp == 0) {
+  // the 32 warps' lists -> one: four warps fold eight lists each as a tree of interleaved
+  // merges, then one warp folds those four (two barriers instead of ten)
 #pragma unroll
-    for (int r = 0; r < E; ++r) s_best[r * 32 + lane] = v[r];
+  for (int r = 0; r < E; ++r) scratch[(size_t)warp * KK + r * 32 + lane] = v[r];
+  __syncthreads();
+  if (warp < 4) {
+    // 8 -> 4 (two lists at a time: 1024 threads leave 64 registers each), 4 -> 2, 2 -> 1
+    u64 m[4][E];
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+      u64 a[2][E], c[2][E];
+#pragma unroll
+      for (int i = 0; i < 2; ++i)
+#pragma unroll
+        for (int r = 0; r < E; ++r) {
+          a[i][r] = scratch[(size_t)(warp * 8 + 2 * h + i) * KK + r * 32 + lane];
+          c[i][r] = scratch[(size_t)(warp * 8 + 4 + 2 * h + i) * KK + r * 32 + lane];
+        }
+      warp_merge_desc_batch<2, E>(a, c, lane);
+#pragma unroll
+      for (int r = 0; r < E; ++r) { m[2 * h][r] = a[0][r]; m[2 * h + 1][r] = a[1][r]; }
+    }
+    u64 a2[2][E], c2[2][E];
+#pragma unroll
+    for (int r = 0; r < E; ++r) { a2[0][r] = m[0][r]; a2[1][r] = m[1][r]; c2[0][r] = m[2][r]; c2[1][r] = m[3][r]; }
+    warp_merge_desc_batch<2, E>(a2, c2, lane);               // 4 -> 2
+    warp_merge_desc<E>(a2[0], a2[1], lane);                  // 2 -> 1
+#pragma unroll
+    for (int r = 0; r < E; ++r) v[r] = a2[0][r];
+  }
+  __syncthreads();
+  if (warp < 4) {
+#pragma unroll
+    for (int r = 0; r < E; ++r) scratch[(size_t)warp * KK + r * 32 + lane] = v[r];
+  }
+  __syncthreads();
+  if (warp == 0) {
+    u64 a[2][E], c[2][E];
+#pragma unroll
+    for (int r = 0; r < E; ++r) {
+      a[0][r] = scratch[r * 32 + lane];
+      a[1][r] = scratch[(size_t)KK + r * 32 + lane];
+      c[0][r] = scratch[(size_t)2 * KK + r * 32 + lane];
+      c[1][r] = scratch[(size_t)3 * KK + r * 32 + lane];
+    }
+    warp_merge_desc_batch<2, E>(a, c, lane);
+    warp_merge_desc<E>(a[0], a[1], lane);
+#pragma unroll
+    for (int r = 0; r < E; ++r) s_best[r * 32 + lane] = a[0][r];
   }
   __syncthreads();
 }

@@ -90,9 +90,9 @@ merge_gather_kernel(PoolView pv, const u64* __restrict__ partial, int n_lists, i
   pdl_launch_dependents();
   pdl_wait();   // the scan's candidate lists
   const int valid = q_valid[q];       // consumed after the merge: the load overlaps it
-  if (kk == 32) merge_lists<1>(partial, n_lists, nq, q, scratch, s_best);
-  else if (kk == 64) merge_lists<2>(partial, n_lists, nq, q, scratch, s_best);
-  else merge_lists<4>(partial, n_lists, nq, q, scratch, s_best);
+  if (kk == 32) merge_lists<1>(partial, n_lists, nq, q, k, scratch, s_best);
+  else if (kk == 64) merge_lists<2>(partial, n_lists, nq, q, k, scratch, s_best);
+  else merge_lists<4>(partial, n_lists, nq, q, k, scratch, s_best);
   for (int j = threadIdx.x; j < k; j += kMergeThreads) {
     const u64 key = valid ? s_best[j] : 0;            // NaN/Inf query: no neighbours
     const int idx = key ? candidate_row(key) : -1;

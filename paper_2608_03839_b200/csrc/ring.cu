@@ -114,7 +114,7 @@ ring_merge_kernel(const u64* __restrict__ partial, int n_lists, int nq, int m, i
   pdl_launch_dependents();
   pdl_wait();
   const int lists = q_valid[q] != 0 ? n_lists : 0;
-  merge_lists<1>(partial, lists, nq, q, scratch, s_best);
+  merge_lists<1>(partial, lists, nq, q, m, scratch, s_best);
   if (threadIdx.x == 0) {
     int c = 0;
     while (c < m && s_best[c] != 0) ++c;

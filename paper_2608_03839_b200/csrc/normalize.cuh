@@ -15,9 +15,10 @@ enum { kRowOk = 0, kRowZero = 1, kRowNonFinite = 2 };
 // double precision (products of bf16 values are exact there), the scale 1/sqrt is IEEE
 // double, each element is rounded once to float and once to bf16 (nearest even).
 // Returns kRowOk, or kRowZero / kRowNonFinite, in which case dst is all zero.
-// kHold: keep the row's chunks in registers between the two passes (one read of the row;
-// 32 registers), or read it twice (for kernels that are short of registers).
-template <bool kHold = true>
+// kHold: keep the row's first kHeld chunks per thread in registers between the two passes
+// (one read of the row up to d = kHeld * 2048), or read it twice (for kernels that are short
+// of registers).
+template <bool kHold = true, int kHeld = 4>
 __device__ __forceinline__ int normalize_row(const uint16_t* __restrict__ src, uint16_t* __restrict__ dst,
                               int d) {
   __shared__ double s_part[kNormThreads / 32];
@@ -26,10 +27,9 @@ __device__ __forceinline__ int normalize_row(const uint16_t* __restrict__ src, u
   __shared__ int s_code;
   const int n_chunks = d >> 3;
   const uint4* src4 = reinterpret_cast<const uint4*>(src);
-  // at most 8 chunks of 8 elements per thread (d <= 16384); the first kHeld of them (all
-  // of a row up to d = 8192) stay in registers so that the row is read from memory once
+  // at most 8 chunks of 8 elements per thread (d <= 16384); the first kHeld of them stay
+  // in registers so that a row of up to kHeld * 2048 elements is read from memory once
   constexpr int kMaxChunks = 16384 / 8 / kNormThreads;
-  constexpr int kHeld = 4;
   uint4 held[kHeld];
   double ss = 0.0;
   int bad = 0;

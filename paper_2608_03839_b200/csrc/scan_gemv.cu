@@ -127,7 +127,7 @@ scan_gemv_kernel(PoolView pv, const uint16_t* __restrict__ q_raw, int nq, int k,
     for (int q = 0; q < QT; ++q) {
       uint16_t* dst = reinterpret_cast<uint16_t*>(qs + (size_t)q * n_chunks);
       if (q0 + q < nq) {
-        const int code = normalize_row<false>(q_raw + (size_t)(q0 + q) * d, dst, d);
+        const int code = normalize_row<true, 2>(q_raw + (size_t)(q0 + q) * d, dst, d);
         if (blockIdx.x == 0 && threadIdx.x == 0) {
           q_valid[q0 + q] = code == kRowNonFinite ? 0 : 1;   // NaN/Inf: no neighbours
           if (code == kRowNonFinite) atomicAdd(&stats->nonfinite_queries, 1ull);

@@ -19,6 +19,17 @@
 //     during which the accumulator buffers are full and the key stream stalls;
 //   - at nq = 256 the query tile re-read from L2 per key tile (twice the key bytes) and the
 //     single k-block per accumulator set; the tensor pipe reaches about half its peak.
+// Small pools (a few tiles per SM): a query costs about 40 us plus the key bytes at HBM
+// speed, against 12 us plus the same for the CUDA-core scan.  A tile's scores exist only
+// after its whole K loop, so the first tile's latency chain is not overlapped: with eight
+// ring stages of 18 KB (nq <= 16) and a stage round trip of ~2.9 us (TMA from HBM, MMA,
+// commit, producer wake-up) one SM streams ~45-50 GB/s whatever the rest of the GPU does,
+// i.e. ~23 us per 1 MB tile, then the first tile's epilogue (7-10 us), the query
+// normalisation kernel and the merge.  Cutting the pool into per-CTA row ranges at 32-row
+// granularity (ragged ends fetched as 32-row boxes) so that all SMs get equal rows was
+// measured: no gain (the stage round trip, not the bytes, sets the pace there), as was
+// seeding the first tile's thresholds from per-warp 32-bit sorts of the scores (the sort
+// costs what the smaller crowd saves).
 // Measured and not kept: separate shared-memory rings for keys and query tiles (query
 // tiles queue behind the key requests, so they need the same lead; 5-8 % slower); a
 // 32-deep candidate queue with retry, to buy a ring stage (slower first tiles, no gain from

@@ -21,15 +21,19 @@
 //     single k-block per accumulator set; the tensor pipe reaches about half its peak.
 // Small pools (a few tiles per SM): a query costs about 40 us plus the key bytes at HBM
 // speed, against 12 us plus the same for the CUDA-core scan.  A tile's scores exist only
-// after its whole K loop, so the first tile's latency chain is not overlapped: with eight
-// ring stages of 18 KB (nq <= 16) and a stage round trip of ~2.9 us (TMA from HBM, MMA,
-// commit, producer wake-up) one SM streams ~45-50 GB/s whatever the rest of the GPU does,
-// i.e. ~23 us per 1 MB tile, then the first tile's epilogue (7-10 us), the query
-// normalisation kernel and the merge.  Cutting the pool into per-CTA row ranges at 32-row
-// granularity (ragged ends fetched as 32-row boxes) so that all SMs get equal rows was
-// measured: no gain (the stage round trip, not the bytes, sets the pace there), as was
-// seeding the first tile's thresholds from per-warp 32-bit sorts of the scores (the sort
-// costs what the smaller crowd saves).
+// after its whole K loop, so the first tile's latency chain is not overlapped, and one SM
+// streams at most ~45-65 GB/s whatever the rest of the GPU does: cycle counters in the
+// MMA-issuing thread show ~360 cycles to issue the four tcgen05.mma and the commit of a
+// 16 KB k-block (~70 cycles per instruction, against ~90 cycles of waiting for the data
+// when HBM is idle), i.e. with queries as the N operand a 128 x N x 16 instruction carries
+// only 4 KB of keys and the issue rate, not the tensor pipe, bounds the per-SM rate.  (With
+// the roles swapped, queries as M = 128 and 256 key rows as N, an instruction would carry
+// 8 KB; that is the next step for this kernel, together with an epilogue in which a thread
+// owns a query.)  Then come the first tile's epilogue (7-10 us), the query normalisation
+// kernel and the merge.  Cutting the pool into per-CTA row ranges at 32-row granularity
+// (ragged ends fetched as 32-row boxes) so that all SMs get equal rows, ring depths up to
+// 12 and seeding the first tile's thresholds from per-warp 32-bit sorts of the scores were
+// measured and bring nothing.
 // Measured and not kept: separate shared-memory rings for keys and query tiles (query
 // tiles queue behind the key requests, so they need the same lead; 5-8 % slower); a
 // 32-deep candidate queue with retry, to buy a ring stage (slower first tiles, no gain from

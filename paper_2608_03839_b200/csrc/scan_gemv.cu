@@ -188,7 +188,13 @@ scan_gemv_kernel(PoolView pv, const uint16_t* __restrict__ q_raw, int nq, int k,
         const int row = rb + r;
         if (row >= r_hi) break;                             // warp-uniform
         uint64_t tag = 0;
-        if (exclude_tag) tag = pv.trace_tag[pv.trace_id[row]];
+        if (exclude_tag) {
+          // rows appended by this launch: their trace id and tag were written by another CTA
+          // a moment ago, and this SM's L1 may hold the lines from before (it has read the
+          // neighbouring rows' entries), so those are read through L2
+          tag = (fa.n > 0 && row >= fa.row0) ? __ldcg(&pv.trace_tag[__ldcg(&pv.trace_id[row])])
+                                             : pv.trace_tag[pv.trace_id[row]];
+        }
 #pragma unroll
         for (int q = 0; q < QT; ++q) {
           const float s = warp_sum(acc[r][q]);

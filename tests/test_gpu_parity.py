@@ -365,6 +365,30 @@ def test_step_is_append_plus_query(nq, path):
     assert np.array_equal(keys, ora.keys) and np.array_equal(tok, ora.tokens)
 
 
+def test_step_with_exclusion_tags_sees_the_new_rows_tags():
+    # the rows a fused step appends carry a tag; a query of the same step that excludes that
+    # tag must not return them, and one that excludes another tag must
+    w = W.C1.scaled(n_rows=4096, nq=2)
+    pool, ora = fill_both(w, spare_rows=512)
+    g = torch.Generator(device="cuda").manual_seed(21)
+    for step in range(6):
+        n = 8
+        st = torch.randn(n, w.d, generator=g, device="cuda").to(torch.bfloat16)
+        tk = torch.randint(0, 100, (n,), generator=g, device="cuda", dtype=torch.int32)
+        q = torch.stack([st[3], st[5]]).contiguous()           # both queries equal new rows
+        tag = 9000 + step
+        ex = torch.tensor([tag, 12345], dtype=torch.int64, device="cuda")
+        pr = fixed(4, 4, theta=-2.0)
+        pr.exclude_tag = ex
+        out = pool.step(st, tk, q, pr, tag=tag, new_trace=(step % 2 == 0))
+        ora.append(W.to_bits(st), tk.cpu().numpy(), tag=tag, new_trace=(step % 2 == 0))
+        first_new = len(pool) - n
+        if step % 2 == 0:                                     # a new trace with the excluded tag
+            assert all(int(r) < first_new for r in out.idx[0].tolist())
+        assert int(out.idx[1, 0]) == first_new + 5
+        check_query(out, ora, W.to_bits(q), pr, exclude=ex.cpu().numpy().astype(np.uint64))
+
+
 def test_step_back_to_back_and_small_pools():
     # 300 fused steps without a host synchronisation in between: every step must find the
     # row it has just appended; then a pool too small to host the append inside the scan

@@ -718,9 +718,9 @@ def main():
         args.warmup = 10 if args.warmup is None else max(args.warmup, 3)
         run_merge(args)
         return
-    default_steps = {"C1": 500, "C2": 500, "C3": 300, "C4": 100, "C5": 50}[args.config]
+    default_steps = {"C1": 500, "C2": 500, "C3": 300, "C4": 200, "C5": 50}[args.config]
     args.steps = default_steps if args.steps is None else args.steps
-    args.warmup = 10 if args.warmup is None else max(args.warmup, 3)
+    args.warmup = 20 if args.warmup is None else max(args.warmup, 3)
     if args.sharded:
         run_sharded(args)
         return

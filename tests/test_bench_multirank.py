@@ -7,6 +7,7 @@ import os
 import socket
 import sys
 
+import pytest
 import torch
 import torch.distributed as dist
 import torch.multiprocessing as mp
@@ -67,3 +68,25 @@ def test_reference_arm_on_other_ranks_does_nothing(monkeypatch, capsys):
         config, nq, steps, warmup, cpu_budget = "C1", 0, 1, 1, 1.0
     bench.run_reference(A)
     assert capsys.readouterr().out == ""
+
+
+@pytest.mark.parametrize("keys", ["bf16", "e4m3"])
+def test_reference_arm_prints_one_contract_line(keys):
+    # the reference arm is the CPU oracle timed on the host cores; it needs no GPU
+    import json
+    import subprocess
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    r = subprocess.run([sys.executable, os.path.join(root, "bench.py"), "--impl", "reference",
+                        "--config", "C1", "--steps", "2", "--warmup", "1", "--keys", keys],
+                       capture_output=True, text=True, timeout=300, cwd=root)
+    assert r.returncode == 0, r.stderr[-2000:]
+    lines = [ln for ln in r.stdout.splitlines() if ln.startswith("{")]
+    assert len(lines) == 1
+    j = json.loads(lines[0])
+    assert j["impl"] == "reference" and j["metric"] == "semantic_pool_queries_per_sec"
+    assert j["unit"] == "queries/s" and j["higher_is_better"] is True and j["value"] > 0
+    assert j["n_gpus"] == 1 and j["steps"] == 2 and j["warmup"] == 1
+    assert j["cpu_baseline"]["kind"] == "oracle" and j["cpu_baseline"]["cores"] >= 1
+    assert j["e2e"] == {"value": j["value"], "unit": j["unit"], "h2d_bytes_per_step": 0,
+                        "d2h_bytes_per_step": 0}
+    assert "workload" in j["config"] and "model" not in j["config"]

@@ -125,7 +125,8 @@ cudaError_t launch_scan_gemv_e4m3(const uint8_t* codes, const float* scales, con
                                   const uint16_t* q_raw, int32_t nq, int32_t k, int32_t kk,
                                   const uint64_t* exclude_tag, unsigned long long* partial,
                                   int32_t* q_valid, DeviceStats* stats, int32_t max_lists,
-                                  int32_t num_sms, int32_t* n_lists, cudaStream_t st);
+                                  int32_t num_sms, int32_t* n_lists, const FusedAppend* fused,
+                                  cudaStream_t st);
 
 // CTAs the CUDA-core scan launches for a pool of n_rows rows.
 inline int32_t scan_gemv_grid(int64_t n_rows, int32_t num_sms, int32_t max_lists) {

@@ -429,7 +429,7 @@ static int query_impl(oilbird_pool_t* p, const void* q, int32_t nq, const oilbir
     if (p->r.e4m3) {
       e = launch_scan_gemv_e4m3(p->codes, p->scales, pv, (const uint16_t*)q, nq, pr->k, kk,
                                 pr->exclude_tag, p->partial, p->q_valid, p->stats, p->r.max_lists,
-                                p->num_sms, &n_lists, st);
+                                p->num_sms, &n_lists, fused, st);
       if (e != cudaSuccess) return cuda_fail(e, "8-bit scan kernel launch");
       p->launches += 1;
     } else if (path == OILBIRD_PATH_GEMV) {
@@ -479,8 +479,11 @@ static int step_impl(oilbird_pool_t* p, const void* states, const int32_t* token
   int rc = check_params(p, nq, pr, &gp);          // nothing is appended if the query is invalid
   if (rc) return rc;
   const int64_t rows_after = p->n_rows + n;
-  const bool fuse = !p->r.e4m3 && n >= 1 && n <= kFuseMaxRows &&
-                    resolve_path(pr, nq) == OILBIRD_PATH_GEMV &&
+  // (8-bit pools always use the CUDA-core scan; its passes beyond the first two queries
+  // would find the rows in place, but keep to the single-request case there too)
+  const bool gemv = p->r.e4m3 ? (nq <= 2 && pr->path != OILBIRD_PATH_TENSOR)
+                              : resolve_path(pr, nq) == OILBIRD_PATH_GEMV;
+  const bool fuse = n >= 1 && n <= kFuseMaxRows && gemv &&
                     scan_gemv_grid(rows_after, p->num_sms, p->r.max_lists) >= n;
   if (!fuse) {
     rc = append_impl(p, states, tokens, n, tag, flags, -1, stream);

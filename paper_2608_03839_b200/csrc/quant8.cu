@@ -13,7 +13,8 @@
 // Everything after the scan (merge, firing rule, depth, gather) is format-independent and
 // shared with the 16-bit path.  The tensor-core scan is not offered for 8-bit pools (its
 // query operand would have to be quantised to 8 bits too); batches run the CUDA-core scan
-// two queries per pass.
+// two queries per pass.  As in the 16-bit scan, the rows of a serving step can be appended
+// by the scan's first CTAs themselves (see FusedAppend).
 #include <cuda_fp16.h>
 
 #include "common.cuh"
@@ -41,8 +42,83 @@ __device__ __forceinline__ uint32_t e4m3_encode(double t) {
 }
 
 // --------------------------------------------------------------------- append ---
-// One CTA per row; d is a multiple of 16.  Two passes over the row (it is re-read from
-// L2): squared norm and peak, then the codes.
+// Quantise one raw bf16 row (d a multiple of 16) into codes + scale.  All kNormThreads
+// threads of the block take part; two passes over the row (it is re-read from L2):
+// squared norm and peak, then the codes.  Returns true if the row was usable.
+__device__ __forceinline__ bool quantize_row_e4m3(const uint16_t* __restrict__ src, int d,
+                                                  uint8_t* __restrict__ dst, float* scale_out) {
+  __shared__ double s_ss[kNormThreads / 32];
+  __shared__ float s_mx[kNormThreads / 32];
+  __shared__ int s_bad[kNormThreads / 32];
+  __shared__ double s_inv;
+  __shared__ float s_scale;
+  __shared__ int s_ok;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int n16 = d >> 4;
+  const uint4* src4 = reinterpret_cast<const uint4*>(src);
+  double ss = 0.0;
+  float mx = 0.f;
+  int bad = 0;
+  for (int c = threadIdx.x; c < 2 * n16; c += kNormThreads) {
+    const uint4 hv = __ldg(src4 + c);
+    const uint32_t w[4] = {hv.x, hv.y, hv.z, hv.w};
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const float lo = bf16_lo(w[j]), hi = bf16_hi(w[j]);
+      bad |= ((w[j] & 0x7f80u) == 0x7f80u) | ((w[j] & 0x7f800000u) == 0x7f800000u);
+      ss += (double)lo * (double)lo;
+      ss += (double)hi * (double)hi;
+      mx = fmaxf(mx, fmaxf(fabsf(lo), fabsf(hi)));
+    }
+  }
+#pragma unroll
+  for (int m = 16; m; m >>= 1) {
+    ss += __shfl_xor_sync(0xffffffffu, ss, m);
+    mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, m));
+    bad |= __shfl_xor_sync(0xffffffffu, bad, m);
+  }
+  if (lane == 0) { s_ss[warp] = ss; s_mx[warp] = mx; s_bad[warp] = bad; }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    double tot = 0.0;
+    float peak = 0.f;
+    int b = 0;
+    for (int w = 0; w < kNormThreads / 32; ++w) { tot += s_ss[w]; peak = fmaxf(peak, s_mx[w]); b |= s_bad[w]; }
+    const double nrm = sqrt(tot);
+    const bool ok = !b && nrm > 0.0 && isfinite(nrm);
+    const double inv = ok ? 1.0 / nrm : 0.0;
+    s_inv = inv;
+    s_scale = ok ? (float)((double)peak * inv / 448.0) : 0.f;
+    s_ok = ok ? 1 : 0;
+    *scale_out = s_scale;
+  }
+  __syncthreads();
+  const double inv = s_inv, sc = (double)s_scale;
+  uint4* dst4 = reinterpret_cast<uint4*>(dst);
+  for (int c = threadIdx.x; c < n16; c += kNormThreads) {
+    uint32_t o[4] = {0, 0, 0, 0};
+    if (sc != 0.0) {
+#pragma unroll
+      for (int h = 0; h < 2; ++h) {
+        const uint4 hv = __ldg(src4 + 2 * c + h);
+        const uint32_t w[4] = {hv.x, hv.y, hv.z, hv.w};
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          const uint32_t c0 = e4m3_encode(((double)bf16_lo(w[j]) * inv) / sc);
+          const uint32_t c1 = e4m3_encode(((double)bf16_hi(w[j]) * inv) / sc);
+          const int e = h * 8 + j * 2;                       // element index within the 16
+          o[e >> 2] |= (c0 << ((e & 3) * 8)) | (c1 << (((e + 1) & 3) * 8));
+        }
+      }
+    }
+    dst4[c] = make_uint4(o[0], o[1], o[2], o[3]);
+  }
+  const bool ok = s_ok != 0;
+  __syncthreads();   // the shared scratch is reused by the next row
+  return ok;
+}
+
+// One CTA per row.
 __global__ void __launch_bounds__(kNormThreads, 4)
 append_e4m3_kernel(const uint16_t* __restrict__ states, const int32_t* __restrict__ tokens,
                    int64_t n, int d, uint8_t* __restrict__ codes, float* __restrict__ scales,
@@ -51,82 +127,20 @@ append_e4m3_kernel(const uint16_t* __restrict__ states, const int32_t* __restric
                    uint64_t* __restrict__ trace_tag, uint64_t tag,
                    int64_t* __restrict__ trace_gbase, int64_t gbase, int set_tag,
                    DeviceStats* stats) {
-  __shared__ double s_ss[kNormThreads / 32];
-  __shared__ float s_mx[kNormThreads / 32];
-  __shared__ int s_bad[kNormThreads / 32];
-  __shared__ double s_inv;
-  __shared__ float s_scale;
   pdl_launch_dependents();
   pdl_wait();   // earlier queries may still be reading the trace table and token stream
   if (blockIdx.x == 0 && threadIdx.x == 0) {
     trace_end[trace] = (int32_t)(row0 + n);
     if (set_tag) { trace_tag[trace] = tag; trace_gbase[trace] = gbase; }
   }
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int n16 = d >> 4;
   for (int64_t r = blockIdx.x; r < n; r += gridDim.x) {
     const int64_t row = row0 + r;
-    const uint4* src4 = reinterpret_cast<const uint4*>(states + r * d);
-    double ss = 0.0;
-    float mx = 0.f;
-    int bad = 0;
-    for (int c = threadIdx.x; c < 2 * n16; c += kNormThreads) {
-      const uint4 hv = __ldg(src4 + c);
-      const uint32_t w[4] = {hv.x, hv.y, hv.z, hv.w};
-#pragma unroll
-      for (int j = 0; j < 4; ++j) {
-        const float lo = bf16_lo(w[j]), hi = bf16_hi(w[j]);
-        bad |= ((w[j] & 0x7f80u) == 0x7f80u) | ((w[j] & 0x7f800000u) == 0x7f800000u);
-        ss += (double)lo * (double)lo;
-        ss += (double)hi * (double)hi;
-        mx = fmaxf(mx, fmaxf(fabsf(lo), fabsf(hi)));
-      }
-    }
-#pragma unroll
-    for (int m = 16; m; m >>= 1) {
-      ss += __shfl_xor_sync(0xffffffffu, ss, m);
-      mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, m));
-      bad |= __shfl_xor_sync(0xffffffffu, bad, m);
-    }
-    if (lane == 0) { s_ss[warp] = ss; s_mx[warp] = mx; s_bad[warp] = bad; }
-    __syncthreads();
+    const bool ok = quantize_row_e4m3(states + r * d, d, codes + row * d, scales + row);
     if (threadIdx.x == 0) {
-      double tot = 0.0;
-      float peak = 0.f;
-      int b = 0;
-      for (int w = 0; w < kNormThreads / 32; ++w) { tot += s_ss[w]; peak = fmaxf(peak, s_mx[w]); b |= s_bad[w]; }
-      const double nrm = sqrt(tot);
-      const bool ok = !b && nrm > 0.0 && isfinite(nrm);
-      const double inv = ok ? 1.0 / nrm : 0.0;
-      s_inv = inv;
-      s_scale = ok ? (float)((double)peak * inv / 448.0) : 0.f;
-      scales[row] = s_scale;
       tok[row] = tokens[r];
       trace_id[row] = trace;
       if (!ok) atomicAdd(&stats->degenerate_rows, 1ull);           // stored as a zero key
     }
-    __syncthreads();
-    const double inv = s_inv, sc = (double)s_scale;
-    uint4* dst4 = reinterpret_cast<uint4*>(codes + row * d);
-    for (int c = threadIdx.x; c < n16; c += kNormThreads) {
-      uint32_t o[4] = {0, 0, 0, 0};
-      if (sc != 0.0) {
-#pragma unroll
-        for (int h = 0; h < 2; ++h) {
-          const uint4 hv = __ldg(src4 + 2 * c + h);
-          const uint32_t w[4] = {hv.x, hv.y, hv.z, hv.w};
-#pragma unroll
-          for (int j = 0; j < 4; ++j) {
-            const uint32_t c0 = e4m3_encode(((double)bf16_lo(w[j]) * inv) / sc);
-            const uint32_t c1 = e4m3_encode(((double)bf16_hi(w[j]) * inv) / sc);
-            const int e = h * 8 + j * 2;                       // element index within the 16
-            o[e >> 2] |= (c0 << ((e & 3) * 8)) | (c1 << (((e + 1) & 3) * 8));
-          }
-        }
-      }
-      dst4[c] = make_uint4(o[0], o[1], o[2], o[3]);
-    }
-    __syncthreads();   // the shared scratch is reused by the next row
   }
 }
 
@@ -146,6 +160,19 @@ constexpr int kQ8Threads = kNormThreads;
 constexpr int kQ8Warps = kQ8Threads / 32;
 constexpr int kQ8Rows = 4;        // rows a warp scores together
 
+// coherent loads (L2) for rows that another CTA of the same launch has just written
+__device__ __forceinline__ uint4 ld_cg16(const void* p) {
+  uint4 v;
+  asm volatile("ld.global.cg.v4.u32 {%0,%1,%2,%3}, [%4];"
+               : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+  return v;
+}
+__device__ __forceinline__ unsigned long long ld_acquire_u64(const unsigned long long* p) {
+  unsigned long long v;
+  asm volatile("ld.acquire.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
+  return v;
+}
+
 // two E4M3 codes -> two floats (exact)
 __device__ __forceinline__ float2 e4m3x2_to_float2(uint32_t two_codes) {
   uint32_t h2;
@@ -161,7 +188,7 @@ __global__ void __launch_bounds__(kQ8Threads, 2)
 scan_gemv_e4m3_kernel(const uint8_t* __restrict__ codes, const float* __restrict__ scales,
                       PoolView pv, const uint16_t* __restrict__ q_raw, int nq, int k,
                       const uint64_t* __restrict__ exclude_tag, u64* __restrict__ partial,
-                      int32_t* __restrict__ q_valid, DeviceStats* stats) {
+                      int32_t* __restrict__ q_valid, DeviceStats* stats, FusedAppend fa) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   constexpr int KK = 32 * E;
   pdl_launch_dependents();
@@ -171,10 +198,37 @@ scan_gemv_e4m3_kernel(const uint8_t* __restrict__ codes, const float* __restrict
   u64* scratch = reinterpret_cast<u64*>(smem_raw + (size_t)QT * d * 2);   // [warps][KK]
   __shared__ uint64_t s_ex[QT];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  // contiguous, balanced share of the rows; the fa.n CTAs that first append a row of this
+  // step take 1/16 less (quantising a row costs about twice what normalising one does)
   const int64_t n = pv.n_rows;
-  const int r_lo = (int)((n * blockIdx.x) / gridDim.x);
-  const int r_hi = (int)((n * (blockIdx.x + 1)) / gridDim.x);
+  const int64_t w_lo = 16ll * blockIdx.x - min((int)blockIdx.x, fa.n);
+  const int64_t w_hi = 16ll * (blockIdx.x + 1) - min((int)blockIdx.x + 1, fa.n);
+  const int64_t w_all = 16ll * gridDim.x - min((int)gridDim.x, fa.n);
+  const int r_lo = (int)((n * w_lo) / w_all);
+  const int r_hi = (int)((n * w_hi) / w_all);
   const uint4* codes4 = reinterpret_cast<const uint4*>(codes);
+
+  // the step's append, one row per CTA (as in the 16-bit scan)
+  if ((int)blockIdx.x < fa.n) {
+    const int r = blockIdx.x;
+    const int64_t row = (int64_t)fa.row0 + r;
+    const bool ok = quantize_row_e4m3(fa.states + (size_t)r * d, d,
+                                      const_cast<uint8_t*>(codes) + row * d,
+                                      const_cast<float*>(scales) + row);
+    if (threadIdx.x == 0) {
+      fa.tok[row] = fa.tokens[r];
+      fa.trace_id[row] = fa.trace;
+      if (!ok) atomicAdd(&stats->degenerate_rows, 1ull);
+      if (r == 0) {
+        fa.trace_end[fa.trace] = fa.row0 + fa.n;
+        if (fa.set_tag) { fa.trace_tag[fa.trace] = fa.tag; fa.trace_gbase[fa.trace] = fa.gbase; }
+      }
+    }
+    __threadfence();                   // this thread's part of the row, before the count
+    __syncthreads();
+    if (threadIdx.x == 0) atomicAdd(fa.ready, 1ull);
+  }
+  bool fresh_ok = fa.n == 0;           // this warp has seen the appended rows arrive
 
   for (int q0 = 0; q0 < nq; q0 += QT) {
     __syncthreads();
@@ -217,11 +271,27 @@ scan_gemv_e4m3_kernel(const uint8_t* __restrict__ codes, const float* __restrict
 #pragma unroll
         for (int q = 0; q < QT; ++q) acc[r][q] = 0.f;
 
+      const bool fresh = fa.n > 0 && rb + kQ8Rows > fa.row0;       // warp-uniform
+      if (fresh && !fresh_ok) {
+        // rows of this step's append: wait (bounded) until all of them are in
+        unsigned long long t0 = 0;
+        for (uint32_t spin = 0; ld_acquire_u64(fa.ready) < fa.target; ++spin) {
+          if (spin == 0) asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t0));
+          if ((spin & 255u) == 255u) {
+            unsigned long long t1;
+            asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t1));
+            if (t1 - t0 > 2000000000ull) { atomicExch(&stats->stalled, 1); break; }
+          }
+          __nanosleep(64);
+        }
+        fresh_ok = true;
+      }
 #pragma unroll 4
       for (int c = lane; c < n16; c += 32) {
         uint4 kv[kQ8Rows];
 #pragma unroll
-        for (int r = 0; r < kQ8Rows; ++r) kv[r] = ld_stream16(rowp[r] + c);
+        for (int r = 0; r < kQ8Rows; ++r)
+          kv[r] = fresh ? ld_cg16(rowp[r] + c) : ld_stream16(rowp[r] + c);
         uint4 qv[QT][2];
 #pragma unroll
         for (int q = 0; q < QT; ++q) { qv[q][0] = qs[q * n8 + 2 * c]; qv[q][1] = qs[q * n8 + 2 * c + 1]; }
@@ -256,9 +326,12 @@ scan_gemv_e4m3_kernel(const uint8_t* __restrict__ codes, const float* __restrict
       for (int r = 0; r < kQ8Rows; ++r) {
         const int row = rb + r;
         if (row >= r_hi) break;                             // warp-uniform
-        const float sc = scales[row];
+        const bool fresh_row = fa.n > 0 && row >= fa.row0;     // written by another CTA just now
+        const float sc = fresh_row ? __ldcg(scales + row) : scales[row];
         uint64_t tag = 0;
-        if (exclude_tag) tag = pv.trace_tag[pv.trace_id[row]];
+        if (exclude_tag)
+          tag = fresh_row ? __ldcg(&pv.trace_tag[__ldcg(&pv.trace_id[row])])
+                          : pv.trace_tag[pv.trace_id[row]];
 #pragma unroll
         for (int q = 0; q < QT; ++q) {
           const float s = warp_sum(acc[r][q]) * sc;
@@ -288,35 +361,43 @@ scan_gemv_e4m3_kernel(const uint8_t* __restrict__ codes, const float* __restrict
 template <int QT, int E>
 static cudaError_t launch_q8(const uint8_t* codes, const float* scales, const PoolView& pv,
                              const uint16_t* q_raw, int nq, int k, const uint64_t* ex, u64* partial,
-                             int32_t* q_valid, DeviceStats* stats, int grid, cudaStream_t st) {
+                             int32_t* q_valid, DeviceStats* stats, int grid, const FusedAppend& fa,
+                             cudaStream_t st) {
   const size_t smem = (size_t)QT * pv.d * 2 + (size_t)kQ8Warps * 32 * E * sizeof(u64);
   cudaError_t e = cudaFuncSetAttribute(scan_gemv_e4m3_kernel<QT, E>,
                                        cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
   return launch_pdl(scan_gemv_e4m3_kernel<QT, E>, dim3(grid), dim3(kQ8Threads), smem, st, codes,
-                    scales, pv, q_raw, nq, k, ex, partial, q_valid, stats);
+                    scales, pv, q_raw, nq, k, ex, partial, q_valid, stats, fa);
 }
 
 template <int QT>
 static cudaError_t launch_q8_qt(int kk, const uint8_t* codes, const float* scales,
                                 const PoolView& pv, const uint16_t* q_raw, int nq, int k,
                                 const uint64_t* ex, u64* partial, int32_t* q_valid,
-                                DeviceStats* stats, int grid, cudaStream_t st) {
-  if (kk == 32) return launch_q8<QT, 1>(codes, scales, pv, q_raw, nq, k, ex, partial, q_valid, stats, grid, st);
-  if (kk == 64) return launch_q8<QT, 2>(codes, scales, pv, q_raw, nq, k, ex, partial, q_valid, stats, grid, st);
-  return launch_q8<QT, 4>(codes, scales, pv, q_raw, nq, k, ex, partial, q_valid, stats, grid, st);
+                                DeviceStats* stats, int grid, const FusedAppend& fa,
+                                cudaStream_t st) {
+  if (kk == 32) return launch_q8<QT, 1>(codes, scales, pv, q_raw, nq, k, ex, partial, q_valid, stats, grid, fa, st);
+  if (kk == 64) return launch_q8<QT, 2>(codes, scales, pv, q_raw, nq, k, ex, partial, q_valid, stats, grid, fa, st);
+  return launch_q8<QT, 4>(codes, scales, pv, q_raw, nq, k, ex, partial, q_valid, stats, grid, fa, st);
 }
 
 cudaError_t launch_scan_gemv_e4m3(const uint8_t* codes, const float* scales, const PoolView& pv,
                                   const uint16_t* q_raw, int32_t nq, int32_t k, int32_t kk,
                                   const uint64_t* exclude_tag, unsigned long long* partial,
                                   int32_t* q_valid, DeviceStats* stats, int32_t max_lists,
-                                  int32_t num_sms, int32_t* n_lists, cudaStream_t st) {
+                                  int32_t num_sms, int32_t* n_lists, const FusedAppend* fused,
+                                  cudaStream_t st) {
   const int grid = scan_gemv_grid(pv.n_rows, num_sms, max_lists);
   *n_lists = grid;
+  FusedAppend fa = {};
+  if (fused) {
+    if (fused->n > grid || fused->n > kFuseMaxRows) return cudaErrorInvalidValue;
+    fa = *fused;
+  }
   if (nq >= 2)
-    return launch_q8_qt<2>(kk, codes, scales, pv, q_raw, nq, k, exclude_tag, partial, q_valid, stats, grid, st);
-  return launch_q8_qt<1>(kk, codes, scales, pv, q_raw, nq, k, exclude_tag, partial, q_valid, stats, grid, st);
+    return launch_q8_qt<2>(kk, codes, scales, pv, q_raw, nq, k, exclude_tag, partial, q_valid, stats, grid, fa, st);
+  return launch_q8_qt<1>(kk, codes, scales, pv, q_raw, nq, k, exclude_tag, partial, q_valid, stats, grid, fa, st);
 }
 
 }  // namespace oilbird

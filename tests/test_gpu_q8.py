@@ -148,3 +148,35 @@ def test_retrieval_agrees_with_the_16bit_pool_on_separated_neighbours():
         for r, s in zip(a.idx[i].tolist(), a.score[i].tolist()):
             if r in common:
                 assert abs(s - common[r]) < 0.02
+
+
+def test_fused_steps_on_8bit_pool():
+    # for nq <= 2 and up to 64 rows the 8-bit scan appends the step's rows itself
+    w = W.C1.scaled(n_rows=8192, nq=1)
+    pool, ora = fill_both(w, key_format="e4m3", spare_rows=8192)
+    g = torch.Generator(device="cuda").manual_seed(4)
+    pr = fixed(4, 4, theta=-2.0)
+    steps = 120
+    sizes = [8, 1, 64, 33, 100, 0]                         # 100 and 0: separate append / none
+    outs, chunks = [], []
+    for s in range(steps):
+        n = sizes[s % len(sizes)]
+        st = torch.randn(max(n, 1), w.d, generator=g, device="cuda").to(torch.bfloat16)
+        tk = torch.randint(0, 100, (max(n, 1),), generator=g, device="cuda", dtype=torch.int32)
+        q = st[-1:].contiguous()
+        st, tk = st[:n].contiguous(), tk[:n].contiguous()
+        outs.append((n, pool.step(st, tk, q, pr, tag=700 + s, new_trace=(s % 2 == 0)), len(pool)))
+        chunks.append((st, tk, s))
+    torch.cuda.synchronize()
+    for n, out, rows in outs:
+        if n > 0:
+            assert int(out.idx[0, 0]) == rows - 1
+    for st, tk, s in chunks:
+        ora.append(W.to_bits(st), tk.cpu().numpy(), tag=700 + s, new_trace=(s % 2 == 0))
+    codes, scales = pool.read_codes()
+    assert np.array_equal(codes, ora.codes) and np.array_equal(scales, ora.scales)
+    _, tok, _ = pool.read_rows()
+    assert np.array_equal(tok, ora.tokens)
+    q = chunks[3][0][:1].contiguous()
+    check_query(pool.query(q, pr), ora, W.to_bits(q), pr)
+    assert pool.stats()["stalled"] == 0

@@ -75,6 +75,8 @@ def lib() -> ctypes.CDLL:
         fn = getattr(L, "oracle_pool_" + name)
         fn.restype = vp
         fn.argtypes = [vp]
+    L.oracle_pool_evict_oldest.restype = i64
+    L.oracle_pool_evict_oldest.argtypes = [vp, i32]
     L.oracle_pool_destroy.restype = None
     L.oracle_pool_destroy.argtypes = [vp]
     L.oracle_pool_reset.restype = None
@@ -227,6 +229,10 @@ class OraclePool:
 
     def reset(self) -> None:
         self._L.oracle_pool_reset(self._h)
+
+    def evict_oldest(self, n_traces: int) -> int:
+        """Drop the n_traces oldest traces; rows and traces are renumbered. Returns rows dropped."""
+        return int(self._L.oracle_pool_evict_oldest(self._h, int(n_traces)))
 
     def append(self, states, tokens, tag: int = 0, new_trace: bool = True) -> None:
         states = _u16(states).reshape(-1, self.d)

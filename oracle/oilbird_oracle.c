@@ -299,6 +299,40 @@ int oracle_pool_append(oracle_pool *p, const uint16_t *states, const int32_t *to
   return 0;
 }
 
+/*
+ * Eviction for a bounded store (the paper's Limitations section names eviction as one way
+ * to keep the store bounded and defines no policy; this build's reading: oldest first, by
+ * whole traces).  The first n_traces traces and their rows are dropped; what remains is
+ * exactly the pool that would have been built from the remaining traces alone: rows and
+ * traces are renumbered from zero, order kept.  Returns the number of rows dropped.
+ */
+int64_t oracle_pool_evict_oldest(oracle_pool *p, int32_t n_traces) {
+  if (n_traces <= 0) return 0;
+  if (n_traces > p->n_traces) n_traces = p->n_traces;
+  if (n_traces == 0) return 0;
+  const int64_t drop = p->trace_end[n_traces - 1];
+  const int64_t live = p->n - drop;
+  const int32_t d = p->d;
+  for (int64_t i = 0; i < live; ++i) {
+    if (p->fmt == 0) {
+      for (int32_t j = 0; j < d; ++j) p->key[(size_t)i * d + j] = p->key[(size_t)(i + drop) * d + j];
+    } else {
+      for (int32_t j = 0; j < d; ++j) p->code[(size_t)i * d + j] = p->code[(size_t)(i + drop) * d + j];
+      p->scale[i] = p->scale[i + drop];
+    }
+    p->tok[i] = p->tok[i + drop];
+    p->trace_id[i] = p->trace_id[i + drop] - n_traces;
+  }
+  for (int32_t t = 0; t + n_traces < p->n_traces; ++t) {
+    p->trace_start[t] = p->trace_start[t + n_traces] - drop;
+    p->trace_end[t] = p->trace_end[t + n_traces] - drop;
+    p->trace_tag[t] = p->trace_tag[t + n_traces];
+  }
+  p->n_traces -= n_traces;
+  p->n = live;
+  return drop;
+}
+
 /* --------------------------------------------------------------- scoring -- */
 
 /*

@@ -160,3 +160,65 @@ def test_quantisation_error_of_a_score_is_within_its_bound():
     bound = 2.0 ** -4 + np.sqrt(d) * p8.scales.max() * 2.0 ** -10 + 2.0 ** -8
     assert np.max(np.abs(a - b)) <= bound
     assert np.max(np.abs(a - b)) < 0.02              # and in practice far below it
+
+
+# ---------------------------------------------------------------- eviction ----
+# Oldest-first eviction by whole traces must leave exactly the pool that the remaining
+# traces alone would have built (the append and query paths are pinned elsewhere).
+
+def _traces(rng, d, lens):
+    return [(bits(rng.normal(0, 1, (n, d))), rng.integers(0, 1000, n).astype(np.int32), 100 + i)
+            for i, n in enumerate(lens)]
+
+
+@pytest.mark.parametrize("fmt", ["bf16", "e4m3"])
+@pytest.mark.parametrize("drop", [0, 1, 3, 6, 9])
+def test_evict_oldest_equals_rebuild_from_remaining_traces(fmt, drop):
+    rng = np.random.default_rng(31)
+    d = 32
+    lens = [5, 1, 17, 4, 9, 2]
+    tr = _traces(rng, d, lens)
+    a, b = OraclePool(d, fmt), OraclePool(d, fmt)
+    for st, tk, tag in tr:
+        a.append(st, tk, tag=tag)
+    dropped = a.evict_oldest(drop)
+    keep = tr[min(drop, len(tr)):]
+    for st, tk, tag in keep:
+        b.append(st, tk, tag=tag)
+    assert dropped == sum(lens[:min(drop, len(lens))])
+    assert len(a) == len(b) and a.num_traces == b.num_traces
+    if fmt == "bf16":
+        assert np.array_equal(a.keys, b.keys)
+    else:
+        assert np.array_equal(a.codes, b.codes) and np.array_equal(a.scales, b.scales)
+    assert np.array_equal(a.tokens, b.tokens) and np.array_equal(a.trace_ids, b.trace_ids)
+    assert np.array_equal(a.trace_starts, b.trace_starts)
+    assert np.array_equal(a.trace_ends, b.trace_ends) and np.array_equal(a.trace_tags, b.trace_tags)
+    if len(a):
+        q = bits(rng.normal(0, 1, (2, d)))
+        pr = oracle.QueryParams(k=4, theta=-2.0, depth_mode=oracle.DEPTH_FIXED, cont_len=6)
+        ra, rb = a.query(q, pr), b.query(q, pr)
+        for f in ("idx", "score", "fired", "cont_len", "cont_tok"):
+            assert np.array_equal(getattr(ra, f), getattr(rb, f))
+    # the pool keeps working: an append after the eviction extends / opens traces as usual
+    st, tk, tag = _traces(rng, d, [3])[0]
+    a.append(st, tk, tag=7, new_trace=False)
+    b.append(st, tk, tag=7, new_trace=False)
+    assert np.array_equal(a.trace_ends, b.trace_ends) and np.array_equal(a.tokens, b.tokens)
+
+
+def test_evicted_rows_by_hand():
+    d = 16
+    p = OraclePool(d)
+    e = np.eye(d, dtype=np.float32)
+    p.append(bits(e[0:2]), np.array([10, 11]), tag=1)        # rows 0,1
+    p.append(bits(e[2:5]), np.array([20, 21, 22]), tag=2)    # rows 2,3,4
+    p.append(bits(e[5:6]), np.array([30]), tag=3)            # row 5
+    assert p.evict_oldest(1) == 2
+    assert p.tokens.tolist() == [20, 21, 22, 30]
+    assert p.trace_ids.tolist() == [0, 0, 0, 1]
+    assert p.trace_starts.tolist() == [0, 3] and p.trace_ends.tolist() == [3, 4]
+    assert p.trace_tags.tolist() == [2, 3]
+    r = p.query(bits(e[2:3]), oracle.QueryParams(k=1, theta=0.5, offset=1, depth_mode=oracle.DEPTH_FIXED,
+                                                 cont_len=4))
+    assert r.idx[0, 0] == 0 and r.cont_tok[0, 0].tolist() == [21, 22, -1, -1]   # clipped at the trace end

@@ -556,6 +556,88 @@ def run_ring(args):
     print(json.dumps(line), flush=True)
 
 
+def run_evict(args):
+    """Bounded store: one step = drop the oldest tenth of the traces (the live rows are moved
+    to the front) + append as many fresh traces + one query.  Reported per step; the
+    roofline is the compaction kernel's: live bytes read once and written once."""
+    from paper_2608_03839_b200 import binding as B
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda:0")
+    w = W.CONFIGS[args.config]
+    n0 = args.rows or w.n_rows
+    rpt = w.rows_per_trace
+    n_tr = n0 // rpt
+    drop = max(1, n_tr // 10)
+    K, Wm = args.steps, args.warmup
+    pool = B.Pool(w.d, n_tr * rpt + rpt, max_nq=1, max_k=w.k, max_traces=n_tr + 8,
+                  key_format=args.keys)
+    row_bytes = w.d * 2 if args.keys == "bf16" else w.d + 4
+    fresh = []
+    done = 0
+    for st, tk, tag in w.traces(dev):
+        if done >= n_tr:
+            break
+        pool.append(st, tk, tag=tag)
+        if len(fresh) < drop:
+            fresh.append((st.clone(), tk.clone()))
+        done += 1
+    q, _ = w.queries(dev, nq=1)
+    pr = B.QueryParams(k=w.k, theta=0.8, depth_mode=B.DEPTH_FIXED, cont_len=w.cont_len)
+    out = B.QueryOut.empty(1, w.k, w.cont_len, dev)
+    torch.cuda.synchronize()
+    step_no = [0]
+
+    def step():
+        pool.evict_oldest(drop)
+        for st, tk in fresh:
+            pool.append(st, tk, tag=5_000_000 + step_no[0])
+            step_no[0] += 1
+        pool.query(q, pr, out=out)
+
+    for _ in range(Wm):
+        step()
+    torch.cuda.synchronize()
+    sampler = ClockSampler(physical_device(0))
+    sampler.start()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    l0 = pool.launch_count
+    e0.record()
+    for _ in range(K):
+        step()
+    e1.record()
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    launches = pool.launch_count - l0
+    total_ms = e0.elapsed_time(e1)
+    # the compaction alone
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(2 * K)]
+    for i in range(K):
+        ev[2 * i].record()
+        pool.evict_oldest(drop)
+        ev[2 * i + 1].record()
+        for st, tk in fresh:
+            pool.append(st, tk, tag=6_000_000 + i)
+    torch.cuda.synchronize()
+    ev_ms = float(np.mean([ev[2 * i].elapsed_time(ev[2 * i + 1]) for i in range(K)]))
+    live = (n_tr - drop) * rpt
+    moved = 2.0 * live * (row_bytes + 8)            # keys (+scale), token, trace id: read + write
+    peaks, peak_kind = measured_peaks()
+    line = {"metric": "evict_append_query_steps_per_sec", "value": K / (total_ms / 1e3),
+            "unit": "steps/s", "n_gpus": 1, "steps": K, "warmup": Wm, "ms_per_step": total_ms / K,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": f"{args.keys} keys", "data": "synthetic",
+            "config": {"workload": f"evict: {w.name} recipe, {n_tr} traces x {rpt} rows x d={w.d} "
+                                   f"{args.keys}; per step the oldest {drop} traces are dropped, "
+                                   f"{drop} appended, 1 query"},
+            "evict_ms": ev_ms, "clocks": clocks, "gpu_launches": int(launches),
+            "roofline": {"bound": "hbm", "kernel": "compact_kernel (live rows moved to the front)",
+                         "achieved": moved / (ev_ms * 1e-3) / 1e9, "peak": peaks["hbm_gbs"],
+                         "unit": "GB/s", "frac": moved / (ev_ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
+                         "peak_kind": peak_kind, "bytes_per_launch": moved, "traffic": None}}
+    print(json.dumps(line), flush=True)
+    pool.close()
+
+
 def run_merge(args):
     """Third workload: chain post-filter + tree merge for a batch of requests (paper sizes:
     8 semantic chains of up to 48 tokens + 7 other chains into a 44-node tree, 16 of 60 nodes)."""
@@ -696,7 +778,7 @@ def main():
     ap.add_argument("--keys", default="bf16", choices=["bf16", "e4m3"],
                     help="stored key format: the paper's 16-bit keys, or the bounded-store "
                          "variant with 8-bit keys (FP8 E4M3 + one scale per row)")
-    ap.add_argument("--workload", default="pool", choices=["pool", "ring", "merge"],
+    ap.add_argument("--workload", default="pool", choices=["pool", "ring", "merge", "evict"],
                     help="pool: the trace-store query path (default); ring: the recycled pool")
     ap.add_argument("--sharded", action="store_true",
                     help="one logical pool row-sharded over the ranks (default: one pool per rank)")
@@ -712,6 +794,11 @@ def main():
         args.steps = 500 if args.steps is None else args.steps
         args.warmup = 10 if args.warmup is None else max(args.warmup, 3)
         run_ring(args)
+        return
+    if args.workload == "evict":
+        args.steps = 20 if args.steps is None else args.steps
+        args.warmup = 3 if args.warmup is None else max(args.warmup, 3)
+        run_evict(args)
         return
     if args.workload == "merge":
         args.steps = 200 if args.steps is None else args.steps

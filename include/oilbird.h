@@ -173,6 +173,20 @@ int oilbird_pool_gather(oilbird_pool_t* pool, const int32_t* idx, const float* s
                         const oilbird_query_out* out, void* cuda_stream);
 
 /*
+ * Eviction, for a bounded store (the paper's Limitations section names eviction as one way
+ * to keep the store bounded and defines no policy).  Drops the n_traces oldest traces
+ * (all of them if there are fewer) with their rows and moves the rest to the front: the
+ * pool afterwards is exactly the pool that the remaining traces alone would have built,
+ * rows and traces renumbered from zero, so row numbers returned by earlier queries are
+ * stale.  The global positions given to oilbird_pool_append_global are kept.  The live rows
+ * are read and written once (a cooperative kernel on cuda_stream); the call also waits for
+ * earlier work on cuda_stream when it publishes the renumbered trace table.
+ * *rows_dropped (may be NULL) receives the number of rows removed.
+ */
+int oilbird_pool_evict_oldest(oilbird_pool_t* pool, int32_t n_traces, int64_t* rows_dropped,
+                              void* cuda_stream);
+
+/*
  * One serving step with DEVICE buffers: oilbird_pool_append (the n rows committed since
  * the last step; n may be 0) followed by oilbird_pool_query, in one call, with the same
  * arguments, results and error codes as the two calls (Algorithm 1 runs once per decoding

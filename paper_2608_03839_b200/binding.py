@@ -86,6 +86,7 @@ SYMBOLS = {
                                           ctypes.POINTER(CQueryOut), _vp]),
     "oilbird_pool_gather": (ctypes.c_int, [_vp, _vp, _vp, _i32, ctypes.POINTER(CQueryParams),
                                            ctypes.POINTER(CQueryOut), _vp]),
+    "oilbird_pool_evict_oldest": (ctypes.c_int, [_vp, _i32, ctypes.POINTER(_i64), _vp]),
     "oilbird_pool_step": (ctypes.c_int, [_vp, _vp, _vp, _i64, _u64, _u32, _vp, _i32,
                                          ctypes.POINTER(CQueryParams),
                                          ctypes.POINTER(CQueryOut), _vp]),
@@ -374,6 +375,14 @@ class Pool:
                                           ctypes.byref(out._c), _stream_ptr(stream)),
                "oilbird_pool_query")
         return out
+
+    def evict_oldest(self, n_traces: int, stream=None) -> int:
+        """Drop the n_traces oldest traces and compact; rows and traces are renumbered.
+        Returns the number of rows dropped."""
+        dropped = ctypes.c_int64(0)
+        _check(self._L.oilbird_pool_evict_oldest(self._h, int(n_traces), ctypes.byref(dropped),
+                                                 _stream_ptr(stream)), "oilbird_pool_evict_oldest")
+        return int(dropped.value)
 
     def step(self, states: torch.Tensor, tokens: torch.Tensor, q: torch.Tensor,
              params: QueryParams | None = None, out: QueryOut | None = None, tag: int = 0,

@@ -128,6 +128,12 @@ cudaError_t launch_scan_gemv_e4m3(const uint8_t* codes, const float* scales, con
                                   int32_t num_sms, int32_t* n_lists, const FusedAppend* fused,
                                   cudaStream_t st);
 
+// Eviction: move rows [head, head+live) of every per-row array down to [0, live) in place
+// (cooperative launch; trace ids drop by n_traces).  scales may be nullptr.
+cudaError_t launch_compact(unsigned char* keys, float* scales, int32_t* tok, int32_t* trace_id,
+                           int64_t head, int64_t live, int64_t row_bytes, int32_t n_traces,
+                           int32_t num_sms, cudaStream_t st);
+
 // CTAs the CUDA-core scan launches for a pool of n_rows rows.
 inline int32_t scan_gemv_grid(int64_t n_rows, int32_t num_sms, int32_t max_lists) {
   // at least 32 rows per CTA, at most two CTAs per SM

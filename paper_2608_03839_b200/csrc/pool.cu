@@ -120,6 +120,8 @@ struct oilbird_pool {
   int64_t n_rows;
   std::vector<int64_t> t_start, t_end;
   std::vector<uint64_t> t_tag;
+  std::vector<int64_t> t_gbase;     // global position of each trace's first row, or -1 if
+                                    // it is simply the local one (pool is not a shard)
   int64_t launches;
   // profiling
   bool profile;
@@ -251,7 +253,7 @@ int oilbird_pool_reset(oilbird_pool_t* p, void* stream) {
   CU(cudaSetDevice(p->device));
   CU(cudaMemsetAsync(p->stats, 0, sizeof(DeviceStats), (cudaStream_t)stream));
   p->n_rows = 0;
-  p->t_start.clear(); p->t_end.clear(); p->t_tag.clear();
+  p->t_start.clear(); p->t_end.clear(); p->t_tag.clear(); p->t_gbase.clear();
   return OILBIRD_OK;
 }
 
@@ -278,13 +280,16 @@ static int append_prepare(oilbird_pool_t* p, const void* states, const int32_t* 
     p->t_start.push_back(p->n_rows);
     p->t_end.push_back(p->n_rows);
     p->t_tag.push_back(tag);
+    p->t_gbase.push_back(-1);
   }
   ap->trace = (int32_t)p->t_start.size() - 1;
   ap->row0 = p->n_rows;
   return OILBIRD_OK;
 }
 static void append_rollback(oilbird_pool_t* p, const AppendPlan& ap) {
-  if (ap.open_new) { p->t_start.pop_back(); p->t_end.pop_back(); p->t_tag.pop_back(); }
+  if (ap.open_new) {
+    p->t_start.pop_back(); p->t_end.pop_back(); p->t_tag.pop_back(); p->t_gbase.pop_back();
+  }
   p->n_rows = ap.row0;
   if (!ap.open_new) p->t_end[ap.trace] = ap.row0;
 }
@@ -317,7 +322,48 @@ static int append_impl(oilbird_pool_t* p, const void* states, const int32_t* tok
     return cuda_fail(e, "append kernel launch");
   }
   p->launches += 1;
+  if (ap.open_new && global_row >= 0) p->t_gbase[ap.trace] = global_row;
   append_commit(p, n, ap);
+  return OILBIRD_OK;
+}
+
+int oilbird_pool_evict_oldest(oilbird_pool_t* p, int32_t n_traces, int64_t* rows_dropped,
+                              void* stream) {
+  if (rows_dropped) *rows_dropped = 0;
+  if (!p || n_traces < 0) return OILBIRD_EINVAL;
+  const int32_t have = (int32_t)p->t_start.size();
+  const int32_t nt = n_traces < have ? n_traces : have;
+  if (nt == 0) return OILBIRD_OK;
+  CU(cudaSetDevice(p->device));
+  cudaStream_t st = (cudaStream_t)stream;
+  const int64_t head = p->t_end[nt - 1], live = p->n_rows - head;
+  const int64_t row_bytes = p->r.e4m3 ? p->r.d : (int64_t)p->r.d * 2;
+  cudaError_t e = launch_compact((unsigned char*)p->keys, p->r.e4m3 ? p->scales : nullptr, p->tok,
+                                 p->trace_id, head, live, row_bytes, nt, p->num_sms, st);
+  if (e != cudaSuccess) return cuda_fail(e, "compaction kernel launch");
+  if (live > 0 && head > 0) p->launches += 1;
+  // the host's copy of the trace table is the truth: renumber it, then publish it
+  p->t_start.erase(p->t_start.begin(), p->t_start.begin() + nt);
+  p->t_end.erase(p->t_end.begin(), p->t_end.begin() + nt);
+  p->t_tag.erase(p->t_tag.begin(), p->t_tag.begin() + nt);
+  p->t_gbase.erase(p->t_gbase.begin(), p->t_gbase.begin() + nt);
+  const size_t left = p->t_start.size();
+  std::vector<int32_t> ends(left);
+  std::vector<int64_t> gb(left);
+  for (size_t i = 0; i < left; ++i) {
+    p->t_start[i] -= head;
+    p->t_end[i] -= head;
+    ends[i] = (int32_t)p->t_end[i];
+    gb[i] = p->t_gbase[i] >= 0 ? p->t_gbase[i] : p->t_start[i];
+  }
+  p->n_rows = live;
+  if (left > 0) {
+    // pageable sources: each call returns once its source has been staged
+    CU(cudaMemcpyAsync(p->trace_end, ends.data(), left * 4, cudaMemcpyHostToDevice, st));
+    CU(cudaMemcpyAsync(p->trace_tag, p->t_tag.data(), left * 8, cudaMemcpyHostToDevice, st));
+    CU(cudaMemcpyAsync(p->trace_gbase, gb.data(), left * 8, cudaMemcpyHostToDevice, st));
+  }
+  if (rows_dropped) *rows_dropped = head;
   return OILBIRD_OK;
 }
 

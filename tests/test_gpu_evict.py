@@ -1,0 +1,102 @@
+"""GPU parity for eviction (bounded store): after dropping the oldest traces the CUDA pool
+must hold exactly what the oracle holds after the same eviction, bit for bit, and keep
+answering queries, steps and appends like it."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from oracle import OraclePool
+from paper_2608_03839_b200 import binding as B
+from paper_2608_03839_b200 import workloads as W
+from parity import check_query, fill_both
+
+pytestmark = pytest.mark.gpu
+
+
+def fixed(k, L, theta=0.8, **kw):
+    return B.QueryParams(k=k, theta=theta, depth_mode=B.DEPTH_FIXED, cont_len=L, **kw)
+
+
+def same_store(pool, ora):
+    if pool.key_format == "bf16":
+        keys, tok, tid = pool.read_rows()
+        assert np.array_equal(keys, ora.keys)
+    else:
+        _, tok, tid = pool.read_rows()
+        codes, scales = pool.read_codes()
+        assert np.array_equal(codes, ora.codes) and np.array_equal(scales, ora.scales)
+    assert np.array_equal(tok, ora.tokens) and np.array_equal(tid, ora.trace_ids)
+    st, en, tg = pool.traces()
+    assert np.array_equal(st, ora.trace_starts) and np.array_equal(en, ora.trace_ends)
+    assert np.array_equal(tg, ora.trace_tags)
+    assert len(pool) == len(ora) and pool.num_traces == ora.num_traces
+
+
+@pytest.mark.parametrize("fmt", ["bf16", "e4m3"])
+@pytest.mark.parametrize("drop", [1, 5, 15, 16, 40])
+def test_evict_matches_oracle(fmt, drop):
+    w = W.C1.scaled(nq=4)                       # 16 traces of 256 rows
+    pool, ora = fill_both(w, key_format=fmt, spare_rows=512)
+    n0 = len(pool)
+    dropped = pool.evict_oldest(drop)
+    assert dropped == ora.evict_oldest(drop) == min(drop, 16) * 256
+    assert len(pool) == n0 - dropped
+    same_store(pool, ora)
+    q, _ = w.queries("cuda")
+    if len(pool):
+        paths = (B.PATH_GEMV,) if fmt == "e4m3" else (B.PATH_GEMV, B.PATH_TENSOR)
+        for path in paths:
+            pr = fixed(8, 8, theta=-2.0, path=path)
+            check_query(pool.query(q, pr), ora, W.to_bits(q), pr)
+    # life goes on: a fused step, an append to the open trace, another eviction
+    g = torch.Generator(device="cuda").manual_seed(drop)
+    st = torch.randn(8, w.d, generator=g, device="cuda").to(torch.bfloat16)
+    tk = torch.arange(8, dtype=torch.int32, device="cuda")
+    pr = fixed(4, 4, theta=-2.0)
+    out = pool.step(st, tk, st[5:6].contiguous(), pr, tag=4242)
+    ora.append(W.to_bits(st), tk.cpu().numpy(), tag=4242)
+    assert int(out.idx[0, 0]) == len(pool) - 3
+    pool.append(st[:3].contiguous(), tk[:3].contiguous(), new_trace=False)
+    ora.append(W.to_bits(st[:3]), tk[:3].cpu().numpy(), new_trace=False)
+    same_store(pool, ora)
+    pool.evict_oldest(1)
+    ora.evict_oldest(1)
+    same_store(pool, ora)
+    assert pool.stats()["stalled"] == 0
+
+
+def test_many_waves_a_short_trace_in_front_of_a_long_pool():
+    # dropping 3 rows from in front of ~5000 moves the pool in ~1700 waves of 3 rows
+    d = 64
+    g = torch.Generator(device="cuda").manual_seed(1)
+    pool, ora = B.Pool(d, 6000), OraclePool(d)
+    for n, tag in ((3, 1), (2500, 2), (7, 3), (2490, 4)):
+        st = torch.randn(n, d, generator=g, device="cuda").to(torch.bfloat16)
+        tk = torch.randint(0, 1000, (n,), generator=g, device="cuda", dtype=torch.int32)
+        pool.append(st, tk, tag=tag)
+        ora.append(W.to_bits(st), tk.cpu().numpy(), tag=tag)
+    assert pool.evict_oldest(1) == ora.evict_oldest(1) == 3
+    same_store(pool, ora)
+    assert pool.evict_oldest(2) == ora.evict_oldest(2) == 2507
+    same_store(pool, ora)
+    assert pool.evict_oldest(0) == 0 and pool.evict_oldest(9) == 2490
+    assert len(pool) == 0 and pool.num_traces == 0
+    # an emptied pool starts over
+    st = torch.randn(5, d, generator=g, device="cuda").to(torch.bfloat16)
+    pool.append(st, torch.arange(5, dtype=torch.int32, device="cuda"), tag=9)
+    out = pool.query(st[2:3].contiguous(), fixed(1, 2, theta=-2.0))
+    assert int(out.idx[0, 0]) == 2 and out.cont_tok[0, 0].tolist() == [4, -1]
+
+
+def test_eviction_keeps_global_positions_of_a_shard():
+    d = 32
+    g = torch.Generator(device="cuda").manual_seed(2)
+    pool = B.Pool(d, 1000)
+    bases = [100, 5000, 70000]
+    for i, gb in enumerate(bases):
+        st = torch.randn(10, d, generator=g, device="cuda").to(torch.bfloat16)
+        pool.append_global(st, torch.arange(10, dtype=torch.int32, device="cuda"), gb, tag=i + 1)
+    pool.evict_oldest(1)
+    idx = torch.tensor([0, 9, 10, 19, -1], dtype=torch.int32, device="cuda")
+    assert pool.to_global(idx).tolist() == [5000, 5009, 70000, 70009, -1]

@@ -420,6 +420,10 @@ def cpu_baseline(w, n0, rows_step, nq, budget_s=20.0, steps=None, warmup=1, keys
     rows = min(rows, n0)
     if rows != probe_rows:
         ora = oracle_pool_for(w, rows, keys)
+    if steps is None:
+        # the whole pool fits the budget with room to spare: take more steps (about half the
+        # budget) so that the figure is not a handful of calls
+        n_steps = int(min(200, max(4, 0.5 * budget_s / max(per_row * nq_s * rows, 1e-12))))
     states, toks, queries = step_inputs(w, n_steps + warmup, rows_step, nq_s, "cpu", seed=0)
     def step(i):
         ora.append(W.to_bits(states[i]), toks[i].numpy(), tag=1_000_000 + i)

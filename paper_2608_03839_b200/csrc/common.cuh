@@ -48,6 +48,35 @@ __device__ __forceinline__ uint4 ld_stream16(const void* p) {
   return v;
 }
 
+// coherent 16-byte load (L2): for rows that another CTA of the same launch has just written
+__device__ __forceinline__ uint4 ld_cg16(const void* p) {
+  uint4 v;
+  asm volatile("ld.global.cg.v4.u32 {%0,%1,%2,%3}, [%4];"
+               : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+  return v;
+}
+__device__ __forceinline__ unsigned long long ld_acquire_u64(const unsigned long long* p) {
+  unsigned long long v;
+  asm volatile("ld.acquire.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
+  return v;
+}
+
+// A scan whose first CTAs append the step's rows: wait until all of them are in (every
+// appending CTA adds one to *ready after its row).  Bounded: after about two seconds the
+// pool's `stalled` flag is raised and the caller carries on (the status call reports it).
+__device__ __forceinline__ void wait_fused_rows(const FusedAppend& fa, DeviceStats* stats) {
+  unsigned long long t0 = 0;
+  for (uint32_t spin = 0; ld_acquire_u64(fa.ready) < fa.target; ++spin) {
+    if (spin == 0) asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t0));
+    if ((spin & 255u) == 255u) {
+      unsigned long long t1;
+      asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t1));
+      if (t1 - t0 > 2000000000ull) { atomicExch(&stats->stalled, 1); break; }
+    }
+    __nanosleep(64);
+  }
+}
+
 // ---------------------------------------------------- programmatic launch ------
 // Every kernel of the library is launched with programmatic stream serialization: its
 // blocks may be scheduled while the previous kernel of the stream is still draining, which

@@ -160,19 +160,6 @@ constexpr int kQ8Threads = kNormThreads;
 constexpr int kQ8Warps = kQ8Threads / 32;
 constexpr int kQ8Rows = 4;        // rows a warp scores together
 
-// coherent loads (L2) for rows that another CTA of the same launch has just written
-__device__ __forceinline__ uint4 ld_cg16(const void* p) {
-  uint4 v;
-  asm volatile("ld.global.cg.v4.u32 {%0,%1,%2,%3}, [%4];"
-               : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
-  return v;
-}
-__device__ __forceinline__ unsigned long long ld_acquire_u64(const unsigned long long* p) {
-  unsigned long long v;
-  asm volatile("ld.acquire.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
-  return v;
-}
-
 // two E4M3 codes -> two floats (exact)
 __device__ __forceinline__ float2 e4m3x2_to_float2(uint32_t two_codes) {
   uint32_t h2;
@@ -273,17 +260,7 @@ scan_gemv_e4m3_kernel(const uint8_t* __restrict__ codes, const float* __restrict
 
       const bool fresh = fa.n > 0 && rb + kQ8Rows > fa.row0;       // warp-uniform
       if (fresh && !fresh_ok) {
-        // rows of this step's append: wait (bounded) until all of them are in
-        unsigned long long t0 = 0;
-        for (uint32_t spin = 0; ld_acquire_u64(fa.ready) < fa.target; ++spin) {
-          if (spin == 0) asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t0));
-          if ((spin & 255u) == 255u) {
-            unsigned long long t1;
-            asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t1));
-            if (t1 - t0 > 2000000000ull) { atomicExch(&stats->stalled, 1); break; }
-          }
-          __nanosleep(64);
-        }
+        wait_fused_rows(fa, stats);       // rows of this step's append
         fresh_ok = true;
       }
 #pragma unroll 4

@@ -25,21 +25,6 @@ namespace oilbird {
 constexpr int kScanThreads = kNormThreads;
 constexpr int kScanWarps = kScanThreads / 32;
 constexpr int kRowsPerIter = 4;   // rows a warp scores together (shares each query load)
-constexpr unsigned long long kFuseWaitNs = 2000000000ull;
-
-// coherent 16-byte load (L2): for rows that another CTA of this launch has just written
-__device__ __forceinline__ uint4 ld_cg16(const void* p) {
-  uint4 v;
-  asm volatile("ld.global.cg.v4.u32 {%0,%1,%2,%3}, [%4];"
-               : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
-  return v;
-}
-__device__ __forceinline__ unsigned long long ld_acquire_u64(const unsigned long long* p) {
-  unsigned long long v;
-  asm volatile("ld.acquire.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
-  return v;
-}
-
 // Dot products of kRowsPerIter rows with the QT queries in shared memory; kFresh selects
 // the coherent load for rows written during this launch.
 template <int QT, bool kFresh>
@@ -167,17 +152,8 @@ scan_gemv_kernel(PoolView pv, const uint16_t* __restrict__ q_raw, int nq, int k,
       if (fa.n > 0 && rb + kRowsPerIter > fa.row0) {        // warp-uniform
         // rows of this step's append: wait (bounded) until all of them are in
         if (!fresh_ok) {
-          unsigned long long t0 = 0;
-          for (uint32_t spin = 0; ld_acquire_u64(fa.ready) < fa.target; ++spin) {
-            if (spin == 0) asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t0));
-            if ((spin & 255u) == 255u) {
-              unsigned long long t1;
-              asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t1));
-              if (t1 - t0 > kFuseWaitNs) { atomicExch(&stats->stalled, 1); break; }
-            }
-            __nanosleep(64);
-          }
-          fresh_ok = true;             // (after a time-out the status call reports the stall)
+          wait_fused_rows(fa, stats);
+          fresh_ok = true;
         }
         score_rows<QT, true>(rowp, qs, n_chunks, lane, acc);
       } else {

@@ -29,6 +29,11 @@ compact_kernel(unsigned char* keys, float* scales, int32_t* tok, int32_t* trace_
   const int64_t tid = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   const int64_t nthreads = (int64_t)gridDim.x * blockDim.x;
   const int64_t chunks_per_row = row_bytes >> 4;
+  if (head == 0) {
+    // only empty traces were dropped: nothing moves, but the traces are renumbered
+    for (int64_t i = tid; i < live; i += nthreads) trace_id[i] -= n_traces;
+    return;
+  }
   for (int64_t w0 = 0; w0 < live; w0 += head) {
     const int64_t rows = live - w0 < head ? live - w0 : head;
     // keys: rows [w0, w0+rows) <- rows [w0+head, ...), 16 bytes per thread and step
@@ -57,7 +62,7 @@ compact_kernel(unsigned char* keys, float* scales, int32_t* tok, int32_t* trace_
 cudaError_t launch_compact(unsigned char* keys, float* scales, int32_t* tok, int32_t* trace_id,
                            int64_t head, int64_t live, int64_t row_bytes, int32_t n_traces,
                            int32_t num_sms, cudaStream_t st) {
-  if (live <= 0 || head <= 0) return cudaSuccess;
+  if (live <= 0 || head < 0 || n_traces <= 0) return cudaSuccess;
   int per_sm = 0;
   cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, compact_kernel,
                                                                 kEvictThreads, 0);

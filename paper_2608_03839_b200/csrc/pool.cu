@@ -341,7 +341,7 @@ int oilbird_pool_evict_oldest(oilbird_pool_t* p, int32_t n_traces, int64_t* rows
   cudaError_t e = launch_compact((unsigned char*)p->keys, p->r.e4m3 ? p->scales : nullptr, p->tok,
                                  p->trace_id, head, live, row_bytes, nt, p->num_sms, st);
   if (e != cudaSuccess) return cuda_fail(e, "compaction kernel launch");
-  if (live > 0 && head > 0) p->launches += 1;
+  if (live > 0) p->launches += 1;
   // the host's copy of the trace table is the truth: renumber it, then publish it
   p->t_start.erase(p->t_start.begin(), p->t_start.begin() + nt);
   p->t_end.erase(p->t_end.begin(), p->t_end.begin() + nt);

@@ -89,6 +89,23 @@ def test_many_waves_a_short_trace_in_front_of_a_long_pool():
     assert int(out.idx[0, 0]) == 2 and out.cont_tok[0, 0].tolist() == [4, -1]
 
 
+def test_evicting_empty_traces_still_renumbers():
+    d = 32
+    g = torch.Generator(device="cuda").manual_seed(3)
+    pool, ora = B.Pool(d, 100), OraclePool(d)
+    empty = torch.empty(0, d, dtype=torch.bfloat16, device="cuda")
+    none = torch.empty(0, dtype=torch.int32, device="cuda")
+    for n, tag in ((0, 1), (0, 2), (9, 3), (0, 4), (5, 5)):
+        st = torch.randn(n, d, generator=g, device="cuda").to(torch.bfloat16) if n else empty
+        tk = torch.arange(n, dtype=torch.int32, device="cuda") if n else none
+        pool.append(st, tk, tag=tag)
+        ora.append(W.to_bits(st) if n else np.empty((0, d), np.uint16), tk.cpu().numpy(), tag=tag)
+    assert pool.evict_oldest(2) == ora.evict_oldest(2) == 0        # two empty traces
+    same_store(pool, ora)
+    assert pool.evict_oldest(2) == ora.evict_oldest(2) == 9        # one full, one empty
+    same_store(pool, ora)
+
+
 def test_eviction_keeps_global_positions_of_a_shard():
     d = 32
     g = torch.Generator(device="cuda").manual_seed(2)

@@ -1,0 +1,99 @@
+"""Randomised life cycles: a seeded sequence of appends, fused steps, evictions, resets and
+queries is applied to the CUDA pool and to the oracle alike; after every operation that
+returns results they are compared under the acceptance rule, and at the end (and after every
+eviction) the stored arrays must be identical bit for bit."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from oracle import OraclePool
+from paper_2608_03839_b200 import binding as B
+from paper_2608_03839_b200 import workloads as W
+from parity import check_query
+
+pytestmark = pytest.mark.gpu
+
+
+def same_store(pool, ora):
+    if pool.key_format == "bf16":
+        keys, tok, tid = pool.read_rows()
+        assert np.array_equal(keys, ora.keys)
+    else:
+        _, tok, tid = pool.read_rows()
+        codes, scales = pool.read_codes()
+        assert np.array_equal(codes, ora.codes) and np.array_equal(scales, ora.scales)
+    assert np.array_equal(tok, ora.tokens) and np.array_equal(tid, ora.trace_ids)
+    st, en, tg = pool.traces()
+    assert np.array_equal(st, ora.trace_starts) and np.array_equal(en, ora.trace_ends)
+    assert np.array_equal(tg, ora.trace_tags)
+
+
+@pytest.mark.parametrize("fmt", ["bf16", "e4m3"])
+@pytest.mark.parametrize("seed", range(8))
+def test_random_life_cycle(fmt, seed):
+    rng = np.random.default_rng(1000 + seed)
+    d = int(rng.choice([64, 256, 1024]))
+    cap = 6000
+    pool, ora = B.Pool(d, cap, max_nq=8, max_k=32, max_traces=400, key_format=fmt), OraclePool(d, fmt)
+    g = torch.Generator(device="cuda").manual_seed(seed)
+    cent = torch.randn(16, d, generator=g, device="cuda")
+    next_tag = [1]
+
+    def rows(n):
+        c = torch.randint(0, 16, (n,), generator=g, device="cuda")
+        st = (cent[c] + 0.3 * torch.randn(n, d, generator=g, device="cuda")).to(torch.bfloat16)
+        tk = torch.randint(0, 5000, (n,), generator=g, device="cuda", dtype=torch.int32)
+        return st, tk
+
+    def params(nq):
+        k = int(rng.choice([1, 4, 8, 17, 32]))
+        pr = B.QueryParams(k=k, theta=float(rng.choice([-2.0, 0.5, 0.8])),
+                           depth_mode=int(rng.choice([B.DEPTH_FIXED, B.DEPTH_TIERED])),
+                           cont_len=int(rng.choice([1, 4, 16])), offset=int(rng.choice([0, 1, 2])))
+        if fmt == "bf16" and nq >= 1:
+            pr.path = int(rng.choice([B.PATH_AUTO, B.PATH_GEMV, B.PATH_TENSOR]))
+        return pr
+
+    for op_no in range(100):
+        op = rng.choice(["append", "step", "step", "query", "evict", "reset"],
+                        p=[0.25, 0.2, 0.2, 0.2, 0.12, 0.03])
+        if op in ("append", "step"):
+            n = int(rng.choice([0, 1, 7, 8, 40, 64, 65, 200]))
+            if len(pool) + n > cap or pool.num_traces + 1 > 390:
+                op, n = "evict", 0
+        if op == "append":
+            st, tk = rows(n)
+            new = bool(rng.random() < 0.7) or len(pool) == 0
+            tag = next_tag[0]; next_tag[0] += 1
+            pool.append(st, tk, tag=tag, new_trace=new)
+            ora.append(W.to_bits(st), tk.cpu().numpy(), tag=tag, new_trace=new)
+        elif op == "step":
+            st, tk = rows(n)
+            nq = int(rng.choice([1, 1, 2, 3, 8]))
+            q = rows(nq)[0]
+            if n > 0:
+                q[0] = st[n - 1]
+            new = bool(rng.random() < 0.7) or len(pool) == 0
+            tag = next_tag[0]; next_tag[0] += 1
+            pr = params(nq)
+            out = pool.step(st, tk, q, pr, tag=tag, new_trace=new)
+            ora.append(W.to_bits(st), tk.cpu().numpy(), tag=tag, new_trace=new)
+            if len(ora):
+                check_query(out, ora, W.to_bits(q), pr)
+        elif op == "query":
+            nq = int(rng.choice([1, 2, 5, 8]))
+            q = rows(nq)[0]
+            pr = params(nq)
+            out = pool.query(q, pr)
+            check_query(out, ora, W.to_bits(q), pr)
+        elif op == "evict":
+            nt = int(rng.integers(0, max(2, pool.num_traces // 2 + 1)))
+            assert pool.evict_oldest(nt) == ora.evict_oldest(nt)
+            same_store(pool, ora)
+        else:
+            pool.reset()
+            ora.reset()
+        assert len(pool) == len(ora) and pool.num_traces == ora.num_traces
+    same_store(pool, ora)
+    assert pool.stats()["stalled"] == 0

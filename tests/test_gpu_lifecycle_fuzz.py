@@ -35,7 +35,8 @@ def test_random_life_cycle(fmt, seed):
     rng = np.random.default_rng(1000 + seed)
     d = int(rng.choice([64, 256, 1024]))
     cap = 6000
-    pool, ora = B.Pool(d, cap, max_nq=8, max_k=32, max_traces=400, key_format=fmt), OraclePool(d, fmt)
+    pool = B.Pool(d, cap, max_nq=8, max_k=32, max_traces=400, max_append=256, key_format=fmt)
+    ora = OraclePool(d, fmt)
     g = torch.Generator(device="cuda").manual_seed(seed)
     cent = torch.randn(16, d, generator=g, device="cuda")
     next_tag = [1]
@@ -62,11 +63,15 @@ def test_random_life_cycle(fmt, seed):
             n = int(rng.choice([0, 1, 7, 8, 40, 64, 65, 200]))
             if len(pool) + n > cap or pool.num_traces + 1 > 390:
                 op, n = "evict", 0
+        host = bool(rng.random() < 0.3)          # through the host-buffer entry points
         if op == "append":
             st, tk = rows(n)
             new = bool(rng.random() < 0.7) or len(pool) == 0
             tag = next_tag[0]; next_tag[0] += 1
-            pool.append(st, tk, tag=tag, new_trace=new)
+            if host:
+                pool.append_host(st.cpu(), tk.cpu(), tag=tag, new_trace=new)
+            else:
+                pool.append(st, tk, tag=tag, new_trace=new)
             ora.append(W.to_bits(st), tk.cpu().numpy(), tag=tag, new_trace=new)
         elif op == "step":
             st, tk = rows(n)
@@ -77,7 +82,11 @@ def test_random_life_cycle(fmt, seed):
             new = bool(rng.random() < 0.7) or len(pool) == 0
             tag = next_tag[0]; next_tag[0] += 1
             pr = params(nq)
-            out = pool.step(st, tk, q, pr, tag=tag, new_trace=new)
+            if host:
+                out = B.QueryOut.empty(nq, pr.k, pr.cont_len, "cpu")
+                pool.step_host(st.cpu(), tk.cpu(), q.cpu(), pr, out, tag=tag, new_trace=new)
+            else:
+                out = pool.step(st, tk, q, pr, tag=tag, new_trace=new)
             ora.append(W.to_bits(st), tk.cpu().numpy(), tag=tag, new_trace=new)
             if len(ora):
                 check_query(out, ora, W.to_bits(q), pr)
@@ -85,7 +94,7 @@ def test_random_life_cycle(fmt, seed):
             nq = int(rng.choice([1, 2, 5, 8]))
             q = rows(nq)[0]
             pr = params(nq)
-            out = pool.query(q, pr)
+            out = pool.query_host(q.cpu(), pr) if host else pool.query(q, pr)
             check_query(out, ora, W.to_bits(q), pr)
         elif op == "evict":
             nt = int(rng.integers(0, max(2, pool.num_traces // 2 + 1)))

@@ -311,7 +311,8 @@ __device__ __forceinline__ void merge_lists(const u64* __restrict__ partial, int
   // many lists in flight per warp: the loads, not the merges, set the pace (with two CTAs
   // per SM a warp folds about ten lists, so one round of loads covers the common case)
   constexpr int PF = E == 1 ? 10 : (E == 2 ? 5 : 3);
-  const bool filter = k <= kMergeWarps && n_lists <= kMergeWarps * PF;   // one round of loads
+  // (k == 0: the caller does not want the filter)
+  const bool filter = k >= 1 && k <= kMergeWarps && n_lists <= kMergeWarps * PF;   // one round of loads
   u64 b[PF][E];
   if (filter) {
     u64 best = 0;

@@ -26,11 +26,15 @@
 // MMA-issuing thread show ~360 cycles to issue the four tcgen05.mma and the commit of a
 // 16 KB k-block (~70 cycles per instruction, against ~90 cycles of waiting for the data
 // when HBM is idle), i.e. with queries as the N operand a 128 x N x 16 instruction carries
-// only 4 KB of keys and the issue rate, not the tensor pipe, bounds the per-SM rate.  (With
-// the roles swapped, queries as M = 128 and 256 key rows as N, an instruction would carry
-// 8 KB; that is the next step for this kernel, together with an epilogue in which a thread
-// owns a query.)  Then come the first tile's epilogue (7-10 us), the query normalisation
-// kernel and the merge.  Cutting the pool into per-CTA row ranges at 32-row granularity
+// only 4 KB of keys and the issue rate, not the tensor pipe, bounds the per-SM rate.  Then
+// come the first tile's epilogue (7-10 us), the query normalisation kernel and the merge.
+// A variant with the roles swapped (queries as M = 128, one query per TMEM lane and per
+// epilogue thread with its threshold in a register and a queue only it writes; 256 key rows
+// as N, so that an instruction carries 8 KB of keys) was written and passes the same tests,
+// but is slower everywhere: 0.90 instead of 1.03 of the measured HBM rate at nq = 16 and
+// 0.73 instead of 0.81 at nq = 128 on the 8.6 GB pool (every stage carries a 16 KB query
+// tile whatever nq is), and 2-3x slower on small pools, where only nq/32 of the four
+// epilogue warps share the sorting of a CTA's first tile.  Cutting the pool into per-CTA row ranges at 32-row granularity
 // (ragged ends fetched as 32-row boxes) so that all SMs get equal rows, ring depths up to
 // 12 and seeding the first tile's thresholds from per-warp 32-bit sorts of the scores were
 // measured and bring nothing.

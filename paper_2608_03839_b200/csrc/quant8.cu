@@ -213,7 +213,10 @@ scan_gemv_e4m3_kernel(const uint8_t* __restrict__ codes, const float* __restrict
     }
     __threadfence();                   // this thread's part of the row, before the count
     __syncthreads();
-    if (threadIdx.x == 0) atomicAdd(fa.ready, 1ull);
+    if (threadIdx.x == 0) {
+      __threadfence();                 // cumulative: the whole CTA's row, as seen through the barrier
+      atomicAdd(fa.ready, 1ull);
+    }
   }
   bool fresh_ok = fa.n == 0;           // this warp has seen the appended rows arrive
 

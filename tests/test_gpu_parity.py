@@ -34,6 +34,16 @@ def test_append_matches_oracle_bit_for_bit(d):
     st[7] = 0                                   # zero row
     st[11, d // 2] = float("inf")               # non-finite rows are stored as zero keys
     st[13, 0] = float("nan")
+    # rows that leave the normal-number fast path of the normalisation: a subnormal element,
+    # a negative zero, finite values near the top of the range (sum of squares above 2^256),
+    # a row of subnormals only
+    sub = torch.tensor([1, 0x7f, 0x8003], dtype=torch.int32).to(torch.int16).view(torch.bfloat16).cuda()
+    st[20, 1] = sub[0]
+    st[21, 0] = -0.0
+    st[22] = 3.0e38
+    st[22, d - 1] = -1.5e38
+    st[23] = sub[1]
+    st[23, d // 3] = sub[2]
     tk = torch.randint(0, 50000, (n,), generator=g, device="cuda", dtype=torch.int32)
     pool, ora = B.Pool(d, 1000), OraclePool(d)
     # three traces, the second extended in two pieces, one empty append in between
@@ -50,6 +60,29 @@ def test_append_matches_oracle_bit_for_bit(d):
     assert t.tolist() == ora.trace_tags.tolist()
     assert pool.stats()["degenerate_rows"] == ora.degenerate_rows == 3
     assert np.all(keys[[7, 11, 13]] == 0)
+
+
+@pytest.mark.parametrize("d", [200, 4096, 4104, 8192, 12288])
+def test_bulk_append_matches_oracle_bit_for_bit(d):
+    # thousands of rows per call take the prefetching kernel (a few rows per resident block);
+    # row counts that are not a multiple of the grid, rows held in registers in part only
+    g = torch.Generator(device="cuda").manual_seed(100 + d)
+    n = 3011
+    st = (torch.randn(n, d, generator=g, device="cuda") * 2).to(torch.bfloat16)
+    st[5] = 0
+    st[n - 1, d - 1] = float("inf")
+    st[1500, 3] = float("nan")
+    tk = torch.randint(0, 50000, (n,), generator=g, device="cuda", dtype=torch.int32)
+    pool, ora = B.Pool(d, n + 200), OraclePool(d)
+    for lo, hi, tag in ((0, 100, 3), (100, n, 4)):          # a small call, then a bulk one
+        pool.append(st[lo:hi].contiguous(), tk[lo:hi].contiguous(), tag=tag, new_trace=True)
+        ora.append(W.to_bits(st[lo:hi]), tk[lo:hi].cpu().numpy(), tag=tag, new_trace=True)
+    keys, tok, tid = pool.read_rows()
+    assert np.array_equal(keys, ora.keys)
+    assert np.array_equal(tok, ora.tokens) and np.array_equal(tid, ora.trace_ids)
+    s, e, t = pool.traces()
+    assert e.tolist() == ora.trace_ends.tolist() and t.tolist() == ora.trace_tags.tolist()
+    assert pool.stats()["degenerate_rows"] == ora.degenerate_rows == 3
 
 
 def test_append_capacity_and_argument_errors():

@@ -41,21 +41,135 @@ __device__ __forceinline__ uint32_t e4m3_encode(double t) {
   return sign | (uint32_t)(((e + 7) << 3) | (n - 8));
 }
 
+// The exact code of one element, out of line: the bulk quantiser reaches it for a few
+// elements in a hundred thousand, and sixteen inlined copies per loop body would not fit the
+// instruction cache.
+__device__ __noinline__ uint32_t e4m3_encode_element(float x, double inv, double sc) {
+  return e4m3_encode(((double)x * inv) / sc);
+}
+
 // --------------------------------------------------------------------- append ---
 // Quantise one raw bf16 row (d a multiple of 16) into codes + scale.  All kNormThreads
 // threads of the block take part; two passes over the row (it is re-read from L2):
 // squared norm and peak, then the codes.  Returns true if the row was usable.
+//
+// kFast (the bulk append): rows whose elements are all normal finite numbers avoid the
+// float<->double conversions, the double division and the general encoder, which together
+// held the kernel at a sixth of the memory system's speed.
+//  - the doubles are built from the bf16 bits (exponent field e + 896, fraction on top), the
+//    peak is the largest magnitude pattern; sums, norm and scale are the same numbers in the
+//    same order as on the exact path;
+//  - per element t' = x * g with g = (1/||x||) / scale stands in for t = (x / ||x||) / scale.
+//    The two differ by at most four units in the last place of a double, so they round to the
+//    same code unless a rounding boundary of the code grid lies within that distance of t'.
+//    Boundaries are numbers with five significant bits, so t' is near one when bits 16..0 of
+//    its high word read 0xffff or 0x10000 and the low word is within 256 of wrapping.  (The
+//    high-word pattern alone is common, 5 elements in a thousand: x and the peak are 8-bit
+//    significands and the scale is their ratio rounded to float, which puts many t' within
+//    2^-24 of a boundary; the low word separates those from the true near-ties.)  Near-ties
+//    and elements below the normal range of the format (t' < 2^-6, one in ten thousand) go
+//    through the exact encoder; for all others the code is the high word rounded at bit 17
+//    and rebiased, capped at 448.
+// A row with a zero, subnormal, Inf or NaN anywhere is redone on the exact path.
+template <bool kFast = false>
 __device__ __forceinline__ bool quantize_row_e4m3(const uint16_t* __restrict__ src, int d,
                                                   uint8_t* __restrict__ dst, float* scale_out) {
   __shared__ double s_ss[kNormThreads / 32];
   __shared__ float s_mx[kNormThreads / 32];
   __shared__ int s_bad[kNormThreads / 32];
   __shared__ double s_inv;
+  __shared__ double s_g;
   __shared__ float s_scale;
   __shared__ int s_ok;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int n16 = d >> 4;
   const uint4* src4 = reinterpret_cast<const uint4*>(src);
+  uint4* dst4 = reinterpret_cast<uint4*>(dst);
+
+  if (kFast) {
+    double fs = 0.0;
+    uint32_t umin = 0xffffffffu, umax = 0u;
+    for (int c = threadIdx.x; c < 2 * n16; c += kNormThreads) {
+      const uint4 hv = __ldg(src4 + c);
+      const uint32_t w[4] = {hv.x, hv.y, hv.z, hv.w};
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const uint32_t ul = (w[j] & 0x7fffu) << 13, uh = (w[j] & 0x7fff0000u) >> 3;
+        umin = min(umin, min(ul, uh));
+        umax = max(umax, max(ul, uh));
+        const double lo = __hiloint2double((int)(ul + 0x38000000u), 0);
+        const double hi = __hiloint2double((int)(uh + 0x38000000u), 0);
+        fs += lo * lo;
+        fs += hi * hi;
+      }
+    }
+#pragma unroll
+    for (int m = 16; m; m >>= 1) {
+      fs += __shfl_xor_sync(0xffffffffu, fs, m);
+      umin = min(umin, __shfl_xor_sync(0xffffffffu, umin, m));
+      umax = max(umax, __shfl_xor_sync(0xffffffffu, umax, m));
+    }
+    if (lane == 0) {
+      s_ss[warp] = fs;
+      s_mx[warp] = __uint_as_float(umax << 3);           // the pattern back in float position
+      s_bad[warp] = (umin < 0x00100000u) | (umax >= 0x0ff00000u);   // exponent field 0 or 255
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      double tot = 0.0;
+      float peak = 0.f;
+      int b = 0;
+      for (int w = 0; w < kNormThreads / 32; ++w) { tot += s_ss[w]; peak = fmaxf(peak, s_mx[w]); b |= s_bad[w]; }
+      if (!b) {
+        const double inv = 1.0 / sqrt(tot);
+        const float scale = (float)((double)peak * inv / 448.0);
+        s_inv = inv;
+        s_scale = scale;
+        s_g = inv / (double)scale;
+        *scale_out = scale;
+      }
+      s_ok = b ? -1 : 1;
+    }
+    __syncthreads();
+    if (s_ok == 1) {
+      const double inv = s_inv, sc = (double)s_scale, g = s_g;
+      for (int c = threadIdx.x; c < n16; c += kNormThreads) {
+        uint32_t o[4] = {0, 0, 0, 0};
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+          const uint4 hv = __ldg(src4 + 2 * c + h);
+          const uint32_t w[4] = {hv.x, hv.y, hv.z, hv.w};
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            uint32_t cd[2];
+#pragma unroll
+            for (int half = 0; half < 2; ++half) {
+              const uint32_t u = half ? (w[j] & 0x7fff0000u) >> 3 : (w[j] & 0x7fffu) << 13;
+              const uint32_t sign = half ? (w[j] >> 24) & 0x80u : (w[j] >> 8) & 0x80u;
+              const double t = __hiloint2double((int)(u + 0x38000000u), 0) * g;
+              const uint32_t th = (uint32_t)__double2hiint(t);
+              bool exact = th < 0x3f900000u;
+              if (((th + 1u) & 0x1fffeu) == 0x10000u) {      // 0xffff or 0x10000: low word decides
+                const uint32_t tl = (uint32_t)__double2loint(t);
+                exact |= (th & 1u) ? tl >= 0xffffff00u : tl < 0x100u;
+              }
+              if (exact) {
+                cd[half] = e4m3_encode_element(half ? bf16_hi(w[j]) : bf16_lo(w[j]), inv, sc);
+              } else {
+                cd[half] = min(((th + 0x10000u) >> 17) - (1016u << 3), 0x7eu) | sign;
+              }
+            }
+            const int e = h * 8 + j * 2;                     // element index within the 16
+            o[e >> 2] |= (cd[0] << ((e & 3) * 8)) | (cd[1] << (((e + 1) & 3) * 8));
+          }
+        }
+        dst4[c] = make_uint4(o[0], o[1], o[2], o[3]);
+      }
+      __syncthreads();   // the shared scratch is reused by the next row
+      return true;
+    }
+  }
+
   double ss = 0.0;
   float mx = 0.f;
   int bad = 0;
@@ -94,7 +208,6 @@ __device__ __forceinline__ bool quantize_row_e4m3(const uint16_t* __restrict__ s
   }
   __syncthreads();
   const double inv = s_inv, sc = (double)s_scale;
-  uint4* dst4 = reinterpret_cast<uint4*>(dst);
   for (int c = threadIdx.x; c < n16; c += kNormThreads) {
     uint32_t o[4] = {0, 0, 0, 0};
     if (sc != 0.0) {
@@ -135,7 +248,7 @@ append_e4m3_kernel(const uint16_t* __restrict__ states, const int32_t* __restric
   }
   for (int64_t r = blockIdx.x; r < n; r += gridDim.x) {
     const int64_t row = row0 + r;
-    const bool ok = quantize_row_e4m3(states + r * d, d, codes + row * d, scales + row);
+    const bool ok = quantize_row_e4m3<true>(states + r * d, d, codes + row * d, scales + row);
     if (threadIdx.x == 0) {
       tok[row] = tokens[r];
       trace_id[row] = trace;

@@ -642,6 +642,72 @@ def run_evict(args):
     pool.close()
 
 
+def run_load(args):
+    """Store step in bulk (Section 4 (i), Eq. 1): one step = reset the pool and load the whole
+    configuration's rows again in calls of 4096 rows (a long trace's worth).  Reported in rows
+    per second; the roofline is the append kernel's: every state read once, every key written
+    once."""
+    from paper_2608_03839_b200 import binding as B
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda:0")
+    w = W.CONFIGS[args.config]
+    n0 = args.rows or w.n_rows
+    chunk = 4096
+    n_calls = max(1, n0 // chunk)
+    K, Wm = args.steps, args.warmup
+    pool = B.Pool(w.d, n_calls * chunk, max_nq=1, max_k=w.k, max_traces=n_calls + 8,
+                  key_format=args.keys)
+    # source states: distinct rows for every call (n0 x d bf16 stays resident, as a prefill's
+    # hidden states would)
+    g = torch.Generator(device=dev).manual_seed(1234)
+    src = [(torch.randn(chunk, w.d, generator=g, device=dev)).to(torch.bfloat16)
+           for _ in range(n_calls)]
+    tok = torch.randint(0, 50000, (chunk,), generator=g, device=dev, dtype=torch.int32)
+    torch.cuda.synchronize()
+
+    def step():
+        pool.reset()
+        for i in range(n_calls):
+            pool.append(src[i], tok, tag=i + 1)
+
+    for _ in range(Wm):
+        step()
+    torch.cuda.synchronize()
+    sampler = ClockSampler(physical_device(0))
+    sampler.start()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    l0 = pool.launch_count
+    e0.record()
+    for _ in range(K):
+        step()
+    e1.record()
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    launches = pool.launch_count - l0
+    total_ms = e0.elapsed_time(e1)
+    rows = n_calls * chunk
+    out_bytes = w.d * 2 if args.keys == "bf16" else w.d + 4
+    moved = float(rows) * (w.d * 2 + 4 + out_bytes + 8)   # state + token in, key (+scale) + token + trace id out
+    per_step_ms = total_ms / K
+    peaks, peak_kind = measured_peaks()
+    kern = "append_bulk_kernel" if args.keys == "bf16" else "append_e4m3_kernel"
+    line = {"metric": "rows_appended_per_sec", "value": rows * K / (total_ms / 1e3),
+            "unit": "rows/s", "n_gpus": 1, "steps": K, "warmup": Wm, "ms_per_step": per_step_ms,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": f"{args.keys} keys, fp64 norm", "data": "synthetic",
+            "config": {"workload": f"load: {rows} rows x d={w.d} into a {args.keys} pool in "
+                                   f"{n_calls} calls of {chunk} rows; inputs "
+                                   f"{rows * w.d * 2 / 1e6:.0f} MB (larger than L2)"},
+            "clocks": clocks, "gpu_launches": int(launches),
+            "roofline": {"bound": "hbm", "kernel": kern,
+                         "achieved": moved / (per_step_ms * 1e-3) / 1e9, "peak": peaks["hbm_gbs"],
+                         "unit": "GB/s", "frac": moved / (per_step_ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
+                         "peak_kind": peak_kind, "bytes_per_launch": moved / n_calls,
+                         "traffic": None}}
+    print(json.dumps(line), flush=True)
+    pool.close()
+
+
 def run_merge(args):
     """Third workload: chain post-filter + tree merge for a batch of requests (paper sizes:
     8 semantic chains of up to 48 tokens + 7 other chains into a 44-node tree, 16 of 60 nodes)."""
@@ -782,8 +848,9 @@ def main():
     ap.add_argument("--keys", default="bf16", choices=["bf16", "e4m3"],
                     help="stored key format: the paper's 16-bit keys, or the bounded-store "
                          "variant with 8-bit keys (FP8 E4M3 + one scale per row)")
-    ap.add_argument("--workload", default="pool", choices=["pool", "ring", "merge", "evict"],
-                    help="pool: the trace-store query path (default); ring: the recycled pool")
+    ap.add_argument("--workload", default="pool", choices=["pool", "ring", "merge", "evict", "load"],
+                    help="pool: the trace-store query path (default); ring: the recycled pool; "
+                         "evict: bounded store; merge: chain merge; load: bulk trace load")
     ap.add_argument("--sharded", action="store_true",
                     help="one logical pool row-sharded over the ranks (default: one pool per rank)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -803,6 +870,11 @@ def main():
         args.steps = 20 if args.steps is None else args.steps
         args.warmup = 3 if args.warmup is None else max(args.warmup, 3)
         run_evict(args)
+        return
+    if args.workload == "load":
+        args.steps = 10 if args.steps is None else args.steps
+        args.warmup = 3 if args.warmup is None else max(args.warmup, 3)
+        run_load(args)
         return
     if args.workload == "merge":
         args.steps = 200 if args.steps is None else args.steps

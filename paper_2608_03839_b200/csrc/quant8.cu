@@ -59,7 +59,7 @@ __device__ __noinline__ uint32_t e4m3_encode_element(float x, double inv, double
 //  - the doubles are built from the bf16 bits (exponent field e + 896, fraction on top), the
 //    peak is the largest magnitude pattern; sums, norm and scale are the same numbers in the
 //    same order as on the exact path;
-//  - per element t' = x * g with g = (1/||x||) / scale stands in for t = (x / ||x||) / scale.
+//  - per element t' = |x| * g with g = (1/||x||) / scale stands in for t = (|x| / ||x||) / scale.
 //    The two differ by at most four units in the last place of a double, so they round to the
 //    same code unless a rounding boundary of the code grid lies within that distance of t'.
 //    Boundaries are numbers with five significant bits, so t' is near one when bits 16..0 of
@@ -67,16 +67,22 @@ __device__ __noinline__ uint32_t e4m3_encode_element(float x, double inv, double
 //    high-word pattern alone is common, 5 elements in a thousand: x and the peak are 8-bit
 //    significands and the scale is their ratio rounded to float, which puts many t' within
 //    2^-24 of a boundary; the low word separates those from the true near-ties.)  Near-ties
-//    and elements below the normal range of the format (t' < 2^-6, one in ten thousand) go
-//    through the exact encoder; for all others the code is the high word rounded at bit 17
-//    and rebiased, capped at 448.
-// A row with a zero, subnormal, Inf or NaN anywhere is redone on the exact path.
+//    go through the exact encoder, out of line.
+//  - for all others the code comes from the hardware: t' is handed over as a float that holds
+//    its exponent, the 20 fraction bits of the double's high word and one sticky bit for the
+//    rest, and cvt.rn.satfinite.e4m3x2.f32 rounds two of them to nearest even, subnormal
+//    codes and the cap at 448 included.  (The sticky bit keeps the side of the boundary; a
+//    plain double -> float conversion would round many of the common 2^-24 cases onto the
+//    boundary itself.)  The four sign bits of a word of codes are picked from the inputs.
+// A row with a zero, subnormal, Inf or NaN anywhere, or with an element more than 2^40 below
+// its peak, is redone on the exact path.
 template <bool kFast = false>
 __device__ __forceinline__ bool quantize_row_e4m3(const uint16_t* __restrict__ src, int d,
                                                   uint8_t* __restrict__ dst, float* scale_out) {
   __shared__ double s_ss[kNormThreads / 32];
   __shared__ float s_mx[kNormThreads / 32];
   __shared__ int s_bad[kNormThreads / 32];
+  __shared__ uint32_t s_lo[kNormThreads / 32];
   __shared__ double s_inv;
   __shared__ double s_g;
   __shared__ float s_scale;
@@ -112,14 +118,21 @@ __device__ __forceinline__ bool quantize_row_e4m3(const uint16_t* __restrict__ s
     if (lane == 0) {
       s_ss[warp] = fs;
       s_mx[warp] = __uint_as_float(umax << 3);           // the pattern back in float position
-      s_bad[warp] = (umin < 0x00100000u) | (umax >= 0x0ff00000u);   // exponent field 0 or 255
+      // exponent field 0 or 255 somewhere, or an element more than 2^40 below the peak (its
+      // t' could leave the float range the encoder below works in)
+      s_bad[warp] = (umin < 0x00100000u) | (umax >= 0x0ff00000u);
+      s_lo[warp] = umin;
     }
     __syncthreads();
     if (threadIdx.x == 0) {
       double tot = 0.0;
       float peak = 0.f;
       int b = 0;
-      for (int w = 0; w < kNormThreads / 32; ++w) { tot += s_ss[w]; peak = fmaxf(peak, s_mx[w]); b |= s_bad[w]; }
+      uint32_t lo_all = 0xffffffffu;
+      for (int w = 0; w < kNormThreads / 32; ++w) {
+        tot += s_ss[w]; peak = fmaxf(peak, s_mx[w]); b |= s_bad[w]; lo_all = min(lo_all, s_lo[w]);
+      }
+      b |= ((__float_as_uint(peak) >> 23) - (lo_all >> 20)) >= 40u;
       if (!b) {
         const double inv = 1.0 / sqrt(tot);
         const float scale = (float)((double)peak * inv / 448.0);
@@ -134,34 +147,43 @@ __device__ __forceinline__ bool quantize_row_e4m3(const uint16_t* __restrict__ s
     if (s_ok == 1) {
       const double inv = s_inv, sc = (double)s_scale, g = s_g;
       for (int c = threadIdx.x; c < n16; c += kNormThreads) {
-        uint32_t o[4] = {0, 0, 0, 0};
+        uint32_t o[4];
 #pragma unroll
         for (int h = 0; h < 2; ++h) {
           const uint4 hv = __ldg(src4 + 2 * c + h);
           const uint32_t w[4] = {hv.x, hv.y, hv.z, hv.w};
+          uint32_t c16[4];
 #pragma unroll
           for (int j = 0; j < 4; ++j) {
-            uint32_t cd[2];
-#pragma unroll
-            for (int half = 0; half < 2; ++half) {
-              const uint32_t u = half ? (w[j] & 0x7fff0000u) >> 3 : (w[j] & 0x7fffu) << 13;
-              const uint32_t sign = half ? (w[j] >> 24) & 0x80u : (w[j] >> 8) & 0x80u;
-              const double t = __hiloint2double((int)(u + 0x38000000u), 0) * g;
-              const uint32_t th = (uint32_t)__double2hiint(t);
-              bool exact = th < 0x3f900000u;
-              if (((th + 1u) & 0x1fffeu) == 0x10000u) {      // 0xffff or 0x10000: low word decides
-                const uint32_t tl = (uint32_t)__double2loint(t);
-                exact |= (th & 1u) ? tl >= 0xffffff00u : tl < 0x100u;
-              }
-              if (exact) {
-                cd[half] = e4m3_encode_element(half ? bf16_hi(w[j]) : bf16_lo(w[j]), inv, sc);
-              } else {
-                cd[half] = min(((th + 0x10000u) >> 17) - (1016u << 3), 0x7eu) | sign;
-              }
+            // |x| of the word's two elements as doubles, times g
+            const uint32_t hl = (w[j] & 0x7fffu) * 8192u + 0x38000000u;
+            const uint32_t hh = __umulhi(w[j] & 0x7fff0000u, 0x20000000u) + 0x38000000u;
+            const double t0 = __hiloint2double((int)hl, 0) * g;
+            const double t1 = __hiloint2double((int)hh, 0) * g;
+            const uint32_t a0 = (uint32_t)__double2hiint(t0), b0 = (uint32_t)__double2loint(t0);
+            const uint32_t a1 = (uint32_t)__double2hiint(t1), b1 = (uint32_t)__double2loint(t1);
+            // the same value as a float: exponent rebiased (by -896 << 23, modulo 2^32), the
+            // 20 fraction bits of the high word, and a sticky last bit for the low word, so
+            // that the hardware's round-to-nearest-even into E4M3 (subnormal codes and the
+            // cap at 448 included) sees on which side of a boundary t' lies
+            const float f0 = __uint_as_float(((a0 << 3) + 0x40000000u) | min(b0, 1u));
+            const float f1 = __uint_as_float(((a1 << 3) + 0x40000000u) | min(b1, 1u));
+            uint16_t two;
+            asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(two) : "f"(f1), "f"(f0));
+            uint32_t cd = two;
+            const bool n0 = ((a0 + 1u) & 0x1fffeu) == 0x10000u;   // 0xffff or 0x10000:
+            const bool n1 = ((a1 + 1u) & 0x1fffeu) == 0x10000u;   // the low word decides
+            if (n0 | n1) {
+              if (n0 && ((a0 & 1u) ? b0 >= 0xffffff00u : b0 < 0x100u))
+                cd = (cd & 0xff00u) | (e4m3_encode_element(bf16_lo(w[j]), inv, sc) & 0x7fu);
+              if (n1 && ((a1 & 1u) ? b1 >= 0xffffff00u : b1 < 0x100u))
+                cd = (cd & 0x00ffu) | ((e4m3_encode_element(bf16_hi(w[j]), inv, sc) & 0x7fu) << 8);
             }
-            const int e = h * 8 + j * 2;                     // element index within the 16
-            o[e >> 2] |= (cd[0] << ((e & 3) * 8)) | (cd[1] << (((e + 1) & 3) * 8));
+            c16[j] = cd;
           }
+          // four codes per word, then the four sign bits (bit 15 and 31 of each input word)
+          o[2 * h] = (c16[0] | (c16[1] << 16)) | (__byte_perm(w[0], w[1], 0x7531) & 0x80808080u);
+          o[2 * h + 1] = (c16[2] | (c16[3] << 16)) | (__byte_perm(w[2], w[3], 0x7531) & 0x80808080u);
         }
         dst4[c] = make_uint4(o[0], o[1], o[2], o[3]);
       }

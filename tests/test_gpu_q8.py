@@ -50,6 +50,42 @@ def test_codes_and_scales_match_oracle_bit_for_bit(d):
     assert not codes[7].any() and scales[7] == 0
 
 
+@pytest.mark.parametrize("d", [64, 4096])
+def test_rows_whose_elements_sit_on_code_boundaries(d):
+    # x / peak = 3 * 2^-j or 5 * 2^-j / 7 ... : with a power-of-two peak, 448 x / peak = 21 * 2^m
+    # lies exactly between two codes, and only the rounding of the stored scale (a different
+    # one per row, through the norm) decides the side.  Elements far below the peak (a spread
+    # of more than 2^40) and rows mixing all of it with ordinary values are in as well.
+    rng = np.random.default_rng(7 + d)
+    n = 400
+    rows = np.zeros((n, d), np.float32)
+    for r in range(n):
+        peak = 2.0 ** rng.integers(-20, 20)
+        j = rng.integers(2, 9, size=d)
+        vals = np.where(rng.random(d) < 0.5, 3.0, 1.0) * 2.0 ** (-j) * peak
+        vals *= rng.choice([-1.0, 1.0], size=d)
+        if r % 3 == 1:                                   # ordinary values mixed in: moves the norm
+            m = rng.random(d) < 0.3
+            vals[m] = rng.standard_normal(m.sum()) * 0.05 * peak
+        if r % 7 == 3:
+            vals[rng.integers(0, d)] = peak * 2.0 ** -45  # far below the peak
+        vals[rng.integers(0, d)] = peak
+        rows[r] = vals
+    st = torch.from_numpy(rows).to(torch.bfloat16).cuda()
+    tok = torch.arange(n, dtype=torch.int32, device="cuda")
+    pool = B.Pool(d, n, key_format="e4m3")
+    ora = OraclePool(d, "e4m3")
+    pool.append(st, tok, tag=1)
+    ora.append(W.to_bits(st), tok.cpu().numpy(), tag=1)
+    codes, scales = pool.read_codes()
+    assert np.array_equal(scales.view(np.uint32), ora.scales.view(np.uint32))
+    assert np.array_equal(codes, ora.codes)
+    # the planted boundary values did land on both sides across the rows
+    rb = st.float().cpu().numpy()
+    c84 = codes[(np.abs(rb) == 0.1875 * np.abs(rb).max(1, keepdims=True))] & 0x7f
+    assert len(set(c84.tolist())) >= 2
+
+
 @pytest.mark.parametrize("d", [16, 64, 256, 1024, 4096])
 def test_closed_form_pool_scores_are_exact(d):
     # +-1 rows: every code is +-448 and s = (1 - 2 Hamming / d) * (scale * 448 * sqrt(d)), the

@@ -7,8 +7,9 @@
 //
 // One CTA per row (see normalize.cuh for the arithmetic).  The work is a single pass
 // over n*d*2 bytes in and out.  Measured on bulk loads (tens of thousands of rows per call):
-// 5.7 TB/s read+write at d = 8192 and 4.8 TB/s at d = 4096, where the per-row block
-// reduction (three barriers and one thread's square root and division per 8 KB) weighs more.
+// 5.7 TB/s read+write at d = 8192 and 5.1 TB/s at d = 4096, where the per-row block
+// reduction (three barriers and one thread's square root and division per 8 KB) weighs more
+// and a block therefore takes two rows at a time.
 // Before the conversion-free fast path of normalize.cuh the kernel sat at 4.4 TB/s with the
 // conversion unit as its busiest pipe.
 #include "common.cuh"
@@ -76,6 +77,53 @@ append_bulk_kernel(const uint16_t* __restrict__ states, const int32_t* __restric
   }
 }
 
+// Bulk append of rows that fit two chunks per thread (d <= 4096): a block takes two rows at
+// a time (normalize_two_rows_fast), which halves the barriers and the one-thread arithmetic
+// per row, and loads the next pair while it works on this one.
+__global__ void __launch_bounds__(kNormThreads, 4)
+append_bulk2_kernel(const uint16_t* __restrict__ states, const int32_t* __restrict__ tokens,
+                    int64_t n, int d, uint16_t* __restrict__ keys, int32_t* __restrict__ tok,
+                    int32_t* __restrict__ trace_id, int64_t row0, int32_t trace,
+                    int32_t* __restrict__ trace_end, uint64_t* __restrict__ trace_tag, uint64_t tag,
+                    int64_t* __restrict__ trace_gbase, int64_t gbase, int set_tag,
+                    DeviceStats* stats) {
+  constexpr int kHeld = 2;
+  pdl_launch_dependents();
+  pdl_wait();
+  if (blockIdx.x == 0 && threadIdx.x == 0) {
+    trace_end[trace] = (int32_t)(row0 + n);
+    if (set_tag) { trace_tag[trace] = tag; trace_gbase[trace] = gbase; }
+  }
+  uint4 ca[kHeld], cb[kHeld], na[kHeld], nb[kHeld];
+  const int64_t stride = 2ll * gridDim.x;
+  int64_t r = 2ll * blockIdx.x;
+  if (r < n) load_row_chunks<kHeld>(states + r * d, d, ca);
+  if (r + 1 < n) load_row_chunks<kHeld>(states + (r + 1) * d, d, cb);
+  for (; r < n; r += stride) {
+    const int64_t rn = r + stride;
+    if (rn < n) load_row_chunks<kHeld>(states + rn * d, d, na);
+    if (rn + 1 < n) load_row_chunks<kHeld>(states + (rn + 1) * d, d, nb);
+    const int64_t row = row0 + r;
+    int code_a, code_b = kRowOk;
+    if (r + 1 < n) {
+      normalize_two_rows_fast<kHeld>(ca, cb, keys + row * d, keys + (row + 1) * d, d, code_a, code_b);
+      if (code_a < 0)
+        code_a = normalize_row_regs<true, kHeld, false>(ca, states + r * d, keys + row * d, d);
+      if (code_b < 0)
+        code_b = normalize_row_regs<true, kHeld, false>(cb, states + (r + 1) * d, keys + (row + 1) * d, d);
+    } else {
+      code_a = normalize_row_regs<true, kHeld, true>(ca, states + r * d, keys + row * d, d);
+    }
+    if (threadIdx.x < 2 && r + threadIdx.x < n) {
+      tok[row + threadIdx.x] = tokens[r + threadIdx.x];
+      trace_id[row + threadIdx.x] = trace;
+      if ((threadIdx.x ? code_b : code_a) != kRowOk) atomicAdd(&stats->degenerate_rows, 1ull);
+    }
+#pragma unroll
+    for (int i = 0; i < kHeld; ++i) { ca[i] = na[i]; cb[i] = nb[i]; }
+  }
+}
+
 __global__ void __launch_bounds__(kNormThreads)
 qnorm_kernel(const uint16_t* __restrict__ q, int nq, int d, uint16_t* __restrict__ qn,
              int32_t* __restrict__ q_valid, DeviceStats* stats, float* __restrict__ xchg,
@@ -115,7 +163,7 @@ cudaError_t launch_append(const uint16_t* states, const int32_t* tokens, int64_t
   const int64_t bulk_grid = (int64_t)sms * 4;
   if (n >= bulk_grid * 4) {
     if (d <= 4096)
-      return launch_pdl(append_bulk_kernel<2>, dim3((unsigned)bulk_grid), dim3(kNormThreads), 0, st,
+      return launch_pdl(append_bulk2_kernel, dim3((unsigned)bulk_grid), dim3(kNormThreads), 0, st,
                         states, tokens, n, d, keys, tok, trace_id, row0, trace, trace_end,
                         trace_tag, tag, trace_gbase, gbase, set_tag, stats);
     return launch_pdl(append_bulk_kernel<4>, dim3((unsigned)bulk_grid), dim3(kNormThreads), 0, st,

@@ -171,6 +171,96 @@ __device__ __forceinline__ int normalize_row_regs(const uint4 (&held)[kHeld],
   return code;
 }
 
+// Two rows at once, fast path only (see normalize_row_regs): every chunk of both rows is in
+// registers (d <= kHeld * 2048).  The per-row block reduction, its barriers and the square
+// root and division that one thread does per row are the fixed cost of a row; two rows share
+// the barriers, and threads 0 and 32 take one row's scale each.  Each row's numbers are
+// accumulated in the order of the single-row routine, so the results are the same.  code_a /
+// code_b come back as kRowOk, or -1 for a row that must be redone on the exact path (nothing
+// has been written for it).
+template <int kHeld>
+__device__ __forceinline__ void normalize_two_rows_fast(const uint4 (&ha)[kHeld],
+                                                        const uint4 (&hb)[kHeld],
+                                                        uint16_t* __restrict__ dst_a,
+                                                        uint16_t* __restrict__ dst_b, int d,
+                                                        int& code_a, int& code_b) {
+  __shared__ double s_part2[2][kNormThreads / 32];
+  __shared__ int s_bad2[2][kNormThreads / 32];
+  __shared__ double s_inv2[2];
+  __shared__ int s_code2[2];
+  const int n_chunks = d >> 3;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  double fs[2] = {0.0, 0.0};
+  uint32_t umin[2] = {0xffffffffu, 0xffffffffu};
+#pragma unroll
+  for (int r = 0; r < 2; ++r) {
+#pragma unroll
+    for (int i = 0; i < kHeld; ++i) {
+      if (threadIdx.x + i * kNormThreads >= n_chunks) break;
+      const uint4 hv = r ? hb[i] : ha[i];
+      const uint32_t w[4] = {hv.x, hv.y, hv.z, hv.w};
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const uint32_t ul = (w[j] & 0x7fffu) << 13, uh = (w[j] & 0x7fff0000u) >> 3;
+        umin[r] = min(umin[r], min(ul, uh));
+        const double lo = __hiloint2double((int)(ul + 0x38000000u), 0);
+        const double hi = __hiloint2double((int)(uh + 0x38000000u), 0);
+        fs[r] += lo * lo;
+        fs[r] += hi * hi;
+      }
+    }
+  }
+  int redo[2] = {umin[0] < 0x00100000u, umin[1] < 0x00100000u};
+#pragma unroll
+  for (int m = 16; m; m >>= 1) {
+#pragma unroll
+    for (int r = 0; r < 2; ++r) {
+      fs[r] += __shfl_xor_sync(0xffffffffu, fs[r], m);
+      redo[r] |= __shfl_xor_sync(0xffffffffu, redo[r], m);
+    }
+  }
+  if (lane == 0) {
+    s_part2[0][warp] = fs[0]; s_bad2[0][warp] = redo[0];
+    s_part2[1][warp] = fs[1]; s_bad2[1][warp] = redo[1];
+  }
+  __syncthreads();
+  if (lane == 0 && warp < 2) {
+    double tot = 0.0;
+    int b = 0;
+    for (int w = 0; w < kNormThreads / 32; ++w) { tot += s_part2[warp][w]; b |= s_bad2[warp][w]; }
+    b |= !(tot < 0x1p256);
+    s_inv2[warp] = b ? 0.0 : 1.0 / sqrt(tot);
+    s_code2[warp] = b ? -1 : kRowOk;
+  }
+  __syncthreads();
+#pragma unroll
+  for (int r = 0; r < 2; ++r) {
+    if (s_code2[r] != kRowOk) continue;
+    const double inv = s_inv2[r];
+    uint4* dst4 = reinterpret_cast<uint4*>(r ? dst_b : dst_a);
+#pragma unroll
+    for (int i = 0; i < kHeld; ++i) {
+      const int c = threadIdx.x + i * kNormThreads;
+      if (c >= n_chunks) break;
+      const uint4 hv = r ? hb[i] : ha[i];
+      const uint32_t w[4] = {hv.x, hv.y, hv.z, hv.w};
+      uint32_t o[4];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const uint32_t hl = ((w[j] & 0x8000u) << 16) | (((w[j] & 0x7fffu) << 13) + 0x38000000u);
+        const uint32_t hh = (w[j] & 0x80000000u) | (((w[j] & 0x7fff0000u) >> 3) + 0x38000000u);
+        const float lo = __double2float_rn(__hiloint2double((int)hl, 0) * inv);
+        const float hi = __double2float_rn(__hiloint2double((int)hh, 0) * inv);
+        asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(o[j]) : "f"(hi), "f"(lo));
+      }
+      dst4[c] = make_uint4(o[0], o[1], o[2], o[3]);
+    }
+  }
+  code_a = s_code2[0];
+  code_b = s_code2[1];
+  __syncthreads();   // the shared scratch is reused by the next pair
+}
+
 // Normalise one row of d bf16 values (d % 8 == 0) from src to dst (global or shared).
 // All kNormThreads threads of the block take part.  The squared norm is accumulated in
 // double precision (products of bf16 values are exact there), the scale 1/sqrt is IEEE

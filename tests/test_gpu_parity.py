@@ -72,6 +72,10 @@ def test_bulk_append_matches_oracle_bit_for_bit(d):
     st[5] = 0
     st[n - 1, d - 1] = float("inf")
     st[1500, 3] = float("nan")
+    st[201] = 0                                  # one row of a pair of rows leaves the fast path
+    st[300] = 0                                  # both rows of a pair do
+    st[301] = 0
+    st[400, 7] = 0                               # a single zero element
     tk = torch.randint(0, 50000, (n,), generator=g, device="cuda", dtype=torch.int32)
     pool, ora = B.Pool(d, n + 200), OraclePool(d)
     for lo, hi, tag in ((0, 100, 3), (100, n, 4)):          # a small call, then a bulk one
@@ -82,7 +86,7 @@ def test_bulk_append_matches_oracle_bit_for_bit(d):
     assert np.array_equal(tok, ora.tokens) and np.array_equal(tid, ora.trace_ids)
     s, e, t = pool.traces()
     assert e.tolist() == ora.trace_ends.tolist() and t.tolist() == ora.trace_tags.tolist()
-    assert pool.stats()["degenerate_rows"] == ora.degenerate_rows == 3
+    assert pool.stats()["degenerate_rows"] == ora.degenerate_rows == 6
 
 
 def test_append_capacity_and_argument_errors():

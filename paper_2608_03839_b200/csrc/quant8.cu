@@ -334,7 +334,7 @@ scan_gemv_e4m3_kernel(const uint8_t* __restrict__ codes, const float* __restrict
   if ((int)blockIdx.x < fa.n) {
     const int r = blockIdx.x;
     const int64_t row = (int64_t)fa.row0 + r;
-    const bool ok = quantize_row_e4m3(fa.states + (size_t)r * d, d,
+    const bool ok = quantize_row_e4m3<true>(fa.states + (size_t)r * d, d,
                                       const_cast<uint8_t*>(codes) + row * d,
                                       const_cast<float*>(scales) + row);
     if (threadIdx.x == 0) {

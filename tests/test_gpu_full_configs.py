@@ -23,6 +23,45 @@ def fixed(k, L, theta=0.8, **kw):
     return B.QueryParams(k=k, theta=theta, depth_mode=B.DEPTH_FIXED, cont_len=L, **kw)
 
 
+@pytest.mark.parametrize("key_format", ["bf16", "e4m3"])
+def test_c2_full_size_in_the_launch_configuration_the_bench_times(key_format):
+    # bench.py's step on its default workload: oilbird_pool_step on the full C2 pool, the
+    # 8 rows committed since the last step appended inside the scan kernel, one query, path
+    # chosen by the library.  Every step's output is checked against the oracle, and the
+    # stored rows at the end.
+    w = W.C2
+    pool, ora = fill_both(w, spare_rows=256, max_nq=w.nq, max_k=w.k, max_append=8,
+                          key_format=key_format)
+    q, meta = w.queries("cuda")
+    g = torch.Generator(device="cuda").manual_seed(2)
+    launches0 = pool.launch_count
+    for step in range(6):
+        st = torch.randn(8, w.d, generator=g, device="cuda").to(torch.bfloat16)
+        tk = torch.randint(0, w.vocab, (8,), generator=g, device="cuda", dtype=torch.int32)
+        qs = q.clone()
+        if step % 2:
+            qs[0] = st[5]                       # every other step asks for a row of this step
+        pr = fixed(w.k, w.cont_len, theta=(0.8 if step < 3 else -2.0))
+        out = pool.step(st, tk, qs, pr, tag=1_000_000 + step)
+        ora.append(W.to_bits(st), tk.cpu().numpy(), tag=1_000_000 + step)
+        check_query(out, ora, W.to_bits(qs), pr)
+        if step % 2:
+            assert int(out.idx[0, 0]) == len(pool) - 3
+        elif "planted_row" in meta:
+            assert int(out.idx[0, 0]) == meta["planted_row"]
+    assert len(pool) == w.n_rows + 48 and pool.stats()["stalled"] == 0
+    assert pool.launch_count - launches0 == 12      # two kernels per step: scan, merge + gather
+    _, tok, tid = pool.read_rows(w.n_rows, 48)
+    assert np.array_equal(tok, ora.tokens[w.n_rows:]) and np.array_equal(tid, ora.trace_ids[w.n_rows:])
+    if key_format == "bf16":
+        keys, _, _ = pool.read_rows(w.n_rows, 48)
+        assert np.array_equal(keys, ora.keys[w.n_rows:])
+    else:
+        codes, scales = pool.read_codes(w.n_rows, 48)
+        assert np.array_equal(codes, ora.codes[w.n_rows:])
+        assert np.array_equal(scales.view(np.uint32), ora.scales[w.n_rows:].view(np.uint32))
+
+
 def test_c3_tool_calling_shape_full_size():
     w = W.C3
     pool, ora = fill_both(w)

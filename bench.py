@@ -844,7 +844,7 @@ def main():
     ap.add_argument("--nq", type=int, default=0, help="override the configuration's nq")
     ap.add_argument("--rows", type=int, default=0,
                     help="override the pool size (profiling a smaller case of the same recipe)")
-    ap.add_argument("--path", type=int, default=0, help="0 auto, 1 CUDA-core scan, 2 tensor scan")
+    ap.add_argument("--path", type=int, default=0, help="0 auto, 1 CUDA-core scan, 2 tcgen05 scan, 3 warp-level tensor scan")
     ap.add_argument("--keys", default="bf16", choices=["bf16", "e4m3"],
                     help="stored key format: the paper's 16-bit keys, or the bounded-store "
                          "variant with 8-bit keys (FP8 E4M3 + one scale per row)")

@@ -21,7 +21,7 @@ OK, EINVAL, ECAPACITY, ENOMEM, ECUDA, ESTALL = 0, -1, -2, -3, -4, -5
 NEW_TRACE = 1
 KEYS_E4M3 = 1          # pool flag: 8-bit keys
 DEPTH_FIXED, DEPTH_TIERED = 0, 1
-PATH_AUTO, PATH_GEMV, PATH_TENSOR = 0, 1, 2
+PATH_AUTO, PATH_GEMV, PATH_TENSOR, PATH_MMA = 0, 1, 2, 3
 MAX_NQ, MAX_K, MAX_CONT_LEN, MAX_TIERS = 256, 128, 128, 4
 
 

@@ -401,7 +401,7 @@ static int check_params(const oilbird_pool* p, int32_t nq, const oilbird_query_p
   if (pr->depth_mode != OILBIRD_DEPTH_FIXED && pr->depth_mode != OILBIRD_DEPTH_TIERED)
     return OILBIRD_EINVAL;
   if (pr->n_tiers < 0 || pr->n_tiers > OILBIRD_MAX_TIERS) return OILBIRD_EINVAL;
-  if (pr->path < OILBIRD_PATH_AUTO || pr->path > OILBIRD_PATH_TENSOR) return OILBIRD_EINVAL;
+  if (pr->path < OILBIRD_PATH_AUTO || pr->path > OILBIRD_PATH_MMA) return OILBIRD_EINVAL;
   if (isnan(pr->theta)) return OILBIRD_EINVAL;
   gp->k = pr->k; gp->offset = pr->offset; gp->depth_mode = pr->depth_mode;
   gp->cont_len = pr->cont_len; gp->n_tiers = pr->n_tiers; gp->theta = pr->theta;
@@ -425,10 +425,20 @@ static bool out_ok(const oilbird_query_out* o, bool need_idx) {
   return !need_idx || (o->idx && o->score);
 }
 
-static int resolve_path(const oilbird_query_params* pr, int32_t nq) {
-  // single-request decode streams keys through the CUDA cores; batches go to tcgen05
+// Key bytes up to which a batch of 3 to 8 queries goes to the warp-level tensor scan: it
+// streams keys like the CUDA-core scan and starts within a few microseconds; above, the
+// tcgen05 scan's higher streaming rate has made up for its ~40 us of start-up.
+constexpr int64_t kMmaMaxKeyBytes = 2ll << 30;
+
+static int resolve_path(const oilbird_pool* p, const oilbird_query_params* pr, int32_t nq) {
+  // single-request decode streams keys through the CUDA cores; batches go to tcgen05,
+  // small batches on pools of the paper's size to mma.sync
   if (pr->path != OILBIRD_PATH_AUTO) return pr->path;
-  return nq <= 2 ? OILBIRD_PATH_GEMV : OILBIRD_PATH_TENSOR;
+  if (nq <= 2) return OILBIRD_PATH_GEMV;
+  if (nq <= 8 && !p->r.e4m3 && p->n_rows * (int64_t)p->r.d * 2 <= kMmaMaxKeyBytes &&
+      scan_mma_supports(p->r.d, list_len(pr->k), p->smem_limit))
+    return OILBIRD_PATH_MMA;
+  return OILBIRD_PATH_TENSOR;
 }
 
 // fused: the step's append, to be done by the CUDA-core scan itself (the rows are already
@@ -447,8 +457,11 @@ static int query_impl(oilbird_pool_t* p, const void* q, int32_t nq, const oilbir
   cudaError_t e;
 
   const int path = p->r.e4m3 && pr->path == OILBIRD_PATH_AUTO ? OILBIRD_PATH_GEMV
-                                                              : resolve_path(pr, nq);
-  if (path == OILBIRD_PATH_TENSOR && p->r.e4m3) return OILBIRD_EINVAL;   // 16-bit pools only
+                                                              : resolve_path(p, pr, nq);
+  if ((path == OILBIRD_PATH_TENSOR || path == OILBIRD_PATH_MMA) && p->r.e4m3)
+    return OILBIRD_EINVAL;                                               // 16-bit pools only
+  if (path == OILBIRD_PATH_MMA && !scan_mma_supports(p->r.d, kk, p->smem_limit))
+    return OILBIRD_EINVAL;
   if (path == OILBIRD_PATH_TENSOR && !p->tc) {
     snprintf(g_cuda_err, sizeof g_cuda_err, "tensor-core scan unavailable on this device");
     return OILBIRD_ECUDA;
@@ -482,6 +495,11 @@ static int query_impl(oilbird_pool_t* p, const void* q, int32_t nq, const oilbir
       e = launch_scan_gemv(pv, (const uint16_t*)q, nq, pr->k, kk, pr->exclude_tag, p->partial,
                            p->q_valid, p->stats, p->r.max_lists, p->num_sms, &n_lists, fused, st);
       if (e != cudaSuccess) return cuda_fail(e, "scan kernel launch");
+      p->launches += 1;
+    } else if (path == OILBIRD_PATH_MMA) {
+      e = launch_scan_mma(pv, (const uint16_t*)q, nq, pr->k, kk, pr->exclude_tag, p->partial,
+                          p->q_valid, p->stats, p->r.max_lists, p->num_sms, &n_lists, st);
+      if (e != cudaSuccess) return cuda_fail(e, "warp-level tensor scan kernel launch");
       p->launches += 1;
     } else {
       e = launch_qnorm((const uint16_t*)q, nq, nq_pad, p->r.d, p->qn, p->q_valid, p->stats,
@@ -528,7 +546,7 @@ static int step_impl(oilbird_pool_t* p, const void* states, const int32_t* token
   // (8-bit pools always use the CUDA-core scan; its passes beyond the first two queries
   // would find the rows in place, but keep to the single-request case there too)
   const bool gemv = p->r.e4m3 ? (nq <= 2 && pr->path != OILBIRD_PATH_TENSOR)
-                              : resolve_path(pr, nq) == OILBIRD_PATH_GEMV;
+                              : resolve_path(p, pr, nq) == OILBIRD_PATH_GEMV;
   const bool fuse = n >= 1 && n <= kFuseMaxRows && gemv &&
                     scan_gemv_grid(rows_after, p->num_sms, p->r.max_lists) >= n;
   if (!fuse) {

@@ -103,7 +103,7 @@ int oilbird_query_static(const oilbird_static_pool* sp, const void* q_bf16, int3
     snprintf(g_static_err, sizeof g_static_err, "query parameter out of range");
     return OILBIRD_EINVAL;
   }
-  if (pr->exclude_tag || pr->path == OILBIRD_PATH_TENSOR) {
+  if (pr->exclude_tag || pr->path == OILBIRD_PATH_TENSOR || pr->path == OILBIRD_PATH_MMA) {
     snprintf(g_static_err, sizeof g_static_err,
              "the static variant has no exclusion tags and only the CUDA-core scan");
     return OILBIRD_EINVAL;

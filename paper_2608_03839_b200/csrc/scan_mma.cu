@@ -1,0 +1,333 @@
+// K2b: warp-level tensor-core scan for small batches (3 to 8 queries per pass).
+//
+// Scoring line of Algorithm 1 (cosine of each query with every stored state) fused with the
+// per-CTA part of Eq. 2's top-k, for the batch sizes between single-request decode and the
+// large batches of the tcgen05 scan.  The tcgen05 scan needs whole 128-row tiles and a
+// completed K loop before a score exists, which costs about 40 us per query call on pools of
+// the paper's size (a few hundred MB); the CUDA-core scan runs out of issue slots beyond two
+// queries (64 FMAs per 16 key bytes at eight).  Here the key stream is organised exactly as
+// in the CUDA-core scan (2 CTAs x 8 warps per SM, contiguous row split, 16-byte streaming
+// loads straight into registers) and the arithmetic goes to mma.sync.m16n8k16 (bf16 in,
+// fp32 accumulate): 16 rows x 8 queries x 32 elements cost two loads of keys, one shared
+// memory load of queries and two MMAs per lane, so the kernel stays bound by the key stream.
+//
+// The reduction dimension may be walked in any order as long as keys and queries agree, so
+// a lane's 16-byte load (eight consecutive elements of one row) feeds the k slots of two
+// MMAs directly: lane (g, t) = (lane / 4, lane % 4) holds rows g and g + 8 of the group
+// and elements 8 t .. 8 t + 7 of each 32-element block, and reads the same elements of
+// query g from shared memory.  No shuffles, no staging of keys in shared memory.
+//
+// Each warp keeps one descending register list per query (Eq. 2); a group's 128 scores are
+// tested against the lists' k-th entries and the few that pass are inserted one by one.  At
+// the end warp w merges query w's eight lists; what leaves the CTA is one list per query,
+// as in the other scans.
+#include "common.cuh"
+#include "internal.h"
+#include "normalize.cuh"
+
+namespace oilbird {
+
+constexpr int kMmaThreads = 256;
+constexpr int kMmaWarps = kMmaThreads / 32;
+constexpr int kMmaQ = 8;          // queries per pass = the N of the instruction
+constexpr int kMmaRows = 16;      // rows per warp step = the M of the instruction
+constexpr int kMmaDepth = 4;      // 32-element blocks in flight per lane and row
+constexpr int kMmaPadBytes = 64;  // per query row in shared memory: keeps the 16-byte loads of
+                                  // a quarter warp (two queries x four offsets) on distinct banks
+
+__device__ __forceinline__ void mma_bf16(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2,
+                                         uint32_t a3, uint32_t b0, uint32_t b1) {
+  asm(
+      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, "
+      "{%8,%9}, {%0,%1,%2,%3};"
+      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+// barrier among the four warps of a quad (ids 1 and 2; 0 is __syncthreads)
+__device__ __forceinline__ void quad_bar(int id) {
+  asm volatile("bar.sync %0, 128;" ::"r"(id) : "memory");
+}
+
+// normalize_row done by one warp, with the numbers accumulated in the order of the block
+// routine (lane l plays threads l, l + 32, ... l + 224 of a 256-thread block with one
+// accumulator each), so that a query is normalised to the same bf16 vector on every path.
+__device__ __forceinline__ int normalize_row_warp(const uint16_t* __restrict__ src,
+                                                  uint16_t* __restrict__ dst, int d, int lane) {
+  const int n_chunks = d >> 3;
+  const uint4* src4 = reinterpret_cast<const uint4*>(src);
+  double acc[kNormThreads / 32];
+  int bad = 0;
+#pragma unroll
+  for (int v = 0; v < kNormThreads / 32; ++v) acc[v] = 0.0;
+  for (int base = 0; base < n_chunks; base += kNormThreads) {
+#pragma unroll
+    for (int v = 0; v < kNormThreads / 32; ++v) {
+      const int c = base + 32 * v + lane;
+      if (c < n_chunks) {
+        const uint4 hv = __ldg(src4 + c);
+        const uint32_t w[4] = {hv.x, hv.y, hv.z, hv.w};
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          const float lo = bf16_lo(w[j]), hi = bf16_hi(w[j]);
+          bad |= ((w[j] & 0x7f80u) == 0x7f80u) | ((w[j] & 0x7f800000u) == 0x7f800000u);
+          acc[v] += (double)lo * (double)lo;
+          acc[v] += (double)hi * (double)hi;
+        }
+      }
+    }
+  }
+  double tot = 0.0;
+#pragma unroll
+  for (int v = 0; v < kNormThreads / 32; ++v) {
+#pragma unroll
+    for (int m = 16; m; m >>= 1) acc[v] += __shfl_xor_sync(0xffffffffu, acc[v], m);
+    tot += acc[v];
+  }
+#pragma unroll
+  for (int m = 16; m; m >>= 1) bad |= __shfl_xor_sync(0xffffffffu, bad, m);
+  const double nrm = sqrt(tot);
+  const bool ok = !bad && nrm > 0.0 && isfinite(nrm);
+  const double inv = ok ? 1.0 / nrm : 0.0;
+  uint4* dst4 = reinterpret_cast<uint4*>(dst);
+  for (int c = lane; c < n_chunks; c += 32) {
+    const uint4 hv = __ldg(src4 + c);
+    const uint32_t w[4] = {hv.x, hv.y, hv.z, hv.w};
+    uint32_t o[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      if (inv == 0.0) { o[j] = 0; continue; }
+      const float lo = __double2float_rn((double)bf16_lo(w[j]) * inv);
+      const float hi = __double2float_rn((double)bf16_hi(w[j]) * inv);
+      o[j] = f32_to_bf16_bits(lo) | (f32_to_bf16_bits(hi) << 16);
+    }
+    dst4[c] = make_uint4(o[0], o[1], o[2], o[3]);
+  }
+  return ok ? kRowOk : ((bad || !isfinite(nrm)) ? kRowNonFinite : kRowZero);
+}
+
+template <int E>
+__global__ void __launch_bounds__(kMmaThreads, 2)
+scan_mma_kernel(PoolView pv, const uint16_t* __restrict__ q_raw, int nq, int k,
+                const uint64_t* __restrict__ exclude_tag, u64* __restrict__ partial,
+                int32_t* __restrict__ q_valid, DeviceStats* stats) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  constexpr int KK = 32 * E;
+  pdl_launch_dependents();
+  pdl_wait();   // the rows appended before this query, and the query states themselves
+  const int d = pv.d, n_chunks = d >> 3;
+  const int q_stride = n_chunks + kMmaPadBytes / 16;                     // in 16-byte units
+  uint4* qs = reinterpret_cast<uint4*>(smem_raw);                        // [kMmaQ][q_stride]
+  u64* scratch = reinterpret_cast<u64*>(smem_raw + (size_t)kMmaQ * q_stride * 16);  // [2 quads][kMmaQ][KK]
+  __shared__ uint64_t s_ex[kMmaQ];
+  __shared__ float4 s_part[2 * 2 * 4 * 32];  // [buffer][quad][quarter][lane]: partial scores of a group
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int g = lane >> 2, t = lane & 3;
+  const int64_t n = pv.n_rows;
+  const int r_lo = (int)((n * blockIdx.x) / gridDim.x);
+  const int r_hi = (int)((n * (blockIdx.x + 1)) / gridDim.x);
+  const uint4* keys4 = reinterpret_cast<const uint4*>(pv.keys);
+
+  for (int q0 = 0; q0 < nq; q0 += kMmaQ) {
+    __syncthreads();
+    // query preparation, one warp per query: qs[w] = bf16(q / ||q||), exactly as a key is stored
+    {
+      uint16_t* dst = reinterpret_cast<uint16_t*>(qs + (size_t)warp * q_stride);
+      if (q0 + warp < nq) {
+        const int code = normalize_row_warp(q_raw + (size_t)(q0 + warp) * d, dst, d, lane);
+        if (blockIdx.x == 0 && lane == 0) {
+          q_valid[q0 + warp] = code == kRowNonFinite ? 0 : 1;   // NaN/Inf: no neighbours
+          if (code == kRowNonFinite) atomicAdd(&stats->nonfinite_queries, 1ull);
+        }
+      } else {
+        for (int c = lane; c < n_chunks; c += 32) qs[(size_t)warp * q_stride + c] = make_uint4(0, 0, 0, 0);
+      }
+      if (lane == 0)
+        s_ex[warp] = (exclude_tag && q0 + warp < nq) ? exclude_tag[q0 + warp] : 0;
+    }
+    __syncthreads();
+
+    // Four warps (a quad) share a group of 16 rows, every fourth 32-element block of the row
+    // width each (so that the quad reads a row in contiguous kilobytes); the four partial
+    // sums meet in shared memory and every warp adds them up.  A warp alone on a
+    // group would leave a CTA's 200-odd rows of a paper-size pool as 14 units for 8 warps
+    // (two rounds, the second three-quarters empty); as 7 units per quad the rounds are full.
+    // The lists are shared out as well: warp kq of a quad keeps those of queries 2 kq and
+    // 2 kq + 1 (the scores its lanes with t == kq hold), over all rows of the quad, so a
+    // list sees four times the rows a per-warp list would and far fewer rows pass.
+    const int quad = warp >> 2, kq = warp & 3;
+    const int cq = n_chunks >> 2;                                   // 16-byte units per quarter
+    const uint4* qrow = qs + (size_t)g * q_stride + kq * 4 + t;
+    float4* part = s_part + quad * 4 * 32;                          // [quarter][lane]
+    // descending lists of this warp's two queries; kth = the k-th entry (0 while not full)
+    u64 top[2][E];
+    u64 kth[2] = {0, 0};
+#pragma unroll
+    for (int qq = 0; qq < 2; ++qq)
+#pragma unroll
+      for (int r = 0; r < E; ++r) top[qq][r] = 0;
+    const bool own = t == kq;                                       // this lane's scores are this warp's
+    const bool live_a = own && q0 + 2 * kq < nq, live_b = own && q0 + 2 * kq + 1 < nq;
+    const uint64_t ex_a = s_ex[2 * kq], ex_b = s_ex[2 * kq + 1];
+    int buf = 0;
+
+    // key pointers of this lane's two rows of the group starting at row rbx
+    auto row_ptr = [&](int rbx, int second) {
+      const int row = rbx + g + 8 * second;
+      return keys4 + (size_t)(row < r_hi ? row : r_hi - 1) * n_chunks + kq * 4 + t;
+    };
+    // The key stream of a warp is one sequence of steps of kMmaDepth blocks of 32 elements
+    // over all its groups: the loads of the next step (the first of the next group, at a
+    // group's end) are issued before this step's MMAs, so that the loads in flight never
+    // drain, neither while the tensor pipe works nor across a group's epilogue.
+    int rb = r_lo + quad * kMmaRows;
+    const uint4 *pa = keys4, *pb = keys4;
+    uint4 ka[kMmaDepth], kb[kMmaDepth];
+    if (rb < r_hi) {
+      pa = row_ptr(rb, 0);
+      pb = row_ptr(rb, 1);
+#pragma unroll
+      for (int u = 0; u < kMmaDepth; ++u) {
+        const bool in = 4 * u < cq;
+        ka[u] = in ? ld_stream16(pa + 4 * (4 * u)) : make_uint4(0, 0, 0, 0);
+        kb[u] = in ? ld_stream16(pb + 4 * (4 * u)) : make_uint4(0, 0, 0, 0);
+      }
+    }
+    for (; rb < r_hi; rb += 2 * kMmaRows) {
+      const int row0 = rb + g, row1 = rb + g + 8;
+      const bool has_next = rb + 2 * kMmaRows < r_hi;
+      const uint4* pna = has_next ? row_ptr(rb + 2 * kMmaRows, 0) : pa;
+      const uint4* pnb = has_next ? row_ptr(rb + 2 * kMmaRows, 1) : pb;
+      float c0[4] = {0.f, 0.f, 0.f, 0.f}, c1[4] = {0.f, 0.f, 0.f, 0.f};
+      for (int c = 0; c < cq; c += 4 * kMmaDepth) {
+        uint4 na[kMmaDepth], nb[kMmaDepth];
+        const int cn = c + 4 * kMmaDepth;
+        const bool same = cn < cq;                         // next step: same group or the next one
+        const uint4* sa = same ? pa + 4 * cn : pna;
+        const uint4* sb = same ? pb + 4 * cn : pnb;
+        const int left = same ? cq - cn : (has_next ? cq : 0);
+#pragma unroll
+        for (int u = 0; u < kMmaDepth; ++u) {
+          const bool in = 4 * u < left;
+          na[u] = in ? ld_stream16(sa + 4 * (4 * u)) : make_uint4(0, 0, 0, 0);
+          nb[u] = in ? ld_stream16(sb + 4 * (4 * u)) : make_uint4(0, 0, 0, 0);
+        }
+#pragma unroll
+        for (int u = 0; u < kMmaDepth; ++u) {
+          const uint4 qv = c + 4 * u < cq ? qrow[4 * (c + 4 * u)] : make_uint4(0, 0, 0, 0);
+          mma_bf16(c0, ka[u].x, kb[u].x, ka[u].y, kb[u].y, qv.x, qv.y);
+          mma_bf16(c1, ka[u].z, kb[u].z, ka[u].w, kb[u].w, qv.z, qv.w);
+        }
+#pragma unroll
+        for (int u = 0; u < kMmaDepth; ++u) { ka[u] = na[u]; kb[u] = nb[u]; }
+      }
+      pa = pna;
+      pb = pnb;
+      // partial scores of (row0, 2t), (row0, 2t+1), (row1, 2t), (row1, 2t+1)
+      // two buffers, one barrier per group: a warp reads a group's partials before it starts
+      // the next group, so when it arrives here for group i it is done with group i - 1, and
+      // the barrier of group i - 1 has shown that everyone was done with group i - 2
+      float4* pbuf = part + (buf ? 4 * 32 * 2 : 0);
+      buf ^= 1;
+      pbuf[kq * 32 + lane] = make_float4(c0[0] + c1[0], c0[1] + c1[1], c0[2] + c1[2], c0[3] + c1[3]);
+      quad_bar(1 + quad);                    // this group's partials are in
+      float4 sc;
+      {
+        const float4 p0 = pbuf[lane], p1 = pbuf[32 + lane], p2 = pbuf[64 + lane], p3 = pbuf[96 + lane];
+        sc.x = ((p0.x + p1.x) + p2.x) + p3.x;
+        sc.y = ((p0.y + p1.y) + p2.y) + p3.y;
+        sc.z = ((p0.z + p1.z) + p2.z) + p3.z;
+        sc.w = ((p0.w + p1.w) + p2.w) + p3.w;
+      }
+      uint64_t tag0 = 0, tag1 = 0;
+      if (exclude_tag && own) {
+        if (row0 < r_hi) tag0 = pv.trace_tag[pv.trace_id[row0]];
+        if (row1 < r_hi) tag1 = pv.trace_tag[pv.trace_id[row1]];
+      }
+      u64 key[4];
+      key[0] = (row0 < r_hi && live_a && !(ex_a != 0 && tag0 == ex_a)) ? pack_candidate(sc.x, (uint32_t)row0) : 0;
+      key[1] = (row0 < r_hi && live_b && !(ex_b != 0 && tag0 == ex_b)) ? pack_candidate(sc.y, (uint32_t)row0) : 0;
+      key[2] = (row1 < r_hi && live_a && !(ex_a != 0 && tag1 == ex_a)) ? pack_candidate(sc.z, (uint32_t)row1) : 0;
+      key[3] = (row1 < r_hi && live_b && !(ex_b != 0 && tag1 == ex_b)) ? pack_candidate(sc.w, (uint32_t)row1) : 0;
+      const bool any = (key[0] > kth[0]) | (key[1] > kth[1]) | (key[2] > kth[0]) | (key[3] > kth[1]);
+      if (__any_sync(0xffffffffu, any)) {
+#pragma unroll
+        for (int qq = 0; qq < 2; ++qq) {
+#pragma unroll
+          for (int half = 0; half < 2; ++half) {
+            const u64 mine = key[qq + 2 * half];
+            unsigned b = __ballot_sync(0xffffffffu, mine > kth[qq]);
+            while (b) {
+              const int src = __ffs(b) - 1;
+              b &= b - 1;
+              const uint32_t lo = __shfl_sync(0xffffffffu, (uint32_t)mine, src);
+              const uint32_t hi = __shfl_sync(0xffffffffu, (uint32_t)(mine >> 32), src);
+              const u64 cand = ((u64)hi << 32) | lo;
+              if (cand > kth[qq]) {
+                warp_sorted_insert<E>(top[qq], cand, lane);
+                kth[qq] = warp_list_get<E>(top[qq], k - 1);
+              }
+            }
+          }
+        }
+      }
+    }
+
+    // warp w merges the two quads' lists of query w and publishes the CTA's KK best
+    __syncthreads();
+#pragma unroll
+    for (int qq = 0; qq < 2; ++qq)
+#pragma unroll
+      for (int r = 0; r < E; ++r)
+        scratch[((size_t)quad * kMmaQ + 2 * kq + qq) * KK + r * 32 + lane] = top[qq][r];
+    __syncthreads();
+    if (q0 + warp < nq) {
+      u64 a[E], b[E];
+#pragma unroll
+      for (int r = 0; r < E; ++r) {
+        a[r] = scratch[((size_t)0 * kMmaQ + warp) * KK + r * 32 + lane];
+        b[r] = scratch[((size_t)1 * kMmaQ + warp) * KK + r * 32 + lane];
+      }
+      warp_merge_desc<E>(a, b, lane);
+      u64* dst = partial + ((size_t)blockIdx.x * nq + (q0 + warp)) * KK;
+#pragma unroll
+      for (int r = 0; r < E; ++r) dst[r * 32 + lane] = a[r];
+    }
+  }
+}
+
+size_t scan_mma_smem(int32_t d, int32_t kk) {
+  return (size_t)kMmaQ * ((size_t)d * 2 + kMmaPadBytes) + (size_t)2 * kMmaQ * kk * sizeof(u64);
+}
+
+bool scan_mma_supports(int32_t d, int32_t kk, size_t smem_limit) {
+  return d % 128 == 0 && kk <= 64 && scan_mma_smem(d, kk) <= smem_limit;
+}
+
+template <int E>
+static cudaError_t launch_mma_one(const PoolView& pv, const uint16_t* q_raw, int nq, int k,
+                                  const uint64_t* ex, u64* partial, int32_t* q_valid,
+                                  DeviceStats* stats, int grid, cudaStream_t st) {
+  const size_t smem = scan_mma_smem(pv.d, 32 * E);
+  cudaError_t e = cudaFuncSetAttribute(scan_mma_kernel<E>,
+                                       cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (e != cudaSuccess) return e;
+  return launch_pdl(scan_mma_kernel<E>, dim3(grid), dim3(kMmaThreads), smem, st, pv, q_raw, nq, k,
+                    ex, partial, q_valid, stats);
+}
+
+cudaError_t launch_scan_mma(const PoolView& pv, const uint16_t* q_raw, int32_t nq, int32_t k,
+                            int32_t kk, const uint64_t* exclude_tag, u64* partial,
+                            int32_t* q_valid, DeviceStats* stats, int32_t max_lists,
+                            int32_t num_sms, int32_t* n_lists, cudaStream_t st) {
+  const int grid = scan_gemv_grid(pv.n_rows, num_sms, max_lists);
+  *n_lists = grid;
+  if (kk == 32)
+    return launch_mma_one<1>(pv, q_raw, nq, k, exclude_tag, partial, q_valid, stats, grid, st);
+  if (kk == 64)
+    return launch_mma_one<2>(pv, q_raw, nq, k, exclude_tag, partial, q_valid, stats, grid, st);
+  return cudaErrorInvalidValue;
+}
+
+}  // namespace oilbird

@@ -55,7 +55,7 @@ extern "C" {
 #define OILBIRD_DEPTH_TIERED  1  /* D(s): first tier whose floor the score reaches     */
 
 /* which scoring kernel runs */
-#define OILBIRD_PATH_AUTO    0   /* chosen from nq                                     */
+#define OILBIRD_PATH_AUTO    0   /* chosen from nq, the pool's size and its key format  */
 #define OILBIRD_PATH_GEMV    1   /* CUDA-core scan (single-request decode)             */
 #define OILBIRD_PATH_TENSOR  2   /* tcgen05 tensor-core scan (batched queries)         */
 #define OILBIRD_PATH_MMA     3   /* warp-level tensor-core scan (batches of 3 to 8):

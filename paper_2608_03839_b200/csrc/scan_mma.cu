@@ -56,6 +56,64 @@ __device__ __forceinline__ int normalize_row_warp(const uint16_t* __restrict__ s
                                                   uint16_t* __restrict__ dst, int d, int lane) {
   const int n_chunks = d >> 3;
   const uint4* src4 = reinterpret_cast<const uint4*>(src);
+  uint4* dst4 = reinterpret_cast<uint4*>(dst);
+  // Rows of normal finite numbers first (see normalize_row_regs: doubles built from the bits,
+  // the same numbers as the conversions give): eight queries of three conversions per
+  // element in every CTA would keep the conversion unit busy for microseconds.
+  {
+    double acc[kNormThreads / 32];
+    uint32_t umin = 0xffffffffu;
+#pragma unroll
+    for (int v = 0; v < kNormThreads / 32; ++v) acc[v] = 0.0;
+    for (int base = 0; base < n_chunks; base += kNormThreads) {
+#pragma unroll
+      for (int v = 0; v < kNormThreads / 32; ++v) {
+        const int c = base + 32 * v + lane;
+        if (c < n_chunks) {
+          const uint4 hv = __ldg(src4 + c);
+          const uint32_t w[4] = {hv.x, hv.y, hv.z, hv.w};
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            const uint32_t ul = (w[j] & 0x7fffu) << 13, uh = (w[j] & 0x7fff0000u) >> 3;
+            umin = min(umin, min(ul, uh));
+            const double lo = __hiloint2double((int)(ul + 0x38000000u), 0);
+            const double hi = __hiloint2double((int)(uh + 0x38000000u), 0);
+            acc[v] += lo * lo;
+            acc[v] += hi * hi;
+          }
+        }
+      }
+    }
+    double tot = 0.0;
+#pragma unroll
+    for (int v = 0; v < kNormThreads / 32; ++v) {
+#pragma unroll
+      for (int m = 16; m; m >>= 1) acc[v] += __shfl_xor_sync(0xffffffffu, acc[v], m);
+      tot += acc[v];
+    }
+    int redo = umin < 0x00100000u;                 // an element with exponent field 0
+#pragma unroll
+    for (int m = 16; m; m >>= 1) redo |= __shfl_xor_sync(0xffffffffu, redo, m);
+    if (!redo && tot < 0x1p256) {                  // no Inf/NaN pattern either
+      const double inv = 1.0 / sqrt(tot);
+      for (int c = lane; c < n_chunks; c += 32) {
+        const uint4 hv = __ldg(src4 + c);
+        const uint32_t w[4] = {hv.x, hv.y, hv.z, hv.w};
+        uint32_t o[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          const uint32_t hl = ((w[j] & 0x8000u) << 16) | (((w[j] & 0x7fffu) << 13) + 0x38000000u);
+          const uint32_t hh = (w[j] & 0x80000000u) | (((w[j] & 0x7fff0000u) >> 3) + 0x38000000u);
+          const float lo = __double2float_rn(__hiloint2double((int)hl, 0) * inv);
+          const float hi = __double2float_rn(__hiloint2double((int)hh, 0) * inv);
+          asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(o[j]) : "f"(hi), "f"(lo));
+        }
+        dst4[c] = make_uint4(o[0], o[1], o[2], o[3]);
+      }
+      return kRowOk;
+    }
+  }
+  // every other row: conversions for all elements, Inf/NaN found from the bits
   double acc[kNormThreads / 32];
   int bad = 0;
 #pragma unroll
@@ -89,7 +147,6 @@ __device__ __forceinline__ int normalize_row_warp(const uint16_t* __restrict__ s
   const double nrm = sqrt(tot);
   const bool ok = !bad && nrm > 0.0 && isfinite(nrm);
   const double inv = ok ? 1.0 / nrm : 0.0;
-  uint4* dst4 = reinterpret_cast<uint4*>(dst);
   for (int c = lane; c < n_chunks; c += 32) {
     const uint4 hv = __ldg(src4 + c);
     const uint32_t w[4] = {hv.x, hv.y, hv.z, hv.w};

@@ -32,6 +32,7 @@ constexpr int kMmaWarps = kMmaThreads / 32;
 constexpr int kMmaQ = 8;          // queries per pass = the N of the instruction
 constexpr int kMmaRows = 16;      // rows per warp step = the M of the instruction
 constexpr int kMmaDepth = 4;      // 32-element blocks in flight per lane and row
+constexpr int kMmaBatchInsert = 5; // candidates of a group and query from which they are merged in as a sorted vector
 constexpr int kMmaPadBytes = 64;  // per query row in shared memory: keeps the 16-byte loads of
                                   // a quarter warp (two queries x four offsets) on distinct banks
 
@@ -258,7 +259,10 @@ scan_mma_kernel(PoolView pv, const uint16_t* __restrict__ q_raw, int nq, int k,
       const uint4* pnb = has_next ? row_ptr(rb + 2 * kMmaRows, 1) : pb;
       float c0[4] = {0.f, 0.f, 0.f, 0.f}, c1[4] = {0.f, 0.f, 0.f, 0.f};
       for (int c = 0; c < cq; c += 4 * kMmaDepth) {
-        uint4 na[kMmaDepth], nb[kMmaDepth];
+        uint4 na[kMmaDepth], nb[kMmaDepth], qv[kMmaDepth];
+#pragma unroll
+        for (int u = 0; u < kMmaDepth; ++u)                // query fragments of this step
+          qv[u] = c + 4 * u < cq ? qrow[4 * (c + 4 * u)] : make_uint4(0, 0, 0, 0);
         const int cn = c + 4 * kMmaDepth;
         const bool same = cn < cq;                         // next step: same group or the next one
         const uint4* sa = same ? pa + 4 * cn : pna;
@@ -272,9 +276,8 @@ scan_mma_kernel(PoolView pv, const uint16_t* __restrict__ q_raw, int nq, int k,
         }
 #pragma unroll
         for (int u = 0; u < kMmaDepth; ++u) {
-          const uint4 qv = c + 4 * u < cq ? qrow[4 * (c + 4 * u)] : make_uint4(0, 0, 0, 0);
-          mma_bf16(c0, ka[u].x, kb[u].x, ka[u].y, kb[u].y, qv.x, qv.y);
-          mma_bf16(c1, ka[u].z, kb[u].z, ka[u].w, kb[u].w, qv.z, qv.w);
+          mma_bf16(c0, ka[u].x, kb[u].x, ka[u].y, kb[u].y, qv[u].x, qv[u].y);
+          mma_bf16(c1, ka[u].z, kb[u].z, ka[u].w, kb[u].w, qv[u].z, qv[u].w);
         }
 #pragma unroll
         for (int u = 0; u < kMmaDepth; ++u) { ka[u] = na[u]; kb[u] = nb[u]; }
@@ -311,10 +314,32 @@ scan_mma_kernel(PoolView pv, const uint16_t* __restrict__ q_raw, int nq, int k,
       if (__any_sync(0xffffffffu, any)) {
 #pragma unroll
         for (int qq = 0; qq < 2; ++qq) {
+          const unsigned b0 = __ballot_sync(0xffffffffu, key[qq] > kth[qq]);
+          const unsigned b1 = __ballot_sync(0xffffffffu, key[qq + 2] > kth[qq]);
+          if (__popc(b0) + __popc(b1) >= kMmaBatchInsert) {
+            // many rows pass (a list's first groups): the group's 16 scores of this query
+            // are sorted as one vector and merged in, which costs about four insertions
+            const int src = (lane & 7) * 4 + kq;
+            const uint32_t l0 = __shfl_sync(0xffffffffu, (uint32_t)key[qq], src);
+            const uint32_t h0 = __shfl_sync(0xffffffffu, (uint32_t)(key[qq] >> 32), src);
+            const uint32_t l1 = __shfl_sync(0xffffffffu, (uint32_t)key[qq + 2], src);
+            const uint32_t h1 = __shfl_sync(0xffffffffu, (uint32_t)(key[qq + 2] >> 32), src);
+            u64 v[1];
+            v[0] = lane < 8 ? (((u64)h0 << 32) | l0) : lane < 16 ? (((u64)h1 << 32) | l1) : 0;
+            v[0] = v[0] > kth[qq] ? v[0] : 0;
+            warp_sort_desc<1>(v, lane);
+            u64 add[E];
+            add[0] = v[0];
+#pragma unroll
+            for (int r = 1; r < E; ++r) add[r] = 0;
+            warp_merge_desc<E>(top[qq], add, lane);
+            kth[qq] = warp_list_get<E>(top[qq], k - 1);
+            continue;
+          }
 #pragma unroll
           for (int half = 0; half < 2; ++half) {
             const u64 mine = key[qq + 2 * half];
-            unsigned b = __ballot_sync(0xffffffffu, mine > kth[qq]);
+            unsigned b = half ? b1 : b0;
             while (b) {
               const int src = __ffs(b) - 1;
               b &= b - 1;

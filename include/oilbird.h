@@ -58,7 +58,7 @@ extern "C" {
 #define OILBIRD_PATH_AUTO    0   /* chosen from nq, the pool's size and its key format  */
 #define OILBIRD_PATH_GEMV    1   /* CUDA-core scan (single-request decode)             */
 #define OILBIRD_PATH_TENSOR  2   /* tcgen05 tensor-core scan (batched queries)         */
-#define OILBIRD_PATH_MMA     3   /* warp-level tensor-core scan (batches of 3 to 8):
+#define OILBIRD_PATH_MMA     3   /* warp-level tensor-core scan (small batches):
                                     16-bit keys, d a multiple of 128, k <= 64           */
 
 typedef struct oilbird_pool oilbird_pool_t;   /* opaque */

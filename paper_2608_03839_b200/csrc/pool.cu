@@ -425,19 +425,25 @@ static bool out_ok(const oilbird_query_out* o, bool need_idx) {
   return !need_idx || (o->idx && o->score);
 }
 
-// Key bytes up to which a batch of 3 to 8 queries goes to the warp-level tensor scan: it
+// Key bytes up to which a batch of 3 to 16 queries goes to the warp-level tensor scan: it
 // streams keys like the CUDA-core scan and starts within a few microseconds; above, the
 // tcgen05 scan's higher streaming rate has made up for its ~40 us of start-up.
 constexpr int64_t kMmaMaxKeyBytes = 2ll << 30;
+// 9 to 16 queries (two 8-query tiles per pass, one CTA per SM) stream at two thirds of that
+// rate: only pools that the start-up dominates (8,192 rows x 4096: 41 us against 53)
+constexpr int64_t kMma16MaxKeyBytes = 128ll << 20;
 
 static int resolve_path(const oilbird_pool* p, const oilbird_query_params* pr, int32_t nq) {
   // single-request decode streams keys through the CUDA cores; batches go to tcgen05,
   // small batches on pools of the paper's size to mma.sync
   if (pr->path != OILBIRD_PATH_AUTO) return pr->path;
   if (nq <= 2) return OILBIRD_PATH_GEMV;
-  if (nq <= 8 && !p->r.e4m3 && p->n_rows * (int64_t)p->r.d * 2 <= kMmaMaxKeyBytes &&
-      scan_mma_supports(p->r.d, list_len(pr->k), p->smem_limit))
-    return OILBIRD_PATH_MMA;
+  const int64_t key_bytes = p->n_rows * (int64_t)p->r.d * 2;
+  if (nq <= 16 && !p->r.e4m3 && key_bytes <= (nq <= 8 ? kMmaMaxKeyBytes : kMma16MaxKeyBytes)) {
+    // up to 8 queries in one pass of 8; 9 to 16 only where 16 fit in one pass
+    const int nt = scan_mma_tiles(p->r.d, list_len(pr->k), nq, p->smem_limit);
+    if (nt == 2 || (nt == 1 && nq <= 8)) return OILBIRD_PATH_MMA;
+  }
   return OILBIRD_PATH_TENSOR;
 }
 
@@ -498,7 +504,8 @@ static int query_impl(oilbird_pool_t* p, const void* q, int32_t nq, const oilbir
       p->launches += 1;
     } else if (path == OILBIRD_PATH_MMA) {
       e = launch_scan_mma(pv, (const uint16_t*)q, nq, pr->k, kk, pr->exclude_tag, p->partial,
-                          p->q_valid, p->stats, p->r.max_lists, p->num_sms, &n_lists, st);
+                          p->q_valid, p->stats, p->r.max_lists, p->num_sms, p->smem_limit,
+                          &n_lists, st);
       if (e != cudaSuccess) return cuda_fail(e, "warp-level tensor scan kernel launch");
       p->launches += 1;
     } else {

@@ -1,4 +1,4 @@
-// K2b: warp-level tensor-core scan for small batches (3 to 8 queries per pass).
+// K2b: warp-level tensor-core scan for small batches (8 or 16 queries per pass).
 //
 // Scoring line of Algorithm 1 (cosine of each query with every stored state) fused with the
 // per-CTA part of Eq. 2's top-k, for the batch sizes between single-request decode and the
@@ -164,21 +164,28 @@ __device__ __forceinline__ int normalize_row_warp(const uint16_t* __restrict__ s
   return ok ? kRowOk : ((bad || !isfinite(nrm)) ? kRowNonFinite : kRowZero);
 }
 
-template <int E>
-__global__ void __launch_bounds__(kMmaThreads, 2)
+// NT = number of 8-query tiles a pass scores (1: up to 8 queries, 2 CTAs of 8 warps per SM;
+// 2: up to 16 queries, one CTA of 16 warps per SM, since sixteen normalised queries take the
+// shared memory of both).
+template <int E, int NT>
+__global__ void __launch_bounds__(kMmaThreads * NT, 2 / NT)
 scan_mma_kernel(PoolView pv, const uint16_t* __restrict__ q_raw, int nq, int k,
                 const uint64_t* __restrict__ exclude_tag, u64* __restrict__ partial,
                 int32_t* __restrict__ q_valid, DeviceStats* stats) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   constexpr int KK = 32 * E;
+  constexpr int QP = kMmaQ * NT;             // queries per pass
+  constexpr int kQuads = 2 * NT;             // quads of four warps per CTA
   pdl_launch_dependents();
   pdl_wait();   // the rows appended before this query, and the query states themselves
   const int d = pv.d, n_chunks = d >> 3;
   const int q_stride = n_chunks + kMmaPadBytes / 16;                     // in 16-byte units
-  uint4* qs = reinterpret_cast<uint4*>(smem_raw);                        // [kMmaQ][q_stride]
-  u64* scratch = reinterpret_cast<u64*>(smem_raw + (size_t)kMmaQ * q_stride * 16);  // [2 quads][kMmaQ][KK]
-  __shared__ uint64_t s_ex[kMmaQ];
-  __shared__ float4 s_part[2 * 2 * 4 * 32];  // [buffer][quad][quarter][lane]: partial scores of a group
+  uint4* qs = reinterpret_cast<uint4*>(smem_raw);                        // [QP][q_stride]
+  u64* scratch = reinterpret_cast<u64*>(smem_raw + (size_t)QP * q_stride * 16);   // [quads][QP][KK]
+  // partial scores of a group: [buffer][quad][quarter][tile][lane]
+  float4* s_part = reinterpret_cast<float4*>(smem_raw + (size_t)QP * q_stride * 16 +
+                                             (size_t)kQuads * QP * KK * sizeof(u64));
+  __shared__ uint64_t s_ex[QP];
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int g = lane >> 2, t = lane & 3;
@@ -187,7 +194,7 @@ scan_mma_kernel(PoolView pv, const uint16_t* __restrict__ q_raw, int nq, int k,
   const int r_hi = (int)((n * (blockIdx.x + 1)) / gridDim.x);
   const uint4* keys4 = reinterpret_cast<const uint4*>(pv.keys);
 
-  for (int q0 = 0; q0 < nq; q0 += kMmaQ) {
+  for (int q0 = 0; q0 < nq; q0 += QP) {
     __syncthreads();
     // query preparation, one warp per query: qs[w] = bf16(q / ||q||), exactly as a key is stored
     {
@@ -212,22 +219,27 @@ scan_mma_kernel(PoolView pv, const uint16_t* __restrict__ q_raw, int nq, int k,
     // group would leave a CTA's 200-odd rows of a paper-size pool as 14 units for 8 warps
     // (two rounds, the second three-quarters empty); as 7 units per quad the rounds are full.
     // The lists are shared out as well: warp kq of a quad keeps those of queries 2 kq and
-    // 2 kq + 1 (the scores its lanes with t == kq hold), over all rows of the quad, so a
-    // list sees four times the rows a per-warp list would and far fewer rows pass.
+    // 2 kq + 1 of every tile (the scores its lanes with t == kq hold), over all rows of the
+    // quad, so a list sees four times the rows a per-warp list would and far fewer rows pass.
     const int quad = warp >> 2, kq = warp & 3;
     const int cq = n_chunks >> 2;                                   // 16-byte units per quarter
-    const uint4* qrow = qs + (size_t)g * q_stride + kq * 4 + t;
-    float4* part = s_part + quad * 4 * 32;                          // [quarter][lane]
-    // descending lists of this warp's two queries; kth = the k-th entry (0 while not full)
-    u64 top[2][E];
-    u64 kth[2] = {0, 0};
-#pragma unroll
-    for (int qq = 0; qq < 2; ++qq)
-#pragma unroll
-      for (int r = 0; r < E; ++r) top[qq][r] = 0;
+    const uint4* qrow = qs + (size_t)g * q_stride + kq * 4 + t;     // tile i: + 8 i rows
+    float4* part = s_part + quad * 4 * NT * 32;                     // [quarter][tile][lane]
+    // descending lists of this warp's 2 NT queries; kth = the k-th entry (0 while not full)
+    u64 top[2 * NT][E];
+    u64 kth[2 * NT];
+    bool live[2 * NT];
+    uint64_t ex[2 * NT];
     const bool own = t == kq;                                       // this lane's scores are this warp's
-    const bool live_a = own && q0 + 2 * kq < nq, live_b = own && q0 + 2 * kq + 1 < nq;
-    const uint64_t ex_a = s_ex[2 * kq], ex_b = s_ex[2 * kq + 1];
+#pragma unroll
+    for (int l = 0; l < 2 * NT; ++l) {
+      kth[l] = 0;
+#pragma unroll
+      for (int r = 0; r < E; ++r) top[l][r] = 0;
+      const int qi = 8 * (l >> 1) + 2 * kq + (l & 1);               // query of list l within the pass
+      live[l] = own && q0 + qi < nq;
+      ex[l] = s_ex[qi];
+    }
     int buf = 0;
 
     // key pointers of this lane's two rows of the group starting at row rbx
@@ -252,17 +264,18 @@ scan_mma_kernel(PoolView pv, const uint16_t* __restrict__ q_raw, int nq, int k,
         kb[u] = in ? ld_stream16(pb + 4 * (4 * u)) : make_uint4(0, 0, 0, 0);
       }
     }
-    for (; rb < r_hi; rb += 2 * kMmaRows) {
+    for (; rb < r_hi; rb += kQuads * kMmaRows) {
       const int row0 = rb + g, row1 = rb + g + 8;
-      const bool has_next = rb + 2 * kMmaRows < r_hi;
-      const uint4* pna = has_next ? row_ptr(rb + 2 * kMmaRows, 0) : pa;
-      const uint4* pnb = has_next ? row_ptr(rb + 2 * kMmaRows, 1) : pb;
-      float c0[4] = {0.f, 0.f, 0.f, 0.f}, c1[4] = {0.f, 0.f, 0.f, 0.f};
-      for (int c = 0; c < cq; c += 4 * kMmaDepth) {
-        uint4 na[kMmaDepth], nb[kMmaDepth], qv[kMmaDepth];
+      const bool has_next = rb + kQuads * kMmaRows < r_hi;
+      const uint4* pna = has_next ? row_ptr(rb + kQuads * kMmaRows, 0) : pa;
+      const uint4* pnb = has_next ? row_ptr(rb + kQuads * kMmaRows, 1) : pb;
+      float c0[NT][4], c1[NT][4];
 #pragma unroll
-        for (int u = 0; u < kMmaDepth; ++u)                // query fragments of this step
-          qv[u] = c + 4 * u < cq ? qrow[4 * (c + 4 * u)] : make_uint4(0, 0, 0, 0);
+      for (int i = 0; i < NT; ++i)
+#pragma unroll
+        for (int e = 0; e < 4; ++e) c0[i][e] = c1[i][e] = 0.f;
+      for (int c = 0; c < cq; c += 4 * kMmaDepth) {
+        uint4 na[kMmaDepth], nb[kMmaDepth];
         const int cn = c + 4 * kMmaDepth;
         const bool same = cn < cq;                         // next step: same group or the next one
         const uint4* sa = same ? pa + 4 * cn : pna;
@@ -276,69 +289,78 @@ scan_mma_kernel(PoolView pv, const uint16_t* __restrict__ q_raw, int nq, int k,
         }
 #pragma unroll
         for (int u = 0; u < kMmaDepth; ++u) {
-          mma_bf16(c0, ka[u].x, kb[u].x, ka[u].y, kb[u].y, qv[u].x, qv[u].y);
-          mma_bf16(c1, ka[u].z, kb[u].z, ka[u].w, kb[u].w, qv[u].z, qv[u].w);
+#pragma unroll
+          for (int i = 0; i < NT; ++i) {
+            const uint4 qv = c + 4 * u < cq ? qrow[(size_t)8 * i * q_stride + 4 * (c + 4 * u)]
+                                            : make_uint4(0, 0, 0, 0);
+            mma_bf16(c0[i], ka[u].x, kb[u].x, ka[u].y, kb[u].y, qv.x, qv.y);
+            mma_bf16(c1[i], ka[u].z, kb[u].z, ka[u].w, kb[u].w, qv.z, qv.w);
+          }
         }
 #pragma unroll
         for (int u = 0; u < kMmaDepth; ++u) { ka[u] = na[u]; kb[u] = nb[u]; }
       }
       pa = pna;
       pb = pnb;
-      // partial scores of (row0, 2t), (row0, 2t+1), (row1, 2t), (row1, 2t+1)
-      // two buffers, one barrier per group: a warp reads a group's partials before it starts
+      // partial scores of (row0, 2t), (row0, 2t+1), (row1, 2t), (row1, 2t+1) of every tile.
+      // Two buffers, one barrier per group: a warp reads a group's partials before it starts
       // the next group, so when it arrives here for group i it is done with group i - 1, and
       // the barrier of group i - 1 has shown that everyone was done with group i - 2
-      float4* pbuf = part + (buf ? 4 * 32 * 2 : 0);
+      float4* pbuf = part + (buf ? kQuads * 4 * NT * 32 : 0);
       buf ^= 1;
-      pbuf[kq * 32 + lane] = make_float4(c0[0] + c1[0], c0[1] + c1[1], c0[2] + c1[2], c0[3] + c1[3]);
+#pragma unroll
+      for (int i = 0; i < NT; ++i)
+        pbuf[(kq * NT + i) * 32 + lane] = make_float4(c0[i][0] + c1[i][0], c0[i][1] + c1[i][1],
+                                                      c0[i][2] + c1[i][2], c0[i][3] + c1[i][3]);
       quad_bar(1 + quad);                    // this group's partials are in
-      float4 sc;
-      {
-        const float4 p0 = pbuf[lane], p1 = pbuf[32 + lane], p2 = pbuf[64 + lane], p3 = pbuf[96 + lane];
-        sc.x = ((p0.x + p1.x) + p2.x) + p3.x;
-        sc.y = ((p0.y + p1.y) + p2.y) + p3.y;
-        sc.z = ((p0.z + p1.z) + p2.z) + p3.z;
-        sc.w = ((p0.w + p1.w) + p2.w) + p3.w;
-      }
       uint64_t tag0 = 0, tag1 = 0;
       if (exclude_tag && own) {
         if (row0 < r_hi) tag0 = pv.trace_tag[pv.trace_id[row0]];
         if (row1 < r_hi) tag1 = pv.trace_tag[pv.trace_id[row1]];
       }
-      u64 key[4];
-      key[0] = (row0 < r_hi && live_a && !(ex_a != 0 && tag0 == ex_a)) ? pack_candidate(sc.x, (uint32_t)row0) : 0;
-      key[1] = (row0 < r_hi && live_b && !(ex_b != 0 && tag0 == ex_b)) ? pack_candidate(sc.y, (uint32_t)row0) : 0;
-      key[2] = (row1 < r_hi && live_a && !(ex_a != 0 && tag1 == ex_a)) ? pack_candidate(sc.z, (uint32_t)row1) : 0;
-      key[3] = (row1 < r_hi && live_b && !(ex_b != 0 && tag1 == ex_b)) ? pack_candidate(sc.w, (uint32_t)row1) : 0;
-      const bool any = (key[0] > kth[0]) | (key[1] > kth[1]) | (key[2] > kth[0]) | (key[3] > kth[1]);
+      u64 key[2 * NT][2];                    // [list][row0 / row1]
+      bool any = false;
+#pragma unroll
+      for (int i = 0; i < NT; ++i) {
+        const float4 p0 = pbuf[(0 * NT + i) * 32 + lane], p1 = pbuf[(1 * NT + i) * 32 + lane],
+                     p2 = pbuf[(2 * NT + i) * 32 + lane], p3 = pbuf[(3 * NT + i) * 32 + lane];
+        const float sx = ((p0.x + p1.x) + p2.x) + p3.x, sy = ((p0.y + p1.y) + p2.y) + p3.y;
+        const float sz = ((p0.z + p1.z) + p2.z) + p3.z, sw = ((p0.w + p1.w) + p2.w) + p3.w;
+        const int la = 2 * i, lb = 2 * i + 1;
+        key[la][0] = (row0 < r_hi && live[la] && !(ex[la] != 0 && tag0 == ex[la])) ? pack_candidate(sx, (uint32_t)row0) : 0;
+        key[lb][0] = (row0 < r_hi && live[lb] && !(ex[lb] != 0 && tag0 == ex[lb])) ? pack_candidate(sy, (uint32_t)row0) : 0;
+        key[la][1] = (row1 < r_hi && live[la] && !(ex[la] != 0 && tag1 == ex[la])) ? pack_candidate(sz, (uint32_t)row1) : 0;
+        key[lb][1] = (row1 < r_hi && live[lb] && !(ex[lb] != 0 && tag1 == ex[lb])) ? pack_candidate(sw, (uint32_t)row1) : 0;
+        any |= (key[la][0] > kth[la]) | (key[la][1] > kth[la]) | (key[lb][0] > kth[lb]) | (key[lb][1] > kth[lb]);
+      }
       if (__any_sync(0xffffffffu, any)) {
 #pragma unroll
-        for (int qq = 0; qq < 2; ++qq) {
-          const unsigned b0 = __ballot_sync(0xffffffffu, key[qq] > kth[qq]);
-          const unsigned b1 = __ballot_sync(0xffffffffu, key[qq + 2] > kth[qq]);
+        for (int l = 0; l < 2 * NT; ++l) {
+          const unsigned b0 = __ballot_sync(0xffffffffu, key[l][0] > kth[l]);
+          const unsigned b1 = __ballot_sync(0xffffffffu, key[l][1] > kth[l]);
           if (__popc(b0) + __popc(b1) >= kMmaBatchInsert) {
             // many rows pass (a list's first groups): the group's 16 scores of this query
             // are sorted as one vector and merged in, which costs about four insertions
             const int src = (lane & 7) * 4 + kq;
-            const uint32_t l0 = __shfl_sync(0xffffffffu, (uint32_t)key[qq], src);
-            const uint32_t h0 = __shfl_sync(0xffffffffu, (uint32_t)(key[qq] >> 32), src);
-            const uint32_t l1 = __shfl_sync(0xffffffffu, (uint32_t)key[qq + 2], src);
-            const uint32_t h1 = __shfl_sync(0xffffffffu, (uint32_t)(key[qq + 2] >> 32), src);
+            const uint32_t l0 = __shfl_sync(0xffffffffu, (uint32_t)key[l][0], src);
+            const uint32_t h0 = __shfl_sync(0xffffffffu, (uint32_t)(key[l][0] >> 32), src);
+            const uint32_t l1 = __shfl_sync(0xffffffffu, (uint32_t)key[l][1], src);
+            const uint32_t h1 = __shfl_sync(0xffffffffu, (uint32_t)(key[l][1] >> 32), src);
             u64 v[1];
             v[0] = lane < 8 ? (((u64)h0 << 32) | l0) : lane < 16 ? (((u64)h1 << 32) | l1) : 0;
-            v[0] = v[0] > kth[qq] ? v[0] : 0;
+            v[0] = v[0] > kth[l] ? v[0] : 0;
             warp_sort_desc<1>(v, lane);
             u64 add[E];
             add[0] = v[0];
 #pragma unroll
             for (int r = 1; r < E; ++r) add[r] = 0;
-            warp_merge_desc<E>(top[qq], add, lane);
-            kth[qq] = warp_list_get<E>(top[qq], k - 1);
+            warp_merge_desc<E>(top[l], add, lane);
+            kth[l] = warp_list_get<E>(top[l], k - 1);
             continue;
           }
 #pragma unroll
           for (int half = 0; half < 2; ++half) {
-            const u64 mine = key[qq + 2 * half];
+            const u64 mine = key[l][half];
             unsigned b = half ? b1 : b0;
             while (b) {
               const int src = __ffs(b) - 1;
@@ -346,9 +368,9 @@ scan_mma_kernel(PoolView pv, const uint16_t* __restrict__ q_raw, int nq, int k,
               const uint32_t lo = __shfl_sync(0xffffffffu, (uint32_t)mine, src);
               const uint32_t hi = __shfl_sync(0xffffffffu, (uint32_t)(mine >> 32), src);
               const u64 cand = ((u64)hi << 32) | lo;
-              if (cand > kth[qq]) {
-                warp_sorted_insert<E>(top[qq], cand, lane);
-                kth[qq] = warp_list_get<E>(top[qq], k - 1);
+              if (cand > kth[l]) {
+                warp_sorted_insert<E>(top[l], cand, lane);
+                kth[l] = warp_list_get<E>(top[l], k - 1);
               }
             }
           }
@@ -356,22 +378,26 @@ scan_mma_kernel(PoolView pv, const uint16_t* __restrict__ q_raw, int nq, int k,
       }
     }
 
-    // warp w merges the two quads' lists of query w and publishes the CTA's KK best
+    // warp w merges the quads' lists of query w and publishes the CTA's KK best
     __syncthreads();
 #pragma unroll
-    for (int qq = 0; qq < 2; ++qq)
+    for (int l = 0; l < 2 * NT; ++l) {
+      const int qi = 8 * (l >> 1) + 2 * kq + (l & 1);
 #pragma unroll
       for (int r = 0; r < E; ++r)
-        scratch[((size_t)quad * kMmaQ + 2 * kq + qq) * KK + r * 32 + lane] = top[qq][r];
+        scratch[((size_t)quad * QP + qi) * KK + r * 32 + lane] = top[l][r];
+    }
     __syncthreads();
     if (q0 + warp < nq) {
-      u64 a[E], b[E];
+      u64 a[E];
 #pragma unroll
-      for (int r = 0; r < E; ++r) {
-        a[r] = scratch[((size_t)0 * kMmaQ + warp) * KK + r * 32 + lane];
-        b[r] = scratch[((size_t)1 * kMmaQ + warp) * KK + r * 32 + lane];
+      for (int r = 0; r < E; ++r) a[r] = scratch[((size_t)0 * QP + warp) * KK + r * 32 + lane];
+      for (int qd = 1; qd < kQuads; ++qd) {
+        u64 b[E];
+#pragma unroll
+        for (int r = 0; r < E; ++r) b[r] = scratch[((size_t)qd * QP + warp) * KK + r * 32 + lane];
+        warp_merge_desc<E>(a, b, lane);
       }
-      warp_merge_desc<E>(a, b, lane);
       u64* dst = partial + ((size_t)blockIdx.x * nq + (q0 + warp)) * KK;
 #pragma unroll
       for (int r = 0; r < E; ++r) dst[r * 32 + lane] = a[r];
@@ -379,37 +405,53 @@ scan_mma_kernel(PoolView pv, const uint16_t* __restrict__ q_raw, int nq, int k,
   }
 }
 
-size_t scan_mma_smem(int32_t d, int32_t kk) {
-  return (size_t)kMmaQ * ((size_t)d * 2 + kMmaPadBytes) + (size_t)2 * kMmaQ * kk * sizeof(u64);
+size_t scan_mma_smem(int32_t d, int32_t kk, int32_t nt) {
+  const size_t qp = (size_t)kMmaQ * nt, quads = 2 * (size_t)nt;
+  return qp * ((size_t)d * 2 + kMmaPadBytes) + quads * qp * kk * sizeof(u64) +
+         2 * quads * 4 * nt * 32 * sizeof(float4);
+}
+
+// 8-query tiles per pass (1 or 2) for a call of nq queries, or 0 if the kernel cannot take
+// the pool's width or the list length
+int scan_mma_tiles(int32_t d, int32_t kk, int32_t nq, size_t smem_limit) {
+  if (d % 128 != 0 || kk > 64) return 0;
+  if (nq > kMmaQ && scan_mma_smem(d, kk, 2) <= smem_limit) return 2;
+  return scan_mma_smem(d, kk, 1) <= smem_limit ? 1 : 0;
 }
 
 bool scan_mma_supports(int32_t d, int32_t kk, size_t smem_limit) {
-  return d % 128 == 0 && kk <= 64 && scan_mma_smem(d, kk) <= smem_limit;
+  return scan_mma_tiles(d, kk, 1, smem_limit) != 0;
 }
 
-template <int E>
+template <int E, int NT>
 static cudaError_t launch_mma_one(const PoolView& pv, const uint16_t* q_raw, int nq, int k,
                                   const uint64_t* ex, u64* partial, int32_t* q_valid,
                                   DeviceStats* stats, int grid, cudaStream_t st) {
-  const size_t smem = scan_mma_smem(pv.d, 32 * E);
-  cudaError_t e = cudaFuncSetAttribute(scan_mma_kernel<E>,
+  const size_t smem = scan_mma_smem(pv.d, 32 * E, NT);
+  cudaError_t e = cudaFuncSetAttribute(scan_mma_kernel<E, NT>,
                                        cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
-  return launch_pdl(scan_mma_kernel<E>, dim3(grid), dim3(kMmaThreads), smem, st, pv, q_raw, nq, k,
-                    ex, partial, q_valid, stats);
+  return launch_pdl(scan_mma_kernel<E, NT>, dim3(grid), dim3(kMmaThreads * NT), smem, st, pv, q_raw,
+                    nq, k, ex, partial, q_valid, stats);
 }
 
 cudaError_t launch_scan_mma(const PoolView& pv, const uint16_t* q_raw, int32_t nq, int32_t k,
                             int32_t kk, const uint64_t* exclude_tag, u64* partial,
                             int32_t* q_valid, DeviceStats* stats, int32_t max_lists,
-                            int32_t num_sms, int32_t* n_lists, cudaStream_t st) {
-  const int grid = scan_gemv_grid(pv.n_rows, num_sms, max_lists);
+                            int32_t num_sms, size_t smem_limit, int32_t* n_lists,
+                            cudaStream_t st) {
+  const int nt = scan_mma_tiles(pv.d, kk, nq, smem_limit);
+  if (nt == 0) return cudaErrorInvalidValue;
+  int grid = scan_gemv_grid(pv.n_rows, num_sms, max_lists);      // two CTAs of 8 warps per SM
+  if (nt == 2) grid = (grid + 1) / 2;                             // one CTA of 16 warps per SM
   *n_lists = grid;
+  if (kk == 32 && nt == 1)
+    return launch_mma_one<1, 1>(pv, q_raw, nq, k, exclude_tag, partial, q_valid, stats, grid, st);
+  if (kk == 64 && nt == 1)
+    return launch_mma_one<2, 1>(pv, q_raw, nq, k, exclude_tag, partial, q_valid, stats, grid, st);
   if (kk == 32)
-    return launch_mma_one<1>(pv, q_raw, nq, k, exclude_tag, partial, q_valid, stats, grid, st);
-  if (kk == 64)
-    return launch_mma_one<2>(pv, q_raw, nq, k, exclude_tag, partial, q_valid, stats, grid, st);
-  return cudaErrorInvalidValue;
+    return launch_mma_one<1, 2>(pv, q_raw, nq, k, exclude_tag, partial, q_valid, stats, grid, st);
+  return launch_mma_one<2, 2>(pv, q_raw, nq, k, exclude_tag, partial, q_valid, stats, grid, st);
 }
 
 }  // namespace oilbird

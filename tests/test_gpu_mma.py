@@ -49,9 +49,10 @@ def test_hamming_pool_exact_scores_and_tie_order(d):
     assert np.array_equal(o.cont_len.numpy(), ref.cont_len)
 
 
-@pytest.mark.parametrize("nq,k", [(1, 8), (3, 8), (5, 32), (8, 16), (8, 33), (11, 64), (17, 5)])
+@pytest.mark.parametrize("nq,k", [(1, 8), (3, 8), (5, 32), (8, 16), (8, 33), (9, 8), (11, 64), (16, 16), (17, 5), (35, 40)])
 def test_nq_and_k_combinations(nq, k):
-    # nq above 8 runs in several passes over the keys; k above 32 uses two registers per lane
+    # 9 to 16 queries take two 8-query tiles per pass, more run in several passes over the
+    # keys; k above 32 uses two registers per lane
     w = W.C1.scaled(nq=nq, k=k, n_rows=3000, d=512, cont_len=5)
     for wl in (w, w.separated()):
         pool, ora = fill_both(wl)
@@ -122,7 +123,13 @@ def test_auto_path_uses_it_for_small_batches_only():
                torch.zeros(64, dtype=torch.int32, device="cuda"), tag=1)
     l0 = big.launch_count
     big.query(torch.randn(9, 256, device="cuda").to(torch.bfloat16), pr)
-    assert big.launch_count - l0 == 3                        # query normalisation + tcgen05 scan + merge
+    assert big.launch_count - l0 == 2                        # sixteen queries per pass fit: still this scan
+    big17 = B.Pool(256, 64, max_nq=32)
+    big17.append(torch.randn(64, 256, device="cuda").to(torch.bfloat16),
+                 torch.zeros(64, dtype=torch.int32, device="cuda"), tag=1)
+    l0 = big17.launch_count
+    big17.query(torch.randn(17, 256, device="cuda").to(torch.bfloat16), pr)
+    assert big17.launch_count - l0 == 3                      # query normalisation + tcgen05 scan + merge
     # widths that are not a multiple of 128 and k above 64 stay on the other scans
     odd = B.Pool(200, 64, max_nq=8, max_k=128)
     odd.append(torch.randn(64, 200, device="cuda").to(torch.bfloat16),

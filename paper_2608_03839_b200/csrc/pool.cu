@@ -429,6 +429,9 @@ static bool out_ok(const oilbird_query_out* o, bool need_idx) {
 // streams keys like the CUDA-core scan and starts within a few microseconds; above, the
 // tcgen05 scan's higher streaming rate has made up for its ~40 us of start-up.
 constexpr int64_t kMmaMaxKeyBytes = 2ll << 30;
+// rows wider than 4096 elements stream ~10 % slower there (d = 5120: 5.2-5.6 TB/s; d = 8192
+// leaves room for one CTA per SM only): 116 against 124 us at 532 MB, 206 against 184 at 1 GB
+constexpr int64_t kMmaMaxKeyBytesWide = 768ll << 20;
 // 9 to 16 queries (two 8-query tiles per pass, one CTA per SM) stream at two thirds of that
 // rate: only pools that the start-up dominates (8,192 rows x 4096: 41 us against 53)
 constexpr int64_t kMma16MaxKeyBytes = 128ll << 20;
@@ -439,7 +442,8 @@ static int resolve_path(const oilbird_pool* p, const oilbird_query_params* pr, i
   if (pr->path != OILBIRD_PATH_AUTO) return pr->path;
   if (nq <= 2) return OILBIRD_PATH_GEMV;
   const int64_t key_bytes = p->n_rows * (int64_t)p->r.d * 2;
-  if (nq <= 16 && !p->r.e4m3 && key_bytes <= (nq <= 8 ? kMmaMaxKeyBytes : kMma16MaxKeyBytes)) {
+  const int64_t mma_max = nq > 8 ? kMma16MaxKeyBytes : p->r.d <= 4096 ? kMmaMaxKeyBytes : kMmaMaxKeyBytesWide;
+  if (nq <= 16 && !p->r.e4m3 && key_bytes <= mma_max) {
     // up to 8 queries in one pass of 8; 9 to 16 only where 16 fit in one pass
     const int nt = scan_mma_tiles(p->r.d, list_len(pr->k), nq, p->smem_limit);
     if (nt == 2 || (nt == 1 && nq <= 8)) return OILBIRD_PATH_MMA;

@@ -194,7 +194,9 @@ int oilbird_pool_evict_oldest(oilbird_pool_t* pool, int32_t n_traces, int64_t* r
  * arguments, results and error codes as the two calls (Algorithm 1 runs once per decoding
  * step: the accepted tokens' states are stored, then the new last position is looked up).
  * Nothing is appended if the query arguments are invalid.  For the single-request scan
- * (nq <= 2; 16-bit and 8-bit pools) and up to 64 rows the append has no kernel of its own: the first n CTAs of the
+ * (nq <= 2; 16-bit and 8-bit pools) and the warp-level tensor scan in its 8-query form
+ * (OILBIRD_PATH_MMA, nq <= 8), and up to 64 rows, the append has no kernel of its own: the
+ * first n CTAs of the
  * scan normalise one row each before they start scanning, and the warps that reach the
  * appended rows (the last rows of the pool) first wait, bounded, for a counter that says
  * all n have been written (a time-out raises the `stalled` status, see oilbird_pool_status).

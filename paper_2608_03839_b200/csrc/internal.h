@@ -152,7 +152,7 @@ cudaError_t launch_scan_mma(const PoolView& pv, const uint16_t* q_raw, int32_t n
                             int32_t kk, const uint64_t* exclude_tag, unsigned long long* partial,
                             int32_t* q_valid, DeviceStats* stats, int32_t max_lists,
                             int32_t num_sms, size_t smem_limit, int32_t* n_lists,
-                            cudaStream_t st);
+                            const FusedAppend* fused, cudaStream_t st);
 
 // a2+a3 (tensor cores): the same contract for queries [q0, q0+nq_c) of a call whose
 // normalised queries already sit in qn.  TcCache holds the pool's TMA tensor maps

@@ -509,7 +509,7 @@ static int query_impl(oilbird_pool_t* p, const void* q, int32_t nq, const oilbir
     } else if (path == OILBIRD_PATH_MMA) {
       e = launch_scan_mma(pv, (const uint16_t*)q, nq, pr->k, kk, pr->exclude_tag, p->partial,
                           p->q_valid, p->stats, p->r.max_lists, p->num_sms, p->smem_limit,
-                          &n_lists, st);
+                          &n_lists, fused, st);
       if (e != cudaSuccess) return cuda_fail(e, "warp-level tensor scan kernel launch");
       p->launches += 1;
     } else {
@@ -556,9 +556,13 @@ static int step_impl(oilbird_pool_t* p, const void* states, const int32_t* token
   const int64_t rows_after = p->n_rows + n;
   // (8-bit pools always use the CUDA-core scan; its passes beyond the first two queries
   // would find the rows in place, but keep to the single-request case there too)
+  const int path = p->r.e4m3 ? OILBIRD_PATH_AUTO : resolve_path(p, pr, nq);
   const bool gemv = p->r.e4m3 ? (nq <= 2 && pr->path != OILBIRD_PATH_TENSOR)
-                              : resolve_path(p, pr, nq) == OILBIRD_PATH_GEMV;
-  const bool fuse = n >= 1 && n <= kFuseMaxRows && gemv &&
+                              : path == OILBIRD_PATH_GEMV;
+  // the warp-level tensor scan appends the step's rows itself in its 8-query form
+  const bool mma8 = path == OILBIRD_PATH_MMA &&
+                    scan_mma_tiles(p->r.d, list_len(pr->k), nq, p->smem_limit) == 1;
+  const bool fuse = n >= 1 && n <= kFuseMaxRows && (gemv || mma8) &&
                     scan_gemv_grid(rows_after, p->num_sms, p->r.max_lists) >= n;
   if (!fuse) {
     rc = append_impl(p, states, tokens, n, tag, flags, -1, stream);

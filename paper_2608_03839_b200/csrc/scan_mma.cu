@@ -45,6 +45,15 @@ __device__ __forceinline__ void mma_bf16(float (&c)[4], uint32_t a0, uint32_t a1
       : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 
+struct BoolTrue { static constexpr bool value = true; };
+struct BoolFalse { static constexpr bool value = false; };
+
+// 16 bytes of a key: the read-only streaming path, or through L2 for rows that another CTA
+// of this launch has just written
+__device__ __forceinline__ uint4 ld_key16(const uint4* p, bool fresh) {
+  return fresh ? ld_cg16(p) : ld_stream16(p);
+}
+
 // barrier among the four warps of a quad (ids 1 and 2; 0 is __syncthreads)
 __device__ __forceinline__ void quad_bar(int id) {
   asm volatile("bar.sync %0, 128;" ::"r"(id) : "memory");
@@ -171,7 +180,7 @@ template <int E, int NT>
 __global__ void __launch_bounds__(kMmaThreads * NT, 2 / NT)
 scan_mma_kernel(PoolView pv, const uint16_t* __restrict__ q_raw, int nq, int k,
                 const uint64_t* __restrict__ exclude_tag, u64* __restrict__ partial,
-                int32_t* __restrict__ q_valid, DeviceStats* stats) {
+                int32_t* __restrict__ q_valid, DeviceStats* stats, FusedAppend fa) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   constexpr int KK = 32 * E;
   constexpr int QP = kMmaQ * NT;             // queries per pass
@@ -189,10 +198,41 @@ scan_mma_kernel(PoolView pv, const uint16_t* __restrict__ q_raw, int nq, int k,
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int g = lane >> 2, t = lane & 3;
+  // contiguous, balanced share of the rows for this CTA; the fa.n CTAs that first append a
+  // row of this step take 1/32 less than the others (as in the CUDA-core scan)
   const int64_t n = pv.n_rows;
-  const int r_lo = (int)((n * blockIdx.x) / gridDim.x);
-  const int r_hi = (int)((n * (blockIdx.x + 1)) / gridDim.x);
+  const int64_t w_lo = 32ll * blockIdx.x - min((int)blockIdx.x, fa.n);
+  const int64_t w_hi = 32ll * (blockIdx.x + 1) - min((int)blockIdx.x + 1, fa.n);
+  const int64_t w_all = 32ll * gridDim.x - min((int)gridDim.x, fa.n);
+  const int r_lo = (int)((n * w_lo) / w_all);
+  const int r_hi = (int)((n * w_hi) / w_all);
   const uint4* keys4 = reinterpret_cast<const uint4*>(pv.keys);
+
+  // the step's append (Section 4 "(i) Store", Eq. 1), one row per CTA; the 8-query form only
+  // (the block routine wants kNormThreads threads)
+  if (NT == 1 && (int)blockIdx.x < fa.n) {
+    const int r = blockIdx.x;
+    const int64_t row = (int64_t)fa.row0 + r;
+    const int code = normalize_row<false>(fa.states + (size_t)r * d, fa.keys + row * d, d);
+    if (threadIdx.x == 0) {
+      fa.tok[row] = fa.tokens[r];
+      fa.trace_id[row] = fa.trace;
+      if (code != kRowOk) atomicAdd(&stats->degenerate_rows, 1ull);  // stored as a zero key
+      if (r == 0) {
+        fa.trace_end[fa.trace] = fa.row0 + fa.n;
+        if (fa.set_tag) { fa.trace_tag[fa.trace] = fa.tag; fa.trace_gbase[fa.trace] = fa.gbase; }
+      }
+    }
+    __threadfence();                   // this thread's part of the row, before the count
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      __threadfence();                 // cumulative: the whole CTA's row, as seen through the barrier
+      atomicAdd(fa.ready, 1ull);
+    }
+  }
+  bool waited = fa.n == 0;             // this warp has seen the appended rows arrive
+  // a group of rows that holds rows of this step's append: read through L2, after the wait
+  auto fresh_at = [&](int rbx) { return fa.n > 0 && rbx + kMmaRows > fa.row0; };
 
   for (int q0 = 0; q0 < nq; q0 += QP) {
     __syncthreads();
@@ -254,19 +294,28 @@ scan_mma_kernel(PoolView pv, const uint16_t* __restrict__ q_raw, int nq, int k,
     int rb = r_lo + quad * kMmaRows;
     const uint4 *pa = keys4, *pb = keys4;
     uint4 ka[kMmaDepth], kb[kMmaDepth];
+    bool cur_fresh = rb < r_hi && fresh_at(rb);
     if (rb < r_hi) {
+      if (cur_fresh && !waited) {
+        wait_fused_rows(fa, stats);
+        waited = true;
+      }
       pa = row_ptr(rb, 0);
       pb = row_ptr(rb, 1);
 #pragma unroll
       for (int u = 0; u < kMmaDepth; ++u) {
         const bool in = 4 * u < cq;
-        ka[u] = in ? ld_stream16(pa + 4 * (4 * u)) : make_uint4(0, 0, 0, 0);
-        kb[u] = in ? ld_stream16(pb + 4 * (4 * u)) : make_uint4(0, 0, 0, 0);
+        ka[u] = in ? ld_key16(pa + 4 * (4 * u), cur_fresh) : make_uint4(0, 0, 0, 0);
+        kb[u] = in ? ld_key16(pb + 4 * (4 * u), cur_fresh) : make_uint4(0, 0, 0, 0);
       }
     }
     for (; rb < r_hi; rb += kQuads * kMmaRows) {
       const int row0 = rb + g, row1 = rb + g + 8;
       const bool has_next = rb + kQuads * kMmaRows < r_hi;
+      const bool next_fresh = has_next && fresh_at(rb + kQuads * kMmaRows);
+      // the next group's first step is fetched early unless it holds rows that this launch
+      // appends and the wait for them is still ahead
+      const bool pre_next = has_next && (!next_fresh || waited);
       const uint4* pna = has_next ? row_ptr(rb + kQuads * kMmaRows, 0) : pa;
       const uint4* pnb = has_next ? row_ptr(rb + kQuads * kMmaRows, 1) : pb;
       float c0[NT][4], c1[NT][4];
@@ -274,32 +323,45 @@ scan_mma_kernel(PoolView pv, const uint16_t* __restrict__ q_raw, int nq, int k,
       for (int i = 0; i < NT; ++i)
 #pragma unroll
         for (int e = 0; e < 4; ++e) c0[i][e] = c1[i][e] = 0.f;
-      for (int c = 0; c < cq; c += 4 * kMmaDepth) {
-        uint4 na[kMmaDepth], nb[kMmaDepth];
-        const int cn = c + 4 * kMmaDepth;
-        const bool same = cn < cq;                         // next step: same group or the next one
-        const uint4* sa = same ? pa + 4 * cn : pna;
-        const uint4* sb = same ? pb + 4 * cn : pnb;
-        const int left = same ? cq - cn : (has_next ? cq : 0);
+      // the steps of a group; kMixed = some of its loads (its own or the next group's first
+      // step) go to rows appended by this launch and must not use the read-only path
+      auto run_steps = [&](auto mixed) {
+        constexpr bool kMixed = decltype(mixed)::value;
+        for (int c = 0; c < cq; c += 4 * kMmaDepth) {
+          uint4 na[kMmaDepth], nb[kMmaDepth];
+          const int cn = c + 4 * kMmaDepth;
+          const bool same = cn < cq;                       // next step: same group or the next one
+          const uint4* sa = same ? pa + 4 * cn : pna;
+          const uint4* sb = same ? pb + 4 * cn : pnb;
+          const int left = same ? cq - cn : (pre_next ? cq : 0);
+          const bool ld_fresh = kMixed && (same ? cur_fresh : next_fresh);
 #pragma unroll
-        for (int u = 0; u < kMmaDepth; ++u) {
-          const bool in = 4 * u < left;
-          na[u] = in ? ld_stream16(sa + 4 * (4 * u)) : make_uint4(0, 0, 0, 0);
-          nb[u] = in ? ld_stream16(sb + 4 * (4 * u)) : make_uint4(0, 0, 0, 0);
-        }
-#pragma unroll
-        for (int u = 0; u < kMmaDepth; ++u) {
-#pragma unroll
-          for (int i = 0; i < NT; ++i) {
-            const uint4 qv = c + 4 * u < cq ? qrow[(size_t)8 * i * q_stride + 4 * (c + 4 * u)]
-                                            : make_uint4(0, 0, 0, 0);
-            mma_bf16(c0[i], ka[u].x, kb[u].x, ka[u].y, kb[u].y, qv.x, qv.y);
-            mma_bf16(c1[i], ka[u].z, kb[u].z, ka[u].w, kb[u].w, qv.z, qv.w);
+          for (int u = 0; u < kMmaDepth; ++u) {
+            const bool in = 4 * u < left;
+            if (kMixed) {
+              na[u] = in ? ld_key16(sa + 4 * (4 * u), ld_fresh) : make_uint4(0, 0, 0, 0);
+              nb[u] = in ? ld_key16(sb + 4 * (4 * u), ld_fresh) : make_uint4(0, 0, 0, 0);
+            } else {
+              na[u] = in ? ld_stream16(sa + 4 * (4 * u)) : make_uint4(0, 0, 0, 0);
+              nb[u] = in ? ld_stream16(sb + 4 * (4 * u)) : make_uint4(0, 0, 0, 0);
+            }
           }
-        }
 #pragma unroll
-        for (int u = 0; u < kMmaDepth; ++u) { ka[u] = na[u]; kb[u] = nb[u]; }
-      }
+          for (int u = 0; u < kMmaDepth; ++u) {
+#pragma unroll
+            for (int i = 0; i < NT; ++i) {
+              const uint4 qv = c + 4 * u < cq ? qrow[(size_t)8 * i * q_stride + 4 * (c + 4 * u)]
+                                              : make_uint4(0, 0, 0, 0);
+              mma_bf16(c0[i], ka[u].x, kb[u].x, ka[u].y, kb[u].y, qv.x, qv.y);
+              mma_bf16(c1[i], ka[u].z, kb[u].z, ka[u].w, kb[u].w, qv.z, qv.w);
+            }
+          }
+#pragma unroll
+          for (int u = 0; u < kMmaDepth; ++u) { ka[u] = na[u]; kb[u] = nb[u]; }
+        }
+      };
+      if (cur_fresh || next_fresh) run_steps(BoolTrue{});
+      else run_steps(BoolFalse{});
       pa = pna;
       pb = pnb;
       // partial scores of (row0, 2t), (row0, 2t+1), (row1, 2t), (row1, 2t+1) of every tile.
@@ -315,8 +377,12 @@ scan_mma_kernel(PoolView pv, const uint16_t* __restrict__ q_raw, int nq, int k,
       quad_bar(1 + quad);                    // this group's partials are in
       uint64_t tag0 = 0, tag1 = 0;
       if (exclude_tag && own) {
-        if (row0 < r_hi) tag0 = pv.trace_tag[pv.trace_id[row0]];
-        if (row1 < r_hi) tag1 = pv.trace_tag[pv.trace_id[row1]];
+        // rows appended by this launch: their trace id and tag were written by another CTA a
+        // moment ago, so those are read through L2
+        if (row0 < r_hi)
+          tag0 = cur_fresh ? __ldcg(&pv.trace_tag[__ldcg(&pv.trace_id[row0])]) : pv.trace_tag[pv.trace_id[row0]];
+        if (row1 < r_hi)
+          tag1 = cur_fresh ? __ldcg(&pv.trace_tag[__ldcg(&pv.trace_id[row1])]) : pv.trace_tag[pv.trace_id[row1]];
       }
       u64 key[2 * NT][2];                    // [list][row0 / row1]
       bool any = false;
@@ -376,6 +442,19 @@ scan_mma_kernel(PoolView pv, const uint16_t* __restrict__ q_raw, int nq, int k,
           }
         }
       }
+      if (has_next && !pre_next) {
+        // the next group holds rows of this step's append: wait (bounded) until all of them
+        // are in, then fetch its first step
+        wait_fused_rows(fa, stats);
+        waited = true;
+#pragma unroll
+        for (int u = 0; u < kMmaDepth; ++u) {
+          const bool in = 4 * u < cq;
+          ka[u] = in ? ld_key16(pa + 4 * (4 * u), true) : make_uint4(0, 0, 0, 0);
+          kb[u] = in ? ld_key16(pb + 4 * (4 * u), true) : make_uint4(0, 0, 0, 0);
+        }
+      }
+      cur_fresh = next_fresh;
     }
 
     // warp w merges the quads' lists of query w and publishes the CTA's KK best
@@ -426,32 +505,41 @@ bool scan_mma_supports(int32_t d, int32_t kk, size_t smem_limit) {
 template <int E, int NT>
 static cudaError_t launch_mma_one(const PoolView& pv, const uint16_t* q_raw, int nq, int k,
                                   const uint64_t* ex, u64* partial, int32_t* q_valid,
-                                  DeviceStats* stats, int grid, cudaStream_t st) {
+                                  DeviceStats* stats, int grid, const FusedAppend& fa,
+                                  cudaStream_t st) {
   const size_t smem = scan_mma_smem(pv.d, 32 * E, NT);
   cudaError_t e = cudaFuncSetAttribute(scan_mma_kernel<E, NT>,
                                        cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
   return launch_pdl(scan_mma_kernel<E, NT>, dim3(grid), dim3(kMmaThreads * NT), smem, st, pv, q_raw,
-                    nq, k, ex, partial, q_valid, stats);
+                    nq, k, ex, partial, q_valid, stats, fa);
 }
 
 cudaError_t launch_scan_mma(const PoolView& pv, const uint16_t* q_raw, int32_t nq, int32_t k,
                             int32_t kk, const uint64_t* exclude_tag, u64* partial,
                             int32_t* q_valid, DeviceStats* stats, int32_t max_lists,
                             int32_t num_sms, size_t smem_limit, int32_t* n_lists,
-                            cudaStream_t st) {
+                            const FusedAppend* fused, cudaStream_t st) {
   const int nt = scan_mma_tiles(pv.d, kk, nq, smem_limit);
   if (nt == 0) return cudaErrorInvalidValue;
   int grid = scan_gemv_grid(pv.n_rows, num_sms, max_lists);      // two CTAs of 8 warps per SM
   if (nt == 2) grid = (grid + 1) / 2;                             // one CTA of 16 warps per SM
   *n_lists = grid;
+  FusedAppend fa = {};
+  if (fused) {
+    // every appending CTA must exist, and all CTAs be resident together (they are: at most
+    // two per SM are launched), because scanning warps wait for the appending ones; the
+    // 8-query form only
+    if (nt != 1 || fused->n > grid || fused->n > kFuseMaxRows) return cudaErrorInvalidValue;
+    fa = *fused;
+  }
   if (kk == 32 && nt == 1)
-    return launch_mma_one<1, 1>(pv, q_raw, nq, k, exclude_tag, partial, q_valid, stats, grid, st);
+    return launch_mma_one<1, 1>(pv, q_raw, nq, k, exclude_tag, partial, q_valid, stats, grid, fa, st);
   if (kk == 64 && nt == 1)
-    return launch_mma_one<2, 1>(pv, q_raw, nq, k, exclude_tag, partial, q_valid, stats, grid, st);
+    return launch_mma_one<2, 1>(pv, q_raw, nq, k, exclude_tag, partial, q_valid, stats, grid, fa, st);
   if (kk == 32)
-    return launch_mma_one<1, 2>(pv, q_raw, nq, k, exclude_tag, partial, q_valid, stats, grid, st);
-  return launch_mma_one<2, 2>(pv, q_raw, nq, k, exclude_tag, partial, q_valid, stats, grid, st);
+    return launch_mma_one<1, 2>(pv, q_raw, nq, k, exclude_tag, partial, q_valid, stats, grid, fa, st);
+  return launch_mma_one<2, 2>(pv, q_raw, nq, k, exclude_tag, partial, q_valid, stats, grid, fa, st);
 }
 
 }  // namespace oilbird

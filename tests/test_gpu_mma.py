@@ -156,3 +156,37 @@ def test_paper_scale_pool_batch_of_eight_full_width():
         out = pool.query(q, pr)
         assert pool.launch_count - l0 == 2
         check_query(out, ora, W.to_bits(q), pr)
+
+
+def test_fused_step_appends_inside_the_scan_and_sees_the_new_rows_tags():
+    # 3 to 8 queries and up to 64 new rows: the scan's first CTAs append the step's rows
+    # (two launches per step); a query of the same step finds them, honours their tag, and the
+    # stored rows equal the oracle's
+    w = W.C1.scaled(n_rows=4096, nq=5)
+    pool, ora = fill_both(w, spare_rows=1024)
+    g = torch.Generator(device="cuda").manual_seed(33)
+    for step in range(8):
+        n = [8, 1, 64, 33, 8, 16, 2, 8][step]
+        st = torch.randn(n, w.d, generator=g, device="cuda").to(torch.bfloat16)
+        tk = torch.randint(0, 100, (n,), generator=g, device="cuda", dtype=torch.int32)
+        q = torch.randn(5, w.d, generator=g, device="cuda").to(torch.bfloat16)
+        q[0] = st[n - 1]
+        q[3] = st[0]
+        tag = 9000 + step
+        ex = torch.tensor([tag, 12345, 0, 0, tag], dtype=torch.int64, device="cuda")
+        pr = fixed(4, 4, theta=-2.0)
+        pr.exclude_tag = ex
+        new_trace = step % 2 == 0
+        l0 = pool.launch_count
+        out = pool.step(st, tk, q, pr, tag=tag, new_trace=new_trace)
+        assert pool.launch_count - l0 == 2
+        ora.append(W.to_bits(st), tk.cpu().numpy(), tag=tag, new_trace=new_trace)
+        first_new = len(pool) - n
+        if new_trace:                                         # a new trace with the excluded tag
+            assert all(int(r) < first_new for r in out.idx[0].tolist())
+        assert int(out.idx[3, 0]) == first_new
+        check_query(out, ora, W.to_bits(q), pr, exclude=ex.cpu().numpy().astype(np.uint64))
+    assert pool.stats()["stalled"] == 0
+    keys, tok, tid = pool.read_rows()
+    assert np.array_equal(keys, ora.keys) and np.array_equal(tok, ora.tokens)
+    assert np.array_equal(tid, ora.trace_ids)

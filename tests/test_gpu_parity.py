@@ -370,7 +370,8 @@ def test_caller_provided_arena():
     check_query(pool.query(q, fixed(8, 8)), ora, W.to_bits(q), fixed(8, 8))
 
 
-@pytest.mark.parametrize("nq,path", [(1, "gemv"), (2, "gemv"), (4, "tensor")])
+@pytest.mark.parametrize("nq,path", [(1, "gemv"), (2, "gemv"), (4, "tensor"), (3, "mma"), (8, "mma"),
+                                     (11, "mma")])
 def test_step_is_append_plus_query(nq, path):
     # the fused step lets the scan run next to its own append; results must not change,
     # and the rows appended in the same step must be found
@@ -379,7 +380,7 @@ def test_step_is_append_plus_query(nq, path):
     pool2, _ = fill_both(w, spare_rows=512)
     g = torch.Generator(device="cuda").manual_seed(11)
     pr = fixed(8, 8, theta=-2.0)
-    pr.path = B.PATH_GEMV if path == "gemv" else B.PATH_TENSOR
+    pr.path = {"gemv": B.PATH_GEMV, "tensor": B.PATH_TENSOR, "mma": B.PATH_MMA}[path]
     for step in range(8):
         n = [8, 1, 0, 33, 64, 100, 8, 2][step]      # up to 64 rows ride inside the scan kernel
         st = torch.randn(n, w.d, generator=g, device="cuda").to(torch.bfloat16)

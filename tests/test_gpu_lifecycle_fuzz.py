@@ -53,7 +53,8 @@ def test_random_life_cycle(fmt, seed):
                            depth_mode=int(rng.choice([B.DEPTH_FIXED, B.DEPTH_TIERED])),
                            cont_len=int(rng.choice([1, 4, 16])), offset=int(rng.choice([0, 1, 2])))
         if fmt == "bf16" and nq >= 1:
-            pr.path = int(rng.choice([B.PATH_AUTO, B.PATH_GEMV, B.PATH_TENSOR]))
+            paths = [B.PATH_AUTO, B.PATH_GEMV, B.PATH_TENSOR] + ([B.PATH_MMA] * 2 if d % 128 == 0 else [])
+            pr.path = int(rng.choice(paths))
         return pr
 
     for op_no in range(100):

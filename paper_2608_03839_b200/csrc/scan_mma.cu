@@ -268,17 +268,12 @@ scan_mma_kernel(PoolView pv, const uint16_t* __restrict__ q_raw, int nq, int k,
     // descending lists of this warp's 2 NT queries; kth = the k-th entry (0 while not full)
     u64 top[2 * NT][E];
     u64 kth[2 * NT];
-    bool live[2 * NT];
-    uint64_t ex[2 * NT];
     const bool own = t == kq;                                       // this lane's scores are this warp's
 #pragma unroll
     for (int l = 0; l < 2 * NT; ++l) {
       kth[l] = 0;
 #pragma unroll
       for (int r = 0; r < E; ++r) top[l][r] = 0;
-      const int qi = 8 * (l >> 1) + 2 * kq + (l & 1);               // query of list l within the pass
-      live[l] = own && q0 + qi < nq;
-      ex[l] = s_ex[qi];
     }
     int buf = 0;
 
@@ -393,10 +388,14 @@ scan_mma_kernel(PoolView pv, const uint16_t* __restrict__ q_raw, int nq, int k,
         const float sx = ((p0.x + p1.x) + p2.x) + p3.x, sy = ((p0.y + p1.y) + p2.y) + p3.y;
         const float sz = ((p0.z + p1.z) + p2.z) + p3.z, sw = ((p0.w + p1.w) + p2.w) + p3.w;
         const int la = 2 * i, lb = 2 * i + 1;
-        key[la][0] = (row0 < r_hi && live[la] && !(ex[la] != 0 && tag0 == ex[la])) ? pack_candidate(sx, (uint32_t)row0) : 0;
-        key[lb][0] = (row0 < r_hi && live[lb] && !(ex[lb] != 0 && tag0 == ex[lb])) ? pack_candidate(sy, (uint32_t)row0) : 0;
-        key[la][1] = (row1 < r_hi && live[la] && !(ex[la] != 0 && tag1 == ex[la])) ? pack_candidate(sz, (uint32_t)row1) : 0;
-        key[lb][1] = (row1 < r_hi && live[lb] && !(ex[lb] != 0 && tag1 == ex[lb])) ? pack_candidate(sw, (uint32_t)row1) : 0;
+        const int qa = 8 * i + 2 * kq;                     // queries of lists la, lb within the pass
+        const bool live_a = own && q0 + qa < nq, live_b = own && q0 + qa + 1 < nq;
+        // exclusion tags are read where they are used: they are rare, registers are not
+        const uint64_t ex_a = exclude_tag ? s_ex[qa] : 0, ex_b = exclude_tag ? s_ex[qa + 1] : 0;
+        key[la][0] = (row0 < r_hi && live_a && !(ex_a != 0 && tag0 == ex_a)) ? pack_candidate(sx, (uint32_t)row0) : 0;
+        key[lb][0] = (row0 < r_hi && live_b && !(ex_b != 0 && tag0 == ex_b)) ? pack_candidate(sy, (uint32_t)row0) : 0;
+        key[la][1] = (row1 < r_hi && live_a && !(ex_a != 0 && tag1 == ex_a)) ? pack_candidate(sz, (uint32_t)row1) : 0;
+        key[lb][1] = (row1 < r_hi && live_b && !(ex_b != 0 && tag1 == ex_b)) ? pack_candidate(sw, (uint32_t)row1) : 0;
         any |= (key[la][0] > kth[la]) | (key[la][1] > kth[la]) | (key[lb][0] > kth[lb]) | (key[lb][1] > kth[lb]);
       }
       if (__any_sync(0xffffffffu, any)) {

@@ -196,8 +196,8 @@ int oilbird_pool_evict_oldest(oilbird_pool_t* pool, int32_t n_traces, int64_t* r
  * Nothing is appended if the query arguments are invalid.  For the single-request scan
  * (nq <= 2; 16-bit and 8-bit pools) and the warp-level tensor scan in its 8-query form
  * (OILBIRD_PATH_MMA, nq <= 8), and up to 64 rows, the append has no kernel of its own: the
- * first n CTAs of the
- * scan normalise one row each before they start scanning, and the warps that reach the
+ * first CTAs of the scan normalise the rows before they start scanning (a row per CTA, or a
+ * row per warp that has no query to prepare), and the warps that reach the
  * appended rows (the last rows of the pool) first wait, bounded, for a counter that says
  * all n have been written (a time-out raises the `stalled` status, see oilbird_pool_status).
  */

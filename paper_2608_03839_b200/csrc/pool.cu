@@ -429,11 +429,8 @@ static bool out_ok(const oilbird_query_out* o, bool need_idx) {
 // streams keys like the CUDA-core scan and starts within a few microseconds; above, the
 // tcgen05 scan's higher streaming rate has made up for its ~40 us of start-up.
 constexpr int64_t kMmaMaxKeyBytes = 2ll << 30;
-// rows wider than 4096 elements stream ~10 % slower there (d = 5120: 5.2-5.6 TB/s; d = 8192
-// leaves room for one CTA per SM only): 116 against 124 us at 532 MB, 206 against 184 at 1 GB
-constexpr int64_t kMmaMaxKeyBytesWide = 768ll << 20;
 // 9 to 16 queries (two 8-query tiles per pass, one CTA per SM) stream at two thirds of that
-// rate: only pools that the start-up dominates (8,192 rows x 4096: 41 us against 53)
+// rate: only pools that the start-up dominates (8,192 rows x 4096: 33 us against 53)
 constexpr int64_t kMma16MaxKeyBytes = 128ll << 20;
 
 static int resolve_path(const oilbird_pool* p, const oilbird_query_params* pr, int32_t nq) {
@@ -442,7 +439,7 @@ static int resolve_path(const oilbird_pool* p, const oilbird_query_params* pr, i
   if (pr->path != OILBIRD_PATH_AUTO) return pr->path;
   if (nq <= 2) return OILBIRD_PATH_GEMV;
   const int64_t key_bytes = p->n_rows * (int64_t)p->r.d * 2;
-  const int64_t mma_max = nq > 8 ? kMma16MaxKeyBytes : p->r.d <= 4096 ? kMmaMaxKeyBytes : kMmaMaxKeyBytesWide;
+  const int64_t mma_max = nq > 8 ? kMma16MaxKeyBytes : kMmaMaxKeyBytes;
   if (nq <= 16 && !p->r.e4m3 && key_bytes <= mma_max) {
     // up to 8 queries in one pass of 8; 9 to 16 only where 16 fit in one pass
     const int nt = scan_mma_tiles(p->r.d, list_len(pr->k), nq, p->smem_limit);
@@ -562,8 +559,10 @@ static int step_impl(oilbird_pool_t* p, const void* states, const int32_t* token
   // the warp-level tensor scan appends the step's rows itself in its 8-query form
   const bool mma8 = path == OILBIRD_PATH_MMA &&
                     scan_mma_tiles(p->r.d, list_len(pr->k), nq, p->smem_limit) == 1;
-  const bool fuse = n >= 1 && n <= kFuseMaxRows && (gemv || mma8) &&
-                    scan_gemv_grid(rows_after, p->num_sms, p->r.max_lists) >= n;
+  const bool fuse =
+      n >= 1 && n <= kFuseMaxRows &&
+      ((gemv && scan_gemv_grid(rows_after, p->num_sms, p->r.max_lists) >= n) ||
+       (mma8 && 8 * (int64_t)scan_mma_grid(rows_after, p->num_sms, p->r.max_lists) >= n));
   if (!fuse) {
     rc = append_impl(p, states, tokens, n, tag, flags, -1, stream);
     if (rc) return rc;

@@ -5,9 +5,9 @@
 // large batches of the tcgen05 scan.  The tcgen05 scan needs whole 128-row tiles and a
 // completed K loop before a score exists, which costs about 40 us per query call on pools of
 // the paper's size (a few hundred MB); the CUDA-core scan runs out of issue slots beyond two
-// queries (64 FMAs per 16 key bytes at eight).  Here the key stream is organised exactly as
-// in the CUDA-core scan (2 CTAs x 8 warps per SM, contiguous row split, 16-byte streaming
-// loads straight into registers) and the arithmetic goes to mma.sync.m16n8k16 (bf16 in,
+// queries (64 FMAs per 16 key bytes at eight).  Here the key stream is organised as in the
+// CUDA-core scan (16 warps per SM, contiguous row split, 16-byte streaming loads straight
+// into registers) and the arithmetic goes to mma.sync.m16n8k16 (bf16 in,
 // fp32 accumulate): 16 rows x 8 queries x 32 elements cost two loads of keys, one shared
 // memory load of queries and two MMAs per lane, so the kernel stays bound by the key stream.
 //
@@ -27,7 +27,7 @@
 
 namespace oilbird {
 
-constexpr int kMmaThreads = 256;
+constexpr int kMmaThreads = 512;
 constexpr int kMmaWarps = kMmaThreads / 32;
 constexpr int kMmaQ = 8;          // queries per pass = the N of the instruction
 constexpr int kMmaRows = 16;      // rows per warp step = the M of the instruction
@@ -76,11 +76,17 @@ __device__ __forceinline__ int normalize_row_warp(const uint16_t* __restrict__ s
 #pragma unroll
     for (int v = 0; v < kNormThreads / 32; ++v) acc[v] = 0.0;
     for (int base = 0; base < n_chunks; base += kNormThreads) {
+      uint4 hv8[kNormThreads / 32];
+#pragma unroll
+      for (int v = 0; v < kNormThreads / 32; ++v) {
+        const int c = base + 32 * v + lane;
+        hv8[v] = c < n_chunks ? __ldg(src4 + c) : make_uint4(0, 0, 0, 0);
+      }
 #pragma unroll
       for (int v = 0; v < kNormThreads / 32; ++v) {
         const int c = base + 32 * v + lane;
         if (c < n_chunks) {
-          const uint4 hv = __ldg(src4 + c);
+          const uint4 hv = hv8[v];
           const uint32_t w[4] = {hv.x, hv.y, hv.z, hv.w};
 #pragma unroll
           for (int j = 0; j < 4; ++j) {
@@ -106,19 +112,30 @@ __device__ __forceinline__ int normalize_row_warp(const uint16_t* __restrict__ s
     for (int m = 16; m; m >>= 1) redo |= __shfl_xor_sync(0xffffffffu, redo, m);
     if (!redo && tot < 0x1p256) {                  // no Inf/NaN pattern either
       const double inv = 1.0 / sqrt(tot);
-      for (int c = lane; c < n_chunks; c += 32) {
-        const uint4 hv = __ldg(src4 + c);
-        const uint32_t w[4] = {hv.x, hv.y, hv.z, hv.w};
-        uint32_t o[4];
+      // eight chunks per lane at a time, their loads issued together (the row comes from L2)
+      for (int base = 0; base < n_chunks; base += kNormThreads) {
+        uint4 hv[kNormThreads / 32];
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {
-          const uint32_t hl = ((w[j] & 0x8000u) << 16) | (((w[j] & 0x7fffu) << 13) + 0x38000000u);
-          const uint32_t hh = (w[j] & 0x80000000u) | (((w[j] & 0x7fff0000u) >> 3) + 0x38000000u);
-          const float lo = __double2float_rn(__hiloint2double((int)hl, 0) * inv);
-          const float hi = __double2float_rn(__hiloint2double((int)hh, 0) * inv);
-          asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(o[j]) : "f"(hi), "f"(lo));
+        for (int v = 0; v < kNormThreads / 32; ++v) {
+          const int c = base + 32 * v + lane;
+          hv[v] = c < n_chunks ? __ldg(src4 + c) : make_uint4(0, 0, 0, 0);
         }
-        dst4[c] = make_uint4(o[0], o[1], o[2], o[3]);
+#pragma unroll
+        for (int v = 0; v < kNormThreads / 32; ++v) {
+          const int c = base + 32 * v + lane;
+          if (c >= n_chunks) continue;
+          const uint32_t w[4] = {hv[v].x, hv[v].y, hv[v].z, hv[v].w};
+          uint32_t o[4];
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            const uint32_t hl = ((w[j] & 0x8000u) << 16) | (((w[j] & 0x7fffu) << 13) + 0x38000000u);
+            const uint32_t hh = (w[j] & 0x80000000u) | (((w[j] & 0x7fff0000u) >> 3) + 0x38000000u);
+            const float lo = __double2float_rn(__hiloint2double((int)hl, 0) * inv);
+            const float hi = __double2float_rn(__hiloint2double((int)hh, 0) * inv);
+            asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(o[j]) : "f"(hi), "f"(lo));
+          }
+          dst4[c] = make_uint4(o[0], o[1], o[2], o[3]);
+        }
       }
       return kRowOk;
     }
@@ -173,18 +190,20 @@ __device__ __forceinline__ int normalize_row_warp(const uint16_t* __restrict__ s
   return ok ? kRowOk : ((bad || !isfinite(nrm)) ? kRowNonFinite : kRowZero);
 }
 
-// NT = number of 8-query tiles a pass scores (1: up to 8 queries, 2 CTAs of 8 warps per SM;
-// 2: up to 16 queries, one CTA of 16 warps per SM, since sixteen normalised queries take the
-// shared memory of both).
+// NT = number of 8-query tiles a pass scores (1: up to 8 queries, 2: up to 16).  One CTA of
+// four quads (16 warps) per SM: it holds the normalised queries once (two CTAs of two quads,
+// each with its own copy, were measured 3-15 % slower at every width, and rows wider than 6144
+// elements leave no room for two copies), leaves half as many lists to the final merge, and
+// its row share splits evenly over the quads.
 template <int E, int NT>
-__global__ void __launch_bounds__(kMmaThreads * NT, 2 / NT)
+__global__ void __launch_bounds__(kMmaThreads, 1)
 scan_mma_kernel(PoolView pv, const uint16_t* __restrict__ q_raw, int nq, int k,
                 const uint64_t* __restrict__ exclude_tag, u64* __restrict__ partial,
                 int32_t* __restrict__ q_valid, DeviceStats* stats, FusedAppend fa) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   constexpr int KK = 32 * E;
   constexpr int QP = kMmaQ * NT;             // queries per pass
-  constexpr int kQuads = 2 * NT;             // quads of four warps per CTA
+  constexpr int kQuads = kMmaThreads / 128;  // quads of four warps per CTA
   pdl_launch_dependents();
   pdl_wait();   // the rows appended before this query, and the query states themselves
   const int d = pv.d, n_chunks = d >> 3;
@@ -198,23 +217,20 @@ scan_mma_kernel(PoolView pv, const uint16_t* __restrict__ q_raw, int nq, int k,
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int g = lane >> 2, t = lane & 3;
-  // contiguous, balanced share of the rows for this CTA; the fa.n CTAs that first append a
-  // row of this step take 1/32 less than the others (as in the CUDA-core scan)
+  // contiguous, balanced share of the rows for this CTA
   const int64_t n = pv.n_rows;
-  const int64_t w_lo = 32ll * blockIdx.x - min((int)blockIdx.x, fa.n);
-  const int64_t w_hi = 32ll * (blockIdx.x + 1) - min((int)blockIdx.x + 1, fa.n);
-  const int64_t w_all = 32ll * gridDim.x - min((int)gridDim.x, fa.n);
-  const int r_lo = (int)((n * w_lo) / w_all);
-  const int r_hi = (int)((n * w_hi) / w_all);
+  const int r_lo = (int)((n * blockIdx.x) / gridDim.x);
+  const int r_hi = (int)((n * (blockIdx.x + 1)) / gridDim.x);
   const uint4* keys4 = reinterpret_cast<const uint4*>(pv.keys);
 
-  // the step's append (Section 4 "(i) Store", Eq. 1), one row per CTA; the 8-query form only
-  // (the block routine wants kNormThreads threads)
-  if (NT == 1 && (int)blockIdx.x < fa.n) {
-    const int r = blockIdx.x;
+  // the step's append (Section 4 "(i) Store", Eq. 1): in the 8-query form warps 8 to 15 have
+  // no query to prepare, so each of them in the first CTAs normalises one row meanwhile
+  // (row 8 b + w - 8 in CTA b), with the numbers of the block routine, and counts it in
+  if (NT == 1 && warp >= 8 && (int)blockIdx.x * 8 + (warp - 8) < fa.n) {
+    const int r = blockIdx.x * 8 + (warp - 8);
     const int64_t row = (int64_t)fa.row0 + r;
-    const int code = normalize_row<false>(fa.states + (size_t)r * d, fa.keys + row * d, d);
-    if (threadIdx.x == 0) {
+    const int code = normalize_row_warp(fa.states + (size_t)r * d, fa.keys + row * d, d, lane);
+    if (lane == 0) {
       fa.tok[row] = fa.tokens[r];
       fa.trace_id[row] = fa.trace;
       if (code != kRowOk) atomicAdd(&stats->degenerate_rows, 1ull);  // stored as a zero key
@@ -223,10 +239,10 @@ scan_mma_kernel(PoolView pv, const uint16_t* __restrict__ q_raw, int nq, int k,
         if (fa.set_tag) { fa.trace_tag[fa.trace] = fa.tag; fa.trace_gbase[fa.trace] = fa.gbase; }
       }
     }
-    __threadfence();                   // this thread's part of the row, before the count
-    __syncthreads();
-    if (threadIdx.x == 0) {
-      __threadfence();                 // cumulative: the whole CTA's row, as seen through the barrier
+    __threadfence();                   // this lane's part of the row, before the count
+    __syncwarp();
+    if (lane == 0) {
+      __threadfence();                 // cumulative: the whole warp's row, as seen through the barrier
       atomicAdd(fa.ready, 1ull);
     }
   }
@@ -237,7 +253,7 @@ scan_mma_kernel(PoolView pv, const uint16_t* __restrict__ q_raw, int nq, int k,
   for (int q0 = 0; q0 < nq; q0 += QP) {
     __syncthreads();
     // query preparation, one warp per query: qs[w] = bf16(q / ||q||), exactly as a key is stored
-    {
+    if (warp < QP) {
       uint16_t* dst = reinterpret_cast<uint16_t*>(qs + (size_t)warp * q_stride);
       if (q0 + warp < nq) {
         const int code = normalize_row_warp(q_raw + (size_t)(q0 + warp) * d, dst, d, lane);
@@ -466,7 +482,7 @@ scan_mma_kernel(PoolView pv, const uint16_t* __restrict__ q_raw, int nq, int k,
         scratch[((size_t)quad * QP + qi) * KK + r * 32 + lane] = top[l][r];
     }
     __syncthreads();
-    if (q0 + warp < nq) {
+    if (warp < QP && q0 + warp < nq) {
       u64 a[E];
 #pragma unroll
       for (int r = 0; r < E; ++r) a[r] = scratch[((size_t)0 * QP + warp) * KK + r * 32 + lane];
@@ -484,7 +500,7 @@ scan_mma_kernel(PoolView pv, const uint16_t* __restrict__ q_raw, int nq, int k,
 }
 
 size_t scan_mma_smem(int32_t d, int32_t kk, int32_t nt) {
-  const size_t qp = (size_t)kMmaQ * nt, quads = 2 * (size_t)nt;
+  const size_t qp = (size_t)kMmaQ * nt, quads = kMmaThreads / 128;
   return qp * ((size_t)d * 2 + kMmaPadBytes) + quads * qp * kk * sizeof(u64) +
          2 * quads * 4 * nt * 32 * sizeof(float4);
 }
@@ -501,6 +517,13 @@ bool scan_mma_supports(int32_t d, int32_t kk, size_t smem_limit) {
   return scan_mma_tiles(d, kk, 1, smem_limit) != 0;
 }
 
+// CTAs the scan launches: at least 64 rows each, at most one per SM
+int32_t scan_mma_grid(int64_t n_rows, int32_t num_sms, int32_t max_lists) {
+  const int64_t want = (n_rows + 63) / 64;
+  const int32_t grid = (int32_t)(want < 1 ? 1 : (want > num_sms ? num_sms : want));
+  return grid > max_lists ? max_lists : grid;
+}
+
 template <int E, int NT>
 static cudaError_t launch_mma_one(const PoolView& pv, const uint16_t* q_raw, int nq, int k,
                                   const uint64_t* ex, u64* partial, int32_t* q_valid,
@@ -510,8 +533,8 @@ static cudaError_t launch_mma_one(const PoolView& pv, const uint16_t* q_raw, int
   cudaError_t e = cudaFuncSetAttribute(scan_mma_kernel<E, NT>,
                                        cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
-  return launch_pdl(scan_mma_kernel<E, NT>, dim3(grid), dim3(kMmaThreads * NT), smem, st, pv, q_raw,
-                    nq, k, ex, partial, q_valid, stats, fa);
+  return launch_pdl(scan_mma_kernel<E, NT>, dim3(grid), dim3(kMmaThreads), smem, st, pv, q_raw, nq,
+                    k, ex, partial, q_valid, stats, fa);
 }
 
 cudaError_t launch_scan_mma(const PoolView& pv, const uint16_t* q_raw, int32_t nq, int32_t k,
@@ -521,15 +544,14 @@ cudaError_t launch_scan_mma(const PoolView& pv, const uint16_t* q_raw, int32_t n
                             const FusedAppend* fused, cudaStream_t st) {
   const int nt = scan_mma_tiles(pv.d, kk, nq, smem_limit);
   if (nt == 0) return cudaErrorInvalidValue;
-  int grid = scan_gemv_grid(pv.n_rows, num_sms, max_lists);      // two CTAs of 8 warps per SM
-  if (nt == 2) grid = (grid + 1) / 2;                             // one CTA of 16 warps per SM
+  const int grid = scan_mma_grid(pv.n_rows, num_sms, max_lists);
   *n_lists = grid;
   FusedAppend fa = {};
   if (fused) {
-    // every appending CTA must exist, and all CTAs be resident together (they are: at most
-    // two per SM are launched), because scanning warps wait for the appending ones; the
-    // 8-query form only
-    if (nt != 1 || fused->n > grid || fused->n > kFuseMaxRows) return cudaErrorInvalidValue;
+    // every appending warp must exist (eight per CTA), and all CTAs be resident together
+    // (they are: at most one per SM is launched), because scanning warps wait for the
+    // appending ones; the 8-query form only
+    if (nt != 1 || fused->n > 8 * grid || fused->n > kFuseMaxRows) return cudaErrorInvalidValue;
     fa = *fused;
   }
   if (kk == 32 && nt == 1)

@@ -190,3 +190,27 @@ def test_fused_step_appends_inside_the_scan_and_sees_the_new_rows_tags():
     keys, tok, tid = pool.read_rows()
     assert np.array_equal(keys, ora.keys) and np.array_equal(tok, ora.tokens)
     assert np.array_equal(tid, ora.trace_ids)
+
+
+@pytest.mark.parametrize("d", [6144, 8192])
+def test_wide_rows(d):
+    # the eight normalised queries of a CTA take 96 to 128 KB of shared memory here
+    w = W.C1.scaled(n_rows=1500, nq=7, d=d, k=8)
+    pool, ora = fill_both(w, spare_rows=64)
+    q, _ = w.queries("cuda")
+    for theta in (0.8, -2.0):
+        pr = fixed(8, 8, theta=theta, path=B.PATH_MMA)
+        check_query(pool.query(q, pr), ora, W.to_bits(q), pr)
+    g = torch.Generator(device="cuda").manual_seed(d)
+    st = torch.randn(8, d, generator=g, device="cuda").to(torch.bfloat16)
+    tk = torch.randint(0, 100, (8,), generator=g, device="cuda", dtype=torch.int32)
+    qs = q.clone()
+    qs[2] = st[6]
+    pr = fixed(8, 8, theta=-2.0)
+    l0 = pool.launch_count
+    out = pool.step(st, tk, qs, pr, tag=777)
+    assert pool.launch_count - l0 == 2
+    ora.append(W.to_bits(st), tk.cpu().numpy(), tag=777)
+    check_query(out, ora, W.to_bits(qs), pr)
+    assert int(out.idx[2, 0]) == len(pool) - 2
+    assert pool.stats()["stalled"] == 0

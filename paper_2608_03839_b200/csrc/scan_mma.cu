@@ -31,7 +31,8 @@ constexpr int kMmaThreads = 512;
 constexpr int kMmaWarps = kMmaThreads / 32;
 constexpr int kMmaQ = 8;          // queries per pass = the N of the instruction
 constexpr int kMmaRows = 16;      // rows per warp step = the M of the instruction
-constexpr int kMmaDepth = 4;      // 32-element blocks in flight per lane and row
+constexpr int kMmaDepth1 = 4;     // 32-element blocks per lane, row and step: 8-query form
+constexpr int kMmaDepth2 = 2;     // 16-query form (its accumulators and lists need the registers)
 constexpr int kMmaBatchInsert = 5; // candidates of a group and query from which they are merged in as a sorted vector
 constexpr int kMmaPadBytes = 64;  // per query row in shared memory: keeps the 16-byte loads of
                                   // a quarter warp (two queries x four offsets) on distinct banks
@@ -204,6 +205,7 @@ scan_mma_kernel(PoolView pv, const uint16_t* __restrict__ q_raw, int nq, int k,
   constexpr int KK = 32 * E;
   constexpr int QP = kMmaQ * NT;             // queries per pass
   constexpr int kQuads = kMmaThreads / 128;  // quads of four warps per CTA
+  constexpr int kMmaDepth = NT == 1 ? kMmaDepth1 : kMmaDepth2;
   pdl_launch_dependents();
   pdl_wait();   // the rows appended before this query, and the query states themselves
   const int d = pv.d, n_chunks = d >> 3;

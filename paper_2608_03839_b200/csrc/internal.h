@@ -145,13 +145,15 @@ inline int32_t scan_gemv_grid(int64_t n_rows, int32_t num_sms, int32_t max_lists
 // a2+a3 (warp-level tensor cores, small batches): the same contract as the CUDA-core scan,
 // eight or sixteen queries per pass over the keys.  Needs d % 128 == 0, kk <= 64 and room for the eight
 // normalised queries in shared memory.
-bool scan_mma_supports(int32_t d, int32_t kk, size_t smem_limit);
+// (8-bit pools: codes and scales given, d % 256 == 0, f16 MMAs, no appended rows.)
+bool scan_mma_supports(int32_t d, int32_t kk, size_t smem_limit, bool fp8);
 // 8-query tiles per pass the kernel would use for nq queries (1 or 2; 0 = unsupported; with
-// one tile it can append a step's rows itself), and the CTAs it launches
-int scan_mma_tiles(int32_t d, int32_t kk, int32_t nq, size_t smem_limit);
+// one tile and 16-bit keys it can append a step's rows itself), and the CTAs it launches
+int scan_mma_tiles(int32_t d, int32_t kk, int32_t nq, size_t smem_limit, bool fp8);
 int32_t scan_mma_grid(int64_t n_rows, int32_t num_sms, int32_t max_lists);
-cudaError_t launch_scan_mma(const PoolView& pv, const uint16_t* q_raw, int32_t nq, int32_t k,
-                            int32_t kk, const uint64_t* exclude_tag, unsigned long long* partial,
+cudaError_t launch_scan_mma(const PoolView& pv, const uint8_t* codes, const float* scales,
+                            const uint16_t* q_raw, int32_t nq, int32_t k, int32_t kk,
+                            const uint64_t* exclude_tag, unsigned long long* partial,
                             int32_t* q_valid, DeviceStats* stats, int32_t max_lists,
                             int32_t num_sms, size_t smem_limit, int32_t* n_lists,
                             const FusedAppend* fused, cudaStream_t st);

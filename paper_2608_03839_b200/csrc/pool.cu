@@ -438,11 +438,17 @@ static int resolve_path(const oilbird_pool* p, const oilbird_query_params* pr, i
   // small batches on pools of the paper's size to mma.sync
   if (pr->path != OILBIRD_PATH_AUTO) return pr->path;
   if (nq <= 2) return OILBIRD_PATH_GEMV;
+  if (p->r.e4m3) {
+    // 8-bit pools have no tcgen05 scan: the warp-level tensor scan scores 8 or 16 queries
+    // per pass over the codes, the CUDA-core scan two
+    return scan_mma_tiles(p->r.d, list_len(pr->k), nq, p->smem_limit, true) ? OILBIRD_PATH_MMA
+                                                                             : OILBIRD_PATH_GEMV;
+  }
   const int64_t key_bytes = p->n_rows * (int64_t)p->r.d * 2;
   const int64_t mma_max = nq > 8 ? kMma16MaxKeyBytes : kMmaMaxKeyBytes;
-  if (nq <= 16 && !p->r.e4m3 && key_bytes <= mma_max) {
+  if (nq <= 16 && key_bytes <= mma_max) {
     // up to 8 queries in one pass of 8; 9 to 16 only where 16 fit in one pass
-    const int nt = scan_mma_tiles(p->r.d, list_len(pr->k), nq, p->smem_limit);
+    const int nt = scan_mma_tiles(p->r.d, list_len(pr->k), nq, p->smem_limit, false);
     if (nt == 2 || (nt == 1 && nq <= 8)) return OILBIRD_PATH_MMA;
   }
   return OILBIRD_PATH_TENSOR;
@@ -463,11 +469,9 @@ static int query_impl(oilbird_pool_t* p, const void* q, int32_t nq, const oilbir
   PoolView pv = view_of(p);
   cudaError_t e;
 
-  const int path = p->r.e4m3 && pr->path == OILBIRD_PATH_AUTO ? OILBIRD_PATH_GEMV
-                                                              : resolve_path(p, pr, nq);
-  if ((path == OILBIRD_PATH_TENSOR || path == OILBIRD_PATH_MMA) && p->r.e4m3)
-    return OILBIRD_EINVAL;                                               // 16-bit pools only
-  if (path == OILBIRD_PATH_MMA && !scan_mma_supports(p->r.d, kk, p->smem_limit))
+  const int path = resolve_path(p, pr, nq);
+  if (path == OILBIRD_PATH_TENSOR && p->r.e4m3) return OILBIRD_EINVAL;   // 16-bit pools only
+  if (path == OILBIRD_PATH_MMA && !scan_mma_supports(p->r.d, kk, p->smem_limit, p->r.e4m3))
     return OILBIRD_EINVAL;
   if (path == OILBIRD_PATH_TENSOR && !p->tc) {
     snprintf(g_cuda_err, sizeof g_cuda_err, "tensor-core scan unavailable on this device");
@@ -492,7 +496,13 @@ static int query_impl(oilbird_pool_t* p, const void* q, int32_t nq, const oilbir
       e0 = p->ev[p->ev_used]; e1 = p->ev[p->ev_used + 1];
       CU(cudaEventRecord(e0, st));
     }
-    if (p->r.e4m3) {
+    if (p->r.e4m3 && path == OILBIRD_PATH_MMA) {
+      e = launch_scan_mma(pv, p->codes, p->scales, (const uint16_t*)q, nq, pr->k, kk,
+                          pr->exclude_tag, p->partial, p->q_valid, p->stats, p->r.max_lists,
+                          p->num_sms, p->smem_limit, &n_lists, nullptr, st);
+      if (e != cudaSuccess) return cuda_fail(e, "8-bit warp-level tensor scan kernel launch");
+      p->launches += 1;
+    } else if (p->r.e4m3) {
       e = launch_scan_gemv_e4m3(p->codes, p->scales, pv, (const uint16_t*)q, nq, pr->k, kk,
                                 pr->exclude_tag, p->partial, p->q_valid, p->stats, p->r.max_lists,
                                 p->num_sms, &n_lists, fused, st);
@@ -504,7 +514,7 @@ static int query_impl(oilbird_pool_t* p, const void* q, int32_t nq, const oilbir
       if (e != cudaSuccess) return cuda_fail(e, "scan kernel launch");
       p->launches += 1;
     } else if (path == OILBIRD_PATH_MMA) {
-      e = launch_scan_mma(pv, (const uint16_t*)q, nq, pr->k, kk, pr->exclude_tag, p->partial,
+      e = launch_scan_mma(pv, nullptr, nullptr, (const uint16_t*)q, nq, pr->k, kk, pr->exclude_tag, p->partial,
                           p->q_valid, p->stats, p->r.max_lists, p->num_sms, p->smem_limit,
                           &n_lists, fused, st);
       if (e != cudaSuccess) return cuda_fail(e, "warp-level tensor scan kernel launch");
@@ -553,12 +563,11 @@ static int step_impl(oilbird_pool_t* p, const void* states, const int32_t* token
   const int64_t rows_after = p->n_rows + n;
   // (8-bit pools always use the CUDA-core scan; its passes beyond the first two queries
   // would find the rows in place, but keep to the single-request case there too)
-  const int path = p->r.e4m3 ? OILBIRD_PATH_AUTO : resolve_path(p, pr, nq);
-  const bool gemv = p->r.e4m3 ? (nq <= 2 && pr->path != OILBIRD_PATH_TENSOR)
-                              : path == OILBIRD_PATH_GEMV;
-  // the warp-level tensor scan appends the step's rows itself in its 8-query form
-  const bool mma8 = path == OILBIRD_PATH_MMA &&
-                    scan_mma_tiles(p->r.d, list_len(pr->k), nq, p->smem_limit) == 1;
+  const int path = resolve_path(p, pr, nq);
+  const bool gemv = p->r.e4m3 ? (nq <= 2 && path == OILBIRD_PATH_GEMV) : path == OILBIRD_PATH_GEMV;
+  // the warp-level tensor scan appends the step's rows itself in its 8-query form (16-bit keys)
+  const bool mma8 = !p->r.e4m3 && path == OILBIRD_PATH_MMA &&
+                    scan_mma_tiles(p->r.d, list_len(pr->k), nq, p->smem_limit, false) == 1;
   const bool fuse =
       n >= 1 && n <= kFuseMaxRows &&
       ((gemv && scan_gemv_grid(rows_after, p->num_sms, p->r.max_lists) >= n) ||

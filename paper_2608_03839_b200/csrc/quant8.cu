@@ -11,9 +11,10 @@
 // the scan, which is bound by the key stream, moves half the bytes.
 //
 // Everything after the scan (merge, firing rule, depth, gather) is format-independent and
-// shared with the 16-bit path.  The tensor-core scan is not offered for 8-bit pools (its
-// query operand would have to be quantised to 8 bits too); batches run the CUDA-core scan
-// two queries per pass.  As in the 16-bit scan, the rows of a serving step can be appended
+// shared with the 16-bit path.  The tcgen05 scan is not offered for 8-bit pools (its query
+// operand would have to be quantised to 8 bits too); batches of three queries and more go
+// to the warp-level tensor scan (scan_mma.cu, codes as f16) where the width allows, else
+// they run here two queries per pass.  As in the 16-bit scan, the rows of a serving step can be appended
 // by the scan's first CTAs themselves (see FusedAppend).
 #include <cuda_fp16.h>
 

@@ -19,8 +19,13 @@
 //
 // Each warp keeps one descending register list per query (Eq. 2); a group's 128 scores are
 // tested against the lists' k-th entries and the few that pass are inserted one by one.  At
-// the end warp w merges query w's eight lists; what leaves the CTA is one list per query,
-// as in the other scans.
+// the end warp w merges query w's lists; what leaves the CTA is one list per query, as in
+// the other scans.
+//
+// Pools with 8-bit keys (E4M3 codes + one scale per row) run the same kernel with f16
+// operands: a code is an f16 number exactly, the query is held as f16 scaled by 2^14.
+#include <cuda_fp16.h>
+
 #include "common.cuh"
 #include "internal.h"
 #include "normalize.cuh"
@@ -59,6 +64,25 @@ __device__ __forceinline__ uint4 ld_key16(const uint4* p, bool fresh) {
 __device__ __forceinline__ void quad_bar(int id) {
   asm volatile("bar.sync %0, 128;" ::"r"(id) : "memory");
 }
+
+// the same with f16 operands: pools with 8-bit keys (an E4M3 code is an f16 number exactly)
+__device__ __forceinline__ void mma_f16(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2,
+                                        uint32_t a3, uint32_t b0, uint32_t b1) {
+  asm(
+      "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, "
+      "{%8,%9}, {%0,%1,%2,%3};"
+      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+// two E4M3 codes (low 16 bits) -> f16x2, first code in the low half
+__device__ __forceinline__ uint32_t e4m3x2_to_f16x2(uint32_t two_codes) {
+  uint32_t h2;
+  asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(h2) : "h"((unsigned short)two_codes));
+  return h2;
+}
+// queries of an 8-bit pool are held as f16 scaled by 2^14 (|q| <= 1 after normalisation; the
+// scale keeps their small elements out of f16's subnormal range); the score is scaled back
+constexpr float kFp8QueryScale = 16384.f;
 
 // normalize_row done by one warp, with the numbers accumulated in the order of the block
 // routine (lane l plays threads l, l + 32, ... l + 224 of a 256-thread block with one
@@ -196,9 +220,12 @@ __device__ __forceinline__ int normalize_row_warp(const uint16_t* __restrict__ s
 // each with its own copy, were measured 3-15 % slower at every width, and rows wider than 6144
 // elements leave no room for two copies), leaves half as many lists to the final merge, and
 // its row share splits evenly over the quads.
-template <int E, int NT>
+// kFp8: the pool holds E4M3 codes + one fp32 scale per row (16 elements per 16-byte load, four
+// f16 MMAs per pair of loads; score = scale * sum, as in the CUDA-core scan of such pools).
+template <int E, int NT, bool kFp8>
 __global__ void __launch_bounds__(kMmaThreads, 1)
-scan_mma_kernel(PoolView pv, const uint16_t* __restrict__ q_raw, int nq, int k,
+scan_mma_kernel(PoolView pv, const uint8_t* __restrict__ codes, const float* __restrict__ scales,
+                const uint16_t* __restrict__ q_raw, int nq, int k,
                 const uint64_t* __restrict__ exclude_tag, u64* __restrict__ partial,
                 int32_t* __restrict__ q_valid, DeviceStats* stats, FusedAppend fa) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
@@ -209,6 +236,7 @@ scan_mma_kernel(PoolView pv, const uint16_t* __restrict__ q_raw, int nq, int k,
   pdl_launch_dependents();
   pdl_wait();   // the rows appended before this query, and the query states themselves
   const int d = pv.d, n_chunks = d >> 3;
+  const int k_units = kFp8 ? d >> 4 : d >> 3;                            // 16-byte units of a key row
   const int q_stride = n_chunks + kMmaPadBytes / 16;                     // in 16-byte units
   uint4* qs = reinterpret_cast<uint4*>(smem_raw);                        // [QP][q_stride]
   u64* scratch = reinterpret_cast<u64*>(smem_raw + (size_t)QP * q_stride * 16);   // [quads][QP][KK]
@@ -223,12 +251,13 @@ scan_mma_kernel(PoolView pv, const uint16_t* __restrict__ q_raw, int nq, int k,
   const int64_t n = pv.n_rows;
   const int r_lo = (int)((n * blockIdx.x) / gridDim.x);
   const int r_hi = (int)((n * (blockIdx.x + 1)) / gridDim.x);
-  const uint4* keys4 = reinterpret_cast<const uint4*>(pv.keys);
+  const uint4* keys4 = kFp8 ? reinterpret_cast<const uint4*>(codes)
+                            : reinterpret_cast<const uint4*>(pv.keys);
 
   // the step's append (Section 4 "(i) Store", Eq. 1): in the 8-query form warps 8 to 15 have
   // no query to prepare, so each of them in the first CTAs normalises one row meanwhile
   // (row 8 b + w - 8 in CTA b), with the numbers of the block routine, and counts it in
-  if (NT == 1 && warp >= 8 && (int)blockIdx.x * 8 + (warp - 8) < fa.n) {
+  if (!kFp8 && NT == 1 && warp >= 8 && (int)blockIdx.x * 8 + (warp - 8) < fa.n) {
     const int r = blockIdx.x * 8 + (warp - 8);
     const int64_t row = (int64_t)fa.row0 + r;
     const int code = normalize_row_warp(fa.states + (size_t)r * d, fa.keys + row * d, d, lane);
@@ -259,6 +288,16 @@ scan_mma_kernel(PoolView pv, const uint16_t* __restrict__ q_raw, int nq, int k,
       uint16_t* dst = reinterpret_cast<uint16_t*>(qs + (size_t)warp * q_stride);
       if (q0 + warp < nq) {
         const int code = normalize_row_warp(q_raw + (size_t)(q0 + warp) * d, dst, d, lane);
+        if (kFp8) {
+          // the normalised bf16 query, as f16 scaled by 2^14 (exact but for elements below 2^-38)
+          __syncwarp();
+          uint32_t* w32 = reinterpret_cast<uint32_t*>(dst);
+          for (int i = lane; i < d / 2; i += 32) {
+            const uint32_t w = w32[i];
+            const __half2 h = __floats2half2_rn(bf16_lo(w) * kFp8QueryScale, bf16_hi(w) * kFp8QueryScale);
+            w32[i] = *reinterpret_cast<const uint32_t*>(&h);
+          }
+        }
         if (blockIdx.x == 0 && lane == 0) {
           q_valid[q0 + warp] = code == kRowNonFinite ? 0 : 1;   // NaN/Inf: no neighbours
           if (code == kRowNonFinite) atomicAdd(&stats->nonfinite_queries, 1ull);
@@ -280,8 +319,10 @@ scan_mma_kernel(PoolView pv, const uint16_t* __restrict__ q_raw, int nq, int k,
     // 2 kq + 1 of every tile (the scores its lanes with t == kq hold), over all rows of the
     // quad, so a list sees four times the rows a per-warp list would and far fewer rows pass.
     const int quad = warp >> 2, kq = warp & 3;
-    const int cq = n_chunks >> 2;                                   // 16-byte units per quarter
-    const uint4* qrow = qs + (size_t)g * q_stride + kq * 4 + t;     // tile i: + 8 i rows
+    const int cq = k_units >> 2;                                    // 16-byte key units per quarter
+    // query fragments: the 16 bytes (8 elements) that go with a 16-byte key unit, two of them
+    // for a unit of 16 codes; tile i: + 8 i rows
+    const uint4* qrow = qs + (size_t)g * q_stride + (kFp8 ? 2 : 1) * (kq * 4 + t);
     float4* part = s_part + quad * 4 * NT * 32;                     // [quarter][tile][lane]
     // descending lists of this warp's 2 NT queries; kth = the k-th entry (0 while not full)
     u64 top[2 * NT][E];
@@ -298,7 +339,7 @@ scan_mma_kernel(PoolView pv, const uint16_t* __restrict__ q_raw, int nq, int k,
     // key pointers of this lane's two rows of the group starting at row rbx
     auto row_ptr = [&](int rbx, int second) {
       const int row = rbx + g + 8 * second;
-      return keys4 + (size_t)(row < r_hi ? row : r_hi - 1) * n_chunks + kq * 4 + t;
+      return keys4 + (size_t)(row < r_hi ? row : r_hi - 1) * k_units + kq * 4 + t;
     };
     // The key stream of a warp is one sequence of steps of kMmaDepth blocks of 32 elements
     // over all its groups: the loads of the next step (the first of the next group, at a
@@ -363,10 +404,25 @@ scan_mma_kernel(PoolView pv, const uint16_t* __restrict__ q_raw, int nq, int k,
           for (int u = 0; u < kMmaDepth; ++u) {
 #pragma unroll
             for (int i = 0; i < NT; ++i) {
-              const uint4 qv = c + 4 * u < cq ? qrow[(size_t)8 * i * q_stride + 4 * (c + 4 * u)]
-                                              : make_uint4(0, 0, 0, 0);
-              mma_bf16(c0[i], ka[u].x, kb[u].x, ka[u].y, kb[u].y, qv.x, qv.y);
-              mma_bf16(c1[i], ka[u].z, kb[u].z, ka[u].w, kb[u].w, qv.z, qv.w);
+              if (kFp8) {
+                const bool in = c + 4 * u < cq;
+                const uint4* qp = qrow + (size_t)8 * i * q_stride + 8 * (c + 4 * u);
+                const uint4 ql = in ? qp[0] : make_uint4(0, 0, 0, 0);
+                const uint4 qh = in ? qp[1] : make_uint4(0, 0, 0, 0);
+                mma_f16(c0[i], e4m3x2_to_f16x2(ka[u].x), e4m3x2_to_f16x2(kb[u].x),
+                        e4m3x2_to_f16x2(ka[u].x >> 16), e4m3x2_to_f16x2(kb[u].x >> 16), ql.x, ql.y);
+                mma_f16(c1[i], e4m3x2_to_f16x2(ka[u].y), e4m3x2_to_f16x2(kb[u].y),
+                        e4m3x2_to_f16x2(ka[u].y >> 16), e4m3x2_to_f16x2(kb[u].y >> 16), ql.z, ql.w);
+                mma_f16(c0[i], e4m3x2_to_f16x2(ka[u].z), e4m3x2_to_f16x2(kb[u].z),
+                        e4m3x2_to_f16x2(ka[u].z >> 16), e4m3x2_to_f16x2(kb[u].z >> 16), qh.x, qh.y);
+                mma_f16(c1[i], e4m3x2_to_f16x2(ka[u].w), e4m3x2_to_f16x2(kb[u].w),
+                        e4m3x2_to_f16x2(ka[u].w >> 16), e4m3x2_to_f16x2(kb[u].w >> 16), qh.z, qh.w);
+              } else {
+                const uint4 qv = c + 4 * u < cq ? qrow[(size_t)8 * i * q_stride + 4 * (c + 4 * u)]
+                                                : make_uint4(0, 0, 0, 0);
+                mma_bf16(c0[i], ka[u].x, kb[u].x, ka[u].y, kb[u].y, qv.x, qv.y);
+                mma_bf16(c1[i], ka[u].z, kb[u].z, ka[u].w, kb[u].w, qv.z, qv.w);
+              }
             }
           }
 #pragma unroll
@@ -397,14 +453,21 @@ scan_mma_kernel(PoolView pv, const uint16_t* __restrict__ q_raw, int nq, int k,
         if (row1 < r_hi)
           tag1 = cur_fresh ? __ldcg(&pv.trace_tag[__ldcg(&pv.trace_id[row1])]) : pv.trace_tag[pv.trace_id[row1]];
       }
+      // 8-bit pools: the rows' scales (and the queries' 2^14 taken back)
+      float sc0 = 1.f, sc1 = 1.f;
+      if (kFp8 && own) {
+        sc0 = row0 < r_hi ? scales[row0] * (1.f / kFp8QueryScale) : 0.f;
+        sc1 = row1 < r_hi ? scales[row1] * (1.f / kFp8QueryScale) : 0.f;
+      }
       u64 key[2 * NT][2];                    // [list][row0 / row1]
       bool any = false;
 #pragma unroll
       for (int i = 0; i < NT; ++i) {
         const float4 p0 = pbuf[(0 * NT + i) * 32 + lane], p1 = pbuf[(1 * NT + i) * 32 + lane],
                      p2 = pbuf[(2 * NT + i) * 32 + lane], p3 = pbuf[(3 * NT + i) * 32 + lane];
-        const float sx = ((p0.x + p1.x) + p2.x) + p3.x, sy = ((p0.y + p1.y) + p2.y) + p3.y;
-        const float sz = ((p0.z + p1.z) + p2.z) + p3.z, sw = ((p0.w + p1.w) + p2.w) + p3.w;
+        float sx = ((p0.x + p1.x) + p2.x) + p3.x, sy = ((p0.y + p1.y) + p2.y) + p3.y;
+        float sz = ((p0.z + p1.z) + p2.z) + p3.z, sw = ((p0.w + p1.w) + p2.w) + p3.w;
+        if (kFp8) { sx *= sc0; sy *= sc0; sz *= sc1; sw *= sc1; }
         const int la = 2 * i, lb = 2 * i + 1;
         const int qa = 8 * i + 2 * kq;                     // queries of lists la, lb within the pass
         const bool live_a = own && q0 + qa < nq, live_b = own && q0 + qa + 1 < nq;
@@ -508,15 +571,16 @@ size_t scan_mma_smem(int32_t d, int32_t kk, int32_t nt) {
 }
 
 // 8-query tiles per pass (1 or 2) for a call of nq queries, or 0 if the kernel cannot take
-// the pool's width or the list length
-int scan_mma_tiles(int32_t d, int32_t kk, int32_t nq, size_t smem_limit) {
-  if (d % 128 != 0 || kk > 64) return 0;
+// the pool's width (a quad's warps take whole blocks of 32 elements, 64 codes for 8-bit
+// keys) or the list length
+int scan_mma_tiles(int32_t d, int32_t kk, int32_t nq, size_t smem_limit, bool fp8) {
+  if (d % (fp8 ? 256 : 128) != 0 || kk > 64) return 0;
   if (nq > kMmaQ && scan_mma_smem(d, kk, 2) <= smem_limit) return 2;
   return scan_mma_smem(d, kk, 1) <= smem_limit ? 1 : 0;
 }
 
-bool scan_mma_supports(int32_t d, int32_t kk, size_t smem_limit) {
-  return scan_mma_tiles(d, kk, 1, smem_limit) != 0;
+bool scan_mma_supports(int32_t d, int32_t kk, size_t smem_limit, bool fp8) {
+  return scan_mma_tiles(d, kk, 1, smem_limit, fp8) != 0;
 }
 
 // CTAs the scan launches: at least 64 rows each, at most one per SM
@@ -526,25 +590,27 @@ int32_t scan_mma_grid(int64_t n_rows, int32_t num_sms, int32_t max_lists) {
   return grid > max_lists ? max_lists : grid;
 }
 
-template <int E, int NT>
-static cudaError_t launch_mma_one(const PoolView& pv, const uint16_t* q_raw, int nq, int k,
-                                  const uint64_t* ex, u64* partial, int32_t* q_valid,
-                                  DeviceStats* stats, int grid, const FusedAppend& fa,
-                                  cudaStream_t st) {
+template <int E, int NT, bool kFp8>
+static cudaError_t launch_mma_one(const PoolView& pv, const uint8_t* codes, const float* scales,
+                                  const uint16_t* q_raw, int nq, int k, const uint64_t* ex,
+                                  u64* partial, int32_t* q_valid, DeviceStats* stats, int grid,
+                                  const FusedAppend& fa, cudaStream_t st) {
   const size_t smem = scan_mma_smem(pv.d, 32 * E, NT);
-  cudaError_t e = cudaFuncSetAttribute(scan_mma_kernel<E, NT>,
+  cudaError_t e = cudaFuncSetAttribute(scan_mma_kernel<E, NT, kFp8>,
                                        cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
-  return launch_pdl(scan_mma_kernel<E, NT>, dim3(grid), dim3(kMmaThreads), smem, st, pv, q_raw, nq,
-                    k, ex, partial, q_valid, stats, fa);
+  return launch_pdl(scan_mma_kernel<E, NT, kFp8>, dim3(grid), dim3(kMmaThreads), smem, st, pv, codes,
+                    scales, q_raw, nq, k, ex, partial, q_valid, stats, fa);
 }
 
-cudaError_t launch_scan_mma(const PoolView& pv, const uint16_t* q_raw, int32_t nq, int32_t k,
-                            int32_t kk, const uint64_t* exclude_tag, u64* partial,
-                            int32_t* q_valid, DeviceStats* stats, int32_t max_lists,
-                            int32_t num_sms, size_t smem_limit, int32_t* n_lists,
-                            const FusedAppend* fused, cudaStream_t st) {
-  const int nt = scan_mma_tiles(pv.d, kk, nq, smem_limit);
+cudaError_t launch_scan_mma(const PoolView& pv, const uint8_t* codes, const float* scales,
+                            const uint16_t* q_raw, int32_t nq, int32_t k, int32_t kk,
+                            const uint64_t* exclude_tag, u64* partial, int32_t* q_valid,
+                            DeviceStats* stats, int32_t max_lists, int32_t num_sms,
+                            size_t smem_limit, int32_t* n_lists, const FusedAppend* fused,
+                            cudaStream_t st) {
+  const bool fp8 = codes != nullptr;
+  const int nt = scan_mma_tiles(pv.d, kk, nq, smem_limit, fp8);
   if (nt == 0) return cudaErrorInvalidValue;
   const int grid = scan_mma_grid(pv.n_rows, num_sms, max_lists);
   *n_lists = grid;
@@ -552,17 +618,24 @@ cudaError_t launch_scan_mma(const PoolView& pv, const uint16_t* q_raw, int32_t n
   if (fused) {
     // every appending warp must exist (eight per CTA), and all CTAs be resident together
     // (they are: at most one per SM is launched), because scanning warps wait for the
-    // appending ones; the 8-query form only
-    if (nt != 1 || fused->n > 8 * grid || fused->n > kFuseMaxRows) return cudaErrorInvalidValue;
+    // appending ones; the 8-query form on 16-bit keys only
+    if (fp8 || nt != 1 || fused->n > 8 * grid || fused->n > kFuseMaxRows) return cudaErrorInvalidValue;
     fa = *fused;
   }
-  if (kk == 32 && nt == 1)
-    return launch_mma_one<1, 1>(pv, q_raw, nq, k, exclude_tag, partial, q_valid, stats, grid, fa, st);
-  if (kk == 64 && nt == 1)
-    return launch_mma_one<2, 1>(pv, q_raw, nq, k, exclude_tag, partial, q_valid, stats, grid, fa, st);
-  if (kk == 32)
-    return launch_mma_one<1, 2>(pv, q_raw, nq, k, exclude_tag, partial, q_valid, stats, grid, fa, st);
-  return launch_mma_one<2, 2>(pv, q_raw, nq, k, exclude_tag, partial, q_valid, stats, grid, fa, st);
+#define OILBIRD_MMA_CASE(E_, NT_, F_)                                                          \
+  if (kk == 32 * E_ && nt == NT_ && fp8 == F_)                                                 \
+    return launch_mma_one<E_, NT_, F_>(pv, codes, scales, q_raw, nq, k, exclude_tag, partial,  \
+                                       q_valid, stats, grid, fa, st);
+  OILBIRD_MMA_CASE(1, 1, false)
+  OILBIRD_MMA_CASE(2, 1, false)
+  OILBIRD_MMA_CASE(1, 2, false)
+  OILBIRD_MMA_CASE(2, 2, false)
+  OILBIRD_MMA_CASE(1, 1, true)
+  OILBIRD_MMA_CASE(2, 1, true)
+  OILBIRD_MMA_CASE(1, 2, true)
+  OILBIRD_MMA_CASE(2, 2, true)
+#undef OILBIRD_MMA_CASE
+  return cudaErrorInvalidValue;
 }
 
 }  // namespace oilbird

@@ -138,11 +138,12 @@ def test_auto_path_uses_it_for_small_batches_only():
     with pytest.raises(B.OilbirdError) as e:
         odd.query(torch.randn(4, 200, device="cuda").to(torch.bfloat16), fixed(8, 8, path=B.PATH_MMA))
     assert e.value.code == B.EINVAL
-    q8 = B.Pool(256, 64, max_nq=8, key_format="e4m3")
-    q8.append(torch.randn(64, 256, device="cuda").to(torch.bfloat16),
+    # 8-bit pools take it from widths that are multiples of 256 (tests/test_gpu_q8.py)
+    q8 = B.Pool(128, 64, max_nq=8, key_format="e4m3")
+    q8.append(torch.randn(64, 128, device="cuda").to(torch.bfloat16),
               torch.zeros(64, dtype=torch.int32, device="cuda"), tag=1)
     with pytest.raises(B.OilbirdError):
-        q8.query(torch.randn(4, 256, device="cuda").to(torch.bfloat16), fixed(8, 8, path=B.PATH_MMA))
+        q8.query(torch.randn(4, 128, device="cuda").to(torch.bfloat16), fixed(8, 8, path=B.PATH_MMA))
 
 
 def test_paper_scale_pool_batch_of_eight_full_width():

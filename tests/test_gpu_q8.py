@@ -216,3 +216,76 @@ def test_fused_steps_on_8bit_pool():
     q = chunks[3][0][:1].contiguous()
     check_query(pool.query(q, pr), ora, W.to_bits(q), pr)
     assert pool.stats()["stalled"] == 0
+
+
+# ------------------------------------------- warp-level tensor scan on 8-bit pools ----
+
+@pytest.mark.parametrize("d", [256, 1024, 4096])
+def test_mma_scan_closed_form_pool_scores_are_exact(d):
+    # +-1 rows (codes +-448) and +-1 queries: f16 products and their sums are exact, so the
+    # batch scan must return the oracle's scores, order and ties bit for bit
+    rng = np.random.default_rng(d)
+    n = 600
+    rows = rng.choice([-1.0, 1.0], size=(n, d)).astype(np.float32)
+    q = rng.choice([-1.0, 1.0], size=(5, d)).astype(np.float32)
+    rows[5] = q[0]; rows[300] = q[0]; rows[599] = q[0]
+    rows[17] = -q[1]
+    pool = B.Pool(d, n, max_nq=8, key_format="e4m3")
+    ora = OraclePool(d, "e4m3")
+    rb = oracle.f32_to_bf16_bits(rows)
+    tok = np.arange(n, dtype=np.int32)
+    pool.append(bits_to_dev(rb), torch.from_numpy(tok).cuda(), tag=1)
+    ora.append(rb, tok, tag=1)
+    qb = oracle.f32_to_bf16_bits(q)
+    pr = fixed(8, 2, theta=-2.0, path=B.PATH_MMA)
+    l0 = pool.launch_count
+    out = pool.query(bits_to_dev(qb), pr).cpu()
+    assert pool.launch_count - l0 == 2
+    ref = ora.query(qb, oracle.QueryParams(k=8, theta=-2.0, depth_mode=oracle.DEPTH_FIXED, cont_len=2))
+    assert out.idx.numpy().tolist() == ref.idx.tolist()
+    assert np.array_equal(out.score.numpy(), ref.score)
+    assert out.idx[0, :3].tolist() == [5, 300, 599]
+
+
+@pytest.mark.parametrize("nq,k", [(1, 8), (3, 8), (8, 16), (8, 40), (11, 8), (16, 64), (19, 5)])
+def test_mma_scan_matches_oracle_and_the_cuda_core_scan(nq, k):
+    w = W.C1.scaled(n_rows=6000, nq=nq, d=512)
+    pool, ora = fill_both(w, key_format="e4m3", max_k=k, max_nq=32)
+    q, _ = w.queries("cuda", nq=nq)
+    for theta in (0.8, -2.0):
+        pr = fixed(k, 8, theta=theta, path=B.PATH_MMA)
+        out = pool.query(q, pr)
+        check_query(out, ora, W.to_bits(q), pr)
+        ref = pool.query(q, fixed(k, 8, theta=theta, path=B.PATH_GEMV))
+        assert torch.allclose(out.score, ref.score, atol=2e-5, rtol=0)
+    # the automatic choice for three queries and more is this scan: one launch (its passes of
+    # 8 or 16 queries run inside the kernel) plus the merge
+    if nq >= 3:
+        l0 = pool.launch_count
+        pool.query(q, fixed(k, 8))
+        assert pool.launch_count - l0 == 2
+    assert pool.stats()["stalled"] == 0
+
+
+def test_mma_scan_wide_rows_exclusion_and_ragged_sizes():
+    w = W.C2.scaled(n_rows=3000, nq=6)
+    pool, ora = fill_both(w, key_format="e4m3", spare_rows=64)
+    q, _ = w.queries("cuda", nq=6)
+    tags = [t for _, _, t in w.traces("cpu")][:2]
+    ex = torch.tensor([tags[0], 0, tags[1], 0, 0, 12345], dtype=torch.int64, device="cuda")
+    pr = fixed(16, 16, theta=-2.0)
+    pr.exclude_tag = ex
+    check_query(pool.query(q, pr), ora, W.to_bits(q), pr, exclude=ex.cpu().numpy().astype(np.uint64))
+    for n_rows in (1, 15, 17, 129, 1000):
+        ws = W.C1.scaled(nq=4, d=256)
+        pool2, ora2 = fill_both(ws, n_rows=n_rows, key_format="e4m3")
+        q2, _ = ws.queries("cuda")
+        pr2 = fixed(ws.k, ws.cont_len, theta=-2.0)
+        check_query(pool2.query(q2, pr2), ora2, W.to_bits(q2), pr2)
+    # a width that is not a multiple of 256 keeps the CUDA-core scan
+    odd = B.Pool(384, 64, max_nq=8, key_format="e4m3")
+    odd.append(torch.randn(64, 384, device="cuda").to(torch.bfloat16),
+               torch.zeros(64, dtype=torch.int32, device="cuda"), tag=1)
+    odd.query(torch.randn(4, 384, device="cuda").to(torch.bfloat16), fixed(8, 8))
+    with pytest.raises(B.OilbirdError):
+        odd.query(torch.randn(4, 384, device="cuda").to(torch.bfloat16), fixed(8, 8, path=B.PATH_MMA))

@@ -437,7 +437,11 @@ static int resolve_path(const oilbird_pool* p, const oilbird_query_params* pr, i
   // single-request decode streams keys through the CUDA cores; batches go to tcgen05,
   // small batches on pools of the paper's size to mma.sync
   if (pr->path != OILBIRD_PATH_AUTO) return pr->path;
-  if (nq <= 2) return OILBIRD_PATH_GEMV;
+  // (two queries on an 8-bit pool: the CUDA-core scan converts every code once per query and
+  // is bound by that, 78 us against 63 at 268 MB of codes; below 128 MB its fused append
+  // makes up for it)
+  if (nq <= 1 || (nq == 2 && !(p->r.e4m3 && p->n_rows * (int64_t)p->r.d >= (128ll << 20))))
+    return OILBIRD_PATH_GEMV;
   if (p->r.e4m3) {
     // 8-bit pools have no tcgen05 scan: the warp-level tensor scan scores 8 or 16 queries
     // per pass over the codes, the CUDA-core scan two

@@ -43,8 +43,26 @@ def test_random_configuration(seed):
                        offset=int(rng.integers(0, 4)), depth_mode=mode, cont_len=L,
                        tier_thr=tuple(tiers), tier_depth=tuple(depths),
                        exclude_tag=None if ex is None else torch.from_numpy(ex.view(np.int64)).cuda())
-    for path in (B.PATH_GEMV, B.PATH_TENSOR, B.PATH_AUTO):
+    paths = [B.PATH_GEMV, B.PATH_TENSOR, B.PATH_AUTO]
+    if d % 128 == 0 and k <= 64:
+        paths.append(B.PATH_MMA)                         # the warp-level tensor scan takes these
+    for path in paths:
         pr.path = path
         out = pool.query(q, pr)
         check_query(out, ora, W.to_bits(q), pr, exclude=ex)
     assert pool.stats()["stalled"] == 0
+    # the same pool with 8-bit keys (widths that are multiples of 16), every scan it has
+    if d % 16 == 0 and n_rows <= 20000:
+        pool8 = B.Pool(w.d, w.n_rows, max_k=128, max_nq=256, max_traces=w.num_traces + 1,
+                       key_format="e4m3")
+        ora8 = OraclePool(w.d, "e4m3")
+        rng2 = np.random.default_rng(1000 + seed)
+        for t, (st, tk, _) in enumerate(w.traces("cuda")):
+            tag = int(rng2.integers(1, 4))
+            pool8.append(st, tk, tag=tag)
+            ora8.append(W.to_bits(st), tk.cpu().numpy(), tag=tag)
+        paths8 = [B.PATH_GEMV, B.PATH_AUTO] + ([B.PATH_MMA] if d % 256 == 0 and k <= 64 else [])
+        for path in paths8:
+            pr.path = path
+            check_query(pool8.query(q, pr), ora8, W.to_bits(q), pr, exclude=ex)
+        assert pool8.stats()["stalled"] == 0

@@ -503,7 +503,7 @@ static int query_impl(oilbird_pool_t* p, const void* q, int32_t nq, const oilbir
     if (p->r.e4m3 && path == OILBIRD_PATH_MMA) {
       e = launch_scan_mma(pv, p->codes, p->scales, (const uint16_t*)q, nq, pr->k, kk,
                           pr->exclude_tag, p->partial, p->q_valid, p->stats, p->r.max_lists,
-                          p->num_sms, p->smem_limit, &n_lists, nullptr, st);
+                          p->num_sms, p->smem_limit, &n_lists, fused, st);
       if (e != cudaSuccess) return cuda_fail(e, "8-bit warp-level tensor scan kernel launch");
       p->launches += 1;
     } else if (p->r.e4m3) {
@@ -569,13 +569,14 @@ static int step_impl(oilbird_pool_t* p, const void* states, const int32_t* token
   // would find the rows in place, but keep to the single-request case there too)
   const int path = resolve_path(p, pr, nq);
   const bool gemv = p->r.e4m3 ? (nq <= 2 && path == OILBIRD_PATH_GEMV) : path == OILBIRD_PATH_GEMV;
-  // the warp-level tensor scan appends the step's rows itself in its 8-query form (16-bit keys)
-  const bool mma8 = !p->r.e4m3 && path == OILBIRD_PATH_MMA &&
-                    scan_mma_tiles(p->r.d, list_len(pr->k), nq, p->smem_limit, false) == 1;
+  // the warp-level tensor scan appends the step's rows itself in its 8-query form (eight rows
+  // per CTA on 16-bit keys, one on 8-bit keys)
+  const bool mma8 = path == OILBIRD_PATH_MMA &&
+                    scan_mma_tiles(p->r.d, list_len(pr->k), nq, p->smem_limit, p->r.e4m3) == 1;
   const bool fuse =
       n >= 1 && n <= kFuseMaxRows &&
       ((gemv && scan_gemv_grid(rows_after, p->num_sms, p->r.max_lists) >= n) ||
-       (mma8 && 8 * (int64_t)scan_mma_grid(rows_after, p->num_sms, p->r.max_lists) >= n));
+       (mma8 && (p->r.e4m3 ? 1 : 8) * (int64_t)scan_mma_grid(rows_after, p->num_sms, p->r.max_lists) >= n));
   if (!fuse) {
     rc = append_impl(p, states, tokens, n, tag, flags, -1, stream);
     if (rc) return rc;

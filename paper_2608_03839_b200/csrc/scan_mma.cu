@@ -29,6 +29,7 @@
 #include "common.cuh"
 #include "internal.h"
 #include "normalize.cuh"
+#include "quant8.cuh"
 
 namespace oilbird {
 
@@ -277,6 +278,30 @@ scan_mma_kernel(PoolView pv, const uint8_t* __restrict__ codes, const float* __r
       atomicAdd(fa.ready, 1ull);
     }
   }
+  // 8-bit pools: the same eight warps quantise one row per CTA together (the block routine,
+  // meeting at a named barrier of their own)
+  if (kFp8 && NT == 1 && warp >= 8 && (int)blockIdx.x < fa.n) {
+    const int r = blockIdx.x;
+    const int64_t row = (int64_t)fa.row0 + r;
+    const bool ok = quantize_row_e4m3<true, 256, 5>(fa.states + (size_t)r * d, d,
+                                                    const_cast<uint8_t*>(codes) + row * d,
+                                                    const_cast<float*>(scales) + row);
+    if (threadIdx.x == 256) {
+      fa.tok[row] = fa.tokens[r];
+      fa.trace_id[row] = fa.trace;
+      if (!ok) atomicAdd(&stats->degenerate_rows, 1ull);           // stored as a zero key
+      if (r == 0) {
+        fa.trace_end[fa.trace] = fa.row0 + fa.n;
+        if (fa.set_tag) { fa.trace_tag[fa.trace] = fa.tag; fa.trace_gbase[fa.trace] = fa.gbase; }
+      }
+    }
+    __threadfence();                   // this thread's part of the row, before the count
+    asm volatile("bar.sync 5, 256;" ::: "memory");
+    if (threadIdx.x == 256) {
+      __threadfence();                 // cumulative: the eight warps' row, as seen through the barrier
+      atomicAdd(fa.ready, 1ull);
+    }
+  }
   bool waited = fa.n == 0;             // this warp has seen the appended rows arrive
   // a group of rows that holds rows of this step's append: read through L2, after the wait
   auto fresh_at = [&](int rbx) { return fa.n > 0 && rbx + kMmaRows > fa.row0; };
@@ -456,8 +481,9 @@ scan_mma_kernel(PoolView pv, const uint8_t* __restrict__ codes, const float* __r
       // 8-bit pools: the rows' scales (and the queries' 2^14 taken back)
       float sc0 = 1.f, sc1 = 1.f;
       if (kFp8 && own) {
-        sc0 = row0 < r_hi ? scales[row0] * (1.f / kFp8QueryScale) : 0.f;
-        sc1 = row1 < r_hi ? scales[row1] * (1.f / kFp8QueryScale) : 0.f;
+        // (a row appended by this launch: its scale was written a moment ago, read it through L2)
+        sc0 = row0 < r_hi ? (cur_fresh ? __ldcg(&scales[row0]) : scales[row0]) * (1.f / kFp8QueryScale) : 0.f;
+        sc1 = row1 < r_hi ? (cur_fresh ? __ldcg(&scales[row1]) : scales[row1]) * (1.f / kFp8QueryScale) : 0.f;
       }
       u64 key[2 * NT][2];                    // [list][row0 / row1]
       bool any = false;
@@ -618,8 +644,8 @@ cudaError_t launch_scan_mma(const PoolView& pv, const uint8_t* codes, const floa
   if (fused) {
     // every appending warp must exist (eight per CTA), and all CTAs be resident together
     // (they are: at most one per SM is launched), because scanning warps wait for the
-    // appending ones; the 8-query form on 16-bit keys only
-    if (fp8 || nt != 1 || fused->n > 8 * grid || fused->n > kFuseMaxRows) return cudaErrorInvalidValue;
+    // appending ones; the 8-query form only (8-bit keys: one row per CTA)
+    if (nt != 1 || fused->n > (fp8 ? 1 : 8) * grid || fused->n > kFuseMaxRows) return cudaErrorInvalidValue;
     fa = *fused;
   }
 #define OILBIRD_MMA_CASE(E_, NT_, F_)                                                          \

@@ -289,3 +289,41 @@ def test_mma_scan_wide_rows_exclusion_and_ragged_sizes():
     odd.query(torch.randn(4, 384, device="cuda").to(torch.bfloat16), fixed(8, 8))
     with pytest.raises(B.OilbirdError):
         odd.query(torch.randn(4, 384, device="cuda").to(torch.bfloat16), fixed(8, 8, path=B.PATH_MMA))
+
+
+def test_mma_scan_appends_the_rows_of_a_step_itself():
+    # three queries and more on an 8-bit pool: eight warps of the scan's first CTAs quantise
+    # one row per CTA (two launches per step); codes and scales equal the oracle's, and a
+    # query of the same step finds the new rows and honours their tag
+    w = W.C1.scaled(n_rows=4096, nq=5, d=512)
+    pool, ora = fill_both(w, key_format="e4m3", spare_rows=1024)
+    g = torch.Generator(device="cuda").manual_seed(44)
+    for step in range(8):
+        n = [8, 1, 64, 33, 8, 16, 2, 8][step]
+        st = torch.randn(n, w.d, generator=g, device="cuda").to(torch.bfloat16)
+        if step == 3:
+            st[5] = 0                                     # a zero row among the new ones
+        tk = torch.randint(0, 100, (n,), generator=g, device="cuda", dtype=torch.int32)
+        q = torch.randn(5, w.d, generator=g, device="cuda").to(torch.bfloat16)
+        q[0] = st[n - 1]
+        q[3] = st[0]
+        tag = 9000 + step
+        ex = torch.tensor([tag, 12345, 0, 0, tag], dtype=torch.int64, device="cuda")
+        pr = fixed(4, 4, theta=-2.0)
+        pr.exclude_tag = ex
+        new_trace = step % 2 == 0
+        l0 = pool.launch_count
+        out = pool.step(st, tk, q, pr, tag=tag, new_trace=new_trace)
+        assert pool.launch_count - l0 == 2
+        ora.append(W.to_bits(st), tk.cpu().numpy(), tag=tag, new_trace=new_trace)
+        first_new = len(pool) - n
+        if new_trace:
+            assert all(int(r) < first_new for r in out.idx[0].tolist())
+        assert int(out.idx[3, 0]) == first_new
+        check_query(out, ora, W.to_bits(q), pr, exclude=ex.cpu().numpy().astype(np.uint64))
+    assert pool.stats()["stalled"] == 0 and pool.stats()["degenerate_rows"] == 1
+    codes, scales = pool.read_codes()
+    assert np.array_equal(codes, ora.codes)
+    assert np.array_equal(scales.view(np.uint32), ora.scales.view(np.uint32))
+    _, tok, tid = pool.read_rows()
+    assert np.array_equal(tok, ora.tokens) and np.array_equal(tid, ora.trace_ids)

@@ -33,15 +33,14 @@
 
 namespace oilbird {
 
-constexpr int kMmaThreads = 512;
-constexpr int kMmaWarps = kMmaThreads / 32;
+constexpr int kMmaThreads = 512;   // one CTA of four quads of four warps per SM
 constexpr int kMmaQ = 8;          // queries per pass = the N of the instruction
 constexpr int kMmaRows = 16;      // rows per warp step = the M of the instruction
 constexpr int kMmaDepth1 = 4;     // 32-element blocks per lane, row and step: 8-query form
 constexpr int kMmaDepth2 = 2;     // 16-query form (its accumulators and lists need the registers)
 constexpr int kMmaBatchInsert = 5; // candidates of a group and query from which they are merged in as a sorted vector
-constexpr int kMmaPadBytes = 64;  // per query row in shared memory: keeps the 16-byte loads of
-                                  // a quarter warp (two queries x four offsets) on distinct banks
+constexpr int kMmaPadBytes = 64;   // per query row in shared memory: keeps the 16-byte loads of
+                                   // a quarter warp (two queries x four offsets) on distinct banks
 
 __device__ __forceinline__ void mma_bf16(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2,
                                          uint32_t a3, uint32_t b0, uint32_t b1) {
@@ -61,7 +60,8 @@ __device__ __forceinline__ uint4 ld_key16(const uint4* p, bool fresh) {
   return fresh ? ld_cg16(p) : ld_stream16(p);
 }
 
-// barrier among the four warps of a quad (ids 1 and 2; 0 is __syncthreads)
+// barrier among the four warps of a quad (ids 1 to 4; 0 is __syncthreads, 5 the quantising
+// warps of an 8-bit step)
 __device__ __forceinline__ void quad_bar(int id) {
   asm volatile("bar.sync %0, 128;" ::"r"(id) : "memory");
 }

@@ -22,8 +22,10 @@ import sys
 import threading
 import time
 
-import numpy as np
-import torch
+os.environ.setdefault("CUDA_MODULE_LOADING", "EAGER")   # see paper_2608_03839_b200/binding.py
+
+import numpy as np  # noqa: E402
+import torch  # noqa: E402
 
 ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:

@@ -128,6 +128,13 @@ size_t oilbird_pool_arena_bytes(const oilbird_pool_config* cfg);
  * Lifecycle.  create() validates cfg, allocates (or carves the arena) and sets the
  * pool empty.  reset() empties it (rows = traces = 0, counters cleared) in stream
  * order without freeing anything.  destroy() synchronises the device and frees.
+ *
+ * Module loading.  The kernels of a step are chained with programmatic launches.  With
+ * CUDA's lazy module loading (the default) the first steps of a process were seen to
+ * dead-lock now and then on the largest configuration; with eager loading never.  create
+ * therefore loads all of the library's kernels before anything is launched, and callers
+ * should run with CUDA_MODULE_LOADING=EAGER set before CUDA is initialised (the Python
+ * binding, bench.py and the tests do).
  */
 int oilbird_pool_create (oilbird_pool_t** out, const oilbird_pool_config* cfg);
 int oilbird_pool_reset  (oilbird_pool_t* pool, void* cuda_stream);

@@ -11,8 +11,16 @@ import ctypes
 import os
 from dataclasses import dataclass, field
 
-import numpy as np
-import torch
+# The library chains the kernels of a step with programmatic launches; with CUDA's lazy
+# module loading the first steps of a process dead-locked now and then on the largest
+# configuration (a kernel loading at its first launch while others of the chain were resident
+# and waiting; with eager loading: never in the runs made).  The library loads its own
+# kernels before it launches any, and the process is asked to load all modules eagerly too,
+# which takes effect if CUDA has not been initialised yet (importing torch does not do that).
+os.environ.setdefault("CUDA_MODULE_LOADING", "EAGER")
+
+import numpy as np  # noqa: E402
+import torch  # noqa: E402
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "liboilbird.so")

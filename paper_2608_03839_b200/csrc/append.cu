@@ -183,4 +183,12 @@ cudaError_t launch_qnorm(const uint16_t* q, int32_t nq, int32_t nq_pad, int32_t 
                     stats, xchg, n_xchg);
 }
 
+cudaError_t preload_append_kernels() {
+  cudaError_t e;
+  if ((e = preload_kernel(append_kernel)) != cudaSuccess) return e;
+  if ((e = preload_kernel(append_bulk_kernel<4>)) != cudaSuccess) return e;
+  if ((e = preload_kernel(append_bulk2_kernel)) != cudaSuccess) return e;
+  return preload_kernel(qnorm_kernel);
+}
+
 }  // namespace oilbird

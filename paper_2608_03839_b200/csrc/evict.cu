@@ -75,4 +75,6 @@ cudaError_t launch_compact(unsigned char* keys, float* scales, int32_t* tok, int
                                      st);
 }
 
+cudaError_t preload_evict_kernels() { return preload_kernel(compact_kernel); }
+
 }  // namespace oilbird

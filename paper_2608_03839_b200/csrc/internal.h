@@ -30,6 +30,32 @@ inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, s
   return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
 }
 
+// With lazy module loading (the CUDA default) a kernel is loaded at its first launch, and
+// that load can wait for the device to go idle.  The kernels of a step are chained with
+// programmatic launches: a kernel may already be resident and waiting for its predecessor
+// when the host reaches the first launch of the next one.  On B200 with driver 580 this
+// dead-locked about three process starts in ten on the largest configuration (the first
+// steps of a process never finished; CUDA_MODULE_LOADING=EAGER: none in ten).  So every
+// kernel of the library is loaded explicitly, once per device, before any of them is
+// launched: asking for a function's attributes loads it.
+template <typename K>
+inline cudaError_t preload_kernel(K kernel) {
+  cudaFuncAttributes attr;
+  return cudaFuncGetAttributes(&attr, kernel);
+}
+cudaError_t preload_append_kernels();
+cudaError_t preload_evict_kernels();
+cudaError_t preload_merge_kernels();
+cudaError_t preload_merge_tree_kernels();
+cudaError_t preload_quant8_kernels();
+cudaError_t preload_ring_kernels();
+cudaError_t preload_scan_gemv_kernels();
+cudaError_t preload_scan_mma_kernels();
+cudaError_t preload_scan_tc_kernels();
+cudaError_t preload_shard_kernels();
+// all of the above, once per device (the current device); thread-safe
+cudaError_t preload_all_kernels();
+
 // Device counters (one struct in device memory per pool).
 struct DeviceStats {
   unsigned long long degenerate_rows;

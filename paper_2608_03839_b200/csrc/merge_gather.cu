@@ -137,4 +137,9 @@ cudaError_t launch_gather_only(const PoolView& pv, const int32_t* idx, const flo
   return launch_pdl(gather_only_kernel, dim3(nq), dim3(128), 0, st, pv, idx, score, gp, out);
 }
 
+cudaError_t preload_merge_kernels() {
+  cudaError_t e = preload_kernel(merge_gather_kernel);
+  return e != cudaSuccess ? e : preload_kernel(gather_only_kernel);
+}
+
 }  // namespace oilbird

@@ -145,6 +145,8 @@ merge_tree_kernel(int nq, const int32_t* __restrict__ sem_tok, const int32_t* __
   if (lane == 0) n_nodes[q] = n;
 }
 
+cudaError_t preload_merge_tree_kernels() { return preload_kernel(merge_tree_kernel); }
+
 }  // namespace oilbird
 
 using namespace oilbird;
@@ -175,6 +177,7 @@ int oilbird_merge_chains(int32_t nq, const int32_t* sem_tok, const int32_t* sem_
       mp->min_len < 0)
     return OILBIRD_EINVAL;
   if (cudaSetDevice(device) != cudaSuccess) return OILBIRD_ECUDA;
+  if (preload_all_kernels() != cudaSuccess) return OILBIRD_ECUDA;
   const int grid = (nq + kMergeTreeWarps - 1) / kMergeTreeWarps;
   cudaError_t e = launch_pdl(merge_tree_kernel, dim3(grid), dim3(kMergeTreeWarps * 32), 0,
                              (cudaStream_t)cuda_stream, nq, sem_tok, sem_len, k, L, extra_tok,

@@ -5,6 +5,7 @@
 #include <stdio.h>
 #include <string.h>
 
+#include <mutex>
 #include <new>
 #include <vector>
 
@@ -13,6 +14,31 @@
 using namespace oilbird;
 
 static thread_local char g_cuda_err[256] = "";
+
+namespace oilbird {
+cudaError_t preload_all_kernels() {
+  static std::mutex mu;
+  static bool done[64] = {};
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  std::lock_guard<std::mutex> lock(mu);
+  if (dev >= 0 && dev < 64 && done[dev]) return cudaSuccess;
+  if ((e = preload_append_kernels()) != cudaSuccess) return e;
+  if ((e = preload_evict_kernels()) != cudaSuccess) return e;
+  if ((e = preload_merge_kernels()) != cudaSuccess) return e;
+  if ((e = preload_merge_tree_kernels()) != cudaSuccess) return e;
+  if ((e = preload_quant8_kernels()) != cudaSuccess) return e;
+  if ((e = preload_ring_kernels()) != cudaSuccess) return e;
+  if ((e = preload_scan_gemv_kernels()) != cudaSuccess) return e;
+  if ((e = preload_scan_mma_kernels()) != cudaSuccess) return e;
+  if ((e = preload_scan_tc_kernels()) != cudaSuccess) return e;
+  if ((e = preload_shard_kernels()) != cudaSuccess) return e;
+  if (dev >= 0 && dev < 64) done[dev] = true;
+  return cudaSuccess;
+}
+}  // namespace oilbird
+
 
 static int cuda_fail(cudaError_t e, const char* what) {
   snprintf(g_cuda_err, sizeof g_cuda_err, "%s: %s", what, cudaGetErrorString(e));
@@ -183,6 +209,7 @@ int oilbird_pool_create(oilbird_pool_t** out, const oilbird_pool_config* cfg) {
   CU(cudaGetDeviceCount(&n_dev));
   if (cfg->device < 0 || cfg->device >= n_dev) return OILBIRD_EINVAL;
   CU(cudaSetDevice(cfg->device));
+  CU(preload_all_kernels());       // before anything of the library is launched on this device
   cudaDeviceProp prop;
   CU(cudaGetDeviceProperties(&prop, cfg->device));
   Resolved r;

@@ -287,4 +287,15 @@ cudaError_t launch_scan_gemv_e4m3(const uint8_t* codes, const float* scales, con
   return launch_q8_qt<1>(kk, codes, scales, pv, q_raw, nq, k, exclude_tag, partial, q_valid, stats, grid, fa, st);
 }
 
+cudaError_t preload_quant8_kernels() {
+  cudaError_t e;
+  if ((e = preload_kernel(append_e4m3_kernel)) != cudaSuccess) return e;
+  if ((e = preload_kernel(scan_gemv_e4m3_kernel<1, 1>)) != cudaSuccess) return e;
+  if ((e = preload_kernel(scan_gemv_e4m3_kernel<1, 2>)) != cudaSuccess) return e;
+  if ((e = preload_kernel(scan_gemv_e4m3_kernel<1, 4>)) != cudaSuccess) return e;
+  if ((e = preload_kernel(scan_gemv_e4m3_kernel<2, 1>)) != cudaSuccess) return e;
+  if ((e = preload_kernel(scan_gemv_e4m3_kernel<2, 2>)) != cudaSuccess) return e;
+  return preload_kernel(scan_gemv_e4m3_kernel<2, 4>);
+}
+
 }  // namespace oilbird

@@ -40,6 +40,10 @@ static char g_static_err[256] = "";
 
 static int static_setup(int device) {
   if (g_scratch_ptr[device]) return OILBIRD_OK;
+  if (preload_all_kernels() != cudaSuccess) {      // first use on this device
+    snprintf(g_static_err, sizeof g_static_err, "loading the library's kernels failed");
+    return OILBIRD_ECUDA;
+  }
   void* p = nullptr;
   cudaError_t e = cudaGetSymbolAddress(&p, g_static_scratch);
   if (e != cudaSuccess || !p) {

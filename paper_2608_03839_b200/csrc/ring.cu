@@ -143,6 +143,13 @@ ring_merge_kernel(const u64* __restrict__ partial, int n_lists, int nq, int m, i
   }
 }
 
+cudaError_t preload_ring_kernels() {
+  cudaError_t e;
+  if ((e = preload_kernel(ring_append_kernel)) != cudaSuccess) return e;
+  if ((e = preload_kernel(ring_scan_kernel)) != cudaSuccess) return e;
+  return preload_kernel(ring_merge_kernel);
+}
+
 }  // namespace oilbird
 
 using namespace oilbird;
@@ -181,6 +188,7 @@ int oilbird_ring_create(oilbird_ring_t** out, const oilbird_ring_config* cfg) {
   RCU(cudaGetDeviceCount(&n_dev));
   if (cfg->device < 0 || cfg->device >= n_dev) return OILBIRD_EINVAL;
   RCU(cudaSetDevice(cfg->device));
+  RCU(preload_all_kernels());      // before anything of the library is launched on this device
   int sms = 0;
   RCU(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, cfg->device));
   oilbird_ring* r = new (std::nothrow) oilbird_ring();

@@ -243,4 +243,14 @@ cudaError_t launch_scan_gemv(const PoolView& pv, const uint16_t* q_raw, int32_t 
   return launch_qt<1>(kk, pv, q_raw, nq, k, exclude_tag, partial, q_valid, stats, grid, fa, st);
 }
 
+cudaError_t preload_scan_gemv_kernels() {
+  cudaError_t e;
+  if ((e = preload_kernel(scan_gemv_kernel<1, 1>)) != cudaSuccess) return e;
+  if ((e = preload_kernel(scan_gemv_kernel<1, 2>)) != cudaSuccess) return e;
+  if ((e = preload_kernel(scan_gemv_kernel<1, 4>)) != cudaSuccess) return e;
+  if ((e = preload_kernel(scan_gemv_kernel<2, 1>)) != cudaSuccess) return e;
+  if ((e = preload_kernel(scan_gemv_kernel<2, 2>)) != cudaSuccess) return e;
+  return preload_kernel(scan_gemv_kernel<2, 4>);
+}
+
 }  // namespace oilbird

@@ -664,4 +664,16 @@ cudaError_t launch_scan_mma(const PoolView& pv, const uint8_t* codes, const floa
   return cudaErrorInvalidValue;
 }
 
+cudaError_t preload_scan_mma_kernels() {
+  cudaError_t e;
+  if ((e = preload_kernel(scan_mma_kernel<1, 1, false>)) != cudaSuccess) return e;
+  if ((e = preload_kernel(scan_mma_kernel<2, 1, false>)) != cudaSuccess) return e;
+  if ((e = preload_kernel(scan_mma_kernel<1, 2, false>)) != cudaSuccess) return e;
+  if ((e = preload_kernel(scan_mma_kernel<2, 2, false>)) != cudaSuccess) return e;
+  if ((e = preload_kernel(scan_mma_kernel<1, 1, true>)) != cudaSuccess) return e;
+  if ((e = preload_kernel(scan_mma_kernel<2, 1, true>)) != cudaSuccess) return e;
+  if ((e = preload_kernel(scan_mma_kernel<1, 2, true>)) != cudaSuccess) return e;
+  return preload_kernel(scan_mma_kernel<2, 2, true>);
+}
+
 }  // namespace oilbird

@@ -739,4 +739,6 @@ cudaError_t launch_scan_tc(TcCache* cache, const PoolView& pv, int32_t q0, int32
                     xchg);
 }
 
+cudaError_t preload_scan_tc_kernels() { return preload_kernel(scan_tc_kernel); }
+
 }  // namespace oilbird

@@ -123,6 +123,11 @@ cudaError_t launch_to_global(const int32_t* idx, int64_t* out, int64_t n, const 
                     trace_end, trace_gbase, n_rows);
 }
 
+cudaError_t preload_shard_kernels() {
+  cudaError_t e = preload_kernel(to_global_kernel);
+  return e != cudaSuccess ? e : preload_kernel(merge_shards_kernel);
+}
+
 }  // namespace oilbird
 
 using namespace oilbird;
@@ -138,6 +143,7 @@ extern "C" int oilbird_merge_shards(int32_t n_shards, int32_t nq, int32_t k, int
       !out_len || !out_tok || theta != theta || (off_gidx % 8) || (shard_stride % 8))
     return OILBIRD_EINVAL;
   if (cudaSetDevice(device) != cudaSuccess) return OILBIRD_ECUDA;
+  if (preload_all_kernels() != cudaSuccess) return OILBIRD_ECUDA;
   cudaError_t e = launch_pdl(merge_shards_kernel, dim3(nq), dim3(kShardThreads), 0,
                              (cudaStream_t)cuda_stream, n_shards, nq, k, L, theta,
                              (const unsigned char*)gathered, shard_stride, off_gidx, off_score,

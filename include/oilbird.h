@@ -20,6 +20,11 @@
  *     append on the same stream.  Using different streams for append and query is
  *     the caller's synchronisation problem.  One host thread per pool at a time.
  *   - There is no CPU fallback: without a CUDA device create() fails.
+ *   - Alignment: bf16 matrices passed in (states, q, and the keys of
+ *     oilbird_query_static) must start on a 16-byte boundary, int32 / float arrays on a
+ *     4-byte boundary, exclude_tag on an 8-byte boundary; rows are then aligned by
+ *     themselves because d is a multiple of 8.  The kernels read them with vector loads, so a
+ *     misaligned pointer is refused with OILBIRD_EINVAL before anything is launched.
  */
 #ifndef OILBIRD_H_
 #define OILBIRD_H_
@@ -37,6 +42,7 @@ extern "C" {
 #define OILBIRD_ENOMEM    (-3)  /* device or host allocation failed                    */
 #define OILBIRD_ECUDA     (-4)  /* a CUDA call failed; see oilbird_last_cuda_error()   */
 #define OILBIRD_ESTALL    (-5)  /* a bounded device-side wait gave up (status only)    */
+#define OILBIRD_EGUARD    (-6)  /* oilbird_pool_check_guards found sentinel bytes changed */
 
 #define OILBIRD_MAX_NQ        256   /* queries per call                                */
 #define OILBIRD_MAX_K         128   /* neighbours per query                            */
@@ -46,6 +52,10 @@ extern "C" {
 /* pool flags (oilbird_pool_config.flags) */
 #define OILBIRD_KEYS_E4M3  1u   /* keys are stored as FP8 E4M3 codes with one fp32 scale
                                    per row instead of bf16 (see "8-bit keys" below)     */
+#define OILBIRD_DEBUG_GUARDS 2u /* debugging aid: every array of the pool's allocation is
+                                   followed by sentinel bytes (from its last byte to the
+                                   next array, at least 256) that no kernel may touch;
+                                   see oilbird_pool_check_guards                        */
 
 /* append flags */
 #define OILBIRD_NEW_TRACE  1u   /* the rows open a new trace (a finished request)      */
@@ -75,7 +85,7 @@ typedef struct {
   int32_t  max_k;          /* largest k (<= OILBIRD_MAX_K); 0 = 64                      */
   int32_t  max_append;     /* largest n of the *_host append variant; 0 = 4096          */
   int32_t  device;         /* CUDA ordinal                                              */
-  uint32_t flags;          /* 0 or OILBIRD_KEYS_E4M3                                    */
+  uint32_t flags;          /* 0, OILBIRD_KEYS_E4M3, OILBIRD_DEBUG_GUARDS                */
   void*    arena;          /* dev, optional: caller-provided memory (256-B aligned) of  */
   size_t   arena_bytes;    /*   at least oilbird_pool_arena_bytes(); NULL = cudaMalloc  */
 } oilbird_pool_config;
@@ -97,7 +107,13 @@ typedef struct {
   const uint64_t* exclude_tag;              /* dev [nq] or NULL: rows of traces whose
                                                tag equals a non-zero entry are skipped
                                                (a request must not draft from a stored
-                                               copy of its own prompt's trace)          */
+                                               copy of its own prompt's trace).  A
+                                               DEVICE pointer on purpose, like q: the
+                                               scan reads it, and a host pointer would
+                                               cost a copy and a staging buffer on the
+                                               latency path; the *_host entry points
+                                               take a host pointer and upload it with
+                                               the queries                              */
   int32_t  path;                            /* OILBIRD_PATH_*                           */
 } oilbird_query_params;
 
@@ -129,12 +145,20 @@ size_t oilbird_pool_arena_bytes(const oilbird_pool_config* cfg);
  * pool empty.  reset() empties it (rows = traces = 0, counters cleared) in stream
  * order without freeing anything.  destroy() synchronises the device and frees.
  *
- * Module loading.  The kernels of a step are chained with programmatic launches.  With
- * CUDA's lazy module loading (the default) the first steps of a process were seen to
- * dead-lock now and then on the largest configuration; with eager loading never.  create
- * therefore loads all of the library's kernels before anything is launched, and callers
- * should run with CUDA_MODULE_LOADING=EAGER set before CUDA is initialised (the Python
- * binding, bench.py and the tests do).
+ * Module loading and programmatic launches.  create loads all of the library's kernels and
+ * sets their attributes before anything is launched, so that a query's first call does
+ * nothing a later call does not do.  The kernels of a step can be chained with programmatic
+ * stream serialization (a kernel is set up on the GPU while its predecessor still runs:
+ * about 6 us per step on a 90 us step).  The library does that only when the process loads
+ * CUDA modules eagerly (CUDA_MODULE_LOADING=EAGER in the environment before CUDA is
+ * initialised; the Python binding, bench.py and the tests set it) and only for scans short
+ * enough to gain from it (pools up to 4 GB of keys); in every other case, lazy loading (the
+ * CUDA default) included, its launches are plain ones, and nothing needs to be set for the
+ * library to be safe.  Reason: with lazy loading and chained launches the first steps of a
+ * process were seen to dead-lock now and then on the largest configuration; the mechanism
+ * inside the driver was not established, so the combination is simply not used.  A chained
+ * kernel releases its successor only after its own predecessor has finished: at most two of
+ * the library's grids are on the GPU at a time.
  */
 int oilbird_pool_create (oilbird_pool_t** out, const oilbird_pool_config* cfg);
 int oilbird_pool_reset  (oilbird_pool_t* pool, void* cuda_stream);
@@ -200,7 +224,8 @@ int oilbird_pool_evict_oldest(oilbird_pool_t* pool, int32_t n_traces, int64_t* r
  * the last step; n may be 0) followed by oilbird_pool_query, in one call, with the same
  * arguments, results and error codes as the two calls (Algorithm 1 runs once per decoding
  * step: the accepted tokens' states are stored, then the new last position is looked up).
- * Nothing is appended if the query arguments are invalid.  For the single-request scan
+ * Nothing is appended if the call is refused (invalid arguments or parameters, or a scan
+ * path this pool does not offer).  For the single-request scan
  * (nq <= 2; 16-bit and 8-bit pools) and the warp-level tensor scan in its 8-query form
  * (OILBIRD_PATH_MMA, nq <= 8), and up to 64 rows, the append has no kernel of its own: the
  * first CTAs of the scan normalise the rows before they start scanning (a row per CTA, or a
@@ -245,6 +270,27 @@ int32_t oilbird_pool_num_traces(const oilbird_pool_t* pool);
 /* Synchronises cuda_stream, then reports the device counters. Returns OILBIRD_ESTALL
  * if a device-side wait ever gave up, else OILBIRD_OK. */
 int oilbird_pool_status(oilbird_pool_t* pool, oilbird_pool_stats* stats, void* cuda_stream);
+/*
+ * Bounded waits.  The library's kernels wait on the device in two places only: a scan that
+ * also appends the step's rows waits for a row counter, and the tensor-core scan's warps wait
+ * on shared-memory barriers for each other.  Every such wait gives up after limit_ns
+ * nanoseconds (0 = the default, two seconds): the kernel raises the `stalled` status, lets
+ * the copies it has in flight land, frees what it holds and returns, so the context stays
+ * usable; oilbird_pool_status then returns OILBIRD_ESTALL until reset().  set_wait_limit
+ * takes effect in stream order.  stall_selftest runs one small kernel that performs both
+ * kinds of wait on things that never happen (a counter nobody advances, a barrier nobody
+ * arrives at), so the give-up path can be exercised: after it, status reports the stall.
+ */
+int oilbird_pool_set_wait_limit(oilbird_pool_t* pool, uint64_t limit_ns, void* cuda_stream);
+int oilbird_pool_stall_selftest(oilbird_pool_t* pool, void* cuda_stream);
+/*
+ * Guard zones (pools created with OILBIRD_DEBUG_GUARDS).  Synchronises cuda_stream and
+ * compares every sentinel byte behind the pool's arrays (keys, tokens, trace tables,
+ * normalised queries, candidate lists, counters, exchange buffers, host staging) with the
+ * value written at creation.  Returns OILBIRD_OK, or OILBIRD_EGUARD with the array and the
+ * offset in oilbird_last_cuda_error().  EINVAL for a pool without guard zones.
+ */
+int oilbird_pool_check_guards(oilbird_pool_t* pool, void* cuda_stream);
 /* Copy stored data to host memory (synchronous; for tests and debugging).
  * keys: [n,d] bf16; tokens, trace_ids: [n] int32; rows [row0, row0+n). */
 int oilbird_pool_read_rows(oilbird_pool_t* pool, int64_t row0, int64_t n, void* keys_host,
@@ -383,7 +429,9 @@ int oilbird_merge_shards(int32_t n_shards, int32_t nq, int32_t k, int32_t L, flo
  * and later chains are not reached).  cost = length - longest prefix already in the tree.
  * With root_attached != 0 nothing is shared: every chain hangs from the root as its own
  * branch (the paper's ablation arm).
- * Tree layout per request: node 0 is the root (the anchor token), tree_parent[0] = -1;
+ * Tree layout per request: node 0 is the root (the anchor token), tree_parent[0] = -1 (a
+ * parent entry that does not name another node of the tree is read as -1: that node is
+ * detached, nothing is followed out of range);
  * tree_tok / tree_parent [nq,max_nodes] and n_nodes [nq] are read and updated in place
  * (new nodes are numbered in the order they are bought); depth [nq,max_nodes] and mask
  * [nq,max_nodes] are written: bit j of mask[i] is set iff node j is node i or one of its

@@ -25,9 +25,10 @@ import torch  # noqa: E402
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "liboilbird.so")
 
-OK, EINVAL, ECAPACITY, ENOMEM, ECUDA, ESTALL = 0, -1, -2, -3, -4, -5
+OK, EINVAL, ECAPACITY, ENOMEM, ECUDA, ESTALL, EGUARD = 0, -1, -2, -3, -4, -5, -6
 NEW_TRACE = 1
 KEYS_E4M3 = 1          # pool flag: 8-bit keys
+DEBUG_GUARDS = 2       # pool flag: sentinel bytes behind every array (see Pool.check_guards)
 DEPTH_FIXED, DEPTH_TIERED = 0, 1
 PATH_AUTO, PATH_GEMV, PATH_TENSOR, PATH_MMA = 0, 1, 2, 3
 MAX_NQ, MAX_K, MAX_CONT_LEN, MAX_TIERS = 256, 128, 128, 4
@@ -107,6 +108,9 @@ SYMBOLS = {
     "oilbird_pool_size": (_i64, [_vp]),
     "oilbird_pool_num_traces": (_i32, [_vp]),
     "oilbird_pool_status": (ctypes.c_int, [_vp, ctypes.POINTER(PoolStats), _vp]),
+    "oilbird_pool_set_wait_limit": (ctypes.c_int, [_vp, _u64, _vp]),
+    "oilbird_pool_stall_selftest": (ctypes.c_int, [_vp, _vp]),
+    "oilbird_pool_check_guards": (ctypes.c_int, [_vp, _vp]),
     "oilbird_pool_read_rows": (ctypes.c_int, [_vp, _i64, _i64, _vp, _vp, _vp]),
     "oilbird_pool_read_codes": (ctypes.c_int, [_vp, _i64, _i64, _vp, _vp]),
     "oilbird_pool_read_traces": (_i32, [_vp, _vp, _vp, _vp, _i32]),
@@ -142,6 +146,18 @@ SYMBOLS = {
 }
 
 _lib = None
+# Pools made without an explicit debug_guards argument take this (the GPU tests switch it on).
+DEFAULT_DEBUG_GUARDS = False
+GUARD_FAILURES: list = []      # pools whose guard check failed inside __del__
+
+
+def _torch_empty(shape, dtype, device):
+    return torch.empty(shape, dtype=dtype, device=device)
+
+
+# Every result tensor this module creates comes from ALLOC(shape, dtype, device); the GPU
+# tests replace it with an allocator that surrounds each tensor with sentinel bytes.
+ALLOC = _torch_empty
 
 
 def lib() -> ctypes.CDLL:
@@ -164,7 +180,8 @@ class OilbirdError(RuntimeError):
     def __init__(self, code: int, where: str):
         L = lib()
         msg = L.oilbird_strerror(code).decode()
-        if code == ECUDA or code == ENOMEM:
+        if code in (ECUDA, ENOMEM, EGUARD) or (code == EINVAL and "aligned" in
+                                                  L.oilbird_last_cuda_error().decode()):
             msg += " (" + L.oilbird_last_cuda_error().decode() + ")"
         super().__init__(f"{where}: {msg} [{code}]")
         self.code = code
@@ -222,12 +239,11 @@ class QueryOut:
 
     @staticmethod
     def empty(nq: int, k: int, L: int, device) -> "QueryOut":
-        kw = dict(device=device)
-        o = QueryOut(torch.empty((nq, k), dtype=torch.int32, **kw),
-                     torch.empty((nq, k), dtype=torch.float32, **kw),
-                     torch.empty((nq,), dtype=torch.int32, **kw),
-                     torch.empty((nq, k), dtype=torch.int32, **kw),
-                     torch.empty((nq, k, L), dtype=torch.int32, **kw))
+        o = QueryOut(ALLOC((nq, k), torch.int32, device),
+                     ALLOC((nq, k), torch.float32, device),
+                     ALLOC((nq,), torch.int32, device),
+                     ALLOC((nq, k), torch.int32, device),
+                     ALLOC((nq, k, L), torch.int32, device))
         o._c = CQueryOut(o.idx.data_ptr(), o.score.data_ptr(), o.fired.data_ptr(),
                          o.cont_len.data_ptr(), o.cont_tok.data_ptr())
         return o
@@ -282,18 +298,22 @@ class Pool:
 
     def __init__(self, d: int, capacity_rows: int, *, max_traces: int = 0, max_nq: int = 0,
                  max_k: int = 0, max_append: int = 0, device: int = 0, use_torch_arena=False,
-                 key_format: str = "bf16"):
-        """key_format: "bf16" (the paper's store) or "e4m3" (8-bit keys, one scale per row)."""
+                 key_format: str = "bf16", debug_guards: bool | None = None):
+        """key_format: "bf16" (the paper's store) or "e4m3" (8-bit keys, one scale per row).
+        debug_guards: sentinel bytes behind every array of the pool (check_guards() verifies
+        them); None takes the module default DEFAULT_DEBUG_GUARDS."""
         self._L = lib()
         if key_format not in ("bf16", "e4m3"):
             raise ValueError("key_format must be 'bf16' or 'e4m3'")
         self.key_format = key_format
+        self.debug_guards = DEFAULT_DEBUG_GUARDS if debug_guards is None else bool(debug_guards)
         if not torch.cuda.is_available():
             raise RuntimeError("oilbird pool needs a CUDA device; there is no CPU fallback")
         self.d, self.device = int(d), int(device)
         cfg = PoolConfig(d=d, capacity_rows=capacity_rows, max_traces=max_traces, max_nq=max_nq,
                          max_k=max_k, max_append=max_append, device=device,
-                         flags=KEYS_E4M3 if key_format == "e4m3" else 0,
+                         flags=(KEYS_E4M3 if key_format == "e4m3" else 0) |
+                               (DEBUG_GUARDS if self.debug_guards else 0),
                          arena=None, arena_bytes=0)
         self._arena = None
         if use_torch_arena:
@@ -311,9 +331,36 @@ class Pool:
     def close(self) -> None:
         h, self._h = getattr(self, "_h", None), None
         if h:
+            rc = OK
+            if self.debug_guards:
+                rc = self._L.oilbird_pool_check_guards(h, _stream_ptr(None))
             self._L.oilbird_pool_destroy(h)
+            _check(rc, "oilbird_pool_check_guards (at close)")
 
-    __del__ = close
+    def __del__(self):
+        try:
+            self.close()
+        except OilbirdError:
+            import traceback
+            traceback.print_exc()
+            GUARD_FAILURES.append(self)
+
+    def check_guards(self, stream=None) -> None:
+        """Raises OilbirdError(EGUARD) if a kernel wrote behind one of the pool's arrays."""
+        _check(self._L.oilbird_pool_check_guards(self._h, _stream_ptr(stream)),
+               "oilbird_pool_check_guards")
+
+    def set_wait_limit(self, limit_ns: int, stream=None) -> None:
+        _check(self._L.oilbird_pool_set_wait_limit(self._h, int(limit_ns), _stream_ptr(stream)),
+               "oilbird_pool_set_wait_limit")
+
+    def stall_selftest(self, stream=None) -> None:
+        _check(self._L.oilbird_pool_stall_selftest(self._h, _stream_ptr(stream)),
+               "oilbird_pool_stall_selftest")
+
+    def status(self, stream=None) -> int:
+        """The code of oilbird_pool_status: OK, or ESTALL after a device-side wait gave up."""
+        return int(self._L.oilbird_pool_status(self._h, None, _stream_ptr(stream)))
 
     def __len__(self) -> int:
         return int(self._L.oilbird_pool_size(self._h))
@@ -359,7 +406,7 @@ class Pool:
         """Local rows (int32) -> global positions (int64); -1 stays -1."""
         assert idx.is_cuda and idx.dtype == torch.int32 and idx.is_contiguous()
         if out is None:
-            out = torch.empty(idx.shape, dtype=torch.int64, device=idx.device)
+            out = ALLOC(tuple(idx.shape), torch.int64, idx.device)
         _check(self._L.oilbird_pool_to_global(self._h, idx.data_ptr(), out.data_ptr(),
                                               idx.numel(), _stream_ptr(stream)),
                "oilbird_pool_to_global")
@@ -588,12 +635,11 @@ class Ring:
         nq = q.shape[0]
         assert anchors.is_cuda and anchors.dtype == torch.int32 and anchors.numel() == nq
         if out is None:
-            kw = dict(device=self._dev)
-            out = RingOut(torch.empty((nq, m), dtype=torch.int32, **kw),
-                          torch.empty((nq, m), dtype=torch.float32, **kw),
-                          torch.empty((nq,), dtype=torch.int32, **kw),
-                          torch.empty((nq, m, self.max_rollout), dtype=torch.int32, **kw),
-                          torch.empty((nq, m), dtype=torch.int32, **kw))
+            out = RingOut(ALLOC((nq, m), torch.int32, self._dev),
+                          ALLOC((nq, m), torch.float32, self._dev),
+                          ALLOC((nq,), torch.int32, self._dev),
+                          ALLOC((nq, m, self.max_rollout), torch.int32, self._dev),
+                          ALLOC((nq, m), torch.int32, self._dev))
         co = CRingOut(out.slot.data_ptr(), out.score.data_ptr(), out.count.data_ptr(),
                       out.rollout.data_ptr(), out.rollout_len.data_ptr())
         _check(self._L.oilbird_ring_query(self._h, q.data_ptr(), anchors.data_ptr(), nq, int(m),
@@ -644,11 +690,11 @@ def merge_chains(tree_tok: torch.Tensor, tree_parent: torch.Tensor, n_nodes: tor
     ne, Le = (extra_tok.shape[1], extra_tok.shape[2]) if extra_tok is not None else (0, 1)
     for t in (tree_tok, tree_parent, n_nodes, sem_tok, sem_len, extra_tok, extra_len):
         assert t is None or (t.is_cuda and t.dtype == torch.int32 and t.is_contiguous())
-    depth = torch.empty((nq, max_nodes), dtype=torch.int32, device=dev)
-    mask = torch.empty((nq, max_nodes), dtype=torch.int64, device=dev)
-    status = torch.empty((nq, k + ne), dtype=torch.int32, device=dev)
-    bought = torch.empty_like(status)
-    walked = torch.empty_like(status)
+    depth = ALLOC((nq, max_nodes), torch.int32, dev)
+    mask = ALLOC((nq, max_nodes), torch.int64, dev)
+    status = ALLOC((nq, k + ne), torch.int32, dev)
+    bought = ALLOC((nq, k + ne), torch.int32, dev)
+    walked = ALLOC((nq, k + ne), torch.int32, dev)
     mp = MergeParams(budget, max_nodes, min_len, int(bool(root_attached)))
     ptr = lambda t: None if t is None else t.data_ptr()
     _check(lib().oilbird_merge_chains(nq, ptr(sem_tok), ptr(sem_len), k, L, ptr(extra_tok),

@@ -24,8 +24,7 @@ append_kernel(const uint16_t* __restrict__ states, const int32_t* __restrict__ t
               int32_t* __restrict__ trace_id, int64_t row0, int32_t trace,
               int32_t* __restrict__ trace_end, uint64_t* __restrict__ trace_tag, uint64_t tag,
               int64_t* __restrict__ trace_gbase, int64_t gbase, int set_tag, DeviceStats* stats) {
-  pdl_launch_dependents();
-  pdl_wait();   // earlier queries may still be reading the trace table and token stream
+  pdl_enter();   // earlier queries may still be reading the trace table and token stream
   if (blockIdx.x == 0 && threadIdx.x == 0) {
     trace_end[trace] = (int32_t)(row0 + n);
     if (set_tag) { trace_tag[trace] = tag; trace_gbase[trace] = gbase; }
@@ -53,8 +52,7 @@ append_bulk_kernel(const uint16_t* __restrict__ states, const int32_t* __restric
                    int32_t* __restrict__ trace_end, uint64_t* __restrict__ trace_tag, uint64_t tag,
                    int64_t* __restrict__ trace_gbase, int64_t gbase, int set_tag,
                    DeviceStats* stats) {
-  pdl_launch_dependents();
-  pdl_wait();
+  pdl_enter();
   if (blockIdx.x == 0 && threadIdx.x == 0) {
     trace_end[trace] = (int32_t)(row0 + n);
     if (set_tag) { trace_tag[trace] = tag; trace_gbase[trace] = gbase; }
@@ -88,8 +86,7 @@ append_bulk2_kernel(const uint16_t* __restrict__ states, const int32_t* __restri
                     int64_t* __restrict__ trace_gbase, int64_t gbase, int set_tag,
                     DeviceStats* stats) {
   constexpr int kHeld = 2;
-  pdl_launch_dependents();
-  pdl_wait();
+  pdl_enter();
   if (blockIdx.x == 0 && threadIdx.x == 0) {
     trace_end[trace] = (int32_t)(row0 + n);
     if (set_tag) { trace_tag[trace] = tag; trace_gbase[trace] = gbase; }
@@ -128,8 +125,7 @@ __global__ void __launch_bounds__(kNormThreads)
 qnorm_kernel(const uint16_t* __restrict__ q, int nq, int d, uint16_t* __restrict__ qn,
              int32_t* __restrict__ q_valid, DeviceStats* stats, float* __restrict__ xchg,
              int n_xchg) {
-  pdl_launch_dependents();
-  pdl_wait();
+  pdl_enter();
   // the tensor scan's cross-CTA threshold exchange starts every call at -inf
   for (int i = blockIdx.x * kNormThreads + threadIdx.x; i < n_xchg; i += gridDim.x * kNormThreads)
     xchg[i] = -INFINITY;
@@ -152,15 +148,9 @@ cudaError_t launch_append(const uint16_t* states, const int32_t* tokens, int64_t
                           uint16_t* keys, int32_t* tok, int32_t* trace_id, int64_t row0,
                           int32_t trace, int32_t* trace_end, uint64_t* trace_tag, uint64_t tag,
                           int64_t* trace_gbase, int64_t gbase, int set_tag, DeviceStats* stats,
-                          cudaStream_t st) {
+                          int32_t num_sms, cudaStream_t st) {
   // from a few rows per resident block on, the prefetching kernel
-  static int sms = 0;
-  if (!sms) {
-    int dev = 0;
-    cudaGetDevice(&dev);
-    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-  }
-  const int64_t bulk_grid = (int64_t)sms * 4;
+  const int64_t bulk_grid = (int64_t)num_sms * 4;
   if (n >= bulk_grid * 4) {
     if (d <= 4096)
       return launch_pdl(append_bulk2_kernel, dim3((unsigned)bulk_grid), dim3(kNormThreads), 0, st,

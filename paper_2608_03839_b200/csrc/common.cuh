@@ -61,32 +61,50 @@ __device__ __forceinline__ unsigned long long ld_acquire_u64(const unsigned long
   return v;
 }
 
+// The pool's limit for device-side waits (two seconds unless the caller set another).
+__device__ __forceinline__ unsigned long long wait_limit_ns(const DeviceStats* stats) {
+  const unsigned long long v = *reinterpret_cast<const volatile unsigned long long*>(&stats->wait_limit_ns);
+  return v ? v : kDefaultWaitNs;
+}
+
 // A scan whose first CTAs append the step's rows: wait until all of them are in (every
-// appending CTA adds one to *ready after its row).  Bounded: after about two seconds the
-// pool's `stalled` flag is raised and the caller carries on (the status call reports it).
-__device__ __forceinline__ void wait_fused_rows(const FusedAppend& fa, DeviceStats* stats) {
-  unsigned long long t0 = 0;
-  for (uint32_t spin = 0; ld_acquire_u64(fa.ready) < fa.target; ++spin) {
-    if (spin == 0) asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t0));
-    if ((spin & 255u) == 255u) {
+// appending CTA adds one to *ready after its row).  Bounded: after the pool's wait limit the
+// `stalled` flag is raised and the caller carries on (the status call reports it).
+__device__ __forceinline__ void wait_fused_rows(const unsigned long long* ready,
+                                                unsigned long long target, DeviceStats* stats) {
+  unsigned long long t0 = 0, limit = 0;
+  for (uint32_t spin = 0; ld_acquire_u64(ready) < target; ++spin) {
+    if (spin == 0) {
+      asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t0));
+      limit = wait_limit_ns(stats);
+    }
+    if ((spin & 15u) == 15u) {
       unsigned long long t1;
       asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t1));
-      if (t1 - t0 > 2000000000ull) { atomicExch(&stats->stalled, 1); break; }
+      if (t1 - t0 > limit) { atomicExch(&stats->stalled, 1); break; }
     }
     __nanosleep(64);
   }
 }
+__device__ __forceinline__ void wait_fused_rows(const FusedAppend& fa, DeviceStats* stats) {
+  wait_fused_rows(fa.ready, fa.target, stats);
+}
 
 // ---------------------------------------------------- programmatic launch ------
-// Every kernel of the library is launched with programmatic stream serialization: its
-// blocks may be scheduled while the previous kernel of the stream is still draining, which
-// hides the launch latency between the three or four kernels of a step.  pdl_wait() must
-// come before the first access to anything an earlier kernel wrote (it waits for that
-// kernel to finish and its writes to be visible); both are no-ops for a plain launch.
-__device__ __forceinline__ void pdl_launch_dependents() {
+// The kernels of a step may be launched with programmatic stream serialization (see
+// launch_pdl in internal.h): a kernel's blocks can then be scheduled, and run their set-up,
+// while the previous kernel of the stream is still working, which hides the launch latency
+// between the three or four kernels of a step.  pdl_enter() must come before the first
+// access to anything an earlier kernel wrote: it waits for that kernel to finish and its
+// writes to be visible, and only then lets the NEXT kernel of the stream be scheduled.
+// Releasing the successor after the wait, not before it, bounds the chain: at most two
+// grids are on the GPU at any time, the one that works and the one that is set up and
+// waiting for it; a kernel never sits behind a predecessor that is itself still waiting.
+// Both instructions are no-ops for a plain launch.
+__device__ __forceinline__ void pdl_enter() {
+  asm volatile("griddepcontrol.wait;" ::: "memory");
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 }
-__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 
 // ------------------------------------------------------------------ warp ops ---
 __device__ __forceinline__ u64 shfl_xor_u64(u64 v, int m) {

@@ -13,7 +13,26 @@ __host__ __device__ inline int next_pow2(int v) {
   return p;
 }
 
-// Launch with programmatic stream serialization (see pdl_wait() in common.cuh).
+// ---- programmatic launches ---------------------------------------------------------
+// Whether this process may chain kernels with programmatic stream serialization at all:
+// only when the driver loads modules eagerly (CUDA_MODULE_LOADING=EAGER before CUDA starts).
+// With lazy loading, the first steps of a process were seen to dead-lock now and then on
+// the largest configuration while kernels of the chain were resident and waiting; the
+// mechanism inside the driver was never established, so under lazy loading (or when the
+// mode cannot be read) every launch of the library is a plain one.  Evaluated once.
+bool pdl_process_ok();
+// Set by an entry point for the calls it is about to make: plain launches for this call
+// (scans that run for milliseconds gain nothing from overlapping a 5 us neighbour).
+extern thread_local bool tl_pdl_off;
+struct PdlScope {
+  bool prev;
+  explicit PdlScope(bool off) : prev(tl_pdl_off) { tl_pdl_off = tl_pdl_off || off; }
+  ~PdlScope() { tl_pdl_off = prev; }
+};
+
+// Launch, with programmatic stream serialization where the policy above allows it (see
+// pdl_enter() in common.cuh; for a plain launch the kernel's griddepcontrol instructions
+// are no-ops).
 template <typename... KArgs, typename... Args>
 inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem,
                               cudaStream_t st, Args&&... args) {
@@ -25,23 +44,29 @@ inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, s
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[0].val.programmaticStreamSerializationAllowed = 1;
-  cfg.attrs = attr;
-  cfg.numAttrs = 1;
+  const bool pdl = !tl_pdl_off && pdl_process_ok();
+  cfg.attrs = pdl ? attr : nullptr;
+  cfg.numAttrs = pdl ? 1 : 0;
   return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
 }
 
-// With lazy module loading (the CUDA default) a kernel is loaded at its first launch, and
-// that load can wait for the device to go idle.  The kernels of a step are chained with
-// programmatic launches: a kernel may already be resident and waiting for its predecessor
-// when the host reaches the first launch of the next one.  On B200 with driver 580 this
-// dead-locked about three process starts in ten on the largest configuration (the first
-// steps of a process never finished; CUDA_MODULE_LOADING=EAGER: none in ten).  So every
-// kernel of the library is loaded explicitly, once per device, before any of them is
-// launched: asking for a function's attributes loads it.
+// Everything a kernel needs before its first launch is done once per device, before any
+// kernel of the library is launched there (oilbird_pool_create and the first use of the
+// ring, merge, shard and static entry points): asking for a function's attributes loads
+// it (with lazy module loading a kernel is otherwise loaded at its first launch, which can
+// wait for the device to go idle), and kernels with dynamic shared memory get their limit
+// raised to the device's maximum here instead of at every launch.
 template <typename K>
-inline cudaError_t preload_kernel(K kernel) {
+inline cudaError_t preload_kernel(K kernel, bool dynamic_smem = false) {
   cudaFuncAttributes attr;
-  return cudaFuncGetAttributes(&attr, kernel);
+  cudaError_t e = cudaFuncGetAttributes(&attr, kernel);
+  if (e != cudaSuccess || !dynamic_smem) return e;
+  int dev = 0, optin = 0;
+  if ((e = cudaGetDevice(&dev)) != cudaSuccess) return e;
+  if ((e = cudaDeviceGetAttribute(&optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev)) != cudaSuccess)
+    return e;
+  const int room = optin - (int)attr.sharedSizeBytes;
+  return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, room > 0 ? room : 0);
 }
 cudaError_t preload_append_kernels();
 cudaError_t preload_evict_kernels();
@@ -62,7 +87,12 @@ struct DeviceStats {
   unsigned long long nonfinite_queries;
   int stalled;
   int pad;
+  // how long a device-side wait may spin before it gives up, in nanoseconds of %globaltimer
+  // (0 = kDefaultWaitNs); survives reset()
+  unsigned long long wait_limit_ns;
 };
+constexpr unsigned long long kDefaultWaitNs = 2000000000ull;
+constexpr size_t kStatsCounterBytes = 24;      // the part of DeviceStats that reset() clears
 
 // Views of the pool's device arrays handed to the kernels.
 struct PoolView {
@@ -81,6 +111,10 @@ struct GatherParams {
   float tier_thr[OILBIRD_MAX_TIERS];
   int32_t tier_depth[OILBIRD_MAX_TIERS];
 };
+
+// Range checks of the retrieval parameters shared by every query entry point; fills gp.
+int check_query_params(int32_t nq, int32_t max_nq, int32_t max_k, const oilbird_query_params* pr,
+                       GatherParams* gp);
 
 // The append of one serving step, done by the first n CTAs of the CUDA-core scan itself
 // instead of by a kernel of its own (n == 0: nothing to append).  CTA i normalises row i
@@ -109,7 +143,7 @@ cudaError_t launch_append(const uint16_t* states, const int32_t* tokens, int64_t
                           uint16_t* keys, int32_t* tok, int32_t* trace_id, int64_t row0,
                           int32_t trace, int32_t* trace_end, uint64_t* trace_tag, uint64_t tag,
                           int64_t* trace_gbase, int64_t gbase, int set_tag, DeviceStats* stats,
-                          cudaStream_t st);
+                          int32_t num_sms, cudaStream_t st);
 
 // Row sharding over several pools: local rows -> caller-assigned global positions, and the
 // merge of the shards' gathered query results (see shard.cu).
@@ -196,6 +230,13 @@ cudaError_t launch_scan_tc(TcCache* cache, const PoolView& pv, int32_t q0, int32
                            int32_t nq_total, int32_t k, int32_t kk, const uint64_t* exclude_tag,
                            unsigned long long* partial, DeviceStats* stats, float* xchg,
                            int32_t num_sms, size_t smem_limit, int32_t* n_lists, cudaStream_t st);
+
+// Exercises the give-up path of the two kinds of device-side wait the library has (the
+// fused append's row counter and an mbarrier of the tensor scan) on a counter nobody
+// advances and a barrier nobody arrives at: both waits run out after the pool's wait limit,
+// raise `stalled` and return.  One small CTA; nothing else is touched.
+cudaError_t launch_stall_selftest(const unsigned long long* ready, DeviceStats* stats,
+                                  cudaStream_t st);
 
 // a3 (final merge) + a4 + a5 + a6: one CTA per query.
 cudaError_t launch_merge_gather(const PoolView& pv, const unsigned long long* partial,

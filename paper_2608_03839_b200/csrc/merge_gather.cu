@@ -87,8 +87,7 @@ merge_gather_kernel(PoolView pv, const u64* __restrict__ partial, int n_lists, i
   __shared__ int32_t s_len[OILBIRD_MAX_K];
   const int q = blockIdx.x;
   const int k = gp.k;
-  pdl_launch_dependents();
-  pdl_wait();   // the scan's candidate lists
+  pdl_enter();   // the scan's candidate lists
   const int valid = q_valid[q];       // consumed after the merge: the load overlaps it
   if (kk == 32) merge_lists<1>(partial, n_lists, nq, q, k, scratch, s_best);
   else if (kk == 64) merge_lists<2>(partial, n_lists, nq, q, k, scratch, s_best);
@@ -113,8 +112,7 @@ gather_only_kernel(PoolView pv, const int32_t* __restrict__ idx, const float* __
   __shared__ float s_score[OILBIRD_MAX_K];
   __shared__ int32_t s_len[OILBIRD_MAX_K];
   const int q = blockIdx.x, k = gp.k;
-  pdl_launch_dependents();
-  pdl_wait();
+  pdl_enter();
   for (int j = threadIdx.x; j < k; j += blockDim.x) {
     s_idx[j] = idx[(size_t)q * k + j];
     s_score[j] = score[(size_t)q * k + j];

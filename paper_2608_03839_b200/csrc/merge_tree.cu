@@ -54,8 +54,7 @@ merge_tree_kernel(int nq, const int32_t* __restrict__ sem_tok, const int32_t* __
   __shared__ int32_t s_chain[kMergeTreeWarps][OILBIRD_MAX_CONT_LEN];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int q = blockIdx.x * kMergeTreeWarps + warp;
-  pdl_launch_dependents();
-  pdl_wait();
+  pdl_enter();
   if (q >= nq) return;
   int32_t* tok = s_tok[warp];
   int32_t* par = s_par[warp];
@@ -65,7 +64,10 @@ merge_tree_kernel(int nq, const int32_t* __restrict__ sem_tok, const int32_t* __
   n = n < 1 ? 1 : (n > max_nodes ? max_nodes : n);
   for (int j = lane; j < kMaxNodes; j += 32) {
     tok[j] = j < n ? tree_tok[(size_t)q * max_nodes + j] : -1;
-    par[j] = j < n ? tree_parent[(size_t)q * max_nodes + j] : -1;
+    // parents come from caller memory and index shared memory below: one that is not
+    // another node of the tree detaches its node (parent -1) instead of being followed
+    int p = (j >= 1 && j < n) ? tree_parent[(size_t)q * max_nodes + j] : -1;
+    par[j] = (p >= 0 && p < n && p != j) ? p : -1;
   }
   __syncwarp();
   int left = mp.budget;

@@ -1,6 +1,7 @@
 // C-ABI layer: argument checks, memory layout of the pool in HBM, host-side trace
 // bookkeeping and the launch sequence of each entry point.  No arithmetic of the
 // method lives here.
+#include <cuda.h>
 #include <math.h>
 #include <stdio.h>
 #include <string.h>
@@ -16,6 +17,25 @@ using namespace oilbird;
 static thread_local char g_cuda_err[256] = "";
 
 namespace oilbird {
+thread_local bool tl_pdl_off = false;
+
+// The driver's module loading mode, read once (CUDA must be initialised: every caller has
+// launched or is about to launch).  Anything but "eager" switches programmatic launches off.
+bool pdl_process_ok() {
+  static const bool ok = [] {
+    typedef CUresult (*GetModeFn)(CUmoduleLoadingMode*);
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuModuleGetLoadingMode", &fn, cudaEnableDefault, &qres) !=
+            cudaSuccess || qres != cudaDriverEntryPointSuccess || !fn)
+      return false;
+    CUmoduleLoadingMode mode;
+    if (((GetModeFn)fn)(&mode) != CUDA_SUCCESS) return false;
+    return mode == CU_MODULE_EAGER_LOADING;
+  }();
+  return ok;
+}
+
 cudaError_t preload_all_kernels() {
   static std::mutex mu;
   static bool done[64] = {};
@@ -24,6 +44,8 @@ cudaError_t preload_all_kernels() {
   if (e != cudaSuccess) return e;
   std::lock_guard<std::mutex> lock(mu);
   if (dev >= 0 && dev < 64 && done[dev]) return cudaSuccess;
+  if ((e = cudaFree(nullptr)) != cudaSuccess) return e;      // the context exists from here on
+  (void)pdl_process_ok();
   if ((e = preload_append_kernels()) != cudaSuccess) return e;
   if ((e = preload_evict_kernels()) != cudaSuccess) return e;
   if ((e = preload_merge_kernels()) != cudaSuccess) return e;
@@ -56,16 +78,24 @@ constexpr int kMaxProfile = 4096;
 size_t align_up(size_t v) { return (v + kAlign - 1) / kAlign * kAlign; }
 
 // Byte offsets of every device array inside one allocation.
+constexpr int kMaxGuards = 24;
 struct Layout {
   size_t keys, tok, trace_id, trace_end, trace_tag, trace_gbase, qn, q_valid, partial, stats;
   size_t xchg;
   size_t q_stage, ex_stage, st_stage, tok_stage, stage_end, fuse_ready, scales;
   size_t total;
+  // OILBIRD_DEBUG_GUARDS: sentinel bytes [g_lo, g_hi) behind every array (from its last
+  // byte to the next array's first), named after the array they follow
+  int n_guards;
+  size_t g_lo[kMaxGuards], g_hi[kMaxGuards];
+  const char* g_name[kMaxGuards];
 };
+constexpr unsigned char kGuardByte = 0xA5;
 
 struct Resolved {
   int32_t d, max_traces, max_nq, max_k, max_append, max_lists;
   int32_t e4m3;              // keys are E4M3 codes with one scale per row
+  int32_t guards;            // guard zones between the arrays (debugging aid)
   int64_t capacity;
 };
 
@@ -73,8 +103,9 @@ bool resolve(const oilbird_pool_config* c, int num_sms, Resolved* r) {
   if (!c) return false;
   if (c->d < 8 || c->d > 16384 || (c->d % 8) != 0) return false;
   if (c->capacity_rows < 1 || c->capacity_rows > 2147483000LL) return false;
-  if (c->flags & ~(uint32_t)OILBIRD_KEYS_E4M3) return false;
+  if (c->flags & ~(uint32_t)(OILBIRD_KEYS_E4M3 | OILBIRD_DEBUG_GUARDS)) return false;
   r->e4m3 = (c->flags & OILBIRD_KEYS_E4M3) ? 1 : 0;
+  r->guards = (c->flags & OILBIRD_DEBUG_GUARDS) ? 1 : 0;
   if (r->e4m3 && (c->d % 16) != 0) return false;      // 16 codes per 16-byte load
   r->d = c->d;
   r->capacity = c->capacity_rows;
@@ -95,28 +126,42 @@ bool resolve(const oilbird_pool_config* c, int num_sms, Resolved* r) {
 Layout make_layout(const Resolved& r) {
   Layout L;
   size_t off = 0;
-  auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes); return o; };
+  L.n_guards = 0;
+  bool guards = r.guards != 0;
+  auto take = [&](size_t bytes, const char* name) {
+    const size_t o = off;
+    off = align_up(off + bytes);
+    if (guards && L.n_guards < kMaxGuards) {
+      L.g_lo[L.n_guards] = o + bytes;
+      off += kAlign;                       // one more aligned block of sentinel bytes
+      L.g_hi[L.n_guards] = off;
+      L.g_name[L.n_guards++] = name;
+    }
+    return o;
+  };
   const size_t nq_pad = (size_t)(r.max_nq + 15) / 16 * 16;
   const size_t k_pad = (size_t)list_len(r.max_k);
-  L.keys = take((size_t)r.capacity * r.d * (r.e4m3 ? 1 : 2));
-  L.scales = take(r.e4m3 ? (size_t)r.capacity * 4 : 0);
-  L.tok = take((size_t)r.capacity * 4);
-  L.trace_id = take((size_t)r.capacity * 4);
-  L.trace_end = take((size_t)r.max_traces * 4);
-  L.trace_tag = take((size_t)r.max_traces * 8);
-  L.trace_gbase = take((size_t)r.max_traces * 8);
-  L.qn = take(nq_pad * r.d * 2);
-  L.q_valid = take(nq_pad * 4);
-  L.partial = take((size_t)r.max_lists * r.max_nq * k_pad * 8);
-  L.stats = take(sizeof(DeviceStats));
-  L.fuse_ready = take(8);
-  L.xchg = take((size_t)kTcXchgFloats * 4);
+  L.keys = take((size_t)r.capacity * r.d * (r.e4m3 ? 1 : 2), "keys");
+  L.scales = take(r.e4m3 ? (size_t)r.capacity * 4 : 0, "scales");
+  L.tok = take((size_t)r.capacity * 4, "tokens");
+  L.trace_id = take((size_t)r.capacity * 4, "trace ids");
+  L.trace_end = take((size_t)r.max_traces * 4, "trace ends");
+  L.trace_tag = take((size_t)r.max_traces * 8, "trace tags");
+  L.trace_gbase = take((size_t)r.max_traces * 8, "trace global bases");
+  L.qn = take(nq_pad * r.d * 2, "normalised queries");
+  L.q_valid = take(nq_pad * 4, "query-valid flags");
+  L.partial = take((size_t)r.max_lists * r.max_nq * k_pad * 8, "candidate lists");
+  L.stats = take(sizeof(DeviceStats), "counters");
+  L.fuse_ready = take(8, "fused-append counter");
+  L.xchg = take((size_t)kTcXchgFloats * 4, "threshold exchange");
   // staging for the *_host variants (adjacent: query_host/step_host fill them with one copy)
-  L.q_stage = take((size_t)r.max_nq * r.d * 2);
-  L.ex_stage = take((size_t)r.max_nq * 8);
-  L.st_stage = take((size_t)r.max_append * r.d * 2);
-  L.tok_stage = take((size_t)r.max_append * 4);
-  L.stage_end = off;
+  guards = false;                          // no sentinels inside the one-copy staging block
+  L.q_stage = take((size_t)r.max_nq * r.d * 2, "");
+  L.ex_stage = take((size_t)r.max_nq * 8, "");
+  L.st_stage = take((size_t)r.max_append * r.d * 2, "");
+  guards = r.guards != 0;
+  L.tok_stage = take((size_t)r.max_append * 4, "host staging");
+  L.stage_end = L.tok_stage + align_up((size_t)r.max_append * 4);   // (a guard may follow)
   L.total = off;
   return L;
 }
@@ -174,6 +219,7 @@ const char* oilbird_strerror(int code) {
     case OILBIRD_ENOMEM: return "out of memory";
     case OILBIRD_ECUDA: return "CUDA error";
     case OILBIRD_ESTALL: return "a bounded device-side wait gave up";
+    case OILBIRD_EGUARD: return "a guard zone of the pool's memory was overwritten";
     default: return "unknown error";
   }
 }
@@ -250,6 +296,8 @@ int oilbird_pool_create(oilbird_pool_t** out, const oilbird_pool_config* cfg) {
   p->fuse_target = 0;
   cudaError_t e = cudaMemset(p->stats, 0, sizeof(DeviceStats));
   if (e == cudaSuccess) e = cudaMemset(p->fuse_ready, 0, 8);
+  for (int g = 0; g < lay.n_guards && e == cudaSuccess; ++g)
+    e = cudaMemset(p->base + lay.g_lo[g], kGuardByte, lay.g_hi[g] - lay.g_lo[g]);
   if (e != cudaSuccess) {
     if (p->owns_mem) cudaFree(p->base);
     delete p;
@@ -278,7 +326,7 @@ int oilbird_pool_destroy(oilbird_pool_t* p) {
 int oilbird_pool_reset(oilbird_pool_t* p, void* stream) {
   if (!p) return OILBIRD_EINVAL;
   CU(cudaSetDevice(p->device));
-  CU(cudaMemsetAsync(p->stats, 0, sizeof(DeviceStats), (cudaStream_t)stream));
+  CU(cudaMemsetAsync(p->stats, 0, kStatsCounterBytes, (cudaStream_t)stream));   // not the wait limit
   p->n_rows = 0;
   p->t_start.clear(); p->t_end.clear(); p->t_tag.clear(); p->t_gbase.clear();
   return OILBIRD_OK;
@@ -287,6 +335,21 @@ int oilbird_pool_reset(oilbird_pool_t* p, void* stream) {
 int64_t oilbird_pool_size(const oilbird_pool_t* p) { return p ? p->n_rows : 0; }
 int32_t oilbird_pool_num_traces(const oilbird_pool_t* p) { return p ? (int32_t)p->t_start.size() : 0; }
 int64_t oilbird_pool_launch_count(const oilbird_pool_t* p) { return p ? p->launches : 0; }
+
+// The kernels read bf16 rows with 16-byte vector loads and the integer arrays word by word;
+// a misaligned pointer would fault on the device, so it is turned away here.
+static bool aligned(const void* p, uintptr_t a) { return ((uintptr_t)p & (a - 1)) == 0; }
+static int misaligned(const char* what) {
+  snprintf(g_cuda_err, sizeof g_cuda_err, "%s is not aligned as the header requires", what);
+  return OILBIRD_EINVAL;
+}
+
+// Scans of pools this large run for about a millisecond and more: chaining their kernels
+// programmatically would gain a few microseconds on that, so they are launched plainly.
+constexpr int64_t kPdlMaxKeyBytes = 4ll << 30;
+static bool long_scan(const oilbird_pool* p) {
+  return p->n_rows * (int64_t)p->r.d * (p->r.e4m3 ? 1 : 2) > kPdlMaxKeyBytes;
+}
 
 // Host side of an append: checks, then the trace bookkeeping (enqueue-time truth).
 struct AppendPlan {
@@ -299,6 +362,8 @@ static int append_prepare(oilbird_pool_t* p, const void* states, const int32_t* 
                           uint64_t tag, uint32_t flags, AppendPlan* ap, bool* nothing) {
   *nothing = false;
   if (!p || n < 0 || (n > 0 && (!states || !tokens))) return OILBIRD_EINVAL;
+  if (n > 0 && !aligned(states, 16)) return misaligned("states");
+  if (n > 0 && !aligned(tokens, 4)) return misaligned("tokens");
   ap->open_new = (flags & OILBIRD_NEW_TRACE) || p->t_start.empty();
   if (n == 0 && !ap->open_new) { *nothing = true; return OILBIRD_OK; }
   if (p->n_rows + n > p->r.capacity) return OILBIRD_ECAPACITY;
@@ -333,6 +398,7 @@ static int append_impl(oilbird_pool_t* p, const void* states, const int32_t* tok
   int rc = append_prepare(p, states, tokens, n, tag, flags, &ap, &nothing);
   if (rc || nothing) return rc;
   CU(cudaSetDevice(p->device));
+  PdlScope plain(long_scan(p));
   const int64_t gbase = global_row >= 0 ? global_row : ap.row0;
   cudaError_t e =
       p->r.e4m3
@@ -342,7 +408,7 @@ static int append_impl(oilbird_pool_t* p, const void* states, const int32_t* tok
                                (cudaStream_t)stream)
           : launch_append((const uint16_t*)states, tokens, n, p->r.d, p->keys, p->tok,
                           p->trace_id, ap.row0, ap.trace, p->trace_end, p->trace_tag, tag,
-                          p->trace_gbase, gbase, ap.open_new ? 1 : 0, p->stats,
+                          p->trace_gbase, gbase, ap.open_new ? 1 : 0, p->stats, p->num_sms,
                           (cudaStream_t)stream);
   if (e != cudaSuccess) {
     append_rollback(p, ap);
@@ -418,11 +484,14 @@ int oilbird_pool_to_global(oilbird_pool_t* p, const int32_t* idx, int64_t* globa
   return OILBIRD_OK;
 }
 
-static int check_params(const oilbird_pool* p, int32_t nq, const oilbird_query_params* pr,
-                        GatherParams* gp) {
+}  // extern "C"
+
+namespace oilbird {
+int check_query_params(int32_t nq, int32_t max_nq, int32_t max_k, const oilbird_query_params* pr,
+                       GatherParams* gp) {
   if (!pr) return OILBIRD_EINVAL;
-  if (nq < 1 || nq > p->r.max_nq) return OILBIRD_EINVAL;
-  if (pr->k < 1 || pr->k > p->r.max_k) return OILBIRD_EINVAL;
+  if (nq < 1 || nq > max_nq) return OILBIRD_EINVAL;
+  if (pr->k < 1 || pr->k > max_k) return OILBIRD_EINVAL;
   if (pr->cont_len < 1 || pr->cont_len > OILBIRD_MAX_CONT_LEN) return OILBIRD_EINVAL;
   if (pr->offset < 0 || pr->offset > (1 << 20)) return OILBIRD_EINVAL;
   if (pr->depth_mode != OILBIRD_DEPTH_FIXED && pr->depth_mode != OILBIRD_DEPTH_TIERED)
@@ -439,6 +508,14 @@ static int check_params(const oilbird_pool* p, int32_t nq, const oilbird_query_p
   }
   return OILBIRD_OK;
 }
+}  // namespace oilbird
+
+extern "C" {
+
+static int check_params(const oilbird_pool* p, int32_t nq, const oilbird_query_params* pr,
+                        GatherParams* gp) {
+  return check_query_params(nq, p->r.max_nq, p->r.max_k, pr, gp);
+}
 
 static PoolView view_of(const oilbird_pool* p) {
   PoolView pv;
@@ -449,7 +526,9 @@ static PoolView view_of(const oilbird_pool* p) {
 
 static bool out_ok(const oilbird_query_out* o, bool need_idx) {
   if (!o || !o->fired || !o->cont_len || !o->cont_tok) return false;
-  return !need_idx || (o->idx && o->score);
+  if (!aligned(o->fired, 4) || !aligned(o->cont_len, 4) || !aligned(o->cont_tok, 4)) return false;
+  if (!need_idx) return true;
+  return o->idx && o->score && aligned(o->idx, 4) && aligned(o->score, 4);
 }
 
 // Key bytes up to which a batch of 3 to 16 queries goes to the warp-level tensor scan: it
@@ -460,14 +539,15 @@ constexpr int64_t kMmaMaxKeyBytes = 2ll << 30;
 // rate: only pools that the start-up dominates (8,192 rows x 4096: 33 us against 53)
 constexpr int64_t kMma16MaxKeyBytes = 128ll << 20;
 
-static int resolve_path(const oilbird_pool* p, const oilbird_query_params* pr, int32_t nq) {
+static int resolve_path(const oilbird_pool* p, const oilbird_query_params* pr, int32_t nq,
+                        int64_t n_rows) {
   // single-request decode streams keys through the CUDA cores; batches go to tcgen05,
   // small batches on pools of the paper's size to mma.sync
   if (pr->path != OILBIRD_PATH_AUTO) return pr->path;
   // (two queries on an 8-bit pool: the CUDA-core scan converts every code once per query and
   // is bound by that, 78 us against 63 at 268 MB of codes; below 128 MB its fused append
   // makes up for it)
-  if (nq <= 1 || (nq == 2 && !(p->r.e4m3 && p->n_rows * (int64_t)p->r.d >= (128ll << 20))))
+  if (nq <= 1 || (nq == 2 && !(p->r.e4m3 && n_rows * (int64_t)p->r.d >= (128ll << 20))))
     return OILBIRD_PATH_GEMV;
   if (p->r.e4m3) {
     // 8-bit pools have no tcgen05 scan: the warp-level tensor scan scores 8 or 16 queries
@@ -475,7 +555,7 @@ static int resolve_path(const oilbird_pool* p, const oilbird_query_params* pr, i
     return scan_mma_tiles(p->r.d, list_len(pr->k), nq, p->smem_limit, true) ? OILBIRD_PATH_MMA
                                                                              : OILBIRD_PATH_GEMV;
   }
-  const int64_t key_bytes = p->n_rows * (int64_t)p->r.d * 2;
+  const int64_t key_bytes = n_rows * (int64_t)p->r.d * 2;
   const int64_t mma_max = nq > 8 ? kMma16MaxKeyBytes : kMmaMaxKeyBytes;
   if (nq <= 16 && key_bytes <= mma_max) {
     // up to 8 queries in one pass of 8; 9 to 16 only where 16 fit in one pass
@@ -485,29 +565,44 @@ static int resolve_path(const oilbird_pool* p, const oilbird_query_params* pr, i
   return OILBIRD_PATH_TENSOR;
 }
 
+// Everything about a query that can be refused, checked before anything is enqueued (and,
+// for a step, before anything is appended): arguments, parameters, and whether the scan the
+// call resolves to exists for this pool.  Returns the scan through *path.
+static int check_query(const oilbird_pool* p, const void* q, int32_t nq,
+                       const oilbird_query_params* pr, const oilbird_query_out* out,
+                       int64_t n_rows, GatherParams* gp, int* path) {
+  if (!p || !q || !out_ok(out, true)) return OILBIRD_EINVAL;
+  if (!aligned(q, 16)) return misaligned("q");
+  int rc = check_params(p, nq, pr, gp);
+  if (rc) return rc;
+  if (pr->exclude_tag && !aligned(pr->exclude_tag, 8)) return misaligned("exclude_tag");
+  *path = resolve_path(p, pr, nq, n_rows);     // n_rows: the pool's size when the scan runs
+  if (*path == OILBIRD_PATH_TENSOR && p->r.e4m3) return OILBIRD_EINVAL;   // 16-bit pools only
+  if (*path == OILBIRD_PATH_MMA &&
+      !scan_mma_supports(p->r.d, list_len(pr->k), p->smem_limit, p->r.e4m3))
+    return OILBIRD_EINVAL;
+  if (*path == OILBIRD_PATH_TENSOR && !p->tc) {
+    snprintf(g_cuda_err, sizeof g_cuda_err, "tensor-core scan unavailable on this device");
+    return OILBIRD_ECUDA;
+  }
+  return OILBIRD_OK;
+}
+
 // fused: the step's append, to be done by the CUDA-core scan itself (the rows are already
 // counted in p->n_rows), or nullptr.
 static int query_impl(oilbird_pool_t* p, const void* q, int32_t nq, const oilbird_query_params* pr,
                       const oilbird_query_out* out, void* stream, const FusedAppend* fused) {
-  if (!p || !q || !out_ok(out, true)) return OILBIRD_EINVAL;
   GatherParams gp;
-  int rc = check_params(p, nq, pr, &gp);
+  int path = 0;
+  int rc = check_query(p, q, nq, pr, out, p ? p->n_rows : 0, &gp, &path);
   if (rc) return rc;
   CU(cudaSetDevice(p->device));
+  PdlScope plain(long_scan(p));
   cudaStream_t st = (cudaStream_t)stream;
   const int kk = list_len(pr->k);
   const int nq_pad = (nq + 15) / 16 * 16;
   PoolView pv = view_of(p);
   cudaError_t e;
-
-  const int path = resolve_path(p, pr, nq);
-  if (path == OILBIRD_PATH_TENSOR && p->r.e4m3) return OILBIRD_EINVAL;   // 16-bit pools only
-  if (path == OILBIRD_PATH_MMA && !scan_mma_supports(p->r.d, kk, p->smem_limit, p->r.e4m3))
-    return OILBIRD_EINVAL;
-  if (path == OILBIRD_PATH_TENSOR && !p->tc) {
-    snprintf(g_cuda_err, sizeof g_cuda_err, "tensor-core scan unavailable on this device");
-    return OILBIRD_ECUDA;
-  }
 
   int32_t n_lists = 0;
   if (p->n_rows == 0) {
@@ -518,12 +613,7 @@ static int query_impl(oilbird_pool_t* p, const void* q, int32_t nq, const oilbir
     p->launches += 1;
   } else {
     cudaEvent_t e0 = nullptr, e1 = nullptr;
-    if (p->profile && p->ev_used + 2 <= 2 * kMaxProfile) {
-      while ((int)p->ev.size() < p->ev_used + 2) {
-        cudaEvent_t ne;
-        CU(cudaEventCreate(&ne));
-        p->ev.push_back(ne);
-      }
+    if (p->profile && p->ev_used + 2 <= (int)p->ev.size()) {
       e0 = p->ev[p->ev_used]; e1 = p->ev[p->ev_used + 1];
       CU(cudaEventRecord(e0, st));
     }
@@ -587,14 +677,16 @@ int oilbird_pool_query(oilbird_pool_t* p, const void* q, int32_t nq,
 static int step_impl(oilbird_pool_t* p, const void* states, const int32_t* tokens, int64_t n,
                      uint64_t tag, uint32_t flags, const void* q, int32_t nq,
                      const oilbird_query_params* pr, const oilbird_query_out* out, void* stream) {
-  if (!p || !q || !out_ok(out, true)) return OILBIRD_EINVAL;
   GatherParams gp;
-  int rc = check_params(p, nq, pr, &gp);          // nothing is appended if the query is invalid
-  if (rc) return rc;
+  int path = 0;
+  // nothing is appended if the query would be refused (arguments, parameters, or a scan this
+  // pool does not have)
+  if (!p) return OILBIRD_EINVAL;
   const int64_t rows_after = p->n_rows + n;
+  int rc = check_query(p, q, nq, pr, out, rows_after, &gp, &path);
+  if (rc) return rc;
   // (8-bit pools always use the CUDA-core scan; its passes beyond the first two queries
   // would find the rows in place, but keep to the single-request case there too)
-  const int path = resolve_path(p, pr, nq);
   const bool gemv = p->r.e4m3 ? (nq <= 2 && path == OILBIRD_PATH_GEMV) : path == OILBIRD_PATH_GEMV;
   // the warp-level tensor scan appends the step's rows itself in its 8-query form (eight rows
   // per CTA on 16-bit keys, one on 8-bit keys)
@@ -642,6 +734,7 @@ int oilbird_pool_gather(oilbird_pool_t* p, const int32_t* idx, const float* scor
                         const oilbird_query_params* pr, const oilbird_query_out* out,
                         void* stream) {
   if (!p || !idx || !score || !out_ok(out, false)) return OILBIRD_EINVAL;
+  if (!aligned(idx, 4) || !aligned(score, 4)) return misaligned("idx / score");
   GatherParams gp;
   int rc = check_params(p, nq, pr, &gp);
   if (rc) return rc;
@@ -684,8 +777,11 @@ static int ensure_pinned(oilbird_pool* p) {
   const size_t o_bytes =
       (size_t)p->r.max_nq * ((size_t)p->r.max_k * (8 + 4 + 4 * OILBIRD_MAX_CONT_LEN) + 4);
   unsigned char* h = nullptr;
-  cudaError_t e = cudaHostAlloc((void**)&h, align_up(a_bytes) + b_bytes + o_bytes,
-                                cudaHostAllocMapped);
+  // page-locking memory is a device-wide operation of the driver: let the device go idle
+  // first rather than have it happen under kernels that are chained and waiting
+  cudaError_t e = cudaDeviceSynchronize();
+  if (e != cudaSuccess) return cuda_fail(e, "cudaDeviceSynchronize");
+  e = cudaHostAlloc((void**)&h, align_up(a_bytes) + b_bytes + o_bytes, cudaHostAllocMapped);
   if (e != cudaSuccess) return cuda_fail(e, "cudaHostAlloc");
   void* dptr = nullptr;
   e = cudaHostGetDevicePointer(&dptr, h, 0);
@@ -832,6 +928,46 @@ int oilbird_pool_status(oilbird_pool_t* p, oilbird_pool_stats* stats, void* stre
   return ds.stalled ? OILBIRD_ESTALL : OILBIRD_OK;
 }
 
+int oilbird_pool_set_wait_limit(oilbird_pool_t* p, uint64_t limit_ns, void* stream) {
+  if (!p) return OILBIRD_EINVAL;
+  CU(cudaSetDevice(p->device));
+  const unsigned long long v = limit_ns;
+  // (pageable source: the call returns once the value has been staged)
+  CU(cudaMemcpyAsync(&p->stats->wait_limit_ns, &v, sizeof v, cudaMemcpyHostToDevice,
+                     (cudaStream_t)stream));
+  return OILBIRD_OK;
+}
+
+int oilbird_pool_stall_selftest(oilbird_pool_t* p, void* stream) {
+  if (!p) return OILBIRD_EINVAL;
+  CU(cudaSetDevice(p->device));
+  cudaError_t e = launch_stall_selftest(p->fuse_ready, p->stats, (cudaStream_t)stream);
+  if (e != cudaSuccess) return cuda_fail(e, "self-test kernel launch");
+  p->launches += 1;
+  return OILBIRD_OK;
+}
+
+int oilbird_pool_check_guards(oilbird_pool_t* p, void* stream) {
+  if (!p) return OILBIRD_EINVAL;
+  if (!p->r.guards) return OILBIRD_EINVAL;
+  CU(cudaSetDevice(p->device));
+  CU(cudaStreamSynchronize((cudaStream_t)stream));
+  std::vector<unsigned char> buf;
+  for (int g = 0; g < p->lay.n_guards; ++g) {
+    const size_t n = p->lay.g_hi[g] - p->lay.g_lo[g];
+    buf.resize(n);
+    CU(cudaMemcpy(buf.data(), p->base + p->lay.g_lo[g], n, cudaMemcpyDeviceToHost));
+    for (size_t i = 0; i < n; ++i) {
+      if (buf[i] != kGuardByte) {
+        snprintf(g_cuda_err, sizeof g_cuda_err, "guard zone behind '%s' overwritten at byte %zu",
+                 p->lay.g_name[g], i);
+        return OILBIRD_EGUARD;
+      }
+    }
+  }
+  return OILBIRD_OK;
+}
+
 int oilbird_pool_read_rows(oilbird_pool_t* p, int64_t row0, int64_t n, void* keys,
                            int32_t* tokens, int32_t* trace_ids) {
   if (!p || row0 < 0 || n < 0 || row0 + n > p->n_rows) return OILBIRD_EINVAL;
@@ -876,6 +1012,15 @@ int32_t oilbird_pool_read_traces(const oilbird_pool_t* p, int64_t* start, int64_
 
 int oilbird_pool_profile(oilbird_pool_t* p, int32_t enable) {
   if (!p) return OILBIRD_EINVAL;
+  if (enable) {
+    // all events now, none on the query path
+    CU(cudaSetDevice(p->device));
+    while ((int)p->ev.size() < 2 * kMaxProfile) {
+      cudaEvent_t ne;
+      CU(cudaEventCreate(&ne));
+      p->ev.push_back(ne);
+    }
+  }
   p->profile = enable != 0;
   return OILBIRD_OK;
 }

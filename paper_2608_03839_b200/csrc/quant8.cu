@@ -34,8 +34,7 @@ append_e4m3_kernel(const uint16_t* __restrict__ states, const int32_t* __restric
                    uint64_t* __restrict__ trace_tag, uint64_t tag,
                    int64_t* __restrict__ trace_gbase, int64_t gbase, int set_tag,
                    DeviceStats* stats) {
-  pdl_launch_dependents();
-  pdl_wait();   // earlier queries may still be reading the trace table and token stream
+  pdl_enter();   // earlier queries may still be reading the trace table and token stream
   if (blockIdx.x == 0 && threadIdx.x == 0) {
     trace_end[trace] = (int32_t)(row0 + n);
     if (set_tag) { trace_tag[trace] = tag; trace_gbase[trace] = gbase; }
@@ -85,8 +84,7 @@ scan_gemv_e4m3_kernel(const uint8_t* __restrict__ codes, const float* __restrict
                       int32_t* __restrict__ q_valid, DeviceStats* stats, FusedAppend fa) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   constexpr int KK = 32 * E;
-  pdl_launch_dependents();
-  pdl_wait();
+  pdl_enter();
   const int d = pv.d, n8 = d >> 3, n16 = d >> 4;
   uint4* qs = reinterpret_cast<uint4*>(smem_raw);                        // [QT][n8] bf16
   u64* scratch = reinterpret_cast<u64*>(smem_raw + (size_t)QT * d * 2);   // [warps][KK]
@@ -251,9 +249,6 @@ static cudaError_t launch_q8(const uint8_t* codes, const float* scales, const Po
                              int32_t* q_valid, DeviceStats* stats, int grid, const FusedAppend& fa,
                              cudaStream_t st) {
   const size_t smem = (size_t)QT * pv.d * 2 + (size_t)kQ8Warps * 32 * E * sizeof(u64);
-  cudaError_t e = cudaFuncSetAttribute(scan_gemv_e4m3_kernel<QT, E>,
-                                       cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-  if (e != cudaSuccess) return e;
   return launch_pdl(scan_gemv_e4m3_kernel<QT, E>, dim3(grid), dim3(kQ8Threads), smem, st, codes,
                     scales, pv, q_raw, nq, k, ex, partial, q_valid, stats, fa);
 }
@@ -290,12 +285,12 @@ cudaError_t launch_scan_gemv_e4m3(const uint8_t* codes, const float* scales, con
 cudaError_t preload_quant8_kernels() {
   cudaError_t e;
   if ((e = preload_kernel(append_e4m3_kernel)) != cudaSuccess) return e;
-  if ((e = preload_kernel(scan_gemv_e4m3_kernel<1, 1>)) != cudaSuccess) return e;
-  if ((e = preload_kernel(scan_gemv_e4m3_kernel<1, 2>)) != cudaSuccess) return e;
-  if ((e = preload_kernel(scan_gemv_e4m3_kernel<1, 4>)) != cudaSuccess) return e;
-  if ((e = preload_kernel(scan_gemv_e4m3_kernel<2, 1>)) != cudaSuccess) return e;
-  if ((e = preload_kernel(scan_gemv_e4m3_kernel<2, 2>)) != cudaSuccess) return e;
-  return preload_kernel(scan_gemv_e4m3_kernel<2, 4>);
+  if ((e = preload_kernel(scan_gemv_e4m3_kernel<1, 1>, true)) != cudaSuccess) return e;
+  if ((e = preload_kernel(scan_gemv_e4m3_kernel<1, 2>, true)) != cudaSuccess) return e;
+  if ((e = preload_kernel(scan_gemv_e4m3_kernel<1, 4>, true)) != cudaSuccess) return e;
+  if ((e = preload_kernel(scan_gemv_e4m3_kernel<2, 1>, true)) != cudaSuccess) return e;
+  if ((e = preload_kernel(scan_gemv_e4m3_kernel<2, 2>, true)) != cudaSuccess) return e;
+  return preload_kernel(scan_gemv_e4m3_kernel<2, 4>, true);
 }
 
 }  // namespace oilbird

@@ -101,15 +101,25 @@ int oilbird_query_static(const oilbird_static_pool* sp, const void* q_bf16, int3
              sp->d, (long long)sp->n_rows);
     return OILBIRD_EINVAL;
   }
-  if (pr->cont_len < 1 || pr->cont_len > OILBIRD_MAX_CONT_LEN || pr->offset < 0 ||
-      pr->n_tiers < 0 || pr->n_tiers > OILBIRD_MAX_TIERS || pr->theta != pr->theta ||
-      (pr->depth_mode != OILBIRD_DEPTH_FIXED && pr->depth_mode != OILBIRD_DEPTH_TIERED)) {
+  GatherParams gp;
+  if (check_query_params(nq, kStaticMaxNq, OILBIRD_MAX_K, pr, &gp) != OILBIRD_OK) {
     snprintf(g_static_err, sizeof g_static_err, "query parameter out of range");
     return OILBIRD_EINVAL;
   }
   if (pr->exclude_tag || pr->path == OILBIRD_PATH_TENSOR || pr->path == OILBIRD_PATH_MMA) {
     snprintf(g_static_err, sizeof g_static_err,
              "the static variant has no exclusion tags and only the CUDA-core scan");
+    return OILBIRD_EINVAL;
+  }
+  // the kernels read keys and queries with 16-byte loads and the integer arrays word by word
+  const uintptr_t a16 = (uintptr_t)q_bf16 | (sp->n_rows > 0 ? (uintptr_t)sp->keys : 0);
+  const uintptr_t a4 = (uintptr_t)out->idx | (uintptr_t)out->score | (uintptr_t)out->fired |
+                       (uintptr_t)out->cont_len | (uintptr_t)out->cont_tok |
+                       (sp->n_rows > 0 ? (uintptr_t)sp->tokens | (uintptr_t)sp->trace_id |
+                                             (uintptr_t)sp->trace_end : 0);
+  if ((a16 & 15) || (a4 & 3)) {
+    snprintf(g_static_err, sizeof g_static_err,
+             "misaligned pointer (keys and q: 16 bytes; integer and score arrays: 4 bytes)");
     return OILBIRD_EINVAL;
   }
   cudaError_t e = cudaSetDevice(sp->device);
@@ -125,13 +135,6 @@ int oilbird_query_static(const oilbird_static_pool* sp, const void* q_bf16, int3
   DeviceStats* stats = (DeviceStats*)(base + kStaticListBytes + kStaticFlagBytes);
   cudaStream_t st = (cudaStream_t)cuda_stream;
 
-  GatherParams gp;
-  gp.k = pr->k; gp.offset = pr->offset; gp.depth_mode = pr->depth_mode;
-  gp.cont_len = pr->cont_len; gp.n_tiers = pr->n_tiers; gp.theta = pr->theta;
-  for (int t = 0; t < OILBIRD_MAX_TIERS; ++t) {
-    gp.tier_thr[t] = t < pr->n_tiers ? pr->tier_thr[t] : INFINITY;
-    gp.tier_depth[t] = t < pr->n_tiers ? pr->tier_depth[t] : 0;
-  }
   PoolView pv;
   pv.keys = (const uint16_t*)sp->keys; pv.tok = sp->tokens; pv.trace_id = sp->trace_id;
   pv.trace_end = sp->trace_end; pv.trace_tag = nullptr; pv.d = sp->d;

@@ -31,8 +31,7 @@ ring_append_kernel(const uint16_t* __restrict__ states, const int32_t* __restric
                    const int32_t* __restrict__ rollouts, int64_t n, int d, int R, int64_t start,
                    int64_t cap, uint16_t* __restrict__ keys, int32_t* __restrict__ anchor,
                    int32_t* __restrict__ rollout) {
-  pdl_launch_dependents();
-  pdl_wait();   // an earlier lookup may still be reading the slots this append overwrites
+  pdl_enter();   // an earlier lookup may still be reading the slots this append overwrites
   for (int64_t r = blockIdx.x; r < n; r += gridDim.x) {
     const int64_t slot = (start + r) % cap;
     normalize_row(states + r * d, keys + slot * d, d);
@@ -53,8 +52,7 @@ ring_scan_kernel(const uint16_t* __restrict__ keys, const int32_t* __restrict__ 
   u64* scratch = reinterpret_cast<u64*>(smem_raw + (size_t)d * 2);          // [warps][32]
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int q = blockIdx.y;
-  pdl_launch_dependents();
-  pdl_wait();
+  pdl_enter();
   const int code = normalize_row<false>(q_raw + (size_t)q * d, reinterpret_cast<uint16_t*>(qs), d);
   if (blockIdx.x == 0 && threadIdx.x == 0) {
     q_valid[q] = code == kRowNonFinite ? 0 : 1;
@@ -111,8 +109,7 @@ ring_merge_kernel(const u64* __restrict__ partial, int n_lists, int nq, int m, i
   __shared__ u64 scratch[kMergeWarps * kRingList];
   __shared__ u64 s_best[kRingList];
   const int q = blockIdx.x;
-  pdl_launch_dependents();
-  pdl_wait();
+  pdl_enter();
   const int lists = q_valid[q] != 0 ? n_lists : 0;
   // no head filter here: the lookup moves under 1 MB and is bound by launch latency; with
   // the filter's two extra barriers an append + lookup step was measured 4.5 us slower
@@ -146,7 +143,7 @@ ring_merge_kernel(const u64* __restrict__ partial, int n_lists, int nq, int m, i
 cudaError_t preload_ring_kernels() {
   cudaError_t e;
   if ((e = preload_kernel(ring_append_kernel)) != cudaSuccess) return e;
-  if ((e = preload_kernel(ring_scan_kernel)) != cudaSuccess) return e;
+  if ((e = preload_kernel(ring_scan_kernel, true)) != cudaSuccess) return e;
   return preload_kernel(ring_merge_kernel);
 }
 
@@ -273,8 +270,6 @@ int oilbird_ring_query(oilbird_ring_t* r, const void* q, const int32_t* q_anchor
   int64_t want = (n_slots + 255) / 256;
   int slices = (int)(want < 1 ? 1 : (want > r->max_lists ? r->max_lists : want));
   const size_t smem = (size_t)r->d * 2 + (size_t)kRingWarps * kRingList * sizeof(u64);
-  RCU(cudaFuncSetAttribute(ring_scan_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                           (int)smem));
   cudaError_t e = launch_pdl(ring_scan_kernel, dim3(slices, nq), dim3(kRingThreads), smem, st,
                              (const uint16_t*)r->keys, (const int32_t*)r->anchor, n_slots, r->d,
                              (const uint16_t*)q, q_anchor, nq, m, floor_s, r->partial, r->q_valid,

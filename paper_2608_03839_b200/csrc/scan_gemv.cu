@@ -67,8 +67,7 @@ scan_gemv_kernel(PoolView pv, const uint16_t* __restrict__ q_raw, int nq, int k,
                  int32_t* __restrict__ q_valid, DeviceStats* stats, FusedAppend fa) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   constexpr int KK = 32 * E;
-  pdl_launch_dependents();
-  pdl_wait();   // the rows appended just before this query, and the query states themselves
+  pdl_enter();   // the rows appended just before this query, and the query states themselves
   const int d = pv.d, n_chunks = d >> 3;
   uint4* qs = reinterpret_cast<uint4*>(smem_raw);                       // [QT][n_chunks]
   u64* scratch = reinterpret_cast<u64*>(smem_raw + (size_t)QT * d * 2);  // [warps][KK]
@@ -207,9 +206,6 @@ static cudaError_t launch_one(const PoolView& pv, const uint16_t* q_raw, int nq,
                               DeviceStats* stats, int grid, const FusedAppend& fa,
                               cudaStream_t st) {
   size_t smem = (size_t)QT * pv.d * 2 + (size_t)kScanWarps * 32 * E * sizeof(u64);
-  cudaError_t e = cudaFuncSetAttribute(scan_gemv_kernel<QT, E>,
-                                       cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-  if (e != cudaSuccess) return e;
   return launch_pdl(scan_gemv_kernel<QT, E>, dim3(grid), dim3(kScanThreads), smem, st, pv, q_raw,
                     nq, k, ex, partial, q_valid, stats, fa);
 }
@@ -245,12 +241,12 @@ cudaError_t launch_scan_gemv(const PoolView& pv, const uint16_t* q_raw, int32_t 
 
 cudaError_t preload_scan_gemv_kernels() {
   cudaError_t e;
-  if ((e = preload_kernel(scan_gemv_kernel<1, 1>)) != cudaSuccess) return e;
-  if ((e = preload_kernel(scan_gemv_kernel<1, 2>)) != cudaSuccess) return e;
-  if ((e = preload_kernel(scan_gemv_kernel<1, 4>)) != cudaSuccess) return e;
-  if ((e = preload_kernel(scan_gemv_kernel<2, 1>)) != cudaSuccess) return e;
-  if ((e = preload_kernel(scan_gemv_kernel<2, 2>)) != cudaSuccess) return e;
-  return preload_kernel(scan_gemv_kernel<2, 4>);
+  if ((e = preload_kernel(scan_gemv_kernel<1, 1>, true)) != cudaSuccess) return e;
+  if ((e = preload_kernel(scan_gemv_kernel<1, 2>, true)) != cudaSuccess) return e;
+  if ((e = preload_kernel(scan_gemv_kernel<1, 4>, true)) != cudaSuccess) return e;
+  if ((e = preload_kernel(scan_gemv_kernel<2, 1>, true)) != cudaSuccess) return e;
+  if ((e = preload_kernel(scan_gemv_kernel<2, 2>, true)) != cudaSuccess) return e;
+  return preload_kernel(scan_gemv_kernel<2, 4>, true);
 }
 
 }  // namespace oilbird

@@ -234,8 +234,7 @@ scan_mma_kernel(PoolView pv, const uint8_t* __restrict__ codes, const float* __r
   constexpr int QP = kMmaQ * NT;             // queries per pass
   constexpr int kQuads = kMmaThreads / 128;  // quads of four warps per CTA
   constexpr int kMmaDepth = NT == 1 ? kMmaDepth1 : kMmaDepth2;
-  pdl_launch_dependents();
-  pdl_wait();   // the rows appended before this query, and the query states themselves
+  pdl_enter();   // the rows appended before this query, and the query states themselves
   const int d = pv.d, n_chunks = d >> 3;
   const int k_units = kFp8 ? d >> 4 : d >> 3;                            // 16-byte units of a key row
   const int q_stride = n_chunks + kMmaPadBytes / 16;                     // in 16-byte units
@@ -622,9 +621,6 @@ static cudaError_t launch_mma_one(const PoolView& pv, const uint8_t* codes, cons
                                   u64* partial, int32_t* q_valid, DeviceStats* stats, int grid,
                                   const FusedAppend& fa, cudaStream_t st) {
   const size_t smem = scan_mma_smem(pv.d, 32 * E, NT);
-  cudaError_t e = cudaFuncSetAttribute(scan_mma_kernel<E, NT, kFp8>,
-                                       cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-  if (e != cudaSuccess) return e;
   return launch_pdl(scan_mma_kernel<E, NT, kFp8>, dim3(grid), dim3(kMmaThreads), smem, st, pv, codes,
                     scales, q_raw, nq, k, ex, partial, q_valid, stats, fa);
 }
@@ -666,14 +662,14 @@ cudaError_t launch_scan_mma(const PoolView& pv, const uint8_t* codes, const floa
 
 cudaError_t preload_scan_mma_kernels() {
   cudaError_t e;
-  if ((e = preload_kernel(scan_mma_kernel<1, 1, false>)) != cudaSuccess) return e;
-  if ((e = preload_kernel(scan_mma_kernel<2, 1, false>)) != cudaSuccess) return e;
-  if ((e = preload_kernel(scan_mma_kernel<1, 2, false>)) != cudaSuccess) return e;
-  if ((e = preload_kernel(scan_mma_kernel<2, 2, false>)) != cudaSuccess) return e;
-  if ((e = preload_kernel(scan_mma_kernel<1, 1, true>)) != cudaSuccess) return e;
-  if ((e = preload_kernel(scan_mma_kernel<2, 1, true>)) != cudaSuccess) return e;
-  if ((e = preload_kernel(scan_mma_kernel<1, 2, true>)) != cudaSuccess) return e;
-  return preload_kernel(scan_mma_kernel<2, 2, true>);
+  if ((e = preload_kernel(scan_mma_kernel<1, 1, false>, true)) != cudaSuccess) return e;
+  if ((e = preload_kernel(scan_mma_kernel<2, 1, false>, true)) != cudaSuccess) return e;
+  if ((e = preload_kernel(scan_mma_kernel<1, 2, false>, true)) != cudaSuccess) return e;
+  if ((e = preload_kernel(scan_mma_kernel<2, 2, false>, true)) != cudaSuccess) return e;
+  if ((e = preload_kernel(scan_mma_kernel<1, 1, true>, true)) != cudaSuccess) return e;
+  if ((e = preload_kernel(scan_mma_kernel<2, 1, true>, true)) != cudaSuccess) return e;
+  if ((e = preload_kernel(scan_mma_kernel<1, 2, true>, true)) != cudaSuccess) return e;
+  return preload_kernel(scan_mma_kernel<2, 2, true>, true);
 }
 
 }  // namespace oilbird

@@ -49,7 +49,6 @@
 // Every mbarrier wait is bounded: after about two seconds it raises the pool's `stalled`
 // flag, the CTA drains what it has in flight, frees its TMEM and returns.
 #include <cuda.h>
-#include <stdlib.h>
 
 #include <new>
 
@@ -68,7 +67,6 @@ constexpr int kATileBytes = kTileM * kBlockK * 2;   // 16 KB
 constexpr int kColsPerRound = 16;      // score columns filtered between two drains
 constexpr int kQueueCap = kTileM * kColsPerRound;
 constexpr int kMaxStages = 8;
-constexpr unsigned long long kWaitLimitNs = 2000000000ull;
 
 // ------------------------------------------------------------------ PTX wrappers ---
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
@@ -105,12 +103,12 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
                                           DeviceStats* stats) {
   if (mbar_try_wait(bar, parity)) return true;
-  const unsigned long long t0 = global_ns();
+  const unsigned long long t0 = global_ns(), limit = wait_limit_ns(stats);
   for (uint32_t spin = 0;; ++spin) {
     if (mbar_try_wait(bar, parity)) return true;
     if ((spin & 63u) == 63u) {
       if (*abort_flag) return false;
-      if (global_ns() - t0 > kWaitLimitNs) {
+      if (global_ns() - t0 > limit) {
         *abort_flag = 1;
         atomicExch(&stats->stalled, 1);
         return false;
@@ -313,7 +311,6 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap key_map,
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int a_bytes = mt * kATileBytes;
   const int stage_bytes = a_bytes + n_pad * kBlockK * 2;
-  pdl_launch_dependents();
   // dynamic shared memory: [stages][mt key tiles | query tile] | lists | queue | state
   unsigned char* base = (unsigned char*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
   unsigned char* ring = base;
@@ -363,7 +360,7 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap key_map,
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = sh.tmem_base;
-  pdl_wait();   // appended rows, normalised queries, exclusion tags; set-up above overlapped
+  pdl_enter();   // appended rows, normalised queries, exclusion tags; set-up above overlapped
   for (int i = threadIdx.x; i < n_pad; i += kTcThreads) {
     thr_s[i] = i < nq_c ? -INFINITY : INFINITY;        // padded columns never pass the filter
     s_ex[i] = (exclude_tag && i < nq_c) ? exclude_tag[q0 + i] : 0;
@@ -437,7 +434,8 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap key_map,
       // nothing may still be writing TMEM when it is freed
       tc_commit(&sh.drain);
       const unsigned long long t0 = global_ns();
-      while (!mbar_try_wait(&sh.drain, 0) && global_ns() - t0 < kWaitLimitNs) {}
+      const unsigned long long limit = wait_limit_ns(stats);
+      while (!mbar_try_wait(&sh.drain, 0) && global_ns() - t0 < limit) {}
     }
   } else {
     // ===================================================== epilogue ==============
@@ -635,6 +633,10 @@ TcCache* tc_cache_create(const void* keys, int64_t capacity, int32_t d, const vo
     delete c;
     return nullptr;
   }
+  // every box height a query of this pool can ask for, encoded now: nothing is left to do
+  // on the first call that uses one
+  for (int n_pad = 16; n_pad <= OILBIRD_MAX_NQ && n_pad <= qn_rows; n_pad += 16)
+    c->q_ok[n_pad / 16 - 1] = make_bf16_map(&c->q_map[n_pad / 16 - 1], qn, qn_rows, d, n_pad);
   return c;
 }
 
@@ -642,11 +644,7 @@ void tc_cache_destroy(TcCache* c) { delete c; }
 
 static const CUtensorMap* tc_q_map(TcCache* c, int n_pad) {
   const int slot = n_pad / 16 - 1;
-  if (!c->q_ok[slot]) {
-    if (!make_bf16_map(&c->q_map[slot], c->qn, c->qn_rows, c->d, n_pad)) return nullptr;
-    c->q_ok[slot] = true;
-  }
-  return &c->q_map[slot];
+  return (slot >= 0 && slot < OILBIRD_MAX_NQ / 16 && c->q_ok[slot]) ? &c->q_map[slot] : nullptr;
 }
 
 static size_t tc_fixed_smem(int nq_c, int n_pad, int kk, bool compact) {
@@ -713,10 +711,7 @@ cudaError_t launch_scan_tc(TcCache* cache, const PoolView& pv, int32_t q0, int32
                            int32_t num_sms, size_t smem_limit, int32_t* n_lists, cudaStream_t st) {
   const int n_pad = (nq_c + 15) / 16 * 16;
   const int n_tiles128 = (pv.n_rows + kTileM - 1) / kTileM;
-  static const int force_mt = getenv("OILBIRD_TC_MT") ? atoi(getenv("OILBIRD_TC_MT")) : 0;
-  TcPlan plan = tc_plan(nq_c, k, n_tiles128, num_sms, smem_limit, force_mt);
-  static const int cap_stages = getenv("OILBIRD_TC_STAGES") ? atoi(getenv("OILBIRD_TC_STAGES")) : 0;
-  if (cap_stages >= 2 && plan.stages > cap_stages) plan.stages = cap_stages;
+  TcPlan plan = tc_plan(nq_c, k, n_tiles128, num_sms, smem_limit, 0);
   const size_t stage = (size_t)plan.mt * kATileBytes + (size_t)n_pad * kBlockK * 2;
   const size_t fixed = tc_fixed_smem(nq_c, n_pad, kk, plan.compact != 0);
   if (plan.stages < 2) return cudaErrorInvalidConfiguration;
@@ -730,15 +725,42 @@ cudaError_t launch_scan_tc(TcCache* cache, const PoolView& pv, int32_t q0, int32
   int grid = n_tiles < num_sms ? n_tiles : num_sms;
   if (grid < 1) grid = 1;
   *n_lists = grid;
-  cudaError_t e = cudaFuncSetAttribute(scan_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                       (int)smem);
-  if (e != cudaSuccess) return e;
   return launch_pdl(scan_tc_kernel, dim3(grid), dim3(kTcThreads), smem, st,
                     cache->key_map, *q_map, pv, q0, nq_c, nq_total, n_pad, k, kk, plan.stages,
                     tmem_cols, plan.mt, plan.n_bufs, plan.compact, exclude_tag, partial, stats,
                     xchg);
 }
 
-cudaError_t preload_scan_tc_kernels() { return preload_kernel(scan_tc_kernel); }
+// Both kinds of bounded wait on things that never happen (see launch_stall_selftest).
+__global__ void __launch_bounds__(64)
+stall_selftest_kernel(const unsigned long long* ready, DeviceStats* stats, int* gave_up) {
+  __shared__ uint64_t bar;
+  __shared__ int abort_flag;
+  pdl_enter();
+  if (threadIdx.x == 0) {
+    mbar_init(&bar, 1);
+    abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+  if (threadIdx.x < 32) {
+    // a row counter that nobody advances: the target is one past whatever it holds
+    wait_fused_rows(ready, ld_acquire_u64(ready) + 1ull, stats);
+  } else if (threadIdx.x == 32) {
+    // phase 0 of a barrier nobody arrives at never completes
+    const bool ok = mbar_wait(&bar, 0, &abort_flag, stats);
+    if (gave_up) *gave_up = ok ? 0 : 1;
+  }
+}
+
+cudaError_t launch_stall_selftest(const unsigned long long* ready, DeviceStats* stats,
+                                  cudaStream_t st) {
+  return launch_pdl(stall_selftest_kernel, dim3(1), dim3(64), 0, st, ready, stats, (int*)nullptr);
+}
+
+cudaError_t preload_scan_tc_kernels() {
+  cudaError_t e = preload_kernel(scan_tc_kernel, true);
+  return e != cudaSuccess ? e : preload_kernel(stall_selftest_kernel);
+}
 
 }  // namespace oilbird

@@ -24,8 +24,7 @@ __global__ void __launch_bounds__(256)
 to_global_kernel(const int32_t* __restrict__ idx, int64_t* __restrict__ out, int64_t n,
                  const int32_t* __restrict__ trace_id, const int32_t* __restrict__ trace_end,
                  const int64_t* __restrict__ trace_gbase, int32_t n_rows) {
-  pdl_launch_dependents();
-  pdl_wait();
+  pdl_enter();
   const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= n) return;
   const int32_t r = idx[i];
@@ -55,8 +54,7 @@ merge_shards_kernel(int n_shards, int nq, int k, int L, float theta,
   __shared__ int s_src[OILBIRD_MAX_K];     // winning candidate of each output rank
   __shared__ int s_fired;
   const int q = blockIdx.x;
-  pdl_launch_dependents();
-  pdl_wait();
+  pdl_enter();
   const int n_cand = n_shards * k;         // <= kShardThreads (checked by the host)
   const int c = threadIdx.x;
   float my_s = -INFINITY;

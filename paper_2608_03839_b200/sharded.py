@@ -104,11 +104,11 @@ def merge_gathered(gathered: torch.Tensor, lay: RecordLayout, theta: float, stre
     n_shards = gathered.shape[0]
     dev = gathered.device
     nq, k, L = lay.nq, lay.k, lay.L
-    out = ShardedOut(torch.empty((nq, k), dtype=torch.int64, device=dev),
-                     torch.empty((nq, k), dtype=torch.float32, device=dev),
-                     torch.empty((nq,), dtype=torch.int32, device=dev),
-                     torch.empty((nq, k), dtype=torch.int32, device=dev),
-                     torch.empty((nq, k, L), dtype=torch.int32, device=dev))
+    out = ShardedOut(B.ALLOC((nq, k), torch.int64, dev),
+                     B.ALLOC((nq, k), torch.float32, dev),
+                     B.ALLOC((nq,), torch.int32, dev),
+                     B.ALLOC((nq, k), torch.int32, dev),
+                     B.ALLOC((nq, k, L), torch.int32, dev))
     B._check(B.lib().oilbird_merge_shards(
         n_shards, nq, k, L, float(theta), gathered.data_ptr(), gathered.stride(0), lay.off_gidx,
         lay.off_score, lay.off_len, lay.off_tok, out.gidx.data_ptr(), out.score.data_ptr(),

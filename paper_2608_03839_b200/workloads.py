@@ -133,6 +133,14 @@ class Workload:
             raise ValueError(self.kind)
         return states.to(torch.bfloat16), toks, self.trace_tag(t)
 
+    def trace_assign(self, t: int, device="cpu") -> torch.Tensor:
+        """Clustered pools: the centroid each row of trace t was drawn around (the labels
+        only, without materialising the states: the trace generator's first draw)."""
+        if self.kind != "clustered":
+            raise ValueError("only clustered pools have centroid labels")
+        g = _gen(device, self.seed, 3, t)
+        return torch.randint(0, self.n_centroids, (self.trace_rows(t),), generator=g, device=device)
+
     def traces(self, device="cpu"):
         C = self._centroids(device) if self.kind == "clustered" else None
         for t in range(self.num_traces):
@@ -162,6 +170,9 @@ class Workload:
             st, _, _ = self.trace(t, device, C)
             q[0] = st[r].float() + self.query_noise * noise[0]
             meta["planted_row"] = row
+            cl = c.tolist()
+            cl[0] = int(self.trace_assign(t, device)[r])
+            meta["centroid"] = cl              # the centroid each query was drawn around
         elif self.kind == "template":
             gi = _gen("cpu", self.seed, 7, step)
             P = self.rows_per_trace

@@ -51,7 +51,7 @@ def test_struct_layout_constants_match_header():
         m = re.search(rf"#define\s+{name}\s+(\d+)", text)
         assert m and int(m.group(1)) == val
     for name, val in [("EINVAL", B.EINVAL), ("ECAPACITY", B.ECAPACITY), ("ENOMEM", B.ENOMEM),
-                      ("ECUDA", B.ECUDA), ("ESTALL", B.ESTALL)]:
+                      ("ECUDA", B.ECUDA), ("ESTALL", B.ESTALL), ("EGUARD", B.EGUARD)]:
         m = re.search(rf"#define\s+OILBIRD_{name}\s+\((-\d+)\)", text)
         assert m and int(m.group(1)) == val
 

@@ -67,7 +67,7 @@ def test_evict_matches_oracle(fmt, drop):
 
 
 def test_many_waves_a_short_trace_in_front_of_a_long_pool():
-    # dropping 3 rows from in front of ~5000 moves the pool in ~1700 waves of 3 rows
+    # 3 rows dropped in front of ~5000 (a prefix far smaller than what remains)
     d = 64
     g = torch.Generator(device="cuda").manual_seed(1)
     pool, ora = B.Pool(d, 6000), OraclePool(d)
@@ -87,6 +87,42 @@ def test_many_waves_a_short_trace_in_front_of_a_long_pool():
     pool.append(st, torch.arange(5, dtype=torch.int32, device="cuda"), tag=9)
     out = pool.query(st[2:3].contiguous(), fixed(1, 2, theta=-2.0))
     assert int(out.idx[0, 0]) == 2 and out.cont_tok[0, 0].tolist() == [4, -1]
+
+
+@pytest.mark.parametrize("fmt", ["bf16", "e4m3"])
+def test_one_row_dropped_in_front_of_a_pool_of_several_waves(fmt):
+    # a one-row trace in front of 20,000 rows: the fixed-size register-staged waves (about
+    # 600,000 16-byte chunks each on a B200) pass several times, with a ragged last wave; the
+    # barrier count must not depend on the size of the dropped prefix
+    d = 1024
+    g = torch.Generator(device="cuda").manual_seed(11)
+    pool, ora = B.Pool(d, 21000, key_format=fmt), OraclePool(d, fmt)
+    for n, tag in ((1, 1), (9000, 2), (2, 3), (10997, 4)):
+        st = torch.randn(n, d, generator=g, device="cuda").to(torch.bfloat16)
+        tk = torch.randint(0, 1000, (n,), generator=g, device="cuda", dtype=torch.int32)
+        pool.append(st, tk, tag=tag)
+        ora.append(W.to_bits(st), tk.cpu().numpy(), tag=tag)
+    assert pool.evict_oldest(1) == ora.evict_oldest(1) == 1
+    same_store(pool, ora)
+    q = torch.randn(1, d, generator=g, device="cuda").to(torch.bfloat16)
+    pr = fixed(8, 4, theta=-2.0)
+    check_query(pool.query(q, pr), ora, W.to_bits(q), pr)
+    assert pool.evict_oldest(2) == ora.evict_oldest(2) == 9002
+    same_store(pool, ora)
+
+
+def test_large_prefix_takes_the_streaming_form():
+    # 1,700 rows of 8 KB in front (14 MB, more than one staged wave): waves of `head` rows
+    d = 4096
+    g = torch.Generator(device="cuda").manual_seed(12)
+    pool, ora = B.Pool(d, 6000), OraclePool(d)
+    for n, tag in ((1700, 1), (2100, 2), (1500, 3)):
+        st = torch.randn(n, d, generator=g, device="cuda").to(torch.bfloat16)
+        tk = torch.randint(0, 1000, (n,), generator=g, device="cuda", dtype=torch.int32)
+        pool.append(st, tk, tag=tag)
+        ora.append(W.to_bits(st), tk.cpu().numpy(), tag=tag)
+    assert pool.evict_oldest(1) == ora.evict_oldest(1) == 1700
+    same_store(pool, ora)
 
 
 def test_evicting_empty_traces_still_renumbers():

@@ -1,12 +1,15 @@
 """Full-size benchmark configurations on the GPU against the CPU oracle.
 
-C3 and C4 are checked with the whole pool in the oracle (C4 on a subset of its 64
-queries: the oracle needs about a second per query at a million rows).  C5 (17-34 GB of
-keys) is checked on sampled rows: the oracle is run, unchanged, on a small pool made of
-the rows the GPU returned, the planted rows and a random sample of the rest; every
-property that holds for the full pool restricted to those rows is asserted.
+Every configuration is checked with the WHOLE pool in the oracle: C3 all queries, C4 on 16
+of its 64 queries (the oracle needs about a second per query at a million rows), C5 (17 GB
+of keys growing to 34 GB) on one to four queries of every batch size of its sweep at the
+start of the stream and at its far end.  Where the host cannot hold a second copy of the C5
+pool, and as a cross-check where it can, the oracle is also run, unchanged, on a small pool
+made of the rows the GPU returned, ALL rows drawn around the query's centroid (the only rows
+that can reach the top-k, see siblings_check) and a random sample of the rest.
 """
 import numpy as np
+import psutil
 import pytest
 import torch
 
@@ -97,7 +100,7 @@ def test_c4_batched_shared_pool_full_size_sampled_queries():
     out = pool.query(q, pr)                     # all 64 queries on the tensor path
     o = out.cpu()
     assert o.idx[0, 0] == meta["planted_row"]
-    sel = [0, 1, 31, 63]                        # the oracle scores these four
+    sel = [0, 1, 2, 7, 8, 15, 16, 17, 31, 32, 33, 47, 48, 55, 62, 63]   # the oracle scores these
     sub = B.QueryOut(o.idx[sel], o.score[sel], o.fired[sel], o.cont_len[sel], o.cont_tok[sel])
     st = check_query(sub, ora, W.to_bits(q)[sel], pr)
     assert st["max_score_err"] < SCORE_BUG
@@ -115,96 +118,141 @@ def test_c4_batched_shared_pool_full_size_sampled_queries():
     assert pool.stats()["stalled"] == 0
 
 
-def sampled_check(pool, w, C, q, out, n_rows, extra_rows, rng, params):
-    """Oracle on {returned rows} U extra_rows U random sample; see module docstring."""
+def take(out: B.QueryOut, sel) -> B.QueryOut:
     o = out.cpu()
+    return B.QueryOut(o.idx[sel], o.score[sel], o.fired[sel], o.cont_len[sel], o.cont_tok[sel])
+
+
+def siblings_check(pool, w, C, q, out, sel, q_centroid, assign, n_rows, extra_rows, rng, params):
+    """The oracle on a sub-pool that holds every row that can matter.
+
+    A clustered pool's rows are centroid + 0.2 * noise: two rows of the same centroid have
+    cosine ~0.96, rows of different centroids ~N(0, 1/d) (sigma 0.011 at d = 8192).  The k
+    best of a query are therefore rows of its own centroid as long as that centroid has at
+    least k rows, and a row of another centroid would have to sit ~80 sigma out to reach
+    them.  The sub-pool is: ALL rows of the selected queries' centroids (from the
+    generator's labels, without materialising the pool), the rows the GPU returned, the rows
+    in extra_rows and 1,500 random rows.  On it the unchanged oracle must reproduce the GPU's
+    answer under the full acceptance rule (so a sibling the scan dropped fails the test),
+    and the random rows must stay far below the k-th score (which is what makes the
+    restriction to siblings exact rather than sampled).
+    """
+    o = take(out, sel)
     idx = o.idx.numpy()
-    nq, k = idx.shape
-    rows = set(idx[idx >= 0].tolist()) | set(extra_rows)
-    rows |= set(rng.integers(0, n_rows, size=1500).tolist())
+    k = idx.shape[1]
+    lab = torch.cat(assign)[:n_rows].cpu().numpy()
+    rows = set(idx[idx >= 0].tolist()) | set(int(r) for r in extra_rows)
+    sib = {}
+    for j, qi in enumerate(sel):
+        sib[j] = np.nonzero(lab == q_centroid[qi])[0]
+        assert len(sib[j]) >= k, "centroid with fewer than k rows: the argument above does not apply"
+        rows |= set(sib[j].tolist())
+    rnd = rng.integers(0, n_rows, size=1500)
+    rows |= set(rnd.tolist())
     rows = np.array(sorted(rows))
     ora = OraclePool(w.d)
     by_trace = {}
     for r in rows:
         by_trace.setdefault(int(r) // w.rows_per_trace, []).append(int(r))
-    hits_by_trace = {}
-    for qi in range(nq):
-        for j in range(k):
-            if idx[qi, j] >= 0 and o.fired[qi]:
-                hits_by_trace.setdefault(int(idx[qi, j]) // w.rows_per_trace, []).append((qi, j))
-    order = []
+    toks = {}
     for t, rr in sorted(by_trace.items()):
         st, tk, tag = w.trace(t, "cuda", C)
         loc = torch.tensor([r - t * w.rows_per_trace for r in rr], device="cuda")
+        # one trace per sampled trace: a continuation never crosses into the next one
         ora.append(W.to_bits(st[loc]), tk[loc].cpu().numpy(), tag=tag)
-        order += rr
-        # gather is checked against the regenerated token stream of the neighbour's trace
-        tk_host = tk.cpu().tolist()
-        for qi, j in hits_by_trace.get(t, ()):
-            s0 = int(idx[qi, j]) - t * w.rows_per_trace + params.offset
-            want = tk_host[s0: s0 + params.cont_len]          # clipped at the trace end
-            assert o.cont_len[qi, j] == len(want)
-            assert o.cont_tok[qi, j].tolist() == want + [-1] * (params.cont_len - len(want))
-    order = np.array(order)
-    # keys of the sampled rows are bit-identical to the oracle's
-    pos = {int(g): i for i, g in enumerate(order)}
-    for g in list(idx[0, :4]) + list(extra_rows)[:4]:
+        toks[t] = tk.cpu().tolist()
+    pos = {int(g): i for i, g in enumerate(rows)}
+    # stored keys of a few of those rows are bit-identical to the oracle's
+    for g in list(idx[0, :3]) + [int(r) for r in list(extra_rows)[:2]]:
         keys, _, _ = pool.read_rows(int(g), 1)
         assert np.array_equal(keys[0], ora.keys[pos[int(g)]])
-    ref = ora.query(W.to_bits(q), oracle_params(params), want_all_scores=True)
-    for qi in range(nq):
-        s_loc = ref.all_scores[qi]
-        got = idx[qi]
+    # the GPU's answer, renumbered into the sub-pool (the order of rows is kept, so ties
+    # break the same way), checked by the same rule as everywhere else but for the gather,
+    # which is compared with the regenerated token stream of the neighbour's own trace
+    ref = ora.query(W.to_bits(q)[sel], oracle_params(params), want_all_scores=True)
+    for j, qi in enumerate(sel):
+        s_loc = ref.all_scores[j]
+        got = idx[j]
         loc = np.array([pos[int(g)] for g in got])
-        err = np.abs(o.score[qi].numpy() - s_loc[loc])
-        assert err.max() < SCORE_BUG
-        # nothing in the sample beats the k-th returned score by more than the tie band
-        kth = float(o.score[qi, -1])
-        better = order[np.where(s_loc > kth + GAP)[0]]
-        assert set(better.tolist()) <= set(got.tolist())
-        assert np.all(np.diff(o.score[qi].numpy()) <= 0)
-        assert len(set(got.tolist())) == k
+        assert np.abs(o.score[j].numpy() - s_loc[loc]).max() < SCORE_BUG
+        assert len(set(got.tolist())) == k and np.all(np.diff(o.score[j].numpy()) <= 0)
+        s_k = float(ref.score[j, k - 1])
+        assert np.all(s_loc[loc] >= s_k - GAP), "a returned row is not among the k best"
+        must = rows[np.where(s_loc > s_k + GAP)[0]]
+        assert set(must.tolist()) <= set(got.tolist()), "a row that beats the k-th by more than the tie band is missing"
+        # every row of another centroid in the sample is far below the k-th score
+        other = np.array([pos[int(r)] for r in rnd if int(lab[int(r)]) != q_centroid[qi]])
+        assert s_k - float(s_loc[other].max()) > 0.5
+        for jj in range(k):
+            t, r0 = divmod(int(got[jj]), w.rows_per_trace)
+            want = (toks[t][r0 + params.offset: r0 + params.offset + params.cont_len]
+                    if o.fired[j] else [])                    # clipped at the trace end
+            assert o.cont_len[j, jj] == len(want)
+            assert o.cont_tok[j, jj].tolist() == want + [-1] * (params.cont_len - len(want))
 
 
-@pytest.mark.parametrize("nq", [1, 8, 64, 256])
-def test_c5_streaming_large_width(nq):
+def test_c5_streaming_large_width_whole_pool_in_the_oracle():
     w = W.C5
-    steps_a, steps_b = 6, 6
     n_start, n_end = W.C5_START_ROWS, w.n_rows
-    pool = B.Pool(w.d, n_end, max_nq=nq, max_k=w.k, max_traces=w.num_traces + 8)
-    C = w._centroids("cuda")
-    rng = np.random.default_rng(nq)
-    g = torch.Generator(device="cuda").manual_seed(1000 + nq)
     pr = fixed(w.k, w.cont_len)
+    # the oracle keeps its own copy of the keys (uint16): 17 GB at the start, 34 GB at the end
+    need = n_end * w.d * 2
+    full = psutil.virtual_memory().available > need + (12 << 30)
+    pool = B.Pool(w.d, n_end, max_nq=256, max_k=w.k, max_traces=w.num_traces + 8)
+    ora = OraclePool(w.d) if full else None
+    C = w._centroids("cuda")
+    rng = np.random.default_rng(5)
+    g = torch.Generator(device="cuda").manual_seed(1005)
+    assign = []
     t = 0
 
     def append_trace():
         nonlocal t
         st, tk, tag = w.trace(t, "cuda", C)
         pool.append(st, tk, tag=tag)
+        if ora is not None:
+            ora.append(W.to_bits(st), tk.cpu().numpy(), tag=tag)
+        assign.append(w.trace_assign(t, "cuda"))
         t += 1
         return st
 
-    def step(check):
+    def step(nq, n_oracle):
+        """One step of the stream (256 rows appended, nq queries, no synchronisation in
+        between); n_oracle of the queries are checked against the whole-pool oracle."""
         st = append_trace()
         n_rows = len(pool)
-        q, _ = w.queries("cuda", nq=nq, step=t)
+        q, meta = w.queries("cuda", nq=nq, step=t)
+        cent = list(meta["centroid"])
         r = int(rng.integers(0, st.shape[0]))
         q[nq - 1] = (st[r].float() + 0.05 * torch.randn(w.d, generator=g, device="cuda")).to(
             torch.bfloat16)
-        out = pool.query(q, pr)                               # no synchronisation in between
+        cent[nq - 1] = int(assign[-1][r])
+        out = pool.query(q, pr)
         assert out.cpu().idx[nq - 1, 0] == n_rows - st.shape[0] + r, "appended row not visible"
-        if check:
-            extra = [n_rows - st.shape[0] + r]
-            sampled_check(pool, w, C, q, out, n_rows, extra, rng, pr)
+        if n_oracle == 0:
+            return
+        sel = sorted({nq - 1, 0, nq // 3, (2 * nq) // 3})[-n_oracle:]
+        if ora is not None:
+            assert len(ora) == n_rows
+            stt = check_query(take(out, sel), ora, W.to_bits(q)[sel], pr)
+            assert stt["max_score_err"] < SCORE_BUG
+        extra = [n_rows - st.shape[0] + r]
+        if meta["planted_row"] < n_rows:              # (drawn over the final size of the pool)
+            extra.append(meta["planted_row"])
+        siblings_check(pool, w, C, q, out, sel, cent, assign, n_rows, extra, rng, pr)
 
     while len(pool) < n_start:
         append_trace()
-    for i in range(steps_a):
-        step(check=(i in (0, steps_a - 1)))
-    while len(pool) < n_end - steps_b * w.rows_per_trace:
+    # the start of the stream (N = 2^20 + a few steps): every batch size of the sweep
+    for nq, n_oracle in ((1, 1), (8, 4), (64, 4), (256, 4), (1, 0), (256, 0)):
+        step(nq, n_oracle)
+    while len(pool) < n_end - 4 * w.rows_per_trace:
         append_trace()
-    for i in range(steps_b):
-        step(check=(i == steps_b - 1))
+    # the far end (N -> 2^21): the compact-list path (nq = 256, k = 64) where it is used,
+    # and the single-request scan over 34 GB
+    for nq, n_oracle in ((64, 2), (8, 0), (256, 4), (1, 1)):
+        step(nq, n_oracle)
     assert len(pool) == n_end
     assert pool.stats() == dict(degenerate_rows=0, nonfinite_queries=0, stalled=0)
+    print(f"C5: whole-pool oracle {'used' if full else 'NOT used (host memory)'}; "
+          f"host memory available at start {psutil.virtual_memory().available / 2**30:.0f} GiB")

@@ -5,15 +5,18 @@ the whole GPU at start-up, say) and therefore cannot let this library allocate i
 scratch: the candidate lists live in a fixed array inside the library instead.  The test
 calls it through the C-ABI on pool arrays held in torch tensors and requires the very
 same results as oilbird_pool_query on the same pool, on two calls in a row (the second
-with other sizes, so that contents left by the first call would show).  The file is named
-so that pytest collects it last; it passes alone in a fresh process and after the others.
+with other sizes, so that contents left by the first call would show), and checks the same
+results against the CPU oracle directly.  The file is named so that pytest collects it
+last; it passes alone in a fresh process and after the others.
 """
 import numpy as np
 import pytest
 import torch
 
+from oracle import OraclePool
 from paper_2608_03839_b200 import binding as B
 from paper_2608_03839_b200 import workloads as W
+from parity import check_query
 
 pytestmark = pytest.mark.gpu
 
@@ -22,9 +25,10 @@ FIELDS = ("idx", "score", "fired", "cont_len", "cont_tok")
 
 def test_static_query_matches_pool_query_on_two_calls_in_a_row():
     w = W.C1.scaled(n_rows=3000, d=512, nq=2, seed=77)
-    pool = B.Pool(w.d, w.n_rows)
+    pool, ora = B.Pool(w.d, w.n_rows), OraclePool(w.d)
     for st, tk, tag in w.traces("cuda"):
         pool.append(st, tk, tag=tag)
+        ora.append(W.to_bits(st), tk.cpu().numpy(), tag=tag)
     # the caller's own copy of the pool arrays, in the layout append produces
     keys, tok, tid = pool.read_rows()
     _, ends, _ = pool.traces()
@@ -42,7 +46,9 @@ def test_static_query_matches_pool_query_on_two_calls_in_a_row():
         out = B.QueryOut.empty(qq.shape[0], pr.k, pr.cont_len, "cuda")
         for t in (out.idx, out.fired, out.cont_len, out.cont_tok):
             t.fill_(-7)                                  # every output word must be written
-        got = B.query_static(keys_t, tok_t, tid_t, end_t, qq, pr, out=out).cpu()
+        got = B.query_static(keys_t, tok_t, tid_t, end_t, qq, pr, out=out)
+        check_query(got, ora, W.to_bits(qq), pr)           # the oracle, not only the other entry point
+        got = got.cpu()
         for f in FIELDS:
             a, b = getattr(got, f), getattr(want, f)
             if f == "score":

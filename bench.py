@@ -35,7 +35,7 @@ from paper_2608_03839_b200 import workloads as W  # noqa: E402
 
 METRIC = "semantic_pool_queries_per_sec"
 UNIT = "queries/s"
-APPEND_ROWS = {"C1": 8, "C2": 8, "C3": 64, "C4": 512, "C5": 256}   # rows committed per step
+APPEND_ROWS = {"C1": 8, "C2": 8, "C3": 64, "C4": 128, "C5": 256}   # rows committed per step
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
 
@@ -178,45 +178,60 @@ def step_inputs(w: W.Workload, n_steps: int, rows: int, nq: int, device, seed: i
     return states, toks, queries
 
 
-def run_ours(args):
+MIN_REGION_S = 0.5        # every timed pass is repeated until it covers this much device time
+MAX_GROWTH = 0.06         # ... or until the appended rows have grown the pool by this fraction
+
+
+def fill_pool(pool, w, n_rows, dev, keep_raw=False):
+    """Append the configuration's seeded traces up to n_rows (not timed).  keep_raw: also
+    return the raw states and tokens, so that the pool can be rebuilt between repeats."""
+    raw = []
+    done = len(pool)
+    t0 = done // w.rows_per_trace
+    C = w._centroids(dev) if w.kind == "clustered" else None
+    for t in range(t0, w.num_traces):
+        if done >= n_rows:
+            break
+        st, tk, tag = w.trace(t, dev, C)
+        if done + st.shape[0] > n_rows:
+            st, tk = st[: n_rows - done].contiguous(), tk[: n_rows - done].contiguous()
+        pool.append(st, tk, tag=tag)
+        if keep_raw:
+            raw.append((st, tk, tag))
+        done += st.shape[0]
+    torch.cuda.synchronize()
+    return raw
+
+
+def measure(pool, w, nq, rows_step, K, Wm, dev, world, rank, local, args, n0, raw=None,
+            traffic_key=None):
+    """All passes of one workload on a filled pool.  Returns the fields of a bench line.
+
+    timed region   R repeats of EXACTLY K steps each, inputs resident in HBM, nothing but the
+                   steps between a repeat's two events; R is chosen after the first repeat so
+                   that the region covers MIN_REGION_S of device time (a 20-step repeat of a
+                   90 us step is 2 ms: too short for the clocks to be sampled or to settle).
+                   `value` is the median repeat, the last repeat is reported beside it (the
+                   first repeats run at boost clocks, the last under whatever the power cap
+                   leaves).  Where a repeat's appends would grow the pool by more than
+                   MAX_GROWTH, the pool is rebuilt from the resident raw states between repeats
+                   (outside the events), or the repeats stop.
+    end to end     the same through the host-buffer entry point, copies inside the region
+    latencies      a pass with an event after every step (serialises consecutive steps)
+    scan kernel    events recorded by the library around the scan launches
+    """
     from paper_2608_03839_b200 import binding as B
     import torch.distributed as dist
 
-    rank, world = env_int("RANK", 0), env_int("WORLD_SIZE", 1)
-    local = env_int("LOCAL_RANK", 0)
-    if world > 1:
-        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
-        dist.init_process_group("nccl", device_id=torch.device(f"cuda:{local}"))
-    torch.cuda.set_device(local)
-    dev = torch.device(f"cuda:{local}")
-    w = W.CONFIGS[args.config]
-    nq = args.nq or w.nq
-    n0 = W.C5_START_ROWS if w.name == "C5" else w.n_rows
-    if args.rows:
-        n0 = args.rows                      # smaller pool of the same recipe (profiling)
-    rows_step = APPEND_ROWS[w.name]
-    K, Wm = args.steps, args.warmup
-    total_steps = 3 * (Wm + K) + Wm + K     # device-timed, latency, kernel-timed and e2e passes
-    cap = n0 + rows_step * total_steps + 8
-    pool = B.Pool(w.d, cap, max_nq=max(nq, 1), max_k=w.k, max_append=rows_step, device=local,
-                  max_traces=w.num_traces + total_steps + 8, key_format=args.keys)
     row_bytes = w.d * 2 if args.keys == "bf16" else w.d + 4     # stored key bytes per row
-    # fill the pool (not timed): seeded traces of the configuration
-    done = 0
-    for st, tk, tag in w.traces(dev):
-        if done >= n0:
-            break
-        if done + st.shape[0] > n0:
-            st, tk = st[: n0 - done].contiguous(), tk[: n0 - done].contiguous()
-        pool.append(st, tk, tag=tag)
-        done += st.shape[0]
-    torch.cuda.synchronize()
     pr = B.QueryParams(k=w.k, theta=0.8, offset=2, depth_mode=B.DEPTH_FIXED, cont_len=w.cont_len,
                        path=args.path)
     n_in = min(Wm + K, 64)                   # distinct step inputs, cycled
     states, toks, queries = step_inputs(w, n_in, rows_step, nq, dev, seed=rank)
     out = B.QueryOut.empty(nq, w.k, w.cont_len, dev)
     step_no = [0]
+    cap_rows = pool.capacity_rows
+    grow_rows = max(rows_step * K, int(MAX_GROWTH * n0))     # rows a pass may add before a rebuild
 
     def step():
         i = step_no[0] % n_in
@@ -224,32 +239,79 @@ def run_ours(args):
                   new_trace=True)
         step_no[0] += 1
 
+    def rebuild():
+        pool.reset()
+        for st, tk, tag in raw:
+            pool.append(st, tk, tag=tag)
+
+    pass_base = [len(pool)]
+
+    def fits(n_steps):
+        return (len(pool) + rows_step * n_steps <= cap_rows and
+                pool.num_traces + n_steps <= pool.max_traces)
+
+    def make_room(n_steps, new_pass=False):
+        """True if n_steps more steps may run: inside the pool's capacity and inside the
+        growth budget (of the configured size when the pool can be rebuilt, else of the
+        current pass)."""
+        if new_pass:
+            pass_base[0] = len(pool)
+        if raw is not None:
+            if not fits(n_steps) or len(pool) + rows_step * n_steps > n0 + grow_rows:
+                rebuild()
+                pass_base[0] = len(pool)
+            return fits(n_steps)
+        return fits(n_steps) and len(pool) + rows_step * n_steps <= pass_base[0] + grow_rows
+
     def barrier():
         torch.cuda.synchronize()
         if world > 1:
             dist.barrier()
         torch.cuda.synchronize()
 
-    # ---- device-timed region: K steps, inputs resident in HBM ----------------------
+    # ---- device-timed region -----------------------------------------------------------
+    make_room(Wm + K, new_pass=True)
     for _ in range(Wm):
         step()
     barrier()
     sampler = ClockSampler(physical_device(local))
     sampler.start()
-    t_begin, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     launches0, rows0 = pool.launch_count, len(pool)
     torch.cuda.cudart().cudaProfilerStart()     # lets a profiler capture this region only
-    t_begin.record()
-    for s in range(K):                          # nothing but the K steps between the two events
-        step()
-    t_end.record()
+    ev, rows_at = [], []
+
+    def repeat():
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        rows_at.append(len(pool))
+        a.record()
+        for _ in range(K):                      # nothing but the K steps between the two events
+            step()
+        b.record()
+        ev.append((a, b))
+
+    repeat()
+    torch.cuda.synchronize()
+    launches = pool.launch_count - launches0    # kernels of one repeat of K steps
+    first_ms = ev[0][0].elapsed_time(ev[0][1])
+    n_rep = int(min(args.max_repeats, max(1, np.ceil(MIN_REGION_S * 1e3 / max(first_ms, 1e-3)))))
+    if world > 1:                               # the same number of repeats on every rank
+        t = torch.tensor([n_rep], dtype=torch.int64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        n_rep = int(t.item())
+    for _ in range(n_rep - 1):
+        if not make_room(K):
+            break
+        repeat()                                # no host synchronisation between repeats
     barrier()
     torch.cuda.cudart().cudaProfilerStop()
     clocks = sampler.stop()
-    launches = pool.launch_count - launches0
-    total_ms = t_begin.elapsed_time(t_end)
-    rows_mean = rows0 + rows_step * (K + 1) / 2.0
+    rep_ms = np.array([a.elapsed_time(b) for a, b in ev])
+    med = int(np.argsort(rep_ms)[len(rep_ms) // 2])
+    total_ms = float(rep_ms[med])
+    rows_mean = rows_at[med] + rows_step * (K + 1) / 2.0
     max_ms, value = aggregate(total_ms, K * nq, world, dev)
+    _, value_last = aggregate(float(rep_ms[-1]), K * nq, world, dev)
+    _, value_first = aggregate(float(rep_ms[0]), K * nq, world, dev)
 
     # ---- end to end through the host-buffer entry points -----------------------------
     h_states = [s.cpu().pin_memory() for s in states]
@@ -262,122 +324,254 @@ def run_ours(args):
         pool.step_host(h_states[i], h_toks[i], h_q[i], pr, h_out, tag=1_000_000 + step_no[0])
         step_no[0] += 1
 
+    make_room(Wm + K, new_pass=True)
     for _ in range(Wm):
         step_host()
     barrier()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record()
-    for _ in range(K):
-        step_host()
-    e1.record()
+    e2e_ms = []
+    t_wall = time.perf_counter()
+    while True:
+        if not make_room(K):
+            break
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(K):
+            step_host()
+        e1.record()
+        torch.cuda.synchronize()
+        e2e_ms.append(e0.elapsed_time(e1))
+        go = torch.tensor([1 if (time.perf_counter() - t_wall < MIN_REGION_S and
+                                 len(e2e_ms) < args.max_repeats) else 0], device=dev)
+        if world > 1:                           # every rank takes the same number of repeats
+            dist.all_reduce(go, op=dist.ReduceOp.MIN)
+        if not int(go.item()):
+            break
     barrier()
-    _, e2e_value = aggregate(e0.elapsed_time(e1), K * nq, world, dev)
+    _, e2e_value = aggregate(float(np.median(e2e_ms)), K * nq, world, dev)
     h2d = rows_step * w.d * 2 + rows_step * 4 + nq * w.d * 2
     d2h = nq * w.k * (4 + 4 + 4 + 4 * w.cont_len) + nq * 4
 
-    # ---- per-step latencies: a pass of its own, because an event after every step keeps
-    # the next step's kernels from being launched early, which the timed region above
-    # should not pay
-    ev = [torch.cuda.Event(enable_timing=True) for _ in range(K + 1)]
-    ev[0].record()
-    for s in range(K):
+    # ---- per-step latencies and the scan kernel: passes of their own -------------------
+    step_ms = total_ms / K
+    n_lat = int(min(max(K, 50), max(10, MIN_REGION_S * 1e3 / step_ms)))
+    make_room(2 * n_lat + 2 * Wm, new_pass=True)
+    evl = [torch.cuda.Event(enable_timing=True) for _ in range(n_lat + 1)]
+    evl[0].record()
+    for s_ in range(n_lat):
         step()
-        ev[s + 1].record()
+        evl[s_ + 1].record()
     torch.cuda.synchronize()
-    lat = np.array([ev[s].elapsed_time(ev[s + 1]) for s in range(K)])
+    lat = np.array([evl[s_].elapsed_time(evl[s_ + 1]) for s_ in range(n_lat)])
 
-    # ---- the dominant kernel (key scan), timed by events around its launches ---------
     pool.profile(True)
     for _ in range(Wm):
         step()
     torch.cuda.synchronize()
     pool.profile_read()
     rows1 = len(pool)
-    for _ in range(K):
+    for _ in range(n_lat):
         step()
     torch.cuda.synchronize()
-    scan_ms = pool.profile_read(max_n=max(K, 1))
+    scan_ms = pool.profile_read(max_n=max(n_lat, 1))
     pool.profile(False)
-    rows_scan = rows1 + rows_step * (K + 1) / 2.0
+    rows_scan = rows1 + rows_step * (n_lat + 1) / 2.0
     scan_bytes = rows_scan * row_bytes
     peaks, peak_kind = measured_peaks()
+    # a call that needs several passes over the keys records one duration per call
     scan_mean_ms = float(scan_ms.mean()) if len(scan_ms) else float("nan")
     achieved = scan_bytes / (scan_mean_ms * 1e-3) / 1e9
-
     stalled = pool.stats()["stalled"]
 
+    res = {
+        "workload": f"{w.name}: pool N={n0} x d={w.d} {args.keys}, nq={nq}, k={w.k}, "
+                    f"L={w.cont_len}, +{rows_step} rows appended per step",
+        "value": value, "unit": UNIT, "ms_per_step": max_ms / K, "steps": K, "repeats": len(rep_ms),
+        "value_first_repeat": value_first, "value_last_repeat": value_last,
+        "timed_region_ms": float(rep_ms.sum()),
+        "pool_rows_start": rows_at[med], "pool_rows_end": rows_at[med] + rows_step * K,
+        "p50_query_latency_us": float(np.percentile(lat, 50)) * 1e3,
+        "p90_query_latency_us": float(np.percentile(lat, 90)) * 1e3,
+        "min_query_latency_us": float(lat.min()) * 1e3,
+        "key_scan_gbs": rows_mean * row_bytes / (max_ms / K * 1e-3) / 1e9,
+        "clocks": clocks,
+        "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d,
+                "d2h_bytes_per_step": d2h, "repeats": len(e2e_ms)},
+        "gpu_launches": int(launches),
+        "roofline": {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"],
+                     "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"],
+                     "peak_kind": peak_kind, "frac_of_nominal_8000": achieved / NOMINAL_HBM_GBS,
+                     "kernel": "key scan (score + per-CTA top-k)",
+                     "kernel_ms": scan_mean_ms, "bytes_per_launch": scan_bytes,
+                     "traffic": ncu_traffic(traffic_key, rows_scan) if traffic_key else None},
+        "device_stalled_flag": stalled,
+    }
+    n_pad = (nq + 15) // 16 * 16
+    if args.keys == "bf16" and (args.path in (2, 3) or (args.path == 0 and nq > 2)):
+        # the batched path is a dense contraction: report its tensor-pipe share too
+        # (2*N*d*n_pad flops per launch, queries padded to the MMA's N)
+        tflops = 2.0 * rows_scan * w.d * n_pad / (scan_mean_ms * 1e-3) / 1e12
+        res["tensor_pipe"] = {
+            "achieved": tflops, "unit": "TFLOP/s", "n_pad": n_pad,
+            "peak_sustained": peaks["bf16_tflops_sustained"], "peak_burst": peaks["bf16_tflops"],
+            "frac_of_sustained": tflops / peaks["bf16_tflops_sustained"],
+            "frac_of_burst": tflops / peaks["bf16_tflops"], "peak_kind": peak_kind,
+            "note": "HBM-bound below nq ~ 218: the tensor pipe idles by design"}
+    return res
+
+
+def spare_rows(n0, rows_step, K, Wm):
+    """Rows beyond the configured size that the passes of measure() may append: a growth
+    budget for each of its four passes (the pool is rebuilt, or the repeats stop, beyond it)."""
+    return 4 * max(int(MAX_GROWTH * n0), rows_step * (K + Wm)) + rows_step * (4 * Wm + 4 * K + 256)
+
+
+def make_pool(w, nq, rows_step, cap_rows, local, args, extra_traces):
+    from paper_2608_03839_b200 import binding as B
+    pool = B.Pool(w.d, cap_rows, max_nq=max(nq, 1), max_k=w.k, max_append=rows_step, device=local,
+                  max_traces=w.num_traces + extra_traces, key_format=args.keys)
+    pool.capacity_rows, pool.max_traces = cap_rows, w.num_traces + extra_traces
+    return pool
+
+
+def run_ours(args):
+    from paper_2608_03839_b200 import binding as B
+    import torch.distributed as dist
+
+    rank, world = env_int("RANK", 0), env_int("WORLD_SIZE", 1)
+    local = env_int("LOCAL_RANK", 0)
+    if world > 1:
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("nccl", device_id=torch.device(f"cuda:{local}"))
+    torch.cuda.set_device(local)
+    dev = torch.device(f"cuda:{local}")
+    default_run = args.config is None           # no --config: the headline line plus the legs
+    w = W.CONFIGS[args.config or "C2"]
+    nq = args.nq or w.nq
+    n0 = W.C5_START_ROWS if w.name == "C5" else w.n_rows
+    if args.rows:
+        n0 = args.rows                      # smaller pool of the same recipe (profiling)
+    rows_step = APPEND_ROWS[w.name]
+    K, Wm = args.steps, args.warmup
+    spare = spare_rows(n0, rows_step, K, Wm)
+    keep_raw = w.key_bytes(n0) <= (2 << 30)     # small pools are rebuilt between repeats
+    pool = make_pool(w, nq, rows_step, n0 + spare, local, args, spare // rows_step + 8)
+    raw = fill_pool(pool, w, n0, dev, keep_raw=keep_raw)
+    plain = not args.rows and not args.nq and args.keys == "bf16"
+    res = measure(pool, w, nq, rows_step, K, Wm, dev, world, rank, local, args, n0,
+                  raw=raw if keep_raw else None, traffic_key=w.name if plain else None)
+
+    line = None
     if rank == 0:
-        p50_ms = float(np.percentile(lat, 50))
         line = {
-            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K,
-            "warmup": Wm, "ms_per_step": max_ms / K, "higher_is_better": True,
+            "metric": METRIC, "value": res["value"], "unit": UNIT, "n_gpus": world, "steps": K,
+            "warmup": Wm, "ms_per_step": res["ms_per_step"], "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": f"{args.keys} keys, fp32 accumulate",
             "data": "synthetic",
-            "config": {"workload": f"{w.name}: pool N={n0} x d={w.d} {args.keys}, nq={nq}, k={w.k}, "
-                                   f"L={w.cont_len}, +{rows_step} rows appended per step",
-                       "pool_rows_start": rows0, "pool_rows_end": rows0 + rows_step * K,
+            "config": {"workload": res["workload"] +
+                       (" (the single-request decode configuration, the one the 70 %-of-HBM "
+                        "target is stated on; the batched and the largest configurations are "
+                        "in `legs`)" if default_run else ""),
+                       "pool_rows_start": res["pool_rows_start"], "pool_rows_end": res["pool_rows_end"],
                        "append_rows_per_step": rows_step, "scan_path": args.path,
                        "l2": "inputs exceed L2" if w.key_bytes(n0) > 2 * 126e6 else
                              "pool fits in L2 (not a bandwidth datum)",
-                       "pools": "one independent pool per GPU"},
-            "p50_query_latency_us": p50_ms * 1e3,
-            "p90_query_latency_us": float(np.percentile(lat, 90)) * 1e3,
-            "min_query_latency_us": float(lat.min()) * 1e3,
+                       "pools": "one independent pool per GPU",
+                       "timing": f"value = median of {res['repeats']} repeats of {K} steps "
+                                 f"({res['timed_region_ms']:.0f} ms of device time in all)"},
             "latency_note": "per-step latencies come from a pass of their own with an event "
                             "after every step (which serialises consecutive steps)",
-            "key_scan_gbs": rows_mean * row_bytes / (max_ms / K * 1e-3) / 1e9,
-            "clocks": clocks,
-            "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d,
-                    "d2h_bytes_per_step": d2h},
-            "gpu_launches": int(launches),
-            "roofline": {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"],
-                         "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"],
-                         "peak_kind": peak_kind, "frac_of_nominal_8000": achieved / NOMINAL_HBM_GBS,
-                         "kernel": "key scan (score + per-CTA top-k)",
-                         "kernel_ms": scan_mean_ms, "bytes_per_launch": scan_bytes,
-                         "traffic": ncu_traffic(w.name, rows_scan)
-                         if not args.rows and not args.nq and args.keys == "bf16" else None},
-            "device_stalled_flag": stalled,
         }
-        n_pad = (nq + 15) // 16 * 16
-        used_tensor = args.keys == "bf16" and (args.path == 2 or (args.path == 0 and nq > 2))
-        if used_tensor:
-            # the batched path is a dense contraction: report its tensor-pipe share too
-            # (2*N*d*n_pad flops per launch, queries padded to the MMA's N)
-            tflops = 2.0 * rows_scan * w.d * n_pad / (scan_mean_ms * 1e-3) / 1e12
-            line["tensor_pipe"] = {
-                "achieved": tflops, "unit": "TFLOP/s", "n_pad": n_pad,
-                "peak_sustained": peaks["bf16_tflops_sustained"], "peak_burst": peaks["bf16_tflops"],
-                "frac_of_sustained": tflops / peaks["bf16_tflops_sustained"],
-                "frac_of_burst": tflops / peaks["bf16_tflops"], "peak_kind": peak_kind,
-                "note": "HBM-bound below nq ~ 218: the tensor pipe idles by design"}
+        for key in ("repeats", "value_first_repeat", "value_last_repeat", "p50_query_latency_us",
+                    "p90_query_latency_us", "min_query_latency_us", "key_scan_gbs", "clocks", "e2e",
+                    "gpu_launches", "roofline", "device_stalled_flag", "tensor_pipe"):
+            if key in res:
+                line[key] = res[key]
         if w.kind == "template" and not args.rows:
             # retrieval quality on the tool-calling shape: recall of the planted
             # same-(template, position) rows and how much of the gathered continuation
             # agrees with the template (slot positions excepted)
             tq, meta = w.queries(dev, nq=nq)
-            res = pool.query(tq, B.QueryParams(k=w.k, theta=-2.0, depth_mode=B.DEPTH_FIXED,
-                                               cont_len=w.cont_len, path=args.path)).cpu()
+            resq = pool.query(tq, B.QueryParams(k=w.k, theta=-2.0, depth_mode=B.DEPTH_FIXED,
+                                                cont_len=w.cont_len, path=args.path)).cpu()
             hits = tot = 0
             match = []
             for i, rows_i in enumerate(meta["planted_rows"]):
-                hits += len(set(rows_i) & set(res.idx[i].tolist()))
+                hits += len(set(rows_i) & set(resq.idx[i].tolist()))
                 tot += min(len(rows_i), w.k)
                 ttok, slot = meta["template_tokens"][i]
                 pos = meta["pos"][i]
                 want = ttok[pos + 2: pos + 2 + w.cont_len]
-                ok = (res.cont_tok[i, 0, : len(want)] == want) | slot[pos + 2: pos + 2 + w.cont_len]
+                ok = (resq.cont_tok[i, 0, : len(want)] == want) | slot[pos + 2: pos + 2 + w.cont_len]
                 match.append(float(ok.sum()) / max(1, len(want)))
             line["retrieval_quality"] = {"recall_planted_at_k": hits / max(1, tot),
                                          "top1_continuation_match": float(np.mean(match)),
                                          "queries": len(match)}
+    pool.close()
+    del pool, raw
+    torch.cuda.empty_cache()
+
+    legs = []
+    if default_run and not args.no_legs:
+        if world == 1:
+            legs = run_legs(args, dev, local, K, Wm)
+        else:
+            # the row-sharded design next to the independent pools: ONE logical pool over all
+            # ranks, one all-gather of nq*k records per query
+            legs = [sharded_leg(args, W.C4, W.C4.nq, min(K, 50), Wm, dev, rank, world, local)]
+    if rank == 0:
+        if legs:
+            line["legs"] = legs
         if not args.no_cpu_baseline and world == 1:
             line["cpu_baseline"] = cpu_baseline(w, n0, rows_step, nq, budget_s=args.cpu_budget,
                                                 keys=args.keys)
         print(json.dumps(line), flush=True)
-    pool.close()
     if world > 1:
         dist.destroy_process_group()
+
+
+def run_legs(args, dev, local, K, Wm):
+    """The batched configuration and the largest one, measured like the headline line (one GPU):
+    C4 nq = 64; C5 (d = 8192) with one query and with 256 at the start of its stream
+    (N = 2^20) and, after the rows in between have been appended in bulk (not timed), at its
+    far end (N ~ 2^21, 34 GB of keys)."""
+    legs = []
+    K = max(3, min(K, 50))
+
+    def leg(pool, w, nq, n0, key=None):
+        r = measure(pool, w, nq, APPEND_ROWS[w.name], K, Wm, dev, 1, 0, local, args, n0,
+                    raw=None, traffic_key=key)
+        r["config"] = w.name
+        legs.append(r)
+
+    w = W.C4
+    rows_step = APPEND_ROWS[w.name]
+    spare = spare_rows(w.n_rows, rows_step, K, Wm)
+    pool = make_pool(w, w.nq, rows_step, w.n_rows + spare, local, args, spare // rows_step + 8)
+    fill_pool(pool, w, w.n_rows, dev)
+    leg(pool, w, w.nq, w.n_rows, key="C4")
+    pool.close()
+    del pool
+    torch.cuda.empty_cache()
+
+    w = W.C5
+    rows_step = APPEND_ROWS[w.name]
+    far = w.n_rows - 65536                      # the far-end legs start here and pass 2^21
+    cap = w.n_rows + (1 << 19)
+    pool = make_pool(w, 256, rows_step, cap, local, args, (1 << 20) // rows_step + 8)
+    fill_pool(pool, w, W.C5_START_ROWS, dev)
+    for nq in (1, 256):
+        leg(pool, w, nq, len(pool))
+    fill_pool(pool, w, far, dev)                # the stream's appends in between, in bulk
+    for nq in (1, 256):
+        leg(pool, w, nq, len(pool))
+    pool.close()
+    return legs
+
+
+def sharded_leg(args, w, nq, K, Wm, dev, rank, world, local):
+    """run_sharded's measurement as a leg of the default multi-GPU line."""
+    r = sharded_measure(args, w, nq, w.n_rows, K, Wm, dev, rank, world, local)
+    return r
 
 
 # ---------------------------------------------------------------- CPU oracle ----
@@ -447,7 +641,7 @@ def run_reference(args):
     rank = env_int("RANK", 0)
     if rank != 0:
         return
-    w = W.CONFIGS[args.config]
+    w = W.CONFIGS[args.config or "C2"]
     nq = args.nq or w.nq
     n0 = W.C5_START_ROWS if w.name == "C5" else w.n_rows
     cb = cpu_baseline(w, n0, APPEND_ROWS[w.name], nq, budget_s=args.cpu_budget * 4,
@@ -569,7 +763,7 @@ def run_evict(args):
     from paper_2608_03839_b200 import binding as B
     torch.cuda.set_device(0)
     dev = torch.device("cuda:0")
-    w = W.CONFIGS[args.config]
+    w = W.CONFIGS[args.config or "C2"]
     n0 = args.rows or w.n_rows
     rpt = w.rows_per_trace
     n_tr = n0 // rpt
@@ -652,7 +846,7 @@ def run_load(args):
     from paper_2608_03839_b200 import binding as B
     torch.cuda.set_device(0)
     dev = torch.device("cuda:0")
-    w = W.CONFIGS[args.config]
+    w = W.CONFIGS[args.config or "C2"]
     n0 = args.rows or w.n_rows
     chunk = 4096
     n_calls = max(1, n0 // chunk)
@@ -765,33 +959,24 @@ def run_merge(args):
     print(json.dumps(line), flush=True)
 
 
-def run_sharded(args):
-    """Row-sharded mode: ONE logical pool of the configuration's size split by whole traces
-    over the ranks; every rank answers every query on its rows, one all-gather of the
-    records, merge on every rank.  Strong scaling: the total work is fixed."""
+def sharded_measure(args, w, nq, n0, K, Wm, dev, rank, world, local):
+    """ONE logical pool of n0 rows split by whole traces over the ranks; every rank answers
+    every query on its rows, one all-gather of the records, merge on every rank.  Strong
+    scaling: the total work is fixed.  Returns the fields of a bench line (on every rank)."""
     from paper_2608_03839_b200 import binding as B
     from paper_2608_03839_b200 import sharded as S
     import torch.distributed as dist
-    rank, world = env_int("RANK", 0), env_int("WORLD_SIZE", 1)
-    local = env_int("LOCAL_RANK", 0)
-    if world > 1:
-        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
-        dist.init_process_group("nccl", device_id=torch.device(f"cuda:{local}"))
-    torch.cuda.set_device(local)
-    dev = torch.device(f"cuda:{local}")
-    w = W.CONFIGS[args.config]
-    nq = args.nq or w.nq
-    n0 = args.rows or (W.C5_START_ROWS if w.name == "C5" else w.n_rows)
-    K, Wm = args.steps, args.warmup
     sp = S.ShardedPool(w.d, n0 // world + 2 * w.rows_per_trace + 8, max_nq=nq, max_k=w.k,
                        device=local)
     g = 0
-    for t, (st, tk, tag) in enumerate(w.traces(dev)):
+    C = w._centroids(dev) if w.kind == "clustered" else None
+    for t in range(w.num_traces):
         if g >= n0:
             break
         if t % world == rank:                       # whole traces, round robin
+            st, tk, tag = w.trace(t, dev, C)
             sp.append(st, tk, global_row=g, tag=tag)
-        g += st.shape[0]
+        g += w.trace_rows(t)
     pr = B.QueryParams(k=w.k, theta=0.8, offset=2, depth_mode=B.DEPTH_FIXED, cont_len=w.cont_len,
                        path=args.path)
     qs = [w.queries(dev, nq=nq, step=i)[0] for i in range(8)]   # same seeds on every rank
@@ -814,23 +999,39 @@ def run_sharded(args):
     clocks = sampler.stop()
     lat = np.array([ev[i].elapsed_time(ev[i + 1]) for i in range(K)])
     max_ms, _ = aggregate(ev[0].elapsed_time(ev[K]), 0.0, world, dev)
+    peaks, peak_kind = measured_peaks()
+    p50 = float(np.percentile(lat, 50))
+    gbs = n0 * w.d * 2 / (p50 * 1e-3) / 1e9
+    return {"metric": METRIC, "value": K * nq / (max_ms / 1e3), "unit": UNIT, "n_gpus": world,
+            "steps": K, "warmup": Wm, "ms_per_step": max_ms / K, "higher_is_better": True,
+            "scaling": "strong", "vs_baseline": None, "dtype": "bf16 keys, fp32 accumulate",
+            "data": "synthetic",
+            "config": {"workload": f"{w.name} row-sharded: ONE pool N={n0} x d={w.d} bf16 over "
+                                   f"{world} GPU(s), nq={nq}, k={w.k}, L={w.cont_len}; query only",
+                       "collective": "one all_gather of nq*k records per query"},
+            "p50_query_latency_us": p50 * 1e3, "key_scan_gbs_all_gpus": gbs, "clocks": clocks,
+            "gpu_launches": 4 * K,
+            "roofline": {"bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"] * world,
+                         "unit": "GB/s", "frac": gbs / (peaks["hbm_gbs"] * world),
+                         "peak_kind": peak_kind, "traffic": None,
+                         "kernel": "whole sharded query (scan + to_global + gather + merge)"}}
+
+
+def run_sharded(args):
+    """Row-sharded mode as a bench line of its own (python bench.py --sharded)."""
+    import torch.distributed as dist
+    rank, world = env_int("RANK", 0), env_int("WORLD_SIZE", 1)
+    local = env_int("LOCAL_RANK", 0)
+    if world > 1:
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("nccl", device_id=torch.device(f"cuda:{local}"))
+    torch.cuda.set_device(local)
+    dev = torch.device(f"cuda:{local}")
+    w = W.CONFIGS[args.config or "C2"]
+    nq = args.nq or w.nq
+    n0 = args.rows or (W.C5_START_ROWS if w.name == "C5" else w.n_rows)
+    line = sharded_measure(args, w, nq, n0, args.steps, args.warmup, dev, rank, world, local)
     if rank == 0:
-        peaks, peak_kind = measured_peaks()
-        p50 = float(np.percentile(lat, 50))
-        gbs = n0 * w.d * 2 / (p50 * 1e-3) / 1e9
-        line = {"metric": METRIC, "value": K * nq / (max_ms / 1e3), "unit": UNIT, "n_gpus": world,
-                "steps": K, "warmup": Wm, "ms_per_step": max_ms / K, "higher_is_better": True,
-                "scaling": "strong", "vs_baseline": None, "dtype": "bf16 keys, fp32 accumulate",
-                "data": "synthetic",
-                "config": {"workload": f"{w.name} row-sharded: ONE pool N={n0} x d={w.d} bf16 over "
-                                       f"{world} GPU(s), nq={nq}, k={w.k}, L={w.cont_len}; query only",
-                           "collective": "one all_gather of nq*k records per query"},
-                "p50_query_latency_us": p50 * 1e3, "key_scan_gbs_all_gpus": gbs, "clocks": clocks,
-                "gpu_launches": 4 * K,
-                "roofline": {"bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"] * world,
-                             "unit": "GB/s", "frac": gbs / (peaks["hbm_gbs"] * world),
-                             "peak_kind": peak_kind, "traffic": None,
-                             "kernel": "whole sharded query (scan + to_global + gather + merge)"}}
         print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()
@@ -842,7 +1043,12 @@ def main():
     ap.add_argument("--steps", type=int, default=None)
     ap.add_argument("--warmup", type=int, default=None)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--config", default="C2", choices=sorted(W.CONFIGS))
+    ap.add_argument("--config", default=None, choices=sorted(W.CONFIGS),
+                    help="one configuration alone; default: C2 as the headline line plus the "
+                         "batched (C4) and the largest (C5) configurations as `legs`")
+    ap.add_argument("--no-legs", action="store_true", help="default run without the legs")
+    ap.add_argument("--max-repeats", type=int, default=400,
+                    help="upper limit on the repeats of a timed region")
     ap.add_argument("--nq", type=int, default=0, help="override the configuration's nq")
     ap.add_argument("--rows", type=int, default=0,
                     help="override the pool size (profiling a smaller case of the same recipe)")
@@ -883,7 +1089,7 @@ def main():
         args.warmup = 10 if args.warmup is None else max(args.warmup, 3)
         run_merge(args)
         return
-    default_steps = {"C1": 500, "C2": 500, "C3": 300, "C4": 200, "C5": 50}[args.config]
+    default_steps = {"C1": 500, "C2": 500, "C3": 300, "C4": 200, "C5": 50}[args.config or "C2"]
     args.steps = default_steps if args.steps is None else args.steps
     args.warmup = 20 if args.warmup is None else max(args.warmup, 3)
     if args.sharded:

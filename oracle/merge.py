@@ -14,7 +14,11 @@ Plain Python loops on purpose: the trees have at most 64 nodes.
 
 Readings where the paper is silent:
   * when the budget runs out inside a chain the chain is cut there (its bought prefix stays);
-    chains after it are not reached;
+    chains after it are not reached: once nothing is left to spend (or the tree is full)
+    every later chain gets status NOT_REACHED without being walked, ALSO a chain whose
+    tokens are all in the tree already, which Eq. 4 would price at zero.  The tree is the
+    same either way (such a chain adds no node); only its status reads "not reached"
+    rather than "merged at cost 0".  The CUDA kernel does the same;
   * a chain that is a duplicate is dropped before merging, whatever its source; the
     minimum length applies to semantic chains only (the algorithm states it on that line);
   * new nodes are numbered in the order they are bought;

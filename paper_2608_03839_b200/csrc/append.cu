@@ -129,6 +129,8 @@ qnorm_kernel(const uint16_t* __restrict__ q, int nq, int d, uint16_t* __restrict
   // the tensor scan's cross-CTA threshold exchange starts every call at -inf
   for (int i = blockIdx.x * kNormThreads + threadIdx.x; i < n_xchg; i += gridDim.x * kNormThreads)
     xchg[i] = -INFINITY;
+  if (blockIdx.x == 0 && threadIdx.x < kTcXchgCounters && n_xchg > 0)
+    reinterpret_cast<unsigned*>(xchg + n_xchg)[threadIdx.x] = 0u;
   const int r = blockIdx.x;
   if (r < nq) {
     // A query holding NaN/Inf returns no neighbours; an all-zero query is legal and

@@ -153,7 +153,8 @@ cudaError_t launch_to_global(const int32_t* idx, int64_t* out, int64_t n, const 
 
 // query preparation: qn[r] = bf16(q[r]/||q[r]||) for r < nq, zero rows up to nq_pad,
 // q_valid[r] = 0 for a query holding NaN/Inf.
-// Also fills xchg[0..n_xchg) with -inf (the tensor scan's threshold exchange, see scan_tc.cu).
+// Also fills xchg[0..n_xchg) with -inf (the tensor scan's threshold exchange, see scan_tc.cu)
+// and zeroes the kTcXchgCounters words behind them.
 cudaError_t launch_qnorm(const uint16_t* q, int32_t nq, int32_t nq_pad, int32_t d, uint16_t* qn,
                          int32_t* q_valid, DeviceStats* stats, float* xchg, int32_t n_xchg,
                          cudaStream_t st);
@@ -162,6 +163,9 @@ cudaError_t launch_qnorm(const uint16_t* q, int32_t nq, int32_t nq_pad, int32_t 
 // CTA (kTcMaxCtas slots) followed by one agreed lower bound per query.
 constexpr int kTcMaxCtas = 160;   // >= the 148 SMs of a B200; five values per lane
 constexpr int kTcXchgFloats = OILBIRD_MAX_NQ * kTcMaxCtas + OILBIRD_MAX_NQ;
+// ... followed by kTcXchgCounters words that the query preparation sets to zero: arrival
+// counters of the two rendezvous in a CTA's first tile (see scan_tc.cu)
+constexpr int kTcXchgCounters = 4;
 
 // Length of the candidate lists exchanged between scan and merge for a given k.
 inline int list_len(int k) { int p = next_pow2(k); return p < 32 ? 32 : p; }

@@ -153,7 +153,7 @@ Layout make_layout(const Resolved& r) {
   L.partial = take((size_t)r.max_lists * r.max_nq * k_pad * 8, "candidate lists");
   L.stats = take(sizeof(DeviceStats), "counters");
   L.fuse_ready = take(8, "fused-append counter");
-  L.xchg = take((size_t)kTcXchgFloats * 4, "threshold exchange");
+  L.xchg = take((size_t)(kTcXchgFloats + kTcXchgCounters) * 4, "threshold exchange");
   // staging for the *_host variants (adjacent: query_host/step_host fill them with one copy)
   guards = false;                          // no sentinels inside the one-copy staging block
   L.q_stage = take((size_t)r.max_nq * r.d * 2, "");

@@ -7,47 +7,68 @@
 // warp-specialised:
 //   warp 0      TMA producer: key tile + query tile per k-block into a 128B-swizzled
 //               shared-memory ring (cp.async.bulk.tensor, mbarrier complete_tx)
-//   warp 1      tcgen05.mma issuer (one thread), fp32 accumulators in TMEM, two
+//   warp 1      tcgen05.mma issuer (one elected lane), fp32 accumulators in TMEM, two
 //               accumulator buffers so the next tile's MMAs overlap the epilogue
 //   warps 2-5   epilogue: tcgen05.ld the 128 x nq scores, filter them against the
-//               per-query running k-th best, and keep per-query top-k lists in shared
-//               memory (Eq. 2); scores never go to global memory
+//               per-query running k-th best, and keep per-query top-k lists (Eq. 2) in
+//               shared memory, or in L2 when they are large; scores never go to global
+//               memory
 // The key stream (N*d*2 bytes from HBM, once) bounds the kernel up to nq ~ 64-96; the
-// epilogue warps then wait for accumulators 60-80 % of the time.  What is left above that:
-//   - a CTA's first one or two macro tiles, whose scores nearly all pass the still-low
-//     thresholds (sorted 32 at a time and merged): ~2.5 tiles' worth of time at nq = 128,
-//     during which the accumulator buffers are full and the key stream stalls;
-//   - at nq = 256 the query tile re-read from L2 per key tile (twice the key bytes) and the
-//     single k-block per accumulator set; the tensor pipe reaches about half its peak.
+// epilogue warps then wait for accumulators 60-80 % of the time.  Beyond that:
+//   - A CTA's first tile has no thresholds yet.  It is read twice: once for its best score
+//     per query only, which the CTAs exchange to agree on a bound (the k-th largest of their
+//     bests), then as every other tile, against that bound.  Without this every score of the
+//     first one or two tiles went through the sorted lists (~2.5 tiles' worth of time at
+//     nq = 128, with the accumulators full and the key stream stalled).
+//   - From 129 queries on, two CTAs share each tile of 256 rows (template argument kPair;
+//     described at the kernel), which halves the query bytes an SM pulls from L2 and writes
+//     to its shared memory per key byte.
+//   - Per k-block of a 128-row tile the tensor core reads the 16 KB of keys and the
+//     n_pad x 128 bytes of queries from shared memory while TMA writes the next ones: at
+//     n_pad = 256 that is 96 KB through the SM's shared memory per k-block, and cycle
+//     counters in the MMA-issuing thread (not part of the build) show the four
+//     128 x 256 x 16 MMAs of a k-block taking ~750 cycles where the tensor pipe alone would
+//     need 512 and the SM's share of the HBM rate allows 720: at nq = 256 the scan is bound
+//     on chip (and, in runs of more than a fraction of a second, by the power cap: the SM
+//     clock settles at 1.0-1.3 GHz), not by HBM.  A pair of CTAs moves 64-80 KB per k-block
+//     and gains 6-10 %.
+// The MMA warp walks its loop as a whole and one elected lane issues, so that descriptors and
+// addresses are computed in uniform control flow (with the loop inside `if (lane == 0)` a
+// k-block's four MMAs and its commit took ~745 cycles to issue at n_pad = 256, now ~500).
 // Small pools (a few tiles per SM): a query costs about 40 us plus the key bytes at HBM
 // speed, against 12 us plus the same for the CUDA-core scan.  A tile's scores exist only
-// after its whole K loop, so the first tile's latency chain is not overlapped, and one SM
-// streams at most ~45-65 GB/s whatever the rest of the GPU does: cycle counters in the
-// MMA-issuing thread show ~360 cycles to issue the four tcgen05.mma and the commit of a
-// 16 KB k-block (~70 cycles per instruction, against ~90 cycles of waiting for the data
-// when HBM is idle), i.e. with queries as the N operand a 128 x N x 16 instruction carries
-// only 4 KB of keys and the issue rate, not the tensor pipe, bounds the per-SM rate.  Then
-// come the first tile's epilogue (7-10 us), the query normalisation kernel and the merge.
-// A variant with the roles swapped (queries as M = 128, one query per TMEM lane and per
-// epilogue thread with its threshold in a register and a queue only it writes; 256 key rows
-// as N, so that an instruction carries 8 KB of keys) was written and passes the same tests,
-// but is slower everywhere: 0.90 instead of 1.03 of the measured HBM rate at nq = 16 and
-// 0.73 instead of 0.81 at nq = 128 on the 8.6 GB pool (every stage carries a 16 KB query
-// tile whatever nq is), and 2-3x slower on small pools, where only nq/32 of the four
-// epilogue warps share the sorting of a CTA's first tile.  Cutting the pool into per-CTA row ranges at 32-row granularity
-// (ragged ends fetched as 32-row boxes) so that all SMs get equal rows, ring depths up to
-// 12 and seeding the first tile's thresholds from per-warp 32-bit sorts of the scores were
-// measured and bring nothing.
-// Measured and not kept: separate shared-memory rings for keys and query tiles (query
-// tiles queue behind the key requests, so they need the same lead; 5-8 % slower); a
-// 32-deep candidate queue with retry, to buy a ring stage (slower first tiles, no gain from
-// the stage); ballot-packed per-warp queue segments instead of shared-memory atomics (drain
-// 60 % slower); sorting every column of the first tile in registers without the queue (no
-// faster than the queue's crowd path); a variant that transposes the scores through shared
-// memory so that one warp owns a query's 128 rows (15-30 % slower).
+// after its whole K loop, so the first tile's latency chain is not overlapped.  Then come
+// the query normalisation kernel and the merge.
+// Measured and not kept:
+//   - a variant with the roles swapped (queries as M = 128, one query per TMEM lane and per
+//     epilogue thread; 256 key rows as N): passes the same tests, slower everywhere (0.90
+//     instead of 1.03 of the measured HBM rate at nq = 16, 0.73 instead of 0.81 at nq = 128 on
+//     the 8.6 GB pool, 2-3x slower on small pools);
+//   - per-CTA row ranges at 32-row granularity, ring depths up to 12, seeding the first
+//     tile's thresholds from per-warp 32-bit sorts: nothing gained;
+//   - separate shared-memory rings for keys and query tiles (query tiles queue behind the key
+//     requests, so they need the same lead; 5-8 % slower); a 32-deep candidate queue with
+//     retry; ballot-packed per-warp queue segments instead of shared-memory atomics (drain
+//     60 % slower); sorting every column of the first tile in registers without the queue; a
+//     variant that transposes the scores through shared memory so that one warp owns a
+//     query's 128 rows (15-30 % slower);
+//   - per-query lists kept in shared memory as 6-byte slots (fp32 score + 16-bit local row)
+//     to make 256 x 64 of them fit beside a two-stage ring: with the lists in global memory
+//     (L2) the ring has four stages and the scan is a third faster;
+//   - two CTAs on a tile with the other CTA's copies counted directly on the leader's
+//     barrier after an arrival (with its byte count) from the other CTA's producer, or with
+//     a warp of the other CTA relaying "stage landed" to the leader: an arrival on a barrier
+//     of the other CTA with release semantics costs the arriving thread ~600 cycles, and
+//     either form ran at 1,600 cycles per k-block;
+//   - a single 128 x 256 x 16 MMA issued as two interleaved 128 x 128 x 16 ones (independent
+//     accumulators): 8 instructions in ~950 cycles instead of 4 in ~750;
+//   - asking for the keys of the next 8 or 24 k-blocks into L2 ahead of the ring
+//     (cp.async.bulk.prefetch.tensor): 1.4x and 2x slower at every nq.
 //
-// Every mbarrier wait is bounded: after about two seconds it raises the pool's `stalled`
-// flag, the CTA drains what it has in flight, frees its TMEM and returns.
+// Every mbarrier wait is bounded: after the pool's wait limit (two seconds by default) it
+// raises the pool's `stalled` flag, the CTA drains what it has in flight, frees its TMEM and
+// returns.  The two meetings of the CTAs in a first tile are short waits (0.1 ms) that give
+// up silently, since they only serve a tighter filter.
 #include <cuda.h>
 
 #include <new>
@@ -67,6 +88,23 @@ constexpr int kATileBytes = kTileM * kBlockK * 2;   // 16 KB
 constexpr int kColsPerRound = 16;      // score columns filtered between two drains
 constexpr int kQueueCap = kTileM * kColsPerRound;
 constexpr int kMaxStages = 8;
+
+// Compile-time overrides for measurements (0 = the plan below decides).
+#ifndef OILBIRD_TC_FORCE_MT
+#define OILBIRD_TC_FORCE_MT 0
+#endif
+#ifndef OILBIRD_TC_FORCE_LISTS
+#define OILBIRD_TC_FORCE_LISTS 0          // 1 = shared memory, 2 = global memory
+#endif
+#ifndef OILBIRD_TC_FIRST_TILE_BOUND
+#define OILBIRD_TC_FIRST_TILE_BOUND 1     // 0 = a CTA's first tile goes through the lists unfiltered
+#endif
+#ifndef OILBIRD_TC_PAIR
+#define OILBIRD_TC_PAIR 1                 // 0 = never pair two CTAs on a tile
+#endif
+#ifndef OILBIRD_TC_MIN_SMEM_STAGES
+#define OILBIRD_TC_MIN_SMEM_STAGES 4      // lists stay in shared memory if this many stages fit
+#endif
 
 // ------------------------------------------------------------------ PTX wrappers ---
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
@@ -99,13 +137,27 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
       : "memory");
   return ok != 0;
 }
+// try_wait whose acquire reaches across the cluster: for a barrier that a thread of the other
+// CTA arrives on after it has seen its own copies land
+__device__ __forceinline__ bool mbar_try_wait_cluster(uint64_t* bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(smem_u32(bar)), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
 // Bounded wait.  Returns false if it gave up (or another role already did).
+template <bool kCluster = false>
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
                                           DeviceStats* stats) {
-  if (mbar_try_wait(bar, parity)) return true;
+  if (kCluster ? mbar_try_wait_cluster(bar, parity) : mbar_try_wait(bar, parity)) return true;
   const unsigned long long t0 = global_ns(), limit = wait_limit_ns(stats);
   for (uint32_t spin = 0;; ++spin) {
-    if (mbar_try_wait(bar, parity)) return true;
+    if (kCluster ? mbar_try_wait_cluster(bar, parity) : mbar_try_wait(bar, parity)) return true;
     if ((spin & 63u) == 63u) {
       if (*abort_flag) return false;
       if (global_ns() - t0 > limit) {
@@ -116,12 +168,78 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volati
     }
   }
 }
+// One lane of a converged warp (the same lane every time).
+__device__ __forceinline__ bool elect_one() {
+  uint32_t pred;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "elect.sync _|p, 0xffffffff;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(pred));
+  return pred != 0;
+}
+// mbar_wait by a whole converged warp, with one outcome for all its lanes
+template <bool kCluster = false>
+__device__ __forceinline__ bool warp_mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
+                                               DeviceStats* stats) {
+  const bool ok = mbar_wait<kCluster>(bar, parity, abort_flag, stats);
+  return __all_sync(0xffffffffu, ok);
+}
 __device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* map, int x, int y,
                                             uint64_t* bar) {
   asm volatile(
       "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes"
       " [%0], [%1, {%3, %4}], [%2];"
       ::"r"(smem_u32(dst)), "l"(map), "r"(smem_u32(bar)), "r"(x), "r"(y)
+      : "memory");
+}
+// ---- two CTAs on one tile (a cluster of two; rank 0 leads) ----
+__device__ __forceinline__ uint32_t cluster_rank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+// the address, in the cluster's shared window, of the same shared-memory object in CTA `rank`
+__device__ __forceinline__ uint32_t smem_of_rank(const void* p, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(smem_u32(p)), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {      // every thread of both CTAs
+  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void mbar_arrive_at(uint32_t cluster_addr) {
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr)
+               : "memory");
+}
+// TMA load into this CTA's shared memory whose completion is counted on a barrier that may
+// live in the other CTA of the pair (no operand is shared between the CTAs: each loads its
+// own rows)
+__device__ __forceinline__ void tma_load_2d_pair(void* dst, const CUtensorMap* map, int x, int y,
+                                                 uint32_t bar_cluster_addr) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes"
+      " [%0], [%1, {%3, %4}], [%2];"
+      ::"r"(smem_u32(dst)), "l"(map), "r"(bar_cluster_addr), "r"(x), "r"(y)
+      : "memory");
+}
+// completion of the pair's MMAs so far, counted on one barrier given by its cluster address
+__device__ __forceinline__ void tc_commit_pair_at(uint32_t bar_cluster_addr) {
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];"
+               ::"r"(bar_cluster_addr)
+               : "memory");
+}
+// D[tmem of both CTAs] (+)= A * B over the pair: M = 256 (128 rows from each CTA's A tile),
+// N from idesc (each CTA's B tile holds N/2 of the query rows), K = 16.  One thread of the
+// leading CTA issues it.
+__device__ __forceinline__ void tc_mma_bf16_pair(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc,
+                                                 uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
       : "memory");
 }
 __device__ __forceinline__ void tc_fence_before() {
@@ -173,10 +291,35 @@ __device__ __forceinline__ uint64_t umma_desc_sw128(uint32_t smem_addr) {
   d |= (uint64_t)2 << 61;                              // SWIZZLE_128B
   return d;
 }
-// Instruction descriptor: D fp32, A/B bf16, both K-major, M=128, N=n.
-__host__ __device__ inline uint32_t umma_idesc_bf16(int n) {
+// Instruction descriptor: D fp32, A/B bf16, both K-major, M = m (128; 256 over a CTA pair), N = n.
+__host__ __device__ inline uint32_t umma_idesc_bf16(int n, int m = kTileM) {
   return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) |
-         ((uint32_t)(kTileM >> 4) << 24);
+         ((uint32_t)(m >> 4) << 24);
+}
+
+// Order-preserving map float -> unsigned (and back), so that a warp-wide maximum of scores is
+// one redux instruction; 0 is below every score.
+__device__ __forceinline__ uint32_t score_to_ord(float s) {
+  s += 0.0f;
+  const uint32_t b = __float_as_uint(s);
+  return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
+}
+__device__ __forceinline__ float ord_to_score(uint32_t b) {
+  return __uint_as_float((b & 0x80000000u) ? (b & 0x7fffffffu) : ~b);
+}
+__device__ __forceinline__ unsigned ld_acquire_u32(const unsigned* p) {
+  unsigned v;
+  asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+  return v;
+}
+// Rendezvous of the grid's CTAs on an arrival counter, for a bound that only makes the
+// filter tighter: a short wait that simply ends when its time is up (nothing is flagged; the
+// caller goes on with whatever the other CTAs have published by then).
+constexpr unsigned long long kRendezvousNs = 100000ull;
+__device__ __forceinline__ void rendezvous_wait(const unsigned* counter, unsigned want) {
+  if (ld_acquire_u32(counter) >= want) return;
+  const unsigned long long t0 = global_ns();
+  while (ld_acquire_u32(counter) < want && global_ns() - t0 < kRendezvousNs) __nanosleep(100);
 }
 
 // ------------------------------------------------------------- per-query lists ---
@@ -189,33 +332,25 @@ struct TcShared {
   int q_cnt[kColsPerRound];     // ... per score column of the round
 };
 
-// Per-query candidate lists in shared memory.  Wide form: one packed 64-bit key per slot.
-// Compact form (6 bytes per slot: fp32 score + 16-bit position), chosen when it lets a call
-// run in fewer passes over the keys: a CTA's rows are numbered locally, its it-th macro tile
-// holding local rows [it*rows_per_tile, (it+1)*rows_per_tile), so 16 bits cover the 65,536
-// rows one CTA scans in pools of up to ~9.7 million rows.  An empty slot is key 0 / -inf.
+// Per-query candidate lists of one CTA: kk packed 64-bit keys per query, descending, empty
+// slots 0.  They live in shared memory while that leaves the operand ring deep enough; for
+// many queries and large k (256 x 64 slots are 128 KB) they live in global memory instead,
+// directly in the CTA's slice of the scan's output, where they stay in L2: a list is read
+// and written only by the warp that owns its query and, once the thresholds have settled,
+// only a few times per tile, while the shared memory it would take is worth two or three
+// ring stages of operands in flight (the key stream of one SM needs ~45 KB in flight to
+// run at its share of the HBM rate).
 struct ListStore {
-  u64* wide;
-  float* sc;
-  uint16_t* loc;
-  int kk, shift;          // rows per macro tile = 1 << shift
-  bool compact;
+  u64* slots;
+  int kk;
+  bool global;
 
   __device__ __forceinline__ u64 load(int q, int i) const {
-    if (!compact) return wide[(size_t)q * kk + i];
-    const float s = sc[(size_t)q * kk + i];
-    if (s == -INFINITY) return 0;
-    const uint32_t l = loc[(size_t)q * kk + i];
-    const uint32_t tile = blockIdx.x + (l >> shift) * gridDim.x;
-    return pack_candidate(s, (tile << shift) | (l & ((1u << shift) - 1u)));
+    return global ? __ldcg(slots + (size_t)q * kk + i) : slots[(size_t)q * kk + i];
   }
   __device__ __forceinline__ void store(int q, int i, u64 key) const {
-    if (!compact) { wide[(size_t)q * kk + i] = key; return; }
-    if (key == 0) { sc[(size_t)q * kk + i] = -INFINITY; loc[(size_t)q * kk + i] = 0; return; }
-    const uint32_t row = (uint32_t)candidate_row(key);
-    const uint32_t it = ((row >> shift) - blockIdx.x) / gridDim.x;
-    sc[(size_t)q * kk + i] = candidate_score(key);
-    loc[(size_t)q * kk + i] = (uint16_t)((it << shift) | (row & ((1u << shift) - 1u)));
+    if (global) __stcg(slots + (size_t)q * kk + i, key);
+    else slots[(size_t)q * kk + i] = key;
   }
 };
 
@@ -294,38 +429,85 @@ __device__ __forceinline__ void drain_round(const ListStore& lists, int kk, cons
   }
 }
 
+// The k-th largest of the CTAs' published best scores for query q (one per CTA), by k rounds
+// of warp-wide maximum extraction; -inf while fewer than k CTAs have published one.  Each is
+// the score of a distinct row, so k rows of the pool reach the value returned.
+__device__ __forceinline__ float kth_largest_best(const float* lmax, int q, int k, int lane) {
+  float mine[kTcMaxCtas / 32];
+#pragma unroll
+  for (int i = 0; i < kTcMaxCtas / 32; ++i) {
+    const int c = i * 32 + lane;
+    mine[i] = c < (int)gridDim.x ? __ldcg(&lmax[(size_t)q * kTcMaxCtas + c]) : -INFINITY;
+  }
+  float kth_best = -INFINITY;
+  for (int r = 0; r < k; ++r) {
+    float m = mine[0];
+#pragma unroll
+    for (int i = 1; i < kTcMaxCtas / 32; ++i) m = fmaxf(m, mine[i]);
+    float w = m;
+#pragma unroll
+    for (int o = 16; o; o >>= 1) w = fmaxf(w, __shfl_xor_sync(0xffffffffu, w, o));
+    kth_best = w;
+    if (w == -INFINITY) break;                                     // fewer than k bests yet
+    const int owner = __ffs(__ballot_sync(0xffffffffu, m == w)) - 1;
+    if (lane == owner) {                                           // remove one instance
+      bool done = false;
+#pragma unroll
+      for (int i = 0; i < kTcMaxCtas / 32; ++i)
+        if (!done && mine[i] == w) { mine[i] = -INFINITY; done = true; }
+    }
+  }
+  return kth_best;
+}
+
 // ------------------------------------------------------------------- the kernel ---
 // Queries [q0, q0+nq_c) of the call; n_pad = nq_c rounded up to 16 = MMA N.
 // mt (1 or 2) key tiles of 128 rows share each query tile: with mt = 2 the query bytes
 // pulled from L2 per key byte halve, which is what limits the kernel from nq ~ 64 up.
 // n_bufs accumulator sets of mt*n_pad TMEM columns each (2 = the next macro tile's MMAs
 // overlap the epilogue; 1 when 2*mt*n_pad would exceed the 512 columns).
+//
+// kPair: two CTAs (a cluster of two, on neighbouring SMs) work on one tile of 256 rows, for
+// batches of more than 128 queries.  There the accumulators of 128 rows x n_pad queries take
+// half of an SM's TMEM, so a lone CTA can share a query tile between no more than one key
+// tile at a time: 2 bytes of query per byte of key through the SM's L2 port, which is then
+// what bounds the kernel (~1,100 cycles per 16 KB of keys against ~720 at the HBM rate).  In
+// a pair each CTA loads its own 128 key rows and HALF of the query rows, and one
+// tcgen05.mma over both CTAs (M = 256) reads both halves: 1 byte of query per byte of key.
+// No load is shared or broadcast between the CTAs: each CTA's copies land in its own shared
+// memory.  The leading CTA (rank 0) issues the MMAs and owns the `full` and `tmem_empty`
+// barriers, on which both CTAs' copies and both CTAs' epilogue warps are counted; `empty`
+// and `tmem_full` exist in both CTAs and the leader's commits are counted on both.  mt is 1
+// in this form.
+template <bool kPair>
 __global__ void __launch_bounds__(kTcThreads, 1)
 scan_tc_kernel(const __grid_constant__ CUtensorMap key_map,
                const __grid_constant__ CUtensorMap q_map, PoolView pv, int q0, int nq_c,
                int nq_total, int n_pad, int k, int kk, int n_stages, int tmem_cols, int mt,
-               int n_bufs, int compact, const uint64_t* __restrict__ exclude_tag,
+               int n_bufs, int global_lists, const uint64_t* __restrict__ exclude_tag,
                u64* __restrict__ partial, DeviceStats* stats, float* xchg) {
   extern __shared__ __align__(1024) unsigned char smem_raw[];
   __shared__ TcShared sh;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t rank = kPair ? cluster_rank() : 0u;       // 0 = the CTA that issues the MMAs
+  const int n_ctas = kPair ? 2 : 1;
+  const int b_rows = n_pad / n_ctas;                       // query rows this CTA loads
   const int a_bytes = mt * kATileBytes;
-  const int stage_bytes = a_bytes + n_pad * kBlockK * 2;
+  const int stage_bytes = a_bytes + b_rows * kBlockK * 2;
   // dynamic shared memory: [stages][mt key tiles | query tile] | lists | queue | state
   unsigned char* base = (unsigned char*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
   unsigned char* ring = base;
   unsigned char* list_mem = ring + (size_t)n_stages * stage_bytes;              // [nq_c][kk]
   ListStore lists;
-  lists.wide = reinterpret_cast<u64*>(list_mem);
-  lists.sc = reinterpret_cast<float*>(list_mem);
-  lists.loc = reinterpret_cast<uint16_t*>(list_mem + (size_t)nq_c * kk * 4);
+  lists.global = global_lists != 0;
+  lists.slots = lists.global ? partial + ((size_t)blockIdx.x * nq_total + q0) * kk
+                             : reinterpret_cast<u64*>(list_mem);
   lists.kk = kk;
-  lists.shift = mt == 2 ? 8 : 7;
-  lists.compact = compact != 0;
-  u64* q_key = reinterpret_cast<u64*>(list_mem + (size_t)nq_c * kk * (compact ? 6 : 8));
+  u64* q_key = reinterpret_cast<u64*>(list_mem + (lists.global ? 0 : (size_t)nq_c * kk * 8));
                                                                // [kColsPerRound][kTileM]
   uint64_t* s_ex = reinterpret_cast<uint64_t*>(q_key + kQueueCap);              // [n_pad]
   float* thr_s = reinterpret_cast<float*>(s_ex + n_pad);                        // [n_pad]
+  uint32_t* s_qmax = reinterpret_cast<uint32_t*>(thr_s + n_pad);                // [n_pad]
   // Cross-CTA threshold exchange (global memory, reset to -inf by the query preparation):
   // lmax[q][cta] = best score CTA `cta` has seen for query q; gthr[q] = a score that at
   // least k distinct rows of the pool are known to reach, namely the k-th largest of the
@@ -336,33 +518,53 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap key_map,
   // orders of magnitude.  Values only grow, so stale reads are merely weaker bounds.
   float* lmax = xchg;
   float* gthr = xchg + (size_t)OILBIRD_MAX_NQ * kTcMaxCtas;
+  unsigned* arrivals = reinterpret_cast<unsigned*>(xchg + kTcXchgFloats);       // two counters
   const bool use_xchg = (int)gridDim.x >= k && (int)gridDim.x <= kTcMaxCtas;
 
-  const int n_tiles = (pv.n_rows + mt * kTileM - 1) / (mt * kTileM);   // macro tiles
+  // a macro tile: mt tiles of 128 rows of this CTA, or one of each CTA of the pair; the
+  // tiles of a grid are dealt out to its units (CTAs or pairs) round robin
+  const int rows_per_macro = (kPair ? 2 : mt) * kTileM;
+  const int n_tiles = (pv.n_rows + rows_per_macro - 1) / rows_per_macro;
+  const int unit = kPair ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;
+  const int n_units = kPair ? (int)(gridDim.x >> 1) : (int)gridDim.x;
   const int n_kb = (pv.d + kBlockK - 1) / kBlockK;
   volatile int* abort_flag = &sh.abort_flag;
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < n_stages; ++s) { mbar_init(&sh.full[s], 1); mbar_init(&sh.empty[s], 1); }
-    for (int b = 0; b < 2; ++b) { mbar_init(&sh.tmem_full[b], 1); mbar_init(&sh.tmem_empty[b], 4); }
+    for (int s = 0; s < n_stages; ++s) {
+      mbar_init(&sh.full[s], 1);
+      mbar_init(&sh.empty[s], 1);
+    }
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(&sh.tmem_full[b], 1);
+      mbar_init(&sh.tmem_empty[b], 4 * n_ctas);
+    }
     mbar_init(&sh.drain, 1);
     sh.abort_flag = 0;
     sh.q_total = 0;
     for (int j = 0; j < kColsPerRound; ++j) sh.q_cnt[j] = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  if (warp == 1) {   // TMEM allocation is a whole-warp operation
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
-                 ::"r"(smem_u32(&sh.tmem_base)), "r"((uint32_t)tmem_cols) : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  if (warp == 1) {   // TMEM allocation is a whole-warp operation (the same warp of both CTAs of a pair)
+    if (kPair) {
+      asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;"
+                   ::"r"(smem_u32(&sh.tmem_base)), "r"((uint32_t)tmem_cols) : "memory");
+      asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+    } else {
+      asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                   ::"r"(smem_u32(&sh.tmem_base)), "r"((uint32_t)tmem_cols) : "memory");
+      asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
   }
   tc_fence_before();
   __syncthreads();
+  if (kPair) cluster_sync_all();     // the other CTA's barriers exist before anything is counted on them
   tc_fence_after();
   const uint32_t tmem_base = sh.tmem_base;
   pdl_enter();   // appended rows, normalised queries, exclusion tags; set-up above overlapped
   for (int i = threadIdx.x; i < n_pad; i += kTcThreads) {
     thr_s[i] = i < nq_c ? -INFINITY : INFINITY;        // padded columns never pass the filter
+    s_qmax[i] = 0u;
     s_ex[i] = (exclude_tag && i < nq_c) ? exclude_tag[q0 + i] : 0;
   }
   for (int i = threadIdx.x; i < nq_c * kk; i += kTcThreads) lists.store(i / kk, i % kk, 0);
@@ -375,40 +577,62 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap key_map,
       asm volatile("prefetch.tensormap [%0];" ::"l"(&q_map) : "memory");
       uint32_t it = 0;
       bool ok = true;
-      for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
+      for (int tile = unit; tile < n_tiles && ok; tile += n_units) {
         for (int kb = 0; kb < n_kb; ++kb, ++it) {
           const int s = it % n_stages;
           const uint32_t ph = (it / n_stages) & 1u;
           if (!mbar_wait(&sh.empty[s], ph ^ 1u, abort_flag, stats)) { ok = false; break; }
           unsigned char* a_dst = ring + (size_t)s * stage_bytes;
-          mbar_arrive_expect_tx(&sh.full[s], (uint32_t)stage_bytes);
-          for (int sub = 0; sub < mt; ++sub)    // rows past the pool's capacity read as zero
-            tma_load_2d(a_dst + sub * kATileBytes, &key_map, kb * kBlockK,
-                        (tile * mt + sub) * kTileM, &sh.full[s]);
-          tma_load_2d(a_dst + a_bytes, &q_map, kb * kBlockK, q0, &sh.full[s]);
+          if (kPair) {
+            // Both CTAs' bytes are counted on the leader's barrier, and the leader's producer
+            // announces them all (the other CTA's bytes may land first: the count then
+            // dips below zero until the announcement, and the phase cannot complete before
+            // the leader's arrival).  Nothing but the copies' own completions crosses between
+            // the CTAs here: an arrival from the other CTA with release semantics was
+            // measured at ~600 cycles per stage for the thread that makes it.
+            const uint32_t full_at = smem_of_rank(&sh.full[s], 0);
+            if (rank == 0) mbar_arrive_expect_tx(&sh.full[s], 2u * (uint32_t)stage_bytes);
+            tma_load_2d_pair(a_dst, &key_map, kb * kBlockK, (tile * 2 + (int)rank) * kTileM, full_at);
+            tma_load_2d_pair(a_dst + a_bytes, &q_map, kb * kBlockK, q0 + (int)rank * b_rows, full_at);
+          } else {
+            mbar_arrive_expect_tx(&sh.full[s], (uint32_t)stage_bytes);
+            for (int sub = 0; sub < mt; ++sub)    // rows past the pool's capacity read as zero
+              tma_load_2d(a_dst + sub * kATileBytes, &key_map, kb * kBlockK,
+                          (tile * mt + sub) * kTileM, &sh.full[s]);
+            tma_load_2d(a_dst + a_bytes, &q_map, kb * kBlockK, q0, &sh.full[s]);
+          }
         }
       }
       if (!ok) {
         // gave up: let the copies already issued land before the CTA's memory goes away
         const uint32_t back = it < (uint32_t)n_stages ? it : (uint32_t)n_stages;
-        for (uint32_t j = 0; j < back; ++j) {
+        for (uint32_t j = 0; j < back && rank == 0; ++j) {   // (a pair's copies are counted in the leader)
           const uint32_t i2 = it - 1 - j;
           const unsigned long long t0 = global_ns();
           while (!mbar_try_wait(&sh.full[i2 % n_stages], (i2 / n_stages) & 1u) &&
                  global_ns() - t0 < 2000000ull) {}
         }
+        if (rank != 0) {                                     // let this CTA's own copies land
+          const unsigned long long t0 = global_ns();
+          while (global_ns() - t0 < 20000ull) {}
+        }
       }
     }
   } else if (warp == 1) {
     // ===================================================== MMA issuer ============
-    if (lane == 0) {
-      const uint32_t idesc = umma_idesc_bf16(n_pad);
+    // The whole warp walks the loop and one elected lane issues: everything the MMAs take
+    // (descriptors, accumulator address, barrier addresses) is then computed in uniform
+    // control flow, where the compiler can keep it in uniform registers, which is where
+    // tcgen05.mma takes its operands from.
+    if (rank == 0) {
+      const bool issuer = elect_one();
+      const uint32_t idesc = umma_idesc_bf16(n_pad, kPair ? 2 * kTileM : kTileM);
       uint32_t it = 0, iter = 0;
       bool ok = true;
-      for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x, ++iter) {
+      for (int tile = unit; tile < n_tiles && ok; tile += n_units, ++iter) {
         const uint32_t buf = iter % (uint32_t)n_bufs;
-        if (!mbar_wait(&sh.tmem_empty[buf], ((iter / (uint32_t)n_bufs) & 1u) ^ 1u, abort_flag,
-                       stats)) {
+        if (!warp_mbar_wait(&sh.tmem_empty[buf], ((iter / (uint32_t)n_bufs) & 1u) ^ 1u, abort_flag,
+                            stats)) {
           ok = false;
           break;
         }
@@ -416,26 +640,61 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap key_map,
         const uint32_t d_tmem = tmem_base + buf * (uint32_t)(mt * n_pad);
         for (int kb = 0; kb < n_kb; ++kb, ++it) {
           const int s = it % n_stages;
-          if (!mbar_wait(&sh.full[s], (it / n_stages) & 1u, abort_flag, stats)) { ok = false; break; }
+          if (!warp_mbar_wait(&sh.full[s], (it / n_stages) & 1u, abort_flag, stats)) { ok = false; break; }
           tc_fence_after();
           const uint32_t a_addr = smem_u32(ring + (size_t)s * stage_bytes);
+          const uint64_t a_desc = umma_desc_sw128(a_addr);
           const uint64_t b_desc = umma_desc_sw128(a_addr + a_bytes);
-          for (int sub = 0; sub < mt; ++sub) {
-            const uint64_t a_desc = umma_desc_sw128(a_addr + sub * kATileBytes);
+          const uint32_t acc = (uint32_t)(kb != 0);
+          if (kPair) {
+            const uint32_t empty0 = smem_of_rank(&sh.empty[s], 0), empty1 = smem_of_rank(&sh.empty[s], 1);
+            if (issuer) {
 #pragma unroll
-            for (int kq = 0; kq < kBlockK / 16; ++kq)      // 32 bytes along K per MMA
-              tc_mma_bf16(d_tmem + (uint32_t)(sub * n_pad), a_desc + (uint64_t)(kq * 2),
-                          b_desc + (uint64_t)(kq * 2), idesc, (kb | kq) != 0 ? 1u : 0u);
+              for (int kq = 0; kq < kBlockK / 16; ++kq)
+                tc_mma_bf16_pair(d_tmem, a_desc + (uint64_t)(kq * 2), b_desc + (uint64_t)(kq * 2),
+                                 idesc, kq != 0 ? 1u : acc);
+              // the stage is reusable in both CTAs once the MMAs retire
+              tc_commit_pair_at(empty0);
+              tc_commit_pair_at(empty1);
+            }
+          } else {
+            const uint64_t a_desc1 = a_desc + (uint64_t)(kATileBytes >> 4);     // second key tile
+            const uint32_t d_tmem1 = d_tmem + (uint32_t)n_pad;
+            if (issuer) {
+#pragma unroll
+              for (int kq = 0; kq < kBlockK / 16; ++kq)      // 32 bytes along K per MMA
+                tc_mma_bf16(d_tmem, a_desc + (uint64_t)(kq * 2), b_desc + (uint64_t)(kq * 2), idesc,
+                            kq != 0 ? 1u : acc);
+              if (mt == 2) {
+#pragma unroll
+                for (int kq = 0; kq < kBlockK / 16; ++kq)
+                  tc_mma_bf16(d_tmem1, a_desc1 + (uint64_t)(kq * 2), b_desc + (uint64_t)(kq * 2), idesc,
+                              kq != 0 ? 1u : acc);
+              }
+              tc_commit(&sh.empty[s]);                        // stage reusable once the MMAs retire
+            }
           }
-          tc_commit(&sh.empty[s]);                          // stage reusable once the MMAs retire
         }
-        if (ok) tc_commit(&sh.tmem_full[buf]);
+        __syncwarp();
+        if (ok && issuer) {
+          if (kPair) {
+            tc_commit_pair_at(smem_of_rank(&sh.tmem_full[buf], 0));
+            tc_commit_pair_at(smem_of_rank(&sh.tmem_full[buf], 1));
+          } else {
+            tc_commit(&sh.tmem_full[buf]);
+          }
+        }
       }
       // nothing may still be writing TMEM when it is freed
-      tc_commit(&sh.drain);
-      const unsigned long long t0 = global_ns();
-      const unsigned long long limit = wait_limit_ns(stats);
-      while (!mbar_try_wait(&sh.drain, 0) && global_ns() - t0 < limit) {}
+      __syncwarp();
+      if (issuer) {
+        if (kPair) tc_commit_pair_at(smem_of_rank(&sh.drain, 0));
+        else tc_commit(&sh.drain);
+        const unsigned long long t0 = global_ns();
+        const unsigned long long limit = wait_limit_ns(stats);
+        while (!mbar_try_wait(&sh.drain, 0) && global_ns() - t0 < limit) {}
+      }
+      __syncwarp();
     }
   } else {
     // ===================================================== epilogue ==============
@@ -444,12 +703,67 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap key_map,
     const int et = threadIdx.x - 64;            // 0..127
     uint32_t iter = 0;
     bool ok = true;
-    for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x, ++iter) {
+    for (int tile = unit; tile < n_tiles && ok; tile += n_units, ++iter) {
       const uint32_t buf = iter % (uint32_t)n_bufs;
       mbar_wait(&sh.tmem_full[buf], (iter / (uint32_t)n_bufs) & 1u, abort_flag, stats);
       // one decision for all four warps, so that the barriers below always match up
       epilogue_bar();
       if (et == 0) sh.epi_go = *abort_flag ? 0 : 1;
+      epilogue_bar();
+      if (!sh.epi_go) { ok = false; break; }
+      tc_fence_after();
+      if (OILBIRD_TC_FIRST_TILE_BOUND && use_xchg && iter == 0) {
+        // A CTA's first tile, before any threshold exists: every score would be a candidate
+        // (sorted 32*E at a time and merged, a couple of tiles' worth of time during which
+        // the accumulators stay full and the key stream stalls).  Instead the tile is read
+        // twice.  First only its best score per query is taken (one redux per column and
+        // warp) and published; the CTAs meet; the CTA responsible for a query takes the k-th
+        // largest of the CTAs' bests, which k distinct rows of the pool reach, as the bound;
+        // the CTAs meet again and adopt it.  The second reading of the tile is the regular
+        // filter, now against a bound that a few rows per query pass.  The two meetings are
+        // short waits that give up silently: a missing bound only means a weaker filter.
+        for (int sub = 0; sub < mt; ++sub) {
+          const int row = (kPair ? tile * 2 + (int)rank : tile * mt + sub) * kTileM + lane_grp * 32 + lane;
+          const bool row_ok = row < pv.n_rows;
+          uint64_t tag = 0;
+          if (exclude_tag && row_ok) tag = pv.trace_tag[pv.trace_id[row]];
+          const uint32_t t_row = tmem_base + ((uint32_t)(lane_grp * 32) << 16) +
+                                 (uint32_t)sub * (uint32_t)n_pad;               // buffer 0
+          for (int c0 = 0; c0 < n_pad; c0 += kColsPerRound) {
+            float v[kColsPerRound];
+            tc_ld16(t_row + (uint32_t)c0, v);
+            uint32_t mine = 0;
+#pragma unroll
+            for (int j = 0; j < kColsPerRound; ++j) {
+              const bool skip = !row_ok || (s_ex[c0 + j] != 0 && tag == s_ex[c0 + j]);
+              const uint32_t m = __reduce_max_sync(0xffffffffu, skip ? 0u : score_to_ord(v[j]));
+              mine = lane == j ? m : mine;
+            }
+            if (lane < kColsPerRound && mine != 0u) atomicMax(&s_qmax[c0 + lane], mine);
+          }
+        }
+        epilogue_bar();
+        for (int q = et; q < nq_c; q += 128)
+          if (s_qmax[q] != 0u)
+            __stcg(&lmax[(size_t)(q0 + q) * kTcMaxCtas + blockIdx.x], ord_to_score(s_qmax[q]));
+        __threadfence();
+        epilogue_bar();
+        if (et == 0) atomicAdd(&arrivals[0], 1u);
+        for (int q = ew; q < nq_c; q += 4) {
+          if ((q0 + q) % (int)gridDim.x != (int)blockIdx.x) continue;     // warp-uniform
+          rendezvous_wait(&arrivals[0], gridDim.x);
+          const float kth_best = kth_largest_best(lmax, q0 + q, k, lane);
+          if (lane == 0 && kth_best > -INFINITY && kth_best > __ldcg(&gthr[q0 + q]))
+            __stcg(&gthr[q0 + q], kth_best);
+        }
+        __threadfence();
+        epilogue_bar();
+        if (et == 0) {
+          atomicAdd(&arrivals[1], 1u);
+          rendezvous_wait(&arrivals[1], gridDim.x);
+        }
+        epilogue_bar();
+      }
       if (use_xchg) {
         // adopt the agreed bounds: v > max(local, prev(g))  <=>  v > local and v >= g
         for (int q = et; q < nq_c; q += 128) {
@@ -458,10 +772,8 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap key_map,
         }
       }
       epilogue_bar();
-      if (!sh.epi_go) { ok = false; break; }
-      tc_fence_after();
       for (int sub = 0; sub < mt; ++sub) {      // sub-tiles in row order: ties stay exact
-      const int row = (tile * mt + sub) * kTileM + lane_grp * 32 + lane;
+      const int row = (kPair ? tile * 2 + (int)rank : tile * mt + sub) * kTileM + lane_grp * 32 + lane;
       const bool row_ok = row < pv.n_rows;
       uint64_t tag = 0;
       if (exclude_tag && row_ok) tag = pv.trace_tag[pv.trace_id[row]];
@@ -474,7 +786,10 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap key_map,
           // all of this macro tile's scores have been read: hand the accumulators back
           tc_fence_before();
           __syncwarp();
-          if (lane == 0) mbar_arrive(&sh.tmem_empty[buf]);
+          if (lane == 0) {
+            if (kPair) mbar_arrive_at(smem_of_rank(&sh.tmem_empty[buf], 0));
+            else mbar_arrive(&sh.tmem_empty[buf]);
+          }
         }
         // The round's sixteen thresholds are fetched together and compared without a
         // branch; only the (rare) passing columns are visited.  Comparing column by column
@@ -532,48 +847,35 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap key_map,
         // largest of all CTAs' bests, by k rounds of warp-wide maximum extraction
         for (int q = ew; q < nq_c; q += 4) {
           if ((q0 + q) % (int)gridDim.x != (int)blockIdx.x) continue;     // warp-uniform
-          float mine[kTcMaxCtas / 32];
-#pragma unroll
-          for (int i = 0; i < kTcMaxCtas / 32; ++i) {
-            const int c = i * 32 + lane;
-            mine[i] = c < (int)gridDim.x ? __ldcg(&lmax[(size_t)(q0 + q) * kTcMaxCtas + c]) : -INFINITY;
-          }
-          float kth_best = -INFINITY;
-          for (int r = 0; r < k; ++r) {
-            float m = mine[0];
-#pragma unroll
-            for (int i = 1; i < kTcMaxCtas / 32; ++i) m = fmaxf(m, mine[i]);
-            float w = m;
-#pragma unroll
-            for (int o = 16; o; o >>= 1) w = fmaxf(w, __shfl_xor_sync(0xffffffffu, w, o));
-            kth_best = w;
-            if (w == -INFINITY) break;                                     // fewer than k bests yet
-            const int owner = __ffs(__ballot_sync(0xffffffffu, m == w)) - 1;
-            if (lane == owner) {                                           // remove one instance
-              bool done = false;
-#pragma unroll
-              for (int i = 0; i < kTcMaxCtas / 32; ++i)
-                if (!done && mine[i] == w) { mine[i] = -INFINITY; done = true; }
-            }
-          }
+          const float kth_best = kth_largest_best(lmax, q0 + q, k, lane);
           if (lane == 0 && kth_best > -INFINITY && kth_best > __ldcg(&gthr[q0 + q]))
             __stcg(&gthr[q0 + q], kth_best);
         }
       }
     }
-    // publish this CTA's per-query lists: already descending, empty slots are 0
+    // publish this CTA's per-query lists: already descending, empty slots are 0 (lists
+    // kept in global memory are in place already)
     epilogue_bar();
-    for (int i = et; i < nq_c * kk; i += 128) {
-      const int q = i / kk, j = i - q * kk;
-      partial[((size_t)blockIdx.x * nq_total + (q0 + q)) * kk + j] = lists.load(q, j);
+    if (!lists.global) {
+      for (int i = et; i < nq_c * kk; i += 128) {
+        const int q = i / kk, j = i - q * kk;
+        partial[((size_t)blockIdx.x * nq_total + (q0 + q)) * kk + j] = lists.load(q, j);
+      }
     }
   }
   tc_fence_before();
   __syncthreads();
+  // a pair: neither CTA goes away, nor is TMEM freed, while the other may still read this
+  // CTA's shared memory, count on its barriers or run MMAs into its TMEM
+  if (kPair) cluster_sync_all();
   if (warp == 1) {
     tc_fence_after();
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;"
-                 ::"r"(tmem_base), "r"((uint32_t)tmem_cols) : "memory");
+    if (kPair)
+      asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;"
+                   ::"r"(tmem_base), "r"((uint32_t)tmem_cols) : "memory");
+    else
+      asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;"
+                   ::"r"(tmem_base), "r"((uint32_t)tmem_cols) : "memory");
   }
 }
 
@@ -647,88 +949,157 @@ static const CUtensorMap* tc_q_map(TcCache* c, int n_pad) {
   return (slot >= 0 && slot < OILBIRD_MAX_NQ / 16 && c->q_ok[slot]) ? &c->q_map[slot] : nullptr;
 }
 
-static size_t tc_fixed_smem(int nq_c, int n_pad, int kk, bool compact) {
-  return (size_t)nq_c * kk * (compact ? 6 : 8) + (size_t)kQueueCap * 8 +
-         (size_t)n_pad * (8 + 4) + 1024 /* alignment slack */;
+static size_t tc_fixed_smem(int nq_c, int n_pad, int kk, bool global_lists) {
+  return (global_lists ? 0 : (size_t)nq_c * kk * 8) + (size_t)kQueueCap * 8 +
+         (size_t)n_pad * (8 + 4 + 4) + 1024 /* alignment slack */;
 }
 
-// How a call is cut up: queries per pass, list format, key tiles per query tile, ring
-// stages, accumulator buffers.  Fewest passes first (every pass re-reads the keys): the
-// compact list format is taken when it saves a pass (two ring stages are then enough: ring
-// depth was measured not to matter once the epilogue sets the pace); then two key tiles per
-// query tile if at least three ring stages still fit, else one.
-struct TcPlan { int per_pass, mt, stages, n_bufs, compact; };
+// How a call is cut up: queries per pass, where the lists live, key tiles per query tile,
+// ring stages, accumulator buffers.  With the lists in global memory any call (256 queries,
+// k = 128) fits one pass over the keys.
+struct TcPlan { int per_pass, n_pad, mt, stages, n_bufs, global_lists, pair; };
 
-static bool tc_fits(int n, int kk, int mt, bool compact, int min_stages, size_t smem_limit,
-                    int* stages) {
-  const size_t stage = (size_t)mt * kATileBytes + (size_t)n * kBlockK * 2;
+static bool tc_fits(int n, int kk, int mt, bool global_lists, int min_stages, size_t smem_limit,
+                    int* stages, bool pair = false) {
+  const size_t stage = (size_t)mt * kATileBytes + (size_t)(pair ? n / 2 : n) * kBlockK * 2;
   // static shared memory (barriers etc.) is padded to the 1024-byte alignment of the ring
-  const size_t fixed = tc_fixed_smem(n, n, kk, compact) + 1024 + 256;
+  const size_t fixed = tc_fixed_smem(n, n, kk, global_lists) + 1024 + 256;
   if (fixed + (size_t)min_stages * stage > smem_limit) return false;
   int st = (int)((smem_limit - fixed) / stage);
   *stages = st > kMaxStages ? kMaxStages : st;
   return true;
 }
 
-static TcPlan tc_plan(int nq, int k, int n_tiles128, int num_sms, size_t smem_limit, int force_mt) {
+static TcPlan tc_plan_single(int nq, int k, int n_tiles128, int num_sms, size_t smem_limit);
+
+static TcPlan tc_plan(int nq, int k, int n_tiles128, int num_sms, size_t smem_limit) {
+  // More than 128 queries on a large pool: two CTAs per tile of 256 rows (see the kernel);
+  // each loads half of the query rows, so their number is a multiple of 32
+  if (OILBIRD_TC_PAIR && nq > 128 && n_tiles128 >= 4 * num_sms && num_sms >= 2) {
+    TcPlan p;
+    p.per_pass = OILBIRD_MAX_NQ;
+    p.n_pad = (nq + 31) / 32 * 32;
+    p.pair = 1; p.mt = 1; p.global_lists = 1; p.n_bufs = 2; p.stages = 0;
+    if (tc_fits(p.n_pad, list_len(k), 1, true, 3, smem_limit, &p.stages, true)) return p;
+  }
+  return tc_plan_single(nq, k, n_tiles128, num_sms, smem_limit);
+}
+
+static TcPlan tc_plan_single(int nq, int k, int n_tiles128, int num_sms, size_t smem_limit) {
   const int kk = list_len(k);
-  int max_pass = 16, max_pass_c = 16, st = 0;
-  for (int n = 16; n <= OILBIRD_MAX_NQ; n += 16) {
-    if (tc_fits(n, kk, 1, false, 3, smem_limit, &st)) max_pass = n;
-    if (tc_fits(n, kk, 1, true, 2, smem_limit, &st)) max_pass_c = n;
-  }
-  int n_pass = (nq + max_pass - 1) / max_pass;
-  // 16-bit local positions: the rows one CTA scans must number at most 65,536
-  const int grid = n_tiles128 < num_sms ? (n_tiles128 > 0 ? n_tiles128 : 1) : num_sms;
-  const bool can_compact = ((int64_t)(n_tiles128 + grid - 1) / grid + 1) * kTileM <= 65536;
   TcPlan p;
-  p.compact = 0;
-  if (can_compact && (nq + max_pass_c - 1) / max_pass_c < n_pass) {
-    p.compact = 1;
-    n_pass = (nq + max_pass_c - 1) / max_pass_c;
-  }
-  const bool cp = p.compact != 0;
-  p.per_pass = ((nq + n_pass - 1) / n_pass + 15) / 16 * 16;      // balanced passes
-  const int n_pad = p.per_pass < nq ? p.per_pass : (nq + 15) / 16 * 16;
-  // sharing a query tile between two key tiles pays at every nq measured (fewer, larger
-  // stages and half the query bytes from L2), given enough tiles to keep every SM busy
-  bool two = n_tiles128 >= 4 * num_sms && tc_fits(n_pad, kk, 2, cp, 3, smem_limit, &st);
-  if (force_mt == 1) two = false;
-  if (force_mt == 2) two = tc_fits(n_pad, kk, 2, cp, 2, smem_limit, &st);
-  p.mt = two ? 2 : 1;
-  tc_fits(n_pad, kk, p.mt, cp, 2, smem_limit, &p.stages);
+  p.per_pass = OILBIRD_MAX_NQ;
+  const int n_pad = (nq + 15) / 16 * 16;
+  int st = 0;
+  p.pair = 0;
+  p.n_pad = n_pad;
+  // Sharing a query tile between two key tiles pays at every nq measured (fewer, larger
+  // stages and half the query bytes from L2), given enough tiles to keep every SM busy and
+  // room for both tiles' accumulators twice (a second accumulator set lets the next tile's
+  // MMAs overlap this tile's epilogue).  Then the lists: in shared memory while the ring
+  // beside them keeps its depth, else in global memory; a deep ring of two-tile stages with
+  // the lists in L2 beats a shallower or one-tile ring with the lists on chip (nq = 128,
+  // k = 64 at d = 8192: 2.61 ms against 3.11).
+  const bool many_tiles = n_tiles128 >= 2 * num_sms;
+  bool two = many_tiles && 2 * 2 * n_pad <= 512 && tc_fits(n_pad, kk, 2, true, 3, smem_limit, &st);
+  if (OILBIRD_TC_FORCE_MT == 1) two = false;
+  if (OILBIRD_TC_FORCE_MT == 2) two = 2 * n_pad <= 512 && tc_fits(n_pad, kk, 2, true, 2, smem_limit, &st);
+  const int mt = two ? 2 : 1;
+  bool gl = !tc_fits(n_pad, kk, mt, false, OILBIRD_TC_MIN_SMEM_STAGES, smem_limit, &st);
+  if (OILBIRD_TC_FORCE_LISTS == 1) gl = !tc_fits(n_pad, kk, mt, false, 2, smem_limit, &st);
+  if (OILBIRD_TC_FORCE_LISTS == 2) gl = true;
+  p.global_lists = gl ? 1 : 0;
+  p.mt = mt;
+  p.stages = 0;
+  tc_fits(n_pad, kk, p.mt, gl, 2, smem_limit, &p.stages);
   p.n_bufs = 2 * p.mt * n_pad <= 512 ? 2 : 1;
   return p;
 }
 
 int tc_queries_per_pass(int nq, int k, int n_rows, int num_sms, size_t smem_limit) {
-  return tc_plan(nq, k, (n_rows + kTileM - 1) / kTileM, num_sms, smem_limit, 0).per_pass;
+  return tc_plan(nq, k, (n_rows + kTileM - 1) / kTileM, num_sms, smem_limit).per_pass;
+}
+
+// CTA pairs that can be resident at once for a given amount of dynamic shared memory
+// (cached: the answer only depends on the device and the size).
+static int max_pairs(size_t smem, int num_sms) {
+  static size_t known_smem = 0;
+  static int known = 0;
+  if (known_smem == smem && known > 0) return known;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(num_sms / 2 * 2);
+  cfg.blockDim = dim3(kTcThreads);
+  cfg.dynamicSmemBytes = smem;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  int n = 0;
+  if (cudaOccupancyMaxActiveClusters(&n, scan_tc_kernel<true>, &cfg) != cudaSuccess) {
+    cudaGetLastError();
+    return 0;
+  }
+  known_smem = smem;
+  known = n;
+  return n;
 }
 
 cudaError_t launch_scan_tc(TcCache* cache, const PoolView& pv, int32_t q0, int32_t nq_c,
                            int32_t nq_total, int32_t k, int32_t kk, const uint64_t* exclude_tag,
                            unsigned long long* partial, DeviceStats* stats, float* xchg,
                            int32_t num_sms, size_t smem_limit, int32_t* n_lists, cudaStream_t st) {
-  const int n_pad = (nq_c + 15) / 16 * 16;
   const int n_tiles128 = (pv.n_rows + kTileM - 1) / kTileM;
-  TcPlan plan = tc_plan(nq_c, k, n_tiles128, num_sms, smem_limit, 0);
-  const size_t stage = (size_t)plan.mt * kATileBytes + (size_t)n_pad * kBlockK * 2;
-  const size_t fixed = tc_fixed_smem(nq_c, n_pad, kk, plan.compact != 0);
-  if (plan.stages < 2) return cudaErrorInvalidConfiguration;
-  const CUtensorMap* q_map = tc_q_map(cache, n_pad);
-  if (!q_map) return cudaErrorInvalidValue;
-  size_t smem = fixed + (size_t)plan.stages * stage;
-  if (smem < 120 * 1024) smem = 120 * 1024;   // one CTA per SM: TMEM is allocated per CTA
-  int tmem_cols = 32;
-  while (tmem_cols < plan.n_bufs * plan.mt * n_pad) tmem_cols <<= 1;
-  const int n_tiles = (n_tiles128 + plan.mt - 1) / plan.mt;
-  int grid = n_tiles < num_sms ? n_tiles : num_sms;
-  if (grid < 1) grid = 1;
-  *n_lists = grid;
-  return launch_pdl(scan_tc_kernel, dim3(grid), dim3(kTcThreads), smem, st,
-                    cache->key_map, *q_map, pv, q0, nq_c, nq_total, n_pad, k, kk, plan.stages,
-                    tmem_cols, plan.mt, plan.n_bufs, plan.compact, exclude_tag, partial, stats,
-                    xchg);
+  TcPlan plan = tc_plan(nq_c, k, n_tiles128, num_sms, smem_limit);
+  for (int attempt = 0; attempt < 2; ++attempt) {
+    const int n_pad = plan.n_pad;
+    const size_t stage = (size_t)plan.mt * kATileBytes +
+                         (size_t)(plan.pair ? n_pad / 2 : n_pad) * kBlockK * 2;
+    const size_t fixed = tc_fixed_smem(nq_c, n_pad, kk, plan.global_lists != 0);
+    if (plan.stages < 2) return cudaErrorInvalidConfiguration;
+    const CUtensorMap* q_map = tc_q_map(cache, plan.pair ? n_pad / 2 : n_pad);
+    if (!q_map) return cudaErrorInvalidValue;
+    size_t smem = fixed + (size_t)plan.stages * stage;
+    if (smem < 120 * 1024) smem = 120 * 1024;   // one CTA per SM: TMEM is allocated per CTA
+    int tmem_cols = 32;
+    while (tmem_cols < plan.n_bufs * plan.mt * n_pad) tmem_cols <<= 1;
+    if (plan.pair) {
+      const int pairs_fit = max_pairs(smem, num_sms);
+      if (pairs_fit < num_sms / 2 - 2) {        // the device will not seat (nearly) every SM in a pair
+        plan = tc_plan_single(nq_c, k, n_tiles128, num_sms, smem_limit);
+        continue;
+      }
+      const int n_tiles = (n_tiles128 + 1) / 2;
+      int pairs = n_tiles < pairs_fit ? n_tiles : pairs_fit;
+      if (pairs > num_sms / 2) pairs = num_sms / 2;
+      *n_lists = 2 * pairs;
+      cudaLaunchConfig_t cfg = {};
+      cfg.gridDim = dim3(2 * pairs);
+      cfg.blockDim = dim3(kTcThreads);
+      cfg.dynamicSmemBytes = smem;
+      cfg.stream = st;
+      cudaLaunchAttribute attr[2];
+      attr[0].id = cudaLaunchAttributeClusterDimension;
+      attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+      attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+      attr[1].val.programmaticStreamSerializationAllowed = 1;
+      cfg.attrs = attr;
+      cfg.numAttrs = (!tl_pdl_off && pdl_process_ok()) ? 2 : 1;
+      return cudaLaunchKernelEx(&cfg, scan_tc_kernel<true>, cache->key_map, *q_map, pv, (int)q0,
+                                (int)nq_c, (int)nq_total, n_pad, (int)k, (int)kk, plan.stages,
+                                tmem_cols, plan.mt, plan.n_bufs, plan.global_lists, exclude_tag,
+                                (u64*)partial, stats, xchg);
+    }
+    const int n_tiles = (n_tiles128 + plan.mt - 1) / plan.mt;
+    int grid = n_tiles < num_sms ? n_tiles : num_sms;
+    if (grid < 1) grid = 1;
+    *n_lists = grid;
+    return launch_pdl(scan_tc_kernel<false>, dim3(grid), dim3(kTcThreads), smem, st,
+                      cache->key_map, *q_map, pv, q0, nq_c, nq_total, n_pad, k, kk, plan.stages,
+                      tmem_cols, plan.mt, plan.n_bufs, plan.global_lists, exclude_tag, partial, stats,
+                      xchg);
+  }
+  return cudaErrorInvalidConfiguration;
 }
 
 // Both kinds of bounded wait on things that never happen (see launch_stall_selftest).
@@ -759,7 +1130,8 @@ cudaError_t launch_stall_selftest(const unsigned long long* ready, DeviceStats* 
 }
 
 cudaError_t preload_scan_tc_kernels() {
-  cudaError_t e = preload_kernel(scan_tc_kernel, true);
+  cudaError_t e = preload_kernel(scan_tc_kernel<false>, true);
+  if (e == cudaSuccess) e = preload_kernel(scan_tc_kernel<true>, true);
   return e != cudaSuccess ? e : preload_kernel(stall_selftest_kernel);
 }
 

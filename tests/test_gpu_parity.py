@@ -485,9 +485,9 @@ def test_step_host_is_append_host_plus_query_host():
 
 
 @pytest.mark.parametrize("nq,k", [(256, 128), (100, 128), (256, 64), (33, 100)])
-def test_largest_nq_and_k_run_in_several_passes(nq, k):
-    """Per-query lists for nq*k beyond shared memory: the tensor path cuts the call into
-    balanced query passes; results must not depend on the cut."""
+def test_largest_nq_and_k(nq, k):
+    """Per-query lists for nq*k beyond shared memory: the tensor path keeps them in global
+    memory (its slice of the scan's output) and still scans the keys once."""
     w = W.C1.scaled(nq=nq, k=k, n_rows=2500, d=256, cont_len=3)
     pool, ora = fill_both(w, max_k=128, max_nq=256)
     q, _ = w.queries("cuda")
@@ -501,6 +501,34 @@ def test_largest_nq_and_k_run_in_several_passes(nq, k):
     if k <= 100:
         gem = pool.query(q[:2].contiguous(), fixed(k, 3, theta=-2.0, path=B.PATH_GEMV))
         check_query(gem, ora, W.to_bits(q)[:2], pr)
+
+
+@pytest.mark.parametrize("nq,k", [(129, 8), (160, 64), (200, 16), (256, 64), (256, 128), (131, 1)])
+def test_pairs_of_ctas_on_batches_above_128_queries(nq, k):
+    """More than 128 queries on a pool of at least four tiles per SM: two CTAs share each
+    tile of 256 rows (one MMA over both, each loading half of the query rows).  Ragged last
+    tile whose second half is empty or partly filled, query counts that are no multiple of
+    32, rows beyond the pool's size inside the last tile."""
+    for n_rows in (148 * 128 * 4 + 77, 148 * 128 * 4 + 128 + 5):
+        w = W.C1.scaled(nq=nq, k=k, n_rows=n_rows, d=192, cont_len=3, n_centroids=2048,
+                        rows_per_trace=1024, seed=40 + k)
+        pool, ora = fill_both(w, max_k=128, max_nq=256)
+        q, meta = w.queries("cuda")
+        pr = fixed(k, 3, theta=-2.0, path=B.PATH_TENSOR)
+        out = pool.query(q, pr)
+        check_query(out, ora, W.to_bits(q), pr)
+        assert int(out.idx[0, 0]) == meta["planted_row"]
+        assert pool.stats()["stalled"] == 0
+    ws = w.separated()
+    pool, ora = fill_both(ws, max_k=128, max_nq=256)
+    q, _ = ws.queries("cuda")
+    check_query(pool.query(q, pr), ora, W.to_bits(q), pr)
+    # exclusion tags: every query skips the trace that holds its best neighbour
+    best = pool.query(q, pr).cpu().idx[:, 0].numpy()
+    ex = np.array([ws.trace_tag(int(b) // ws.rows_per_trace) for b in best], dtype=np.int64)
+    pr_ex = fixed(k, 3, theta=-2.0, path=B.PATH_TENSOR, exclude_tag=torch.from_numpy(ex).cuda())
+    check_query(pool.query(q, pr_ex), ora, W.to_bits(q), pr_ex, exclude=ex.astype(np.uint64))
+    assert pool.stats()["stalled"] == 0
 
 
 @pytest.mark.parametrize("d", [8, 72, 200, 1000])
@@ -527,6 +555,18 @@ def test_exact_ties_spread_over_all_ctas_keep_the_lowest_rows():
     ora.append(bits, tk, tag=1)
     qb = np.stack([np.where(base > 0, P1, M1).astype(np.uint16)] * 3)
     qb[1, :2] = np.where(base[:2] > 0, M1, P1)              # a second, slightly different query
+    # the same three queries 50 times over: the two-CTA form of the tensor scan (> 128 queries)
+    qmany = np.concatenate([qb] * 50)
+    pool.close()
+    pool = B.Pool(d, n, max_k=128, max_nq=256)
+    pool.append(bits_to_dev(bits), torch.from_numpy(tk).cuda(), tag=1)
+    for k in (8, 128):
+        pr = fixed(k, 2, theta=-2.0, path=B.PATH_TENSOR)
+        out = pool.query(bits_to_dev(qmany), pr).cpu()
+        ref = ora.query(qb, __import__("parity").oracle_params(pr))
+        for r in range(50):
+            assert out.idx.numpy()[3 * r:3 * r + 3].tolist() == ref.idx.tolist(), (k, r)
+            assert np.array_equal(out.score.numpy()[3 * r:3 * r + 3], ref.score)
     for k in (1, 8, 64, 128):
         for path in (B.PATH_TENSOR, B.PATH_GEMV):
             pr = fixed(k, 2, theta=-2.0, path=path)

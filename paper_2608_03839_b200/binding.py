@@ -340,10 +340,11 @@ class Pool:
     def __del__(self):
         try:
             self.close()
-        except OilbirdError:
-            import traceback
-            traceback.print_exc()
-            GUARD_FAILURES.append(self)
+        except Exception as e:           # (module globals may be gone at interpreter exit)
+            if type(e).__name__ == "OilbirdError":
+                import traceback
+                traceback.print_exc()
+                GUARD_FAILURES.append(self)
 
     def check_guards(self, stream=None) -> None:
         """Raises OilbirdError(EGUARD) if a kernel wrote behind one of the pool's arrays."""

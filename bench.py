@@ -62,8 +62,9 @@ def measured_peaks():
 # profiles/ (file named per entry), with the pool rows held at capture time.  Traffic is
 # proportional to the rows scanned, so it is scaled to the rows of the timed launches.
 NCU_TRAFFIC = {
-    "C2": (540625920.0, 65560),      # profiles/scan_gemv_C2_ncu.md
-    "C4": (2172068528.0, 264192),    # profiles/scan_tc_C4_quarter_ncu.md (quarter-size pool)
+    "C2": (540625920.0, 65560),        # profiles/scan_gemv_C2_ncu.md
+    "C4": (2162393280.0, 262784),      # profiles/scan_tc_C4_quarter_ncu.md (quarter-size pool)
+    "C5nq256": (2657778952.0, 152832), # profiles/scan_tc_C5_nq256_eighth_ncu.md (151,552-row pool)
 }
 
 
@@ -560,10 +561,10 @@ def run_legs(args, dev, local, K, Wm):
     pool = make_pool(w, 256, rows_step, cap, local, args, (1 << 20) // rows_step + 8)
     fill_pool(pool, w, W.C5_START_ROWS, dev)
     for nq in (1, 256):
-        leg(pool, w, nq, len(pool))
+        leg(pool, w, nq, len(pool), key="C5nq256" if nq == 256 else None)
     fill_pool(pool, w, far, dev)                # the stream's appends in between, in bulk
     for nq in (1, 256):
-        leg(pool, w, nq, len(pool))
+        leg(pool, w, nq, len(pool), key="C5nq256" if nq == 256 else None)
     pool.close()
     return legs
 
@@ -819,6 +820,17 @@ def run_evict(args):
             pool.append(st, tk, tag=6_000_000 + i)
     torch.cuda.synchronize()
     ev_ms = float(np.mean([ev[2 * i].elapsed_time(ev[2 * i + 1]) for i in range(K)]))
+    # a small evicted prefix (one trace in front of all the others): the fixed-size,
+    # register-staged waves of the compaction, whose barrier count does not depend on it
+    ev1 = [torch.cuda.Event(enable_timing=True) for _ in range(2 * K)]
+    for i in range(K):
+        ev1[2 * i].record()
+        pool.evict_oldest(1)
+        ev1[2 * i + 1].record()
+        pool.append(fresh[0][0], fresh[0][1], tag=7_000_000 + i)
+    torch.cuda.synchronize()
+    ev1_ms = float(np.mean([ev1[2 * i].elapsed_time(ev1[2 * i + 1]) for i in range(K)]))
+    moved1 = 2.0 * (n_tr - 1) * rpt * (row_bytes + 8)
     live = (n_tr - drop) * rpt
     moved = 2.0 * live * (row_bytes + 8)            # keys (+scale), token, trace id: read + write
     peaks, peak_kind = measured_peaks()
@@ -830,6 +842,8 @@ def run_evict(args):
                                    f"{args.keys}; per step the oldest {drop} traces are dropped, "
                                    f"{drop} appended, 1 query"},
             "evict_ms": ev_ms, "clocks": clocks, "gpu_launches": int(launches),
+            "evict_one_trace": {"ms": ev1_ms, "gbs": moved1 / (ev1_ms * 1e-3) / 1e9,
+                                "note": f"1 trace of {rpt} rows dropped in front of {n_tr - 1}"},
             "roofline": {"bound": "hbm", "kernel": "compact_kernel (live rows moved to the front)",
                          "achieved": moved / (ev_ms * 1e-3) / 1e9, "peak": peaks["hbm_gbs"],
                          "unit": "GB/s", "frac": moved / (ev_ms * 1e-3) / 1e9 / peaks["hbm_gbs"],

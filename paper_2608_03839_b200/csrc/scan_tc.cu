@@ -61,7 +61,11 @@
 //     of the other CTA with release semantics costs the arriving thread ~600 cycles, and
 //     either form ran at 1,600 cycles per k-block;
 //   - a single 128 x 256 x 16 MMA issued as two interleaved 128 x 128 x 16 ones (independent
-//     accumulators): 8 instructions in ~950 cycles instead of 4 in ~750;
+//     accumulators): 8 instructions in ~950 cycles instead of 4 in ~750; the same two halves
+//     issued by two warps at once: 857 cycles per k-block against 856 with one issuer, so
+//     what bounds the loop is the operands' way through shared memory, not the issue;
+//   - a suspend-time hint (2 or 20 us) on the mbarrier waits, to spin less under the power
+//     cap: no change in sustained runs;
 //   - asking for the keys of the next 8 or 24 k-blocks into L2 ahead of the ring
 //     (cp.async.bulk.prefetch.tensor): 1.4x and 2x slower at every nq.
 //

@@ -468,10 +468,10 @@ def run_ours(args):
             "warmup": Wm, "ms_per_step": res["ms_per_step"], "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": f"{args.keys} keys, fp32 accumulate",
             "data": "synthetic",
-            "config": {"workload": res["workload"] +
-                       (" (the single-request decode configuration, the one the 70 %-of-HBM "
-                        "target is stated on; the batched and the largest configurations are "
-                        "in `legs`)" if default_run else ""),
+            "config": {"workload": res["workload"],
+                       "note": ("the single-request decode configuration, the one the 70 %-of-HBM "
+                                "target is stated on; the batched and the largest configurations "
+                                "are in `legs`") if default_run else "one configuration alone",
                        "pool_rows_start": res["pool_rows_start"], "pool_rows_end": res["pool_rows_end"],
                        "append_rows_per_step": rows_step, "scan_path": args.path,
                        "l2": "inputs exceed L2" if w.key_bytes(n0) > 2 * 126e6 else

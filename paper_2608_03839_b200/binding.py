@@ -11,12 +11,12 @@ import ctypes
 import os
 from dataclasses import dataclass, field
 
-# The library chains the kernels of a step with programmatic launches; with CUDA's lazy
-# module loading the first steps of a process dead-locked now and then on the largest
-# configuration (a kernel loading at its first launch while others of the chain were resident
-# and waiting; with eager loading: never in the runs made).  The library loads its own
-# kernels before it launches any, and the process is asked to load all modules eagerly too,
-# which takes effect if CUDA has not been initialised yet (importing torch does not do that).
+# The library chains the kernels of a step with programmatic launches only when the process
+# loads CUDA modules eagerly (under lazy loading, the CUDA default, it launches plainly: the
+# combination of lazy loading and chained launches was seen to dead-lock the first steps of a
+# process now and then).  Asking for eager loading here buys those ~6 us per step on small
+# pools; it takes effect if CUDA has not been initialised yet (importing torch does not do
+# that), and the library is safe either way.
 os.environ.setdefault("CUDA_MODULE_LOADING", "EAGER")
 
 import numpy as np  # noqa: E402

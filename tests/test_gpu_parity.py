@@ -519,6 +519,13 @@ def test_pairs_of_ctas_on_batches_above_128_queries(nq, k):
         check_query(out, ora, W.to_bits(q), pr)
         assert int(out.idx[0, 0]) == meta["planted_row"]
         assert pool.stats()["stalled"] == 0
+        # which candidates reach the lists depends on when the CTAs' bounds arrive; the
+        # answer must not: three more runs, bit for bit
+        a = out.cpu()
+        for _ in range(3):
+            b = pool.query(q, pr).cpu()
+            assert torch.equal(a.idx, b.idx) and torch.equal(a.score, b.score)
+            assert torch.equal(a.cont_tok, b.cont_tok) and torch.equal(a.cont_len, b.cont_len)
     ws = w.separated()
     pool, ora = fill_both(ws, max_k=128, max_nq=256)
     q, _ = ws.queries("cuda")

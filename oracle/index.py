@@ -1,0 +1,107 @@
+"""CPU oracle for the coarse index over the pool (test infrastructure).
+
+The paper's Limitations section names "an index" as one of three ways to keep the cost of
+the cosine lookup bounded as the store grows, and defines none.  The one built here is an
+inverted file over centroids the caller supplies; what it computes, in the order the steps
+are taken:
+
+  assign   every stored row belongs to the list of the centroid that is the best neighbour
+           of the row's STORED key taken as a query state (the lookup of Algorithm 1 with
+           k = 1 against the centroids: cosine of the normalised vectors, ties to the lowest
+           centroid);
+  probe    a query's lists are the n_probe best centroids for the query state (the same
+           lookup with k = n_probe);
+  scan     the candidates are the rows of the probed lists plus every row appended since
+           the index was last refreshed (the tail, which is always scanned); among them the
+           answer is exactly Eq. 2 and Eq. 3: top-k by (score descending, row ascending),
+           theta on the best, depth, continuation clipped at the trace end.
+
+So the result is the brute-force result restricted to the candidate rows: with every list
+probed it IS the brute-force result, which is the first pin.  Everything is built from
+OraclePool (full scores in double, full sort); plain numpy and Python loops on purpose.
+"""
+from __future__ import annotations
+
+import numpy as np
+
+from . import DEPTH_FIXED, OraclePool, QueryParams, QueryResult, depth as oracle_depth
+
+
+class OracleIndex:
+    def __init__(self, pool: OraclePool, centroids_bits: np.ndarray):
+        """centroids_bits: raw bf16 states [n_lists, d] (uint16 bit patterns)."""
+        c = np.ascontiguousarray(centroids_bits, dtype=np.uint16).reshape(-1, pool.d)
+        self.pool = pool
+        self.n_lists = c.shape[0]
+        self.cent = OraclePool(pool.d)
+        self.cent.append(c, np.arange(self.n_lists, dtype=np.int32), tag=0)
+        self.assign = np.empty(0, dtype=np.int64)      # list of every indexed row
+
+    @property
+    def n_indexed(self) -> int:
+        return int(self.assign.shape[0])
+
+    def reset(self) -> None:
+        self.assign = np.empty(0, dtype=np.int64)
+
+    def refresh(self) -> None:
+        """Assign the rows appended since the last refresh."""
+        n = len(self.pool)
+        if n <= self.n_indexed:
+            return
+        keys = self.pool.keys[self.n_indexed:n]        # stored (normalised) keys, as queries
+        one = QueryParams(k=1, theta=-np.inf, depth_mode=DEPTH_FIXED, cont_len=1)
+        new = np.empty(keys.shape[0], dtype=np.int64)
+        step = 4096
+        for r0 in range(0, keys.shape[0], step):
+            new[r0:r0 + step] = self.cent.query(keys[r0:r0 + step], one).idx[:, 0]
+        self.assign = np.concatenate([self.assign, new])
+
+    def lists(self) -> list[np.ndarray]:
+        return [np.nonzero(self.assign == l)[0] for l in range(self.n_lists)]
+
+    def probes(self, q_bits: np.ndarray, n_probe: int) -> np.ndarray:
+        """[nq, n_probe] centroid ids, best first, -1 where fewer than n_probe exist."""
+        pr = QueryParams(k=n_probe, theta=-np.inf, depth_mode=DEPTH_FIXED, cont_len=1)
+        return self.cent.query(q_bits, pr).idx
+
+    def candidates(self, probes_q: np.ndarray) -> np.ndarray:
+        """Row mask [N]: rows of the probed lists, and the tail."""
+        n = len(self.pool)
+        mask = np.zeros(n, dtype=bool)
+        good = probes_q[probes_q >= 0]
+        mask[: self.n_indexed] = np.isin(self.assign, good)
+        mask[self.n_indexed:] = True
+        return mask
+
+    def query(self, q_bits: np.ndarray, n_probe: int, params: QueryParams | None = None,
+              want_all_scores: bool = False) -> QueryResult:
+        pr = params or QueryParams()
+        q = np.ascontiguousarray(q_bits, dtype=np.uint16).reshape(-1, self.pool.d)
+        nq, k, L = q.shape[0], int(pr.k), int(pr.cont_len)
+        full = self.pool.query(q, pr, want_all_scores=True)    # scores of EVERY row (exclusion applied)
+        probes = self.probes(q, n_probe)
+        idx = np.full((nq, k), -1, dtype=np.int64)
+        score = np.full((nq, k), -np.inf, dtype=np.float32)
+        fired = np.zeros(nq, dtype=np.int32)
+        clen = np.zeros((nq, k), dtype=np.int32)
+        ctok = np.full((nq, k, L), -1, dtype=np.int32)
+        alls = np.full((nq, len(self.pool)), -np.inf, dtype=np.float32)
+        for i in range(nq):
+            s = full.all_scores[i].copy()
+            s[~self.candidates(probes[i])] = -np.inf           # only candidates can be neighbours
+            alls[i] = s
+            rows = np.nonzero(np.isfinite(s))[0]
+            order = rows[np.lexsort((rows, -s[rows].astype(np.float64)))]   # score desc, row asc
+            top = order[:k]
+            idx[i, : len(top)] = top
+            score[i, : len(top)] = s[top]
+            fired[i] = int(len(top) > 0 and np.float32(s[top[0]]) >= np.float32(pr.theta))
+            for j, r in enumerate(top):
+                dep = 0
+                if fired[i]:
+                    dep = L if pr.depth_mode == DEPTH_FIXED else oracle_depth(
+                        float(s[r]), pr.tier_thr, pr.tier_depth)
+                tok, n = self.pool.gather_one(int(r), dep, pr.offset, L)
+                ctok[i, j], clen[i, j] = tok, n
+        return QueryResult(idx, score, fired, clen, ctok, alls if want_all_scores else None)

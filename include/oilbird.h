@@ -460,6 +460,48 @@ int oilbird_merge_chains(int32_t nq, const int32_t* sem_tok, const int32_t* sem_
                          int32_t device, void* cuda_stream);
 
 /*
+ * Coarse index (the paper's Limitations section names "an index" next to eviction and
+ * quantisation as a way to keep the lookup's cost from growing with the store, and defines
+ * none; this is the library's reading): an inverted file over n_lists centroids the caller
+ * supplies (raw states, dev [n_lists,d] bf16, normalised like keys; e.g. a sample of stored
+ * states).  The pool is left as it is; the index adds, per row, the number of a list.
+ *   - A row belongs to the list of the centroid that is the best neighbour of its STORED key
+ *     taken as a query state (this library's lookup with k = 1 against the centroids; ties to
+ *     the lowest centroid).
+ *   - refresh() assigns every row appended since the last refresh and rebuilds the lists.
+ *     Rows appended since then (the tail) have no list yet and are always scanned.
+ *   - query() takes each query's n_probe best centroids (the same lookup, k = n_probe, at most
+ *     OILBIRD_MAX_K), scores the rows of those lists and the tail exactly as
+ *     oilbird_pool_query scores them, and returns the k best of them by (score descending,
+ *     row ascending) with the firing rule, depths and continuations of Eq. 2 and Eq. 3.
+ * The answer is oilbird_pool_query's answer restricted to the candidate rows: identical when
+ * every list is probed, otherwise approximate (rows of lists that were not probed cannot be
+ * found).  16-bit pools only.  create() copies the centroids (enqueued on cuda_stream); the
+ * caller's array is free again once that work has completed.  After oilbird_pool_reset or
+ * oilbird_pool_evict_oldest the row numbers the index holds are stale: call
+ * oilbird_index_reset (all rows become tail) and refresh again; refresh and query refuse with
+ * EINVAL while the pool holds fewer rows than the index covers.  Index calls enqueue on
+ * cuda_stream and use the pool's scratch, so they follow the pool's one-stream, one-thread
+ * rule.  Destroy the index before its pool.
+ */
+typedef struct oilbird_index oilbird_index_t;   /* opaque */
+int oilbird_index_create (oilbird_index_t** out, oilbird_pool_t* pool, const void* centroids_bf16,
+                          int32_t n_lists /* 1..65536 */, void* cuda_stream);
+int oilbird_index_refresh(oilbird_index_t* index, void* cuda_stream);
+int oilbird_index_reset  (oilbird_index_t* index, void* cuda_stream);
+int oilbird_index_query  (oilbird_index_t* index, const void* q_bf16 /* dev [nq,d] */, int32_t nq,
+                          int32_t n_probe, const oilbird_query_params* params,
+                          const oilbird_query_out* out, void* cuda_stream);
+int oilbird_index_destroy(oilbird_index_t* index);
+int64_t oilbird_index_rows(const oilbird_index_t* index);        /* rows that have a list   */
+/* Copy the index to host memory (synchronous; tests): assign [rows] (list of each row),
+ * list_off [n_lists+1], list_rows [rows] (the rows of list l are list_rows[list_off[l] ..
+ * list_off[l+1]), in no particular order).  Any pointer may be NULL. */
+int oilbird_index_read(oilbird_index_t* index, int32_t* assign_host, int32_t* list_off_host,
+                       int32_t* list_rows_host);
+const char* oilbird_index_last_error(void);
+
+/*
  * Query without any allocation (the paper has no counterpart; this serves hosts of the
  * library that own all device memory themselves and must not let a library allocate:
  * for instance a serving engine that reserved the whole of HBM at start-up, where a

@@ -137,6 +137,15 @@ SYMBOLS = {
     "oilbird_merge_chains": (ctypes.c_int, [_i32, _vp, _vp, _i32, _i32, _vp, _vp, _i32, _i32, _vp,
                                             _vp, _vp, _vp, _vp, _vp, _vp, _vp,
                                             ctypes.POINTER(MergeParams), _i32, _vp]),
+    "oilbird_index_create": (ctypes.c_int, [ctypes.POINTER(_vp), _vp, _vp, _i32, _vp]),
+    "oilbird_index_refresh": (ctypes.c_int, [_vp, _vp]),
+    "oilbird_index_reset": (ctypes.c_int, [_vp, _vp]),
+    "oilbird_index_query": (ctypes.c_int, [_vp, _vp, _i32, _i32, ctypes.POINTER(CQueryParams),
+                                           ctypes.POINTER(CQueryOut), _vp]),
+    "oilbird_index_destroy": (ctypes.c_int, [_vp]),
+    "oilbird_index_rows": (_i64, [_vp]),
+    "oilbird_index_read": (ctypes.c_int, [_vp, _vp, _vp, _vp]),
+    "oilbird_index_last_error": (ctypes.c_char_p, []),
     "oilbird_query_static": (ctypes.c_int, [ctypes.POINTER(StaticPool), _vp, _i32,
                                             ctypes.POINTER(CQueryParams),
                                             ctypes.POINTER(CQueryOut), _vp]),
@@ -567,6 +576,69 @@ class Pool:
         buf = np.empty(max_n, dtype=np.float32)
         n = self._L.oilbird_pool_profile_read(self._h, buf.ctypes.data, max_n)
         return buf[:n].copy()
+
+
+# ------------------------------------------------------------------ coarse index ----
+class Index:
+    """Inverted-file index over a Pool (oilbird_index_* of the C-ABI): centroids the caller
+    supplies, rows assigned by the library's own k = 1 lookup, queries answered from the
+    n_probe best lists plus the rows appended since the last refresh."""
+
+    def __init__(self, pool: Pool, centroids: torch.Tensor, stream=None):
+        assert centroids.is_cuda and centroids.dtype == torch.bfloat16 and centroids.is_contiguous()
+        assert centroids.dim() == 2 and centroids.shape[1] == pool.d
+        self._L, self.pool, self.n_lists = lib(), pool, int(centroids.shape[0])
+        h = ctypes.c_void_p()
+        _check(self._L.oilbird_index_create(ctypes.byref(h), pool._h, centroids.data_ptr(),
+                                            self.n_lists, _stream_ptr(stream)), "oilbird_index_create")
+        self._h = h
+
+    def close(self) -> None:
+        h, self._h = getattr(self, "_h", None), None
+        if h:
+            self._L.oilbird_index_destroy(h)
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def __len__(self) -> int:
+        return int(self._L.oilbird_index_rows(self._h))
+
+    def refresh(self, stream=None) -> None:
+        _check(self._L.oilbird_index_refresh(self._h, _stream_ptr(stream)), "oilbird_index_refresh")
+
+    def reset(self, stream=None) -> None:
+        _check(self._L.oilbird_index_reset(self._h, _stream_ptr(stream)), "oilbird_index_reset")
+
+    def query(self, q: torch.Tensor, n_probe: int, params: QueryParams | None = None,
+              out: QueryOut | None = None, stream=None) -> QueryOut:
+        pr = params or QueryParams()
+        assert q.is_cuda and q.dtype == torch.bfloat16 and q.is_contiguous()
+        q = q.reshape(-1, self.pool.d)
+        nq = q.shape[0]
+        ex_ptr = None
+        if pr.exclude_tag is not None:
+            ex = pr.exclude_tag
+            assert ex.is_cuda and ex.dtype in (torch.int64, torch.uint64) and ex.numel() == nq
+            ex_ptr = ex.data_ptr()
+        if out is None:
+            out = QueryOut.empty(nq, pr.k, pr.cont_len, self.pool._dev)
+        cp = pr.to_c(ex_ptr)
+        _check(self._L.oilbird_index_query(self._h, q.data_ptr(), nq, int(n_probe), ctypes.byref(cp),
+                                           ctypes.byref(out._c), _stream_ptr(stream)),
+               "oilbird_index_query")
+        return out
+
+    def read(self):
+        """(assign int32 [rows], list_off int32 [n_lists+1], list_rows int32 [rows])."""
+        n = len(self)
+        a, o, r = np.empty(n, np.int32), np.empty(self.n_lists + 1, np.int32), np.empty(n, np.int32)
+        _check(self._L.oilbird_index_read(self._h, a.ctypes.data, o.ctypes.data, r.ctypes.data),
+               "oilbird_index_read")
+        return a, o, r
 
 
 # ------------------------------------------------------------------ recycled pool ----

@@ -90,6 +90,43 @@ __device__ __forceinline__ void wait_fused_rows(const FusedAppend& fa, DeviceSta
   wait_fused_rows(fa.ready, fa.target, stats);
 }
 
+// ------------------------------------------------- scoring rows (CUDA cores) ---
+constexpr int kRowsPerIter = 4;   // rows a warp scores together (shares each query load)
+// Dot products of kRowsPerIter rows with the QT queries in shared memory; kFresh selects
+// the coherent load for rows written during this launch.
+template <int QT, bool kFresh>
+__device__ __forceinline__ void score_rows(const uint4* const (&rowp)[kRowsPerIter], const uint4* qs,
+                                           int n_chunks, int lane,
+                                           float (&acc)[kRowsPerIter][QT]) {
+#pragma unroll 2
+  for (int c = lane; c < n_chunks; c += 32) {
+    uint4 kv[kRowsPerIter];
+#pragma unroll
+    for (int r = 0; r < kRowsPerIter; ++r)
+      kv[r] = kFresh ? ld_cg16(rowp[r] + c) : ld_stream16(rowp[r] + c);
+#pragma unroll
+    for (int q = 0; q < QT; ++q) {
+      const uint4 qv = qs[q * n_chunks + c];
+      const float q0f = bf16_lo(qv.x), q1f = bf16_hi(qv.x), q2f = bf16_lo(qv.y),
+                  q3f = bf16_hi(qv.y), q4f = bf16_lo(qv.z), q5f = bf16_hi(qv.z),
+                  q6f = bf16_lo(qv.w), q7f = bf16_hi(qv.w);
+#pragma unroll
+      for (int r = 0; r < kRowsPerIter; ++r) {
+        float a = acc[r][q];
+        a = fmaf(bf16_lo(kv[r].x), q0f, a);
+        a = fmaf(bf16_hi(kv[r].x), q1f, a);
+        a = fmaf(bf16_lo(kv[r].y), q2f, a);
+        a = fmaf(bf16_hi(kv[r].y), q3f, a);
+        a = fmaf(bf16_lo(kv[r].z), q4f, a);
+        a = fmaf(bf16_hi(kv[r].z), q5f, a);
+        a = fmaf(bf16_lo(kv[r].w), q6f, a);
+        a = fmaf(bf16_hi(kv[r].w), q7f, a);
+        acc[r][q] = a;
+      }
+    }
+  }
+}
+
 // ---------------------------------------------------- programmatic launch ------
 // The kernels of a step may be launched with programmatic stream serialization (see
 // launch_pdl in internal.h): a kernel's blocks can then be scheduled, and run their set-up,

@@ -1,0 +1,408 @@
+// Coarse index over a pool: an inverted file over centroids the caller supplies.
+//
+// The paper's Limitations section names "an index" next to eviction and quantisation as a way
+// to keep the cost of the cosine lookup from growing with the store, and defines none.  The
+// one here leaves the pool as it is (rows stay where they were appended, so positions, traces
+// and continuations are untouched) and adds, per row, the number of a list:
+//   assign   a row belongs to the list of the centroid that is the best neighbour of the row's
+//            STORED key taken as a query (the library's own lookup with k = 1 against a small
+//            pool that holds the centroids; ties to the lowest centroid);
+//   probe    a query's lists are its n_probe best centroids (the same lookup, k = n_probe);
+//   scan     the rows of those lists, found through row numbers kept list by list, plus every
+//            row appended since the last refresh (the tail) are scored exactly as the full
+//            scan scores them, and the k best by (score, lowest row) go through the same merge,
+//            firing rule, depth and gather (Eq. 2, Eq. 3).
+// The answer is the full scan's answer restricted to the candidate rows: exact with every
+// list probed, approximate otherwise (recall is measured by the benchmark).  A key row is
+// 2d contiguous bytes, so fetching rows by number costs HBM nothing in efficiency; a lookup
+// moves n_lists*d*2 bytes of centroids plus the candidates' keys instead of the whole pool.
+#include <math.h>
+#include <stdio.h>
+
+#include <new>
+
+#include "common.cuh"
+#include "internal.h"
+#include "normalize.cuh"
+#include "pool_priv.h"
+
+namespace oilbird {
+
+constexpr int kIndexMaxLists = 65536;
+constexpr int kIndexMaxProbe = OILBIRD_MAX_K;        // the probes are a k-lookup on the centroids
+constexpr int kIndexAssignBatch = 256;               // rows assigned per lookup
+
+// ------------------------------------------------------------------ list building ---
+__global__ void __launch_bounds__(256)
+index_count_kernel(const int32_t* __restrict__ assign, int n, int32_t* __restrict__ counts,
+                   int n_lists) {
+  pdl_enter();
+  for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < n; i += gridDim.x * blockDim.x) {
+    const int l = assign[i];
+    if (l >= 0 && l < n_lists) atomicAdd(&counts[l], 1);
+  }
+}
+
+// list_off[l] = rows in lists below l (one block); cursor starts at zero.
+__global__ void __launch_bounds__(1024)
+index_offsets_kernel(const int32_t* __restrict__ counts, int32_t* __restrict__ list_off,
+                     int32_t* __restrict__ cursor, int n_lists) {
+  __shared__ int s_sum[1024];
+  pdl_enter();
+  const int per = (n_lists + 1023) / 1024;
+  const int lo = threadIdx.x * per, hi = min(n_lists, lo + per);
+  int sum = 0;
+  for (int l = lo; l < hi; ++l) sum += counts[l];
+  s_sum[threadIdx.x] = sum;
+  __syncthreads();
+  for (int o = 1; o < 1024; o <<= 1) {                  // inclusive scan of the threads' sums
+    const int v = threadIdx.x >= o ? s_sum[threadIdx.x - o] : 0;
+    __syncthreads();
+    s_sum[threadIdx.x] += v;
+    __syncthreads();
+  }
+  int run = s_sum[threadIdx.x] - sum;
+  for (int l = lo; l < hi; ++l) {
+    list_off[l] = run;
+    cursor[l] = 0;
+    run += counts[l];
+  }
+  if (threadIdx.x == 1023) list_off[n_lists] = s_sum[1023];
+}
+
+__global__ void __launch_bounds__(256)
+index_scatter_kernel(const int32_t* __restrict__ assign, int n, const int32_t* __restrict__ list_off,
+                     int32_t* __restrict__ cursor, int32_t* __restrict__ list_rows, int n_lists) {
+  pdl_enter();
+  for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < n; i += gridDim.x * blockDim.x) {
+    const int l = assign[i];
+    if (l >= 0 && l < n_lists) list_rows[list_off[l] + atomicAdd(&cursor[l], 1)] = i;
+  }
+}
+
+// ------------------------------------------------------------- scan of the candidates ---
+// Grid (G, nq): CTA (b, q) scores a contiguous share of query q's candidates (the rows of its
+// probed lists in probe order, then the tail) and leaves one descending list of KK packed
+// candidates in partial[b][q], as the full scans do.  Rows are fetched by number; everything
+// else (query preparation, scoring, per-warp lists, block merge) is the CUDA-core scan's.
+template <int E>
+__global__ void __launch_bounds__(kNormThreads, 2)
+scan_ids_kernel(PoolView pv, const uint16_t* __restrict__ q_raw, int nq, int k,
+                const int32_t* __restrict__ probes, int n_probe,
+                const int32_t* __restrict__ list_off, const int32_t* __restrict__ list_rows,
+                int n_indexed, const uint64_t* __restrict__ exclude_tag, u64* __restrict__ partial,
+                int32_t* __restrict__ q_valid, DeviceStats* stats) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  constexpr int KK = 32 * E;
+  constexpr int kWarps = kNormThreads / 32;
+  __shared__ int s_pref[kIndexMaxProbe + 1], s_base[kIndexMaxProbe];
+  pdl_enter();
+  const int d = pv.d, n_chunks = d >> 3;
+  uint4* qs = reinterpret_cast<uint4*>(smem_raw);                        // [n_chunks]
+  u64* scratch = reinterpret_cast<u64*>(smem_raw + (size_t)d * 2);        // [warps][KK]
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int q = blockIdx.y;
+
+  const int code = normalize_row<true, 2>(q_raw + (size_t)q * d, reinterpret_cast<uint16_t*>(qs), d);
+  if (blockIdx.x == 0 && threadIdx.x == 0) {
+    q_valid[q] = code == kRowNonFinite ? 0 : 1;          // NaN/Inf: no neighbours
+    if (code == kRowNonFinite) atomicAdd(&stats->nonfinite_queries, 1ull);
+  }
+  // the probed lists of this query, laid end to end
+  if (threadIdx.x < n_probe) {
+    const int l = probes[(size_t)q * n_probe + threadIdx.x];
+    s_base[threadIdx.x] = l >= 0 ? list_off[l] : 0;
+    s_pref[threadIdx.x + 1] = l >= 0 ? list_off[l + 1] - list_off[l] : 0;
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    s_pref[0] = 0;
+    for (int p = 0; p < n_probe; ++p) s_pref[p + 1] += s_pref[p];
+  }
+  __syncthreads();
+  const int in_lists = s_pref[n_probe];
+  const int total = in_lists + (pv.n_rows - n_indexed);
+  const uint64_t ex = exclude_tag ? exclude_tag[q] : 0;
+  const int c_lo = (int)(((long long)total * blockIdx.x) / gridDim.x);
+  const int c_hi = (int)(((long long)total * (blockIdx.x + 1)) / gridDim.x);
+  const uint4* keys4 = reinterpret_cast<const uint4*>(pv.keys);
+
+  auto row_of = [&](int c) -> int {
+    if (c >= in_lists) return n_indexed + (c - in_lists);          // the tail
+    int lo = 0, hi = n_probe;                                      // last p with s_pref[p] <= c
+    while (hi - lo > 1) {
+      const int mid = (lo + hi) >> 1;
+      if (s_pref[mid] <= c) lo = mid; else hi = mid;
+    }
+    return list_rows[s_base[lo] + (c - s_pref[lo])];
+  };
+
+  u64 top[1][E];
+  u64 kth = 0;
+#pragma unroll
+  for (int r = 0; r < E; ++r) top[0][r] = 0;
+  for (int cb = c_lo + warp * kRowsPerIter; cb < c_hi; cb += kWarps * kRowsPerIter) {
+    int rows[kRowsPerIter];
+    const uint4* rowp[kRowsPerIter];
+#pragma unroll
+    for (int r = 0; r < kRowsPerIter; ++r) {
+      rows[r] = row_of(cb + r < c_hi ? cb + r : c_hi - 1);          // clamp: result discarded below
+      rowp[r] = keys4 + (size_t)rows[r] * n_chunks;
+    }
+    float acc[kRowsPerIter][1];
+#pragma unroll
+    for (int r = 0; r < kRowsPerIter; ++r) acc[r][0] = 0.f;
+    score_rows<1, false>(rowp, qs, n_chunks, lane, acc);
+#pragma unroll
+    for (int r = 0; r < kRowsPerIter; ++r) {
+      if (cb + r >= c_hi) break;                                    // warp-uniform
+      const float s = warp_sum(acc[r][0]);
+      if (ex != 0 && pv.trace_tag[pv.trace_id[rows[r]]] == ex) continue;   // same-prompt trace
+      const u64 key = pack_candidate(s, (uint32_t)rows[r]);
+      if (key > kth) {
+        warp_sorted_insert<E>(top[0], key, lane);
+        kth = warp_list_get<E>(top[0], k - 1);
+      }
+    }
+  }
+  block_merge_desc<E>(top[0], scratch, kWarps);
+  if (threadIdx.x < 32) {
+    u64* dst = partial + ((size_t)blockIdx.x * nq + q) * KK;
+#pragma unroll
+    for (int r = 0; r < E; ++r) dst[r * 32 + lane] = top[0][r];
+  }
+}
+
+template <int E>
+static cudaError_t launch_scan_ids(const PoolView& pv, const uint16_t* q, int nq, int k,
+                                   const int32_t* probes, int n_probe, const int32_t* list_off,
+                                   const int32_t* list_rows, int n_indexed, const uint64_t* ex,
+                                   u64* partial, int32_t* q_valid, DeviceStats* stats, int grid,
+                                   cudaStream_t st) {
+  const size_t smem = (size_t)pv.d * 2 + (size_t)(kNormThreads / 32) * 32 * E * sizeof(u64);
+  return launch_pdl(scan_ids_kernel<E>, dim3(grid, nq), dim3(kNormThreads), smem, st, pv, q, nq, k,
+                    probes, n_probe, list_off, list_rows, n_indexed, ex, partial, q_valid, stats);
+}
+
+cudaError_t preload_index_kernels() {
+  cudaError_t e;
+  if ((e = preload_kernel(index_count_kernel)) != cudaSuccess) return e;
+  if ((e = preload_kernel(index_offsets_kernel)) != cudaSuccess) return e;
+  if ((e = preload_kernel(index_scatter_kernel)) != cudaSuccess) return e;
+  if ((e = preload_kernel(scan_ids_kernel<1>, true)) != cudaSuccess) return e;
+  if ((e = preload_kernel(scan_ids_kernel<2>, true)) != cudaSuccess) return e;
+  return preload_kernel(scan_ids_kernel<4>, true);
+}
+
+}  // namespace oilbird
+
+using namespace oilbird;
+
+struct oilbird_index {
+  oilbird_pool* pool;
+  oilbird_pool* cent;            // the centroids, as a pool of n_lists rows
+  int32_t n_lists;
+  int64_t n_indexed;             // rows that have a list (enqueue-time truth)
+  unsigned char* mem;
+  int32_t *assign, *list_rows, *list_off, *cursor, *counts;
+  // results of the lookups on the centroids
+  int32_t* probe_idx; float* probe_score; int32_t *probe_fired, *probe_len, *probe_tok;
+  float* a_score; int32_t *a_fired, *a_len, *a_tok;
+};
+
+static thread_local char g_index_err[256] = "";
+static int index_fail(cudaError_t e, const char* what) {
+  snprintf(g_index_err, sizeof g_index_err, "%s: %s", what, cudaGetErrorString(e));
+  return e == cudaErrorMemoryAllocation ? OILBIRD_ENOMEM : OILBIRD_ECUDA;
+}
+#define ICU(call)                                         \
+  do {                                                    \
+    cudaError_t e_ = (call);                              \
+    if (e_ != cudaSuccess) return index_fail(e_, #call);  \
+  } while (0)
+
+extern "C" {
+
+const char* oilbird_index_last_error(void) { return g_index_err; }
+
+int oilbird_index_create(oilbird_index_t** out, oilbird_pool_t* pool, const void* centroids_bf16,
+                         int32_t n_lists, void* cuda_stream) {
+  if (!out) return OILBIRD_EINVAL;
+  *out = nullptr;
+  if (!pool || !centroids_bf16 || n_lists < 1 || n_lists > kIndexMaxLists) return OILBIRD_EINVAL;
+  if (pool->r.e4m3) return OILBIRD_EINVAL;                       // rows are fetched as bf16 keys
+  if ((uintptr_t)centroids_bf16 & 15) return OILBIRD_EINVAL;
+  ICU(cudaSetDevice(pool->device));
+  oilbird_index* ix = new (std::nothrow) oilbird_index();
+  if (!ix) return OILBIRD_ENOMEM;
+  ix->pool = pool; ix->n_lists = n_lists; ix->n_indexed = 0; ix->cent = nullptr; ix->mem = nullptr;
+  oilbird_pool_config cc = {};
+  cc.d = pool->r.d; cc.capacity_rows = n_lists; cc.max_traces = 1; cc.max_nq = OILBIRD_MAX_NQ;
+  cc.max_k = OILBIRD_MAX_K; cc.max_append = 1; cc.device = pool->device;
+  cc.flags = pool->r.guards ? OILBIRD_DEBUG_GUARDS : 0;
+  int rc = oilbird_pool_create(&ix->cent, &cc);
+  if (rc) { delete ix; return rc; }
+  const size_t cap = (size_t)pool->r.capacity, nl = (size_t)n_lists;
+  const size_t rows_i32 = cap > nl ? cap : nl;
+  auto up = [](size_t v) { return (v + 255) / 256 * 256; };
+  const size_t o_assign = 0, o_rows = o_assign + up(rows_i32 * 4), o_off = o_rows + up(rows_i32 * 4),
+               o_cur = o_off + up((nl + 1) * 4), o_cnt = o_cur + up(nl * 4),
+               o_pidx = o_cnt + up(nl * 4),
+               o_psc = o_pidx + up((size_t)OILBIRD_MAX_NQ * kIndexMaxProbe * 4),
+               o_pf = o_psc + up((size_t)OILBIRD_MAX_NQ * kIndexMaxProbe * 4),
+               o_pl = o_pf + up((size_t)OILBIRD_MAX_NQ * 4),
+               o_pt = o_pl + up((size_t)OILBIRD_MAX_NQ * kIndexMaxProbe * 4),
+               o_as = o_pt + up((size_t)OILBIRD_MAX_NQ * kIndexMaxProbe * 4),
+               o_af = o_as + up(kIndexAssignBatch * 4), o_al = o_af + up(kIndexAssignBatch * 4),
+               o_at = o_al + up(kIndexAssignBatch * 4), total = o_at + up(kIndexAssignBatch * 4);
+  cudaError_t e = cudaMalloc((void**)&ix->mem, total);
+  if (e != cudaSuccess) { oilbird_pool_destroy(ix->cent); delete ix; return index_fail(e, "cudaMalloc(index)"); }
+  ix->assign = (int32_t*)(ix->mem + o_assign); ix->list_rows = (int32_t*)(ix->mem + o_rows);
+  ix->list_off = (int32_t*)(ix->mem + o_off); ix->cursor = (int32_t*)(ix->mem + o_cur);
+  ix->counts = (int32_t*)(ix->mem + o_cnt);
+  ix->probe_idx = (int32_t*)(ix->mem + o_pidx); ix->probe_score = (float*)(ix->mem + o_psc);
+  ix->probe_fired = (int32_t*)(ix->mem + o_pf); ix->probe_len = (int32_t*)(ix->mem + o_pl);
+  ix->probe_tok = (int32_t*)(ix->mem + o_pt);
+  ix->a_score = (float*)(ix->mem + o_as); ix->a_fired = (int32_t*)(ix->mem + o_af);
+  ix->a_len = (int32_t*)(ix->mem + o_al); ix->a_tok = (int32_t*)(ix->mem + o_at);
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  // the centroids become the rows of a one-trace pool (their tokens are never looked at);
+  // all lists start empty
+  e = cudaMemsetAsync(ix->mem, 0, o_pidx, st);
+  if (e == cudaSuccess)
+    rc = oilbird_pool_append(ix->cent, centroids_bf16, ix->list_rows, n_lists, 0, OILBIRD_NEW_TRACE, st);
+  if (e != cudaSuccess || rc) {
+    cudaFree(ix->mem); oilbird_pool_destroy(ix->cent); delete ix;
+    return e != cudaSuccess ? index_fail(e, "cudaMemsetAsync(index)") : rc;
+  }
+  *out = ix;
+  return OILBIRD_OK;
+}
+
+int oilbird_index_destroy(oilbird_index_t* ix) {
+  if (!ix) return OILBIRD_EINVAL;
+  cudaSetDevice(ix->pool->device);
+  cudaDeviceSynchronize();
+  oilbird_pool_destroy(ix->cent);
+  cudaFree(ix->mem);
+  delete ix;
+  return OILBIRD_OK;
+}
+
+int64_t oilbird_index_rows(const oilbird_index_t* ix) { return ix ? ix->n_indexed : 0; }
+
+int oilbird_index_reset(oilbird_index_t* ix, void* cuda_stream) {
+  if (!ix) return OILBIRD_EINVAL;
+  ICU(cudaSetDevice(ix->pool->device));
+  // every list empty again: offsets all zero
+  ICU(cudaMemsetAsync(ix->list_off, 0, ((size_t)ix->n_lists + 1) * 4, (cudaStream_t)cuda_stream));
+  ix->n_indexed = 0;
+  return OILBIRD_OK;
+}
+
+int oilbird_index_refresh(oilbird_index_t* ix, void* cuda_stream) {
+  if (!ix) return OILBIRD_EINVAL;
+  oilbird_pool* p = ix->pool;
+  ICU(cudaSetDevice(p->device));
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  const int64_t n = p->n_rows;
+  if (n < ix->n_indexed) return OILBIRD_EINVAL;          // the pool was reset or evicted from: reset the index
+  if (n == ix->n_indexed) return OILBIRD_OK;
+  // assign the new rows: their stored keys, a batch at a time, as queries against the centroids
+  oilbird_query_params pr;
+  oilbird_query_params_default(&pr);
+  pr.k = 1; pr.theta = -INFINITY; pr.depth_mode = OILBIRD_DEPTH_FIXED; pr.cont_len = 1;
+  for (int64_t r0 = ix->n_indexed; r0 < n; r0 += kIndexAssignBatch) {
+    const int32_t nq = (int32_t)(n - r0 < kIndexAssignBatch ? n - r0 : kIndexAssignBatch);
+    oilbird_query_out o;
+    o.idx = ix->assign + r0; o.score = ix->a_score; o.fired = ix->a_fired;
+    o.cont_len = ix->a_len; o.cont_tok = ix->a_tok;
+    int rc = oilbird_pool_query(ix->cent, p->keys + (size_t)r0 * p->r.d, nq, &pr, &o, st);
+    if (rc) return rc;
+  }
+  // rebuild the lists over all indexed rows: count, offsets, scatter
+  const int n_all = (int)n;
+  int grid = (n_all + 255) / 256;
+  if (grid > 4 * p->num_sms) grid = 4 * p->num_sms;
+  ICU(cudaMemsetAsync(ix->counts, 0, (size_t)ix->n_lists * 4, st));
+  cudaError_t e = launch_pdl(index_count_kernel, dim3(grid), dim3(256), 0, st,
+                             (const int32_t*)ix->assign, n_all, ix->counts, ix->n_lists);
+  if (e == cudaSuccess)
+    e = launch_pdl(index_offsets_kernel, dim3(1), dim3(1024), 0, st, (const int32_t*)ix->counts,
+                   ix->list_off, ix->cursor, ix->n_lists);
+  if (e == cudaSuccess)
+    e = launch_pdl(index_scatter_kernel, dim3(grid), dim3(256), 0, st, (const int32_t*)ix->assign,
+                   n_all, (const int32_t*)ix->list_off, ix->cursor, ix->list_rows, ix->n_lists);
+  if (e != cudaSuccess) return index_fail(e, "index list kernels");
+  p->launches += 3;
+  ix->n_indexed = n;
+  return OILBIRD_OK;
+}
+
+int oilbird_index_query(oilbird_index_t* ix, const void* q_bf16, int32_t nq, int32_t n_probe,
+                        const oilbird_query_params* pr, const oilbird_query_out* out,
+                        void* cuda_stream) {
+  if (!ix || !q_bf16 || !pr || !out || !out->idx || !out->score || !out->fired || !out->cont_len ||
+      !out->cont_tok)
+    return OILBIRD_EINVAL;
+  oilbird_pool* p = ix->pool;
+  GatherParams gp;
+  int rc = check_query_params(nq, p->r.max_nq, p->r.max_k, pr, &gp);
+  if (rc) return rc;
+  if (n_probe < 1) return OILBIRD_EINVAL;
+  if (n_probe > kIndexMaxProbe) n_probe = kIndexMaxProbe;
+  if (((uintptr_t)q_bf16 & 15) || ((uintptr_t)pr->exclude_tag & 7) ||
+      (((uintptr_t)out->idx | (uintptr_t)out->score | (uintptr_t)out->fired |
+        (uintptr_t)out->cont_len | (uintptr_t)out->cont_tok) & 3)) {
+    snprintf(g_index_err, sizeof g_index_err, "misaligned pointer");
+    return OILBIRD_EINVAL;
+  }
+  if (p->n_rows < ix->n_indexed) return OILBIRD_EINVAL;   // pool reset or evicted from: reset the index
+  ICU(cudaSetDevice(p->device));
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  // probe: the n_probe best centroids of every query
+  oilbird_query_params pp;
+  oilbird_query_params_default(&pp);
+  pp.k = n_probe; pp.theta = -INFINITY; pp.depth_mode = OILBIRD_DEPTH_FIXED; pp.cont_len = 1;
+  oilbird_query_out po;
+  po.idx = ix->probe_idx; po.score = ix->probe_score; po.fired = ix->probe_fired;
+  po.cont_len = ix->probe_len; po.cont_tok = ix->probe_tok;
+  rc = oilbird_pool_query(ix->cent, q_bf16, nq, &pp, &po, st);
+  if (rc) return rc;
+  // scan the candidates, merge, fire, gather
+  const int kk = list_len(pr->k);
+  int grid = 2 * p->num_sms;
+  if (grid > p->r.max_lists) grid = p->r.max_lists;
+  PoolView pv = pool_view(p);
+  cudaError_t e;
+  const uint16_t* q = (const uint16_t*)q_bf16;
+  if (kk == 32)
+    e = launch_scan_ids<1>(pv, q, nq, pr->k, ix->probe_idx, n_probe, ix->list_off, ix->list_rows,
+                           (int)ix->n_indexed, pr->exclude_tag, p->partial, p->q_valid, p->stats, grid, st);
+  else if (kk == 64)
+    e = launch_scan_ids<2>(pv, q, nq, pr->k, ix->probe_idx, n_probe, ix->list_off, ix->list_rows,
+                           (int)ix->n_indexed, pr->exclude_tag, p->partial, p->q_valid, p->stats, grid, st);
+  else
+    e = launch_scan_ids<4>(pv, q, nq, pr->k, ix->probe_idx, n_probe, ix->list_off, ix->list_rows,
+                           (int)ix->n_indexed, pr->exclude_tag, p->partial, p->q_valid, p->stats, grid, st);
+  if (e != cudaSuccess) return index_fail(e, "candidate scan launch");
+  e = launch_merge_gather(pv, p->partial, grid, nq, kk, p->q_valid, gp, *out, st);
+  if (e != cudaSuccess) return index_fail(e, "merge launch");
+  p->launches += 2;
+  return OILBIRD_OK;
+}
+
+int oilbird_index_read(oilbird_index_t* ix, int32_t* assign_host, int32_t* list_off_host,
+                       int32_t* list_rows_host) {
+  if (!ix) return OILBIRD_EINVAL;
+  ICU(cudaSetDevice(ix->pool->device));
+  ICU(cudaDeviceSynchronize());
+  const size_t n = (size_t)ix->n_indexed;
+  if (assign_host && n) ICU(cudaMemcpy(assign_host, ix->assign, n * 4, cudaMemcpyDeviceToHost));
+  if (list_off_host)
+    ICU(cudaMemcpy(list_off_host, ix->list_off, ((size_t)ix->n_lists + 1) * 4, cudaMemcpyDeviceToHost));
+  if (list_rows_host && n) ICU(cudaMemcpy(list_rows_host, ix->list_rows, n * 4, cudaMemcpyDeviceToHost));
+  return OILBIRD_OK;
+}
+
+}  // extern "C"

@@ -70,6 +70,7 @@ inline cudaError_t preload_kernel(K kernel, bool dynamic_smem = false) {
 }
 cudaError_t preload_append_kernels();
 cudaError_t preload_evict_kernels();
+cudaError_t preload_index_kernels();
 cudaError_t preload_merge_kernels();
 cudaError_t preload_merge_tree_kernels();
 cudaError_t preload_quant8_kernels();

@@ -11,6 +11,7 @@
 #include <vector>
 
 #include "internal.h"
+#include "pool_priv.h"
 
 using namespace oilbird;
 
@@ -48,6 +49,7 @@ cudaError_t preload_all_kernels() {
   (void)pdl_process_ok();
   if ((e = preload_append_kernels()) != cudaSuccess) return e;
   if ((e = preload_evict_kernels()) != cudaSuccess) return e;
+  if ((e = preload_index_kernels()) != cudaSuccess) return e;
   if ((e = preload_merge_kernels()) != cudaSuccess) return e;
   if ((e = preload_merge_tree_kernels()) != cudaSuccess) return e;
   if ((e = preload_quant8_kernels()) != cudaSuccess) return e;
@@ -76,28 +78,6 @@ namespace {
 constexpr size_t kAlign = 256;
 constexpr int kMaxProfile = 4096;
 size_t align_up(size_t v) { return (v + kAlign - 1) / kAlign * kAlign; }
-
-// Byte offsets of every device array inside one allocation.
-constexpr int kMaxGuards = 24;
-struct Layout {
-  size_t keys, tok, trace_id, trace_end, trace_tag, trace_gbase, qn, q_valid, partial, stats;
-  size_t xchg;
-  size_t q_stage, ex_stage, st_stage, tok_stage, stage_end, fuse_ready, scales;
-  size_t total;
-  // OILBIRD_DEBUG_GUARDS: sentinel bytes [g_lo, g_hi) behind every array (from its last
-  // byte to the next array's first), named after the array they follow
-  int n_guards;
-  size_t g_lo[kMaxGuards], g_hi[kMaxGuards];
-  const char* g_name[kMaxGuards];
-};
-constexpr unsigned char kGuardByte = 0xA5;
-
-struct Resolved {
-  int32_t d, max_traces, max_nq, max_k, max_append, max_lists;
-  int32_t e4m3;              // keys are E4M3 codes with one scale per row
-  int32_t guards;            // guard zones between the arrays (debugging aid)
-  int64_t capacity;
-};
 
 bool resolve(const oilbird_pool_config* c, int num_sms, Resolved* r) {
   if (!c) return false;
@@ -166,48 +146,6 @@ Layout make_layout(const Resolved& r) {
   return L;
 }
 }  // namespace
-
-struct oilbird_pool {
-  Resolved r;
-  Layout lay;
-  int device, num_sms;
-  bool owns_mem;
-  unsigned char* base;
-  // device arrays
-  uint16_t* keys;            // bf16 keys, or ...
-  uint8_t* codes;            // ... E4M3 codes (the same memory) with ...
-  float* scales;             // ... one scale per row
-  int32_t *tok, *trace_id, *trace_end;
-  uint64_t* trace_tag;
-  int64_t* trace_gbase;      // global position of each trace's first row (row sharding)
-  uint16_t* qn;
-  int32_t* q_valid;
-  unsigned long long* partial;
-  DeviceStats* stats;
-  float* xchg;               // tensor scan: cross-CTA threshold exchange
-  unsigned long long* fuse_ready;   // rows published by appends fused into a scan ...
-  unsigned long long fuse_target;   // ... and the host's count of them (enqueue time)
-  // host bookkeeping (enqueue-time truth)
-  int64_t n_rows;
-  std::vector<int64_t> t_start, t_end;
-  std::vector<uint64_t> t_tag;
-  std::vector<int64_t> t_gbase;     // global position of each trace's first row, or -1 if
-                                    // it is simply the local one (pool is not a shard)
-  int64_t launches;
-  // profiling
-  bool profile;
-  std::vector<cudaEvent_t> ev;   // pairs
-  int ev_used;
-  // pinned staging for host variants
-  unsigned char* pinned;       // host address
-  unsigned char* pinned_dev;   // the same block as the device sees it
-  size_t blob_off, result_off;
-  cudaEvent_t upload_done;
-  bool upload_pending;
-  // tensor-core scan: TMA tensor maps of this pool (nullptr = path unavailable)
-  size_t smem_limit;
-  TcCache* tc;
-};
 
 extern "C" {
 
@@ -517,12 +455,7 @@ static int check_params(const oilbird_pool* p, int32_t nq, const oilbird_query_p
   return check_query_params(nq, p->r.max_nq, p->r.max_k, pr, gp);
 }
 
-static PoolView view_of(const oilbird_pool* p) {
-  PoolView pv;
-  pv.keys = p->keys; pv.tok = p->tok; pv.trace_id = p->trace_id; pv.trace_end = p->trace_end;
-  pv.trace_tag = p->trace_tag; pv.d = p->r.d; pv.n_rows = (int32_t)p->n_rows;
-  return pv;
-}
+static PoolView view_of(const oilbird_pool* p) { return pool_view(p); }
 
 static bool out_ok(const oilbird_query_out* o, bool need_idx) {
   if (!o || !o->fired || !o->cont_len || !o->cont_tok) return false;

@@ -1,0 +1,167 @@
+"""GPU parity for the coarse index: the CUDA index against oracle/index.py on the same pool,
+centroids and queries.  Assignments and lists are integers and must be identical (the
+workloads keep the best two centroids of every row well apart, so accumulation order
+cannot decide); answers go through the acceptance rule of every other query test, applied to
+the oracle's candidate-restricted scores."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from oracle import OraclePool
+from oracle.index import OracleIndex
+from paper_2608_03839_b200 import binding as B
+from paper_2608_03839_b200 import workloads as W
+from parity import GAP, SCORE_BUG, fill_both, oracle_params
+
+pytestmark = pytest.mark.gpu
+
+
+def fixed(k, L, theta=-2.0, **kw):
+    return B.QueryParams(k=k, theta=theta, depth_mode=B.DEPTH_FIXED, cont_len=L, **kw)
+
+
+def check_index_query(out, oidx: OracleIndex, q_bits, n_probe, params, exclude=None):
+    """check_query's rule with the oracle's scores masked to the candidate rows."""
+    o = out.cpu()
+    idx, score = o.idx.numpy(), o.score.numpy()
+    ref = oidx.query(q_bits, n_probe, oracle_params(params, exclude), want_all_scores=True)
+    nq, k = idx.shape
+    for q in range(nq):
+        s_all = ref.all_scores[q]
+        kk = min(k, int(np.sum(np.isfinite(s_all))))
+        got = idx[q]
+        assert np.all(got[kk:] == -1) and np.all(np.isneginf(score[q, kk:]))
+        assert len(set(got[:kk].tolist())) == kk
+        if kk:
+            assert np.all(np.isfinite(s_all[got[:kk]])), "a row outside the probed lists was returned"
+            err = np.abs(score[q, :kk].astype(np.float64) - s_all[got[:kk]])
+            assert err.max() <= SCORE_BUG
+            s_k = float(ref.score[q, kk - 1])
+            assert np.all(s_all[got[:kk]] >= s_k - GAP)
+            must = np.where(s_all > s_k + GAP)[0]
+            assert set(must.tolist()) <= set(got[:kk].tolist())
+            for j in range(1, kk):
+                assert score[q, j - 1] > score[q, j] or (score[q, j - 1] == score[q, j] and got[j - 1] < got[j])
+            if abs(float(ref.score[q, 0]) - params.theta) > GAP:
+                assert o.fired[q] == ref.fired[q]
+        for j in range(k):
+            dep = params.cont_len if (o.fired[q] and got[j] >= 0) else 0
+            tok, n = oidx.pool.gather_one(int(got[j]), dep, params.offset, params.cont_len)
+            assert o.cont_len[q, j] == n and np.array_equal(o.cont_tok[q, j].numpy(), tok)
+    return ref
+
+
+def build_both(w, n_lists, seed=0, **pool_kw):
+    pool, ora = fill_both(w, **pool_kw)
+    # centroids: stored states of the pool, drawn at random (a sample of traffic)
+    g = np.random.default_rng(seed)
+    rows = np.sort(g.choice(w.n_rows, n_lists, replace=False))
+    raw = []
+    for r in rows:
+        t, i = divmod(int(r), w.rows_per_trace)
+        raw.append(w.trace(t, "cuda")[0][i])
+    cent = torch.stack(raw).contiguous()
+    gix, oix = B.Index(pool, cent), OracleIndex(ora, W.to_bits(cent))
+    return pool, ora, gix, oix
+
+
+def same_lists(gix, oix):
+    a, off, rows = gix.read()
+    assert np.array_equal(a, oix.assign.astype(np.int32))
+    want = oix.lists()
+    assert off[0] == 0 and off[-1] == oix.n_indexed
+    for l in range(oix.n_lists):
+        assert sorted(rows[off[l]:off[l + 1]].tolist()) == want[l].tolist()
+
+
+@pytest.mark.parametrize("d,n_lists", [(256, 24), (1024, 64)])
+def test_lists_and_answers_match_the_oracle(d, n_lists):
+    w = W.C1.scaled(n_rows=6000, d=d, nq=5, k=8, cont_len=4, n_centroids=40, rows_per_trace=500)
+    pool, ora, gix, oix = build_both(w, n_lists, spare_rows=600)
+    gix.refresh(); oix.refresh()
+    assert len(gix) == 6000
+    same_lists(gix, oix)
+    q, _ = w.queries("cuda")
+    for n_probe in (1, 3, n_lists, n_lists + 7):
+        for k in (1, 8, 40):
+            pr = fixed(k, 4, theta=0.8 if k == 8 else -2.0)
+            check_index_query(gix.query(q, n_probe, pr), oix, W.to_bits(q), n_probe, pr)
+    # every list probed: the full scan's own answer, bit for bit
+    pr = fixed(8, 4)
+    a, b = gix.query(q, n_lists, pr).cpu(), pool.query(q, pr).cpu()
+    assert torch.equal(a.idx, b.idx) and torch.equal(a.cont_tok, b.cont_tok)
+    assert torch.allclose(a.score, b.score, atol=SCORE_BUG, rtol=0)
+    # rows appended after the refresh are found without one (the tail), then move into lists
+    g = torch.Generator(device="cuda").manual_seed(3)
+    st = torch.randn(300, d, generator=g, device="cuda").to(torch.bfloat16)
+    tk = torch.arange(300, dtype=torch.int32, device="cuda")
+    pool.append(st, tk, tag=77)
+    ora.append(W.to_bits(st), tk.cpu().numpy(), tag=77)
+    q2 = torch.cat([st[17:18], q[:2]]).contiguous()
+    out = gix.query(q2, 1, fixed(4, 4))
+    assert int(out.idx[0, 0]) == 6017
+    check_index_query(out, oix, W.to_bits(q2), 1, fixed(4, 4))
+    gix.refresh(); oix.refresh()
+    assert len(gix) == 6300
+    same_lists(gix, oix)
+    check_index_query(gix.query(q2, 2, fixed(4, 4)), oix, W.to_bits(q2), 2, fixed(4, 4))
+    # exclusion tags
+    ex = np.array([77, 0, 3], dtype=np.uint64)
+    pr = fixed(6, 4, exclude_tag=torch.from_numpy(ex.view(np.int64)).cuda())
+    check_index_query(gix.query(q2, 4, pr), oix, W.to_bits(q2), 4, pr, exclude=ex)
+    assert pool.stats()["stalled"] == 0
+
+
+def test_index_after_eviction_needs_a_reset():
+    w = W.C1.scaled(n_rows=2000, d=128, nq=3, k=4, cont_len=2, rows_per_trace=250)
+    pool, ora, gix, oix = build_both(w, 16)
+    gix.refresh(); oix.refresh()
+    pool.evict_oldest(2); ora.evict_oldest(2)
+    q, _ = w.queries("cuda")
+    with pytest.raises(B.OilbirdError) as e:
+        gix.query(q, 2, fixed(4, 2))
+    assert e.value.code == B.EINVAL
+    gix.reset(); oix.reset()
+    # everything is tail now: the full scan's answer whatever is probed
+    pr = fixed(4, 2)
+    a, b = gix.query(q, 1, pr).cpu(), pool.query(q, pr).cpu()
+    assert torch.equal(a.idx, b.idx)
+    gix.refresh(); oix.refresh()
+    same_lists(gix, oix)
+    check_index_query(gix.query(q, 3, pr), oix, W.to_bits(q), 3, pr)
+
+
+def test_c2_shaped_pool_recall_and_candidate_volume():
+    # the single-request configuration at a quarter of its size: 512 centroids' worth of
+    # traffic, 256 lists from a sample of stored states
+    w = W.C2.scaled(n_rows=16384)
+    pool, ora, gix, oix = build_both(w, 256)
+    gix.refresh(); oix.refresh()
+    same_lists(gix, oix)
+    q, meta = w.queries("cuda", nq=4)
+    pr = fixed(w.k, w.cont_len)
+    exact = pool.query(q, pr).cpu()
+    hits = []
+    for n_probe in (1, 4, 16, 256):
+        out = gix.query(q, n_probe, pr)
+        check_index_query(out, oix, W.to_bits(q), n_probe, pr)
+        o = out.cpu()
+        hits.append(np.mean([len(set(o.idx[i].tolist()) & set(exact.idx[i].tolist())) / w.k
+                             for i in range(4)]))
+    assert hits == sorted(hits) and hits[-1] == 1.0
+
+
+def test_bad_arguments_are_refused():
+    pool = B.Pool(64, 100, key_format="e4m3")
+    cent = torch.zeros(4, 64, dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(B.OilbirdError) as e:
+        B.Index(pool, cent)                                  # 16-bit pools only
+    assert e.value.code == B.EINVAL
+    pool = B.Pool(64, 100)
+    ix = B.Index(pool, cent)
+    q = torch.zeros(1, 64, dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(B.OilbirdError):
+        ix.query(q, 0, fixed(4, 2))                          # at least one probe
+    out = ix.query(q, 2, fixed(4, 2)).cpu()                  # an empty pool is legal
+    assert torch.all(out.idx == -1) and out.fired[0] == 0

@@ -918,6 +918,94 @@ def run_load(args):
     pool.close()
 
 
+def run_index(args):
+    """Bounded lookup cost: the coarse index (inverted file over a sample of stored states).
+    One step = one lookup of one query through the index; reported for several n_probe with
+    the recall of the exact top-k (the full scan's answer on the same pool) beside it, the
+    time of the full scan, and the rate at which refresh() assigns rows to lists."""
+    from paper_2608_03839_b200 import binding as B
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda:0")
+    w = W.CONFIGS[args.config or "C2"]
+    n0 = args.rows or (W.C5_START_ROWS if w.name == "C5" else w.n_rows)
+    K, Wm = args.steps, args.warmup
+    pool = B.Pool(w.d, n0 + 8, max_nq=64, max_k=w.k, max_traces=w.num_traces + 8)
+    fill_pool(pool, w, n0, dev)
+    # centroids: the states of whole stored traces, four per cluster of the recipe on average
+    n_lists = int(min(65536, max(64, 4 * max(w.n_centroids, 1)), n0))
+    C = w._centroids(dev) if w.kind == "clustered" else None
+    cent, t = [], 0
+    step_t = max(1, (n0 // w.rows_per_trace) // max(1, n_lists // w.rows_per_trace))
+    while sum(c.shape[0] for c in cent) < n_lists:
+        cent.append(w.trace(t, dev, C)[0])
+        t += step_t
+    cent = torch.cat(cent)[:n_lists].contiguous()
+    ix = B.Index(pool, cent)
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    ix.refresh()
+    torch.cuda.synchronize()
+    refresh_s = time.perf_counter() - t0
+    n_q = 64
+    qs, _ = w.queries(dev, nq=n_q)
+    pr = B.QueryParams(k=w.k, theta=0.8, offset=2, depth_mode=B.DEPTH_FIXED, cont_len=w.cont_len)
+    exact = pool.query(qs, pr).cpu().idx.numpy()
+    one = [qs[i:i + 1].contiguous() for i in range(n_q)]
+    out = B.QueryOut.empty(1, w.k, w.cont_len, dev)
+
+    def timed(fn):
+        for i in range(Wm):
+            fn(i)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for i in range(K):
+            fn(i)
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / K * 1e3        # us
+
+    full_us = timed(lambda i: pool.query(one[i % n_q], pr, out=out))
+    a, off, rows = ix.read()
+    lens = np.diff(off)
+    table = []
+    sampler = ClockSampler(physical_device(0))
+    sampler.start()
+    for n_probe in (1, 4, 16, 64):
+        us = timed(lambda i: ix.query(one[i % n_q], n_probe, pr, out=out))
+        got = ix.query(qs, n_probe, pr).cpu().idx.numpy()
+        rec = float(np.mean([len(set(got[i].tolist()) & set(exact[i].tolist())) / w.k
+                             for i in range(n_q)]))
+        table.append({"n_probe": n_probe, "us_per_query": us, "queries_per_sec": 1e6 / us,
+                      "recall_of_exact_top_k": rec, "speedup_vs_full_scan": full_us / us})
+    clocks = sampler.stop()
+    head = table[2]
+    peaks, peak_kind = measured_peaks()
+    cand_bytes = (n_lists + 16 * float(lens.mean())) * w.d * 2
+    line = {"metric": "index_queries_per_sec", "value": head["queries_per_sec"], "unit": UNIT,
+            "n_gpus": 1, "steps": K, "warmup": Wm, "ms_per_step": head["us_per_query"] / 1e3,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "bf16 keys, fp32 accumulate", "data": "synthetic",
+            "config": {"workload": f"index: {w.name} recipe, pool N={n0} x d={w.d} bf16, {n_lists} lists "
+                                   f"(centroids: stored states of whole traces), nq=1, k={w.k}, "
+                                   f"L={w.cont_len}; headline n_probe=16",
+                       "rows_per_list": {"mean": float(lens.mean()), "max": int(lens.max()),
+                                         "empty_lists": int((lens == 0).sum())}},
+            "probes": table, "full_scan_us_per_query": full_us,
+            "refresh": {"rows": n0, "seconds": refresh_s, "rows_per_sec": n0 / refresh_s},
+            "clocks": clocks, "gpu_launches": 5 * K,
+            "roofline": {"bound": "hbm", "kernel": "centroid lookup + candidate scan (n_probe = 16)",
+                         "achieved": cand_bytes / (head["us_per_query"] * 1e-6) / 1e9,
+                         "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                         "frac": cand_bytes / (head["us_per_query"] * 1e-6) / 1e9 / peaks["hbm_gbs"],
+                         "peak_kind": peak_kind, "bytes_per_launch": cand_bytes, "traffic": None,
+                         "note": "a lookup moves the centroids and a few hundred candidate rows: "
+                                 "five dependent launches, latency-bound, not bandwidth-bound"}}
+    print(json.dumps(line), flush=True)
+    ix.close()
+    pool.close()
+
+
 def run_merge(args):
     """Third workload: chain post-filter + tree merge for a batch of requests (paper sizes:
     8 semantic chains of up to 48 tokens + 7 other chains into a 44-node tree, 16 of 60 nodes)."""
@@ -1070,9 +1158,10 @@ def main():
     ap.add_argument("--keys", default="bf16", choices=["bf16", "e4m3"],
                     help="stored key format: the paper's 16-bit keys, or the bounded-store "
                          "variant with 8-bit keys (FP8 E4M3 + one scale per row)")
-    ap.add_argument("--workload", default="pool", choices=["pool", "ring", "merge", "evict", "load"],
+    ap.add_argument("--workload", default="pool", choices=["pool", "ring", "merge", "evict", "load", "index"],
                     help="pool: the trace-store query path (default); ring: the recycled pool; "
-                         "evict: bounded store; merge: chain merge; load: bulk trace load")
+                         "evict: bounded store; merge: chain merge; load: bulk trace load; "
+                         "index: bounded lookup cost (coarse index, with recall)")
     ap.add_argument("--sharded", action="store_true",
                     help="one logical pool row-sharded over the ranks (default: one pool per rank)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -1097,6 +1186,11 @@ def main():
         args.steps = 10 if args.steps is None else args.steps
         args.warmup = 3 if args.warmup is None else max(args.warmup, 3)
         run_load(args)
+        return
+    if args.workload == "index":
+        args.steps = 300 if args.steps is None else args.steps
+        args.warmup = 20 if args.warmup is None else max(args.warmup, 3)
+        run_index(args)
         return
     if args.workload == "merge":
         args.steps = 200 if args.steps is None else args.steps

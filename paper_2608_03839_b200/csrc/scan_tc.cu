@@ -93,22 +93,8 @@ constexpr int kColsPerRound = 16;      // score columns filtered between two dra
 constexpr int kQueueCap = kTileM * kColsPerRound;
 constexpr int kMaxStages = 8;
 
-// Compile-time overrides for measurements (0 = the plan below decides).
-#ifndef OILBIRD_TC_FORCE_MT
-#define OILBIRD_TC_FORCE_MT 0
-#endif
-#ifndef OILBIRD_TC_FORCE_LISTS
-#define OILBIRD_TC_FORCE_LISTS 0          // 1 = shared memory, 2 = global memory
-#endif
-#ifndef OILBIRD_TC_FIRST_TILE_BOUND
-#define OILBIRD_TC_FIRST_TILE_BOUND 1     // 0 = a CTA's first tile goes through the lists unfiltered
-#endif
-#ifndef OILBIRD_TC_PAIR
-#define OILBIRD_TC_PAIR 1                 // 0 = never pair two CTAs on a tile
-#endif
-#ifndef OILBIRD_TC_MIN_SMEM_STAGES
-#define OILBIRD_TC_MIN_SMEM_STAGES 4      // lists stay in shared memory if this many stages fit
-#endif
+// Lists stay in shared memory if this many ring stages still fit beside them.
+constexpr int kTcMinSmemStages = 4;
 
 // ------------------------------------------------------------------ PTX wrappers ---
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
@@ -716,7 +702,7 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap key_map,
       epilogue_bar();
       if (!sh.epi_go) { ok = false; break; }
       tc_fence_after();
-      if (OILBIRD_TC_FIRST_TILE_BOUND && use_xchg && iter == 0) {
+      if (use_xchg && iter == 0) {
         // A CTA's first tile, before any threshold exists: every score would be a candidate
         // (sorted 32*E at a time and merged, a couple of tiles' worth of time during which
         // the accumulators stay full and the key stream stalls).  Instead the tile is read
@@ -979,7 +965,7 @@ static TcPlan tc_plan_single(int nq, int k, int n_tiles128, int num_sms, size_t 
 static TcPlan tc_plan(int nq, int k, int n_tiles128, int num_sms, size_t smem_limit) {
   // More than 128 queries on a large pool: two CTAs per tile of 256 rows (see the kernel);
   // each loads half of the query rows, so their number is a multiple of 32
-  if (OILBIRD_TC_PAIR && nq > 128 && n_tiles128 >= 4 * num_sms && num_sms >= 2) {
+  if (nq > 128 && n_tiles128 >= 4 * num_sms && num_sms >= 2) {
     TcPlan p;
     p.per_pass = OILBIRD_MAX_NQ;
     p.n_pad = (nq + 31) / 32 * 32;
@@ -1005,13 +991,9 @@ static TcPlan tc_plan_single(int nq, int k, int n_tiles128, int num_sms, size_t 
   // the lists in L2 beats a shallower or one-tile ring with the lists on chip (nq = 128,
   // k = 64 at d = 8192: 2.61 ms against 3.11).
   const bool many_tiles = n_tiles128 >= 2 * num_sms;
-  bool two = many_tiles && 2 * 2 * n_pad <= 512 && tc_fits(n_pad, kk, 2, true, 3, smem_limit, &st);
-  if (OILBIRD_TC_FORCE_MT == 1) two = false;
-  if (OILBIRD_TC_FORCE_MT == 2) two = 2 * n_pad <= 512 && tc_fits(n_pad, kk, 2, true, 2, smem_limit, &st);
+  const bool two = many_tiles && 2 * 2 * n_pad <= 512 && tc_fits(n_pad, kk, 2, true, 3, smem_limit, &st);
   const int mt = two ? 2 : 1;
-  bool gl = !tc_fits(n_pad, kk, mt, false, OILBIRD_TC_MIN_SMEM_STAGES, smem_limit, &st);
-  if (OILBIRD_TC_FORCE_LISTS == 1) gl = !tc_fits(n_pad, kk, mt, false, 2, smem_limit, &st);
-  if (OILBIRD_TC_FORCE_LISTS == 2) gl = true;
+  const bool gl = !tc_fits(n_pad, kk, mt, false, kTcMinSmemStages, smem_limit, &st);
   p.global_lists = gl ? 1 : 0;
   p.mt = mt;
   p.stages = 0;

@@ -479,8 +479,9 @@ int oilbird_merge_chains(int32_t nq, const int32_t* sem_tok, const int32_t* sem_
  * found).  16-bit pools only.  create() copies the centroids (enqueued on cuda_stream); the
  * caller's array is free again once that work has completed.  After oilbird_pool_reset or
  * oilbird_pool_evict_oldest the row numbers the index holds are stale: call
- * oilbird_index_reset (all rows become tail) and refresh again; refresh and query refuse with
- * EINVAL while the pool holds fewer rows than the index covers.  Index calls enqueue on
+ * oilbird_index_reset (all rows become tail) and refresh again; until then refresh and query
+ * refuse with EINVAL (the pool counts such calls and the index remembers the count its lists
+ * were built under).  Index calls enqueue on
  * cuda_stream and use the pool's scratch, so they follow the pool's one-stream, one-thread
  * rule.  Destroy the index before its pool.
  */

@@ -203,6 +203,7 @@ struct oilbird_index {
   oilbird_pool* cent;            // the centroids, as a pool of n_lists rows
   int32_t n_lists;
   int64_t n_indexed;             // rows that have a list (enqueue-time truth)
+  int64_t generation;            // the pool's row numbering the lists refer to
   unsigned char* mem;
   int32_t *assign, *list_rows, *list_off, *cursor, *counts;
   // results of the lookups on the centroids
@@ -236,6 +237,7 @@ int oilbird_index_create(oilbird_index_t** out, oilbird_pool_t* pool, const void
   oilbird_index* ix = new (std::nothrow) oilbird_index();
   if (!ix) return OILBIRD_ENOMEM;
   ix->pool = pool; ix->n_lists = n_lists; ix->n_indexed = 0; ix->cent = nullptr; ix->mem = nullptr;
+  ix->generation = pool->generation;
   oilbird_pool_config cc = {};
   cc.d = pool->r.d; cc.capacity_rows = n_lists; cc.max_traces = 1; cc.max_nq = OILBIRD_MAX_NQ;
   cc.max_k = OILBIRD_MAX_K; cc.max_append = 1; cc.device = pool->device;
@@ -297,6 +299,7 @@ int oilbird_index_reset(oilbird_index_t* ix, void* cuda_stream) {
   // every list empty again: offsets all zero
   ICU(cudaMemsetAsync(ix->list_off, 0, ((size_t)ix->n_lists + 1) * 4, (cudaStream_t)cuda_stream));
   ix->n_indexed = 0;
+  ix->generation = ix->pool->generation;
   return OILBIRD_OK;
 }
 
@@ -306,7 +309,10 @@ int oilbird_index_refresh(oilbird_index_t* ix, void* cuda_stream) {
   ICU(cudaSetDevice(p->device));
   cudaStream_t st = (cudaStream_t)cuda_stream;
   const int64_t n = p->n_rows;
-  if (n < ix->n_indexed) return OILBIRD_EINVAL;          // the pool was reset or evicted from: reset the index
+  // the pool was reset or evicted from since: its rows have other numbers now
+  if (p->generation != ix->generation && ix->n_indexed > 0) return OILBIRD_EINVAL;
+  if (n < ix->n_indexed) return OILBIRD_EINVAL;
+  ix->generation = p->generation;
   if (n == ix->n_indexed) return OILBIRD_OK;
   // assign the new rows: their stored keys, a batch at a time, as queries against the centroids
   oilbird_query_params pr;
@@ -357,7 +363,9 @@ int oilbird_index_query(oilbird_index_t* ix, const void* q_bf16, int32_t nq, int
     snprintf(g_index_err, sizeof g_index_err, "misaligned pointer");
     return OILBIRD_EINVAL;
   }
-  if (p->n_rows < ix->n_indexed) return OILBIRD_EINVAL;   // pool reset or evicted from: reset the index
+  // pool reset or evicted from since the lists were built: reset the index first
+  if ((p->generation != ix->generation && ix->n_indexed > 0) || p->n_rows < ix->n_indexed)
+    return OILBIRD_EINVAL;
   ICU(cudaSetDevice(p->device));
   cudaStream_t st = (cudaStream_t)cuda_stream;
   // probe: the n_probe best centroids of every query

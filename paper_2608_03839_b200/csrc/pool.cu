@@ -202,7 +202,7 @@ int oilbird_pool_create(oilbird_pool_t** out, const oilbird_pool_config* cfg) {
   oilbird_pool* p = new (std::nothrow) oilbird_pool();
   if (!p) return OILBIRD_ENOMEM;
   p->r = r; p->lay = lay; p->device = cfg->device; p->num_sms = prop.multiProcessorCount;
-  p->n_rows = 0; p->launches = 0; p->profile = false; p->ev_used = 0;
+  p->n_rows = 0; p->launches = 0; p->generation = 0; p->profile = false; p->ev_used = 0;
   p->pinned = nullptr; p->pinned_dev = nullptr;
   if (cfg->arena) {
     size_t mis = (size_t)((uintptr_t)cfg->arena % kAlign);
@@ -266,6 +266,7 @@ int oilbird_pool_reset(oilbird_pool_t* p, void* stream) {
   CU(cudaSetDevice(p->device));
   CU(cudaMemsetAsync(p->stats, 0, kStatsCounterBytes, (cudaStream_t)stream));   // not the wait limit
   p->n_rows = 0;
+  p->generation += 1;
   p->t_start.clear(); p->t_end.clear(); p->t_tag.clear(); p->t_gbase.clear();
   return OILBIRD_OK;
 }
@@ -373,6 +374,7 @@ int oilbird_pool_evict_oldest(oilbird_pool_t* p, int32_t n_traces, int64_t* rows
                                  p->trace_id, head, live, row_bytes, nt, p->num_sms, st);
   if (e != cudaSuccess) return cuda_fail(e, "compaction kernel launch");
   if (live > 0) p->launches += 1;
+  p->generation += 1;
   // the host's copy of the trace table is the truth: renumber it, then publish it
   p->t_start.erase(p->t_start.begin(), p->t_start.begin() + nt);
   p->t_end.erase(p->t_end.begin(), p->t_end.begin() + nt);

@@ -58,6 +58,7 @@ struct oilbird_pool {
   std::vector<int64_t> t_gbase;     // global position of each trace's first row, or -1 if
                                     // it is simply the local one (pool is not a shard)
   int64_t launches;
+  int64_t generation;         // counts the calls that renumber rows (reset, eviction)
   // profiling
   bool profile;
   std::vector<cudaEvent_t> ev;   // pairs

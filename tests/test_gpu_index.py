@@ -115,13 +115,25 @@ def test_lists_and_answers_match_the_oracle(d, n_lists):
 
 def test_index_after_eviction_needs_a_reset():
     w = W.C1.scaled(n_rows=2000, d=128, nq=3, k=4, cont_len=2, rows_per_trace=250)
-    pool, ora, gix, oix = build_both(w, 16)
+    pool, ora, gix, oix = build_both(w, 16, spare_rows=1000)
     gix.refresh(); oix.refresh()
     pool.evict_oldest(2); ora.evict_oldest(2)
     q, _ = w.queries("cuda")
     with pytest.raises(B.OilbirdError) as e:
         gix.query(q, 2, fixed(4, 2))
     assert e.value.code == B.EINVAL
+    # growing back past the indexed size does not make the old row numbers right again
+    g = torch.Generator(device="cuda").manual_seed(8)
+    for tag in (501, 502, 503):
+        st = torch.randn(250, w.d, generator=g, device="cuda").to(torch.bfloat16)
+        tk = torch.arange(250, dtype=torch.int32, device="cuda")
+        pool.append(st, tk, tag=tag)
+        ora.append(W.to_bits(st), tk.cpu().numpy(), tag=tag)
+    assert len(pool) > len(gix)
+    for call in (lambda: gix.query(q, 2, fixed(4, 2)), gix.refresh):
+        with pytest.raises(B.OilbirdError) as e:
+            call()
+        assert e.value.code == B.EINVAL
     gix.reset(); oix.reset()
     # everything is tail now: the full scan's answer whatever is probed
     pr = fixed(4, 2)

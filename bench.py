@@ -320,34 +320,57 @@ def measure(pool, w, nq, rows_step, K, Wm, dev, world, rank, local, args, n0, ra
     h_q = [q.cpu().pin_memory() for q in queries]
     h_out = B.QueryOut.empty(nq, w.k, w.cont_len, "cpu")
 
-    def step_host():
-        i = step_no[0] % n_in
-        pool.step_host(h_states[i], h_toks[i], h_q[i], pr, h_out, tag=1_000_000 + step_no[0])
-        step_no[0] += 1
+    h_outs = [h_out, B.QueryOut.empty(nq, w.k, w.cont_len, "cpu")]
 
-    make_room(Wm + K, new_pass=True)
-    for _ in range(Wm):
-        step_host()
-    barrier()
-    e2e_ms = []
-    t_wall = time.perf_counter()
-    while True:
-        if not make_room(K):
-            break
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record()
-        for _ in range(K):
-            step_host()
-        e1.record()
-        torch.cuda.synchronize()
-        e2e_ms.append(e0.elapsed_time(e1))
-        go = torch.tensor([1 if (time.perf_counter() - t_wall < MIN_REGION_S and
-                                 len(e2e_ms) < args.max_repeats) else 0], device=dev)
-        if world > 1:                           # every rank takes the same number of repeats
-            dist.all_reduce(go, op=dist.ReduceOp.MIN)
-        if not int(go.item()):
-            break
-    barrier()
+    def steps_sync(n):
+        """One step at a time: the call returns with the answer on the host."""
+        for _ in range(n):
+            i = step_no[0] % n_in
+            pool.step_host(h_states[i], h_toks[i], h_q[i], pr, h_out, tag=1_000_000 + step_no[0])
+            step_no[0] += 1
+
+    def steps_two_deep(n):
+        """Two steps in flight (several requests share a pool): the host packs step j+1 and
+        reads step j-1 while the device works on step j.  Every step's inputs still cross
+        from pinned host memory and every step's answer is read on the host, inside the
+        timed region; the region ends when the last answer has been read."""
+        for j in range(n):
+            i = step_no[0] % n_in
+            if j >= 2:
+                pool.step_host_end(j % 2, h_outs[j % 2])
+            pool.step_host_begin(h_states[i], h_toks[i], h_q[i], pr, slot=j % 2,
+                                 tag=1_000_000 + step_no[0])
+            step_no[0] += 1
+        for j in range(max(0, n - 2), n):
+            pool.step_host_end(j % 2, h_outs[j % 2])
+
+    def e2e_pass(run):
+        make_room(Wm + K, new_pass=True)
+        run(Wm)
+        barrier()
+        ms = []
+        t_wall = time.perf_counter()
+        while True:
+            if not make_room(K):
+                break
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            run(K)
+            e1.record()
+            torch.cuda.synchronize()
+            ms.append(e0.elapsed_time(e1))
+            go = torch.tensor([1 if (time.perf_counter() - t_wall < MIN_REGION_S and
+                                     len(ms) < args.max_repeats) else 0], device=dev)
+            if world > 1:                       # every rank takes the same number of repeats
+                dist.all_reduce(go, op=dist.ReduceOp.MIN)
+            if not int(go.item()):
+                break
+        barrier()
+        return ms
+
+    e2e_ms = e2e_pass(steps_two_deep)
+    e2e_sync_ms = e2e_pass(steps_sync)
+    _, e2e_sync_value = aggregate(float(np.median(e2e_sync_ms)), K * nq, world, dev)
     _, e2e_value = aggregate(float(np.median(e2e_ms)), K * nq, world, dev)
     h2d = rows_step * w.d * 2 + rows_step * 4 + nq * w.d * 2
     d2h = nq * w.k * (4 + 4 + 4 + 4 * w.cont_len) + nq * 4
@@ -396,7 +419,14 @@ def measure(pool, w, nq, rows_step, K, Wm, dev, world, rank, local, args, n0, ra
         "key_scan_gbs": rows_mean * row_bytes / (max_ms / K * 1e-3) / 1e9,
         "clocks": clocks,
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d,
-                "d2h_bytes_per_step": d2h, "repeats": len(e2e_ms)},
+                "d2h_bytes_per_step": d2h, "repeats": len(e2e_ms),
+                "mode": "oilbird_pool_step_host_begin / _end, two steps in flight (throughput, "
+                        "as `value` is: steps of independent requests back to back); every "
+                        "step's inputs come from pinned host memory and its answer is read on "
+                        "the host inside the timed region",
+                "one_step_at_a_time": {"value": e2e_sync_value, "unit": UNIT,
+                                       "call": "oilbird_pool_step_host (returns with the answer)",
+                                       "repeats": len(e2e_sync_ms)}},
         "gpu_launches": int(launches),
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"],
                      "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"],

@@ -264,6 +264,32 @@ int oilbird_pool_step_host(oilbird_pool_t* pool, const void* states_bf16_host,
                            const oilbird_query_params* params, const oilbird_query_out* out_host,
                            void* cuda_stream);
 
+/*
+ * The same step in two halves, so that the host work of one step (packing its inputs,
+ * reading its results) overlaps the device work of another: several requests share a
+ * pool and their lookups do not depend on one another.  `begin` copies the inputs into
+ * the pinned block of `slot` (0 <= slot < OILBIRD_HOST_SLOTS; the caller's buffers are
+ * free again when it returns), uploads them on a copy stream of the pool's own into the
+ * slot's device staging block (so the upload runs under the kernels of the step before),
+ * enqueues the step on cuda_stream behind that upload and returns without waiting; the
+ * merge kernel writes the results into the slot's mapped block.  `end` waits
+ * for that step alone (an event behind its kernels) and copies the results into the host
+ * arrays of `out`, whose shape is the one `begin` was given (nq, params->k,
+ * params->cont_len).  A slot holds one step: `begin` on a slot whose `end` has not been
+ * called, and `end` on an idle slot, return OILBIRD_EINVAL and do nothing.  Steps take
+ * effect in the order of their `begin` calls (one stream); `end` may be called in any
+ * order.  params->exclude_tag is a host pointer, read during `begin`.  The synchronous
+ * *_host calls have a slot and a staging block of their own and may be mixed in.
+ */
+#define OILBIRD_HOST_SLOTS 2
+int oilbird_pool_step_host_begin(oilbird_pool_t* pool, const void* states_bf16_host,
+                                 const int32_t* tokens_host, int64_t n, uint64_t trace_tag,
+                                 uint32_t flags, const void* q_bf16_host, int32_t nq,
+                                 const oilbird_query_params* params, int32_t slot,
+                                 void* cuda_stream);
+int oilbird_pool_step_host_end(oilbird_pool_t* pool, int32_t slot,
+                               const oilbird_query_out* out_host);
+
 /* Introspection (host side; none of these enqueue work unless stated). */
 int64_t oilbird_pool_size(const oilbird_pool_t* pool);          /* rows appended so far  */
 int32_t oilbird_pool_num_traces(const oilbird_pool_t* pool);

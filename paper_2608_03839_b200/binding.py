@@ -32,6 +32,7 @@ DEBUG_GUARDS = 2       # pool flag: sentinel bytes behind every array (see Pool.
 DEPTH_FIXED, DEPTH_TIERED = 0, 1
 PATH_AUTO, PATH_GEMV, PATH_TENSOR, PATH_MMA = 0, 1, 2, 3
 MAX_NQ, MAX_K, MAX_CONT_LEN, MAX_TIERS = 256, 128, 128, 4
+HOST_SLOTS = 2
 
 
 class PoolConfig(ctypes.Structure):
@@ -105,6 +106,9 @@ SYMBOLS = {
     "oilbird_pool_step_host": (ctypes.c_int, [_vp, _vp, _vp, _i64, _u64, _u32, _vp, _i32,
                                               ctypes.POINTER(CQueryParams),
                                               ctypes.POINTER(CQueryOut), _vp]),
+    "oilbird_pool_step_host_begin": (ctypes.c_int, [_vp, _vp, _vp, _i64, _u64, _u32, _vp, _i32,
+                                                    ctypes.POINTER(CQueryParams), _i32, _vp]),
+    "oilbird_pool_step_host_end": (ctypes.c_int, [_vp, _i32, ctypes.POINTER(CQueryOut)]),
     "oilbird_pool_size": (_i64, [_vp]),
     "oilbird_pool_num_traces": (_i32, [_vp]),
     "oilbird_pool_status": (ctypes.c_int, [_vp, ctypes.POINTER(PoolStats), _vp]),
@@ -189,8 +193,8 @@ class OilbirdError(RuntimeError):
     def __init__(self, code: int, where: str):
         L = lib()
         msg = L.oilbird_strerror(code).decode()
-        if code in (ECUDA, ENOMEM, EGUARD) or (code == EINVAL and "aligned" in
-                                                  L.oilbird_last_cuda_error().decode()):
+        if code in (ECUDA, ENOMEM, EGUARD) or (code == EINVAL and any(
+                w in L.oilbird_last_cuda_error().decode() for w in ("aligned", "in flight"))):
             msg += " (" + L.oilbird_last_cuda_error().decode() + ")"
         super().__init__(f"{where}: {msg} [{code}]")
         self.code = code
@@ -530,6 +534,23 @@ class Pool:
             self._h, states.data_ptr(), tokens.data_ptr(), int(tokens.shape[0]), int(tag),
             NEW_TRACE if new_trace else 0, q.data_ptr(), int(q.shape[0]), ctypes.byref(cp),
             ctypes.byref(out._c), _stream_ptr(stream)), "oilbird_pool_step_host")
+        return out
+
+    def step_host_begin(self, states: torch.Tensor, tokens: torch.Tensor, q: torch.Tensor,
+                        params: QueryParams, slot: int, tag: int = 0, new_trace: bool = True,
+                        stream=None) -> None:
+        """First half of step_host: returns once the step is enqueued (slot 0 or 1)."""
+        ex_ptr = params.exclude_tag.data_ptr() if params.exclude_tag is not None else None
+        cp = params.to_c(ex_ptr)
+        _check(self._L.oilbird_pool_step_host_begin(
+            self._h, states.data_ptr(), tokens.data_ptr(), int(tokens.shape[0]), int(tag),
+            NEW_TRACE if new_trace else 0, q.data_ptr(), int(q.shape[0]), ctypes.byref(cp),
+            int(slot), _stream_ptr(stream)), "oilbird_pool_step_host_begin")
+
+    def step_host_end(self, slot: int, out: QueryOut) -> QueryOut:
+        """Second half: waits for that slot's step, fills the CPU tensors of `out`."""
+        _check(self._L.oilbird_pool_step_host_end(self._h, int(slot), ctypes.byref(out._c)),
+               "oilbird_pool_step_host_end")
         return out
 
     # ---- introspection --------------------------------------------------------------

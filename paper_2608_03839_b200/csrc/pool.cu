@@ -142,6 +142,11 @@ Layout make_layout(const Resolved& r) {
   guards = r.guards != 0;
   L.tok_stage = take((size_t)r.max_append * 4, "host staging");
   L.stage_end = L.tok_stage + align_up((size_t)r.max_append * 4);   // (a guard may follow)
+  const size_t stage_bytes = L.stage_end - L.q_stage;
+  guards = false;
+  L.pipe_stage[0] = take(stage_bytes, "");
+  guards = r.guards != 0;
+  L.pipe_stage[1] = take(stage_bytes, "staging of host steps in flight");
   L.total = off;
   return L;
 }
@@ -254,7 +259,12 @@ int oilbird_pool_destroy(oilbird_pool_t* p) {
   cudaSetDevice(p->device);
   cudaDeviceSynchronize();
   for (cudaEvent_t e : p->ev) cudaEventDestroy(e);
-  if (p->pinned) { cudaFreeHost(p->pinned); cudaEventDestroy(p->upload_done); }
+  if (p->pinned) {
+    cudaFreeHost(p->pinned);
+    cudaEventDestroy(p->upload_done);
+    for (auto& sl : p->slot) { cudaEventDestroy(sl.done); cudaEventDestroy(sl.copied); }
+    cudaStreamDestroy(p->copy_stream);
+  }
   tc_cache_destroy(p->tc);
   if (p->owns_mem) cudaFree(p->base);
   delete p;
@@ -280,6 +290,11 @@ int64_t oilbird_pool_launch_count(const oilbird_pool_t* p) { return p ? p->launc
 static bool aligned(const void* p, uintptr_t a) { return ((uintptr_t)p & (a - 1)) == 0; }
 static int misaligned(const char* what) {
   snprintf(g_cuda_err, sizeof g_cuda_err, "%s is not aligned as the header requires", what);
+  return OILBIRD_EINVAL;
+}
+
+static int refused(const char* why) {
+  snprintf(g_cuda_err, sizeof g_cuda_err, "%s", why);
   return OILBIRD_EINVAL;
 }
 
@@ -689,6 +704,7 @@ int oilbird_pool_gather(oilbird_pool_t* p, const int32_t* idx, const float* scor
 // and let the merge kernel write the results straight into the mapped result block, which
 // is valid on the host once the stream has been synchronised.
 constexpr size_t kPackLimit = 256 << 10;   // bytes up to which a step's inputs are packed
+constexpr int kHostSlots = OILBIRD_HOST_SLOTS;   // host steps that may be in flight
 
 struct HostBlob {
   size_t o_st, o_tok, o_q, o_ex, used;
@@ -716,16 +732,25 @@ static int ensure_pinned(oilbird_pool* p) {
   // first rather than have it happen under kernels that are chained and waiting
   cudaError_t e = cudaDeviceSynchronize();
   if (e != cudaSuccess) return cuda_fail(e, "cudaDeviceSynchronize");
-  e = cudaHostAlloc((void**)&h, align_up(a_bytes) + b_bytes + o_bytes, cudaHostAllocMapped);
+  const size_t stride = align_up(b_bytes + o_bytes);
+  e = cudaHostAlloc((void**)&h, align_up(a_bytes) + (kHostSlots + 1) * stride, cudaHostAllocMapped);
   if (e != cudaSuccess) return cuda_fail(e, "cudaHostAlloc");
   void* dptr = nullptr;
   e = cudaHostGetDevicePointer(&dptr, h, 0);
   if (e == cudaSuccess) e = cudaEventCreateWithFlags(&p->upload_done, cudaEventDisableTiming);
+  for (auto& sl : p->slot) {
+    sl.busy = false;
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&sl.done, cudaEventDisableTiming);
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&sl.copied, cudaEventDisableTiming);
+  }
+  // (non-blocking: no implicit ordering against the legacy default stream a caller may use)
+  if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&p->copy_stream, cudaStreamNonBlocking);
   if (e != cudaSuccess) { cudaFreeHost(h); return cuda_fail(e, "pinned staging set-up"); }
   p->pinned = h;
   p->pinned_dev = (unsigned char*)dptr;
   p->blob_off = align_up(a_bytes);
   p->result_off = p->blob_off + b_bytes;
+  p->slot_stride = stride;
   p->upload_pending = false;
   return OILBIRD_OK;
 }
@@ -755,11 +780,29 @@ int oilbird_pool_append_host(oilbird_pool_t* p, const void* states, const int32_
   return oilbird_pool_append(p, d_st, d_tok, n, tag, flags, stream);
 }
 
-// Shared body of query_host (n = 0, no append) and step_host.
-static int host_step(oilbird_pool_t* p, bool do_append, const void* states, const int32_t* tokens,
-                     int64_t n, uint64_t tag, uint32_t flags, const void* q, int32_t nq,
-                     const oilbird_query_params* pr, const oilbird_query_out* out, void* stream) {
-  if (!p || !q || !out_ok(out, true)) return OILBIRD_EINVAL;
+// Result block of a slot: idx | score | cont_len | cont_tok | fired.
+struct HostResult {
+  size_t o_idx, o_score, o_len, o_tok, o_fired;
+};
+static HostResult result_layout(size_t nq, size_t k, size_t L) {
+  HostResult r;
+  r.o_idx = 0;
+  r.o_score = r.o_idx + nq * k * 4;
+  r.o_len = r.o_score + nq * k * 4;
+  r.o_tok = r.o_len + nq * k * 4;
+  r.o_fired = r.o_tok + nq * k * L * 4;
+  return r;
+}
+
+// First half of a host step (query_host: n = 0 and no append): inputs into the slot's
+// pinned blob, one upload, the kernels, the results written by the merge kernel straight
+// into the slot's mapped result block, an event behind them.  `direct` (the synchronous
+// calls only) lets a large step upload from the caller's buffers instead of packing.
+static int host_begin(oilbird_pool_t* p, bool do_append, const void* states, const int32_t* tokens,
+                      int64_t n, uint64_t tag, uint32_t flags, const void* q, int32_t nq,
+                      const oilbird_query_params* pr, int slot, void* stream) {
+  if (!p || !q || slot < 0 || slot > kHostSlots) return OILBIRD_EINVAL;
+  const bool direct = slot == kHostSlots;      // the synchronous calls' own slot
   if (n < 0 || n > p->r.max_append || (n > 0 && (!states || !tokens))) return OILBIRD_EINVAL;
   GatherParams gp;
   int rc = check_params(p, nq, pr, &gp);
@@ -767,28 +810,40 @@ static int host_step(oilbird_pool_t* p, bool do_append, const void* states, cons
   CU(cudaSetDevice(p->device));
   rc = ensure_pinned(p);
   if (rc) return rc;
+  if (p->slot[slot].busy) return refused("host slot still in flight (step_host_end not called)");
   cudaStream_t st = (cudaStream_t)stream;
   const size_t k = pr->k, L = pr->cont_len;
 
-  // inputs: one packed block, one copy (the device staging areas are adjacent in the arena)
+  // inputs: one packed block, one copy (the device staging areas are adjacent in the arena
+  // and are reused in stream order, which is why all host calls of a pool share a stream)
   const HostBlob b = blob_layout(p, n, nq, pr->exclude_tag != nullptr);
-  unsigned char* h_blob = p->pinned + p->blob_off;
-  unsigned char* d_blob = p->base + p->lay.q_stage;
+  unsigned char* h_blob = p->pinned + p->blob_off + (size_t)slot * p->slot_stride;
+  unsigned char* d_blob = p->base + (direct ? p->lay.q_stage : p->lay.pipe_stage[slot]);
   if (b.used > p->lay.stage_end - p->lay.q_stage) return OILBIRD_EINVAL;   // cannot happen
   oilbird_query_params dp = *pr;
   if (pr->exclude_tag) dp.exclude_tag = (const uint64_t*)(d_blob + b.o_ex);
-  if (b.used <= kPackLimit) {
-    // small step: pack, one copy (a copy's fixed cost outweighs the host-side memcpy)
+  if (b.used <= kPackLimit || !direct) {
+    // pack, one copy (for a small step a copy's fixed cost outweighs the host-side memcpy;
+    // a step that stays in flight must not depend on the caller's buffers)
     if (n > 0) {
       memcpy(h_blob + b.o_st, states, (size_t)n * p->r.d * 2);
       memcpy(h_blob + b.o_tok, tokens, (size_t)n * 4);
     }
     memcpy(h_blob + b.o_q, q, (size_t)nq * p->r.d * 2);
     if (pr->exclude_tag) memcpy(h_blob + b.o_ex, pr->exclude_tag, (size_t)nq * 8);
-    CU(cudaMemcpyAsync(d_blob, h_blob, b.used, cudaMemcpyHostToDevice, st));
+    if (direct) {
+      CU(cudaMemcpyAsync(d_blob, h_blob, b.used, cudaMemcpyHostToDevice, st));
+    } else {
+      // the slot's own staging block was last read by the step `end` has already waited
+      // for, so the upload need not queue behind the kernels of the step before this one
+      CU(cudaMemcpyAsync(d_blob, h_blob, b.used, cudaMemcpyHostToDevice, p->copy_stream));
+      CU(cudaEventRecord(p->slot[slot].copied, p->copy_stream));
+      CU(cudaStreamWaitEvent(st, p->slot[slot].copied, 0));
+    }
   } else {
-    // large step: the call synchronises before it returns, so the caller's buffers are
-    // uploaded directly (DMA from pinned memory; the driver stages pageable memory itself)
+    // large synchronous step: the call synchronises before it returns, so the caller's
+    // buffers are uploaded directly (DMA from pinned memory; the driver stages pageable
+    // memory itself)
     cudaError_t ce = cudaSuccess;
     if (n > 0) {
       ce = cudaMemcpyAsync(d_blob + b.o_st, states, (size_t)n * p->r.d * 2, cudaMemcpyHostToDevice, st);
@@ -805,32 +860,69 @@ static int host_step(oilbird_pool_t* p, bool do_append, const void* states, cons
     }
   }
 
-  // results: idx | score | cont_len | cont_tok | fired, written by the kernel into mapped
-  // host memory
-  const size_t o_idx = 0, o_score = o_idx + nq * k * 4, o_len = o_score + nq * k * 4,
-               o_tok = o_len + nq * k * 4, o_fired = o_tok + nq * k * L * 4;
-  unsigned char* h_out = p->pinned + p->result_off;
-  unsigned char* d_out = p->pinned_dev + p->result_off;
+  const HostResult o = result_layout(nq, k, L);
+  unsigned char* d_out = p->pinned_dev + p->result_off + (size_t)slot * p->slot_stride;
   oilbird_query_out dout;
-  dout.idx = (int32_t*)(d_out + o_idx);
-  dout.score = (float*)(d_out + o_score);
-  dout.cont_len = (int32_t*)(d_out + o_len);
-  dout.cont_tok = (int32_t*)(d_out + o_tok);
-  dout.fired = (int32_t*)(d_out + o_fired);
+  dout.idx = (int32_t*)(d_out + o.o_idx);
+  dout.score = (float*)(d_out + o.o_score);
+  dout.cont_len = (int32_t*)(d_out + o.o_len);
+  dout.cont_tok = (int32_t*)(d_out + o.o_tok);
+  dout.fired = (int32_t*)(d_out + o.o_fired);
   if (do_append)
     rc = step_impl(p, d_blob + b.o_st, (const int32_t*)(d_blob + b.o_tok), n, tag, flags,
                    d_blob + b.o_q, nq, &dp, &dout, stream);
   else
     rc = query_impl(p, d_blob + b.o_q, nq, &dp, &dout, stream, nullptr);
-  cudaError_t e = cudaStreamSynchronize(st);     // also frees the caller's buffers on error
-  if (rc) return rc;
-  if (e != cudaSuccess) return cuda_fail(e, "cudaStreamSynchronize");
-  memcpy(out->idx, h_out + o_idx, nq * k * 4);
-  memcpy(out->score, h_out + o_score, nq * k * 4);
-  memcpy(out->cont_len, h_out + o_len, nq * k * 4);
-  memcpy(out->cont_tok, h_out + o_tok, nq * k * L * 4);
-  memcpy(out->fired, h_out + o_fired, (size_t)nq * 4);
+  if (rc) {
+    cudaStreamSynchronize(st);               // also frees the caller's buffers on error
+    return rc;
+  }
+  CU(cudaEventRecord(p->slot[slot].done, st));
+  p->slot[slot].busy = true;
+  p->slot[slot].nq = nq; p->slot[slot].k = (int32_t)k; p->slot[slot].L = (int32_t)L;
   return OILBIRD_OK;
+}
+
+// Second half: wait for the slot's event, hand the results over.
+static int host_end(oilbird_pool_t* p, int slot, const oilbird_query_out* out) {
+  if (!p || slot < 0 || slot > kHostSlots || !out_ok(out, true)) return OILBIRD_EINVAL;
+  if (!p->pinned || !p->slot[slot].busy) return refused("no host step in flight in this slot");
+  CU(cudaSetDevice(p->device));
+  p->slot[slot].busy = false;
+  cudaError_t e = cudaEventSynchronize(p->slot[slot].done);
+  if (e != cudaSuccess) return cuda_fail(e, "cudaEventSynchronize");
+  const size_t nq = p->slot[slot].nq, k = p->slot[slot].k, L = p->slot[slot].L;
+  const HostResult o = result_layout(nq, k, L);
+  const unsigned char* h_out = p->pinned + p->result_off + (size_t)slot * p->slot_stride;
+  memcpy(out->idx, h_out + o.o_idx, nq * k * 4);
+  memcpy(out->score, h_out + o.o_score, nq * k * 4);
+  memcpy(out->cont_len, h_out + o.o_len, nq * k * 4);
+  memcpy(out->cont_tok, h_out + o.o_tok, nq * k * L * 4);
+  memcpy(out->fired, h_out + o.o_fired, nq * 4);
+  return OILBIRD_OK;
+}
+
+static int host_step(oilbird_pool_t* p, bool do_append, const void* states, const int32_t* tokens,
+                     int64_t n, uint64_t tag, uint32_t flags, const void* q, int32_t nq,
+                     const oilbird_query_params* pr, const oilbird_query_out* out, void* stream) {
+  if (!out_ok(out, true)) return OILBIRD_EINVAL;
+  // (a slot and a staging block of their own: steps may be in flight beside this call)
+  int rc = host_begin(p, do_append, states, tokens, n, tag, flags, q, nq, pr, kHostSlots, stream);
+  if (rc) return rc;
+  return host_end(p, kHostSlots, out);
+}
+
+int oilbird_pool_step_host_begin(oilbird_pool_t* p, const void* states, const int32_t* tokens,
+                                 int64_t n, uint64_t tag, uint32_t flags, const void* q,
+                                 int32_t nq, const oilbird_query_params* pr, int32_t slot,
+                                 void* stream) {
+  if (slot < 0 || slot >= kHostSlots) return OILBIRD_EINVAL;
+  return host_begin(p, true, states, tokens, n, tag, flags, q, nq, pr, slot, stream);
+}
+
+int oilbird_pool_step_host_end(oilbird_pool_t* p, int32_t slot, const oilbird_query_out* out) {
+  if (slot < 0 || slot >= kHostSlots) return OILBIRD_EINVAL;
+  return host_end(p, slot, out);
 }
 
 int oilbird_pool_query_host(oilbird_pool_t* p, const void* q, int32_t nq,

@@ -13,6 +13,7 @@ struct Layout {
   size_t keys, tok, trace_id, trace_end, trace_tag, trace_gbase, qn, q_valid, partial, stats;
   size_t xchg;
   size_t q_stage, ex_stage, st_stage, tok_stage, stage_end, fuse_ready, scales;
+  size_t pipe_stage[2];      // two more staging blocks [q_stage, stage_end) for host steps in flight
   size_t total;
   // OILBIRD_DEBUG_GUARDS: sentinel bytes [g_lo, g_hi) behind every array (from its last
   // byte to the next array's first), named after the array they follow
@@ -66,9 +67,15 @@ struct oilbird_pool {
   // pinned staging for host variants
   unsigned char* pinned;       // host address
   unsigned char* pinned_dev;   // the same block as the device sees it
-  size_t blob_off, result_off;
+  size_t blob_off, result_off;   // of slot 0; slot s is slot_stride bytes further on
+  size_t slot_stride;
   cudaEvent_t upload_done;
   bool upload_pending;
+  // host steps: slots 0 and 1 belong to step_host_begin .. step_host_end (inputs uploaded
+  // on copy_stream into a staging block of their own, so that the upload of one step runs
+  // under the kernels of the step before it); the last slot serves the synchronous calls
+  struct HostSlot { bool busy; int32_t nq, k, L; cudaEvent_t copied, done; } slot[3];
+  cudaStream_t copy_stream;
   // tensor-core scan: TMA tensor maps of this pool (nullptr = path unavailable)
   size_t smem_limit;
   oilbird::TcCache* tc;

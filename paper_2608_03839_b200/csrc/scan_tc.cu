@@ -467,8 +467,9 @@ __device__ __forceinline__ float kth_largest_best(const float* lmax, int q, int 
 // No load is shared or broadcast between the CTAs: each CTA's copies land in its own shared
 // memory.  The leading CTA (rank 0) issues the MMAs and owns the `full` and `tmem_empty`
 // barriers, on which both CTAs' copies and both CTAs' epilogue warps are counted; `empty`
-// and `tmem_full` exist in both CTAs and the leader's commits are counted on both.  mt is 1
-// in this form.
+// and `tmem_full` exist in both CTAs and the leader's commits are counted on both.  With
+// mt = 2 each CTA holds two key tiles per stage and the pair's macro tile is 512 rows:
+// sub-tile `sub` of tile t is rows ((t*mt + sub)*2 + rank)*128 onward.
 template <bool kPair>
 __global__ void __launch_bounds__(kTcThreads, 1)
 scan_tc_kernel(const __grid_constant__ CUtensorMap key_map,
@@ -513,7 +514,7 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap key_map,
 
   // a macro tile: mt tiles of 128 rows of this CTA, or one of each CTA of the pair; the
   // tiles of a grid are dealt out to its units (CTAs or pairs) round robin
-  const int rows_per_macro = (kPair ? 2 : mt) * kTileM;
+  const int rows_per_macro = (kPair ? 2 : 1) * mt * kTileM;
   const int n_tiles = (pv.n_rows + rows_per_macro - 1) / rows_per_macro;
   const int unit = kPair ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;
   const int n_units = kPair ? (int)(gridDim.x >> 1) : (int)gridDim.x;
@@ -582,7 +583,9 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap key_map,
             // measured at ~600 cycles per stage for the thread that makes it.
             const uint32_t full_at = smem_of_rank(&sh.full[s], 0);
             if (rank == 0) mbar_arrive_expect_tx(&sh.full[s], 2u * (uint32_t)stage_bytes);
-            tma_load_2d_pair(a_dst, &key_map, kb * kBlockK, (tile * 2 + (int)rank) * kTileM, full_at);
+            for (int sub = 0; sub < mt; ++sub)
+              tma_load_2d_pair(a_dst + sub * kATileBytes, &key_map, kb * kBlockK,
+                               ((tile * mt + sub) * 2 + (int)rank) * kTileM, full_at);
             tma_load_2d_pair(a_dst + a_bytes, &q_map, kb * kBlockK, q0 + (int)rank * b_rows, full_at);
           } else {
             mbar_arrive_expect_tx(&sh.full[s], (uint32_t)stage_bytes);
@@ -638,11 +641,19 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap key_map,
           const uint32_t acc = (uint32_t)(kb != 0);
           if (kPair) {
             const uint32_t empty0 = smem_of_rank(&sh.empty[s], 0), empty1 = smem_of_rank(&sh.empty[s], 1);
+            const uint64_t a_desc1 = a_desc + (uint64_t)(kATileBytes >> 4);     // second key tile
+            const uint32_t d_tmem1 = d_tmem + (uint32_t)n_pad;
             if (issuer) {
 #pragma unroll
               for (int kq = 0; kq < kBlockK / 16; ++kq)
                 tc_mma_bf16_pair(d_tmem, a_desc + (uint64_t)(kq * 2), b_desc + (uint64_t)(kq * 2),
                                  idesc, kq != 0 ? 1u : acc);
+              if (mt == 2) {
+#pragma unroll
+                for (int kq = 0; kq < kBlockK / 16; ++kq)
+                  tc_mma_bf16_pair(d_tmem1, a_desc1 + (uint64_t)(kq * 2), b_desc + (uint64_t)(kq * 2),
+                                   idesc, kq != 0 ? 1u : acc);
+              }
               // the stage is reusable in both CTAs once the MMAs retire
               tc_commit_pair_at(empty0);
               tc_commit_pair_at(empty1);
@@ -713,7 +724,7 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap key_map,
         // filter, now against a bound that a few rows per query pass.  The two meetings are
         // short waits that give up silently: a missing bound only means a weaker filter.
         for (int sub = 0; sub < mt; ++sub) {
-          const int row = (kPair ? tile * 2 + (int)rank : tile * mt + sub) * kTileM + lane_grp * 32 + lane;
+          const int row = (kPair ? (tile * mt + sub) * 2 + (int)rank : tile * mt + sub) * kTileM + lane_grp * 32 + lane;
           const bool row_ok = row < pv.n_rows;
           uint64_t tag = 0;
           if (exclude_tag && row_ok) tag = pv.trace_tag[pv.trace_id[row]];
@@ -763,7 +774,7 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap key_map,
       }
       epilogue_bar();
       for (int sub = 0; sub < mt; ++sub) {      // sub-tiles in row order: ties stay exact
-      const int row = (kPair ? tile * 2 + (int)rank : tile * mt + sub) * kTileM + lane_grp * 32 + lane;
+      const int row = (kPair ? (tile * mt + sub) * 2 + (int)rank : tile * mt + sub) * kTileM + lane_grp * 32 + lane;
       const bool row_ok = row < pv.n_rows;
       uint64_t tag = 0;
       if (exclude_tag && row_ok) tag = pv.trace_tag[pv.trace_id[row]];
@@ -960,17 +971,25 @@ static bool tc_fits(int n, int kk, int mt, bool global_lists, int min_stages, si
   return true;
 }
 
+constexpr int kPairMinNq = 96;   // batches above this many queries go to CTA pairs
 static TcPlan tc_plan_single(int nq, int k, int n_tiles128, int num_sms, size_t smem_limit);
 
 static TcPlan tc_plan(int nq, int k, int n_tiles128, int num_sms, size_t smem_limit) {
-  // More than 128 queries on a large pool: two CTAs per tile of 256 rows (see the kernel);
-  // each loads half of the query rows, so their number is a multiple of 32
-  if (nq > 128 && n_tiles128 >= 4 * num_sms && num_sms >= 2) {
+  // Around a hundred queries and more on a large pool: two CTAs per tile of 256 rows (see the
+  // kernel); each loads half of the query rows, so their number is a multiple of 32.  Up to
+  // 128 queries the accumulators leave room for two such tiles per query tile (a macro tile
+  // of 512 rows), which is what makes the pair pay there: C4 at nq = 128 1.58 ms against
+  // 1.635 for one CTA per two tiles, nq = 96 1.465 against 1.48, both under the power cap at
+  // ~980 MHz; one tile per pair was slower than either (1.75 ms).
+  if (nq > kPairMinNq && num_sms >= 2) {
     TcPlan p;
     p.per_pass = OILBIRD_MAX_NQ;
     p.n_pad = (nq + 31) / 32 * 32;
-    p.pair = 1; p.mt = 1; p.global_lists = 1; p.n_bufs = 2; p.stages = 0;
-    if (tc_fits(p.n_pad, list_len(k), 1, true, 3, smem_limit, &p.stages, true)) return p;
+    p.pair = 1; p.global_lists = 1; p.n_bufs = 2; p.stages = 0;
+    p.mt = 2 * 2 * p.n_pad <= 512 ? 2 : 1;
+    if (n_tiles128 >= 4 * p.mt * num_sms &&       // four macro tiles per pair and more
+        tc_fits(p.n_pad, list_len(k), p.mt, true, 3, smem_limit, &p.stages, true))
+      return p;
   }
   return tc_plan_single(nq, k, n_tiles128, num_sms, smem_limit);
 }
@@ -1055,7 +1074,7 @@ cudaError_t launch_scan_tc(TcCache* cache, const PoolView& pv, int32_t q0, int32
         plan = tc_plan_single(nq_c, k, n_tiles128, num_sms, smem_limit);
         continue;
       }
-      const int n_tiles = (n_tiles128 + 1) / 2;
+      const int n_tiles = (n_tiles128 + 2 * plan.mt - 1) / (2 * plan.mt);
       int pairs = n_tiles < pairs_fit ? n_tiles : pairs_fit;
       if (pairs > num_sms / 2) pairs = num_sms / 2;
       *n_lists = 2 * pairs;

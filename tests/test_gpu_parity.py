@@ -484,6 +484,56 @@ def test_step_host_is_append_host_plus_query_host():
     check_query(pool.query(q, pr), ora, W.to_bits(q), pr)
 
 
+def test_host_steps_in_flight_two_deep_equal_the_oracle_step_by_step():
+    """step_host_begin / step_host_end: two steps in flight, each step's answer is the oracle's
+    answer on the pool as it was after that step's own append (and before the next one's);
+    a busy slot and an idle slot are refused and change nothing."""
+    w = W.C1.scaled(n_rows=1024, nq=2)
+    pool, ora = fill_both(w, spare_rows=200)
+    g = torch.Generator().manual_seed(11)
+    pr = fixed(8, 8, theta=-2.0)
+    sizes = [8, 1, 0, 16, 8, 3, 8]
+    steps = []
+    for n in sizes:
+        st = torch.randn(n, w.d, generator=g).to(torch.bfloat16)
+        qh = torch.randn(2, w.d, generator=g).to(torch.bfloat16)
+        if n:
+            qh[0] = st[n // 2]                   # the first query repeats one of the step's own rows
+        steps.append((st, torch.randint(0, 100, (n,), generator=g, dtype=torch.int32), qh.contiguous()))
+    outs = [B.QueryOut.empty(2, 8, 8, "cpu") for _ in steps]
+    with pytest.raises(B.OilbirdError) as e:
+        pool.step_host_end(0, outs[0])           # nothing in flight yet
+    assert e.value.code == B.EINVAL
+
+    for s, (st, tk, qh) in enumerate(steps):
+        if s >= 2:
+            pool.step_host_end(s % 2, outs[s - 2])   # frees the slot this step takes
+        st_in, tk_in, qh_in = st.clone(), tk.clone(), qh.clone()
+        pool.step_host_begin(st_in, tk_in, qh_in, pr, slot=s % 2, tag=70 + s)
+        st_in.zero_(); tk_in.zero_(); qh_in.zero_()  # the caller's buffers are free after begin
+        if s == 0:
+            rows = len(pool)
+            with pytest.raises(B.OilbirdError) as e:
+                pool.step_host_begin(st, tk, qh, pr, slot=0, tag=999)   # slot 0 is busy
+            assert e.value.code == B.EINVAL and "in flight" in str(e.value) and len(pool) == rows
+    pool.step_host_end((len(steps) - 1) % 2, outs[-1])   # any order
+    pool.step_host_end((len(steps) - 2) % 2, outs[-2])
+    for s, (st, tk, qh) in enumerate(steps):
+        ora.append(W.to_bits(st), tk.numpy(), tag=70 + s)
+        check_query(outs[s], ora, W.to_bits(qh), pr)
+        if sizes[s]:
+            assert int(outs[s].idx[0, 0]) == len(ora) - sizes[s] + sizes[s] // 2
+    assert len(pool) == len(ora) == 1024 + sum(sizes)
+    # a synchronous call beside a step in flight uses the free slot
+    qh = steps[0][2]
+    pool.step_host_begin(torch.empty(0, w.d, dtype=torch.bfloat16), torch.empty(0, dtype=torch.int32),
+                         qh, pr, slot=0, new_trace=False)
+    b = pool.query_host(qh, pr)
+    a = pool.step_host_end(0, B.QueryOut.empty(2, 8, 8, "cpu"))
+    for f in ("idx", "score", "fired", "cont_len", "cont_tok"):
+        assert torch.equal(getattr(a, f), getattr(b, f))
+
+
 @pytest.mark.parametrize("nq,k", [(256, 128), (100, 128), (256, 64), (33, 100)])
 def test_largest_nq_and_k(nq, k):
     """Per-query lists for nq*k beyond shared memory: the tensor path keeps them in global
@@ -531,6 +581,36 @@ def test_pairs_of_ctas_on_batches_above_128_queries(nq, k):
     q, _ = ws.queries("cuda")
     check_query(pool.query(q, pr), ora, W.to_bits(q), pr)
     # exclusion tags: every query skips the trace that holds its best neighbour
+    best = pool.query(q, pr).cpu().idx[:, 0].numpy()
+    ex = np.array([ws.trace_tag(int(b) // ws.rows_per_trace) for b in best], dtype=np.int64)
+    pr_ex = fixed(k, 3, theta=-2.0, path=B.PATH_TENSOR, exclude_tag=torch.from_numpy(ex).cuda())
+    check_query(pool.query(q, pr_ex), ora, W.to_bits(q), pr_ex, exclude=ex.astype(np.uint64))
+    assert pool.stats()["stalled"] == 0
+
+
+@pytest.mark.parametrize("nq,k", [(97, 8), (128, 64), (120, 1)])
+def test_pairs_of_ctas_with_two_tiles_each_from_97_to_128_queries(nq, k):
+    """97 to 128 queries on a pool of at least eight tiles per SM: a pair of CTAs takes macro
+    tiles of 512 rows (two MMAs over both CTAs per query tile).  Last macro tile with one, two
+    and three of its four sub-tiles (partly) filled."""
+    for n_rows in (148 * 128 * 8 + 77, 148 * 128 * 8 + 128 + 5, 148 * 128 * 8 + 3 * 128 - 1):
+        w = W.C1.scaled(nq=nq, k=k, n_rows=n_rows, d=128, cont_len=3, n_centroids=2048,
+                        rows_per_trace=1024, seed=80 + k)
+        pool, ora = fill_both(w, max_k=128, max_nq=256)
+        q, meta = w.queries("cuda")
+        pr = fixed(k, 3, theta=-2.0, path=B.PATH_TENSOR)
+        out = pool.query(q, pr)
+        check_query(out, ora, W.to_bits(q), pr)
+        assert int(out.idx[0, 0]) == meta["planted_row"]
+        assert pool.stats()["stalled"] == 0
+        a = out.cpu()
+        for _ in range(2):
+            b = pool.query(q, pr).cpu()
+            assert torch.equal(a.idx, b.idx) and torch.equal(a.score, b.score)
+    ws = w.separated()
+    pool, ora = fill_both(ws, max_k=128, max_nq=256)
+    q, _ = ws.queries("cuda")
+    check_query(pool.query(q, pr), ora, W.to_bits(q), pr)
     best = pool.query(q, pr).cpu().idx[:, 0].numpy()
     ex = np.array([ws.trace_tag(int(b) // ws.rows_per_trace) for b in best], dtype=np.int64)
     pr_ex = fixed(k, 3, theta=-2.0, path=B.PATH_TENSOR, exclude_tag=torch.from_numpy(ex).cuda())

@@ -80,8 +80,8 @@ class ClockSampler:
 
     def __init__(self, index: int, period_s: float = 0.005):
         self.index, self.period = index, period_s
-        self.samples, self.reasons = [], set()
-        self.max_mhz = None
+        self.samples, self.reasons, self.power = [], set(), []
+        self.max_mhz = self.power_limit_w = None
         self._stop = threading.Event()
         self._thr = None
         try:
@@ -90,6 +90,10 @@ class ClockSampler:
             self.nv = pynvml
             self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
             self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+            try:                                  # (read only: nothing here changes a setting)
+                self.power_limit_w = pynvml.nvmlDeviceGetEnforcedPowerLimit(self.h) / 1e3
+            except Exception:
+                pass
         except Exception:
             self.nv = None
 
@@ -107,6 +111,10 @@ class ClockSampler:
         while not self._stop.is_set():
             try:
                 self.samples.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+                try:
+                    self.power.append(nv.nvmlDeviceGetPowerUsage(self.h) / 1e3)
+                except Exception:
+                    pass
                 try:
                     r = nv.nvmlDeviceGetCurrentClocksEventReasons(self.h)
                 except Exception:
@@ -130,7 +138,9 @@ class ClockSampler:
         reasons = sorted(r for r in self.reasons if r != "GpuIdle")
         med = float(np.median(self.samples)) if self.samples else None
         return {"sm_mhz": med, "sm_max_mhz": self.max_mhz, "reasons": reasons,
-                "samples": len(self.samples)}
+                "samples": len(self.samples),
+                "power_w": float(np.median(self.power)) if self.power else None,
+                "power_limit_w": self.power_limit_w}
 
 
 def aggregate(local_ms: float, local_units: float, world: int, device) -> tuple[float, float]:
@@ -452,8 +462,8 @@ def measure(pool, w, nq, rows_step, K, Wm, dev, world, rank, local, args, n0, ra
 
 def spare_rows(n0, rows_step, K, Wm):
     """Rows beyond the configured size that the passes of measure() may append: a growth
-    budget for each of its four passes (the pool is rebuilt, or the repeats stop, beyond it)."""
-    return 4 * max(int(MAX_GROWTH * n0), rows_step * (K + Wm)) + rows_step * (4 * Wm + 4 * K + 256)
+    budget for each of its five passes (the pool is rebuilt, or the repeats stop, beyond it)."""
+    return 5 * max(int(MAX_GROWTH * n0), rows_step * (K + Wm)) + rows_step * (5 * Wm + 5 * K + 256)
 
 
 def make_pool(w, nq, rows_step, cap_rows, local, args, extra_traces):

@@ -924,6 +924,8 @@ struct TcCache {
   alignas(64) CUtensorMap key_map;
   alignas(64) CUtensorMap q_map[OILBIRD_MAX_NQ / 16];          // [n_pad / 16 - 1]
   bool q_ok[OILBIRD_MAX_NQ / 16];
+  size_t pairs_smem;      // CTA pairs that fit the device at this much shared memory (the last
+  int pairs;              // answer; kept per pool, whose calls are the caller's to serialise)
 };
 
 TcCache* tc_cache_create(const void* keys, int64_t capacity, int32_t d, const void* qn,
@@ -931,6 +933,7 @@ TcCache* tc_cache_create(const void* keys, int64_t capacity, int32_t d, const vo
   TcCache* c = new (std::nothrow) TcCache();
   if (!c) return nullptr;
   c->qn = qn; c->qn_rows = qn_rows; c->d = d;
+  c->pairs_smem = 0; c->pairs = 0;
   for (bool& b : c->q_ok) b = false;
   if (!make_bf16_map(&c->key_map, keys, capacity, d, kTileM)) {
     delete c;
@@ -1026,11 +1029,9 @@ int tc_queries_per_pass(int nq, int k, int n_rows, int num_sms, size_t smem_limi
 }
 
 // CTA pairs that can be resident at once for a given amount of dynamic shared memory
-// (cached: the answer only depends on the device and the size).
-static int max_pairs(size_t smem, int num_sms) {
-  static size_t known_smem = 0;
-  static int known = 0;
-  if (known_smem == smem && known > 0) return known;
+// (remembered in the pool's cache: the answer only depends on the device and the size).
+static int max_pairs(TcCache* cache, size_t smem, int num_sms) {
+  if (cache->pairs_smem == smem && cache->pairs > 0) return cache->pairs;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(num_sms / 2 * 2);
   cfg.blockDim = dim3(kTcThreads);
@@ -1045,8 +1046,8 @@ static int max_pairs(size_t smem, int num_sms) {
     cudaGetLastError();
     return 0;
   }
-  known_smem = smem;
-  known = n;
+  cache->pairs_smem = smem;
+  cache->pairs = n;
   return n;
 }
 
@@ -1069,7 +1070,7 @@ cudaError_t launch_scan_tc(TcCache* cache, const PoolView& pv, int32_t q0, int32
     int tmem_cols = 32;
     while (tmem_cols < plan.n_bufs * plan.mt * n_pad) tmem_cols <<= 1;
     if (plan.pair) {
-      const int pairs_fit = max_pairs(smem, num_sms);
+      const int pairs_fit = max_pairs(cache, smem, num_sms);
       if (pairs_fit < num_sms / 2 - 2) {        // the device will not seat (nearly) every SM in a pair
         plan = tc_plan_single(nq_c, k, n_tiles128, num_sms, smem_limit);
         continue;

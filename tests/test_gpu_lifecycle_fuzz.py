@@ -83,12 +83,24 @@ def test_random_life_cycle(fmt, seed):
             new = bool(rng.random() < 0.7) or len(pool) == 0
             tag = next_tag[0]; next_tag[0] += 1
             pr = params(nq)
-            if host:
+            in_flight = host and bool(rng.random() < 0.5)   # the two-halves form of the host step
+            if in_flight:
+                out = B.QueryOut.empty(nq, pr.k, pr.cont_len, "cpu")
+                slot = int(rng.integers(0, 2))
+                pool.step_host_begin(st.cpu(), tk.cpu(), q.cpu(), pr, slot, tag=tag, new_trace=new)
+            elif host:
                 out = B.QueryOut.empty(nq, pr.k, pr.cont_len, "cpu")
                 pool.step_host(st.cpu(), tk.cpu(), q.cpu(), pr, out, tag=tag, new_trace=new)
             else:
                 out = pool.step(st, tk, q, pr, tag=tag, new_trace=new)
             ora.append(W.to_bits(st), tk.cpu().numpy(), tag=tag, new_trace=new)
+            if in_flight:
+                if len(ora) and rng.random() < 0.7:      # other lookups while the step is in flight
+                    q2 = rows(2)[0]
+                    pr2 = params(2)
+                    o2 = pool.query_host(q2.cpu(), pr2) if rng.random() < 0.5 else pool.query(q2, pr2)
+                    check_query(o2, ora, W.to_bits(q2), pr2)
+                pool.step_host_end(slot, out)
             if len(ora):
                 check_query(out, ora, W.to_bits(q), pr)
         elif op == "query":

@@ -565,6 +565,7 @@ def run_ours(args):
         if not args.no_cpu_baseline and world == 1:
             line["cpu_baseline"] = cpu_baseline(w, n0, rows_step, nq, budget_s=args.cpu_budget,
                                                 keys=args.keys)
+            line["score_check"] = score_check(w, n0, nq, dev, args)
         print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()
@@ -676,6 +677,43 @@ def cpu_baseline(w, n0, rows_step, nq, budget_s=20.0, steps=None, warmup=1, keys
             "sample": f"{n_steps} steps x {nq_s} queries, each scoring {rows} of {n0} pool rows "
                       f"(all d={w.d}) + full sort + gather; value scaled by {frac:.4g}",
             "seconds": dt, "ms_per_step": dt / n_steps * 1e3}
+
+
+def score_check(w, n0, nq, dev, args, max_rows=131072, max_q=8):
+    """Reported beside the baseline, not a gate: the scores the GPU returns against the
+    oracle's scores of the same rows, on a prefix of the workload's pool (whole traces, at
+    most `max_rows` rows) and up to `max_q` of its queries.  Both sides multiply the same
+    bf16 operands, so the difference is accumulation order; anything above 1e-4 is flagged."""
+    import oracle
+    from paper_2608_03839_b200 import binding as B
+    rows = min(n0, max_rows) // w.rows_per_trace * w.rows_per_trace or min(n0, max_rows)
+    pool = B.Pool(w.d, rows + 8, max_nq=max(nq, 1), max_k=w.k, max_traces=w.num_traces + 8,
+                  key_format=args.keys)
+    ora = oracle.OraclePool(w.d, args.keys)
+    for st, tk, tag in fill_pool(pool, w, rows, dev, keep_raw=True):   # the same arrays on both sides
+        ora.append(W.to_bits(st), tk.cpu().numpy(), tag=tag)
+    q, _ = w.queries(dev, nq=nq)
+    q = q[:max_q].contiguous()
+    pr_o = oracle.QueryParams(k=w.k, theta=-2.0, depth_mode=oracle.DEPTH_FIXED, cont_len=w.cont_len)
+    pr = B.QueryParams(k=w.k, theta=-2.0, depth_mode=B.DEPTH_FIXED, cont_len=w.cont_len,
+                       path=args.path)
+    got = pool.query(q, pr).cpu()
+    ref = ora.query(W.to_bits(q), pr_o, want_all_scores=True)
+    idx = got.idx.numpy()
+    ok = idx >= 0
+    err = np.abs(got.score.numpy()[ok].astype(np.float64) -
+                 np.take_along_axis(ref.all_scores, np.maximum(idx, 0), axis=1)[ok])
+    same_sets = int(sum(set(idx[i][ok[i]].tolist()) == set(ref.idx[i][ref.idx[i] >= 0].tolist())
+                        for i in range(idx.shape[0])))
+    pool.close()
+    return {"rows": len(ora), "queries": int(idx.shape[0]), "scores_compared": int(ok.sum()),
+            "max_abs_err": float(err.max()) if err.size else 0.0,
+            "p99_abs_err": float(np.percentile(err, 99)) if err.size else 0.0,
+            "above_1e-4": bool(err.size and err.max() > 1e-4),
+            "identical_top_k_sets": same_sets,
+            "note": "GPU score minus the oracle's score of the same row (double accumulation, "
+                    "one rounding); top-k sets may differ inside near-ties, which the parity "
+                    "tests judge under their acceptance rule"}
 
 
 def run_reference(args):

@@ -1157,6 +1157,102 @@ def run_graph(args):
     pool.close()
 
 
+def run_stream(args):
+    """C5 as the configuration states it: the pool grows from 2^20 to 2^21 rows over 4,096
+    steps, each appending one 256-row trace (the recipe's own traces 4,096 to 8,191) and
+    answering nq queries, the first of which is the row appended last plus small noise (it
+    must come back first: the rows of a step are visible to the step's own lookup).  One
+    sweep per nq; every sweep is timed as a whole, with an event every 256 steps."""
+    from paper_2608_03839_b200 import binding as B
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda:0")
+    w = W.C5
+    n0, n1, rows_step = W.C5_START_ROWS, w.n_rows, w.rows_per_trace
+    n_steps = (n1 - n0) // rows_step
+    if args.steps:                               # a shorter stream (smoke runs)
+        n_steps = min(n_steps, args.steps)
+    chunk = 256 if n_steps >= 512 else max(1, n_steps // 2)
+    t_first = n0 // rows_step
+    C = w._centroids(dev)
+    g = torch.Generator(device=dev).manual_seed(0x57EA)
+    R = torch.empty(n_steps, rows_step, w.d, dtype=torch.bfloat16, device=dev)
+    T = torch.empty(n_steps, rows_step, dtype=torch.int32, device=dev)
+    tags = []
+    for s_ in range(n_steps):
+        st, tk, tag = w.trace(t_first + s_, dev, C)
+        R[s_], T[s_] = st, tk
+        tags.append(tag)
+    planted = (R[:, -1].float() + w.query_noise * torch.randn(n_steps, w.d, generator=g, device=dev)
+               ).to(torch.bfloat16)
+    pool = B.Pool(w.d, n1 + 8, max_nq=256, max_k=w.k, max_traces=n1 // rows_step + 8,
+                  max_append=max(rows_step, 4096))
+    peaks, peak_kind = measured_peaks()
+    pr = B.QueryParams(k=w.k, theta=0.8, offset=2, depth_mode=B.DEPTH_FIXED, cont_len=w.cont_len,
+                       path=args.path)
+    sweeps = []
+    for nq in ((args.nq,) if args.nq else W.C5_NQ_SWEEP):
+        pool.reset()
+        fill_pool(pool, w, n0, dev)
+        base = torch.stack([w.queries(dev, nq=nq, step=100 + j)[0] for j in range(16)])   # fresh draws
+        Q = base[torch.arange(n_steps, device=dev) % 16].contiguous()                      # [steps, nq, d]
+        Q[:, 0] = planted
+        del base
+        out = B.QueryOut.empty(nq, w.k, w.cont_len, dev)
+        kept = {s_: B.QueryOut.empty(nq, w.k, w.cont_len, dev)
+                for s_ in list(range(0, n_steps, chunk)) + [n_steps - 1]}
+        for j in range(3):                        # warm-up lookups on the start pool (no appends)
+            pool.query(Q[j], pr, out=out)
+        torch.cuda.synchronize()
+        sampler = ClockSampler(physical_device(0))
+        sampler.start()
+        launches0 = pool.launch_count
+        ev = [torch.cuda.Event(enable_timing=True) for _ in range(n_steps // chunk + 2)]
+        ev[0].record()
+        n_ev = 1
+        for s_ in range(n_steps):
+            pool.step(R[s_], T[s_], Q[s_], pr, out=kept.get(s_, out), tag=tags[s_], new_trace=True)
+            if (s_ + 1) % chunk == 0 or s_ + 1 == n_steps:
+                ev[n_ev].record()
+                n_ev += 1
+        torch.cuda.synchronize()
+        clocks = sampler.stop()
+        ms = np.array([ev[i].elapsed_time(ev[i + 1]) for i in range(n_ev - 1)])
+        total_s = float(ms.sum()) / 1e3
+        rows_scanned = sum(n0 + (s_ + 1) * rows_step for s_ in range(n_steps))
+        gbs = rows_scanned * w.d * 2 / total_s / 1e9
+        seen = {s_: int(o.idx[0, 0]) for s_, o in kept.items()}
+        want = {s_: n0 + (s_ + 1) * rows_step - 1 for s_ in kept}
+        sweeps.append({
+            "nq": nq, "steps": n_steps, "rows_from": n0, "rows_to": len(pool), "seconds": total_s,
+            "queries_per_sec": n_steps * nq / total_s, "ms_per_step_mean": total_s / n_steps * 1e3,
+            "ms_per_step_first_chunk": float(ms[0]) / chunk, "ms_per_step_last_chunk":
+                float(ms[-1]) / (n_steps - (n_ev - 2) * chunk),
+            "key_scan_gbs": gbs, "frac_of_measured_hbm": gbs / peaks["hbm_gbs"],
+            "tensor_tflops": (2.0 * rows_scanned * w.d * ((nq + 15) // 16 * 16) / total_s / 1e12
+                              if nq > 2 else None),
+            "just_appended_row_ranked_first": seen == want, "steps_checked": len(kept),
+            "gpu_launches": int(pool.launch_count - launches0), "clocks": clocks,
+            "device_stalled_flag": pool.stats()["stalled"]})
+        del Q, kept
+        torch.cuda.empty_cache()
+    head = sweeps[0]
+    line = {"metric": METRIC, "value": head["queries_per_sec"], "unit": UNIT, "n_gpus": 1,
+            "steps": head["steps"], "warmup": 3, "ms_per_step": head["ms_per_step_mean"],
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "bf16 keys, fp32 accumulate", "data": "synthetic",
+            "config": {"workload": f"C5 stream: pool grows N={n0} -> {head['rows_to']} x d={w.d} bf16 "
+                                   f"over {head['steps']} steps of (+{rows_step} rows as a new trace, "
+                                   f"then nq queries), k={w.k}, L={w.cont_len}; headline nq={head['nq']}",
+                       "l2": "inputs exceed L2"},
+            "sweeps": sweeps, "gpu_launches": head["gpu_launches"], "clocks": head["clocks"],
+            "roofline": {"bound": "hbm", "achieved": head["key_scan_gbs"], "peak": peaks["hbm_gbs"],
+                         "unit": "GB/s", "frac": head["frac_of_measured_hbm"], "peak_kind": peak_kind,
+                         "kernel": "whole step (append + scan + merge), mean over the stream",
+                         "traffic": None}}
+    print(json.dumps(line), flush=True)
+    pool.close()
+
+
 def run_merge(args):
     """Third workload: chain post-filter + tree merge for a batch of requests (paper sizes:
     8 semantic chains of up to 48 tokens + 7 other chains into a 44-node tree, 16 of 60 nodes)."""
@@ -1309,7 +1405,7 @@ def main():
     ap.add_argument("--keys", default="bf16", choices=["bf16", "e4m3"],
                     help="stored key format: the paper's 16-bit keys, or the bounded-store "
                          "variant with 8-bit keys (FP8 E4M3 + one scale per row)")
-    ap.add_argument("--workload", default="pool", choices=["pool", "ring", "merge", "evict", "load", "index", "graph"],
+    ap.add_argument("--workload", default="pool", choices=["pool", "ring", "merge", "evict", "load", "index", "graph", "stream"],
                     help="pool: the trace-store query path (default); ring: the recycled pool; "
                          "evict: bounded store; merge: chain merge; load: bulk trace load; "
                          "index: bounded lookup cost (coarse index, with recall)")
@@ -1342,6 +1438,9 @@ def main():
         args.steps = 300 if args.steps is None else args.steps
         args.warmup = 20 if args.warmup is None else max(args.warmup, 3)
         run_index(args)
+        return
+    if args.workload == "stream":
+        run_stream(args)
         return
     if args.workload == "graph":
         args.steps = 500 if args.steps is None else args.steps

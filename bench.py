@@ -559,9 +559,19 @@ def run_ours(args):
             # the row-sharded design next to the independent pools: ONE logical pool over all
             # ranks, one all-gather of nq*k records per query
             legs = [sharded_leg(args, W.C4, W.C4.nq, min(K, 50), Wm, dev, rank, world, local)]
+    stream = None
+    if default_run and not args.no_legs and world == 1:
+        # C5 exactly as stated: the whole stream, every nq of its sweep
+        stream = {"workload": f"C5 stream: pool grows N={W.C5_START_ROWS} -> {W.C5.n_rows} x "
+                              f"d={W.C5.d} bf16 over {(W.C5.n_rows - W.C5_START_ROWS) // W.C5.rows_per_trace} "
+                              f"steps of (+{W.C5.rows_per_trace} rows as a new trace, then nq queries), "
+                              f"k={W.C5.k}, L={W.C5.cont_len}; each sweep timed as a whole",
+                  "sweeps": stream_sweeps(args, W.C5_NQ_SWEEP)}
     if rank == 0:
         if legs:
             line["legs"] = legs
+        if stream:
+            line["stream"] = stream
         if not args.no_cpu_baseline and world == 1:
             line["cpu_baseline"] = cpu_baseline(w, n0, rows_step, nq, budget_s=args.cpu_budget,
                                                 keys=args.keys)
@@ -1157,7 +1167,7 @@ def run_graph(args):
     pool.close()
 
 
-def run_stream(args):
+def stream_sweeps(args, nqs, max_steps=None):
     """C5 as the configuration states it: the pool grows from 2^20 to 2^21 rows over 4,096
     steps, each appending one 256-row trace (the recipe's own traces 4,096 to 8,191) and
     answering nq queries, the first of which is the row appended last plus small noise (it
@@ -1169,8 +1179,8 @@ def run_stream(args):
     w = W.C5
     n0, n1, rows_step = W.C5_START_ROWS, w.n_rows, w.rows_per_trace
     n_steps = (n1 - n0) // rows_step
-    if args.steps:                               # a shorter stream (smoke runs)
-        n_steps = min(n_steps, args.steps)
+    if max_steps:                                # a shorter stream (smoke runs)
+        n_steps = min(n_steps, max_steps)
     chunk = 256 if n_steps >= 512 else max(1, n_steps // 2)
     t_first = n0 // rows_step
     C = w._centroids(dev)
@@ -1190,7 +1200,7 @@ def run_stream(args):
     pr = B.QueryParams(k=w.k, theta=0.8, offset=2, depth_mode=B.DEPTH_FIXED, cont_len=w.cont_len,
                        path=args.path)
     sweeps = []
-    for nq in ((args.nq,) if args.nq else W.C5_NQ_SWEEP):
+    for nq in nqs:
         pool.reset()
         fill_pool(pool, w, n0, dev)
         base = torch.stack([w.queries(dev, nq=nq, step=100 + j)[0] for j in range(16)])   # fresh draws
@@ -1235,6 +1245,17 @@ def run_stream(args):
             "device_stalled_flag": pool.stats()["stalled"]})
         del Q, kept
         torch.cuda.empty_cache()
+    pool.close()
+    del pool, R, T, planted
+    torch.cuda.empty_cache()
+    return sweeps
+
+
+def run_stream(args):
+    w = W.C5
+    n0, rows_step = W.C5_START_ROWS, w.rows_per_trace
+    peaks, peak_kind = measured_peaks()
+    sweeps = stream_sweeps(args, (args.nq,) if args.nq else W.C5_NQ_SWEEP, args.steps)
     head = sweeps[0]
     line = {"metric": METRIC, "value": head["queries_per_sec"], "unit": UNIT, "n_gpus": 1,
             "steps": head["steps"], "warmup": 3, "ms_per_step": head["ms_per_step_mean"],
@@ -1250,7 +1271,6 @@ def run_stream(args):
                          "kernel": "whole step (append + scan + merge), mean over the stream",
                          "traffic": None}}
     print(json.dumps(line), flush=True)
-    pool.close()
 
 
 def run_merge(args):

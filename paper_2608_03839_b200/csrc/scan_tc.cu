@@ -988,11 +988,22 @@ static TcPlan tc_plan(int nq, int k, int n_tiles128, int num_sms, size_t smem_li
     TcPlan p;
     p.per_pass = OILBIRD_MAX_NQ;
     p.n_pad = (nq + 31) / 32 * 32;
-    p.pair = 1; p.global_lists = 1; p.n_bufs = 2; p.stages = 0;
-    p.mt = 2 * 2 * p.n_pad <= 512 ? 2 : 1;
-    if (n_tiles128 >= 4 * p.mt * num_sms &&       // four macro tiles per pair and more
-        tc_fits(p.n_pad, list_len(k), p.mt, true, 3, smem_limit, &p.stages, true))
-      return p;
+    p.pair = 1; p.global_lists = 1; p.stages = 0;
+    // two tiles per CTA and query tile: with both accumulator sets up to 128 columns, with
+    // one set up to 224 (what the shared query tile saves outweighs the epilogue no longer
+    // overlapping the MMAs: C5 nq = 160 3.94 -> 3.63 ms, nq = 192 4.20 -> 3.93, nq = 224
+    // 4.46 -> 4.35; at 256 columns it does not: 4.72 -> 4.71)
+    if (p.n_pad <= 224 && n_tiles128 >= 8 * num_sms) {
+      p.mt = 2;
+      p.n_bufs = 2 * 2 * p.n_pad <= 512 ? 2 : 1;
+      if (tc_fits(p.n_pad, list_len(k), 2, true, 3, smem_limit, &p.stages, true)) return p;
+    }
+    // one tile per CTA: pays above 128 columns only (below, the lone CTA with two tiles is
+    // faster: half the bytes per barrier round here)
+    if (p.n_pad > 128 && n_tiles128 >= 4 * num_sms) {
+      p.mt = 1; p.n_bufs = 2; p.stages = 0;
+      if (tc_fits(p.n_pad, list_len(k), 1, true, 3, smem_limit, &p.stages, true)) return p;
+    }
   }
   return tc_plan_single(nq, k, n_tiles128, num_sms, smem_limit);
 }

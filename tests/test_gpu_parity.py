@@ -588,11 +588,12 @@ def test_pairs_of_ctas_on_batches_above_128_queries(nq, k):
     assert pool.stats()["stalled"] == 0
 
 
-@pytest.mark.parametrize("nq,k", [(97, 8), (128, 64), (120, 1)])
-def test_pairs_of_ctas_with_two_tiles_each_from_97_to_128_queries(nq, k):
-    """97 to 128 queries on a pool of at least eight tiles per SM: a pair of CTAs takes macro
-    tiles of 512 rows (two MMAs over both CTAs per query tile).  Last macro tile with one, two
-    and three of its four sub-tiles (partly) filled."""
+@pytest.mark.parametrize("nq,k", [(97, 8), (128, 64), (120, 1), (160, 16), (224, 64), (129, 8)])
+def test_pairs_of_ctas_with_two_tiles_each_from_97_to_224_queries(nq, k):
+    """97 to 224 queries on a pool of at least eight tiles per SM: a pair of CTAs takes macro
+    tiles of 512 rows (two MMAs over both CTAs per query tile), with two accumulator sets up
+    to 128 queries and one above.  Last macro tile with one, two and three of its four
+    sub-tiles (partly) filled."""
     for n_rows in (148 * 128 * 8 + 77, 148 * 128 * 8 + 128 + 5, 148 * 128 * 8 + 3 * 128 - 1):
         w = W.C1.scaled(nq=nq, k=k, n_rows=n_rows, d=128, cont_len=3, n_centroids=2048,
                         rows_per_trace=1024, seed=80 + k)

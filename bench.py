@@ -387,7 +387,9 @@ def measure(pool, w, nq, rows_step, K, Wm, dev, world, rank, local, args, n0, ra
 
     # ---- per-step latencies and the scan kernel: passes of their own -------------------
     step_ms = total_ms / K
-    n_lat = int(min(max(K, 50), max(10, MIN_REGION_S * 1e3 / step_ms)))
+    # at least 200 timed calls (50 on the millisecond-scale C5), fewer only where half a second
+    # of steps does not hold that many
+    n_lat = int(min(max(K, 50 if w.name == "C5" else 200), max(50, MIN_REGION_S * 1e3 / step_ms)))
     make_room(2 * n_lat + 2 * Wm, new_pass=True)
     evl = [torch.cuda.Event(enable_timing=True) for _ in range(n_lat + 1)]
     evl[0].record()

@@ -12,6 +12,8 @@
 // and a block therefore takes two rows at a time.
 // Before the conversion-free fast path of normalize.cuh the kernel sat at 4.4 TB/s with the
 // conversion unit as its busiest pipe.
+#include <cuda_fp16.h>
+
 #include "common.cuh"
 #include "internal.h"
 #include "normalize.cuh"
@@ -124,7 +126,7 @@ append_bulk2_kernel(const uint16_t* __restrict__ states, const int32_t* __restri
 __global__ void __launch_bounds__(kNormThreads)
 qnorm_kernel(const uint16_t* __restrict__ q, int nq, int d, uint16_t* __restrict__ qn,
              int32_t* __restrict__ q_valid, DeviceStats* stats, float* __restrict__ xchg,
-             int n_xchg) {
+             int n_xchg, int f16_scaled) {
   pdl_enter();
   // the tensor scan's cross-CTA threshold exchange starts every call at -inf
   for (int i = blockIdx.x * kNormThreads + threadIdx.x; i < n_xchg; i += gridDim.x * kNormThreads)
@@ -139,6 +141,17 @@ qnorm_kernel(const uint16_t* __restrict__ q, int nq, int d, uint16_t* __restrict
     if (threadIdx.x == 0) {
       q_valid[r] = code == kRowNonFinite ? 0 : 1;
       if (code == kRowNonFinite) atomicAdd(&stats->nonfinite_queries, 1ull);
+    }
+    if (f16_scaled) {
+      // the normalised bf16 query as f16 scaled by 2^14, as the warp-level scan of 8-bit
+      // pools holds it (exact but for elements below 2^-31)
+      __syncthreads();
+      uint32_t* w32 = reinterpret_cast<uint32_t*>(qn + (size_t)r * d);
+      for (int i = threadIdx.x; i < d / 2; i += kNormThreads) {
+        const uint32_t w = w32[i];
+        const __half2 h = __floats2half2_rn(bf16_lo(w) * 16384.f, bf16_hi(w) * 16384.f);
+        w32[i] = *reinterpret_cast<const uint32_t*>(&h);
+      }
     }
   } else {
     uint4* dst4 = reinterpret_cast<uint4*>(qn + (size_t)r * d);
@@ -170,9 +183,9 @@ cudaError_t launch_append(const uint16_t* states, const int32_t* tokens, int64_t
 
 cudaError_t launch_qnorm(const uint16_t* q, int32_t nq, int32_t nq_pad, int32_t d, uint16_t* qn,
                          int32_t* q_valid, DeviceStats* stats, float* xchg, int32_t n_xchg,
-                         cudaStream_t st) {
+                         bool f16_scaled, cudaStream_t st) {
   return launch_pdl(qnorm_kernel, dim3(nq_pad), dim3(kNormThreads), 0, st, q, nq, d, qn, q_valid,
-                    stats, xchg, n_xchg);
+                    stats, xchg, n_xchg, f16_scaled ? 1 : 0);
 }
 
 cudaError_t preload_append_kernels() {

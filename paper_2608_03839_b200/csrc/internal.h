@@ -156,9 +156,10 @@ cudaError_t launch_to_global(const int32_t* idx, int64_t* out, int64_t n, const 
 // q_valid[r] = 0 for a query holding NaN/Inf.
 // Also fills xchg[0..n_xchg) with -inf (the tensor scan's threshold exchange, see scan_tc.cu)
 // and zeroes the kTcXchgCounters words behind them.
+// f16_scaled: qn holds f16(2^14 * bf16 value) instead (the tensor scan of 8-bit pools).
 cudaError_t launch_qnorm(const uint16_t* q, int32_t nq, int32_t nq_pad, int32_t d, uint16_t* qn,
                          int32_t* q_valid, DeviceStats* stats, float* xchg, int32_t n_xchg,
-                         cudaStream_t st);
+                         bool f16_scaled, cudaStream_t st);
 
 // Cross-CTA threshold exchange of the tensor scan: per query one published best score per
 // CTA (kTcMaxCtas slots) followed by one agreed lower bound per query.
@@ -227,14 +228,17 @@ cudaError_t launch_scan_mma(const PoolView& pv, const uint8_t* codes, const floa
 // normalised queries already sit in qn.  TcCache holds the pool's TMA tensor maps
 // (nullptr from create = tensor path unavailable).
 struct TcCache;
+// fp8: `keys` are E4M3 codes (one byte per element); launch_scan_tc then wants the rows' scales
+// and the queries in qn as f16 scaled by 2^14 (launch_qnorm's f16_scaled).
 TcCache* tc_cache_create(const void* keys, int64_t capacity, int32_t d, const void* qn,
-                         int64_t qn_rows);
+                         int64_t qn_rows, bool fp8);
 void tc_cache_destroy(TcCache* cache);
-int tc_queries_per_pass(int nq, int k, int n_rows, int num_sms, size_t smem_limit);
+int tc_queries_per_pass(int nq, int k, int n_rows, int num_sms, size_t smem_limit, bool fp8);
 cudaError_t launch_scan_tc(TcCache* cache, const PoolView& pv, int32_t q0, int32_t nq_c,
                            int32_t nq_total, int32_t k, int32_t kk, const uint64_t* exclude_tag,
                            unsigned long long* partial, DeviceStats* stats, float* xchg,
-                           int32_t num_sms, size_t smem_limit, int32_t* n_lists, cudaStream_t st);
+                           int32_t num_sms, size_t smem_limit, int32_t* n_lists,
+                           const float* scales, cudaStream_t st);
 
 // Exercises the give-up path of the two kinds of device-side wait the library has (the
 // fused append's row counter and an mbarrier of the tensor scan) on a counter nobody

@@ -247,8 +247,8 @@ int oilbird_pool_create(oilbird_pool_t** out, const oilbird_pool_config* cfg) {
     return cuda_fail(e, "cudaMemset(stats)");
   }
   p->smem_limit = prop.sharedMemPerBlockOptin;
-  p->tc = (prop.major == 10 && !r.e4m3) ? tc_cache_create(p->keys, r.capacity, r.d, p->qn,
-                                             (r.max_nq + 15) / 16 * 16)
+  p->tc = (prop.major == 10) ? tc_cache_create(p->keys, r.capacity, r.d, p->qn,
+                                             (r.max_nq + 15) / 16 * 16, r.e4m3 != 0)
                            : nullptr;
   *out = p;
   return OILBIRD_OK;
@@ -489,6 +489,9 @@ constexpr int64_t kMmaMaxKeyBytes = 2ll << 30;
 // rate: only pools that the start-up dominates (8,192 rows x 4096: 33 us against 53)
 constexpr int64_t kMma16MaxKeyBytes = 128ll << 20;
 
+// 8-bit pools: more than 8 queries go to the tcgen05 scan from this many bytes of codes on
+constexpr int64_t kFp8TensorMinBytes = 32ll << 20;
+
 static int resolve_path(const oilbird_pool* p, const oilbird_query_params* pr, int32_t nq,
                         int64_t n_rows) {
   // single-request decode streams keys through the CUDA cores; batches go to tcgen05,
@@ -500,8 +503,10 @@ static int resolve_path(const oilbird_pool* p, const oilbird_query_params* pr, i
   if (nq <= 1 || (nq == 2 && !(p->r.e4m3 && n_rows * (int64_t)p->r.d >= (128ll << 20))))
     return OILBIRD_PATH_GEMV;
   if (p->r.e4m3) {
-    // 8-bit pools have no tcgen05 scan: the warp-level tensor scan scores 8 or 16 queries
-    // per pass over the codes, the CUDA-core scan two
+    // 8-bit pools: the warp-level tensor scan scores 8 queries per pass over the codes (the
+    // CUDA-core scan two); larger batches take the tcgen05 scan, which turns the codes into
+    // f16 on the way and reads them once for the whole batch
+    if (nq > 8 && p->tc && n_rows * (int64_t)p->r.d >= kFp8TensorMinBytes) return OILBIRD_PATH_TENSOR;
     return scan_mma_tiles(p->r.d, list_len(pr->k), nq, p->smem_limit, true) ? OILBIRD_PATH_MMA
                                                                              : OILBIRD_PATH_GEMV;
   }
@@ -527,7 +532,6 @@ static int check_query(const oilbird_pool* p, const void* q, int32_t nq,
   if (rc) return rc;
   if (pr->exclude_tag && !aligned(pr->exclude_tag, 8)) return misaligned("exclude_tag");
   *path = resolve_path(p, pr, nq, n_rows);     // n_rows: the pool's size when the scan runs
-  if (*path == OILBIRD_PATH_TENSOR && p->r.e4m3) return OILBIRD_EINVAL;   // 16-bit pools only
   if (*path == OILBIRD_PATH_MMA &&
       !scan_mma_supports(p->r.d, list_len(pr->k), p->smem_limit, p->r.e4m3))
     return OILBIRD_EINVAL;
@@ -558,7 +562,7 @@ static int query_impl(oilbird_pool_t* p, const void* q, int32_t nq, const oilbir
   if (p->n_rows == 0) {
     // nothing to scan: only classify the queries (a NaN/Inf query is still counted)
     e = launch_qnorm((const uint16_t*)q, nq, nq_pad, p->r.d, p->qn, p->q_valid, p->stats,
-                     nullptr, 0, st);
+                     nullptr, 0, false, st);
     if (e != cudaSuccess) return cuda_fail(e, "qnorm kernel launch");
     p->launches += 1;
   } else {
@@ -567,7 +571,24 @@ static int query_impl(oilbird_pool_t* p, const void* q, int32_t nq, const oilbir
       e0 = p->ev[p->ev_used]; e1 = p->ev[p->ev_used + 1];
       CU(cudaEventRecord(e0, st));
     }
-    if (p->r.e4m3 && path == OILBIRD_PATH_MMA) {
+    if (path == OILBIRD_PATH_TENSOR) {
+      // (8-bit pools: the queries as f16 scaled by 2^14, the rows' scales applied to the scores)
+      e = launch_qnorm((const uint16_t*)q, nq, nq_pad, p->r.d, p->qn, p->q_valid, p->stats,
+                       p->xchg, kTcXchgFloats, p->r.e4m3 != 0, st);
+      if (e != cudaSuccess) return cuda_fail(e, "qnorm kernel launch");
+      p->launches += 1;
+      // as many queries per pass as shared memory allows next to a 3-stage ring
+      const int per_pass = tc_queries_per_pass(nq, pr->k, pv.n_rows, p->num_sms, p->smem_limit,
+                                               p->r.e4m3 != 0);
+      for (int q0 = 0; q0 < nq; q0 += per_pass) {
+        const int nq_c = nq - q0 < per_pass ? nq - q0 : per_pass;
+        e = launch_scan_tc(p->tc, pv, q0, nq_c, nq, pr->k, kk, pr->exclude_tag, p->partial,
+                           p->stats, p->xchg, p->num_sms, p->smem_limit, &n_lists,
+                           p->r.e4m3 ? p->scales : nullptr, st);
+        if (e != cudaSuccess) return cuda_fail(e, "tensor scan kernel launch");
+        p->launches += 1;
+      }
+    } else if (p->r.e4m3 && path == OILBIRD_PATH_MMA) {
       e = launch_scan_mma(pv, p->codes, p->scales, (const uint16_t*)q, nq, pr->k, kk,
                           pr->exclude_tag, p->partial, p->q_valid, p->stats, p->r.max_lists,
                           p->num_sms, p->smem_limit, &n_lists, fused, st);
@@ -591,19 +612,7 @@ static int query_impl(oilbird_pool_t* p, const void* q, int32_t nq, const oilbir
       if (e != cudaSuccess) return cuda_fail(e, "warp-level tensor scan kernel launch");
       p->launches += 1;
     } else {
-      e = launch_qnorm((const uint16_t*)q, nq, nq_pad, p->r.d, p->qn, p->q_valid, p->stats,
-                       p->xchg, kTcXchgFloats, st);
-      if (e != cudaSuccess) return cuda_fail(e, "qnorm kernel launch");
-      p->launches += 1;
-      // as many queries per pass as shared memory allows next to a 3-stage ring
-      const int per_pass = tc_queries_per_pass(nq, pr->k, pv.n_rows, p->num_sms, p->smem_limit);
-      for (int q0 = 0; q0 < nq; q0 += per_pass) {
-        const int nq_c = nq - q0 < per_pass ? nq - q0 : per_pass;
-        e = launch_scan_tc(p->tc, pv, q0, nq_c, nq, pr->k, kk, pr->exclude_tag, p->partial,
-                           p->stats, p->xchg, p->num_sms, p->smem_limit, &n_lists, st);
-        if (e != cudaSuccess) return cuda_fail(e, "tensor scan kernel launch");
-        p->launches += 1;
-      }
+      return OILBIRD_EINVAL;                   // (resolve_path names one of the scans above)
     }
     if (e0) {
       CU(cudaEventRecord(e1, st));

@@ -83,12 +83,14 @@
 namespace oilbird {
 
 constexpr int kTcThreads = 192;
+constexpr int kTcThreadsFp8 = 320;     // ... plus four warps that turn codes into f16 (8-bit pools)
 constexpr int kTileM = 128;            // key rows per tile = TMEM lanes
 // bf16 elements per k-block = one 128-byte swizzle row.  (32-element blocks with the 64-byte
 // swizzle were measured too: more, finer ring stages, but every 128-byte line is then
 // requested twice and the scan runs 30-40 % slower at every nq.)
 constexpr int kBlockK = 64;
 constexpr int kATileBytes = kTileM * kBlockK * 2;   // 16 KB
+constexpr int kCodeTileBytes = kTileM * kBlockK;    // the same tile as E4M3 codes: 8 KB
 constexpr int kColsPerRound = 16;      // score columns filtered between two drains
 constexpr int kQueueCap = kTileM * kColsPerRound;
 constexpr int kMaxStages = 8;
@@ -287,6 +289,17 @@ __host__ __device__ inline uint32_t umma_idesc_bf16(int n, int m = kTileM) {
          ((uint32_t)(m >> 4) << 24);
 }
 
+// The same with f16 operands (8-bit pools: an E4M3 code is an f16 number exactly).
+__host__ __device__ inline uint32_t umma_idesc_f16(int n, int m = kTileM) {
+  return (1u << 4) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
+}
+// two E4M3 codes (low 16 bits) -> f16x2, first code in the low half
+__device__ __forceinline__ uint32_t e4m3x2_to_f16x2(uint32_t two_codes) {
+  uint32_t h2;
+  asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(h2) : "h"((unsigned short)two_codes));
+  return h2;
+}
+
 // Order-preserving map float -> unsigned (and back), so that a warp-wide maximum of scores is
 // one redux instruction; 0 is below every score.
 __device__ __forceinline__ uint32_t score_to_ord(float s) {
@@ -315,6 +328,7 @@ __device__ __forceinline__ void rendezvous_wait(const unsigned* counter, unsigne
 // ------------------------------------------------------------- per-query lists ---
 struct TcShared {
   uint64_t full[kMaxStages], empty[kMaxStages], tmem_full[2], tmem_empty[2], drain;
+  uint64_t cvt[kMaxStages];     // 8-bit pools: the stage's codes have been turned into f16
   uint32_t tmem_base;
   int abort_flag;
   int epi_go;
@@ -470,13 +484,26 @@ __device__ __forceinline__ float kth_largest_best(const float* lmax, int q, int 
 // and `tmem_full` exist in both CTAs and the leader's commits are counted on both.  With
 // mt = 2 each CTA holds two key tiles per stage and the pair's macro tile is 512 rows:
 // sub-tile `sub` of tile t is rows ((t*mt + sub)*2 + rank)*128 onward.
-template <bool kPair>
-__global__ void __launch_bounds__(kTcThreads, 1)
+//
+// kFp8 (lone CTAs only): the pool holds E4M3 codes and one fp32 scale per row.  The tensor
+// core takes 16-bit operands, so a stage's codes (8 KB per tile, loaded by TMA without
+// swizzle) are turned into the f16 tile the MMA reads by four more warps: 16 codes per
+// 16-byte shared-memory load, `cvt.rn.f16x2.e4m3x2` (exact), two 16-byte stores into the
+// 128-byte-swizzled layout a TMA load would have produced, a proxy fence, and an arrival on
+// the stage's `cvt` barrier, which is what the MMA warp waits for in place of `full`.  The
+// queries arrive as f16 scaled by 2^14 (see the query preparation); a row's scale and the
+// 2^-14 are applied to its scores as they leave TMEM.  HBM carries half the bytes of a
+// 16-bit pool; shared memory carries more (codes in and out, f16 in and out), which is what
+// bounds this form.
+template <bool kPair, bool kFp8 = false>
+__global__ void __launch_bounds__(kFp8 ? kTcThreadsFp8 : kTcThreads, 1)
 scan_tc_kernel(const __grid_constant__ CUtensorMap key_map,
                const __grid_constant__ CUtensorMap q_map, PoolView pv, int q0, int nq_c,
                int nq_total, int n_pad, int k, int kk, int n_stages, int tmem_cols, int mt,
                int n_bufs, int global_lists, const uint64_t* __restrict__ exclude_tag,
-               u64* __restrict__ partial, DeviceStats* stats, float* xchg) {
+               u64* __restrict__ partial, DeviceStats* stats, float* xchg,
+               const float* __restrict__ scales) {
+  static_assert(!(kPair && kFp8), "8-bit pools run lone CTAs");
   extern __shared__ __align__(1024) unsigned char smem_raw[];
   __shared__ TcShared sh;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -484,8 +511,9 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap key_map,
   const int n_ctas = kPair ? 2 : 1;
   const int b_rows = n_pad / n_ctas;                       // query rows this CTA loads
   const int a_bytes = mt * kATileBytes;
-  const int stage_bytes = a_bytes + b_rows * kBlockK * 2;
-  // dynamic shared memory: [stages][mt key tiles | query tile] | lists | queue | state
+  const int raw_off = a_bytes + b_rows * kBlockK * 2;       // 8-bit pools: the stage's codes
+  const int stage_bytes = raw_off + (kFp8 ? mt * kCodeTileBytes : 0);
+  // dynamic shared memory: [stages][mt key tiles | query tile | codes] | lists | queue | state
   unsigned char* base = (unsigned char*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
   unsigned char* ring = base;
   unsigned char* list_mem = ring + (size_t)n_stages * stage_bytes;              // [nq_c][kk]
@@ -525,6 +553,7 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap key_map,
     for (int s = 0; s < n_stages; ++s) {
       mbar_init(&sh.full[s], 1);
       mbar_init(&sh.empty[s], 1);
+      mbar_init(&sh.cvt[s], 4);
     }
     for (int b = 0; b < 2; ++b) {
       mbar_init(&sh.tmem_full[b], 1);
@@ -553,12 +582,12 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap key_map,
   tc_fence_after();
   const uint32_t tmem_base = sh.tmem_base;
   pdl_enter();   // appended rows, normalised queries, exclusion tags; set-up above overlapped
-  for (int i = threadIdx.x; i < n_pad; i += kTcThreads) {
+  for (int i = threadIdx.x; i < n_pad; i += (int)blockDim.x) {
     thr_s[i] = i < nq_c ? -INFINITY : INFINITY;        // padded columns never pass the filter
     s_qmax[i] = 0u;
     s_ex[i] = (exclude_tag && i < nq_c) ? exclude_tag[q0 + i] : 0;
   }
-  for (int i = threadIdx.x; i < nq_c * kk; i += kTcThreads) lists.store(i / kk, i % kk, 0);
+  for (int i = threadIdx.x; i < nq_c * kk; i += (int)blockDim.x) lists.store(i / kk, i % kk, 0);
   __syncthreads();
 
   if (warp == 0) {
@@ -587,6 +616,12 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap key_map,
               tma_load_2d_pair(a_dst + sub * kATileBytes, &key_map, kb * kBlockK,
                                ((tile * mt + sub) * 2 + (int)rank) * kTileM, full_at);
             tma_load_2d_pair(a_dst + a_bytes, &q_map, kb * kBlockK, q0 + (int)rank * b_rows, full_at);
+          } else if (kFp8) {
+            mbar_arrive_expect_tx(&sh.full[s], (uint32_t)(stage_bytes - a_bytes));
+            for (int sub = 0; sub < mt; ++sub)    // codes: 64 bytes x 128 rows, rows as they are
+              tma_load_2d(a_dst + raw_off + sub * kCodeTileBytes, &key_map, kb * kBlockK,
+                          (tile * mt + sub) * kTileM, &sh.full[s]);
+            tma_load_2d(a_dst + a_bytes, &q_map, kb * kBlockK, q0, &sh.full[s]);
           } else {
             mbar_arrive_expect_tx(&sh.full[s], (uint32_t)stage_bytes);
             for (int sub = 0; sub < mt; ++sub)    // rows past the pool's capacity read as zero
@@ -619,7 +654,7 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap key_map,
     // tcgen05.mma takes its operands from.
     if (rank == 0) {
       const bool issuer = elect_one();
-      const uint32_t idesc = umma_idesc_bf16(n_pad, kPair ? 2 * kTileM : kTileM);
+      const uint32_t idesc = kFp8 ? umma_idesc_f16(n_pad) : umma_idesc_bf16(n_pad, kPair ? 2 * kTileM : kTileM);
       uint32_t it = 0, iter = 0;
       bool ok = true;
       for (int tile = unit; tile < n_tiles && ok; tile += n_units, ++iter) {
@@ -633,7 +668,10 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap key_map,
         const uint32_t d_tmem = tmem_base + buf * (uint32_t)(mt * n_pad);
         for (int kb = 0; kb < n_kb; ++kb, ++it) {
           const int s = it % n_stages;
-          if (!warp_mbar_wait(&sh.full[s], (it / n_stages) & 1u, abort_flag, stats)) { ok = false; break; }
+          if (!warp_mbar_wait(kFp8 ? &sh.cvt[s] : &sh.full[s], (it / n_stages) & 1u, abort_flag, stats)) {
+            ok = false;
+            break;
+          }
           tc_fence_after();
           const uint32_t a_addr = smem_u32(ring + (size_t)s * stage_bytes);
           const uint64_t a_desc = umma_desc_sw128(a_addr);
@@ -697,6 +735,39 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap key_map,
       }
       __syncwarp();
     }
+  } else if (kFp8 && warp >= 6) {
+    // ===================================================== codes -> f16 ==========
+    // thread ct takes the 16-byte pieces ct, ct + 128, ... of a stage's codes (consecutive
+    // lanes read consecutive pieces: no bank conflict); piece g is codes 16 (g % 4) onward of
+    // row g / 4, i.e. the row's 16-byte f16 chunks 2 (g % 4) and 2 (g % 4) + 1, which the
+    // 128-byte swizzle keeps at chunk position (chunk ^ (row % 8)) of the row's 128 bytes
+    const int ct = threadIdx.x - 192;
+    uint32_t it = 0;
+    bool ok = true;
+    for (int tile = unit; tile < n_tiles && ok; tile += n_units) {
+      for (int kb = 0; kb < n_kb; ++kb, ++it) {
+        const int s = it % n_stages;
+        if (!mbar_wait(&sh.full[s], (it / n_stages) & 1u, abort_flag, stats)) { ok = false; break; }
+        unsigned char* a_dst = ring + (size_t)s * stage_bytes;
+        const uint4* raw = reinterpret_cast<const uint4*>(a_dst + raw_off);
+        for (int g = ct; g < mt * (kCodeTileBytes / 16); g += 128) {
+          const uint4 c = raw[g];
+          const int row_all = g >> 2, c4 = g & 3;           // row over the stage's tiles
+          unsigned char* row_dst = a_dst + (size_t)row_all * 128;
+          const int sw = row_all & 7;
+          const uint4 lo = make_uint4(e4m3x2_to_f16x2(c.x), e4m3x2_to_f16x2(c.x >> 16),
+                                      e4m3x2_to_f16x2(c.y), e4m3x2_to_f16x2(c.y >> 16));
+          const uint4 hi = make_uint4(e4m3x2_to_f16x2(c.z), e4m3x2_to_f16x2(c.z >> 16),
+                                      e4m3x2_to_f16x2(c.w), e4m3x2_to_f16x2(c.w >> 16));
+          *reinterpret_cast<uint4*>(row_dst + (((2 * c4) ^ sw) << 4)) = lo;
+          *reinterpret_cast<uint4*>(row_dst + (((2 * c4 + 1) ^ sw) << 4)) = hi;
+        }
+        // the tile was written through the generic proxy; the MMA reads it through the async one
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&sh.cvt[s]);
+      }
+    }
   } else {
     // ===================================================== epilogue ==============
     const int ew = warp - 2;                    // 0..3: which queries this warp owns in drains
@@ -730,9 +801,15 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap key_map,
           if (exclude_tag && row_ok) tag = pv.trace_tag[pv.trace_id[row]];
           const uint32_t t_row = tmem_base + ((uint32_t)(lane_grp * 32) << 16) +
                                  (uint32_t)sub * (uint32_t)n_pad;               // buffer 0
+          // 8-bit pools: score = scale(row) * sum / 2^14 (the queries' scaling taken back)
+          const float rs = (kFp8 && row_ok) ? scales[row] * (1.f / 16384.f) : 0.f;
           for (int c0 = 0; c0 < n_pad; c0 += kColsPerRound) {
             float v[kColsPerRound];
             tc_ld16(t_row + (uint32_t)c0, v);
+            if (kFp8) {
+#pragma unroll
+              for (int j = 0; j < kColsPerRound; ++j) v[j] *= rs;
+            }
             uint32_t mine = 0;
 #pragma unroll
             for (int j = 0; j < kColsPerRound; ++j) {
@@ -780,9 +857,14 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap key_map,
       if (exclude_tag && row_ok) tag = pv.trace_tag[pv.trace_id[row]];
       const uint32_t t_row = tmem_base + ((uint32_t)(lane_grp * 32) << 16) +
                              (buf * (uint32_t)mt + (uint32_t)sub) * (uint32_t)n_pad;
+      const float rs = (kFp8 && row_ok) ? scales[row] * (1.f / 16384.f) : 0.f;
       for (int c0 = 0; c0 < n_pad; c0 += kColsPerRound) {
         float v[kColsPerRound];
         tc_ld16(t_row + (uint32_t)c0, v);
+        if (kFp8) {
+#pragma unroll
+          for (int j = 0; j < kColsPerRound; ++j) v[j] *= rs;
+        }
         if (sub == mt - 1 && c0 + kColsPerRound >= n_pad) {
           // all of this macro tile's scores have been read: hand the accumulators back
           tc_fence_before();
@@ -914,6 +996,21 @@ static bool make_bf16_map(CUtensorMap* map_out, const void* base, int64_t rows, 
   return r == CUDA_SUCCESS;
 }
 
+// Tensor map over a row-major matrix of E4M3 codes [rows, d]; box = 64 codes x 128 rows as they
+// are (no swizzle: the codes are read back with plain loads), out-of-range codes read as zero.
+static bool make_code_map(CUtensorMap* map_out, const void* base, int64_t rows, int32_t d) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  cuuint64_t dims[2] = {(cuuint64_t)d, (cuuint64_t)rows};
+  cuuint64_t strides[1] = {(cuuint64_t)d};
+  cuuint32_t box[2] = {(cuuint32_t)kBlockK, (cuuint32_t)kTileM};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult r = fn(map_out, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, (void*)base, dims, strides, box,
+                  estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
+                  CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS;
+}
+
 // Tensor maps of one pool: keys (fixed at creation: the map covers the whole capacity,
 // rows past the current size are masked in the epilogue) and, made on first use, the
 // normalised-query buffer for every box height.
@@ -921,6 +1018,7 @@ struct TcCache {
   const void* qn;
   int64_t qn_rows;
   int32_t d;
+  bool fp8;               // the keys are E4M3 codes (key_map covers bytes, the queries are f16)
   alignas(64) CUtensorMap key_map;
   alignas(64) CUtensorMap q_map[OILBIRD_MAX_NQ / 16];          // [n_pad / 16 - 1]
   bool q_ok[OILBIRD_MAX_NQ / 16];
@@ -929,13 +1027,14 @@ struct TcCache {
 };
 
 TcCache* tc_cache_create(const void* keys, int64_t capacity, int32_t d, const void* qn,
-                         int64_t qn_rows) {
+                         int64_t qn_rows, bool fp8) {
   TcCache* c = new (std::nothrow) TcCache();
   if (!c) return nullptr;
-  c->qn = qn; c->qn_rows = qn_rows; c->d = d;
+  c->qn = qn; c->qn_rows = qn_rows; c->d = d; c->fp8 = fp8;
   c->pairs_smem = 0; c->pairs = 0;
   for (bool& b : c->q_ok) b = false;
-  if (!make_bf16_map(&c->key_map, keys, capacity, d, kTileM)) {
+  if (!(fp8 ? make_code_map(&c->key_map, keys, capacity, d)
+            : make_bf16_map(&c->key_map, keys, capacity, d, kTileM))) {
     delete c;
     return nullptr;
   }
@@ -964,8 +1063,9 @@ static size_t tc_fixed_smem(int nq_c, int n_pad, int kk, bool global_lists) {
 struct TcPlan { int per_pass, n_pad, mt, stages, n_bufs, global_lists, pair; };
 
 static bool tc_fits(int n, int kk, int mt, bool global_lists, int min_stages, size_t smem_limit,
-                    int* stages, bool pair = false) {
-  const size_t stage = (size_t)mt * kATileBytes + (size_t)(pair ? n / 2 : n) * kBlockK * 2;
+                    int* stages, bool pair = false, bool fp8 = false) {
+  const size_t stage = (size_t)mt * (kATileBytes + (fp8 ? kCodeTileBytes : 0)) +
+                       (size_t)(pair ? n / 2 : n) * kBlockK * 2;
   // static shared memory (barriers etc.) is padded to the 1024-byte alignment of the ring
   const size_t fixed = tc_fixed_smem(n, n, kk, global_lists) + 1024 + 256;
   if (fixed + (size_t)min_stages * stage > smem_limit) return false;
@@ -975,9 +1075,12 @@ static bool tc_fits(int n, int kk, int mt, bool global_lists, int min_stages, si
 }
 
 constexpr int kPairMinNq = 96;   // batches above this many queries go to CTA pairs
-static TcPlan tc_plan_single(int nq, int k, int n_tiles128, int num_sms, size_t smem_limit);
+static TcPlan tc_plan_single(int nq, int k, int n_tiles128, int num_sms, size_t smem_limit,
+                             bool fp8 = false);
 
-static TcPlan tc_plan(int nq, int k, int n_tiles128, int num_sms, size_t smem_limit) {
+static TcPlan tc_plan(int nq, int k, int n_tiles128, int num_sms, size_t smem_limit,
+                      bool fp8 = false) {
+  if (fp8) return tc_plan_single(nq, k, n_tiles128, num_sms, smem_limit, true);   // lone CTAs only
   // Around a hundred queries and more on a large pool: two CTAs per tile of 256 rows (see the
   // kernel); each loads half of the query rows, so their number is a multiple of 32.  Up to
   // 128 queries the accumulators leave room for two such tiles per query tile (a macro tile
@@ -1008,7 +1111,8 @@ static TcPlan tc_plan(int nq, int k, int n_tiles128, int num_sms, size_t smem_li
   return tc_plan_single(nq, k, n_tiles128, num_sms, smem_limit);
 }
 
-static TcPlan tc_plan_single(int nq, int k, int n_tiles128, int num_sms, size_t smem_limit) {
+static TcPlan tc_plan_single(int nq, int k, int n_tiles128, int num_sms, size_t smem_limit,
+                             bool fp8) {
   const int kk = list_len(k);
   TcPlan p;
   p.per_pass = OILBIRD_MAX_NQ;
@@ -1024,19 +1128,20 @@ static TcPlan tc_plan_single(int nq, int k, int n_tiles128, int num_sms, size_t 
   // the lists in L2 beats a shallower or one-tile ring with the lists on chip (nq = 128,
   // k = 64 at d = 8192: 2.61 ms against 3.11).
   const bool many_tiles = n_tiles128 >= 2 * num_sms;
-  const bool two = many_tiles && 2 * 2 * n_pad <= 512 && tc_fits(n_pad, kk, 2, true, 3, smem_limit, &st);
+  const bool two = many_tiles && 2 * 2 * n_pad <= 512 &&
+                   tc_fits(n_pad, kk, 2, true, 3, smem_limit, &st, false, fp8);
   const int mt = two ? 2 : 1;
-  const bool gl = !tc_fits(n_pad, kk, mt, false, kTcMinSmemStages, smem_limit, &st);
+  const bool gl = !tc_fits(n_pad, kk, mt, false, kTcMinSmemStages, smem_limit, &st, false, fp8);
   p.global_lists = gl ? 1 : 0;
   p.mt = mt;
   p.stages = 0;
-  tc_fits(n_pad, kk, p.mt, gl, 2, smem_limit, &p.stages);
+  tc_fits(n_pad, kk, p.mt, gl, 2, smem_limit, &p.stages, false, fp8);
   p.n_bufs = 2 * p.mt * n_pad <= 512 ? 2 : 1;
   return p;
 }
 
-int tc_queries_per_pass(int nq, int k, int n_rows, int num_sms, size_t smem_limit) {
-  return tc_plan(nq, k, (n_rows + kTileM - 1) / kTileM, num_sms, smem_limit).per_pass;
+int tc_queries_per_pass(int nq, int k, int n_rows, int num_sms, size_t smem_limit, bool fp8) {
+  return tc_plan(nq, k, (n_rows + kTileM - 1) / kTileM, num_sms, smem_limit, fp8).per_pass;
 }
 
 // CTA pairs that can be resident at once for a given amount of dynamic shared memory
@@ -1065,12 +1170,15 @@ static int max_pairs(TcCache* cache, size_t smem, int num_sms) {
 cudaError_t launch_scan_tc(TcCache* cache, const PoolView& pv, int32_t q0, int32_t nq_c,
                            int32_t nq_total, int32_t k, int32_t kk, const uint64_t* exclude_tag,
                            unsigned long long* partial, DeviceStats* stats, float* xchg,
-                           int32_t num_sms, size_t smem_limit, int32_t* n_lists, cudaStream_t st) {
+                           int32_t num_sms, size_t smem_limit, int32_t* n_lists,
+                           const float* scales, cudaStream_t st) {
   const int n_tiles128 = (pv.n_rows + kTileM - 1) / kTileM;
-  TcPlan plan = tc_plan(nq_c, k, n_tiles128, num_sms, smem_limit);
+  const bool fp8 = cache->fp8;
+  if (fp8 != (scales != nullptr)) return cudaErrorInvalidValue;
+  TcPlan plan = tc_plan(nq_c, k, n_tiles128, num_sms, smem_limit, fp8);
   for (int attempt = 0; attempt < 2; ++attempt) {
     const int n_pad = plan.n_pad;
-    const size_t stage = (size_t)plan.mt * kATileBytes +
+    const size_t stage = (size_t)plan.mt * (kATileBytes + (fp8 ? kCodeTileBytes : 0)) +
                          (size_t)(plan.pair ? n_pad / 2 : n_pad) * kBlockK * 2;
     const size_t fixed = tc_fixed_smem(nq_c, n_pad, kk, plan.global_lists != 0);
     if (plan.stages < 2) return cudaErrorInvalidConfiguration;
@@ -1105,16 +1213,21 @@ cudaError_t launch_scan_tc(TcCache* cache, const PoolView& pv, int32_t q0, int32
       return cudaLaunchKernelEx(&cfg, scan_tc_kernel<true>, cache->key_map, *q_map, pv, (int)q0,
                                 (int)nq_c, (int)nq_total, n_pad, (int)k, (int)kk, plan.stages,
                                 tmem_cols, plan.mt, plan.n_bufs, plan.global_lists, exclude_tag,
-                                (u64*)partial, stats, xchg);
+                                (u64*)partial, stats, xchg, (const float*)nullptr);
     }
     const int n_tiles = (n_tiles128 + plan.mt - 1) / plan.mt;
     int grid = n_tiles < num_sms ? n_tiles : num_sms;
     if (grid < 1) grid = 1;
     *n_lists = grid;
+    if (fp8)
+      return launch_pdl(scan_tc_kernel<false, true>, dim3(grid), dim3(kTcThreadsFp8), smem, st,
+                        cache->key_map, *q_map, pv, q0, nq_c, nq_total, n_pad, k, kk, plan.stages,
+                        tmem_cols, plan.mt, plan.n_bufs, plan.global_lists, exclude_tag, partial,
+                        stats, xchg, scales);
     return launch_pdl(scan_tc_kernel<false>, dim3(grid), dim3(kTcThreads), smem, st,
                       cache->key_map, *q_map, pv, q0, nq_c, nq_total, n_pad, k, kk, plan.stages,
                       tmem_cols, plan.mt, plan.n_bufs, plan.global_lists, exclude_tag, partial, stats,
-                      xchg);
+                      xchg, (const float*)nullptr);
   }
   return cudaErrorInvalidConfiguration;
 }
@@ -1149,6 +1262,7 @@ cudaError_t launch_stall_selftest(const unsigned long long* ready, DeviceStats* 
 cudaError_t preload_scan_tc_kernels() {
   cudaError_t e = preload_kernel(scan_tc_kernel<false>, true);
   if (e == cudaSuccess) e = preload_kernel(scan_tc_kernel<true>, true);
+  if (e == cudaSuccess) e = preload_kernel(scan_tc_kernel<false, true>, true);
   return e != cudaSuccess ? e : preload_kernel(stall_selftest_kernel);
 }
 

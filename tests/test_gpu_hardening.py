@@ -62,12 +62,10 @@ def test_misaligned_pointers_are_refused_before_any_launch():
     assert out.idx[:, 0].tolist() == [3, 4]
 
 
-@pytest.mark.parametrize("fmt,path,d,k", [("e4m3", B.PATH_TENSOR, 256, 8),    # no tcgen05 scan for 8-bit keys
+@pytest.mark.parametrize("fmt,path,d,k", [("e4m3", B.PATH_MMA, 384, 8),       # 8-bit warp-level scan: d a multiple of 256
                                           ("bf16", B.PATH_MMA, 200, 8),       # d not a multiple of 128
                                           ("bf16", B.PATH_MMA, 256, 100)])    # k beyond the warp-level scan
 def test_a_refused_step_appends_nothing(fmt, path, d, k):
-    if fmt == "e4m3":
-        d = 256
     g = torch.Generator(device="cuda").manual_seed(6)
     pool = B.Pool(d, 400, key_format=fmt, max_k=128)
     st = torch.randn(64, d, generator=g, device="cuda").to(torch.bfloat16)

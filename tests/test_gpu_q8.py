@@ -150,9 +150,9 @@ def test_limits_of_8bit_pools():
     st = torch.randn(40, 64, device="cuda").to(torch.bfloat16)
     pool.append(st, torch.arange(40, dtype=torch.int32, device="cuda"))
     pr = fixed(4, 4)
-    pr.path = B.PATH_TENSOR
+    pr.path = 7
     with pytest.raises(B.OilbirdError):
-        pool.query(st[:4].contiguous(), pr)                      # no tensor-core scan for 8-bit keys
+        pool.query(st[:4].contiguous(), pr)                      # no such scan
     keys, tok, tid = pool.read_rows()
     assert keys is None and tok.shape == (40,)
     pool16 = B.Pool(64, 256)
@@ -327,3 +327,100 @@ def test_mma_scan_appends_the_rows_of_a_step_itself():
     assert np.array_equal(scales.view(np.uint32), ora.scales.view(np.uint32))
     _, tok, tid = pool.read_rows()
     assert np.array_equal(tok, ora.tokens) and np.array_equal(tid, ora.trace_ids)
+
+
+# ---- tcgen05 scan of 8-bit pools: codes turned into f16 inside the kernel ---------------
+
+@pytest.mark.parametrize("d", [64, 256, 1024, 4096])
+def test_tensor_scan_closed_form_pool_scores_are_exact(d):
+    # +-1 rows (codes +-448) and +-1 queries: f16 products and their sums are exact, so the
+    # scan must return the oracle's scores, order and ties bit for bit
+    rng = np.random.default_rng(d + 1)
+    n = 700
+    rows = rng.choice([-1.0, 1.0], size=(n, d)).astype(np.float32)
+    q = rng.choice([-1.0, 1.0], size=(12, d)).astype(np.float32)
+    rows[5] = q[0]; rows[300] = q[0]; rows[699] = q[0]
+    rows[17] = -q[1]
+    pool = B.Pool(d, n, max_nq=16, key_format="e4m3")
+    ora = OraclePool(d, "e4m3")
+    rb = oracle.f32_to_bf16_bits(rows)
+    tok = np.arange(n, dtype=np.int32)
+    pool.append(bits_to_dev(rb), torch.from_numpy(tok).cuda(), tag=1)
+    ora.append(rb, tok, tag=1)
+    qb = oracle.f32_to_bf16_bits(q)
+    pr = fixed(8, 2, theta=-2.0, path=B.PATH_TENSOR)
+    l0 = pool.launch_count
+    out = pool.query(bits_to_dev(qb), pr).cpu()
+    assert pool.launch_count - l0 == 3                       # query preparation, scan, merge
+    ref = ora.query(qb, oracle.QueryParams(k=8, theta=-2.0, depth_mode=oracle.DEPTH_FIXED, cont_len=2))
+    assert out.idx.numpy().tolist() == ref.idx.tolist()
+    assert np.array_equal(out.score.numpy(), ref.score)
+    assert out.idx[0, :3].tolist() == [5, 300, 699]
+    assert pool.stats()["stalled"] == 0
+
+
+@pytest.mark.parametrize("nq,k", [(3, 8), (9, 8), (16, 64), (64, 16), (100, 8), (256, 64), (33, 128)])
+def test_tensor_scan_matches_oracle_and_the_other_scans(nq, k):
+    w = W.C1.scaled(n_rows=6000, nq=nq, d=512)
+    pool, ora = fill_both(w, key_format="e4m3", max_k=128, max_nq=256)
+    q, _ = w.queries("cuda", nq=nq)
+    for theta in (0.8, -2.0):
+        pr = fixed(k, 8, theta=theta, path=B.PATH_TENSOR)
+        out = pool.query(q, pr)
+        check_query(out, ora, W.to_bits(q), pr)
+        if k <= 64:
+            ref = pool.query(q, fixed(k, 8, theta=theta, path=B.PATH_MMA))
+            assert torch.allclose(out.score, ref.score, atol=2e-5, rtol=0)
+        again = pool.query(q, pr).cpu()                      # bit-identical from run to run
+        assert torch.equal(out.cpu().idx, again.idx) and torch.equal(out.cpu().score, again.score)
+    assert pool.stats()["stalled"] == 0
+
+
+@pytest.mark.parametrize("n_rows,d", [(148 * 128 * 2 + 77, 256), (148 * 128 * 3 + 128 + 5, 208),
+                                      (1, 64), (127, 128), (129, 1024), (5000, 8192)])
+def test_tensor_scan_tile_shapes_widths_and_exclusion(n_rows, d):
+    # two key tiles per query tile (from two tiles per SM on), a ragged last tile, a width that
+    # is not a multiple of the k-block (the codes beyond it read as zero), one row, wide rows
+    w = W.C1.scaled(n_rows=max(n_rows, 2100), nq=24, k=16, d=d, cont_len=4, rows_per_trace=700,
+                    n_centroids=512, seed=70 + d)
+    pool, ora = fill_both(w, n_rows=n_rows, key_format="e4m3", max_k=64, max_nq=64)
+    q, _ = w.queries("cuda")
+    pr = fixed(16, 4, theta=-2.0, path=B.PATH_TENSOR)
+    out = pool.query(q, pr)
+    check_query(out, ora, W.to_bits(q), pr)
+    if n_rows > 1000:
+        ws = w.separated()
+        pool, ora = fill_both(ws, key_format="e4m3", max_k=64, max_nq=64)
+        q, _ = ws.queries("cuda")
+        check_query(pool.query(q, pr), ora, W.to_bits(q), pr)
+        best = pool.query(q, pr).cpu().idx[:, 0].numpy()
+        ex = np.array([ws.trace_tag(int(b) // ws.rows_per_trace) for b in best], dtype=np.int64)
+        pr_ex = fixed(16, 4, theta=-2.0, path=B.PATH_TENSOR, exclude_tag=torch.from_numpy(ex).cuda())
+        check_query(pool.query(q, pr_ex), ora, W.to_bits(q), pr_ex, exclude=ex.astype(np.uint64))
+    assert pool.stats()["stalled"] == 0
+
+
+def test_batches_on_larger_8bit_pools_take_the_tensor_scan_by_themselves():
+    # more than 8 queries from 32 MB of codes on: query preparation + one scan + merge, where
+    # the warp-level scan would read the codes once per 8 queries; a step adds its append
+    w = W.C1.scaled(n_rows=70000, nq=20, k=8, d=512, cont_len=4, rows_per_trace=1000, seed=77)
+    pool, ora = fill_both(w, key_format="e4m3", max_nq=32, spare_rows=64)
+    q, _ = w.queries("cuda")
+    pr = fixed(8, 4, theta=-2.0)
+    l0 = pool.launch_count
+    out = pool.query(q, pr)
+    assert pool.launch_count - l0 == 3
+    check_query(out, ora, W.to_bits(q), pr)
+    g = torch.Generator(device="cuda").manual_seed(3)
+    st = torch.randn(8, w.d, generator=g, device="cuda").to(torch.bfloat16)
+    tk = torch.arange(8, dtype=torch.int32, device="cuda")
+    q[0] = st[5]
+    l0 = pool.launch_count
+    out = pool.step(st, tk, q, pr, tag=4242)
+    assert pool.launch_count - l0 == 4
+    ora.append(W.to_bits(st), tk.cpu().numpy(), tag=4242)
+    check_query(out, ora, W.to_bits(q), pr)
+    assert int(out.idx[0, 0]) == len(pool) - 3
+    small = pool.query(q[:8].contiguous(), pr)                   # 8 queries stay on the warp-level scan
+    check_query(small, ora, W.to_bits(q[:8]), pr)
+    assert pool.stats()["stalled"] == 0

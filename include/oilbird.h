@@ -330,9 +330,11 @@ int oilbird_pool_read_rows(oilbird_pool_t* pool, int64_t row0, int64_t n, void* 
  * stored as zero codes with scale 0).  A score is fp32(scale * sum_j qn_j * value(c_j)), the
  * query normalised and rounded to bf16 as for 16-bit pools; everything after the scores is
  * unchanged.  A row takes d + 4 bytes instead of 2d.  d must be a multiple of 16.  Such
- * pools use the CUDA-core scan for one or two queries and the warp-level tensor scan for
- * batches (OILBIRD_PATH_MMA: codes as f16, d a multiple of 256, else the CUDA-core scan two
- * queries per pass); OILBIRD_PATH_TENSOR is rejected,
+ * pools use the CUDA-core scan for one or two queries, the warp-level tensor scan for up to
+ * eight (OILBIRD_PATH_MMA: codes as f16, eight queries per pass over the codes, d a multiple
+ * of 256, else the CUDA-core scan two queries per pass) and the tcgen05 scan for larger
+ * batches from 32 MB of codes on (OILBIRD_PATH_TENSOR: the codes are turned into f16 inside
+ * the kernel and read once for the whole batch);
  * oilbird_query_static does not apply, and keys are read back with the call below
  * (oilbird_pool_read_rows then takes keys_host == NULL).
  * codes: [n,d] uint8; scales: [n] fp32; either may be NULL.

@@ -83,7 +83,8 @@
 namespace oilbird {
 
 constexpr int kTcThreads = 192;
-constexpr int kTcThreadsFp8 = 320;     // ... plus four warps that turn codes into f16 (8-bit pools)
+constexpr int kConvWarps = 6;          // warps that turn codes into f16 (8-bit pools)
+constexpr int kTcThreadsFp8 = kTcThreads + 32 * kConvWarps;
 constexpr int kTileM = 128;            // key rows per tile = TMEM lanes
 // bf16 elements per k-block = one 128-byte swizzle row.  (32-element blocks with the 64-byte
 // swizzle were measured too: more, finer ring stages, but every 128-byte line is then
@@ -293,13 +294,15 @@ __host__ __device__ inline uint32_t umma_idesc_bf16(int n, int m = kTileM) {
 __host__ __device__ inline uint32_t umma_idesc_f16(int n, int m = kTileM) {
   return (1u << 4) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
 }
-// two E4M3 codes (low 16 bits) -> f16x2, first code in the low half
-__device__ __forceinline__ uint32_t e4m3x2_to_f16x2(uint32_t two_codes) {
-  uint32_t h2;
-  asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(h2) : "h"((unsigned short)two_codes));
-  return h2;
+// four E4M3 codes (one word) -> two f16x2 (codes 0,1 and codes 2,3)
+__device__ __forceinline__ void e4m3x4_to_f16x4(uint32_t w, uint32_t& h01, uint32_t& h23) {
+  asm("{\n\t.reg .b16 lo, hi;\n\t"
+      "mov.b32 {lo, hi}, %2;\n\t"
+      "cvt.rn.f16x2.e4m3x2 %0, lo;\n\t"
+      "cvt.rn.f16x2.e4m3x2 %1, hi;\n\t}"
+      : "=r"(h01), "=r"(h23)
+      : "r"(w));
 }
-
 // Order-preserving map float -> unsigned (and back), so that a warp-wide maximum of scores is
 // one redux instruction; 0 is below every score.
 __device__ __forceinline__ uint32_t score_to_ord(float s) {
@@ -487,14 +490,20 @@ __device__ __forceinline__ float kth_largest_best(const float* lmax, int q, int 
 //
 // kFp8 (lone CTAs only): the pool holds E4M3 codes and one fp32 scale per row.  The tensor
 // core takes 16-bit operands, so a stage's codes (8 KB per tile, loaded by TMA without
-// swizzle) are turned into the f16 tile the MMA reads by four more warps: 16 codes per
+// swizzle) are turned into the f16 tile the MMA reads by six more warps: 16 codes per
 // 16-byte shared-memory load, `cvt.rn.f16x2.e4m3x2` (exact), two 16-byte stores into the
 // 128-byte-swizzled layout a TMA load would have produced, a proxy fence, and an arrival on
 // the stage's `cvt` barrier, which is what the MMA warp waits for in place of `full`.  The
 // queries arrive as f16 scaled by 2^14 (see the query preparation); a row's scale and the
 // 2^-14 are applied to its scores as they leave TMEM.  HBM carries half the bytes of a
 // 16-bit pool; shared memory carries more (codes in and out, f16 in and out), which is what
-// bounds this form.
+// bounds this form (C4 as codes, nq = 16: 0.95 ms = 4.5 TB/s of codes where the stage's
+// 100 KB through shared memory at 128 B/clock give 0.8).  Measured and dropped: making the
+// f16 numbers with integer shifts and masks (the code's magnitude bits at f16's exponent and
+// fraction read 2^-8 times its value, exactly, subnormal codes included) for all rows or
+// for every other quarter of a tile: 1.30 and 1.11 ms against 0.95; four or eight
+// converting warps in place of six: 1.02 and 0.95 against 0.97; a ring of code stages with
+// two f16 slots of their own: 1.14.
 template <bool kPair, bool kFp8 = false>
 __global__ void __launch_bounds__(kFp8 ? kTcThreadsFp8 : kTcThreads, 1)
 scan_tc_kernel(const __grid_constant__ CUtensorMap key_map,
@@ -553,7 +562,7 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap key_map,
     for (int s = 0; s < n_stages; ++s) {
       mbar_init(&sh.full[s], 1);
       mbar_init(&sh.empty[s], 1);
-      mbar_init(&sh.cvt[s], 4);
+      mbar_init(&sh.cvt[s], kConvWarps);
     }
     for (int b = 0; b < 2; ++b) {
       mbar_init(&sh.tmem_full[b], 1);
@@ -741,7 +750,7 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap key_map,
     // lanes read consecutive pieces: no bank conflict); piece g is codes 16 (g % 4) onward of
     // row g / 4, i.e. the row's 16-byte f16 chunks 2 (g % 4) and 2 (g % 4) + 1, which the
     // 128-byte swizzle keeps at chunk position (chunk ^ (row % 8)) of the row's 128 bytes
-    const int ct = threadIdx.x - 192;
+    const int ct = threadIdx.x - kTcThreads;
     uint32_t it = 0;
     bool ok = true;
     for (int tile = unit; tile < n_tiles && ok; tile += n_units) {
@@ -750,17 +759,30 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap key_map,
         if (!mbar_wait(&sh.full[s], (it / n_stages) & 1u, abort_flag, stats)) { ok = false; break; }
         unsigned char* a_dst = ring + (size_t)s * stage_bytes;
         const uint4* raw = reinterpret_cast<const uint4*>(a_dst + raw_off);
-        for (int g = ct; g < mt * (kCodeTileBytes / 16); g += 128) {
-          const uint4 c = raw[g];
-          const int row_all = g >> 2, c4 = g & 3;           // row over the stage's tiles
-          unsigned char* row_dst = a_dst + (size_t)row_all * 128;
-          const int sw = row_all & 7;
-          const uint4 lo = make_uint4(e4m3x2_to_f16x2(c.x), e4m3x2_to_f16x2(c.x >> 16),
-                                      e4m3x2_to_f16x2(c.y), e4m3x2_to_f16x2(c.y >> 16));
-          const uint4 hi = make_uint4(e4m3x2_to_f16x2(c.z), e4m3x2_to_f16x2(c.z >> 16),
-                                      e4m3x2_to_f16x2(c.w), e4m3x2_to_f16x2(c.w >> 16));
-          *reinterpret_cast<uint4*>(row_dst + (((2 * c4) ^ sw) << 4)) = lo;
-          *reinterpret_cast<uint4*>(row_dst + (((2 * c4 + 1) ^ sw) << 4)) = hi;
+        // All of a thread's pieces are loaded before any is converted (one after the other, each
+        // waiting for its own load, kept the whole scan at a third of its rate).
+        constexpr int kConvThreads = 32 * kConvWarps;
+        constexpr int kMaxPieces = (2 * kCodeTileBytes / 16 + kConvThreads - 1) / kConvThreads;
+        const int n_total = mt * (kCodeTileBytes / 16);                 // 16-byte pieces of the stage
+        uint4 c[kMaxPieces];
+#pragma unroll
+        for (int i = 0; i < kMaxPieces; ++i)
+          if (ct + i * kConvThreads < n_total) c[i] = raw[ct + i * kConvThreads];
+#pragma unroll
+        for (int i = 0; i < kMaxPieces; ++i) {
+          if (ct + i * kConvThreads < n_total) {
+            const int g = ct + i * kConvThreads;
+            const int row_all = g >> 2, c4 = g & 3;         // row over the stage's tiles
+            unsigned char* row_dst = a_dst + (size_t)row_all * 128;
+            const int sw = row_all & 7;
+            uint4 lo, hi;
+            e4m3x4_to_f16x4(c[i].x, lo.x, lo.y);
+            e4m3x4_to_f16x4(c[i].y, lo.z, lo.w);
+            e4m3x4_to_f16x4(c[i].z, hi.x, hi.y);
+            e4m3x4_to_f16x4(c[i].w, hi.z, hi.w);
+            *reinterpret_cast<uint4*>(row_dst + (((2 * c4) ^ sw) << 4)) = lo;
+            *reinterpret_cast<uint4*>(row_dst + (((2 * c4 + 1) ^ sw) << 4)) = hi;
+          }
         }
         // the tile was written through the generic proxy; the MMA reads it through the async one
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");

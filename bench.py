@@ -449,7 +449,8 @@ def measure(pool, w, nq, rows_step, K, Wm, dev, world, rank, local, args, n0, ra
         "device_stalled_flag": stalled,
     }
     n_pad = (nq + 15) // 16 * 16
-    if args.keys == "bf16" and (args.path in (2, 3) or (args.path == 0 and nq > 2)):
+    if (args.keys == "bf16" and (args.path in (2, 3) or (args.path == 0 and nq > 2))) or \
+            (args.keys == "e4m3" and (args.path == 2 or (args.path == 0 and nq > 8))):
         # the batched path is a dense contraction: report its tensor-pipe share too
         # (2*N*d*n_pad flops per launch, queries padded to the MMA's N)
         tflops = 2.0 * rows_scan * w.d * n_pad / (scan_mean_ms * 1e-3) / 1e12
@@ -603,6 +604,21 @@ def run_legs(args, dev, local, K, Wm):
     pool = make_pool(w, w.nq, rows_step, w.n_rows + spare, local, args, spare // rows_step + 8)
     fill_pool(pool, w, w.n_rows, dev)
     leg(pool, w, w.nq, w.n_rows, key="C4")
+    pool.close()
+    del pool
+    torch.cuda.empty_cache()
+
+    # the same configuration as a bounded store: 8-bit keys, half the bytes (tcgen05 scan on
+    # codes turned into f16 on chip)
+    import copy
+    args8 = copy.copy(args)
+    args8.keys = "e4m3"
+    pool = make_pool(w, w.nq, rows_step, w.n_rows + spare, local, args8, spare // rows_step + 8)
+    fill_pool(pool, w, w.n_rows, dev)
+    r = measure(pool, w, w.nq, rows_step, K, Wm, dev, 1, 0, local, args8, w.n_rows, raw=None,
+                traffic_key=None)
+    r["config"] = w.name + " (8-bit keys)"
+    legs.append(r)
     pool.close()
     del pool
     torch.cuda.empty_cache()

@@ -594,7 +594,10 @@ def test_pairs_of_ctas_with_two_tiles_each_from_97_to_224_queries(nq, k):
     tiles of 512 rows (two MMAs over both CTAs per query tile), with two accumulator sets up
     to 128 queries and one above.  Last macro tile with one, two and three of its four
     sub-tiles (partly) filled."""
-    for n_rows in (148 * 128 * 8 + 77, 148 * 128 * 8 + 128 + 5, 148 * 128 * 8 + 3 * 128 - 1):
+    sizes = (148 * 128 * 8 + 77, 148 * 128 * 8 + 128 + 5, 148 * 128 * 8 + 3 * 128 - 1)
+    if (nq, k) not in ((128, 64), (160, 16)):   # the other batch sizes take one ragged size each
+        sizes = sizes[(nq + k) % 3:][:1]
+    for n_rows in sizes:
         w = W.C1.scaled(nq=nq, k=k, n_rows=n_rows, d=128, cont_len=3, n_centroids=2048,
                         rows_per_trace=1024, seed=80 + k)
         pool, ora = fill_both(w, max_k=128, max_nq=256)

@@ -59,6 +59,10 @@ extern "C" {
 
 /* append flags */
 #define OILBIRD_NEW_TRACE  1u   /* the rows open a new trace (a finished request)      */
+#define OILBIRD_EVICT_TO_FIT 2u /* bounded store: if the rows (or the new trace) do not fit,
+                                   the fewest oldest traces are evicted first, as by
+                                   oilbird_pool_evict_oldest (never the trace being extended);
+                                   OILBIRD_ECAPACITY only if that cannot make room        */
 
 /* depth modes (Eq. 3 and the fixed-span variant of the batched harness) */
 #define OILBIRD_DEPTH_FIXED   0  /* every neighbour copies cont_len tokens             */

@@ -27,6 +27,8 @@ LIB_PATH = os.path.join(_HERE, "liboilbird.so")
 
 OK, EINVAL, ECAPACITY, ENOMEM, ECUDA, ESTALL, EGUARD = 0, -1, -2, -3, -4, -5, -6
 NEW_TRACE = 1
+EVICT_TO_FIT = 2
+EVICT_TO_FIT = 2
 KEYS_E4M3 = 1          # pool flag: 8-bit keys
 DEBUG_GUARDS = 2       # pool flag: sentinel bytes behind every array (see Pool.check_guards)
 DEPTH_FIXED, DEPTH_TIERED = 0, 1
@@ -198,6 +200,10 @@ class OilbirdError(RuntimeError):
             msg += " (" + L.oilbird_last_cuda_error().decode() + ")"
         super().__init__(f"{where}: {msg} [{code}]")
         self.code = code
+
+
+def _flags(new_trace: bool, evict_to_fit: bool) -> int:
+    return (NEW_TRACE if new_trace else 0) | (EVICT_TO_FIT if evict_to_fit else 0)
 
 
 def _check(code: int, where: str) -> None:
@@ -392,7 +398,7 @@ class Pool:
 
     # ---- device-buffer entry points -------------------------------------------------
     def append(self, states: torch.Tensor, tokens: torch.Tensor, tag: int = 0,
-               new_trace: bool = True, stream=None) -> None:
+               new_trace: bool = True, evict_to_fit: bool = False, stream=None) -> None:
         n = int(tokens.shape[0])
         if n:
             assert states.is_cuda and tokens.is_cuda and states.dtype == torch.bfloat16
@@ -400,11 +406,11 @@ class Pool:
             assert states.shape == (n, self.d)
         _check(self._L.oilbird_pool_append(self._h, states.data_ptr() if n else None,
                                            tokens.data_ptr() if n else None, n, int(tag),
-                                           NEW_TRACE if new_trace else 0, _stream_ptr(stream)),
+                                           _flags(new_trace, evict_to_fit), _stream_ptr(stream)),
                "oilbird_pool_append")
 
     def append_global(self, states: torch.Tensor, tokens: torch.Tensor, global_row: int,
-                      tag: int = 0, new_trace: bool = True, stream=None) -> None:
+                      tag: int = 0, new_trace: bool = True, evict_to_fit: bool = False, stream=None) -> None:
         """append() for a pool that is one shard of a larger one: global_row is the position
         of the first appended row in the logical pool."""
         n = int(tokens.shape[0])
@@ -412,7 +418,7 @@ class Pool:
         assert tokens.dtype == torch.int32 and states.is_contiguous() and tokens.is_contiguous()
         _check(self._L.oilbird_pool_append_global(
             self._h, states.data_ptr(), tokens.data_ptr(), n, int(tag),
-            NEW_TRACE if new_trace else 0, int(global_row), _stream_ptr(stream)),
+            _flags(new_trace, evict_to_fit), int(global_row), _stream_ptr(stream)),
             "oilbird_pool_append_global")
 
     def to_global(self, idx: torch.Tensor, out: torch.Tensor | None = None, stream=None
@@ -455,7 +461,7 @@ class Pool:
 
     def step(self, states: torch.Tensor, tokens: torch.Tensor, q: torch.Tensor,
              params: QueryParams | None = None, out: QueryOut | None = None, tag: int = 0,
-             new_trace: bool = True, stream=None) -> QueryOut:
+             new_trace: bool = True, evict_to_fit: bool = False, stream=None) -> QueryOut:
         """One serving step on device tensors: append(states, tokens) then query(q), in one
         call (same results as the two calls; the single-request scan overlaps the append)."""
         pr = params or QueryParams()
@@ -476,7 +482,7 @@ class Pool:
         cp = pr.to_c(ex_ptr)
         _check(self._L.oilbird_pool_step(
             self._h, states.data_ptr(), tokens.data_ptr(), n, int(tag),
-            NEW_TRACE if new_trace else 0, q.data_ptr(), nq, ctypes.byref(cp),
+            _flags(new_trace, evict_to_fit), q.data_ptr(), nq, ctypes.byref(cp),
             ctypes.byref(out._c), _stream_ptr(stream)), "oilbird_pool_step")
         return out
 
@@ -496,12 +502,12 @@ class Pool:
 
     # ---- host-buffer entry points ---------------------------------------------------
     def append_host(self, states: torch.Tensor, tokens: torch.Tensor, tag: int = 0,
-                    new_trace: bool = True, stream=None) -> None:
+                    new_trace: bool = True, evict_to_fit: bool = False, stream=None) -> None:
         """states: CPU bf16 tensor [n,d] (ideally pinned); tokens: CPU int32 [n]."""
         n = int(tokens.shape[0])
         assert not states.is_cuda and not tokens.is_cuda and states.is_contiguous()
         _check(self._L.oilbird_pool_append_host(self._h, states.data_ptr(), tokens.data_ptr(), n,
-                                                int(tag), NEW_TRACE if new_trace else 0,
+                                                int(tag), _flags(new_trace, evict_to_fit),
                                                 _stream_ptr(stream)), "oilbird_pool_append_host")
 
     def query_host(self, q: torch.Tensor, params: QueryParams | None = None,
@@ -525,26 +531,26 @@ class Pool:
         return out
 
     def step_host(self, states: torch.Tensor, tokens: torch.Tensor, q: torch.Tensor,
-                  params: QueryParams, out: QueryOut, tag: int = 0, new_trace: bool = True,
+                  params: QueryParams, out: QueryOut, tag: int = 0, new_trace: bool = True, evict_to_fit: bool = False,
                   stream=None) -> QueryOut:
         """One serving step from host memory: append the committed rows, then query.
         All tensors are CPU tensors; `out` must have been made with QueryOut.empty(..., "cpu")."""
         cp = params.to_c(None)
         _check(self._L.oilbird_pool_step_host(
             self._h, states.data_ptr(), tokens.data_ptr(), int(tokens.shape[0]), int(tag),
-            NEW_TRACE if new_trace else 0, q.data_ptr(), int(q.shape[0]), ctypes.byref(cp),
+            _flags(new_trace, evict_to_fit), q.data_ptr(), int(q.shape[0]), ctypes.byref(cp),
             ctypes.byref(out._c), _stream_ptr(stream)), "oilbird_pool_step_host")
         return out
 
     def step_host_begin(self, states: torch.Tensor, tokens: torch.Tensor, q: torch.Tensor,
-                        params: QueryParams, slot: int, tag: int = 0, new_trace: bool = True,
+                        params: QueryParams, slot: int, tag: int = 0, new_trace: bool = True, evict_to_fit: bool = False,
                         stream=None) -> None:
         """First half of step_host: returns once the step is enqueued (slot 0 or 1)."""
         ex_ptr = params.exclude_tag.data_ptr() if params.exclude_tag is not None else None
         cp = params.to_c(ex_ptr)
         _check(self._L.oilbird_pool_step_host_begin(
             self._h, states.data_ptr(), tokens.data_ptr(), int(tokens.shape[0]), int(tag),
-            NEW_TRACE if new_trace else 0, q.data_ptr(), int(q.shape[0]), ctypes.byref(cp),
+            _flags(new_trace, evict_to_fit), q.data_ptr(), int(q.shape[0]), ctypes.byref(cp),
             int(slot), _stream_ptr(stream)), "oilbird_pool_step_host_begin")
 
     def step_host_end(self, slot: int, out: QueryOut) -> QueryOut:

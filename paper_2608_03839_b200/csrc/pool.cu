@@ -344,12 +344,47 @@ static void append_commit(oilbird_pool_t* p, int64_t n, const AppendPlan& ap) {
   p->t_end[ap.trace] = p->n_rows;
 }
 
+// OILBIRD_EVICT_TO_FIT: how many of the oldest traces have to go so that n more rows (and a new
+// trace, if one is opened) fit: the fewest, never the trace that is being extended.  Returns
+// OILBIRD_ECAPACITY if even that does not make room.  *rows = the rows those traces hold.
+static int evict_plan(const oilbird_pool* p, int64_t n, uint32_t flags, int32_t* n_traces,
+                      int64_t* rows) {
+  *n_traces = 0;
+  *rows = 0;
+  if (!(flags & OILBIRD_EVICT_TO_FIT)) return OILBIRD_OK;
+  const bool open_new = (flags & OILBIRD_NEW_TRACE) || p->t_start.empty();
+  const int32_t have = (int32_t)p->t_start.size();
+  const int32_t may_go = open_new ? have : have - 1;          // the open trace stays
+  int32_t nt = 0;
+  int64_t dropped = 0;
+  while ((p->n_rows - dropped + n > p->r.capacity ||
+          (open_new && have - nt >= p->r.max_traces)) && nt < may_go) {
+    dropped = p->t_end[nt];
+    ++nt;
+  }
+  if (p->n_rows - dropped + n > p->r.capacity || (open_new && have - nt >= p->r.max_traces))
+    return OILBIRD_ECAPACITY;
+  *n_traces = nt;
+  *rows = dropped;
+  return OILBIRD_OK;
+}
+static int evict_to_fit(oilbird_pool_t* p, int64_t n, uint32_t flags, void* stream) {
+  int32_t nt;
+  int64_t rows;
+  int rc = evict_plan(p, n, flags, &nt, &rows);
+  if (rc || nt == 0) return rc;
+  return oilbird_pool_evict_oldest(p, nt, nullptr, stream);
+}
+
 // global_row < 0: the pool is not a shard, a trace's global position is its local one.
 static int append_impl(oilbird_pool_t* p, const void* states, const int32_t* tokens, int64_t n,
                        uint64_t tag, uint32_t flags, int64_t global_row, void* stream) {
   AppendPlan ap;
   bool nothing;
-  int rc = append_prepare(p, states, tokens, n, tag, flags, &ap, &nothing);
+  if (!p || n < 0 || (n > 0 && (!states || !tokens))) return OILBIRD_EINVAL;
+  int rc = evict_to_fit(p, n, flags, stream);
+  if (rc) return rc;
+  rc = append_prepare(p, states, tokens, n, tag, flags, &ap, &nothing);
   if (rc || nothing) return rc;
   CU(cudaSetDevice(p->device));
   PdlScope plain(long_scan(p));
@@ -641,9 +676,18 @@ static int step_impl(oilbird_pool_t* p, const void* states, const int32_t* token
   // nothing is appended if the query would be refused (arguments, parameters, or a scan this
   // pool does not have)
   if (!p) return OILBIRD_EINVAL;
-  const int64_t rows_after = p->n_rows + n;
-  int rc = check_query(p, q, nq, pr, out, rows_after, &gp, &path);
+  // (a step that evicts to make room: planned first, done only once the query has passed)
+  int32_t evict_traces = 0;
+  int64_t evict_rows = 0;
+  int rc = evict_plan(p, n, flags, &evict_traces, &evict_rows);
   if (rc) return rc;
+  const int64_t rows_after = p->n_rows - evict_rows + n;
+  rc = check_query(p, q, nq, pr, out, rows_after, &gp, &path);
+  if (rc) return rc;
+  if (evict_traces > 0) {
+    rc = oilbird_pool_evict_oldest(p, evict_traces, nullptr, stream);
+    if (rc) return rc;
+  }
   // (8-bit pools always use the CUDA-core scan; its passes beyond the first two queries
   // would find the rows in place, but keep to the single-request case there too)
   const bool gemv = p->r.e4m3 ? (nq <= 2 && path == OILBIRD_PATH_GEMV) : path == OILBIRD_PATH_GEMV;

@@ -153,3 +153,98 @@ def test_eviction_keeps_global_positions_of_a_shard():
     pool.evict_oldest(1)
     idx = torch.tensor([0, 9, 10, 19, -1], dtype=torch.int32, device="cuda")
     assert pool.to_global(idx).tolist() == [5000, 5009, 70000, 70009, -1]
+
+
+def fewest_traces_to_go(ora, n, capacity, max_traces, open_new):
+    """The definition of OILBIRD_EVICT_TO_FIT, by trying every count in turn."""
+    ends = ora.trace_ends.tolist()
+    have = len(ends)
+    may_go = have if open_new else have - 1
+    for nt in range(0, may_go + 1):
+        dropped = ends[nt - 1] if nt else 0
+        if len(ora) - dropped + n <= capacity and (not open_new or have - nt < max_traces):
+            return nt
+    return None
+
+
+@pytest.mark.parametrize("fmt", ["bf16", "e4m3"])
+def test_appends_and_steps_that_evict_to_fit(fmt):
+    """A bounded store: appends and steps that do not fit drop the fewest oldest traces first,
+    exactly as oilbird_pool_evict_oldest would; everything else is as after that eviction."""
+    d, cap, max_traces = 256, 1000, 7
+    pool = B.Pool(d, cap, max_traces=max_traces, max_nq=8, key_format=fmt)
+    ora = OraclePool(d, fmt)
+    g = torch.Generator(device="cuda").manual_seed(21)
+    next_tag = [100]
+
+    def rows(n):
+        st = torch.randn(n, d, generator=g, device="cuda").to(torch.bfloat16)
+        return st, torch.randint(0, 1000, (n,), generator=g, device="cuda", dtype=torch.int32)
+
+    def both(n, new=True, step_nq=0, host=False):
+        st, tk = rows(n)
+        tag = next_tag[0]; next_tag[0] += 1
+        nt = fewest_traces_to_go(ora, n, cap, max_traces, new or ora.num_traces == 0)
+        assert nt is not None
+        gen0 = pool.num_traces
+        if step_nq:
+            q = rows(step_nq)[0]
+            if n:
+                q[0] = st[n - 1]
+            pr = fixed(4, 4, theta=-2.0)
+            if host:
+                out = B.QueryOut.empty(step_nq, 4, 4, "cpu")
+                pool.step_host(st.cpu(), tk.cpu(), q.cpu(), pr, out, tag=tag, new_trace=new, evict_to_fit=True)
+            else:
+                out = pool.step(st, tk, q, pr, tag=tag, new_trace=new, evict_to_fit=True)
+        elif host:
+            pool.append_host(st.cpu(), tk.cpu(), tag=tag, new_trace=new, evict_to_fit=True)
+        else:
+            pool.append(st, tk, tag=tag, new_trace=new, evict_to_fit=True)
+        ora.evict_oldest(nt)
+        ora.append(W.to_bits(st), tk.cpu().numpy(), tag=tag, new_trace=new)
+        same_store(pool, ora)
+        if step_nq:
+            check_query(out, ora, W.to_bits(q), pr)
+            if n:
+                assert int(out.idx[0, 0]) == len(pool) - 1
+        return nt
+
+    for _ in range(5):
+        assert both(200) == 0                     # 1,000 rows, 5 traces: full
+    assert both(150) == 1                         # one trace goes: 950 rows
+    assert both(50) == 0                          # fits exactly
+    assert both(8, step_nq=1) == 1                # a fused step that has to make room
+    assert both(100, new=False) == 0              # the open trace grows into the room left
+    assert both(300, step_nq=3) >= 1              # a step with its own append kernel
+    assert both(120, host=True) >= 0
+    assert both(64, step_nq=2, host=True) >= 0
+    # the trace table fills before the rows do: one-row traces
+    for _ in range(2 * max_traces):
+        both(1)
+    assert pool.num_traces == max_traces
+    # the open trace is never evicted: extending it beyond what the others can free is refused
+    while ora.num_traces > 1:
+        pool.evict_oldest(1); ora.evict_oldest(1)
+    room = cap - len(ora)
+    st, tk = rows(room + 1)
+    before = (len(pool), pool.num_traces)
+    with pytest.raises(B.OilbirdError) as e:
+        pool.append(st, tk, new_trace=False, evict_to_fit=True)
+    assert e.value.code == B.ECAPACITY and (len(pool), pool.num_traces) == before
+    # ... but as a new trace the same rows fit once the old one has gone
+    assert both(room + 1) == 1
+    # more rows than the pool holds at all
+    st, tk = rows(cap + 1)
+    with pytest.raises(B.OilbirdError) as e:
+        pool.append(st, tk, tag=1, evict_to_fit=True)
+    assert e.value.code == B.ECAPACITY
+    # a refused step evicts nothing
+    both(600)
+    before = (len(pool), pool.num_traces)
+    st, tk = rows(700)
+    with pytest.raises(B.OilbirdError) as e:
+        pool.step(st, tk, st[:2].contiguous(), fixed(4, 4, path=9), tag=5, evict_to_fit=True)
+    assert e.value.code == B.EINVAL and (len(pool), pool.num_traces) == before
+    same_store(pool, ora)
+    assert pool.stats()["stalled"] == 0

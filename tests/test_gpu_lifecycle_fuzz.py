@@ -15,6 +15,17 @@ from parity import check_query
 pytestmark = pytest.mark.gpu
 
 
+def fewest_traces_to_go(ora, n, capacity, max_traces, open_new):
+    """OILBIRD_EVICT_TO_FIT by its definition: the first count that makes room."""
+    ends = ora.trace_ends.tolist()
+    have = len(ends)
+    for nt in range(0, (have if open_new else have - 1) + 1):
+        dropped = ends[nt - 1] if nt else 0
+        if len(ora) - dropped + n <= capacity and (not open_new or have - nt < max_traces):
+            return nt
+    return None
+
+
 def same_store(pool, ora):
     if pool.key_format == "bf16":
         keys, tok, tid = pool.read_rows()
@@ -62,17 +73,23 @@ def test_random_life_cycle(fmt, seed):
                         p=[0.25, 0.2, 0.2, 0.2, 0.12, 0.03])
         if op in ("append", "step"):
             n = int(rng.choice([0, 1, 7, 8, 40, 64, 65, 200]))
+            fit = False
             if len(pool) + n > cap or pool.num_traces + 1 > 390:
-                op, n = "evict", 0
+                if rng.random() < 0.5:
+                    fit = True                   # the call makes its own room
+                else:
+                    op, n = "evict", 0
         host = bool(rng.random() < 0.3)          # through the host-buffer entry points
         if op == "append":
             st, tk = rows(n)
-            new = bool(rng.random() < 0.7) or len(pool) == 0
+            new = bool(rng.random() < 0.7) or len(pool) == 0 or fit
             tag = next_tag[0]; next_tag[0] += 1
             if host:
-                pool.append_host(st.cpu(), tk.cpu(), tag=tag, new_trace=new)
+                pool.append_host(st.cpu(), tk.cpu(), tag=tag, new_trace=new, evict_to_fit=fit)
             else:
-                pool.append(st, tk, tag=tag, new_trace=new)
+                pool.append(st, tk, tag=tag, new_trace=new, evict_to_fit=fit)
+            if fit:
+                ora.evict_oldest(fewest_traces_to_go(ora, n, cap, 400, True))
             ora.append(W.to_bits(st), tk.cpu().numpy(), tag=tag, new_trace=new)
         elif op == "step":
             st, tk = rows(n)
@@ -80,19 +97,23 @@ def test_random_life_cycle(fmt, seed):
             q = rows(nq)[0]
             if n > 0:
                 q[0] = st[n - 1]
-            new = bool(rng.random() < 0.7) or len(pool) == 0
+            new = bool(rng.random() < 0.7) or len(pool) == 0 or fit
             tag = next_tag[0]; next_tag[0] += 1
             pr = params(nq)
             in_flight = host and bool(rng.random() < 0.5)   # the two-halves form of the host step
             if in_flight:
                 out = B.QueryOut.empty(nq, pr.k, pr.cont_len, "cpu")
                 slot = int(rng.integers(0, 2))
-                pool.step_host_begin(st.cpu(), tk.cpu(), q.cpu(), pr, slot, tag=tag, new_trace=new)
+                pool.step_host_begin(st.cpu(), tk.cpu(), q.cpu(), pr, slot, tag=tag, new_trace=new,
+                                     evict_to_fit=fit)
             elif host:
                 out = B.QueryOut.empty(nq, pr.k, pr.cont_len, "cpu")
-                pool.step_host(st.cpu(), tk.cpu(), q.cpu(), pr, out, tag=tag, new_trace=new)
+                pool.step_host(st.cpu(), tk.cpu(), q.cpu(), pr, out, tag=tag, new_trace=new,
+                               evict_to_fit=fit)
             else:
-                out = pool.step(st, tk, q, pr, tag=tag, new_trace=new)
+                out = pool.step(st, tk, q, pr, tag=tag, new_trace=new, evict_to_fit=fit)
+            if fit:
+                ora.evict_oldest(fewest_traces_to_go(ora, n, cap, 400, True))
             ora.append(W.to_bits(st), tk.cpu().numpy(), tag=tag, new_trace=new)
             if in_flight:
                 if len(ora) and rng.random() < 0.7:      # other lookups while the step is in flight

@@ -331,7 +331,7 @@ def test_mma_scan_appends_the_rows_of_a_step_itself():
 
 # ---- tcgen05 scan of 8-bit pools: codes turned into f16 inside the kernel ---------------
 
-@pytest.mark.parametrize("d", [64, 256, 1024, 4096])
+@pytest.mark.parametrize("d", [16, 64, 256, 1024, 4096])
 def test_tensor_scan_closed_form_pool_scores_are_exact(d):
     # +-1 rows (codes +-448) and +-1 queries: f16 products and their sums are exact, so the
     # scan must return the oracle's scores, order and ties bit for bit

@@ -19,6 +19,17 @@ are taken:
 So the result is the brute-force result restricted to the candidate rows: with every list
 probed it IS the brute-force result, which is the first pin.  Everything is built from
 OraclePool (full scores in double, full sort); plain numpy and Python loops on purpose.
+
+  train    Lloyd's iterations on the rows the pool holds (spherical k-means, the textbook
+           procedure; the paper defines none).  One iteration: every row is assigned as
+           above; then each centroid that has rows becomes the mean of its rows' stored
+           keys, and a centroid without rows stays as it is.  So that the mean does not
+           depend on the order of the rows it is taken in fixed point: element x of a stored
+           key contributes trunc(x * 2^30) (an integer, |x| <= 1), the integers are summed
+           exactly, and the new raw centroid element is bf16(float(double(sum) /
+           (count * 2^30))), both roundings to nearest even.  The raw centroids then go
+           through the same normalisation as at creation.  After the last iteration the lists
+           are rebuilt from scratch.
 """
 from __future__ import annotations
 
@@ -33,9 +44,13 @@ class OracleIndex:
         c = np.ascontiguousarray(centroids_bits, dtype=np.uint16).reshape(-1, pool.d)
         self.pool = pool
         self.n_lists = c.shape[0]
-        self.cent = OraclePool(pool.d)
-        self.cent.append(c, np.arange(self.n_lists, dtype=np.int32), tag=0)
+        self.cent_raw = c.copy()                       # raw centroid states (bf16 bit patterns)
+        self._build_centroids()
         self.assign = np.empty(0, dtype=np.int64)      # list of every indexed row
+
+    def _build_centroids(self) -> None:
+        self.cent = OraclePool(self.pool.d)
+        self.cent.append(self.cent_raw, np.arange(self.n_lists, dtype=np.int32), tag=0)
 
     @property
     def n_indexed(self) -> int:
@@ -56,6 +71,25 @@ class OracleIndex:
         for r0 in range(0, keys.shape[0], step):
             new[r0:r0 + step] = self.cent.query(keys[r0:r0 + step], one).idx[:, 0]
         self.assign = np.concatenate([self.assign, new])
+
+    def train(self, iterations: int) -> None:
+        """Lloyd's iterations (see the header); afterwards every row of the pool is indexed."""
+        from . import bf16_bits_to_f32, f32_to_bf16_bits
+        for _ in range(int(iterations)):
+            self.reset()
+            self.refresh()
+            x = bf16_bits_to_f32(self.pool.keys).astype(np.float64)       # stored keys, exact
+            t = np.trunc(x * 2.0 ** 30).astype(np.int64)
+            for l in range(self.n_lists):
+                rows = np.nonzero(self.assign == l)[0]
+                if rows.size == 0:
+                    continue                                              # keeps its centroid
+                total = t[rows].sum(axis=0, dtype=np.int64)               # exact, any order
+                mean = total.astype(np.float64) / (float(rows.size) * 2.0 ** 30)
+                self.cent_raw[l] = f32_to_bf16_bits(mean.astype(np.float32))
+            self._build_centroids()
+        self.reset()
+        self.refresh()
 
     def lists(self) -> list[np.ndarray]:
         return [np.nonzero(self.assign == l)[0] for l in range(self.n_lists)]

@@ -166,3 +166,117 @@ def test_exclusion_and_reset():
     assert idx.n_indexed == 0
     # with nothing indexed every row is tail: brute force whatever is probed
     assert np.array_equal(idx.query(q, 1, fixed(3)).idx, pool.query(q, fixed(3)).idx)
+
+
+# ---- training (Lloyd's iterations) ------------------------------------------------------
+
+def pm1_pool(rows):
+    """Rows of +-1 with d = 16 normalise to +-0.25 exactly, so means can be written down."""
+    pool = OraclePool(16)
+    pool.append(f2b(np.asarray(rows, dtype=np.float32)), np.arange(len(rows), dtype=np.int32), tag=1)
+    return pool
+
+
+def test_one_iteration_by_hand():
+    a = [1.0] * 16
+    b = [1.0] * 12 + [-1.0] * 4          # cos(a, b) = 0.5
+    c = [-1.0] * 16
+    e = [-1.0] * 8 + [1.0] * 8           # cos(c, e) = 0, cos(a, e) = 0
+    pool = pm1_pool([a, b, c, e, a])
+    # centroid 0 near a, centroid 1 near c, centroid 2 = e exactly (but rows tie towards lower
+    # centroids only when scores are equal: e scores 1 against centroid 2)
+    c0 = [1.0] * 15 + [0.5]
+    c1 = [-1.0] * 15 + [-0.5]
+    idx = OracleIndex(pool, f2b(np.array([c0, c1, e, [0.0] * 15 + [1.0]], dtype=np.float32)))
+    idx.train(1)
+    # lists after the iteration's own assignment: {a, b, a} -> 0, {c} -> 1, {e} -> 2, none -> 3
+    got = oracle.bf16_bits_to_f32(idx.cent_raw)
+    mean0 = (2 * np.array(a) * 0.25 + np.array(b) * 0.25) / 3        # 0.25 x 12, 0.25/3 x 4
+    assert np.array_equal(got[0], oracle.bf16_bits_to_f32(f2b(mean0.astype(np.float32))))
+    assert np.array_equal(got[0][:12], np.full(12, 0.25, dtype=np.float32))
+    assert np.array_equal(got[0][12:], oracle.bf16_bits_to_f32(f2b(np.full(4, 0.25 / 3, np.float32))))
+    assert np.array_equal(got[1], np.full(16, -0.25, dtype=np.float32))     # the one row itself
+    assert np.array_equal(got[2], np.array(e, dtype=np.float32) * 0.25)
+    assert np.array_equal(idx.cent_raw[3], f2b(np.array([0.0] * 15 + [1.0], dtype=np.float32)))  # kept
+    assert idx.n_indexed == 5
+    assert [l.tolist() for l in idx.lists()] == [[0, 1, 4], [2], [3], []]
+
+
+def test_fixed_point_sum_is_exact_and_order_free():
+    # many rows whose elements differ wildly in size: the integer sum is the same whatever
+    # the order, and equals the exact rational sum of the truncated terms
+    rng = np.random.default_rng(3)
+    d, n = 8, 200
+    rows = (rng.standard_normal((n, d)) * np.exp(rng.uniform(-12, 0, size=(n, d)))).astype(np.float32)
+    pool = OraclePool(d)
+    pool.append(f2b(rows), np.arange(n, dtype=np.int32), tag=1)
+    idx = OracleIndex(pool, f2b(np.ones((1, d), dtype=np.float32)))
+    idx.train(1)
+    x = oracle.bf16_bits_to_f32(pool.keys).astype(np.float64)
+    from fractions import Fraction
+    for j in range(d):
+        total = sum(int(np.trunc(v * 2.0 ** 30)) for v in x[::-1, j])          # Python ints, reversed
+        mean = Fraction(total, n * 2 ** 30)
+        want = f2b(np.array([np.float32(float(mean))]))[0]                      # float(Fraction) is correctly rounded
+        assert idx.cent_raw[0, j] == want
+
+
+def test_training_is_a_fixed_point_once_converged_and_never_lowers_the_objective():
+    rng = np.random.default_rng(11)
+    d, n, n_lists = 32, 600, 12
+    cent = rng.standard_normal((n_lists, d))
+    rows = cent[rng.integers(0, n_lists, n)] + 0.3 * rng.standard_normal((n, d))
+    pool = OraclePool(d)
+    pool.append(f2b(rows.astype(np.float32)), np.arange(n, dtype=np.int32), tag=1)
+    start = f2b(rows[:n_lists].astype(np.float32))                 # twelve rows as first centroids
+    idx = OracleIndex(pool, start)
+    one = fixed(1)
+
+    def objective(ix):
+        return float(ix.cent.query(pool.keys, one).score[:, 0].astype(np.float64).sum())
+
+    idx.refresh()
+    obj = [objective(idx)]
+    for _ in range(6):
+        idx.train(1)
+        obj.append(objective(idx))
+    assert all(b >= a - 1e-3 for a, b in zip(obj, obj[1:])) and obj[-1] > obj[0] + 1.0
+    # several single iterations equal one call with that many
+    again = OracleIndex(pool, start)
+    again.train(6)
+    assert np.array_equal(again.cent_raw, idx.cent_raw) and np.array_equal(again.assign, idx.assign)
+    # converged: further iterations change nothing
+    for _ in range(20):
+        before = idx.cent_raw.copy()
+        idx.train(1)
+        if np.array_equal(before, idx.cent_raw):
+            break
+    before, lists = idx.cent_raw.copy(), [l.tolist() for l in idx.lists()]
+    idx.train(2)
+    assert np.array_equal(before, idx.cent_raw) and lists == [l.tolist() for l in idx.lists()]
+    # and the answers with every list probed are still brute force
+    q = f2b(rng.standard_normal((4, d)).astype(np.float32))
+    a, b = idx.query(q, n_lists, fixed(9)), pool.query(q, fixed(9))
+    assert np.array_equal(a.idx, b.idx) and np.array_equal(a.score, b.score)
+
+
+def test_training_raises_recall_at_one_probe():
+    rng = np.random.default_rng(5)
+    d, n, n_clusters = 48, 3000, 30
+    cent = rng.standard_normal((n_clusters, d))
+    who = rng.integers(0, n_clusters, n)
+    rows = cent[who] + 0.25 * rng.standard_normal((n, d))
+    pool = OraclePool(d)
+    pool.append(f2b(rows.astype(np.float32)), np.arange(n, dtype=np.int32), tag=1)
+    idx = OracleIndex(pool, f2b(rows[:n_clusters].astype(np.float32)))   # a poor start: the first rows
+    q = f2b((cent[rng.integers(0, n_clusters, 40)] + 0.25 * rng.standard_normal((40, d))).astype(np.float32))
+    exact = pool.query(q, fixed(10)).idx
+
+    def recall(ix):
+        got = ix.query(q, 1, fixed(10)).idx
+        return np.mean([len(set(got[i]) & set(exact[i])) / 10 for i in range(40)])
+
+    idx.refresh()
+    r0 = recall(idx)
+    idx.train(5)
+    assert recall(idx) > r0 + 0.1

@@ -1089,6 +1089,22 @@ def run_index(args):
         table.append({"n_probe": n_probe, "us_per_query": us, "queries_per_sec": 1e6 / us,
                       "recall_of_exact_top_k": rec, "speedup_vs_full_scan": full_us / us})
     clocks = sampler.stop()
+    # the same after Lloyd's iterations on the stored rows (oilbird_index_train)
+    n_train = 4
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    ix.train(n_train)
+    torch.cuda.synchronize()
+    train_s = time.perf_counter() - t0
+    _, off_t, _ = ix.read()
+    lens_t = np.diff(off_t)
+    trained = []
+    for n_probe in (1, 4, 16, 64):
+        us = timed(lambda i: ix.query(one[i % n_q], n_probe, pr, out=out))
+        got = ix.query(qs, n_probe, pr).cpu().idx.numpy()
+        rec = float(np.mean([len(set(got[i].tolist()) & set(exact[i].tolist())) / w.k
+                             for i in range(n_q)]))
+        trained.append({"n_probe": n_probe, "us_per_query": us, "recall_of_exact_top_k": rec})
     head = table[2]
     peaks, peak_kind = measured_peaks()
     cand_bytes = (n_lists + 16 * float(lens.mean())) * w.d * 2
@@ -1102,6 +1118,9 @@ def run_index(args):
                        "rows_per_list": {"mean": float(lens.mean()), "max": int(lens.max()),
                                          "empty_lists": int((lens == 0).sum())}},
             "probes": table, "full_scan_us_per_query": full_us,
+            "after_training": {"iterations": n_train, "seconds": train_s, "probes": trained,
+                               "rows_per_list": {"mean": float(lens_t.mean()), "max": int(lens_t.max()),
+                                                 "empty_lists": int((lens_t == 0).sum())}},
             "refresh": {"rows": n0, "seconds": refresh_s, "rows_per_sec": n0 / refresh_s},
             "clocks": clocks, "gpu_launches": 5 * K,
             "roofline": {"bound": "hbm", "kernel": "centroid lookup + candidate scan (n_probe = 16)",

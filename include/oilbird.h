@@ -532,6 +532,19 @@ int64_t oilbird_index_rows(const oilbird_index_t* index);        /* rows that ha
  * list_off[l+1]), in no particular order).  Any pointer may be NULL. */
 int oilbird_index_read(oilbird_index_t* index, int32_t* assign_host, int32_t* list_off_host,
                        int32_t* list_rows_host);
+/*
+ * Training (optional): `iterations` of Lloyd's algorithm on the rows the pool holds now, from
+ * the centroids the index has.  One iteration assigns every row as refresh() does and then
+ * replaces each centroid that has rows by the mean of its rows' stored keys (a centroid
+ * without rows stays).  The mean is taken in fixed point so that it does not depend on the
+ * order of the rows: element x contributes trunc(x * 2^30), the integers are summed exactly,
+ * and the new raw centroid element is bf16(float(double(sum) / (count * 2^30))), rounded to
+ * nearest even twice; the raw centroids are then normalised like any stored row.  Afterwards
+ * the lists are rebuilt over all rows (as reset() + refresh()).  Deterministic.  d <= 8192.
+ * read_centroids copies the raw centroids ([n_lists, d] bf16) to the host (synchronises).
+ */
+int oilbird_index_train(oilbird_index_t* index, int32_t iterations, void* cuda_stream);
+int oilbird_index_read_centroids(oilbird_index_t* index, void* centroids_bf16_host);
 const char* oilbird_index_last_error(void);
 
 /*

@@ -146,6 +146,8 @@ SYMBOLS = {
     "oilbird_index_create": (ctypes.c_int, [ctypes.POINTER(_vp), _vp, _vp, _i32, _vp]),
     "oilbird_index_refresh": (ctypes.c_int, [_vp, _vp]),
     "oilbird_index_reset": (ctypes.c_int, [_vp, _vp]),
+    "oilbird_index_train": (ctypes.c_int, [_vp, _i32, _vp]),
+    "oilbird_index_read_centroids": (ctypes.c_int, [_vp, _vp]),
     "oilbird_index_query": (ctypes.c_int, [_vp, _vp, _i32, _i32, ctypes.POINTER(CQueryParams),
                                            ctypes.POINTER(CQueryOut), _vp]),
     "oilbird_index_destroy": (ctypes.c_int, [_vp]),
@@ -639,6 +641,18 @@ class Index:
 
     def reset(self, stream=None) -> None:
         _check(self._L.oilbird_index_reset(self._h, _stream_ptr(stream)), "oilbird_index_reset")
+
+    def train(self, iterations: int, stream=None) -> None:
+        """Lloyd's iterations on the pool's rows; the lists are rebuilt afterwards."""
+        _check(self._L.oilbird_index_train(self._h, int(iterations), _stream_ptr(stream)),
+               "oilbird_index_train")
+
+    def centroids(self) -> np.ndarray:
+        """The raw centroid states, [n_lists, d] bf16 bit patterns (uint16)."""
+        out = np.empty((self.n_lists, self.pool.d), dtype=np.uint16)
+        _check(self._L.oilbird_index_read_centroids(self._h, out.ctypes.data),
+               "oilbird_index_read_centroids")
+        return out
 
     def query(self, q: torch.Tensor, n_probe: int, params: QueryParams | None = None,
               out: QueryOut | None = None, stream=None) -> QueryOut:

@@ -80,6 +80,60 @@ index_scatter_kernel(const int32_t* __restrict__ assign, int n, const int32_t* _
   }
 }
 
+// ------------------------------------------------------------------- training ---
+// One Lloyd update: block l turns centroid l into the mean of the stored keys of its list
+// (a list without rows keeps its centroid).  Sums are taken in fixed point, element x
+// contributing trunc(x * 2^30), so that they are exact and do not depend on the order in
+// which the scatter kernel happened to place the rows; the new raw element is
+// bf16(float(double(sum) / (count * 2^30))), both roundings to nearest even.
+constexpr int kMeanChunks = 4;          // 16-byte chunks of the row width per thread: d <= 8192
+__global__ void __launch_bounds__(256)
+index_means_kernel(const uint16_t* __restrict__ keys, int d, const int32_t* __restrict__ list_off,
+                   const int32_t* __restrict__ list_rows, uint16_t* __restrict__ cent_raw) {
+  pdl_enter();
+  const int l = blockIdx.x;
+  const int lo = list_off[l], hi = list_off[l + 1];
+  if (hi == lo) return;
+  const int n_chunks = d >> 3;
+  long long acc[kMeanChunks][8];
+#pragma unroll
+  for (int u = 0; u < kMeanChunks; ++u)
+#pragma unroll
+    for (int j = 0; j < 8; ++j) acc[u][j] = 0;
+  for (int i = lo; i < hi; ++i) {
+    const uint4* row = reinterpret_cast<const uint4*>(keys + (size_t)list_rows[i] * d);
+#pragma unroll
+    for (int u = 0; u < kMeanChunks; ++u) {
+      const int c = threadIdx.x + u * 256;
+      if (c < n_chunks) {
+        const uint4 v = __ldg(row + c);
+        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          acc[u][2 * j] += (long long)((double)bf16_lo(w[j]) * 1073741824.0);      // truncates
+          acc[u][2 * j + 1] += (long long)((double)bf16_hi(w[j]) * 1073741824.0);
+        }
+      }
+    }
+  }
+  const double denom = (double)(hi - lo) * 1073741824.0;
+  uint4* dst = reinterpret_cast<uint4*>(cent_raw + (size_t)l * d);
+#pragma unroll
+  for (int u = 0; u < kMeanChunks; ++u) {
+    const int c = threadIdx.x + u * 256;
+    if (c < n_chunks) {
+      uint32_t o[4];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const float a = __double2float_rn(__ll2double_rn(acc[u][2 * j]) / denom);
+        const float b = __double2float_rn(__ll2double_rn(acc[u][2 * j + 1]) / denom);
+        o[j] = f32_to_bf16_bits(a) | (f32_to_bf16_bits(b) << 16);
+      }
+      dst[c] = make_uint4(o[0], o[1], o[2], o[3]);
+    }
+  }
+}
+
 // ------------------------------------------------------------- scan of the candidates ---
 // Grid (G, nq): CTA (b, q) scores a contiguous share of query q's candidates (the rows of its
 // probed lists in probe order, then the tail) and leaves one descending list of KK packed
@@ -189,6 +243,7 @@ cudaError_t preload_index_kernels() {
   if ((e = preload_kernel(index_count_kernel)) != cudaSuccess) return e;
   if ((e = preload_kernel(index_offsets_kernel)) != cudaSuccess) return e;
   if ((e = preload_kernel(index_scatter_kernel)) != cudaSuccess) return e;
+  if ((e = preload_kernel(index_means_kernel)) != cudaSuccess) return e;
   if ((e = preload_kernel(scan_ids_kernel<1>, true)) != cudaSuccess) return e;
   if ((e = preload_kernel(scan_ids_kernel<2>, true)) != cudaSuccess) return e;
   return preload_kernel(scan_ids_kernel<4>, true);
@@ -206,6 +261,7 @@ struct oilbird_index {
   int64_t generation;            // the pool's row numbering the lists refer to
   unsigned char* mem;
   int32_t *assign, *list_rows, *list_off, *cursor, *counts;
+  uint16_t* cent_raw;            // the raw centroid states the centroid pool was built from
   // results of the lookups on the centroids
   int32_t* probe_idx; float* probe_score; int32_t *probe_fired, *probe_len, *probe_tok;
   float* a_score; int32_t *a_fired, *a_len, *a_tok;
@@ -256,7 +312,8 @@ int oilbird_index_create(oilbird_index_t** out, oilbird_pool_t* pool, const void
                o_pt = o_pl + up((size_t)OILBIRD_MAX_NQ * kIndexMaxProbe * 4),
                o_as = o_pt + up((size_t)OILBIRD_MAX_NQ * kIndexMaxProbe * 4),
                o_af = o_as + up(kIndexAssignBatch * 4), o_al = o_af + up(kIndexAssignBatch * 4),
-               o_at = o_al + up(kIndexAssignBatch * 4), total = o_at + up(kIndexAssignBatch * 4);
+               o_at = o_al + up(kIndexAssignBatch * 4), o_raw = o_at + up(kIndexAssignBatch * 4),
+               total = o_raw + up(nl * (size_t)pool->r.d * 2);
   cudaError_t e = cudaMalloc((void**)&ix->mem, total);
   if (e != cudaSuccess) { oilbird_pool_destroy(ix->cent); delete ix; return index_fail(e, "cudaMalloc(index)"); }
   ix->assign = (int32_t*)(ix->mem + o_assign); ix->list_rows = (int32_t*)(ix->mem + o_rows);
@@ -267,12 +324,16 @@ int oilbird_index_create(oilbird_index_t** out, oilbird_pool_t* pool, const void
   ix->probe_tok = (int32_t*)(ix->mem + o_pt);
   ix->a_score = (float*)(ix->mem + o_as); ix->a_fired = (int32_t*)(ix->mem + o_af);
   ix->a_len = (int32_t*)(ix->mem + o_al); ix->a_tok = (int32_t*)(ix->mem + o_at);
+  ix->cent_raw = (uint16_t*)(ix->mem + o_raw);
   cudaStream_t st = (cudaStream_t)cuda_stream;
   // the centroids become the rows of a one-trace pool (their tokens are never looked at);
   // all lists start empty
   e = cudaMemsetAsync(ix->mem, 0, o_pidx, st);
   if (e == cudaSuccess)
-    rc = oilbird_pool_append(ix->cent, centroids_bf16, ix->list_rows, n_lists, 0, OILBIRD_NEW_TRACE, st);
+    e = cudaMemcpyAsync(ix->cent_raw, centroids_bf16, nl * (size_t)pool->r.d * 2,
+                        cudaMemcpyDeviceToDevice, st);
+  if (e == cudaSuccess)
+    rc = oilbird_pool_append(ix->cent, ix->cent_raw, ix->list_rows, n_lists, 0, OILBIRD_NEW_TRACE, st);
   if (e != cudaSuccess || rc) {
     cudaFree(ix->mem); oilbird_pool_destroy(ix->cent); delete ix;
     return e != cudaSuccess ? index_fail(e, "cudaMemsetAsync(index)") : rc;
@@ -342,6 +403,42 @@ int oilbird_index_refresh(oilbird_index_t* ix, void* cuda_stream) {
   if (e != cudaSuccess) return index_fail(e, "index list kernels");
   p->launches += 3;
   ix->n_indexed = n;
+  return OILBIRD_OK;
+}
+
+int oilbird_index_train(oilbird_index_t* ix, int32_t iterations, void* cuda_stream) {
+  if (!ix || iterations < 0) return OILBIRD_EINVAL;
+  oilbird_pool* p = ix->pool;
+  if (p->r.d > kMeanChunks * 256 * 8) return OILBIRD_EINVAL;
+  ICU(cudaSetDevice(p->device));
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  for (int32_t it = 0; it < iterations; ++it) {
+    int rc = oilbird_index_reset(ix, cuda_stream);
+    if (!rc) rc = oilbird_index_refresh(ix, cuda_stream);
+    if (rc) return rc;
+    if (ix->n_indexed == 0) break;                     // no rows: nothing to learn from
+    cudaError_t e = launch_pdl(index_means_kernel, dim3(ix->n_lists), dim3(256), 0, st,
+                               (const uint16_t*)p->keys, (int)p->r.d, (const int32_t*)ix->list_off,
+                               (const int32_t*)ix->list_rows, ix->cent_raw);
+    if (e != cudaSuccess) return index_fail(e, "index means kernel");
+    p->launches += 1;
+    // the centroid pool, rebuilt from the new raw states (tokens are never looked at)
+    rc = oilbird_pool_reset(ix->cent, cuda_stream);
+    if (!rc)
+      rc = oilbird_pool_append(ix->cent, ix->cent_raw, ix->cursor, ix->n_lists, 0, OILBIRD_NEW_TRACE,
+                               cuda_stream);
+    if (rc) return rc;
+  }
+  int rc = oilbird_index_reset(ix, cuda_stream);
+  return rc ? rc : oilbird_index_refresh(ix, cuda_stream);
+}
+
+int oilbird_index_read_centroids(oilbird_index_t* ix, void* centroids_bf16_host) {
+  if (!ix || !centroids_bf16_host) return OILBIRD_EINVAL;
+  ICU(cudaSetDevice(ix->pool->device));
+  ICU(cudaDeviceSynchronize());
+  ICU(cudaMemcpy(centroids_bf16_host, ix->cent_raw, (size_t)ix->n_lists * ix->pool->r.d * 2,
+                 cudaMemcpyDeviceToHost));
   return OILBIRD_OK;
 }
 

@@ -177,3 +177,64 @@ def test_bad_arguments_are_refused():
         ix.query(q, 0, fixed(4, 2))                          # at least one probe
     out = ix.query(q, 2, fixed(4, 2)).cpu()                  # an empty pool is legal
     assert torch.all(out.idx == -1) and out.fired[0] == 0
+
+
+def test_training_matches_the_oracle_bit_for_bit():
+    """Lloyd's iterations: raw centroids, assignments and lists identical to the oracle's after
+    one, two and five iterations (one starting centroid in each cluster of the recipe, so
+    that no row sits between two centroids), then answers under the acceptance rule."""
+    w = W.C1.scaled(n_rows=6000, nq=6, d=256, n_centroids=24, rows_per_trace=500, seed=31)
+    pool, ora = fill_both(w, max_nq=16)
+    assign = np.concatenate([w.trace_assign(t, "cuda").cpu().numpy() for t in range(w.num_traces)])[: w.n_rows]
+    first = [int(np.nonzero(assign == c)[0][0]) for c in range(24)]      # one row of every cluster
+    keys_raw = torch.cat([st for st, _, _ in w.traces("cuda")])[: w.n_rows]
+    cent = keys_raw[first].contiguous()
+    gix, oix = B.Index(pool, cent), OracleIndex(ora, W.to_bits(cent))
+    assert np.array_equal(gix.centroids(), oix.cent_raw)
+    done = 0
+    for upto in (1, 2, 5):
+        gix.train(upto - done)
+        oix.train(upto - done)
+        done = upto
+        assert np.array_equal(gix.centroids(), oix.cent_raw)
+        same_lists(gix, oix)
+        assert len(gix) == len(pool)
+    q, _ = w.queries("cuda")
+    for n_probe in (1, 3, 24):
+        pr = fixed(8, 4)
+        check_index_query(gix.query(q, n_probe, pr), oix, W.to_bits(q), n_probe, pr)
+    # zero iterations only rebuild the lists; an empty pool has nothing to learn from
+    gix.train(0)
+    same_lists(gix, oix)
+    empty = B.Pool(w.d, 64)
+    eix = B.Index(empty, cent)
+    eix.train(3)
+    assert len(eix) == 0 and np.array_equal(eix.centroids(), W.to_bits(cent))
+
+
+def test_training_on_fewer_lists_than_clusters_keeps_the_index_exact_and_helps_recall():
+    w = W.C1.scaled(n_rows=20000, nq=32, k=8, d=128, n_centroids=96, rows_per_trace=1000, seed=32)
+    pool, ora, gix, oix = build_both(w, 20, seed=3, max_nq=32)
+    q, _ = w.queries("cuda")
+    pr = fixed(8, 4)
+    exact = pool.query(q, fixed(8, 4, path=B.PATH_GEMV)).cpu()    # (the index scores on the CUDA cores)
+    gix.refresh()
+
+    def recall(n_probe):
+        got = gix.query(q, n_probe, pr).cpu().idx.numpy()
+        return float(np.mean([len(set(got[i]) & set(exact.idx[i].tolist())) / 8 for i in range(32)]))
+
+    r_before = recall(1)
+    gix.train(6)
+    a, off, rows = gix.read()
+    assert len(gix) == len(pool) and off[-1] == len(pool)
+    assert sorted(rows.tolist()) == list(range(len(pool)))             # a partition of the rows
+    full = gix.query(q, 20, pr).cpu()                                   # every list probed: the full scan
+    assert torch.equal(full.idx, exact.idx) and torch.equal(full.score, exact.score)
+    assert recall(1) >= r_before - 0.02
+    # the same training twice gives the same centroids (nothing depends on scheduling)
+    c1 = gix.centroids()
+    pool2, _, gix2, _ = build_both(w, 20, seed=3, max_nq=32)
+    gix2.train(6)
+    assert np.array_equal(c1, gix2.centroids())
+    assert pool.stats()["stalled"] == 0

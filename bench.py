@@ -1079,11 +1079,7 @@ def run_index(args):
     sampler = ClockSampler(physical_device(0))
     sampler.start()
     for n_probe in (1, 4, 16, 64):
-        if n_probe == 16:
-            torch.cuda.cudart().cudaProfilerStart()     # lets a profiler capture the headline loop only
         us = timed(lambda i: ix.query(one[i % n_q], n_probe, pr, out=out))
-        if n_probe == 16:
-            torch.cuda.cudart().cudaProfilerStop()
         got = ix.query(qs, n_probe, pr).cpu().idx.numpy()
         rec = float(np.mean([len(set(got[i].tolist()) & set(exact[i].tolist())) / w.k
                              for i in range(n_q)]))
@@ -1101,7 +1097,11 @@ def run_index(args):
     lens_t = np.diff(off_t)
     trained = []
     for n_probe in (1, 4, 16, 64):
+        if n_probe == 4:
+            torch.cuda.cudart().cudaProfilerStart()     # lets a profiler capture the headline loop only
         us = timed(lambda i: ix.query(one[i % n_q], n_probe, pr, out=out))
+        if n_probe == 4:
+            torch.cuda.cudart().cudaProfilerStop()
         got = ix.query(qs, n_probe, pr).cpu().idx.numpy()
         rec = float(np.mean([len(set(got[i].tolist()) & set(exact[i].tolist())) / w.k
                              for i in range(n_q)]))

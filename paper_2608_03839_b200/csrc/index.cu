@@ -476,7 +476,15 @@ int oilbird_index_query(oilbird_index_t* ix, const void* q_bf16, int32_t nq, int
   if (rc) return rc;
   // scan the candidates, merge, fire, gather
   const int kk = list_len(pr->k);
+  // blocks per query: all the SMs twice over for a single lookup (a block holds a few rows
+  // and the lookup is latency-bound), fewer per query as the batch grows (every block
+  // prepares its query first, which a batch would otherwise pay thousands of times over)
   int grid = 2 * p->num_sms;
+  if (nq > 1) {
+    grid = (8 * p->num_sms + nq - 1) / nq;
+    if (grid < 8) grid = 8;
+    if (grid > 2 * p->num_sms) grid = 2 * p->num_sms;
+  }
   if (grid > p->r.max_lists) grid = p->r.max_lists;
   PoolView pv = pool_view(p);
   cudaError_t e;

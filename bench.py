@@ -1106,6 +1106,18 @@ def run_index(args):
         rec = float(np.mean([len(set(got[i].tolist()) & set(exact[i].tolist())) / w.k
                              for i in range(n_q)]))
         trained.append({"n_probe": n_probe, "us_per_query": us, "recall_of_exact_top_k": rec})
+    # lookups in batches (four probes, trained): the queries of concurrent requests together
+    batches = []
+    for nq_b in (8, 64):
+        qb = qs[:nq_b].contiguous()
+        out_b = B.QueryOut.empty(nq_b, w.k, w.cont_len, dev)
+        us = timed(lambda i: ix.query(qb, 4, pr, out=out_b))
+        full_b = timed(lambda i: pool.query(qb, pr, out=out_b))
+        got = ix.query(qb, 4, pr).cpu().idx.numpy()
+        rec = float(np.mean([len(set(got[i].tolist()) & set(exact[i].tolist())) / w.k
+                             for i in range(nq_b)]))
+        batches.append({"nq": nq_b, "n_probe": 4, "us_per_batch": us, "lookups_per_sec": nq_b * 1e6 / us,
+                        "recall_of_exact_top_k": rec, "full_scan_us_per_batch": full_b})
     head = dict(trained[1])                      # four probes after training
     head["queries_per_sec"] = 1e6 / head["us_per_query"]
     peaks, peak_kind = measured_peaks()
@@ -1123,6 +1135,7 @@ def run_index(args):
             "recall_of_exact_top_k": head["recall_of_exact_top_k"],
             "speedup_vs_full_scan": full_us / head["us_per_query"],
             "probes": table, "full_scan_us_per_query": full_us,
+            "batches_after_training": batches,
             "after_training": {"iterations": n_train, "seconds": train_s, "probes": trained,
                                "rows_per_list": {"mean": float(lens_t.mean()), "max": int(lens_t.max()),
                                                  "empty_lists": int((lens_t == 0).sum())}},

@@ -796,8 +796,11 @@ def run_ring(args):
     torch.cuda.synchronize()
 
     def step(i):
-        ring.append(*steps_in[i % n_in])
-        ring.query(qs[i % n_in][0], qs[i % n_in][1], m=4, floor=0.8, out=out)
+        if args.path == 9:                      # (comparison: the two calls of their own)
+            ring.append(*steps_in[i % n_in])
+            ring.query(qs[i % n_in][0], qs[i % n_in][1], m=4, floor=0.8, out=out)
+        else:
+            ring.step(*steps_in[i % n_in], qs[i % n_in][0], qs[i % n_in][1], m=4, floor=0.8, out=out)
 
     for i in range(Wm):
         step(i)
@@ -849,7 +852,7 @@ def run_ring(args):
                                    f"{vocab} tokens (~{matches:.0f} matching records)"},
             "p50_step_latency_us": float(np.percentile(lat, 50)) * 1e3,
             "lookup_us": look_ms * 1e3, "append_us": app_ms * 1e3, "clocks": clocks,
-            "gpu_launches": 3 * K,
+            "gpu_launches": (3 if args.path == 9 else 2) * K,
             "roofline": {"bound": "hbm", "kernel": "ring lookup (anchor filter + matching keys)",
                          "achieved": look_bytes / (look_ms * 1e-3) / 1e9, "peak": peaks["hbm_gbs"],
                          "unit": "GB/s", "frac": look_bytes / (look_ms * 1e-3) / 1e9 / peaks["hbm_gbs"],

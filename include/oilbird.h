@@ -414,6 +414,18 @@ int oilbird_ring_append(oilbird_ring_t* ring, const void* states_bf16, const int
 int oilbird_ring_query(oilbird_ring_t* ring, const void* q_bf16, const int32_t* q_anchor,
                        int32_t nq, int32_t m, float floor, const oilbird_ring_out* out,
                        void* cuda_stream);
+/*
+ * One verification pass in one call: oilbird_ring_append of n records (n may be 0) followed by
+ * oilbird_ring_query, with the same results as the two calls.  The lookup's own kernel stores
+ * the records before it scans (its first blocks take one record each; warps that reach a slot
+ * written by the call wait, bounded, until all records are in), so the pass is two launches
+ * instead of three; where the lookup needs more blocks than the GPU seats at once the append
+ * gets a launch of its own.
+ */
+int oilbird_ring_step(oilbird_ring_t* ring, const void* states_bf16, const int32_t* anchors,
+                      const int32_t* rollouts, int64_t n, const void* q_bf16,
+                      const int32_t* q_anchor, int32_t nq, int32_t m, float floor,
+                      const oilbird_ring_out* out, void* cuda_stream);
 /* Copy stored records to the host (synchronous; tests and debugging). */
 int oilbird_ring_read(oilbird_ring_t* ring, void* keys_host, int32_t* anchors_host,
                       int32_t* rollouts_host);

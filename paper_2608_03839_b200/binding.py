@@ -131,6 +131,8 @@ SYMBOLS = {
     "oilbird_ring_append": (ctypes.c_int, [_vp, _vp, _vp, _vp, _i64, _vp]),
     "oilbird_ring_query": (ctypes.c_int, [_vp, _vp, _vp, _i32, _i32, ctypes.c_float,
                                           ctypes.POINTER(CRingOut), _vp]),
+    "oilbird_ring_step": (ctypes.c_int, [_vp, _vp, _vp, _vp, _i64, _vp, _vp, _i32, _i32,
+                                         ctypes.c_float, ctypes.POINTER(CRingOut), _vp]),
     "oilbird_ring_read": (ctypes.c_int, [_vp, _vp, _vp, _vp]),
     "oilbird_ring_last_error": (ctypes.c_char_p, []),
     "oilbird_pool_append_global": (ctypes.c_int, [_vp, _vp, _vp, _i64, _u64, _u32, _i64, _vp]),
@@ -759,6 +761,33 @@ class Ring:
         _check(self._L.oilbird_ring_query(self._h, q.data_ptr(), anchors.data_ptr(), nq, int(m),
                                           float(floor), ctypes.byref(co), _stream_ptr(stream)),
                "oilbird_ring_query")
+        return out
+
+    def step(self, states: torch.Tensor, anchors: torch.Tensor, rollouts: torch.Tensor,
+             q: torch.Tensor, q_anchors: torch.Tensor, m: int = 4, floor: float = 0.8,
+             out: RingOut | None = None, stream=None) -> RingOut:
+        """One verification pass: append the records, then look up, in one call."""
+        n = int(anchors.shape[0])
+        assert states.is_cuda and states.dtype == torch.bfloat16 and states.is_contiguous()
+        assert anchors.is_cuda and anchors.dtype == torch.int32 and anchors.is_contiguous()
+        assert rollouts.is_cuda and rollouts.dtype == torch.int32 and rollouts.is_contiguous()
+        assert states.shape == (n, self.d) and rollouts.shape == (n, self.max_rollout)
+        assert q.is_cuda and q.dtype == torch.bfloat16 and q.is_contiguous()
+        q = q.reshape(-1, self.d)
+        nq = q.shape[0]
+        assert q_anchors.is_cuda and q_anchors.dtype == torch.int32 and q_anchors.numel() == nq
+        if out is None:
+            out = RingOut(ALLOC((nq, m), torch.int32, self._dev),
+                          ALLOC((nq, m), torch.float32, self._dev),
+                          ALLOC((nq,), torch.int32, self._dev),
+                          ALLOC((nq, m, self.max_rollout), torch.int32, self._dev),
+                          ALLOC((nq, m), torch.int32, self._dev))
+        co = CRingOut(out.slot.data_ptr(), out.score.data_ptr(), out.count.data_ptr(),
+                      out.rollout.data_ptr(), out.rollout_len.data_ptr())
+        _check(self._L.oilbird_ring_step(self._h, states.data_ptr(), anchors.data_ptr(),
+                                         rollouts.data_ptr(), n, q.data_ptr(), q_anchors.data_ptr(),
+                                         nq, int(m), float(floor), ctypes.byref(co),
+                                         _stream_ptr(stream)), "oilbird_ring_step")
         return out
 
     def read(self):

@@ -40,12 +40,29 @@ ring_append_kernel(const uint16_t* __restrict__ states, const int32_t* __restric
   }
 }
 
-// grid (slices, nq): CTA (s, q) scans slots [lo, hi) of the ring for query q.
+// The records of a step that the lookup's own kernel stores before it scans (oilbird_ring_step):
+// n = 0 for a plain lookup.
+struct RingFused {
+  const uint16_t* states;
+  const int32_t *anchors, *rollouts;
+  int32_t* rollout;              // the ring's continuations (written here, read by the merge)
+  int n, R;
+  int64_t start, cap;            // record r goes to slot (start + r) % cap
+  unsigned long long* ready;     // += 1 per stored record
+  unsigned long long target;     // *ready once all n are in
+};
+
+// grid (slices, nq): CTA (s, q) scans slots [lo, hi) of the ring for query q.  With fused
+// records the CTAs first store them, one record per CTA and round (all CTAs of the launch are
+// resident together: at most two per SM are launched), and a warp whose 32 slots include a
+// slot written by this launch waits, bounded, until all of them are in and reads those
+// slots' anchors and keys through L2.
 __global__ void __launch_bounds__(kRingThreads, 2)
-ring_scan_kernel(const uint16_t* __restrict__ keys, const int32_t* __restrict__ anchor,
+ring_scan_kernel(uint16_t* __restrict__ keys, int32_t* __restrict__ anchor,
                  int64_t n_slots, int d, const uint16_t* __restrict__ q_raw,
                  const int32_t* __restrict__ q_anchor, int nq, int m, float floor_s,
-                 u64* __restrict__ partial, int32_t* __restrict__ q_valid, DeviceStats* stats) {
+                 u64* __restrict__ partial, int32_t* __restrict__ q_valid, DeviceStats* stats,
+                 RingFused fa) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   const int n_chunks = d >> 3;
   uint4* qs = reinterpret_cast<uint4*>(smem_raw);                           // [n_chunks]
@@ -53,6 +70,29 @@ ring_scan_kernel(const uint16_t* __restrict__ keys, const int32_t* __restrict__ 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int q = blockIdx.y;
   pdl_enter();
+  if (fa.n > 0) {
+    const int n_blocks = gridDim.x * gridDim.y, b = blockIdx.y * gridDim.x + blockIdx.x;
+    for (int r = b; r < fa.n; r += n_blocks) {
+      const int64_t slot = (fa.start + r) % fa.cap;
+      normalize_row(fa.states + (size_t)r * d, keys + slot * d, d);
+      if (threadIdx.x == 0) anchor[slot] = fa.anchors[r];
+      if (threadIdx.x < fa.R) fa.rollout[slot * fa.R + threadIdx.x] = fa.rollouts[(size_t)r * fa.R + threadIdx.x];
+      __threadfence();                   // this thread's part of the record, before the count
+      __syncthreads();
+      if (threadIdx.x == 0) {
+        __threadfence();                 // cumulative: the whole CTA's record
+        atomicAdd(fa.ready, 1ull);
+      }
+    }
+  }
+  bool fresh_ok = fa.n == 0;             // this warp has seen the step's records arrive
+  // slots written by this launch: [f0, f0 + n) modulo the ring's capacity
+  const int64_t f0 = fa.n > 0 ? fa.start % fa.cap : 0;
+  auto fresh = [&](int64_t slot) {
+    if (fa.n == 0) return false;
+    const int64_t off = slot >= f0 ? slot - f0 : slot + fa.cap - f0;
+    return off < fa.n;
+  };
   const int code = normalize_row<false>(q_raw + (size_t)q * d, reinterpret_cast<uint16_t*>(qs), d);
   if (blockIdx.x == 0 && threadIdx.x == 0) {
     q_valid[q] = code == kRowNonFinite ? 0 : 1;
@@ -67,17 +107,26 @@ ring_scan_kernel(const uint16_t* __restrict__ keys, const int32_t* __restrict__ 
   u64 kth = 0;
   for (int64_t base = lo + warp * 32; base < hi; base += kRingWarps * 32) {
     const int64_t slot = base + lane;
-    const bool hit = slot < hi && anchor[slot] == xq;          // anchor token must be equal
+    const bool mine_fresh = slot < hi && fresh(slot);
+    const bool any_fresh = __any_sync(0xffffffffu, mine_fresh);
+    if (any_fresh && !fresh_ok) {
+      wait_fused_rows(fa.ready, fa.target, stats);
+      fresh_ok = true;
+    }
+    const int a_slot = slot < hi ? (mine_fresh ? __ldcg(&anchor[slot]) : anchor[slot]) : 0;
+    const bool hit = slot < hi && a_slot == xq;                // anchor token must be equal
     unsigned mask = __ballot_sync(0xffffffffu, hit);
+    const unsigned fresh_mask = __ballot_sync(0xffffffffu, mine_fresh);
     while (mask) {
       const int src = __ffs(mask) - 1;
       mask &= mask - 1;
       const int64_t s_row = base + src;
       const uint4* rowp = keys4 + (size_t)s_row * n_chunks;
+      const bool row_fresh = (fresh_mask >> src) & 1u;           // warp-uniform
       float acc = 0.f;
 #pragma unroll 4
       for (int c = lane; c < n_chunks; c += 32) {
-        const uint4 kv = ld_stream16(rowp + c);
+        const uint4 kv = row_fresh ? ld_cg16(rowp + c) : ld_stream16(rowp + c);
         const uint4 qv = qs[c];
         acc = fmaf(bf16_lo(kv.x), bf16_lo(qv.x), acc);
         acc = fmaf(bf16_hi(kv.x), bf16_hi(qv.x), acc);
@@ -169,6 +218,8 @@ struct oilbird_ring {
   int32_t *anchor, *rollout, *q_valid;
   unsigned long long* partial;
   DeviceStats* stats;
+  unsigned long long* ready;       // records stored by lookups that append (device counter) ...
+  unsigned long long ready_target; // ... and the host's count of them (enqueue time)
   unsigned char* base;
 };
 
@@ -198,7 +249,7 @@ int oilbird_ring_create(oilbird_ring_t** out, const oilbird_ring_config* cfg) {
                o_valid = o_roll + up((size_t)r->cap * r->R * 4),
                o_part = o_valid + up((size_t)OILBIRD_RING_MAX_NQ * 4),
                o_stats = o_part + up((size_t)r->max_lists * OILBIRD_RING_MAX_NQ * kRingList * 8),
-               total = o_stats + up(sizeof(DeviceStats));
+               o_ready = o_stats + up(sizeof(DeviceStats)), total = o_ready + 256;
   void* mem = nullptr;
   cudaError_t e = cudaMalloc(&mem, total);
   if (e != cudaSuccess) { delete r; return ring_fail(e, "cudaMalloc(ring)"); }
@@ -209,7 +260,9 @@ int oilbird_ring_create(oilbird_ring_t** out, const oilbird_ring_config* cfg) {
   r->q_valid = (int32_t*)(r->base + o_valid);
   r->partial = (unsigned long long*)(r->base + o_part);
   r->stats = (DeviceStats*)(r->base + o_stats);
-  e = cudaMemset(r->stats, 0, sizeof(DeviceStats));
+  r->ready = (unsigned long long*)(r->base + o_ready);
+  r->ready_target = 0;
+  e = cudaMemset(r->stats, 0, o_ready + 256 - o_stats);       // counters and the fused-store counter
   if (e != cudaSuccess) { cudaFree(mem); delete r; return ring_fail(e, "cudaMemset"); }
   *out = r;
   return OILBIRD_OK;
@@ -256,8 +309,11 @@ int oilbird_ring_append(oilbird_ring_t* r, const void* states, const int32_t* an
   return OILBIRD_OK;
 }
 
-int oilbird_ring_query(oilbird_ring_t* r, const void* q, const int32_t* q_anchor, int32_t nq,
-                       int32_t m, float floor_s, const oilbird_ring_out* out, void* stream) {
+// Lookup, optionally with the records of a step stored by the scan kernel itself.
+static int ring_query_impl(oilbird_ring_t* r, const void* q, const int32_t* q_anchor, int32_t nq,
+                           int32_t m, float floor_s, const oilbird_ring_out* out, void* stream,
+                           const void* states, const int32_t* anchors, const int32_t* rollouts,
+                           int64_t n) {
   if (!r || !q || !q_anchor || !out || !out->slot || !out->score || !out->count ||
       !out->rollout || !out->rollout_len)
     return OILBIRD_EINVAL;
@@ -265,21 +321,51 @@ int oilbird_ring_query(oilbird_ring_t* r, const void* q, const int32_t* q_anchor
     return OILBIRD_EINVAL;
   RCU(cudaSetDevice(r->device));
   cudaStream_t st = (cudaStream_t)stream;
-  const int64_t n_slots = oilbird_ring_size(r);
+  const int64_t total_after = r->total + n;
+  const int64_t n_slots = total_after < r->cap ? total_after : r->cap;
   // at least 256 slots per CTA, at most two CTAs per SM
   int64_t want = (n_slots + 255) / 256;
   int slices = (int)(want < 1 ? 1 : (want > r->max_lists ? r->max_lists : want));
+  RingFused fa = {};
+  if (n > 0) {
+    // the scan's own blocks store the records: they must all be resident together, because
+    // scanning warps wait for the storing ones (else: a launch of its own for the append)
+    if ((int64_t)slices * nq > 2 * r->num_sms || n > r->cap) {
+      int rc = oilbird_ring_append(r, states, anchors, rollouts, n, stream);
+      if (rc) return rc;
+      return ring_query_impl(r, q, q_anchor, nq, m, floor_s, out, stream, nullptr, nullptr, nullptr, 0);
+    }
+    fa.states = (const uint16_t*)states; fa.anchors = anchors; fa.rollouts = rollouts;
+    fa.rollout = r->rollout; fa.n = (int)n; fa.R = r->R; fa.start = r->total; fa.cap = r->cap;
+    fa.ready = r->ready; fa.target = r->ready_target + (unsigned long long)n;
+  }
   const size_t smem = (size_t)r->d * 2 + (size_t)kRingWarps * kRingList * sizeof(u64);
   cudaError_t e = launch_pdl(ring_scan_kernel, dim3(slices, nq), dim3(kRingThreads), smem, st,
-                             (const uint16_t*)r->keys, (const int32_t*)r->anchor, n_slots, r->d,
-                             (const uint16_t*)q, q_anchor, nq, m, floor_s, r->partial, r->q_valid,
-                             r->stats);
+                             r->keys, r->anchor, n_slots, r->d, (const uint16_t*)q, q_anchor, nq, m,
+                             floor_s, r->partial, r->q_valid, r->stats, fa);
   if (e != cudaSuccess) return ring_fail(e, "ring scan launch");
+  if (n > 0) {
+    r->total = total_after;
+    r->ready_target = fa.target;
+  }
   e = launch_pdl(ring_merge_kernel, dim3(nq), dim3(kMergeThreads), 0, st,
                  (const u64*)r->partial, slices, nq, m, r->R, (const int32_t*)r->q_valid,
                  (const int32_t*)r->rollout, *out);
   if (e != cudaSuccess) return ring_fail(e, "ring merge launch");
   return OILBIRD_OK;
+}
+
+int oilbird_ring_query(oilbird_ring_t* r, const void* q, const int32_t* q_anchor, int32_t nq,
+                       int32_t m, float floor_s, const oilbird_ring_out* out, void* stream) {
+  return ring_query_impl(r, q, q_anchor, nq, m, floor_s, out, stream, nullptr, nullptr, nullptr, 0);
+}
+
+int oilbird_ring_step(oilbird_ring_t* r, const void* states, const int32_t* anchors,
+                      const int32_t* rollouts, int64_t n, const void* q, const int32_t* q_anchor,
+                      int32_t nq, int32_t m, float floor_s, const oilbird_ring_out* out,
+                      void* stream) {
+  if (n < 0 || (n > 0 && (!states || !anchors || !rollouts))) return OILBIRD_EINVAL;
+  return ring_query_impl(r, q, q_anchor, nq, m, floor_s, out, stream, states, anchors, rollouts, n);
 }
 
 int oilbird_ring_read(oilbird_ring_t* r, void* keys, int32_t* anchors, int32_t* rollouts) {

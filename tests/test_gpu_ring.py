@@ -132,3 +132,41 @@ def test_more_records_than_slots_in_one_append_and_reset():
     assert out.count[0] == 0                      # a NaN query finds nothing
     with pytest.raises(B.OilbirdError):
         ring.query(st[:1].contiguous(), anc[:1].contiguous(), m=33)
+
+
+@pytest.mark.parametrize("d,cap,vocab,nq", [(256, 1000, 5, 1), (4096, 8192, 40, 1), (512, 257, 3, 4),
+                                             (1024, 90000, 6, 1), (128, 40000, 4, 8)])
+def test_steps_that_store_and_look_up_in_one_call(d, cap, vocab, nq):
+    """oilbird_ring_step = append + query: the stored ring and every answer equal the oracle's
+    after the same append; the query of a step looks for one of the step's own records (it
+    must come back first); rings that wrap, steps of 0, 1, 64 and more records than blocks, and
+    a lookup that needs more blocks than fit at once (its append then gets a launch of its own)."""
+    ring, ora = B.Ring(d, cap), OracleRing(d, cap)
+    cent, st, anc, roll = ring_inputs(cap + 1500, d, vocab, seed=7 + d + nq)
+    # most of the ring first, in bulk; then steps across the wrap-around
+    bulk = max(0, cap - 300)
+    ring.append(st[:bulk].contiguous(), anc[:bulk].contiguous(), roll[:bulk].contiguous())
+    ora.append(W.to_bits(st[:bulk]), anc[:bulk].cpu().numpy(), roll[:bulk].cpu().numpy())
+    g = torch.Generator(device="cuda").manual_seed(5)
+    pos = bulk
+    for n in (64, 0, 1, 64, 333, 64, 7, 64, 700):
+        s_, a_, r_ = st[pos:pos + n].contiguous(), anc[pos:pos + n].contiguous(), roll[pos:pos + n].contiguous()
+        q = (cent[:nq] + 0.3 * torch.randn(nq, d, generator=g, device="cuda")).to(torch.bfloat16)
+        qa = torch.randint(0, vocab, (nq,), generator=g, device="cuda", dtype=torch.int32)
+        if n:
+            q[0] = s_[n - 1]                      # a record stored by this very call
+            qa[0] = a_[n - 1]
+        out = ring.step(s_, a_, r_, q, qa, m=4, floor=0.5)
+        ora.append(W.to_bits(s_), a_.cpu().numpy(), r_.cpu().numpy())
+        pos += n
+        assert len(ring) == len(ora) and ring.total == pos
+        check(out, ora, W.to_bits(q), qa.cpu().numpy(), 4, 0.5)
+        if n:
+            assert int(out.slot[0, 0]) == (pos - 1) % cap
+    keys, a2, r2 = ring.read()
+    assert np.array_equal(keys, ora.keys) and np.array_equal(a2, ora.anchors)
+    assert np.array_equal(r2, ora.rollouts)
+    # a plain lookup afterwards sees the same ring
+    q = (cent[:nq] + 0.3 * torch.randn(nq, d, generator=g, device="cuda")).to(torch.bfloat16)
+    qa = torch.randint(0, vocab, (nq,), generator=g, device="cuda", dtype=torch.int32)
+    check(ring.query(q, qa, m=8, floor=-2.0), ora, W.to_bits(q), qa.cpu().numpy(), 8, -2.0)

@@ -852,7 +852,7 @@ def run_ring(args):
                                    f"{vocab} tokens (~{matches:.0f} matching records)"},
             "p50_step_latency_us": float(np.percentile(lat, 50)) * 1e3,
             "lookup_us": look_ms * 1e3, "append_us": app_ms * 1e3, "clocks": clocks,
-            "gpu_launches": (3 if args.path == 9 else 2) * K,
+            "gpu_launches": (2 if args.path == 9 else 1) * K,
             "roofline": {"bound": "hbm", "kernel": "ring lookup (anchor filter + matching keys)",
                          "achieved": look_bytes / (look_ms * 1e-3) / 1e9, "peak": peaks["hbm_gbs"],
                          "unit": "GB/s", "frac": look_bytes / (look_ms * 1e-3) / 1e9 / peaks["hbm_gbs"],

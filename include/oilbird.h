@@ -418,9 +418,10 @@ int oilbird_ring_query(oilbird_ring_t* ring, const void* q_bf16, const int32_t* 
  * One verification pass in one call: oilbird_ring_append of n records (n may be 0) followed by
  * oilbird_ring_query, with the same results as the two calls.  The lookup's own kernel stores
  * the records before it scans (its first blocks take one record each; warps that reach a slot
- * written by the call wait, bounded, until all records are in), so the pass is two launches
- * instead of three; where the lookup needs more blocks than the GPU seats at once the append
- * gets a launch of its own.
+ * written by the call wait, bounded, until all records are in), and the last block of a query
+ * to finish merges the blocks' candidates and writes the answer, so the pass is one launch
+ * (a plain oilbird_ring_query likewise); where the lookup needs more blocks than the GPU seats
+ * at once the append gets a launch of its own.
  */
 int oilbird_ring_step(oilbird_ring_t* ring, const void* states_bf16, const int32_t* anchors,
                       const int32_t* rollouts, int64_t n, const void* q_bf16,

@@ -10,7 +10,9 @@
 // anchor tokens (4 bytes per slot, coalesced) and streams the 16-byte key chunks of the
 // matching slots only, so its traffic is capacity*4 + matches*d*2 bytes instead of the
 // whole ring; each warp keeps its best records in a sorted register list, CTAs publish
-// one list each and a second kernel merges them and copies the continuations out.
+// one list each, and the last CTA of a query to finish merges them and copies the
+// continuations out (no second launch).  oilbird_ring_step also stores the records of a
+// verification pass inside the same launch.
 #include <math.h>
 #include <stdio.h>
 
@@ -62,7 +64,8 @@ ring_scan_kernel(uint16_t* __restrict__ keys, int32_t* __restrict__ anchor,
                  int64_t n_slots, int d, const uint16_t* __restrict__ q_raw,
                  const int32_t* __restrict__ q_anchor, int nq, int m, float floor_s,
                  u64* __restrict__ partial, int32_t* __restrict__ q_valid, DeviceStats* stats,
-                 RingFused fa) {
+                 RingFused fa, unsigned* __restrict__ done, const int32_t* __restrict__ rollout,
+                 int R, oilbird_ring_out out) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   const int n_chunks = d >> 3;
   uint4* qs = reinterpret_cast<uint4*>(smem_raw);                           // [n_chunks]
@@ -148,39 +151,63 @@ ring_scan_kernel(uint16_t* __restrict__ keys, int32_t* __restrict__ anchor,
     }
   }
   block_merge_desc<1>(top, scratch, kRingWarps);
-  if (threadIdx.x < 32) partial[((size_t)blockIdx.x * nq + q) * kRingList + lane] = top[0];
-}
+  if (threadIdx.x < 32) __stcg(&partial[((size_t)blockIdx.x * nq + q) * kRingList + lane], top[0]);
 
-__global__ void __launch_bounds__(kMergeThreads)
-ring_merge_kernel(const u64* __restrict__ partial, int n_lists, int nq, int m, int R,
-                  const int32_t* __restrict__ q_valid, const int32_t* __restrict__ rollout,
-                  oilbird_ring_out out) {
-  __shared__ u64 scratch[kMergeWarps * kRingList];
+  // The last block of a query to get here merges the blocks' lists and writes the answer:
+  // no launch of its own for that (a lookup moves under a megabyte and is bound by launch
+  // latency; as a second kernel the merge cost a pass 5-6 us).
+  __shared__ int s_last;
   __shared__ u64 s_best[kRingList];
-  const int q = blockIdx.x;
-  pdl_enter();
-  const int lists = q_valid[q] != 0 ? n_lists : 0;
-  // no head filter here: the lookup moves under 1 MB and is bound by launch latency; with
-  // the filter's two extra barriers an append + lookup step was measured 4.5 us slower
-  merge_lists<1>(partial, lists, nq, q, 0, scratch, s_best);
+  __threadfence();                       // this block's list (and any record it stored)
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    const unsigned prev = atomicAdd(&done[q], 1u);
+    s_last = prev == gridDim.x - 1;
+    if (s_last) done[q] = 0;             // everybody has arrived: ready for the next launch
+  }
+  __syncthreads();
+  if (!s_last) return;
+  __threadfence();                       // the other blocks' lists, published before their arrival
+  u64 v[1] = {0};
+  if (code != kRowNonFinite) {           // a NaN/Inf query finds nothing
+    // most blocks found nothing (a few dozen records match among hundreds of blocks): a warp
+    // first looks at the heads of 32 lists at once, then fetches the lists that hold
+    // something four at a time
+    for (int l0 = warp * 32; l0 < (int)gridDim.x; l0 += kRingWarps * 32) {
+      const int l = l0 + lane;
+      const u64 head = l < (int)gridDim.x ? __ldcg(&partial[((size_t)l * nq + q) * kRingList]) : 0;
+      unsigned live = __ballot_sync(0xffffffffu, head != 0);
+      while (live) {
+        u64 b[4][1];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          const int src = live ? __ffs(live) - 1 : -1;
+          if (live) live &= live - 1;
+          b[u][0] = src >= 0 ? __ldcg(&partial[((size_t)(l0 + src) * nq + q) * kRingList + lane]) : 0;
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) warp_merge_desc<1>(v, b[u], lane);
+      }
+    }
+  }
+  block_merge_desc<1>(v, scratch, kRingWarps);
+  if (threadIdx.x < 32) s_best[lane] = v[0];
+  __syncthreads();
   if (threadIdx.x == 0) {
     int c = 0;
     while (c < m && s_best[c] != 0) ++c;
     out.count[q] = c;
   }
-  __syncthreads();
-  for (int j = threadIdx.x; j < m; j += kMergeThreads) {
+  for (int j = threadIdx.x; j < m; j += kRingThreads) {
     const u64 key = s_best[j];
     out.slot[(size_t)q * m + j] = key ? candidate_row(key) : -1;
     out.score[(size_t)q * m + j] = key ? candidate_score(key) : -INFINITY;
-  }
-  // stored continuation up to its first negative entry, -1 behind it
-  for (int j = threadIdx.x; j < m; j += kMergeThreads) {
-    const u64 key = s_best[j];
+    // stored continuation up to its first negative entry, -1 behind it (through L2: the
+    // record may have been stored by another block of this launch)
     int len = 0;
     bool open = key != 0;
     for (int t = 0; t < R; ++t) {
-      int tok = open ? rollout[(size_t)candidate_row(key) * R + t] : -1;
+      int tok = open ? __ldcg(&rollout[(size_t)candidate_row(key) * R + t]) : -1;
       if (tok < 0) open = false;
       out.rollout[((size_t)q * m + j) * R + t] = open ? tok : -1;
       if (open) ++len;
@@ -192,8 +219,7 @@ ring_merge_kernel(const u64* __restrict__ partial, int n_lists, int nq, int m, i
 cudaError_t preload_ring_kernels() {
   cudaError_t e;
   if ((e = preload_kernel(ring_append_kernel)) != cudaSuccess) return e;
-  if ((e = preload_kernel(ring_scan_kernel, true)) != cudaSuccess) return e;
-  return preload_kernel(ring_merge_kernel);
+  return preload_kernel(ring_scan_kernel, true);
 }
 
 }  // namespace oilbird
@@ -218,6 +244,7 @@ struct oilbird_ring {
   int32_t *anchor, *rollout, *q_valid;
   unsigned long long* partial;
   DeviceStats* stats;
+  unsigned* done;                  // per query: blocks of the running lookup that have finished
   unsigned long long* ready;       // records stored by lookups that append (device counter) ...
   unsigned long long ready_target; // ... and the host's count of them (enqueue time)
   unsigned char* base;
@@ -249,7 +276,8 @@ int oilbird_ring_create(oilbird_ring_t** out, const oilbird_ring_config* cfg) {
                o_valid = o_roll + up((size_t)r->cap * r->R * 4),
                o_part = o_valid + up((size_t)OILBIRD_RING_MAX_NQ * 4),
                o_stats = o_part + up((size_t)r->max_lists * OILBIRD_RING_MAX_NQ * kRingList * 8),
-               o_ready = o_stats + up(sizeof(DeviceStats)), total = o_ready + 256;
+               o_ready = o_stats + up(sizeof(DeviceStats)), o_done = o_ready + 256,
+               total = o_done + up((size_t)OILBIRD_RING_MAX_NQ * 4);
   void* mem = nullptr;
   cudaError_t e = cudaMalloc(&mem, total);
   if (e != cudaSuccess) { delete r; return ring_fail(e, "cudaMalloc(ring)"); }
@@ -261,8 +289,9 @@ int oilbird_ring_create(oilbird_ring_t** out, const oilbird_ring_config* cfg) {
   r->partial = (unsigned long long*)(r->base + o_part);
   r->stats = (DeviceStats*)(r->base + o_stats);
   r->ready = (unsigned long long*)(r->base + o_ready);
+  r->done = (unsigned*)(r->base + o_done);
   r->ready_target = 0;
-  e = cudaMemset(r->stats, 0, o_ready + 256 - o_stats);       // counters and the fused-store counter
+  e = cudaMemset(r->stats, 0, total - o_stats);               // counters, fused-store and arrival counters
   if (e != cudaSuccess) { cudaFree(mem); delete r; return ring_fail(e, "cudaMemset"); }
   *out = r;
   return OILBIRD_OK;
@@ -342,16 +371,13 @@ static int ring_query_impl(oilbird_ring_t* r, const void* q, const int32_t* q_an
   const size_t smem = (size_t)r->d * 2 + (size_t)kRingWarps * kRingList * sizeof(u64);
   cudaError_t e = launch_pdl(ring_scan_kernel, dim3(slices, nq), dim3(kRingThreads), smem, st,
                              r->keys, r->anchor, n_slots, r->d, (const uint16_t*)q, q_anchor, nq, m,
-                             floor_s, r->partial, r->q_valid, r->stats, fa);
+                             floor_s, r->partial, r->q_valid, r->stats, fa, r->done,
+                             (const int32_t*)r->rollout, r->R, *out);
   if (e != cudaSuccess) return ring_fail(e, "ring scan launch");
   if (n > 0) {
     r->total = total_after;
     r->ready_target = fa.target;
   }
-  e = launch_pdl(ring_merge_kernel, dim3(nq), dim3(kMergeThreads), 0, st,
-                 (const u64*)r->partial, slices, nq, m, r->R, (const int32_t*)r->q_valid,
-                 (const int32_t*)r->rollout, *out);
-  if (e != cudaSuccess) return ring_fail(e, "ring merge launch");
   return OILBIRD_OK;
 }
 

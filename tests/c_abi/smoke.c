@@ -90,6 +90,25 @@ int main(void) {
   CU(cudaMemcpy(&idx0, out.idx, 4, cudaMemcpyDeviceToHost));
   CU(cudaMemcpy(&clen0, out.cont_len, 4, cudaMemcpyDeviceToHost));
   if (idx0 != 198 || clen0 != 0) { fprintf(stderr, "self: idx %d len %d\n", idx0, clen0); return 8; }
+  /* host steps in two halves, two in flight: plain host arrays in, plain host arrays out */
+  {
+    static int32_t h_idx[2][K], h_fired[2], h_len[2][K], h_tok[2][K][L];
+    static float h_score[2][K];
+    oilbird_query_out ho[2];
+    for (int s = 0; s < 2; ++s) {
+      ho[s].idx = h_idx[s]; ho[s].score = h_score[s]; ho[s].fired = &h_fired[s];
+      ho[s].cont_len = h_len[s]; ho[s].cont_tok = &h_tok[s][0][0];
+    }
+    pr.path = OILBIRD_PATH_AUTO;
+    CHECK(oilbird_pool_step_host_begin(pool, NULL, NULL, 0, 0, 0, q, 1, &pr, 0, NULL));
+    CHECK(oilbird_pool_step_host_begin(pool, NULL, NULL, 0, 0, 0, rows[198], 1, &pr, 1, NULL));
+    if (oilbird_pool_step_host_begin(pool, NULL, NULL, 0, 0, 0, q, 1, &pr, 0, NULL) != OILBIRD_EINVAL) return 12;
+    CHECK(oilbird_pool_step_host_end(pool, 1, &ho[1]));
+    CHECK(oilbird_pool_step_host_end(pool, 0, &ho[0]));
+    if (oilbird_pool_step_host_end(pool, 0, &ho[0]) != OILBIRD_EINVAL) return 13;
+    if (h_idx[0][0] != 17 || h_idx[0][1] != 5 || h_fired[0] != 1 || h_tok[0][0][0] != 1000 + 19) return 14;
+    if (h_idx[1][0] != 198 || h_len[1][0] != 0) return 15;
+  }
   /* misaligned input is refused, nothing is appended */
   if (oilbird_pool_reset(pool, NULL) != 0) return 9;
   if (oilbird_pool_append(pool, (char*)d_rows + 2, d_tok, 1, 1, OILBIRD_NEW_TRACE, NULL) != OILBIRD_EINVAL) return 10;

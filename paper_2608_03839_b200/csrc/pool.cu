@@ -794,15 +794,27 @@ static int ensure_pinned(oilbird_pool* p) {
   if (e != cudaSuccess) return cuda_fail(e, "cudaHostAlloc");
   void* dptr = nullptr;
   e = cudaHostGetDevicePointer(&dptr, h, 0);
-  if (e == cudaSuccess) e = cudaEventCreateWithFlags(&p->upload_done, cudaEventDisableTiming);
+  // events and the copy stream; whatever was created is destroyed again if one of them fails
+  cudaEvent_t made[1 + 2 * (kHostSlots + 1)];
+  int n_made = 0;
+  auto make_event = [&](cudaEvent_t* ev) {
+    if (e != cudaSuccess) return;
+    e = cudaEventCreateWithFlags(ev, cudaEventDisableTiming);
+    if (e == cudaSuccess) made[n_made++] = *ev;
+  };
+  make_event(&p->upload_done);
   for (auto& sl : p->slot) {
     sl.busy = false;
-    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&sl.done, cudaEventDisableTiming);
-    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&sl.copied, cudaEventDisableTiming);
+    make_event(&sl.done);
+    make_event(&sl.copied);
   }
   // (non-blocking: no implicit ordering against the legacy default stream a caller may use)
   if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&p->copy_stream, cudaStreamNonBlocking);
-  if (e != cudaSuccess) { cudaFreeHost(h); return cuda_fail(e, "pinned staging set-up"); }
+  if (e != cudaSuccess) {
+    for (int i = 0; i < n_made; ++i) cudaEventDestroy(made[i]);
+    cudaFreeHost(h);
+    return cuda_fail(e, "pinned staging set-up");
+  }
   p->pinned = h;
   p->pinned_dev = (unsigned char*)dptr;
   p->blob_off = align_up(a_bytes);

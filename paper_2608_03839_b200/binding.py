@@ -821,7 +821,7 @@ def merge_chains(tree_tok: torch.Tensor, tree_parent: torch.Tensor, n_nodes: tor
                  sem_tok: torch.Tensor | None, sem_len: torch.Tensor | None,
                  extra_tok: torch.Tensor | None = None, extra_len: torch.Tensor | None = None,
                  budget: int = 16, min_len: int = 2, root_attached: bool = False,
-                 stream=None) -> MergeOut:
+                 stream=None, out: "MergeOut | None" = None) -> MergeOut:
     """oilbird_merge_chains: post-filter the chains and merge them into each request's tree.
 
     tree_tok / tree_parent: CUDA int32 [nq,max_nodes] (updated in place), n_nodes: [nq].
@@ -833,11 +833,15 @@ def merge_chains(tree_tok: torch.Tensor, tree_parent: torch.Tensor, n_nodes: tor
     ne, Le = (extra_tok.shape[1], extra_tok.shape[2]) if extra_tok is not None else (0, 1)
     for t in (tree_tok, tree_parent, n_nodes, sem_tok, sem_len, extra_tok, extra_len):
         assert t is None or (t.is_cuda and t.dtype == torch.int32 and t.is_contiguous())
-    depth = ALLOC((nq, max_nodes), torch.int32, dev)
-    mask = ALLOC((nq, max_nodes), torch.int64, dev)
-    status = ALLOC((nq, k + ne), torch.int32, dev)
-    bought = ALLOC((nq, k + ne), torch.int32, dev)
-    walked = ALLOC((nq, k + ne), torch.int32, dev)
+    if out is not None:                      # result arrays of an earlier call, written again
+        depth, mask, status, bought, walked = out.depth, out.mask, out.status, out.bought, out.walked
+        assert depth.shape == (nq, max_nodes) and status.shape == (nq, k + ne)
+    else:
+        depth = ALLOC((nq, max_nodes), torch.int32, dev)
+        mask = ALLOC((nq, max_nodes), torch.int64, dev)
+        status = ALLOC((nq, k + ne), torch.int32, dev)
+        bought = ALLOC((nq, k + ne), torch.int32, dev)
+        walked = ALLOC((nq, k + ne), torch.int32, dev)
     mp = MergeParams(budget, max_nodes, min_len, int(bool(root_attached)))
     ptr = lambda t: None if t is None else t.data_ptr()
     _check(lib().oilbird_merge_chains(nq, ptr(sem_tok), ptr(sem_len), k, L, ptr(extra_tok),

@@ -156,3 +156,23 @@ def test_tree_merge_ignores_parents_that_name_no_node():
     assert mo.tree_parent[1, :7].tolist() == [-1, 0, -1, -1, 1, 4, 5]
     assert mo.bought[:, 0].tolist() == [1, 3] and mo.walked[:, 0].tolist() == [3, 1]
     assert mo.mask[1, 2].item() == 1 << 2 and mo.depth[1, 2].item() == 0
+
+
+@pytest.mark.gpu
+def test_tree_merge_returns_on_parents_that_form_a_cycle():
+    # nodes 2 and 3 name each other: neither hangs off the root, so neither is walked, and
+    # the call still returns with the sound part of the tree extended
+    t_tok = torch.full((1, 60), -1, dtype=torch.int32, device="cuda")
+    t_par = torch.full((1, 60), -1, dtype=torch.int32, device="cuda")
+    t_tok[0, :4] = torch.tensor([7, 1, 2, 3], dtype=torch.int32)
+    t_par[0, :4] = torch.tensor([-1, 0, 3, 2], dtype=torch.int32)
+    n = torch.tensor([4], dtype=torch.int32, device="cuda")
+    sem = torch.tensor([[[1, 2, 3, 4]]], dtype=torch.int32, device="cuda")
+    slen = torch.tensor([[4]], dtype=torch.int32, device="cuda")
+    mo = B.merge_chains(t_tok, t_par, n, sem, slen)
+    torch.cuda.synchronize()
+    assert mo.n_nodes.tolist() == [7]
+    assert mo.tree_parent[0, :7].tolist() == [-1, 0, 3, 2, 1, 4, 5]
+    assert mo.bought[0, 0].item() == 3 and mo.walked[0, 0].item() == 1
+    assert mo.depth[0, 4:7].tolist() == [2, 3, 4]
+    assert mo.mask[0, 6].item() == (1 << 6) | (1 << 5) | (1 << 4) | (1 << 1) | 1

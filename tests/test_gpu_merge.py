@@ -88,6 +88,21 @@ def test_random_batches(seed):
         run_both(trees, sems, extras, budget, max_nodes, root_attached=ra, L=12, Le=7)
 
 
+def test_more_chains_than_the_kernel_stages_on_chip():
+    # 70 chains per request: beyond the 64 whose tokens the kernel keeps in shared memory, so
+    # it reads them from global memory chain by chain; same results either way
+    rng = np.random.default_rng(11)
+    trees, sems, extras = [], [], []
+    for _ in range(9):
+        n = int(rng.integers(1, 30))
+        trees.append(([7] + rng.integers(0, 3, n - 1).tolist(),
+                      [-1] + [int(rng.integers(0, j)) for j in range(1, n)]))
+        sems.append([rng.integers(0, 3, rng.integers(0, 12)).tolist() for _ in range(40)])
+        extras.append([rng.integers(0, 3, rng.integers(0, 7)).tolist() for _ in range(30)])
+    for budget, ra in ((16, False), (1000, False), (16, True)):
+        run_both(trees, sems, extras, budget, 64, root_attached=ra, L=12, Le=7)
+
+
 def test_query_output_feeds_the_merge():
     """End of the retrieval path: cont_tok / cont_len of a query go straight into the merge."""
     w = W.C3.scaled(n_rows=6000, n_templates=10, d=512, nq=8, k=8, cont_len=12)

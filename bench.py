@@ -1166,7 +1166,8 @@ def index_line(args):
                          "frac": cand_bytes / (head["us_per_query"] * 1e-6) / 1e9 / peaks["hbm_gbs"],
                          "peak_kind": peak_kind, "bytes_per_launch": cand_bytes, "traffic": None,
                          "note": "a lookup moves the centroids and a few hundred candidate rows: "
-                                 "four dependent launches, latency-bound, not bandwidth-bound"}}
+                                 "one launch of dependent round trips (centroids, probes, candidates, merge), "
+                                 "latency-bound, not bandwidth-bound"}}
     ix.close()
     pool.close()
     del pool

@@ -22,6 +22,7 @@
 #include <new>
 
 #include "common.cuh"
+#include "gather.cuh"
 #include "internal.h"
 #include "normalize.cuh"
 #include "pool_priv.h"
@@ -31,6 +32,12 @@ namespace oilbird {
 constexpr int kIndexMaxLists = 65536;
 constexpr int kIndexMaxProbe = OILBIRD_MAX_K;        // the probes are a k-lookup on the centroids
 constexpr int kIndexAssignBatch = 256;               // rows assigned per lookup
+// Batches up to here take the one-launch lookup.  It splits the CTAs of a launch between the
+// queries, so from two queries on the separate launches (each with every CTA on every
+// query's share, the centroids scanned once for all queries by the batched kernels) are
+// faster: 45.9 against 42.7 us for two queries, 72.9 against 55.6 us for four (C4 pool,
+// 4,096 lists, 4 probes).
+constexpr int kLookupMaxNq = 1;
 
 // ------------------------------------------------------------------ list building ---
 __global__ void __launch_bounds__(256)
@@ -139,32 +146,59 @@ index_means_kernel(const uint16_t* __restrict__ keys, int d, const int32_t* __re
 // probed lists in probe order, then the tail) and leaves one descending list of KK packed
 // candidates in partial[b][q], as the full scans do.  Rows are fetched by number; everything
 // else (query preparation, scoring, per-warp lists, block merge) is the CUDA-core scan's.
+// One row against the query in shared memory with up to kWide 16-byte loads per lane in
+// flight at once (a whole row of d <= 4096 in one round trip): for CTAs that hold a handful of
+// rows, where the round trips, not the bytes, are the cost.  A lane adds its chunks in the
+// order score_rows adds them, so the score has the same bits.
+constexpr int kWide = 16;
+__device__ __forceinline__ float score_row_wide(const uint4* row, const uint4* qs, int n_chunks,
+                                                int lane) {
+  float a = 0.f;
+  for (int c0 = lane; c0 < n_chunks; c0 += 32 * kWide) {
+    uint4 kv[kWide];
+#pragma unroll
+    for (int u = 0; u < kWide; ++u) {
+      const int c = c0 + 32 * u;
+      kv[u] = c < n_chunks ? ld_stream16(row + c) : make_uint4(0, 0, 0, 0);
+    }
+#pragma unroll
+    for (int u = 0; u < kWide; ++u) {
+      const int c = c0 + 32 * u;
+      if (c < n_chunks) {
+        const uint4 qv = qs[c];
+        a = fmaf(bf16_lo(kv[u].x), bf16_lo(qv.x), a);
+        a = fmaf(bf16_hi(kv[u].x), bf16_hi(qv.x), a);
+        a = fmaf(bf16_lo(kv[u].y), bf16_lo(qv.y), a);
+        a = fmaf(bf16_hi(kv[u].y), bf16_hi(qv.y), a);
+        a = fmaf(bf16_lo(kv[u].z), bf16_lo(qv.z), a);
+        a = fmaf(bf16_hi(kv[u].z), bf16_hi(qv.z), a);
+        a = fmaf(bf16_lo(kv[u].w), bf16_lo(qv.w), a);
+        a = fmaf(bf16_hi(kv[u].w), bf16_hi(qv.w), a);
+      }
+    }
+  }
+  return warp_sum(a);
+}
+// CTAs with at most this many rows each take them one row per warp at a time
+constexpr int kWideMaxRows = 64;
+
+// The candidate scan of CTA b of G for query q, whose normalised form is in qs.
 template <int E>
-__global__ void __launch_bounds__(kNormThreads, 2)
-scan_ids_kernel(PoolView pv, const uint16_t* __restrict__ q_raw, int nq, int k,
-                const int32_t* __restrict__ probes, int n_probe,
-                const int32_t* __restrict__ list_off, const int32_t* __restrict__ list_rows,
-                int n_indexed, const uint64_t* __restrict__ exclude_tag, u64* __restrict__ partial,
-                int32_t* __restrict__ q_valid, DeviceStats* stats) {
-  extern __shared__ __align__(16) unsigned char smem_raw[];
+__device__ __forceinline__ void scan_candidates(const PoolView& pv, const uint4* qs, u64* scratch,
+                                                int q, int nq, int k, int b, int G,
+                                                const int32_t* probes, int n_probe,
+                                                const int32_t* __restrict__ list_off,
+                                                const int32_t* __restrict__ list_rows, int n_indexed,
+                                                const uint64_t* __restrict__ exclude_tag,
+                                                u64* __restrict__ partial, int* s_pref, int* s_base) {
   constexpr int KK = 32 * E;
   constexpr int kWarps = kNormThreads / 32;
-  __shared__ int s_pref[kIndexMaxProbe + 1], s_base[kIndexMaxProbe];
-  pdl_enter();
-  const int d = pv.d, n_chunks = d >> 3;
-  uint4* qs = reinterpret_cast<uint4*>(smem_raw);                        // [n_chunks]
-  u64* scratch = reinterpret_cast<u64*>(smem_raw + (size_t)d * 2);        // [warps][KK]
+  const int n_chunks = pv.d >> 3;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int q = blockIdx.y;
-
-  const int code = normalize_row<true, 2>(q_raw + (size_t)q * d, reinterpret_cast<uint16_t*>(qs), d);
-  if (blockIdx.x == 0 && threadIdx.x == 0) {
-    q_valid[q] = code == kRowNonFinite ? 0 : 1;          // NaN/Inf: no neighbours
-    if (code == kRowNonFinite) atomicAdd(&stats->nonfinite_queries, 1ull);
-  }
-  // the probed lists of this query, laid end to end
+  // the probed lists of this query, laid end to end (the probes may have been written by
+  // another CTA of this launch: read through L2)
   if (threadIdx.x < n_probe) {
-    const int l = probes[(size_t)q * n_probe + threadIdx.x];
+    const int l = __ldcg(&probes[(size_t)q * n_probe + threadIdx.x]);
     s_base[threadIdx.x] = l >= 0 ? list_off[l] : 0;
     s_pref[threadIdx.x + 1] = l >= 0 ? list_off[l + 1] - list_off[l] : 0;
   }
@@ -177,8 +211,8 @@ scan_ids_kernel(PoolView pv, const uint16_t* __restrict__ q_raw, int nq, int k,
   const int in_lists = s_pref[n_probe];
   const int total = in_lists + (pv.n_rows - n_indexed);
   const uint64_t ex = exclude_tag ? exclude_tag[q] : 0;
-  const int c_lo = (int)(((long long)total * blockIdx.x) / gridDim.x);
-  const int c_hi = (int)(((long long)total * (blockIdx.x + 1)) / gridDim.x);
+  const int c_lo = (int)(((long long)total * b) / G);
+  const int c_hi = (int)(((long long)total * (b + 1)) / G);
   const uint4* keys4 = reinterpret_cast<const uint4*>(pv.keys);
 
   auto row_of = [&](int c) -> int {
@@ -195,6 +229,18 @@ scan_ids_kernel(PoolView pv, const uint16_t* __restrict__ q_raw, int nq, int k,
   u64 kth = 0;
 #pragma unroll
   for (int r = 0; r < E; ++r) top[0][r] = 0;
+  if (c_hi - c_lo <= kWideMaxRows) {
+    for (int c = c_lo + warp; c < c_hi; c += kWarps) {
+      const int row = row_of(c);
+      const float s = score_row_wide(keys4 + (size_t)row * n_chunks, qs, n_chunks, lane);
+      if (ex != 0 && pv.trace_tag[pv.trace_id[row]] == ex) continue;       // same-prompt trace
+      const u64 key = pack_candidate(s, (uint32_t)row);
+      if (key > kth) {
+        warp_sorted_insert<E>(top[0], key, lane);
+        kth = warp_list_get<E>(top[0], k - 1);
+      }
+    }
+  } else
   for (int cb = c_lo + warp * kRowsPerIter; cb < c_hi; cb += kWarps * kRowsPerIter) {
     int rows[kRowsPerIter];
     const uint4* rowp[kRowsPerIter];
@@ -221,9 +267,299 @@ scan_ids_kernel(PoolView pv, const uint16_t* __restrict__ q_raw, int nq, int k,
   }
   block_merge_desc<E>(top[0], scratch, kWarps);
   if (threadIdx.x < 32) {
-    u64* dst = partial + ((size_t)blockIdx.x * nq + q) * KK;
+    u64* dst = partial + ((size_t)b * nq + q) * KK;
 #pragma unroll
     for (int r = 0; r < E; ++r) dst[r * 32 + lane] = top[0][r];
+  }
+}
+
+template <int E>
+__global__ void __launch_bounds__(kNormThreads, 2)
+scan_ids_kernel(PoolView pv, const uint16_t* __restrict__ q_raw, int nq, int k,
+                const int32_t* __restrict__ probes, int n_probe,
+                const int32_t* __restrict__ list_off, const int32_t* __restrict__ list_rows,
+                int n_indexed, const uint64_t* __restrict__ exclude_tag, u64* __restrict__ partial,
+                int32_t* __restrict__ q_valid, DeviceStats* stats) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  __shared__ int s_pref[kIndexMaxProbe + 1], s_base[kIndexMaxProbe];
+  pdl_enter();
+  const int d = pv.d;
+  uint4* qs = reinterpret_cast<uint4*>(smem_raw);                        // [n_chunks]
+  u64* scratch = reinterpret_cast<u64*>(smem_raw + (size_t)d * 2);        // [warps][KK]
+  const int q = blockIdx.y;
+  const int code = normalize_row<true, 2>(q_raw + (size_t)q * d, reinterpret_cast<uint16_t*>(qs), d);
+  if (blockIdx.x == 0 && threadIdx.x == 0) {
+    q_valid[q] = code == kRowNonFinite ? 0 : 1;          // NaN/Inf: no neighbours
+    if (code == kRowNonFinite) atomicAdd(&stats->nonfinite_queries, 1ull);
+  }
+  scan_candidates<E>(pv, qs, scratch, q, nq, k, blockIdx.x, gridDim.x, probes, n_probe, list_off,
+                     list_rows, n_indexed, exclude_tag, partial, s_pref, s_base);
+}
+
+// ------------------------------------------------------------ folding lists on one CTA ---
+// The `want` best entries of n descending lists (KK = 32*E entries each, `stride` apart, written
+// during this launch: read through L2) into warp 0's registers.  A list's head is its best
+// entry, and the want-th largest of any grouping's best heads is reached by `want` distinct
+// lists, so no list whose head lies below that floor holds one of the `want` best: the heads
+// come first, in one round of loads, then only the lists at or above the floor.
+constexpr int kFoldMaxLists = 2 * kNormThreads;
+template <int E>
+__device__ __forceinline__ void fold_lists(const u64* lists, int n, size_t stride, int want,
+                                           u64 (&v)[E], u64* scratch) {
+  constexpr int kWarps = kNormThreads / 32;
+  constexpr int PF = E == 1 ? 8 : (E == 2 ? 4 : 2);        // lists a warp has in flight
+  __shared__ u64 s_floor, s_wmax[kWarps];
+  __shared__ int s_live[kFoldMaxLists], s_nlive;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, t = threadIdx.x;
+  const u64 h0 = t < n ? __ldcg(lists + (size_t)t * stride) : 0;
+  const u64 h1 = t + kNormThreads < n ? __ldcg(lists + (size_t)(t + kNormThreads) * stride) : 0;
+  const u64 hm = h0 > h1 ? h0 : h1;
+  if (t == 0) s_nlive = 0;
+  if (want <= kWarps) {
+    // few wanted: the warps' best heads are grouping enough, and cheaper than a sort
+    u64 m = hm;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) { const u64 x = shfl_xor_u64(m, o); m = x > m ? x : m; }
+    if (lane == 0) s_wmax[warp] = m;
+    __syncthreads();
+    if (t == 0) {
+      u64 w[kWarps];
+#pragma unroll
+      for (int i = 0; i < kWarps; ++i) w[i] = s_wmax[i];
+      u64 fl = 0;
+#pragma unroll
+      for (int i = 0; i < kWarps; ++i) {                           // want-th largest of eight
+        int above = 0;
+#pragma unroll
+        for (int j = 0; j < kWarps; ++j) above += (w[j] > w[i] || (w[j] == w[i] && j < i)) ? 1 : 0;
+        if (above == want - 1) fl = w[i];
+      }
+      s_floor = fl;
+    }
+  } else {
+    u64 hv[E];
+#pragma unroll
+    for (int r = 0; r < E; ++r) hv[r] = 0;
+    u64 h[1] = {hm};
+    warp_sort_desc<1>(h, lane);
+    hv[0] = h[0];                                                  // sorted, zeros behind it
+    block_merge_desc<E>(hv, scratch, kWarps);
+    const u64 fl = want <= 32 * E ? warp_list_get<E>(hv, want - 1) : 0;   // warp 0 holds the merged heads
+    if (t == 0) s_floor = fl;
+  }
+  __syncthreads();
+  const u64 fl = s_floor;
+  if (h0 != 0 && h0 >= fl) s_live[atomicAdd(&s_nlive, 1)] = t;
+  if (h1 != 0 && h1 >= fl) s_live[atomicAdd(&s_nlive, 1)] = t + kNormThreads;
+  __syncthreads();
+  const int n_live = s_nlive;
+#pragma unroll
+  for (int r = 0; r < E; ++r) v[r] = 0;
+  // (live list i goes to warp i mod kWarps: a handful of lists are spread over the warps)
+  for (int i0 = warp; i0 < n_live; i0 += kWarps * PF) {
+    u64 bl[PF][E];
+#pragma unroll
+    for (int u = 0; u < PF; ++u) {
+      const int i = i0 + u * kWarps;
+      const u64* src = lists + (size_t)s_live[i < n_live ? i : 0] * stride;
+#pragma unroll
+      for (int r = 0; r < E; ++r) bl[u][r] = i < n_live ? __ldcg(src + r * 32 + lane) : 0;
+    }
+#pragma unroll
+    for (int u = 0; u < PF; ++u)
+      if (i0 + u * kWarps < n_live) warp_merge_desc<E>(v, bl[u], lane);
+  }
+  block_merge_desc<E>(v, scratch, kWarps);
+}
+
+// ------------------------------------------------------------ one-launch lookup ---
+// Centroid scan, choice of the probes and candidate scan in one launch (small batches, where
+// a lookup is a chain of short dependent launches and their latencies are its cost).  Grid
+// (g1 + g2, nq).  A CTA draws a ticket for its query when it starts.  The first g1 tickets
+// score a share of the centroids each and leave a list of their 32 best; the last of them to
+// finish merges the g1 lists, publishes the n_probe best centroids and raises the query's
+// flag; none of them ever waits.  Tickets g1 and up prepare their query, wait for the flag
+// (bounded, like every wait of this library) and then scan a share of the candidates.
+// Whoever holds a ticket >= g1 knows that g1 CTAs have started before it, so what it waits
+// for is running whether or not the whole grid fits on the GPU at once.  The last of the
+// candidate CTAs to finish merges their lists and ends the lookup (firing rule, depth,
+// gather: a4..a6), and the last CTA of a query to leave clears the query's words for the
+// next launch.
+struct LookupSync { unsigned ticket, scanned, ready, candidates, finished, pad[3]; };
+
+template <int E>
+__global__ void __launch_bounds__(kNormThreads, 2)
+index_lookup_kernel(PoolView pv, const uint16_t* __restrict__ cent_keys, int n_lists,
+                    const uint16_t* __restrict__ q_raw, int nq, int k, int g1, int n_probe,
+                    int32_t* probes, u64* cpartial, LookupSync* sync,
+                    const int32_t* __restrict__ list_off, const int32_t* __restrict__ list_rows,
+                    int n_indexed, const uint64_t* __restrict__ exclude_tag, u64* __restrict__ partial,
+                    DeviceStats* stats, GatherParams gp, oilbird_query_out out) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  __shared__ int s_pref[kIndexMaxProbe + 1], s_base[kIndexMaxProbe];
+  __shared__ int s_ticket, s_flag;
+  constexpr int kWarps = kNormThreads / 32;
+  pdl_enter();
+  const int d = pv.d, n_chunks = d >> 3;
+  uint4* qs = reinterpret_cast<uint4*>(smem_raw);                        // [n_chunks]
+  u64* scratch = reinterpret_cast<u64*>(smem_raw + (size_t)d * 2);        // [warps][KK]
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int q = blockIdx.y;
+  LookupSync* sy = sync + q;
+  if (threadIdx.x == 0) s_ticket = (int)atomicAdd(&sy->ticket, 1u);
+  const int code = normalize_row<true, 2>(q_raw + (size_t)q * d, reinterpret_cast<uint16_t*>(qs), d);
+  __syncthreads();
+  const int ticket = s_ticket;
+  if (ticket >= (int)gridDim.x) {
+    // words left over from a launch that gave up: no share is this CTA's to take.  The
+    // status call reports it; oilbird_index_reset clears the words.
+    if (threadIdx.x == 0) atomicExch(&stats->stalled, 1);
+    return;
+  }
+  if (ticket < g1) {
+    // ---- a share of the centroids
+    const int r_lo = (int)(((long long)n_lists * ticket) / g1);
+    const int r_hi = (int)(((long long)n_lists * (ticket + 1)) / g1);
+    const uint4* keys4 = reinterpret_cast<const uint4*>(cent_keys);
+    u64 top[1] = {0};
+    u64 kth = 0;
+    if (r_hi - r_lo <= kWideMaxRows) {
+      for (int r = r_lo + warp; r < r_hi; r += kWarps) {
+        const u64 key = pack_candidate(score_row_wide(keys4 + (size_t)r * n_chunks, qs, n_chunks, lane),
+                                       (uint32_t)r);
+        if (key > kth) {
+          warp_sorted_insert<1>(top, key, lane);
+          kth = warp_list_get<1>(top, n_probe - 1);
+        }
+      }
+    } else
+    for (int rb = r_lo + warp * kRowsPerIter; rb < r_hi; rb += kWarps * kRowsPerIter) {
+      const uint4* rowp[kRowsPerIter];
+#pragma unroll
+      for (int r = 0; r < kRowsPerIter; ++r)
+        rowp[r] = keys4 + (size_t)(rb + r < r_hi ? rb + r : r_hi - 1) * n_chunks;
+      float acc[kRowsPerIter][1];
+#pragma unroll
+      for (int r = 0; r < kRowsPerIter; ++r) acc[r][0] = 0.f;
+      score_rows<1, false>(rowp, qs, n_chunks, lane, acc);
+#pragma unroll
+      for (int r = 0; r < kRowsPerIter; ++r) {
+        if (rb + r >= r_hi) break;                                    // warp-uniform
+        const u64 key = pack_candidate(warp_sum(acc[r][0]), (uint32_t)(rb + r));
+        if (key > kth) {
+          warp_sorted_insert<1>(top, key, lane);
+          kth = warp_list_get<1>(top, n_probe - 1);
+        }
+      }
+    }
+    block_merge_desc<1>(top, scratch, kWarps);
+    if (threadIdx.x < 32) {
+      // warp 0 holds the list: it publishes it and arrives (the arrival releases the warp's
+      // stores and, for the last one in, acquires everybody else's)
+      cpartial[((size_t)ticket * nq + q) * 32 + lane] = top[0];
+      __syncwarp();
+      if (lane == 0) {
+        unsigned prev;
+        asm volatile("atom.acq_rel.gpu.global.add.u32 %0, [%1], 1;" : "=r"(prev) : "l"(&sy->scanned) : "memory");
+        s_flag = prev == (unsigned)(g1 - 1);
+      }
+    }
+    __syncthreads();
+    if (s_flag) {
+      // ---- the last share is in: the g1 lists -> the probes
+      u64 v[1];
+      fold_lists<1>(cpartial + (size_t)q * 32, g1, (size_t)nq * 32, n_probe, v, scratch);
+      if (threadIdx.x < 32) {
+        if (lane < n_probe)
+          probes[(size_t)q * n_probe + lane] = (v[0] != 0 && code != kRowNonFinite) ? candidate_row(v[0]) : -1;
+        __syncwarp();
+        if (lane == 0) {
+          sy->scanned = 0;
+          asm volatile("st.release.gpu.global.u32 [%0], %1;" :: "l"(&sy->ready), "r"(1u) : "memory");
+        }
+      }
+    }
+  } else {
+    // ---- a share of the candidates, once the probes are known
+    if (ticket == g1 && threadIdx.x == 0 && code == kRowNonFinite)
+      atomicAdd(&stats->nonfinite_queries, 1ull);
+    if (threadIdx.x == 0) {
+      unsigned long long t0 = 0, limit = 0;
+      int ok = 1;
+      for (uint32_t spin = 0;; ++spin) {
+        unsigned r;
+        asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(r) : "l"(&sy->ready) : "memory");
+        if (r != 0) break;
+        if (spin == 0) {
+          asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t0));
+          limit = wait_limit_ns(stats);
+        }
+        if ((spin & 15u) == 15u) {
+          unsigned long long t1;
+          asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t1));
+          if (t1 - t0 > limit) { atomicExch(&stats->stalled, 1); ok = 0; break; }
+        }
+        __nanosleep(64);
+      }
+      s_flag = ok;
+    }
+    __syncthreads();
+    const int b = ticket - g1, g2 = (int)gridDim.x - g1;
+    const int woke = s_flag;
+    __syncthreads();                                     // s_flag is written again below
+    if (woke) {
+      scan_candidates<E>(pv, qs, scratch, q, nq, k, b, g2, probes, n_probe, list_off, list_rows,
+                         n_indexed, exclude_tag, partial, s_pref, s_base);
+    } else if (threadIdx.x < 32) {                         // gave up: an empty list
+      constexpr int KK = 32 * E;
+#pragma unroll
+      for (int r = 0; r < E; ++r) partial[((size_t)b * nq + q) * KK + r * 32 + lane] = 0;
+    }
+    // ---- the last list in: merge them, fire, gather (warp 0 wrote this CTA's list)
+    if (threadIdx.x < 32) {
+      __syncwarp();
+      if (lane == 0) {
+        unsigned prev;
+        asm volatile("atom.acq_rel.gpu.global.add.u32 %0, [%1], 1;" : "=r"(prev) : "l"(&sy->candidates) : "memory");
+        s_flag = prev == (unsigned)(g2 - 1);
+      }
+    }
+    __syncthreads();
+    if (s_flag) {
+      constexpr int KK = 32 * E;
+      __shared__ u64 s_best[OILBIRD_MAX_K];
+      __shared__ int32_t s_idx[OILBIRD_MAX_K];
+      __shared__ float s_score[OILBIRD_MAX_K];
+      __shared__ int32_t s_len[OILBIRD_MAX_K];
+      u64 v[E];
+      fold_lists<E>(partial + (size_t)q * KK, g2, (size_t)nq * KK, gp.k, v, scratch);
+      if (threadIdx.x < 32) {
+#pragma unroll
+        for (int r = 0; r < E; ++r) s_best[r * 32 + lane] = v[r];
+      }
+      __syncthreads();
+      const int kq = gp.k;
+      for (int j = threadIdx.x; j < kq; j += kNormThreads) {
+        const u64 key = code != kRowNonFinite ? s_best[j] : 0;     // NaN/Inf query: no neighbours
+        const int idx = key ? candidate_row(key) : -1;
+        const float sc = key ? candidate_score(key) : -INFINITY;
+        s_idx[j] = idx;
+        s_score[j] = sc;
+        out.idx[(size_t)q * kq + j] = idx;
+        out.score[(size_t)q * kq + j] = sc;
+      }
+      __syncthreads();
+      fire_depth_copy(pv, gp, q, s_idx, s_score, out, s_len);
+      if (threadIdx.x == 0) sy->candidates = 0;
+    }
+  }
+  // ---- the last CTA of the query leaves its words as it found them
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    __threadfence();
+    if (atomicAdd(&sy->finished, 1u) == gridDim.x - 1) {
+      sy->ticket = 0; sy->ready = 0; sy->finished = 0;
+    }
   }
 }
 
@@ -238,12 +574,29 @@ static cudaError_t launch_scan_ids(const PoolView& pv, const uint16_t* q, int nq
                     probes, n_probe, list_off, list_rows, n_indexed, ex, partial, q_valid, stats);
 }
 
+template <int E>
+static cudaError_t launch_index_lookup(const PoolView& pv, const uint16_t* cent_keys, int n_lists,
+                                       const uint16_t* q, int nq, int k, int g1, int g2, int n_probe,
+                                       int32_t* probes, u64* cpartial, LookupSync* sync,
+                                       const int32_t* list_off, const int32_t* list_rows,
+                                       int n_indexed, const uint64_t* ex, u64* partial,
+                                       DeviceStats* stats, const GatherParams& gp,
+                                       const oilbird_query_out& out, cudaStream_t st) {
+  const size_t smem = (size_t)pv.d * 2 + (size_t)(kNormThreads / 32) * 32 * E * sizeof(u64);
+  return launch_pdl(index_lookup_kernel<E>, dim3(g1 + g2, nq), dim3(kNormThreads), smem, st, pv,
+                    cent_keys, n_lists, q, nq, k, g1, n_probe, probes, cpartial, sync, list_off,
+                    list_rows, n_indexed, ex, partial, stats, gp, out);
+}
+
 cudaError_t preload_index_kernels() {
   cudaError_t e;
   if ((e = preload_kernel(index_count_kernel)) != cudaSuccess) return e;
   if ((e = preload_kernel(index_offsets_kernel)) != cudaSuccess) return e;
   if ((e = preload_kernel(index_scatter_kernel)) != cudaSuccess) return e;
   if ((e = preload_kernel(index_means_kernel)) != cudaSuccess) return e;
+  if ((e = preload_kernel(index_lookup_kernel<1>, true)) != cudaSuccess) return e;
+  if ((e = preload_kernel(index_lookup_kernel<2>, true)) != cudaSuccess) return e;
+  if ((e = preload_kernel(index_lookup_kernel<4>, true)) != cudaSuccess) return e;
   if ((e = preload_kernel(scan_ids_kernel<1>, true)) != cudaSuccess) return e;
   if ((e = preload_kernel(scan_ids_kernel<2>, true)) != cudaSuccess) return e;
   return preload_kernel(scan_ids_kernel<4>, true);
@@ -265,6 +618,7 @@ struct oilbird_index {
   // results of the lookups on the centroids
   int32_t* probe_idx; float* probe_score; int32_t *probe_fired, *probe_len, *probe_tok;
   float* a_score; int32_t *a_fired, *a_len, *a_tok;
+  oilbird::LookupSync* sync;     // one-launch lookups: four words per query, zero between launches
 };
 
 static thread_local char g_index_err[256] = "";
@@ -312,7 +666,8 @@ int oilbird_index_create(oilbird_index_t** out, oilbird_pool_t* pool, const void
                o_pt = o_pl + up((size_t)OILBIRD_MAX_NQ * kIndexMaxProbe * 4),
                o_as = o_pt + up((size_t)OILBIRD_MAX_NQ * kIndexMaxProbe * 4),
                o_af = o_as + up(kIndexAssignBatch * 4), o_al = o_af + up(kIndexAssignBatch * 4),
-               o_at = o_al + up(kIndexAssignBatch * 4), o_raw = o_at + up(kIndexAssignBatch * 4),
+               o_at = o_al + up(kIndexAssignBatch * 4), o_sync = o_at + up(kIndexAssignBatch * 4),
+               o_raw = o_sync + up((size_t)OILBIRD_MAX_NQ * sizeof(LookupSync)),
                total = o_raw + up(nl * (size_t)pool->r.d * 2);
   cudaError_t e = cudaMalloc((void**)&ix->mem, total);
   if (e != cudaSuccess) { oilbird_pool_destroy(ix->cent); delete ix; return index_fail(e, "cudaMalloc(index)"); }
@@ -325,10 +680,12 @@ int oilbird_index_create(oilbird_index_t** out, oilbird_pool_t* pool, const void
   ix->a_score = (float*)(ix->mem + o_as); ix->a_fired = (int32_t*)(ix->mem + o_af);
   ix->a_len = (int32_t*)(ix->mem + o_al); ix->a_tok = (int32_t*)(ix->mem + o_at);
   ix->cent_raw = (uint16_t*)(ix->mem + o_raw);
+  ix->sync = (LookupSync*)(ix->mem + o_sync);
   cudaStream_t st = (cudaStream_t)cuda_stream;
   // the centroids become the rows of a one-trace pool (their tokens are never looked at);
   // all lists start empty
   e = cudaMemsetAsync(ix->mem, 0, o_pidx, st);
+  if (e == cudaSuccess) e = cudaMemsetAsync(ix->sync, 0, (size_t)OILBIRD_MAX_NQ * sizeof(LookupSync), st);
   if (e == cudaSuccess)
     e = cudaMemcpyAsync(ix->cent_raw, centroids_bf16, nl * (size_t)pool->r.d * 2,
                         cudaMemcpyDeviceToDevice, st);
@@ -359,6 +716,7 @@ int oilbird_index_reset(oilbird_index_t* ix, void* cuda_stream) {
   ICU(cudaSetDevice(ix->pool->device));
   // every list empty again: offsets all zero
   ICU(cudaMemsetAsync(ix->list_off, 0, ((size_t)ix->n_lists + 1) * 4, (cudaStream_t)cuda_stream));
+  ICU(cudaMemsetAsync(ix->sync, 0, (size_t)OILBIRD_MAX_NQ * sizeof(LookupSync), (cudaStream_t)cuda_stream));
   ix->n_indexed = 0;
   ix->generation = ix->pool->generation;
   return OILBIRD_OK;
@@ -465,6 +823,36 @@ int oilbird_index_query(oilbird_index_t* ix, const void* q_bf16, int32_t nq, int
     return OILBIRD_EINVAL;
   ICU(cudaSetDevice(p->device));
   cudaStream_t st = (cudaStream_t)cuda_stream;
+  const int kk = list_len(pr->k);
+  PoolView pv = pool_view(p);
+  const uint16_t* q = (const uint16_t*)q_bf16;
+  if (nq <= kLookupMaxNq && n_probe <= 32 && pr->path == OILBIRD_PATH_AUTO) {
+    // small batches: centroid scan, probes and candidate scan in one launch, then the merge
+    if (preload_all_kernels() != cudaSuccess) return OILBIRD_ECUDA;
+    // Twice the CTAs that fit at once (two per SM): the first half takes the centroids and
+    // leaves, the second half moves in behind it, prepares the query while the probes are
+    // being chosen, and takes the candidates; each side has the whole GPU for its round trips.
+    // (Sharing one GPU-full of CTAs between the two sides, six to one: 17.4 us against 20.1 us
+    // for an even split on 4,096 lists and ~1,000 candidates; this form is faster than both.)
+    int g_all = 2 * p->num_sms / nq;
+    if (g_all < 4) g_all = 4;
+    if (g_all > kFoldMaxLists) g_all = kFoldMaxLists;
+    int g1 = g_all, g2 = g_all;
+    if (g1 > ix->cent->r.max_lists) g1 = ix->cent->r.max_lists;
+    if (g2 > p->r.max_lists) g2 = p->r.max_lists;
+    cudaError_t e;
+#define LOOKUP(E)                                                                                     \
+    launch_index_lookup<E>(pv, ix->cent->keys, ix->n_lists, q, nq, pr->k, g1, g2, n_probe, ix->probe_idx, \
+                           ix->cent->partial, ix->sync, ix->list_off, ix->list_rows,                  \
+                           (int)ix->n_indexed, pr->exclude_tag, p->partial, p->stats, gp, *out, st)
+    if (kk == 32) e = LOOKUP(1);
+    else if (kk == 64) e = LOOKUP(2);
+    else e = LOOKUP(4);
+#undef LOOKUP
+    if (e != cudaSuccess) return index_fail(e, "lookup launch");
+    p->launches += 1;
+    return OILBIRD_OK;
+  }
   // probe: the n_probe best centroids of every query
   oilbird_query_params pp;
   oilbird_query_params_default(&pp);
@@ -475,7 +863,6 @@ int oilbird_index_query(oilbird_index_t* ix, const void* q_bf16, int32_t nq, int
   rc = oilbird_pool_query(ix->cent, q_bf16, nq, &pp, &po, st);
   if (rc) return rc;
   // scan the candidates, merge, fire, gather
-  const int kk = list_len(pr->k);
   // blocks per query: all the SMs twice over for a single lookup (a block holds a few rows
   // and the lookup is latency-bound), fewer per query as the batch grows (every block
   // prepares its query first, which a batch would otherwise pay thousands of times over)
@@ -486,9 +873,7 @@ int oilbird_index_query(oilbird_index_t* ix, const void* q_bf16, int32_t nq, int
     if (grid > 2 * p->num_sms) grid = 2 * p->num_sms;
   }
   if (grid > p->r.max_lists) grid = p->r.max_lists;
-  PoolView pv = pool_view(p);
   cudaError_t e;
-  const uint16_t* q = (const uint16_t*)q_bf16;
   if (kk == 32)
     e = launch_scan_ids<1>(pv, q, nq, pr->k, ix->probe_idx, n_probe, ix->list_off, ix->list_rows,
                            (int)ix->n_indexed, pr->exclude_tag, p->partial, p->q_valid, p->stats, grid, st);

@@ -113,6 +113,68 @@ def test_lists_and_answers_match_the_oracle(d, n_lists):
     assert pool.stats()["stalled"] == 0
 
 
+@pytest.mark.parametrize("nq", [1, 2, 3, 4])
+def test_lookups_in_one_launch_match_the_oracle_and_the_separate_launches(nq):
+    # a single query's lookup is one launch (centroids, probes, candidates, merge and gather);
+    # batches, and an explicit scan path, take the separate launches
+    w = W.C1.scaled(n_rows=9000, d=512, nq=nq, k=8, cont_len=4, n_centroids=40, rows_per_trace=500, seed=21)
+    pool, ora, gix, oix = build_both(w, 48, seed=5, spare_rows=400, max_k=128)
+    gix.refresh(); oix.refresh()
+    g = torch.Generator(device="cuda").manual_seed(8)
+    st = torch.randn(130, 512, generator=g, device="cuda").to(torch.bfloat16)     # a tail
+    tk = torch.arange(130, dtype=torch.int32, device="cuda")
+    pool.append(st, tk, tag=99)
+    ora.append(W.to_bits(st), tk.cpu().numpy(), tag=99)
+    q, _ = w.queries("cuda")
+    q[nq - 1] = st[11]                                       # one query whose best row is in the tail
+    launches = pool.launch_count
+    for n_probe in (1, 3, 31, 48):
+        for k in (1, 8, 40, 100):
+            pr = fixed(k, 4, theta=0.8 if k == 8 else -2.0)
+            one = gix.query(q, n_probe, pr)
+            check_index_query(one, oix, W.to_bits(q), n_probe, pr)
+            sep = gix.query(q, n_probe, fixed(k, 4, theta=pr.theta, path=B.PATH_GEMV))
+            a, b = one.cpu(), sep.cpu()
+            assert torch.equal(a.idx, b.idx) and torch.equal(a.cont_tok, b.cont_tok)
+            assert torch.equal(a.fired, b.fired) and torch.equal(a.cont_len, b.cont_len)
+            assert torch.allclose(a.score, b.score, atol=SCORE_BUG, rtol=0)
+    assert int(gix.query(q, 1, fixed(4, 4)).idx[nq - 1, 0]) == 9011
+    # a single query is one launch per lookup up to 32 probes (12 above, one here); more
+    # probes, batches, and lookups that name a scan path are two on this pool (+ two on the
+    # centroids' own)
+    fused = 1 if nq == 1 else 2
+    assert pool.launch_count - launches == (12 + 1) * fused + 4 * 2 + 16 * 2, "the one-launch form was not taken"
+    # exclusion tags and a query that is not finite
+    ex = np.zeros(nq, dtype=np.uint64); ex[0] = 99; ex[-1] = 99
+    pr = fixed(6, 4, exclude_tag=torch.from_numpy(ex.view(np.int64)).cuda())
+    check_index_query(gix.query(q, 4, pr), oix, W.to_bits(q), 4, pr, exclude=ex)
+    bad = q.clone(); bad[0, 5] = float("nan")
+    out = gix.query(bad, 4, fixed(8, 4)).cpu()
+    assert out.idx[0].tolist() == [-1] * 8 and int(out.fired[0]) == 0 and out.cont_len[0].sum() == 0
+    if nq > 1:
+        good = gix.query(q, 4, fixed(8, 4)).cpu()
+        assert torch.equal(out.idx[1:], good.idx[1:])
+    # the words the CTAs of a lookup meet at are left clear: the same lookup as a CUDA graph,
+    # replayed, gives the same answer every time
+    pr = fixed(8, 4)
+    want = gix.query(q, 3, pr).cpu()
+    out = gix.query(q, 3, pr)
+    s = torch.cuda.Stream()
+    with torch.cuda.stream(s):
+        gix.query(q, 3, pr, out=out)
+        s.synchronize()
+        gr = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(gr, stream=s):
+            for _ in range(3):
+                gix.query(q, 3, pr, out=out)
+        for _ in range(4):
+            out.idx.fill_(-7)
+            gr.replay()
+            s.synchronize()
+            assert torch.equal(out.idx.cpu(), want.idx) and torch.equal(out.cont_tok.cpu(), want.cont_tok)
+    assert pool.stats()["stalled"] == 0 and pool.status() == B.OK
+
+
 def test_index_after_eviction_needs_a_reset():
     w = W.C1.scaled(n_rows=2000, d=128, nq=3, k=4, cont_len=2, rows_per_trace=250)
     pool, ora, gix, oix = build_both(w, 16, spare_rows=1000)

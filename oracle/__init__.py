@@ -25,6 +25,7 @@ _LIB = os.path.join(_HERE, "liboilbird_oracle.so")
 
 DEPTH_FIXED = 0
 DEPTH_TIERED = 1
+DEPTH_RANKED = 2          # granularity ablation: depth by neighbour rank (tier_depth[j])
 
 # Constants the paper prints (Algorithm 1's Require line; Eq. 3).
 PAPER_K = 8
@@ -99,6 +100,8 @@ def lib() -> ctypes.CDLL:
     L.oracle_scores.argtypes = [vp, vp, u64, vp]
     L.oracle_depth.restype = i32
     L.oracle_depth.argtypes = [f32, i32, vp, vp]
+    L.oracle_depth_by_rank.restype = i32
+    L.oracle_depth_by_rank.argtypes = [i32, i32, vp]
     L.oracle_gather_one.restype = i32
     L.oracle_gather_one.argtypes = [vp, i64, i32, i32, i32, vp]
     L.oracle_pool_query.restype = ctypes.c_int
@@ -331,6 +334,11 @@ class OraclePool:
         out = np.empty(L, dtype=np.int32)
         n = self._L.oracle_gather_one(self._h, int(idx), int(dep), int(offset), int(L), _ptr(out))
         return out, int(n)
+
+
+def depth_by_rank(j: int, tier_depth=PAPER_TIER_DEPTH) -> int:
+    dep = np.asarray(tier_depth, dtype=np.int32)
+    return int(lib().oracle_depth_by_rank(int(j), int(dep.size), _ptr(dep)))
 
 
 def depth(s: float, tier_thr=PAPER_TIER_THR, tier_depth=PAPER_TIER_DEPTH) -> int:

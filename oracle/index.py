@@ -35,7 +35,8 @@ from __future__ import annotations
 
 import numpy as np
 
-from . import DEPTH_FIXED, OraclePool, QueryParams, QueryResult, depth as oracle_depth
+from . import (DEPTH_FIXED, DEPTH_RANKED, OraclePool, QueryParams, QueryResult, depth as oracle_depth,
+               depth_by_rank)
 
 
 class OracleIndex:
@@ -134,8 +135,12 @@ class OracleIndex:
             for j, r in enumerate(top):
                 dep = 0
                 if fired[i]:
-                    dep = L if pr.depth_mode == DEPTH_FIXED else oracle_depth(
-                        float(s[r]), pr.tier_thr, pr.tier_depth)
+                    if pr.depth_mode == DEPTH_FIXED:
+                        dep = L
+                    elif pr.depth_mode == DEPTH_RANKED:
+                        dep = depth_by_rank(j, pr.tier_depth)
+                    else:
+                        dep = oracle_depth(float(s[r]), pr.tier_thr, pr.tier_depth)
                 tok, n = self.pool.gather_one(int(r), dep, pr.offset, L)
                 ctok[i, j], clen[i, j] = tok, n
         return QueryResult(idx, score, fired, clen, ctok, alls if want_all_scores else None)

@@ -397,6 +397,18 @@ int32_t oracle_depth(float s, int32_t n_tiers, const float *tier_thr, const int3
 }
 
 /*
+ * The granularity ablation's other arm (Section 6, "Retrieval granularity"): the copy depth is
+ * assigned by the neighbour's rank instead of its similarity.  The paper names the arm and
+ * gives no schedule; reading: neighbour j (best first, j from 0) copies tier_depth[j] tokens
+ * for j < n_tiers, and tier_depth[n_tiers - 1] from there on (the paper's table {48, 8}: the
+ * best neighbour copies 48 tokens, every other one 8).  No tier: nothing is copied.
+ */
+int32_t oracle_depth_by_rank(int32_t j, int32_t n_tiers, const int32_t *tier_depth) {
+  if (n_tiers <= 0 || j < 0) return 0;
+  return tier_depth[j < n_tiers ? j : n_tiers - 1];
+}
+
+/*
  * Eq. 3's copy for one neighbour: up to `dep` tokens starting `offset` after
  * row idx, clipped at the end of the trace holding idx and at L; the rest of
  * the L slots are filled with -1.  Returns the number of tokens copied.
@@ -417,7 +429,7 @@ int32_t oracle_gather_one(const oracle_pool *p, int64_t idx, int32_t dep, int32_
 
 /*
  * One retrieval (Algorithm 1's score / top-k / firing / depth / copy lines)
- * for nq queries.  depth_mode 0 = fixed span of L tokens, 1 = tiered D(s).
+ * for nq queries.  depth_mode 0 = fixed span of L tokens, 1 = tiered D(s), 2 = by rank.
  * Outputs (host, caller-owned): idx[nq][k] (-1 where fewer than k rows have a
  * finite score), score[nq][k] (-inf there), fired[nq], cont_len[nq][k],
  * cont_tok[nq][k][L] padded with -1.  all_scores, if not NULL, receives the
@@ -449,6 +461,7 @@ int oracle_pool_query(const oracle_pool *p, const uint16_t *q_raw, int32_t nq, i
       int32_t dep = 0;
       if (f && i >= 0)
         dep = depth_mode == 0 ? L
+            : depth_mode == 2 ? oracle_depth_by_rank(j, n_tiers, tier_depth)
                               : oracle_depth(score[(size_t)q * k + j], n_tiers, tier_thr, tier_depth);
       cont_len[(size_t)q * k + j] =
           oracle_gather_one(p, i, dep, offset, L, cont_tok + ((size_t)q * k + j) * L);

@@ -221,6 +221,40 @@ def test_theta_gates_on_best_only_and_lower_ranked_get_own_depth():
     assert np.all(res2.cont_tok == -1)
 
 
+def test_depth_by_rank_follows_the_table_whatever_the_scores():
+    # the granularity ablation's arm: neighbour j copies tier_depth[j], the last entry from
+    # there on; the scores only order the neighbours and decide the firing
+    d = 1024
+    base = np.ones(d, np.int64)
+    hs = [200, 40, 95, 60, 300]                 # s = .609, .9219, .8145, .8828, .414 (rows 0..4)
+    body = [hamming_row(base, h) for h in hs] + [hamming_row(base, d)] * 60
+    pool = OraclePool(d)
+    pool.append(pm1(body), np.arange(len(body)), tag=1)
+    pr = QueryParams(k=5, cont_len=48, depth_mode=oracle.DEPTH_RANKED)          # the paper's {48, 8}
+    res = pool.query(pm1(base), pr)
+    assert res.idx[0].tolist() == [1, 3, 2, 0, 4] and res.fired[0] == 1
+    assert res.cont_len[0].tolist() == [48, 8, 8, 8, 8]    # by similarity it would be 48, 8, 0, 0, 0
+    assert res.cont_tok[0, 0, :3].tolist() == [3, 4, 5] and res.cont_tok[0, 3, :8].tolist() == list(range(2, 10))
+    assert pool.query(pm1(base), QueryParams(k=5, cont_len=48)).cont_len[0].tolist() == [48, 8, 0, 0, 0]
+    # a longer table, a depth above L (capped at L) and one of zero
+    pr = QueryParams(k=5, cont_len=12, depth_mode=oracle.DEPTH_RANKED, tier_thr=(0, 0, 0), tier_depth=(20, 0, 3))
+    assert pool.query(pm1(base), pr).cont_len[0].tolist() == [12, 0, 3, 3, 3]
+    assert [oracle.depth_by_rank(j, (20, 0, 3)) for j in range(5)] == [20, 0, 3, 3, 3]
+    assert oracle.depth_by_rank(0, ()) == 0
+    # the firing rule is unchanged: best below theta, nothing is copied
+    pr = QueryParams(k=5, theta=0.95, cont_len=48, depth_mode=oracle.DEPTH_RANKED)
+    res = pool.query(pm1(base), pr)
+    assert res.fired[0] == 0 and np.all(res.cont_len == 0) and np.all(res.cont_tok == -1)
+    # clipped at the trace end like every copy: row 64 is the last of 65
+    pr = QueryParams(k=1, theta=-2.0, cont_len=48, depth_mode=oracle.DEPTH_RANKED)
+    far = pool.query(pm1(-base), pr)
+    assert far.idx[0, 0] == 5 and far.cont_len[0, 0] == 48
+    tail = OraclePool(d)
+    tail.append(pm1(body[:6]), np.arange(6), tag=1)
+    assert tail.query(pm1(base), QueryParams(k=2, cont_len=48, depth_mode=oracle.DEPTH_RANKED)
+                      ).cont_len[0].tolist() == [3, 1]          # rows 1 and 3 of six
+
+
 # ------------------------------------------------------------------- T7 gather --
 
 def test_gather_offsets_clipping_and_trace_boundaries():

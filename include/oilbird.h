@@ -67,6 +67,11 @@ extern "C" {
 /* depth modes (Eq. 3 and the fixed-span variant of the batched harness) */
 #define OILBIRD_DEPTH_FIXED   0  /* every neighbour copies cont_len tokens             */
 #define OILBIRD_DEPTH_TIERED  1  /* D(s): first tier whose floor the score reaches     */
+#define OILBIRD_DEPTH_RANKED  2  /* by rank (Section 6, "Retrieval granularity", the arm
+                                    the paper compares D(s) with; it gives no schedule, this
+                                    is the library's reading): neighbour j, best first from
+                                    0, copies tier_depth[j] tokens, the last entry from
+                                    j = n_tiers - 1 on; tier_thr is not looked at         */
 
 /* which scoring kernel runs */
 #define OILBIRD_PATH_AUTO    0   /* chosen from nq, the pool's size and its key format  */

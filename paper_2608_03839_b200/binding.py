@@ -31,7 +31,7 @@ EVICT_TO_FIT = 2
 EVICT_TO_FIT = 2
 KEYS_E4M3 = 1          # pool flag: 8-bit keys
 DEBUG_GUARDS = 2       # pool flag: sentinel bytes behind every array (see Pool.check_guards)
-DEPTH_FIXED, DEPTH_TIERED = 0, 1
+DEPTH_FIXED, DEPTH_TIERED, DEPTH_RANKED = 0, 1, 2
 PATH_AUTO, PATH_GEMV, PATH_TENSOR, PATH_MMA = 0, 1, 2, 3
 MAX_NQ, MAX_K, MAX_CONT_LEN, MAX_TIERS = 256, 128, 128, 4
 HOST_SLOTS = 2

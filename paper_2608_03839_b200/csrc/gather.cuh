@@ -7,9 +7,13 @@
 
 namespace oilbird {
 
-// Eq. 3's D(s): first tier, in the order given, whose floor the score reaches.
-__device__ __forceinline__ int depth_of(float s, const GatherParams& gp) {
+// Eq. 3's D(s): first tier, in the order given, whose floor the score reaches.  By rank (the
+// granularity ablation's arm, Section 6): neighbour j copies tier_depth[j], the last entry
+// from there on, whatever its score.
+__device__ __forceinline__ int depth_of(float s, int j, const GatherParams& gp) {
   if (gp.depth_mode == OILBIRD_DEPTH_FIXED) return gp.cont_len;
+  if (gp.depth_mode == OILBIRD_DEPTH_RANKED)
+    return gp.n_tiers > 0 ? gp.tier_depth[j < gp.n_tiers ? j : gp.n_tiers - 1] : 0;
   for (int t = 0; t < gp.n_tiers; ++t)
     if (s >= gp.tier_thr[t]) return gp.tier_depth[t];
   return 0;
@@ -27,7 +31,7 @@ __device__ __forceinline__ void fire_depth_copy(const PoolView& pv, const Gather
     const int idx = s_idx[j];
     int len = 0;
     if (fired && idx >= 0 && idx < pv.n_rows) {
-      const int dep = depth_of(s_score[j], gp);                       // a5
+      const int dep = depth_of(s_score[j], j, gp);                    // a5
       const long long start = (long long)idx + gp.offset;
       const long long end = pv.trace_end[pv.trace_id[idx]];           // never leave the trace
       long long m = end - start;

@@ -484,7 +484,8 @@ int check_query_params(int32_t nq, int32_t max_nq, int32_t max_k, const oilbird_
   if (pr->k < 1 || pr->k > max_k) return OILBIRD_EINVAL;
   if (pr->cont_len < 1 || pr->cont_len > OILBIRD_MAX_CONT_LEN) return OILBIRD_EINVAL;
   if (pr->offset < 0 || pr->offset > (1 << 20)) return OILBIRD_EINVAL;
-  if (pr->depth_mode != OILBIRD_DEPTH_FIXED && pr->depth_mode != OILBIRD_DEPTH_TIERED)
+  if (pr->depth_mode != OILBIRD_DEPTH_FIXED && pr->depth_mode != OILBIRD_DEPTH_TIERED &&
+      pr->depth_mode != OILBIRD_DEPTH_RANKED)
     return OILBIRD_EINVAL;
   if (pr->n_tiers < 0 || pr->n_tiers > OILBIRD_MAX_TIERS) return OILBIRD_EINVAL;
   if (pr->path < OILBIRD_PATH_AUTO || pr->path > OILBIRD_PATH_MMA) return OILBIRD_EINVAL;

@@ -115,6 +115,7 @@ def check_query(out: B.QueryOut, ora: OraclePool, q_bits: np.ndarray, params: B.
             dep = 0
             if fired[q] and got[j] >= 0:
                 dep = (params.cont_len if params.depth_mode == B.DEPTH_FIXED
+                       else oracle.depth_by_rank(j, params.tier_depth) if params.depth_mode == B.DEPTH_RANKED
                        else oracle.depth(float(score[q, j]), params.tier_thr, params.tier_depth))
             exp_tok, exp_len = ora.gather_one(int(got[j]), dep, params.offset, params.cont_len)
             assert clen[q, j] == exp_len, (q, j, got[j], clen[q, j], exp_len)

@@ -160,6 +160,36 @@ def test_theta_and_depth_tiers_on_exact_scores():
         assert torch.all(out.idx[0, 1:] >= 1)    # theta is not a floor inside the top-k
 
 
+def test_depth_by_rank_on_exact_scores_and_on_every_scan_path():
+    # by hand, as the oracle's pin: scores .609 .9219 .8145 .8828 .414 -> neighbours 1 3 2 0 4
+    d = 1024
+    base = np.ones(d, np.int64)
+    rows = np.stack([np.where(np.arange(d) < h, -base, base) for h in (200, 40, 95, 60, 300)] + [-base] * 60)
+    bits = np.where(rows > 0, P1, M1).astype(np.uint16)
+    pool = B.Pool(d, 80)
+    pool.append(bits_to_dev(bits), torch.arange(65, dtype=torch.int32).cuda(), tag=1)
+    q = bits_to_dev(np.full((1, d), P1, np.uint16))
+    out = pool.query(q, B.QueryParams(k=5, cont_len=48, depth_mode=B.DEPTH_RANKED)).cpu()
+    assert out.idx[0].tolist() == [1, 3, 2, 0, 4] and int(out.fired[0]) == 1
+    assert out.cont_len[0].tolist() == [48, 8, 8, 8, 8]
+    assert out.cont_tok[0, 0, :3].tolist() == [3, 4, 5] and out.cont_tok[0, 3, :8].tolist() == list(range(2, 10))
+    pr = B.QueryParams(k=5, cont_len=12, depth_mode=B.DEPTH_RANKED, tier_thr=(0.0, 0.0, 0.0), tier_depth=(20, 0, 3))
+    assert pool.query(q, pr).cpu().cont_len[0].tolist() == [12, 0, 3, 3, 3]
+    out = pool.query(q, B.QueryParams(k=5, theta=0.95, cont_len=48, depth_mode=B.DEPTH_RANKED)).cpu()
+    assert int(out.fired[0]) == 0 and int(out.cont_len.sum()) == 0 and torch.all(out.cont_tok == -1)
+    with pytest.raises(B.OilbirdError):
+        pool.query(q, B.QueryParams(k=5, cont_len=12, depth_mode=3))
+    # against the oracle on a benchmark-shaped pool, every scan path, several queries
+    w = W.C1.scaled(nq=6, k=12, n_rows=3000, d=512, cont_len=24)
+    big, ora = fill_both(w)
+    qs, _ = w.queries("cuda")
+    for path in (B.PATH_GEMV, B.PATH_MMA, B.PATH_TENSOR):
+        for tiers in ((48, 8), (5, 4, 3, 2)):
+            pr = B.QueryParams(k=8, theta=-2.0, cont_len=24, depth_mode=B.DEPTH_RANKED, path=path,
+                               tier_thr=(0.0,) * len(tiers), tier_depth=tiers)
+            check_query(big.query(qs, pr), ora, W.to_bits(qs), pr)
+
+
 # ------------------------------------------------------------- benchmark shapes ----
 
 def run_workload(w, n_rows=None, nq=None, paths=(B.PATH_AUTO,), thetas=(0.8, -2.0), **kw):

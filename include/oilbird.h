@@ -306,15 +306,18 @@ int32_t oilbird_pool_num_traces(const oilbird_pool_t* pool);
  * if a device-side wait ever gave up, else OILBIRD_OK. */
 int oilbird_pool_status(oilbird_pool_t* pool, oilbird_pool_stats* stats, void* cuda_stream);
 /*
- * Bounded waits.  The library's kernels wait on the device in two places only: a scan that
- * also appends the step's rows waits for a row counter, and the tensor-core scan's warps wait
- * on shared-memory barriers for each other.  Every such wait gives up after limit_ns
+ * Bounded waits.  The library's kernels wait on the device in three places only: a scan that
+ * also appends the step's rows waits for a row counter, the tensor-core scan's warps wait
+ * on shared-memory barriers for each other, and the candidate CTAs of a one-launch index
+ * lookup wait for the flag word that hands them the probes (the recycled pool's fused step
+ * waits like the first).  Every such wait gives up after limit_ns
  * nanoseconds (0 = the default, two seconds): the kernel raises the `stalled` status, lets
  * the copies it has in flight land, frees what it holds and returns, so the context stays
  * usable; oilbird_pool_status then returns OILBIRD_ESTALL until reset().  set_wait_limit
- * takes effect in stream order.  stall_selftest runs one small kernel that performs both
- * kinds of wait on things that never happen (a counter nobody advances, a barrier nobody
- * arrives at), so the give-up path can be exercised: after it, status reports the stall.
+ * takes effect in stream order.  stall_selftest runs one small kernel that performs the
+ * three kinds of wait on things that never happen (a counter nobody advances, a barrier
+ * nobody arrives at, a flag nobody raises), so the give-up path can be exercised: after it,
+ * status reports the stall.
  */
 int oilbird_pool_set_wait_limit(oilbird_pool_t* pool, uint64_t limit_ns, void* cuda_stream);
 int oilbird_pool_stall_selftest(oilbird_pool_t* pool, void* cuda_stream);

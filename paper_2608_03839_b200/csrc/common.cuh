@@ -89,6 +89,26 @@ __device__ __forceinline__ void wait_fused_rows(const unsigned long long* ready,
 __device__ __forceinline__ void wait_fused_rows(const FusedAppend& fa, DeviceStats* stats) {
   wait_fused_rows(fa.ready, fa.target, stats);
 }
+// Wait until another CTA of this launch has raised a flag word (acquire).  Bounded in the same
+// way: false after the pool's wait limit, with `stalled` raised.
+__device__ __forceinline__ bool wait_flag_u32(const unsigned* flag, DeviceStats* stats) {
+  unsigned long long t0 = 0, limit = 0;
+  for (uint32_t spin = 0;; ++spin) {
+    unsigned r;
+    asm volatile("ld.acquire.gpu.u32 %0, [%1];" : "=r"(r) : "l"(flag) : "memory");
+    if (r != 0) return true;
+    if (spin == 0) {
+      asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t0));
+      limit = wait_limit_ns(stats);
+    }
+    if ((spin & 15u) == 15u) {
+      unsigned long long t1;
+      asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t1));
+      if (t1 - t0 > limit) { atomicExch(&stats->stalled, 1); return false; }
+    }
+    __nanosleep(64);
+  }
+}
 
 // ------------------------------------------------- scoring rows (CUDA cores) ---
 constexpr int kRowsPerIter = 4;   // rows a warp scores together (shares each query load)

@@ -483,26 +483,7 @@ index_lookup_kernel(PoolView pv, const uint16_t* __restrict__ cent_keys, int n_l
     // ---- a share of the candidates, once the probes are known
     if (ticket == g1 && threadIdx.x == 0 && code == kRowNonFinite)
       atomicAdd(&stats->nonfinite_queries, 1ull);
-    if (threadIdx.x == 0) {
-      unsigned long long t0 = 0, limit = 0;
-      int ok = 1;
-      for (uint32_t spin = 0;; ++spin) {
-        unsigned r;
-        asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(r) : "l"(&sy->ready) : "memory");
-        if (r != 0) break;
-        if (spin == 0) {
-          asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t0));
-          limit = wait_limit_ns(stats);
-        }
-        if ((spin & 15u) == 15u) {
-          unsigned long long t1;
-          asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t1));
-          if (t1 - t0 > limit) { atomicExch(&stats->stalled, 1); ok = 0; break; }
-        }
-        __nanosleep(64);
-      }
-      s_flag = ok;
-    }
+    if (threadIdx.x == 0) s_flag = wait_flag_u32(&sy->ready, stats) ? 1 : 0;
     __syncthreads();
     const int b = ticket - g1, g2 = (int)gridDim.x - g1;
     const int woke = s_flag;

@@ -1256,15 +1256,17 @@ cudaError_t launch_scan_tc(TcCache* cache, const PoolView& pv, int32_t q0, int32
   return cudaErrorInvalidConfiguration;
 }
 
-// Both kinds of bounded wait on things that never happen (see launch_stall_selftest).
+// The three kinds of bounded wait on things that never happen (see launch_stall_selftest).
 __global__ void __launch_bounds__(64)
 stall_selftest_kernel(const unsigned long long* ready, DeviceStats* stats, int* gave_up) {
   __shared__ uint64_t bar;
   __shared__ int abort_flag;
+  __shared__ unsigned never_raised;
   pdl_enter();
   if (threadIdx.x == 0) {
     mbar_init(&bar, 1);
     abort_flag = 0;
+    never_raised = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   __syncthreads();
@@ -1275,6 +1277,9 @@ stall_selftest_kernel(const unsigned long long* ready, DeviceStats* stats, int* 
     // phase 0 of a barrier nobody arrives at never completes
     const bool ok = mbar_wait(&bar, 0, &abort_flag, stats);
     if (gave_up) *gave_up = ok ? 0 : 1;
+  } else if (threadIdx.x == 33) {
+    // a flag word that no CTA raises (the index lookup's hand-over of the probes)
+    wait_flag_u32(&never_raised, stats);
   }
 }
 

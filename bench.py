@@ -1399,8 +1399,8 @@ def run_merge(args):
             "gpu_launches": K,
             "roofline": {"bound": "alu", "kernel": "merge_tree_kernel", "achieved": None, "peak": None,
                          "frac": None, "traffic": None,
-                         "note": "sequential per request (one warp each), a few hundred tokens: "
-                                 "launch-latency bound, no roofline applies"},
+                         "note": "one warp per request (the chains of a request depend on one another), "
+                                 "a few hundred tokens: latency-bound, no roofline applies"},
             "cpu_baseline": {"value": nq / cpu_dt, "unit": "requests/s", "cores": 1, "kind": "oracle",
                              "sample": f"the same {nq} requests through the Python oracle"}}
     print(json.dumps(line), flush=True)

@@ -171,6 +171,13 @@ scan_gemv_e4m3_kernel(const uint8_t* __restrict__ codes, const float* __restrict
         wait_fused_rows(fa, stats);       // rows of this step's append
         fresh_ok = true;
       }
+      // the rows' scales are asked for ahead of the codes, not behind the sums
+      float sc[kQ8Rows];
+#pragma unroll
+      for (int r = 0; r < kQ8Rows; ++r) {
+        const int row = rb + r < r_hi ? rb + r : r_hi - 1;
+        sc[r] = (fa.n > 0 && row >= fa.row0) ? __ldcg(scales + row) : scales[row];
+      }
 #pragma unroll 4
       for (int c = lane; c < n16; c += 32) {
         uint4 kv[kQ8Rows];
@@ -212,14 +219,13 @@ scan_gemv_e4m3_kernel(const uint8_t* __restrict__ codes, const float* __restrict
         const int row = rb + r;
         if (row >= r_hi) break;                             // warp-uniform
         const bool fresh_row = fa.n > 0 && row >= fa.row0;     // written by another CTA just now
-        const float sc = fresh_row ? __ldcg(scales + row) : scales[row];
         uint64_t tag = 0;
         if (exclude_tag)
           tag = fresh_row ? __ldcg(&pv.trace_tag[__ldcg(&pv.trace_id[row])])
                           : pv.trace_tag[pv.trace_id[row]];
 #pragma unroll
         for (int q = 0; q < QT; ++q) {
-          const float s = warp_sum(acc[r][q]) * sc;
+          const float s = warp_sum(acc[r][q]) * sc[r];
           if (q0 + q >= nq) continue;
           if (s_ex[q] != 0 && tag == s_ex[q]) continue;     // same-prompt trace: skipped
           const u64 key = pack_candidate(s, (uint32_t)row);

@@ -389,6 +389,15 @@ scan_mma_kernel(PoolView pv, const uint8_t* __restrict__ codes, const float* __r
     }
     for (; rb < r_hi; rb += kQuads * kMmaRows) {
       const int row0 = rb + g, row1 = rb + g + 8;
+      // 8-bit pools: the rows' scales (and the queries' 2^14 taken back), asked for before the
+      // group's arithmetic so that the epilogue does not wait a round trip for them (a group
+      // that holds rows appended by this launch has waited for them before its first load)
+      float sc0 = 1.f, sc1 = 1.f;
+      if (kFp8 && own) {
+        // (a row appended by this launch: its scale was written a moment ago, read it through L2)
+        sc0 = row0 < r_hi ? (cur_fresh ? __ldcg(&scales[row0]) : scales[row0]) * (1.f / kFp8QueryScale) : 0.f;
+        sc1 = row1 < r_hi ? (cur_fresh ? __ldcg(&scales[row1]) : scales[row1]) * (1.f / kFp8QueryScale) : 0.f;
+      }
       const bool has_next = rb + kQuads * kMmaRows < r_hi;
       const bool next_fresh = has_next && fresh_at(rb + kQuads * kMmaRows);
       // the next group's first step is fetched early unless it holds rows that this launch
@@ -476,13 +485,6 @@ scan_mma_kernel(PoolView pv, const uint8_t* __restrict__ codes, const float* __r
           tag0 = cur_fresh ? __ldcg(&pv.trace_tag[__ldcg(&pv.trace_id[row0])]) : pv.trace_tag[pv.trace_id[row0]];
         if (row1 < r_hi)
           tag1 = cur_fresh ? __ldcg(&pv.trace_tag[__ldcg(&pv.trace_id[row1])]) : pv.trace_tag[pv.trace_id[row1]];
-      }
-      // 8-bit pools: the rows' scales (and the queries' 2^14 taken back)
-      float sc0 = 1.f, sc1 = 1.f;
-      if (kFp8 && own) {
-        // (a row appended by this launch: its scale was written a moment ago, read it through L2)
-        sc0 = row0 < r_hi ? (cur_fresh ? __ldcg(&scales[row0]) : scales[row0]) * (1.f / kFp8QueryScale) : 0.f;
-        sc1 = row1 < r_hi ? (cur_fresh ? __ldcg(&scales[row1]) : scales[row1]) * (1.f / kFp8QueryScale) : 0.f;
       }
       u64 key[2 * NT][2];                    // [list][row0 / row1]
       bool any = false;

@@ -30,6 +30,14 @@ OraclePool (full scores in double, full sort); plain numpy and Python loops on p
            (count * 2^30))), both roundings to nearest even.  The raw centroids then go
            through the same normalisation as at creation.  After the last iteration the lists
            are rebuilt from scratch.
+
+8-bit pools (FP8 E4M3 codes with one fp32 scale per row).  The paper defines neither the
+quantised store nor the index, so what a stored row IS, as a state, is a reading: element j of
+row i is x = fp32(value(code_ij) * scale_i), the product rounded once to fp32.  Taken as a
+query state (assign), the row is those elements rounded to bf16, like any state the library
+is handed, and goes through the query normalisation.  In the training means the element
+contributes trunc(x * 2^30) with the fp32 x itself.  Scoring, and so the scan step, is the
+8-bit pool's own (OraclePool with key_format "e4m3").
 """
 from __future__ import annotations
 
@@ -60,12 +68,28 @@ class OracleIndex:
     def reset(self) -> None:
         self.assign = np.empty(0, dtype=np.int64)
 
+    def _stored_f32(self, lo: int, hi: int) -> np.ndarray:
+        """Rows lo..hi of the store as fp32 elements (see the header for 8-bit pools)."""
+        from . import bf16_bits_to_f32, e4m3_decode
+        if self.pool.key_format == "bf16":
+            return bf16_bits_to_f32(self.pool.keys[lo:hi])
+        value = np.array([e4m3_decode(c) for c in range(256)], dtype=np.float64)
+        value[~np.isfinite(value)] = 0.0               # NaN codes are never stored
+        codes, scales = self.pool.codes[lo:hi], self.pool.scales[lo:hi]
+        return (value[codes] * scales.astype(np.float64)[:, None]).astype(np.float32)
+
+    def _stored_as_queries(self, lo: int, hi: int) -> np.ndarray:
+        from . import f32_to_bf16_bits
+        if self.pool.key_format == "bf16":
+            return self.pool.keys[lo:hi]               # stored (normalised) keys, as queries
+        return f32_to_bf16_bits(self._stored_f32(lo, hi))
+
     def refresh(self) -> None:
         """Assign the rows appended since the last refresh."""
         n = len(self.pool)
         if n <= self.n_indexed:
             return
-        keys = self.pool.keys[self.n_indexed:n]        # stored (normalised) keys, as queries
+        keys = self._stored_as_queries(self.n_indexed, n)
         one = QueryParams(k=1, theta=-np.inf, depth_mode=DEPTH_FIXED, cont_len=1)
         new = np.empty(keys.shape[0], dtype=np.int64)
         step = 4096
@@ -75,11 +99,11 @@ class OracleIndex:
 
     def train(self, iterations: int) -> None:
         """Lloyd's iterations (see the header); afterwards every row of the pool is indexed."""
-        from . import bf16_bits_to_f32, f32_to_bf16_bits
+        from . import f32_to_bf16_bits
         for _ in range(int(iterations)):
             self.reset()
             self.refresh()
-            x = bf16_bits_to_f32(self.pool.keys).astype(np.float64)       # stored keys, exact
+            x = self._stored_f32(0, len(self.pool)).astype(np.float64)    # stored elements, exact
             t = np.trunc(x * 2.0 ** 30).astype(np.int64)
             for l in range(self.n_lists):
                 rows = np.nonzero(self.assign == l)[0]

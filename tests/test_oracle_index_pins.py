@@ -20,8 +20,8 @@ def fixed(k, L=2, theta=-np.inf, **kw):
     return oracle.QueryParams(k=k, theta=theta, depth_mode=oracle.DEPTH_FIXED, cont_len=L, **kw)
 
 
-def random_pool(rng, n, d, n_traces=4):
-    pool = OraclePool(d)
+def random_pool(rng, n, d, n_traces=4, key_format="bf16"):
+    pool = OraclePool(d, key_format)
     rows = rng.standard_normal((n, d)).astype(np.float32)
     bits = f2b(rows)
     per = n // n_traces
@@ -31,10 +31,11 @@ def random_pool(rng, n, d, n_traces=4):
     return pool, bits
 
 
+@pytest.mark.parametrize("key_format", ["bf16", "e4m3"])
 @pytest.mark.parametrize("n_lists", [1, 3, 16])
-def test_all_lists_probed_is_brute_force(n_lists):
+def test_all_lists_probed_is_brute_force(n_lists, key_format):
     rng = np.random.default_rng(n_lists)
-    pool, bits = random_pool(rng, 300, 32)
+    pool, bits = random_pool(rng, 300, 32, key_format=key_format)
     idx = OracleIndex(pool, f2b(rng.standard_normal((n_lists, 32)).astype(np.float32)))
     idx.refresh()
     assert idx.n_indexed == 300 and sum(len(l) for l in idx.lists()) == 300
@@ -175,6 +176,62 @@ def pm1_pool(rows):
     pool = OraclePool(16)
     pool.append(f2b(np.asarray(rows, dtype=np.float32)), np.arange(len(rows), dtype=np.int32), tag=1)
     return pool
+
+
+# ------------------------------------------------------------------ 8-bit pools ----
+
+def test_8bit_rows_along_axes_and_diagonals_fall_into_the_lists_read_off_by_hand():
+    # A row along an axis keeps one non-zero code, so whatever its scale it dequantises to a
+    # multiple of that axis and, as a query, normalises to the axis exactly; a row with two
+    # equal entries keeps two equal codes and so ties between the two axes, to the lower one.
+    r = np.float32(1.0)
+    rows = np.array([[r, 0, 0, 0], [0, 3 * r, 0, 0], [-r, 0, 0, 0], [0, 0, 0.5 * r, 0],
+                     [r, r, 0, 0], [0, r, r, 0], [0, 0, -2 * r, 0]], dtype=np.float32)
+    pool = OraclePool(4, "e4m3")
+    pool.append(f2b(rows), np.arange(7, dtype=np.int32) + 10, tag=1)
+    idx = OracleIndex(pool, f2b(np.eye(4, dtype=np.float32)[:3]))
+    idx.refresh()
+    #   e0 -> 0, 3 e1 -> 1, -e0 -> scores (-1, 0, 0): tie of lists 1 and 2 -> 1, e2/2 -> 2,
+    #   e0+e1 -> tie 0/1 -> 0, e1+e2 -> tie 1/2 -> 1, -2 e2 -> scores (0, 0, -1) -> tie 0/1 -> 0
+    assert idx.assign.tolist() == [0, 1, 1, 2, 0, 1, 0]
+    # the rows as the index sees them: element = fp32(value(code) * scale), one rounding
+    got = idx._stored_f32(0, 7)
+    codes, scales = pool.codes, pool.scales
+    for i in range(7):
+        for j in range(4):
+            want = np.float32(np.float64(oracle.e4m3_decode(int(codes[i, j]))) * np.float64(scales[i]))
+            assert got[i, j] == want
+        assert np.count_nonzero(got[i]) == np.count_nonzero(rows[i])
+    assert got[4, 0] == got[4, 1] and got[5, 1] == got[5, 2]
+    # and as queries: bf16 of those elements
+    assert np.array_equal(idx._stored_as_queries(0, 7), f2b(got))
+    # a lookup probes by the query, scores by the 8-bit pool's own rule
+    q = f2b(np.array([[1.0, 0.2, 0.0, 0.0]], dtype=np.float32))
+    assert idx.probes(q, 2).tolist() == [[0, 1]]
+    one = idx.query(q, 1, fixed(3))
+    assert one.idx[0].tolist() == [0, 4, 6]                 # list 0 = rows 0, 4, 6: cos .98, .83, 0
+    full = pool.query(q, fixed(3))
+    assert np.array_equal(one.score[0, :2], full.score[0, :2])
+
+
+def test_8bit_training_takes_the_means_of_the_dequantised_elements():
+    rng = np.random.default_rng(5)
+    d, n = 8, 120
+    rows = (rng.standard_normal((n, d)) * np.exp(rng.uniform(-4, 0, size=(n, d)))).astype(np.float32)
+    pool = OraclePool(d, "e4m3")
+    pool.append(f2b(rows), np.arange(n, dtype=np.int32), tag=1)
+    idx = OracleIndex(pool, f2b(np.ones((1, d), dtype=np.float32)))
+    idx.train(1)                                            # one list: the mean of every row
+    from fractions import Fraction
+    codes, scales = pool.codes, pool.scales
+    for j in range(d):
+        total = 0
+        for i in reversed(range(n)):                        # Python ints, another order
+            x = np.float32(np.float64(oracle.e4m3_decode(int(codes[i, j]))) * np.float64(scales[i]))
+            total += int(np.trunc(np.float64(x) * 2.0 ** 30))
+        want = f2b(np.array([np.float32(float(Fraction(total, n * 2 ** 30)))]))[0]
+        assert idx.cent_raw[0, j] == want
+    assert idx.n_indexed == n and idx.assign.tolist() == [0] * n
 
 
 def test_one_iteration_by_hand():

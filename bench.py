@@ -1054,7 +1054,7 @@ def index_line(args):
     w = W.CONFIGS[args.config or "C2"]
     n0 = args.rows or (W.C5_START_ROWS if w.name == "C5" else w.n_rows)
     K, Wm = args.steps, args.warmup
-    pool = B.Pool(w.d, n0 + 8, max_nq=64, max_k=w.k, max_traces=w.num_traces + 8)
+    pool = B.Pool(w.d, n0 + 8, max_nq=64, max_k=w.k, max_traces=w.num_traces + 8, key_format=args.keys)
     fill_pool(pool, w, n0, dev)
     # lists: about sqrt(16 N), a power of two, which balances the centroid scan against the
     # candidates of 16 probed lists; their first centroids: the states of whole stored traces
@@ -1140,12 +1140,15 @@ def index_line(args):
     head = dict(trained[1])                      # four probes after training
     head["queries_per_sec"] = 1e6 / head["us_per_query"]
     peaks, peak_kind = measured_peaks()
-    cand_bytes = (n_lists + 4 * float(lens_t.mean())) * w.d * 2
+    row_bytes = w.d * 2 if args.keys == "bf16" else w.d + 4
+    cand_bytes = n_lists * w.d * 2 + 4 * float(lens_t.mean()) * row_bytes
+    # a single 16-bit lookup is one launch; 8-bit pools take the four separate ones
+    launches_per_lookup = 1 if args.keys == "bf16" else 4
     line = {"metric": "index_queries_per_sec", "value": head["queries_per_sec"], "unit": UNIT,
             "n_gpus": 1, "steps": K, "warmup": Wm, "ms_per_step": head["us_per_query"] / 1e3,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-            "dtype": "bf16 keys, fp32 accumulate", "data": "synthetic",
-            "config": {"workload": f"index: {w.name} recipe, pool N={n0} x d={w.d} bf16, {n_lists} lists "
+            "dtype": f"{args.keys} keys, fp32 accumulate", "data": "synthetic",
+            "config": {"workload": f"index: {w.name} recipe, pool N={n0} x d={w.d} {args.keys}, {n_lists} lists "
                                    f"(first centroids: stored states of whole traces, then "
                                    f"{n_train} iterations of training on the pool), nq=1, k={w.k}, "
                                    f"L={w.cont_len}; headline: n_probe=4 after training",
@@ -1159,7 +1162,7 @@ def index_line(args):
                                "rows_per_list": {"mean": float(lens_t.mean()), "max": int(lens_t.max()),
                                                  "empty_lists": int((lens_t == 0).sum())}},
             "refresh": {"rows": n0, "seconds": refresh_s, "rows_per_sec": n0 / refresh_s},
-            "clocks": clocks, "gpu_launches": 4 * K,
+            "clocks": clocks, "gpu_launches": launches_per_lookup * K,
             "roofline": {"bound": "hbm", "kernel": "centroid lookup + candidate scan (n_probe = 4)",
                          "achieved": cand_bytes / (head["us_per_query"] * 1e-6) / 1e9,
                          "peak": peaks["hbm_gbs"], "unit": "GB/s",

@@ -529,7 +529,11 @@ int oilbird_merge_chains(int32_t nq, const int32_t* sem_tok, const int32_t* sem_
  *     row ascending) with the firing rule, depths and continuations of Eq. 2 and Eq. 3.
  * The answer is oilbird_pool_query's answer restricted to the candidate rows: identical when
  * every list is probed, otherwise approximate (rows of lists that were not probed cannot be
- * found).  16-bit pools only.  create() copies the centroids (enqueued on cuda_stream); the
+ * found).  Pools of either key format.  In an 8-bit pool element j of stored row i is
+ * fp32(value(code_ij) * scale_i), one rounding (the library's reading); a row is assigned
+ * through those elements rounded to bf16, taken as a query state; candidates are scored as
+ * oilbird_pool_query scores the rows of an 8-bit pool; training takes the means of the fp32
+ * elements.  create() copies the centroids (enqueued on cuda_stream); the
  * caller's array is free again once that work has completed.  After oilbird_pool_reset or
  * oilbird_pool_evict_oldest the row numbers the index holds are stale: call
  * oilbird_index_reset (all rows become tail) and refresh again; until then refresh and query
@@ -537,11 +541,11 @@ int oilbird_merge_chains(int32_t nq, const int32_t* sem_tok, const int32_t* sem_
  * were built under).  Index calls enqueue on
  * cuda_stream and use the pool's scratch, so they follow the pool's one-stream, one-thread
  * rule.  Destroy the index before its pool.
- * Launches: a lookup of one query with up to 32 probes and params->path == OILBIRD_PATH_AUTO
- * is a single kernel (centroid scan, choice of the probes, candidate scan, merge, firing
+ * Launches: on a 16-bit pool a lookup of one query with up to 32 probes and params->path ==
+ * OILBIRD_PATH_AUTO is a single kernel (centroid scan, choice of the probes, candidate scan, merge, firing
  * rule and gather; its CTAs meet at four words of device memory per query, with the
  * library's bounded wait: a wait that runs out raises the pool's `stalled` status, and
- * oilbird_index_reset clears the words).  Batches, more probes, and any explicit
+ * oilbird_index_reset clears the words).  Batches, more probes, 8-bit pools and any explicit
  * params->path take four launches: oilbird_pool_query on the centroids (scan + merge), the
  * candidate scan, the merge.  The answers are the same.
  */

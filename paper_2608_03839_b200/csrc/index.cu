@@ -26,6 +26,7 @@
 #include "internal.h"
 #include "normalize.cuh"
 #include "pool_priv.h"
+#include "quant8.cuh"
 
 namespace oilbird {
 
@@ -294,6 +295,211 @@ scan_ids_kernel(PoolView pv, const uint16_t* __restrict__ q_raw, int nq, int k,
   }
   scan_candidates<E>(pv, qs, scratch, q, nq, k, blockIdx.x, gridDim.x, probes, n_probe, list_off,
                      list_rows, n_indexed, exclude_tag, partial, s_pref, s_base);
+}
+
+// ------------------------------------------------------------------- 8-bit pools ---
+// What a stored row of an 8-bit pool is, as a state (the library's reading; the paper defines
+// neither the quantised store nor the index): element j of row i is fp32(value(code_ij) *
+// scale_i), one rounding.  As a query state (the assignment of a row to its list) the row is
+// those elements rounded to bf16, like any state the library is handed.
+__global__ void __launch_bounds__(256)
+dequant_rows_kernel(const uint8_t* __restrict__ codes, const float* __restrict__ scales, int d,
+                    int row0, uint16_t* __restrict__ out) {
+  pdl_enter();
+  const int r = blockIdx.x;
+  const float sc = scales[row0 + r];
+  const uint4* src = reinterpret_cast<const uint4*>(codes + (size_t)(row0 + r) * d);
+  uint4* dst = reinterpret_cast<uint4*>(out + (size_t)r * d);
+  for (int c = threadIdx.x; c < (d >> 4); c += blockDim.x) {
+    const uint4 v = src[c];
+    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+    uint32_t o[8];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const float2 a = e4m3x2_to_float2(w[j] & 0xffffu), b = e4m3x2_to_float2(w[j] >> 16);
+      o[2 * j] = f32_to_bf16_bits(__fmul_rn(a.x, sc)) | (f32_to_bf16_bits(__fmul_rn(a.y, sc)) << 16);
+      o[2 * j + 1] = f32_to_bf16_bits(__fmul_rn(b.x, sc)) | (f32_to_bf16_bits(__fmul_rn(b.y, sc)) << 16);
+    }
+    dst[2 * c] = make_uint4(o[0], o[1], o[2], o[3]);
+    dst[2 * c + 1] = make_uint4(o[4], o[5], o[6], o[7]);
+  }
+}
+
+// The training means over an 8-bit pool: as index_means_kernel, each element contributing
+// trunc(x * 2^30) with x = fp32(value(code) * scale).  A thread holds 16-code chunks.
+constexpr int kMeanChunks8 = 2;         // 16-code chunks of the row width per thread: d <= 8192
+__global__ void __launch_bounds__(256)
+index_means_e4m3_kernel(const uint8_t* __restrict__ codes, const float* __restrict__ scales, int d,
+                        const int32_t* __restrict__ list_off, const int32_t* __restrict__ list_rows,
+                        uint16_t* __restrict__ cent_raw) {
+  pdl_enter();
+  const int l = blockIdx.x;
+  const int lo = list_off[l], hi = list_off[l + 1];
+  if (hi == lo) return;
+  const int n16 = d >> 4;
+  long long acc[kMeanChunks8][16];
+#pragma unroll
+  for (int u = 0; u < kMeanChunks8; ++u)
+#pragma unroll
+    for (int j = 0; j < 16; ++j) acc[u][j] = 0;
+  for (int i = lo; i < hi; ++i) {
+    const int row = list_rows[i];
+    const float sc = scales[row];
+    const uint4* src = reinterpret_cast<const uint4*>(codes + (size_t)row * d);
+#pragma unroll
+    for (int u = 0; u < kMeanChunks8; ++u) {
+      const int c = threadIdx.x + u * 256;
+      if (c < n16) {
+        const uint4 v = __ldg(src + c);
+        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          const float2 a = e4m3x2_to_float2(w[j] & 0xffffu), b = e4m3x2_to_float2(w[j] >> 16);
+          acc[u][4 * j] += (long long)((double)__fmul_rn(a.x, sc) * 1073741824.0);       // truncates
+          acc[u][4 * j + 1] += (long long)((double)__fmul_rn(a.y, sc) * 1073741824.0);
+          acc[u][4 * j + 2] += (long long)((double)__fmul_rn(b.x, sc) * 1073741824.0);
+          acc[u][4 * j + 3] += (long long)((double)__fmul_rn(b.y, sc) * 1073741824.0);
+        }
+      }
+    }
+  }
+  const double denom = (double)(hi - lo) * 1073741824.0;
+  uint4* dst = reinterpret_cast<uint4*>(cent_raw + (size_t)l * d);
+#pragma unroll
+  for (int u = 0; u < kMeanChunks8; ++u) {
+    const int c = threadIdx.x + u * 256;
+    if (c < n16) {
+      uint32_t o[8];
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        const float a = __double2float_rn(__ll2double_rn(acc[u][2 * j]) / denom);
+        const float b = __double2float_rn(__ll2double_rn(acc[u][2 * j + 1]) / denom);
+        o[j] = f32_to_bf16_bits(a) | (f32_to_bf16_bits(b) << 16);
+      }
+      dst[2 * c] = make_uint4(o[0], o[1], o[2], o[3]);
+      dst[2 * c + 1] = make_uint4(o[4], o[5], o[6], o[7]);
+    }
+  }
+}
+
+// One row of codes against the query in shared memory: a lane adds its elements in the order
+// the 8-bit CUDA-core scan adds them (16-code chunks lane, lane + 32, ...; within a chunk
+// element by element), so the score has that scan's bits.  Up to kWide8 chunks in flight.
+constexpr int kWide8 = 8;
+__device__ __forceinline__ float score_code_row(const uint4* row, const uint4* qs, int n16, int lane) {
+  float a = 0.f;
+  for (int c0 = lane; c0 < n16; c0 += 32 * kWide8) {
+    uint4 kv[kWide8];
+#pragma unroll
+    for (int u = 0; u < kWide8; ++u) {
+      const int c = c0 + 32 * u;
+      kv[u] = c < n16 ? ld_stream16(row + c) : make_uint4(0, 0, 0, 0);
+    }
+#pragma unroll
+    for (int u = 0; u < kWide8; ++u) {
+      const int c = c0 + 32 * u;
+      if (c < n16) {
+        const uint4 qa = qs[2 * c], qb = qs[2 * c + 1];
+        const uint32_t w[4] = {kv[u].x, kv[u].y, kv[u].z, kv[u].w};
+        const uint32_t qw[8] = {qa.x, qa.y, qa.z, qa.w, qb.x, qb.y, qb.z, qb.w};
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          const float2 ka = e4m3x2_to_float2(w[j] & 0xffffu), kb = e4m3x2_to_float2(w[j] >> 16);
+          a = fmaf(ka.x, bf16_lo(qw[2 * j]), a);
+          a = fmaf(ka.y, bf16_hi(qw[2 * j]), a);
+          a = fmaf(kb.x, bf16_lo(qw[2 * j + 1]), a);
+          a = fmaf(kb.y, bf16_hi(qw[2 * j + 1]), a);
+        }
+      }
+    }
+  }
+  return warp_sum(a);
+}
+
+// The candidate scan over an 8-bit pool: scan_candidates with the rows' codes and scales.
+template <int E>
+__global__ void __launch_bounds__(kNormThreads, 2)
+scan_ids_e4m3_kernel(PoolView pv, const uint8_t* __restrict__ codes, const float* __restrict__ scales,
+                     const uint16_t* __restrict__ q_raw, int nq, int k,
+                     const int32_t* __restrict__ probes, int n_probe,
+                     const int32_t* __restrict__ list_off, const int32_t* __restrict__ list_rows,
+                     int n_indexed, const uint64_t* __restrict__ exclude_tag, u64* __restrict__ partial,
+                     int32_t* __restrict__ q_valid, DeviceStats* stats) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  __shared__ int s_pref[kIndexMaxProbe + 1], s_base[kIndexMaxProbe];
+  constexpr int KK = 32 * E;
+  constexpr int kWarps = kNormThreads / 32;
+  pdl_enter();
+  const int d = pv.d, n16 = d >> 4;
+  uint4* qs = reinterpret_cast<uint4*>(smem_raw);                        // [d / 8] bf16
+  u64* scratch = reinterpret_cast<u64*>(smem_raw + (size_t)d * 2);        // [warps][KK]
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int q = blockIdx.y, b = blockIdx.x, G = gridDim.x;
+  const int code = normalize_row<true, 2>(q_raw + (size_t)q * d, reinterpret_cast<uint16_t*>(qs), d);
+  if (b == 0 && threadIdx.x == 0) {
+    q_valid[q] = code == kRowNonFinite ? 0 : 1;          // NaN/Inf: no neighbours
+    if (code == kRowNonFinite) atomicAdd(&stats->nonfinite_queries, 1ull);
+  }
+  if (threadIdx.x < n_probe) {
+    const int l = probes[(size_t)q * n_probe + threadIdx.x];
+    s_base[threadIdx.x] = l >= 0 ? list_off[l] : 0;
+    s_pref[threadIdx.x + 1] = l >= 0 ? list_off[l + 1] - list_off[l] : 0;
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    s_pref[0] = 0;
+    for (int p = 0; p < n_probe; ++p) s_pref[p + 1] += s_pref[p];
+  }
+  __syncthreads();
+  const int in_lists = s_pref[n_probe];
+  const int total = in_lists + (pv.n_rows - n_indexed);
+  const uint64_t ex = exclude_tag ? exclude_tag[q] : 0;
+  const int c_lo = (int)(((long long)total * b) / G);
+  const int c_hi = (int)(((long long)total * (b + 1)) / G);
+  const uint4* codes4 = reinterpret_cast<const uint4*>(codes);
+  u64 top[E];
+  u64 kth = 0;
+#pragma unroll
+  for (int r = 0; r < E; ++r) top[r] = 0;
+  for (int c = c_lo + warp; c < c_hi; c += kWarps) {
+    int row;
+    if (c >= in_lists) {
+      row = n_indexed + (c - in_lists);                            // the tail
+    } else {
+      int lo = 0, hi = n_probe;                                    // last p with s_pref[p] <= c
+      while (hi - lo > 1) {
+        const int mid = (lo + hi) >> 1;
+        if (s_pref[mid] <= c) lo = mid; else hi = mid;
+      }
+      row = list_rows[s_base[lo] + (c - s_pref[lo])];
+    }
+    const float sc = scales[row];
+    const float s = score_code_row(codes4 + (size_t)row * n16, qs, n16, lane) * sc;
+    if (ex != 0 && pv.trace_tag[pv.trace_id[row]] == ex) continue;     // same-prompt trace
+    const u64 key = pack_candidate(s, (uint32_t)row);
+    if (key > kth) {
+      warp_sorted_insert<E>(top, key, lane);
+      kth = warp_list_get<E>(top, k - 1);
+    }
+  }
+  block_merge_desc<E>(top, scratch, kWarps);
+  if (threadIdx.x < 32) {
+    u64* dst = partial + ((size_t)b * nq + q) * KK;
+#pragma unroll
+    for (int r = 0; r < E; ++r) dst[r * 32 + lane] = top[r];
+  }
+}
+
+template <int E>
+static cudaError_t launch_scan_ids_e4m3(const PoolView& pv, const uint8_t* codes, const float* scales,
+                                        const uint16_t* q, int nq, int k, const int32_t* probes,
+                                        int n_probe, const int32_t* list_off, const int32_t* list_rows,
+                                        int n_indexed, const uint64_t* ex, u64* partial,
+                                        int32_t* q_valid, DeviceStats* stats, int grid, cudaStream_t st) {
+  const size_t smem = (size_t)pv.d * 2 + (size_t)(kNormThreads / 32) * 32 * E * sizeof(u64);
+  return launch_pdl(scan_ids_e4m3_kernel<E>, dim3(grid, nq), dim3(kNormThreads), smem, st, pv, codes,
+                    scales, q, nq, k, probes, n_probe, list_off, list_rows, n_indexed, ex, partial,
+                    q_valid, stats);
 }
 
 // ------------------------------------------------------------ folding lists on one CTA ---
@@ -575,6 +781,11 @@ cudaError_t preload_index_kernels() {
   if ((e = preload_kernel(index_offsets_kernel)) != cudaSuccess) return e;
   if ((e = preload_kernel(index_scatter_kernel)) != cudaSuccess) return e;
   if ((e = preload_kernel(index_means_kernel)) != cudaSuccess) return e;
+  if ((e = preload_kernel(dequant_rows_kernel)) != cudaSuccess) return e;
+  if ((e = preload_kernel(index_means_e4m3_kernel)) != cudaSuccess) return e;
+  if ((e = preload_kernel(scan_ids_e4m3_kernel<1>, true)) != cudaSuccess) return e;
+  if ((e = preload_kernel(scan_ids_e4m3_kernel<2>, true)) != cudaSuccess) return e;
+  if ((e = preload_kernel(scan_ids_e4m3_kernel<4>, true)) != cudaSuccess) return e;
   if ((e = preload_kernel(index_lookup_kernel<1>, true)) != cudaSuccess) return e;
   if ((e = preload_kernel(index_lookup_kernel<2>, true)) != cudaSuccess) return e;
   if ((e = preload_kernel(index_lookup_kernel<4>, true)) != cudaSuccess) return e;
@@ -600,6 +811,7 @@ struct oilbird_index {
   int32_t* probe_idx; float* probe_score; int32_t *probe_fired, *probe_len, *probe_tok;
   float* a_score; int32_t *a_fired, *a_len, *a_tok;
   oilbird::LookupSync* sync;     // one-launch lookups: four words per query, zero between launches
+  uint16_t* as_query;            // 8-bit pools: a batch of stored rows as bf16 query states
 };
 
 static thread_local char g_index_err[256] = "";
@@ -622,7 +834,6 @@ int oilbird_index_create(oilbird_index_t** out, oilbird_pool_t* pool, const void
   if (!out) return OILBIRD_EINVAL;
   *out = nullptr;
   if (!pool || !centroids_bf16 || n_lists < 1 || n_lists > kIndexMaxLists) return OILBIRD_EINVAL;
-  if (pool->r.e4m3) return OILBIRD_EINVAL;                       // rows are fetched as bf16 keys
   if ((uintptr_t)centroids_bf16 & 15) return OILBIRD_EINVAL;
   ICU(cudaSetDevice(pool->device));
   oilbird_index* ix = new (std::nothrow) oilbird_index();
@@ -649,7 +860,8 @@ int oilbird_index_create(oilbird_index_t** out, oilbird_pool_t* pool, const void
                o_af = o_as + up(kIndexAssignBatch * 4), o_al = o_af + up(kIndexAssignBatch * 4),
                o_at = o_al + up(kIndexAssignBatch * 4), o_sync = o_at + up(kIndexAssignBatch * 4),
                o_raw = o_sync + up((size_t)OILBIRD_MAX_NQ * sizeof(LookupSync)),
-               total = o_raw + up(nl * (size_t)pool->r.d * 2);
+               o_asq = o_raw + up(nl * (size_t)pool->r.d * 2),
+               total = o_asq + (pool->r.e4m3 ? up((size_t)kIndexAssignBatch * pool->r.d * 2) : 0);
   cudaError_t e = cudaMalloc((void**)&ix->mem, total);
   if (e != cudaSuccess) { oilbird_pool_destroy(ix->cent); delete ix; return index_fail(e, "cudaMalloc(index)"); }
   ix->assign = (int32_t*)(ix->mem + o_assign); ix->list_rows = (int32_t*)(ix->mem + o_rows);
@@ -662,6 +874,7 @@ int oilbird_index_create(oilbird_index_t** out, oilbird_pool_t* pool, const void
   ix->a_len = (int32_t*)(ix->mem + o_al); ix->a_tok = (int32_t*)(ix->mem + o_at);
   ix->cent_raw = (uint16_t*)(ix->mem + o_raw);
   ix->sync = (LookupSync*)(ix->mem + o_sync);
+  ix->as_query = pool->r.e4m3 ? (uint16_t*)(ix->mem + o_asq) : nullptr;
   cudaStream_t st = (cudaStream_t)cuda_stream;
   // the centroids become the rows of a one-trace pool (their tokens are never looked at);
   // all lists start empty
@@ -723,7 +936,17 @@ int oilbird_index_refresh(oilbird_index_t* ix, void* cuda_stream) {
     oilbird_query_out o;
     o.idx = ix->assign + r0; o.score = ix->a_score; o.fired = ix->a_fired;
     o.cont_len = ix->a_len; o.cont_tok = ix->a_tok;
-    int rc = oilbird_pool_query(ix->cent, p->keys + (size_t)r0 * p->r.d, nq, &pr, &o, st);
+    const uint16_t* states = p->keys + (size_t)r0 * p->r.d;       // the stored keys as queries
+    if (p->r.e4m3) {
+      // 8-bit pools: the stored rows as bf16 states (fp32(value(code) * scale) rounded to bf16)
+      cudaError_t e = launch_pdl(dequant_rows_kernel, dim3(nq), dim3(256), 0, st,
+                                 (const uint8_t*)p->codes, (const float*)p->scales, (int)p->r.d,
+                                 (int)r0, ix->as_query);
+      if (e != cudaSuccess) return index_fail(e, "dequantise kernel");
+      p->launches += 1;
+      states = ix->as_query;
+    }
+    int rc = oilbird_pool_query(ix->cent, states, nq, &pr, &o, st);
     if (rc) return rc;
   }
   // rebuild the lists over all indexed rows: count, offsets, scatter
@@ -756,7 +979,11 @@ int oilbird_index_train(oilbird_index_t* ix, int32_t iterations, void* cuda_stre
     if (!rc) rc = oilbird_index_refresh(ix, cuda_stream);
     if (rc) return rc;
     if (ix->n_indexed == 0) break;                     // no rows: nothing to learn from
-    cudaError_t e = launch_pdl(index_means_kernel, dim3(ix->n_lists), dim3(256), 0, st,
+    cudaError_t e =
+        p->r.e4m3 ? launch_pdl(index_means_e4m3_kernel, dim3(ix->n_lists), dim3(256), 0, st,
+                               (const uint8_t*)p->codes, (const float*)p->scales, (int)p->r.d,
+                               (const int32_t*)ix->list_off, (const int32_t*)ix->list_rows, ix->cent_raw)
+                  : launch_pdl(index_means_kernel, dim3(ix->n_lists), dim3(256), 0, st,
                                (const uint16_t*)p->keys, (int)p->r.d, (const int32_t*)ix->list_off,
                                (const int32_t*)ix->list_rows, ix->cent_raw);
     if (e != cudaSuccess) return index_fail(e, "index means kernel");
@@ -807,7 +1034,7 @@ int oilbird_index_query(oilbird_index_t* ix, const void* q_bf16, int32_t nq, int
   const int kk = list_len(pr->k);
   PoolView pv = pool_view(p);
   const uint16_t* q = (const uint16_t*)q_bf16;
-  if (nq <= kLookupMaxNq && n_probe <= 32 && pr->path == OILBIRD_PATH_AUTO) {
+  if (nq <= kLookupMaxNq && n_probe <= 32 && pr->path == OILBIRD_PATH_AUTO && !p->r.e4m3) {
     // small batches: centroid scan, probes and candidate scan in one launch, then the merge
     if (preload_all_kernels() != cudaSuccess) return OILBIRD_ECUDA;
     // Twice the CTAs that fit at once (two per SM): the first half takes the centroids and
@@ -855,7 +1082,14 @@ int oilbird_index_query(oilbird_index_t* ix, const void* q_bf16, int32_t nq, int
   }
   if (grid > p->r.max_lists) grid = p->r.max_lists;
   cudaError_t e;
-  if (kk == 32)
+  if (p->r.e4m3) {
+#define SCAN8(E)                                                                                  \
+    launch_scan_ids_e4m3<E>(pv, p->codes, p->scales, q, nq, pr->k, ix->probe_idx, n_probe,       \
+                            ix->list_off, ix->list_rows, (int)ix->n_indexed, pr->exclude_tag,     \
+                            p->partial, p->q_valid, p->stats, grid, st)
+    e = kk == 32 ? SCAN8(1) : (kk == 64 ? SCAN8(2) : SCAN8(4));
+#undef SCAN8
+  } else if (kk == 32)
     e = launch_scan_ids<1>(pv, q, nq, pr->k, ix->probe_idx, n_probe, ix->list_off, ix->list_rows,
                            (int)ix->n_indexed, pr->exclude_tag, p->partial, p->q_valid, p->stats, grid, st);
   else if (kk == 64)

@@ -66,13 +66,6 @@ constexpr int kQ8Threads = kNormThreads;
 constexpr int kQ8Warps = kQ8Threads / 32;
 constexpr int kQ8Rows = 4;        // rows a warp scores together
 
-// two E4M3 codes -> two floats (exact)
-__device__ __forceinline__ float2 e4m3x2_to_float2(uint32_t two_codes) {
-  uint32_t h2;
-  asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(h2) : "h"((unsigned short)two_codes));
-  return __half22float2(*reinterpret_cast<const __half2*>(&h2));
-}
-
 // Same structure as the 16-bit CUDA-core scan: 2 CTAs x 8 warps per SM, contiguous row
 // split, 16-byte streaming loads (16 codes), the normalised bf16 queries in shared memory,
 // fp32 accumulation, per-warp sorted register lists, one list per CTA and query.

@@ -1,10 +1,19 @@
 // Row quantiser of pools with 8-bit keys (FP8 E4M3 codes + one fp32 scale per row), shared by
 // the append kernel and by the scans that append a serving step's rows themselves.
 #pragma once
+#include <cuda_fp16.h>
+
 #include "common.cuh"
 #include "normalize.cuh"
 
 namespace oilbird {
+
+// two E4M3 codes -> two floats (exact)
+__device__ __forceinline__ float2 e4m3x2_to_float2(uint32_t two_codes) {
+  uint32_t h2;
+  asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(h2) : "h"((unsigned short)two_codes));
+  return __half22float2(*reinterpret_cast<const __half2*>(&h2));
+}
 
 // ---------------------------------------------------------------- E4M3 encode ---
 // Nearest E4M3 code of t (double), ties to the even code, |t| >= 448 saturates to 448;

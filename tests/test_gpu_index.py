@@ -227,18 +227,67 @@ def test_c2_shaped_pool_recall_and_candidate_volume():
 
 
 def test_bad_arguments_are_refused():
-    pool = B.Pool(64, 100, key_format="e4m3")
     cent = torch.zeros(4, 64, dtype=torch.bfloat16, device="cuda")
-    with pytest.raises(B.OilbirdError) as e:
-        B.Index(pool, cent)                                  # 16-bit pools only
-    assert e.value.code == B.EINVAL
     pool = B.Pool(64, 100)
+    with pytest.raises(B.OilbirdError) as e:
+        B.Index(pool, torch.zeros(0, 64, dtype=torch.bfloat16, device="cuda"))   # no lists
+    assert e.value.code == B.EINVAL
     ix = B.Index(pool, cent)
     q = torch.zeros(1, 64, dtype=torch.bfloat16, device="cuda")
     with pytest.raises(B.OilbirdError):
         ix.query(q, 0, fixed(4, 2))                          # at least one probe
     out = ix.query(q, 2, fixed(4, 2)).cpu()                  # an empty pool is legal
     assert torch.all(out.idx == -1) and out.fired[0] == 0
+
+
+def test_index_over_an_8bit_pool_matches_the_oracle():
+    """Codes and scales in place of keys: rows are assigned through their dequantised form
+    (fp32(value(code) * scale), rounded to bf16 as a query), candidates are scored by the 8-bit
+    pool's own rule, training takes the means of the dequantised elements."""
+    w = W.C1.scaled(n_rows=6000, nq=5, d=256, k=8, cont_len=4, n_centroids=24, rows_per_trace=500, seed=41)
+    pool, ora = fill_both(w, key_format="e4m3", spare_rows=300, max_nq=16)
+    assign = np.concatenate([w.trace_assign(t, "cuda").cpu().numpy() for t in range(w.num_traces)])[: w.n_rows]
+    first = [int(np.nonzero(assign == c)[0][0]) for c in range(24)]      # one row of every cluster
+    keys_raw = torch.cat([st for st, _, _ in w.traces("cuda")])[: w.n_rows]
+    cent = keys_raw[first].contiguous()
+    gix, oix = B.Index(pool, cent), OracleIndex(ora, W.to_bits(cent))
+    gix.refresh(); oix.refresh()
+    assert len(gix) == 6000
+    same_lists(gix, oix)
+    q, _ = w.queries("cuda")
+    for n_probe in (1, 3, 24, 30):
+        for k in (1, 8, 40):
+            pr = fixed(k, 4, theta=0.8 if k == 8 else -2.0)
+            check_index_query(gix.query(q, n_probe, pr), oix, W.to_bits(q), n_probe, pr)
+    # every list probed: the 8-bit pool's own full scan (single queries share its arithmetic)
+    pr = fixed(8, 4)
+    for i in range(2):
+        a, b = gix.query(q[i:i + 1].contiguous(), 24, pr).cpu(), pool.query(q[i:i + 1].contiguous(), pr).cpu()
+        assert torch.equal(a.idx, b.idx) and torch.equal(a.score, b.score) and torch.equal(a.cont_tok, b.cont_tok)
+    # the tail, then a refresh; exclusion tags
+    g = torch.Generator(device="cuda").manual_seed(3)
+    st = torch.randn(200, w.d, generator=g, device="cuda").to(torch.bfloat16)
+    tk = torch.arange(200, dtype=torch.int32, device="cuda")
+    pool.append(st, tk, tag=77)
+    ora.append(W.to_bits(st), tk.cpu().numpy(), tag=77)
+    q2 = torch.cat([st[17:18], q[:2]]).contiguous()
+    out = gix.query(q2, 1, fixed(4, 4))
+    assert int(out.idx[0, 0]) == 6017
+    check_index_query(out, oix, W.to_bits(q2), 1, fixed(4, 4))
+    gix.refresh(); oix.refresh()
+    same_lists(gix, oix)
+    ex = np.array([77, 0, 3], dtype=np.uint64)
+    pr = fixed(6, 4, exclude_tag=torch.from_numpy(ex.view(np.int64)).cuda())
+    check_index_query(gix.query(q2, 4, pr), oix, W.to_bits(q2), 4, pr, exclude=ex)
+    # training: raw centroids, assignments and lists identical after one and three iterations
+    done = 0
+    for upto in (1, 3):
+        gix.train(upto - done); oix.train(upto - done)
+        done = upto
+        assert np.array_equal(gix.centroids(), oix.cent_raw)
+        same_lists(gix, oix)
+    check_index_query(gix.query(q, 3, fixed(8, 4)), oix, W.to_bits(q), 3, fixed(8, 4))
+    assert pool.stats()["stalled"] == 0
 
 
 def test_training_matches_the_oracle_bit_for_bit():

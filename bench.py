@@ -1142,8 +1142,7 @@ def index_line(args):
     peaks, peak_kind = measured_peaks()
     row_bytes = w.d * 2 if args.keys == "bf16" else w.d + 4
     cand_bytes = n_lists * w.d * 2 + 4 * float(lens_t.mean()) * row_bytes
-    # a single 16-bit lookup is one launch; 8-bit pools take the four separate ones
-    launches_per_lookup = 1 if args.keys == "bf16" else 4
+    launches_per_lookup = 1                       # a single query's lookup is one launch
     line = {"metric": "index_queries_per_sec", "value": head["queries_per_sec"], "unit": UNIT,
             "n_gpus": 1, "steps": K, "warmup": Wm, "ms_per_step": head["us_per_query"] / 1e3,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None,

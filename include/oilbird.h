@@ -541,11 +541,11 @@ int oilbird_merge_chains(int32_t nq, const int32_t* sem_tok, const int32_t* sem_
  * were built under).  Index calls enqueue on
  * cuda_stream and use the pool's scratch, so they follow the pool's one-stream, one-thread
  * rule.  Destroy the index before its pool.
- * Launches: on a 16-bit pool a lookup of one query with up to 32 probes and params->path ==
+ * Launches: a lookup of one query with up to 32 probes and params->path ==
  * OILBIRD_PATH_AUTO is a single kernel (centroid scan, choice of the probes, candidate scan, merge, firing
  * rule and gather; its CTAs meet at four words of device memory per query, with the
  * library's bounded wait: a wait that runs out raises the pool's `stalled` status, and
- * oilbird_index_reset clears the words).  Batches, more probes, 8-bit pools and any explicit
+ * oilbird_index_reset clears the words).  Batches, more probes and any explicit
  * params->path take four launches: oilbird_pool_query on the centroids (scan + merge), the
  * candidate scan, the merge.  The answers are the same.
  */

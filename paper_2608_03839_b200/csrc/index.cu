@@ -183,15 +183,52 @@ __device__ __forceinline__ float score_row_wide(const uint4* row, const uint4* q
 // CTAs with at most this many rows each take them one row per warp at a time
 constexpr int kWideMaxRows = 64;
 
-// The candidate scan of CTA b of G for query q, whose normalised form is in qs.
-template <int E>
+// One row of codes against the query in shared memory: a lane adds its elements in the order
+// the 8-bit CUDA-core scan adds them (16-code chunks lane, lane + 32, ...; within a chunk
+// element by element), so the score has that scan's bits.  Up to kWide8 chunks in flight.
+constexpr int kWide8 = 8;
+__device__ __forceinline__ float score_code_row(const uint4* row, const uint4* qs, int n16, int lane) {
+  float a = 0.f;
+  for (int c0 = lane; c0 < n16; c0 += 32 * kWide8) {
+    uint4 kv[kWide8];
+#pragma unroll
+    for (int u = 0; u < kWide8; ++u) {
+      const int c = c0 + 32 * u;
+      kv[u] = c < n16 ? ld_stream16(row + c) : make_uint4(0, 0, 0, 0);
+    }
+#pragma unroll
+    for (int u = 0; u < kWide8; ++u) {
+      const int c = c0 + 32 * u;
+      if (c < n16) {
+        const uint4 qa = qs[2 * c], qb = qs[2 * c + 1];
+        const uint32_t w[4] = {kv[u].x, kv[u].y, kv[u].z, kv[u].w};
+        const uint32_t qw[8] = {qa.x, qa.y, qa.z, qa.w, qb.x, qb.y, qb.z, qb.w};
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          const float2 ka = e4m3x2_to_float2(w[j] & 0xffffu), kb = e4m3x2_to_float2(w[j] >> 16);
+          a = fmaf(ka.x, bf16_lo(qw[2 * j]), a);
+          a = fmaf(ka.y, bf16_hi(qw[2 * j]), a);
+          a = fmaf(kb.x, bf16_lo(qw[2 * j + 1]), a);
+          a = fmaf(kb.y, bf16_hi(qw[2 * j + 1]), a);
+        }
+      }
+    }
+  }
+  return warp_sum(a);
+}
+
+// The candidate scan of CTA b of G for query q, whose normalised form is in qs.  k8: the pool
+// holds E4M3 codes and one scale per row (scored as the 8-bit CUDA-core scan scores them).
+template <int E, bool k8 = false>
 __device__ __forceinline__ void scan_candidates(const PoolView& pv, const uint4* qs, u64* scratch,
                                                 int q, int nq, int k, int b, int G,
                                                 const int32_t* probes, int n_probe,
                                                 const int32_t* __restrict__ list_off,
                                                 const int32_t* __restrict__ list_rows, int n_indexed,
                                                 const uint64_t* __restrict__ exclude_tag,
-                                                u64* __restrict__ partial, int* s_pref, int* s_base) {
+                                                u64* __restrict__ partial, int* s_pref, int* s_base,
+                                                const uint8_t* __restrict__ codes = nullptr,
+                                                const float* __restrict__ scales = nullptr) {
   constexpr int KK = 32 * E;
   constexpr int kWarps = kNormThreads / 32;
   const int n_chunks = pv.d >> 3;
@@ -230,7 +267,21 @@ __device__ __forceinline__ void scan_candidates(const PoolView& pv, const uint4*
   u64 kth = 0;
 #pragma unroll
   for (int r = 0; r < E; ++r) top[0][r] = 0;
-  if (c_hi - c_lo <= kWideMaxRows) {
+  if (k8) {
+    const uint4* codes4 = reinterpret_cast<const uint4*>(codes);
+    const int n16 = pv.d >> 4;
+    for (int c = c_lo + warp; c < c_hi; c += kWarps) {
+      const int row = row_of(c);
+      const float sc = scales[row];
+      const float s = score_code_row(codes4 + (size_t)row * n16, qs, n16, lane) * sc;
+      if (ex != 0 && pv.trace_tag[pv.trace_id[row]] == ex) continue;       // same-prompt trace
+      const u64 key = pack_candidate(s, (uint32_t)row);
+      if (key > kth) {
+        warp_sorted_insert<E>(top[0], key, lane);
+        kth = warp_list_get<E>(top[0], k - 1);
+      }
+    }
+  } else if (c_hi - c_lo <= kWideMaxRows) {
     for (int c = c_lo + warp; c < c_hi; c += kWarps) {
       const int row = row_of(c);
       const float s = score_row_wide(keys4 + (size_t)row * n_chunks, qs, n_chunks, lane);
@@ -382,41 +433,7 @@ index_means_e4m3_kernel(const uint8_t* __restrict__ codes, const float* __restri
   }
 }
 
-// One row of codes against the query in shared memory: a lane adds its elements in the order
-// the 8-bit CUDA-core scan adds them (16-code chunks lane, lane + 32, ...; within a chunk
-// element by element), so the score has that scan's bits.  Up to kWide8 chunks in flight.
-constexpr int kWide8 = 8;
-__device__ __forceinline__ float score_code_row(const uint4* row, const uint4* qs, int n16, int lane) {
-  float a = 0.f;
-  for (int c0 = lane; c0 < n16; c0 += 32 * kWide8) {
-    uint4 kv[kWide8];
-#pragma unroll
-    for (int u = 0; u < kWide8; ++u) {
-      const int c = c0 + 32 * u;
-      kv[u] = c < n16 ? ld_stream16(row + c) : make_uint4(0, 0, 0, 0);
-    }
-#pragma unroll
-    for (int u = 0; u < kWide8; ++u) {
-      const int c = c0 + 32 * u;
-      if (c < n16) {
-        const uint4 qa = qs[2 * c], qb = qs[2 * c + 1];
-        const uint32_t w[4] = {kv[u].x, kv[u].y, kv[u].z, kv[u].w};
-        const uint32_t qw[8] = {qa.x, qa.y, qa.z, qa.w, qb.x, qb.y, qb.z, qb.w};
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-          const float2 ka = e4m3x2_to_float2(w[j] & 0xffffu), kb = e4m3x2_to_float2(w[j] >> 16);
-          a = fmaf(ka.x, bf16_lo(qw[2 * j]), a);
-          a = fmaf(ka.y, bf16_hi(qw[2 * j]), a);
-          a = fmaf(kb.x, bf16_lo(qw[2 * j + 1]), a);
-          a = fmaf(kb.y, bf16_hi(qw[2 * j + 1]), a);
-        }
-      }
-    }
-  }
-  return warp_sum(a);
-}
-
-// The candidate scan over an 8-bit pool: scan_candidates with the rows' codes and scales.
+// The candidate scan over an 8-bit pool (separate launches).
 template <int E>
 __global__ void __launch_bounds__(kNormThreads, 2)
 scan_ids_e4m3_kernel(PoolView pv, const uint8_t* __restrict__ codes, const float* __restrict__ scales,
@@ -427,67 +444,18 @@ scan_ids_e4m3_kernel(PoolView pv, const uint8_t* __restrict__ codes, const float
                      int32_t* __restrict__ q_valid, DeviceStats* stats) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   __shared__ int s_pref[kIndexMaxProbe + 1], s_base[kIndexMaxProbe];
-  constexpr int KK = 32 * E;
-  constexpr int kWarps = kNormThreads / 32;
   pdl_enter();
-  const int d = pv.d, n16 = d >> 4;
+  const int d = pv.d;
   uint4* qs = reinterpret_cast<uint4*>(smem_raw);                        // [d / 8] bf16
   u64* scratch = reinterpret_cast<u64*>(smem_raw + (size_t)d * 2);        // [warps][KK]
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int q = blockIdx.y, b = blockIdx.x, G = gridDim.x;
+  const int q = blockIdx.y;
   const int code = normalize_row<true, 2>(q_raw + (size_t)q * d, reinterpret_cast<uint16_t*>(qs), d);
-  if (b == 0 && threadIdx.x == 0) {
+  if (blockIdx.x == 0 && threadIdx.x == 0) {
     q_valid[q] = code == kRowNonFinite ? 0 : 1;          // NaN/Inf: no neighbours
     if (code == kRowNonFinite) atomicAdd(&stats->nonfinite_queries, 1ull);
   }
-  if (threadIdx.x < n_probe) {
-    const int l = probes[(size_t)q * n_probe + threadIdx.x];
-    s_base[threadIdx.x] = l >= 0 ? list_off[l] : 0;
-    s_pref[threadIdx.x + 1] = l >= 0 ? list_off[l + 1] - list_off[l] : 0;
-  }
-  __syncthreads();
-  if (threadIdx.x == 0) {
-    s_pref[0] = 0;
-    for (int p = 0; p < n_probe; ++p) s_pref[p + 1] += s_pref[p];
-  }
-  __syncthreads();
-  const int in_lists = s_pref[n_probe];
-  const int total = in_lists + (pv.n_rows - n_indexed);
-  const uint64_t ex = exclude_tag ? exclude_tag[q] : 0;
-  const int c_lo = (int)(((long long)total * b) / G);
-  const int c_hi = (int)(((long long)total * (b + 1)) / G);
-  const uint4* codes4 = reinterpret_cast<const uint4*>(codes);
-  u64 top[E];
-  u64 kth = 0;
-#pragma unroll
-  for (int r = 0; r < E; ++r) top[r] = 0;
-  for (int c = c_lo + warp; c < c_hi; c += kWarps) {
-    int row;
-    if (c >= in_lists) {
-      row = n_indexed + (c - in_lists);                            // the tail
-    } else {
-      int lo = 0, hi = n_probe;                                    // last p with s_pref[p] <= c
-      while (hi - lo > 1) {
-        const int mid = (lo + hi) >> 1;
-        if (s_pref[mid] <= c) lo = mid; else hi = mid;
-      }
-      row = list_rows[s_base[lo] + (c - s_pref[lo])];
-    }
-    const float sc = scales[row];
-    const float s = score_code_row(codes4 + (size_t)row * n16, qs, n16, lane) * sc;
-    if (ex != 0 && pv.trace_tag[pv.trace_id[row]] == ex) continue;     // same-prompt trace
-    const u64 key = pack_candidate(s, (uint32_t)row);
-    if (key > kth) {
-      warp_sorted_insert<E>(top, key, lane);
-      kth = warp_list_get<E>(top, k - 1);
-    }
-  }
-  block_merge_desc<E>(top, scratch, kWarps);
-  if (threadIdx.x < 32) {
-    u64* dst = partial + ((size_t)b * nq + q) * KK;
-#pragma unroll
-    for (int r = 0; r < E; ++r) dst[r * 32 + lane] = top[r];
-  }
+  scan_candidates<E, true>(pv, qs, scratch, q, nq, k, blockIdx.x, gridDim.x, probes, n_probe, list_off,
+                           list_rows, n_indexed, exclude_tag, partial, s_pref, s_base, codes, scales);
 }
 
 template <int E>
@@ -593,9 +561,10 @@ __device__ __forceinline__ void fold_lists(const u64* lists, int n, size_t strid
 // next launch.
 struct LookupSync { unsigned ticket, scanned, ready, candidates, finished, pad[3]; };
 
-template <int E>
+template <int E, bool k8>
 __global__ void __launch_bounds__(kNormThreads, 2)
-index_lookup_kernel(PoolView pv, const uint16_t* __restrict__ cent_keys, int n_lists,
+index_lookup_kernel(PoolView pv, const uint8_t* __restrict__ codes, const float* __restrict__ scales,
+                    const uint16_t* __restrict__ cent_keys, int n_lists,
                     const uint16_t* __restrict__ q_raw, int nq, int k, int g1, int n_probe,
                     int32_t* probes, u64* cpartial, LookupSync* sync,
                     const int32_t* __restrict__ list_off, const int32_t* __restrict__ list_rows,
@@ -695,8 +664,8 @@ index_lookup_kernel(PoolView pv, const uint16_t* __restrict__ cent_keys, int n_l
     const int woke = s_flag;
     __syncthreads();                                     // s_flag is written again below
     if (woke) {
-      scan_candidates<E>(pv, qs, scratch, q, nq, k, b, g2, probes, n_probe, list_off, list_rows,
-                         n_indexed, exclude_tag, partial, s_pref, s_base);
+      scan_candidates<E, k8>(pv, qs, scratch, q, nq, k, b, g2, probes, n_probe, list_off, list_rows,
+                             n_indexed, exclude_tag, partial, s_pref, s_base, codes, scales);
     } else if (threadIdx.x < 32) {                         // gave up: an empty list
       constexpr int KK = 32 * E;
 #pragma unroll
@@ -761,8 +730,9 @@ static cudaError_t launch_scan_ids(const PoolView& pv, const uint16_t* q, int nq
                     probes, n_probe, list_off, list_rows, n_indexed, ex, partial, q_valid, stats);
 }
 
-template <int E>
-static cudaError_t launch_index_lookup(const PoolView& pv, const uint16_t* cent_keys, int n_lists,
+template <int E, bool k8>
+static cudaError_t launch_index_lookup(const PoolView& pv, const uint8_t* codes, const float* scales,
+                                       const uint16_t* cent_keys, int n_lists,
                                        const uint16_t* q, int nq, int k, int g1, int g2, int n_probe,
                                        int32_t* probes, u64* cpartial, LookupSync* sync,
                                        const int32_t* list_off, const int32_t* list_rows,
@@ -770,8 +740,8 @@ static cudaError_t launch_index_lookup(const PoolView& pv, const uint16_t* cent_
                                        DeviceStats* stats, const GatherParams& gp,
                                        const oilbird_query_out& out, cudaStream_t st) {
   const size_t smem = (size_t)pv.d * 2 + (size_t)(kNormThreads / 32) * 32 * E * sizeof(u64);
-  return launch_pdl(index_lookup_kernel<E>, dim3(g1 + g2, nq), dim3(kNormThreads), smem, st, pv,
-                    cent_keys, n_lists, q, nq, k, g1, n_probe, probes, cpartial, sync, list_off,
+  return launch_pdl(index_lookup_kernel<E, k8>, dim3(g1 + g2, nq), dim3(kNormThreads), smem, st, pv,
+                    codes, scales, cent_keys, n_lists, q, nq, k, g1, n_probe, probes, cpartial, sync, list_off,
                     list_rows, n_indexed, ex, partial, stats, gp, out);
 }
 
@@ -786,9 +756,12 @@ cudaError_t preload_index_kernels() {
   if ((e = preload_kernel(scan_ids_e4m3_kernel<1>, true)) != cudaSuccess) return e;
   if ((e = preload_kernel(scan_ids_e4m3_kernel<2>, true)) != cudaSuccess) return e;
   if ((e = preload_kernel(scan_ids_e4m3_kernel<4>, true)) != cudaSuccess) return e;
-  if ((e = preload_kernel(index_lookup_kernel<1>, true)) != cudaSuccess) return e;
-  if ((e = preload_kernel(index_lookup_kernel<2>, true)) != cudaSuccess) return e;
-  if ((e = preload_kernel(index_lookup_kernel<4>, true)) != cudaSuccess) return e;
+  if ((e = preload_kernel(index_lookup_kernel<1, false>, true)) != cudaSuccess) return e;
+  if ((e = preload_kernel(index_lookup_kernel<2, false>, true)) != cudaSuccess) return e;
+  if ((e = preload_kernel(index_lookup_kernel<4, false>, true)) != cudaSuccess) return e;
+  if ((e = preload_kernel(index_lookup_kernel<1, true>, true)) != cudaSuccess) return e;
+  if ((e = preload_kernel(index_lookup_kernel<2, true>, true)) != cudaSuccess) return e;
+  if ((e = preload_kernel(index_lookup_kernel<4, true>, true)) != cudaSuccess) return e;
   if ((e = preload_kernel(scan_ids_kernel<1>, true)) != cudaSuccess) return e;
   if ((e = preload_kernel(scan_ids_kernel<2>, true)) != cudaSuccess) return e;
   return preload_kernel(scan_ids_kernel<4>, true);
@@ -1034,7 +1007,7 @@ int oilbird_index_query(oilbird_index_t* ix, const void* q_bf16, int32_t nq, int
   const int kk = list_len(pr->k);
   PoolView pv = pool_view(p);
   const uint16_t* q = (const uint16_t*)q_bf16;
-  if (nq <= kLookupMaxNq && n_probe <= 32 && pr->path == OILBIRD_PATH_AUTO && !p->r.e4m3) {
+  if (nq <= kLookupMaxNq && n_probe <= 32 && pr->path == OILBIRD_PATH_AUTO) {
     // small batches: centroid scan, probes and candidate scan in one launch, then the merge
     if (preload_all_kernels() != cudaSuccess) return OILBIRD_ECUDA;
     // Twice the CTAs that fit at once (two per SM): the first half takes the centroids and
@@ -1049,13 +1022,13 @@ int oilbird_index_query(oilbird_index_t* ix, const void* q_bf16, int32_t nq, int
     if (g1 > ix->cent->r.max_lists) g1 = ix->cent->r.max_lists;
     if (g2 > p->r.max_lists) g2 = p->r.max_lists;
     cudaError_t e;
-#define LOOKUP(E)                                                                                     \
-    launch_index_lookup<E>(pv, ix->cent->keys, ix->n_lists, q, nq, pr->k, g1, g2, n_probe, ix->probe_idx, \
-                           ix->cent->partial, ix->sync, ix->list_off, ix->list_rows,                  \
-                           (int)ix->n_indexed, pr->exclude_tag, p->partial, p->stats, gp, *out, st)
-    if (kk == 32) e = LOOKUP(1);
-    else if (kk == 64) e = LOOKUP(2);
-    else e = LOOKUP(4);
+#define LOOKUP(E, K8)                                                                             \
+    launch_index_lookup<E, K8>(pv, p->codes, p->scales, ix->cent->keys, ix->n_lists, q, nq, pr->k,    \
+                               g1, g2, n_probe, ix->probe_idx, ix->cent->partial, ix->sync,           \
+                               ix->list_off, ix->list_rows, (int)ix->n_indexed, pr->exclude_tag,      \
+                               p->partial, p->stats, gp, *out, st)
+    if (p->r.e4m3) e = kk == 32 ? LOOKUP(1, true) : (kk == 64 ? LOOKUP(2, true) : LOOKUP(4, true));
+    else e = kk == 32 ? LOOKUP(1, false) : (kk == 64 ? LOOKUP(2, false) : LOOKUP(4, false));
 #undef LOOKUP
     if (e != cudaSuccess) return index_fail(e, "lookup launch");
     p->launches += 1;

@@ -245,7 +245,7 @@ def test_index_over_an_8bit_pool_matches_the_oracle():
     (fp32(value(code) * scale), rounded to bf16 as a query), candidates are scored by the 8-bit
     pool's own rule, training takes the means of the dequantised elements."""
     w = W.C1.scaled(n_rows=6000, nq=5, d=256, k=8, cont_len=4, n_centroids=24, rows_per_trace=500, seed=41)
-    pool, ora = fill_both(w, key_format="e4m3", spare_rows=300, max_nq=16)
+    pool, ora = fill_both(w, key_format="e4m3", spare_rows=300, max_nq=16, max_k=128)
     assign = np.concatenate([w.trace_assign(t, "cuda").cpu().numpy() for t in range(w.num_traces)])[: w.n_rows]
     first = [int(np.nonzero(assign == c)[0][0]) for c in range(24)]      # one row of every cluster
     keys_raw = torch.cat([st for st, _, _ in w.traces("cuda")])[: w.n_rows]
@@ -264,6 +264,17 @@ def test_index_over_an_8bit_pool_matches_the_oracle():
     for i in range(2):
         a, b = gix.query(q[i:i + 1].contiguous(), 24, pr).cpu(), pool.query(q[i:i + 1].contiguous(), pr).cpu()
         assert torch.equal(a.idx, b.idx) and torch.equal(a.score, b.score) and torch.equal(a.cont_tok, b.cont_tok)
+    # a single query's lookup is one launch here too: same neighbours as the separate launches
+    launches = pool.launch_count
+    for n_probe in (1, 3, 30):
+        for k in (1, 8, 100):
+            q1 = q[2:3].contiguous()
+            one = gix.query(q1, n_probe, fixed(k, 4))
+            check_index_query(one, oix, W.to_bits(q1), n_probe, fixed(k, 4))
+            sep = gix.query(q1, n_probe, fixed(k, 4, path=B.PATH_GEMV)).cpu()
+            assert torch.equal(one.cpu().idx, sep.idx) and torch.equal(one.cpu().score, sep.score)
+            assert torch.equal(one.cpu().cont_tok, sep.cont_tok)
+    assert pool.launch_count - launches == 9 * (1 + 2)
     # the tail, then a refresh; exclusion tags
     g = torch.Generator(device="cuda").manual_seed(3)
     st = torch.randn(200, w.d, generator=g, device="cuda").to(torch.bfloat16)

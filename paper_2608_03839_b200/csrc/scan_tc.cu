@@ -944,7 +944,9 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap key_map,
       }
       }
       // The agreed bound tightens like 1/t: after the first tiles every fourth exchange is enough
-      if (use_xchg && (iter < 4 || (iter & 3u) == 3u)) {
+      // (not behind a CTA's last tile: nothing of its own is left to filter, and the others
+      // are at their last tiles too)
+      if (use_xchg && (iter < 4 || (iter & 3u) == 3u) && tile + n_units < n_tiles) {
         // publish this CTA's best per query (the owner warp's lists are quiescent here) ...
         for (int q = ew + 4 * lane; q < nq_c; q += 128) {
           const u64 top = lists.load(q, 0);

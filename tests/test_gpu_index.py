@@ -175,6 +175,26 @@ def test_lookups_in_one_launch_match_the_oracle_and_the_separate_launches(nq):
     assert pool.stats()["stalled"] == 0 and pool.status() == B.OK
 
 
+@pytest.mark.parametrize("key_format", ["bf16", "e4m3"])
+def test_one_launch_lookup_at_the_widest_rows_and_longest_lists(key_format):
+    # d = 8192 (a row is more than one round of a lane's loads), k up to 128 (four registers of
+    # list per lane), 32 probes (the most the one-launch form takes)
+    w = W.C1.scaled(n_rows=3000, d=8192, nq=1, k=8, cont_len=4, n_centroids=40, rows_per_trace=500, seed=23)
+    pool, ora, gix, oix = build_both(w, 40, seed=6, spare_rows=100, max_k=128, key_format=key_format)
+    gix.refresh(); oix.refresh()
+    same_lists(gix, oix)
+    q, _ = w.queries("cuda")
+    launches = pool.launch_count
+    for n_probe, k in ((1, 64), (7, 128), (32, 128), (32, 33)):
+        pr = fixed(k, 4)
+        one = gix.query(q, n_probe, pr)
+        check_index_query(one, oix, W.to_bits(q), n_probe, pr)
+        sep = gix.query(q, n_probe, fixed(k, 4, path=B.PATH_GEMV)).cpu()
+        assert torch.equal(one.cpu().idx, sep.idx) and torch.equal(one.cpu().score, sep.score)
+    assert pool.launch_count - launches == 4 * (1 + 2)
+    assert pool.stats()["stalled"] == 0
+
+
 def test_index_after_eviction_needs_a_reset():
     w = W.C1.scaled(n_rows=2000, d=128, nq=3, k=4, cont_len=2, rows_per_trace=250)
     pool, ora, gix, oix = build_both(w, 16, spare_rows=1000)

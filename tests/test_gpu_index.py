@@ -46,7 +46,11 @@ def check_index_query(out, oidx: OracleIndex, q_bits, n_probe, params, exclude=N
             if abs(float(ref.score[q, 0]) - params.theta) > GAP:
                 assert o.fired[q] == ref.fired[q]
         for j in range(k):
-            dep = params.cont_len if (o.fired[q] and got[j] >= 0) else 0
+            dep = 0
+            if o.fired[q] and got[j] >= 0:
+                dep = (params.cont_len if params.depth_mode == B.DEPTH_FIXED
+                       else oracle.depth_by_rank(j, params.tier_depth) if params.depth_mode == B.DEPTH_RANKED
+                       else oracle.depth(float(score[q, j]), params.tier_thr, params.tier_depth))
             tok, n = oidx.pool.gather_one(int(got[j]), dep, params.offset, params.cont_len)
             assert o.cont_len[q, j] == n and np.array_equal(o.cont_tok[q, j].numpy(), tok)
     return ref

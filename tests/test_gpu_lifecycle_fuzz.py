@@ -61,7 +61,7 @@ def test_random_life_cycle(fmt, seed):
     def params(nq):
         k = int(rng.choice([1, 4, 8, 17, 32]))
         pr = B.QueryParams(k=k, theta=float(rng.choice([-2.0, 0.5, 0.8])),
-                           depth_mode=int(rng.choice([B.DEPTH_FIXED, B.DEPTH_TIERED])),
+                           depth_mode=int(rng.choice([B.DEPTH_FIXED, B.DEPTH_TIERED, B.DEPTH_RANKED])),
                            cont_len=int(rng.choice([1, 4, 16])), offset=int(rng.choice([0, 1, 2])))
         if fmt == "bf16" and nq >= 1:
             paths = [B.PATH_AUTO, B.PATH_GEMV, B.PATH_TENSOR] + ([B.PATH_MMA] * 2 if d % 128 == 0 else [])
@@ -140,3 +140,75 @@ def test_random_life_cycle(fmt, seed):
         assert len(pool) == len(ora) and pool.num_traces == ora.num_traces
     same_store(pool, ora)
     assert pool.stats()["stalled"] == 0
+
+
+@pytest.mark.parametrize("fmt", ["bf16", "e4m3"])
+@pytest.mark.parametrize("seed", range(4))
+def test_random_life_cycle_with_an_index(fmt, seed):
+    """Appends, refreshes, lookups (one launch and separate launches), training, evictions and
+    resets in a seeded order, the coarse index and its oracle side by side: lists identical
+    after every refresh, answers under the acceptance rule on the candidate rows."""
+    from oracle.index import OracleIndex
+    from test_gpu_index import check_index_query, same_lists
+    rng = np.random.default_rng(2000 + seed)
+    d = int(rng.choice([128, 512]))
+    cap, n_lists = 5000, 12
+    pool = B.Pool(d, cap, max_nq=8, max_k=32, max_traces=200, key_format=fmt)
+    ora = OraclePool(d, fmt)
+    g = torch.Generator(device="cuda").manual_seed(50 + seed)
+    cent = torch.randn(n_lists, d, generator=g, device="cuda")
+    cent_bf = cent.to(torch.bfloat16).contiguous()
+    gix, oix = B.Index(pool, cent_bf), OracleIndex(ora, W.to_bits(cent_bf))
+    tag = [1]
+
+    def rows(n):
+        # well inside a cluster: the best two centroids of a row stay apart, so the lists
+        # cannot depend on the accumulation order
+        c = torch.randint(0, n_lists, (n,), generator=g, device="cuda")
+        return (cent[c] + 0.15 * torch.randn(n, d, generator=g, device="cuda")).to(torch.bfloat16), \
+            torch.randint(0, 5000, (n,), generator=g, device="cuda", dtype=torch.int32)
+
+    for _ in range(45):
+        op = rng.choice(["append", "refresh", "lookup", "lookup", "train", "evict", "reset"],
+                        p=[0.3, 0.15, 0.2, 0.2, 0.05, 0.07, 0.03])
+        if op == "append":
+            n = int(rng.choice([1, 8, 60, 300]))
+            if len(pool) + n > cap or pool.num_traces + 1 > 190:
+                op = "evict"
+            else:
+                st, tk = rows(n)
+                pool.append(st, tk, tag=tag[0])
+                ora.append(W.to_bits(st), tk.cpu().numpy(), tag=tag[0])
+                tag[0] += 1
+        if op == "refresh":
+            gix.refresh(); oix.refresh()
+            assert len(gix) == len(pool)
+            same_lists(gix, oix)
+        elif op == "lookup" and len(ora):
+            nq = int(rng.choice([1, 1, 2, 5]))
+            q = rows(nq)[0]
+            pr = B.QueryParams(k=int(rng.choice([1, 8, 32])), theta=float(rng.choice([-2.0, 0.8])),
+                               depth_mode=int(rng.choice([B.DEPTH_FIXED, B.DEPTH_TIERED, B.DEPTH_RANKED])),
+                               cont_len=int(rng.choice([2, 16])),
+                               path=int(rng.choice([B.PATH_AUTO, B.PATH_AUTO, B.PATH_GEMV])))
+            n_probe = int(rng.choice([1, 3, n_lists, 40]))
+            check_index_query(gix.query(q, n_probe, pr), oix, W.to_bits(q), n_probe, pr)
+        elif op == "train" and len(ora):
+            gix.train(1); oix.train(1)
+            assert np.array_equal(gix.centroids(), oix.cent_raw)
+            same_lists(gix, oix)
+        elif op == "evict" and pool.num_traces:
+            nt = int(rng.integers(1, pool.num_traces + 1))
+            assert pool.evict_oldest(nt) == ora.evict_oldest(nt)
+            if len(gix) > 0:
+                with pytest.raises(B.OilbirdError):
+                    gix.refresh()                  # row numbers changed: a reset comes first
+            gix.reset(); oix.reset()
+            gix.refresh(); oix.refresh()
+            same_lists(gix, oix)
+        elif op == "reset":
+            pool.reset(); ora.reset()
+            gix.reset(); oix.reset()
+    gix.refresh(); oix.refresh()
+    same_lists(gix, oix)
+    assert pool.stats()["stalled"] == 0 and pool.status() == B.OK

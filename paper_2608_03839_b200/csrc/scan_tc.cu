@@ -851,8 +851,12 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap key_map,
         __threadfence();
         epilogue_bar();
         if (et == 0) atomicAdd(&arrivals[0], 1u);
-        for (int q = ew; q < nq_c; q += 4) {
-          if ((q0 + q) % (int)gridDim.x != (int)blockIdx.x) continue;     // warp-uniform
+        // (the queries this CTA answers for, q0 + q = blockIdx.x mod gridDim.x, dealt out to
+        // the four warps in turn: they are a stride of gridDim.x apart, which is often a
+        // multiple of four)
+        const int q_first = (((int)blockIdx.x - q0) % (int)gridDim.x + (int)gridDim.x) % (int)gridDim.x;
+        for (int j = 0, q = q_first; q < nq_c; ++j, q += (int)gridDim.x) {
+          if ((j & 3) != ew) continue;                                    // warp-uniform
           rendezvous_wait(&arrivals[0], gridDim.x);
           const float kth_best = kth_largest_best(lmax, q0 + q, k, lane);
           if (lane == 0 && kth_best > -INFINITY && kth_best > __ldcg(&gthr[q0 + q]))
@@ -954,8 +958,9 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap key_map,
         }
         // ... and, for the queries this CTA is responsible for, agree on the bound: the k-th
         // largest of all CTAs' bests, by k rounds of warp-wide maximum extraction
-        for (int q = ew; q < nq_c; q += 4) {
-          if ((q0 + q) % (int)gridDim.x != (int)blockIdx.x) continue;     // warp-uniform
+        const int q_first = (((int)blockIdx.x - q0) % (int)gridDim.x + (int)gridDim.x) % (int)gridDim.x;
+        for (int j = 0, q = q_first; q < nq_c; ++j, q += (int)gridDim.x) {
+          if ((j & 3) != ew) continue;                                    // warp-uniform
           const float kth_best = kth_largest_best(lmax, q0 + q, k, lane);
           if (lane == 0 && kth_best > -INFINITY && kth_best > __ldcg(&gthr[q0 + q]))
             __stcg(&gthr[q0 + q], kth_best);

@@ -272,6 +272,17 @@ __device__ __forceinline__ void tc_ld16(uint32_t taddr, float (&v)[16]) {
 __device__ __forceinline__ void epilogue_bar() {      // the 128 epilogue threads only
   asm volatile("bar.sync 1, 128;" ::: "memory");
 }
+// the same barrier, returning whether any of the 128 threads brought a true flag
+__device__ __forceinline__ bool epilogue_bar_or(bool flag) {
+  uint32_t any;
+  asm volatile(
+      "{\n\t.reg .pred p_in, p_out;\n\t"
+      "setp.ne.u32 p_in, %1, 0;\n\t"
+      "bar.red.or.pred p_out, 1, 128, p_in;\n\t"
+      "selp.u32 %0, 1, 0, p_out;\n\t}"
+      : "=r"(any) : "r"((uint32_t)flag) : "memory");
+  return any != 0;
+}
 
 // Shared-memory matrix descriptor of a K-major bf16 tile whose rows are 128 bytes wide
 // and 128B-swizzled (what the TMA box above produces): 8-row groups 1024 bytes apart.
@@ -335,8 +346,6 @@ struct TcShared {
   uint32_t tmem_base;
   int abort_flag;
   int epi_go;
-  int q_total;                  // nonzero: candidates were queued in the current round
-  int q_cnt[kColsPerRound];     // ... per score column of the round
 };
 
 // Per-query candidate lists of one CTA: kk packed 64-bit keys per query, descending, empty
@@ -372,17 +381,18 @@ constexpr int kDrainQ = kColsPerRound / 4;      // queries per warp and round
 constexpr int kCrowd = 8;
 
 template <int E>
-__device__ __forceinline__ void drain_round(const ListStore& lists, int kk, const u64* q_key,
-                                            const int* q_cnt, int c0, int ew, int nq_c, int k,
-                                            float* thr_s, int lane) {
+__device__ __forceinline__ void drain_cols(const ListStore& lists, const u64* q_key, int q_cap,
+                                           const int* q_cnt, const int (&cols)[kDrainQ], int k,
+                                           float* thr_s, int lane) {
   u64 v[kDrainQ][E];
   u64 kth[kDrainQ];
   int n[kDrainQ];
   int n_max = 0, crowd_max = 0;
 #pragma unroll
   for (int u = 0; u < kDrainQ; ++u) {
-    const int j = ew + 4 * u, q = c0 + j;
-    n[u] = q < nq_c ? q_cnt[j] : 0;
+    const int q = cols[u];
+    n[u] = q >= 0 ? q_cnt[q] : 0;
+    n[u] = n[u] > q_cap ? q_cap : n[u];          // pushes beyond the queue's end were not stored
     if (n[u] > 0) {
 #pragma unroll
       for (int r = 0; r < E; ++r) v[u][r] = lists.load(q, r * 32 + lane);
@@ -404,7 +414,7 @@ __device__ __forceinline__ void drain_round(const ListStore& lists, int kk, cons
 #pragma unroll
       for (int r = 0; r < E; ++r) {
         const int i = i0 + r * 32 + lane;
-        const u64 key = (n[u] >= kCrowd && i < n[u]) ? q_key[(ew + 4 * u) * kTileM + i] : 0;
+        const u64 key = (n[u] >= kCrowd && i < n[u]) ? q_key[(size_t)cols[u] * q_cap + i] : 0;
         b[u][r] = key > kth[u] ? key : 0;
       }
     }
@@ -418,7 +428,7 @@ __device__ __forceinline__ void drain_round(const ListStore& lists, int kk, cons
     for (int u = 0; u < kDrainQ; ++u) {
       // every queued candidate beat the threshold it was filtered with; kth only settles
       // ties and is refreshed after the round (a worse key just falls off the end)
-      u64 key = (n[u] < kCrowd && i < n[u]) ? q_key[(ew + 4 * u) * kTileM + i] : 0;
+      u64 key = (n[u] < kCrowd && i < n[u]) ? q_key[(size_t)cols[u] * q_cap + i] : 0;
       key = key > kth[u] ? key : 0;
       warp_sorted_insert<E>(v[u], key, lane);
     }
@@ -426,7 +436,7 @@ __device__ __forceinline__ void drain_round(const ListStore& lists, int kk, cons
 #pragma unroll
   for (int u = 0; u < kDrainQ; ++u) {
     if (n[u] > 0) {
-      const int q = c0 + ew + 4 * u;
+      const int q = cols[u];
 #pragma unroll
       for (int r = 0; r < E; ++r) lists.store(q, r * 32 + lane, v[u][r]);
       const u64 nk = warp_list_get<E>(v[u], k - 1);
@@ -434,6 +444,40 @@ __device__ __forceinline__ void drain_round(const ListStore& lists, int kk, cons
       if (lane == 0 && nk != 0) thr_s[q] = fmaxf(thr_s[q], candidate_score(nk));
     }
   }
+}
+
+// Warp ew folds everything queued for its queries (ew, ew + 4, ...) into their lists, four
+// queries at a time, and empties those queues.  Candidates wait in per-query queues from the
+// round that found them to the end of their tile (or until a queue is full): a list kept in
+// global memory costs a round trip to L2 to fetch and one to put back, and draining after
+// every round of sixteen columns paid that for the one or two queries of the round that had
+// a candidate (256 queries, k = 64: 198 of 224 rounds drained, 3,650 cycles each, the
+// epilogue busy for 840,000 of the kernel's 1,090,000 cycles and the MMAs waiting for it).
+template <int E>
+__device__ __forceinline__ void flush_queues(const ListStore& lists, const u64* q_key, int q_cap,
+                                             int* q_cnt, int n_pad, int ew, int k, float* thr_s,
+                                             int lane) {
+  const int per_warp = n_pad >> 2;
+  for (int base = 0; base < per_warp; base += 32) {
+    const int i = base + lane;
+    const int cnt = i < per_warp ? q_cnt[ew + 4 * i] : 0;
+    unsigned m = __ballot_sync(0xffffffffu, cnt > 0);
+    while (m) {
+      int cols[kDrainQ];
+#pragma unroll
+      for (int u = 0; u < kDrainQ; ++u) {
+        cols[u] = m ? ew + 4 * (base + __ffs(m) - 1) : -1;
+        m &= m - 1;
+      }
+      drain_cols<E>(lists, q_key, q_cap, q_cnt, cols, k, thr_s, lane);
+      __syncwarp();
+      int mine = -1;
+#pragma unroll
+      for (int u = 0; u < kDrainQ; ++u) mine = lane == u ? cols[u] : mine;
+      if (mine >= 0) q_cnt[mine] = 0;
+    }
+  }
+  __syncwarp();
 }
 
 // The k-th largest of the CTAs' published best scores for query q (one per CTA), by k rounds
@@ -534,10 +578,12 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap key_map,
                              : reinterpret_cast<u64*>(list_mem);
   lists.kk = kk;
   u64* q_key = reinterpret_cast<u64*>(list_mem + (lists.global ? 0 : (size_t)nq_c * kk * 8));
-                                                               // [kColsPerRound][kTileM]
+                                                               // [n_pad][q_cap]
   uint64_t* s_ex = reinterpret_cast<uint64_t*>(q_key + kQueueCap);              // [n_pad]
   float* thr_s = reinterpret_cast<float*>(s_ex + n_pad);                        // [n_pad]
   uint32_t* s_qmax = reinterpret_cast<uint32_t*>(thr_s + n_pad);                // [n_pad]
+  int* q_cnt = reinterpret_cast<int*>(s_qmax + n_pad);                          // [n_pad]
+  const int q_cap = kQueueCap / n_pad;       // queue slots per query (8 at 256 queries)
   // Cross-CTA threshold exchange (global memory, reset to -inf by the query preparation):
   // lmax[q][cta] = best score CTA `cta` has seen for query q; gthr[q] = a score that at
   // least k distinct rows of the pool are known to reach, namely the k-th largest of the
@@ -572,8 +618,6 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap key_map,
     }
     mbar_init(&sh.drain, 1);
     sh.abort_flag = 0;
-    sh.q_total = 0;
-    for (int j = 0; j < kColsPerRound; ++j) sh.q_cnt[j] = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 1) {   // TMEM allocation is a whole-warp operation (the same warp of both CTAs of a pair)
@@ -596,6 +640,7 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap key_map,
   for (int i = threadIdx.x; i < n_pad; i += (int)blockDim.x) {
     thr_s[i] = i < nq_c ? -INFINITY : INFINITY;        // padded columns never pass the filter
     s_qmax[i] = 0u;
+    q_cnt[i] = 0;
     s_ex[i] = (exclude_tag && i < nq_c) ? exclude_tag[q0 + i] : 0;
   }
   for (int i = threadIdx.x; i < nq_c * kk; i += (int)blockDim.x) lists.store(i / kk, i % kk, 0);
@@ -921,32 +966,38 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap key_map,
         // the columns in the same order would serialise on one counter at a time.
         const int rot = lane & (kColsPerRound - 1);
         pass = ((pass >> rot) | (pass << (kColsPerRound - rot))) & ((1u << kColsPerRound) - 1u);
-        while (pass) {
-          const int j = (__ffs(pass) - 1 + rot) & (kColsPerRound - 1);
-          pass &= pass - 1;
-          const int q = c0 + j;
-          if (s_ex[q] != 0 && tag == s_ex[q]) continue;           // same-prompt trace: skipped
-          float vj = v[0];
+        // Passing scores go into their query's queue; the queues are folded into the lists at
+        // the end of the tile, or at once when one is full (the threads it turned away keep
+        // their candidates and queue them again behind the flush).
+        for (;;) {
+          uint32_t retry = 0;
+          while (pass) {
+            const uint32_t low = pass & (0u - pass);
+            const int j = (__ffs(pass) - 1 + rot) & (kColsPerRound - 1);
+            pass &= pass - 1;
+            const int q = c0 + j;
+            if (s_ex[q] != 0 && tag == s_ex[q]) continue;         // same-prompt trace: skipped
+            float vj = v[0];
 #pragma unroll
-          for (int i = 1; i < kColsPerRound; ++i) vj = j == i ? v[i] : vj;
-          const int pos = atomicAdd(&sh.q_cnt[j], 1);
-          q_key[j * kTileM + pos] = pack_candidate(vj, (uint32_t)row);
-          sh.q_total = 1;
-        }
-        epilogue_bar();
-        if (sh.q_total > 0) {
-          // drain: warp ew folds the candidates of columns ew, ew+4, ... into their lists
-          if (kk == 32) drain_round<1>(lists, kk, q_key, sh.q_cnt, c0, ew, nq_c, k, thr_s, lane);
-          else if (kk == 64) drain_round<2>(lists, kk, q_key, sh.q_cnt, c0, ew, nq_c, k, thr_s, lane);
-          else drain_round<4>(lists, kk, q_key, sh.q_cnt, c0, ew, nq_c, k, thr_s, lane);
-          __syncwarp();
-          if (lane < kDrainQ) sh.q_cnt[ew + 4 * lane] = 0;
-          epilogue_bar();
-          if (et == 0) sh.q_total = 0;
-          epilogue_bar();
+            for (int i = 1; i < kColsPerRound; ++i) vj = j == i ? v[i] : vj;
+            const int pos = atomicAdd(&q_cnt[q], 1);
+            if (pos < q_cap) q_key[(size_t)q * q_cap + pos] = pack_candidate(vj, (uint32_t)row);
+            else retry |= low;
+          }
+          if (!epilogue_bar_or(retry != 0)) break;                // every candidate found room
+          if (kk == 32) flush_queues<1>(lists, q_key, q_cap, q_cnt, n_pad, ew, k, thr_s, lane);
+          else if (kk == 64) flush_queues<2>(lists, q_key, q_cap, q_cnt, n_pad, ew, k, thr_s, lane);
+          else flush_queues<4>(lists, q_key, q_cap, q_cnt, n_pad, ew, k, thr_s, lane);
+          epilogue_bar();                                         // the queues are empty again
+          pass = retry;
         }
       }
       }
+      // the tile's candidates, into the lists (the last round's barrier has seen them queued)
+      if (kk == 32) flush_queues<1>(lists, q_key, q_cap, q_cnt, n_pad, ew, k, thr_s, lane);
+      else if (kk == 64) flush_queues<2>(lists, q_key, q_cap, q_cnt, n_pad, ew, k, thr_s, lane);
+      else flush_queues<4>(lists, q_key, q_cap, q_cnt, n_pad, ew, k, thr_s, lane);
+      epilogue_bar();
       // The agreed bound tightens like 1/t: after the first tiles every fourth exchange is enough
       // (not behind a CTA's last tile: nothing of its own is left to filter, and the others
       // are at their last tiles too)
@@ -1085,7 +1136,7 @@ static const CUtensorMap* tc_q_map(TcCache* c, int n_pad) {
 
 static size_t tc_fixed_smem(int nq_c, int n_pad, int kk, bool global_lists) {
   return (global_lists ? 0 : (size_t)nq_c * kk * 8) + (size_t)kQueueCap * 8 +
-         (size_t)n_pad * (8 + 4 + 4) + 1024 /* alignment slack */;
+         (size_t)n_pad * (8 + 4 + 4 + 4) + 1024 /* alignment slack */;
 }
 
 // How a call is cut up: queries per pass, where the lists live, key tiles per query tile,

@@ -92,8 +92,8 @@ constexpr int kTileM = 128;            // key rows per tile = TMEM lanes
 constexpr int kBlockK = 64;
 constexpr int kATileBytes = kTileM * kBlockK * 2;   // 16 KB
 constexpr int kCodeTileBytes = kTileM * kBlockK;    // the same tile as E4M3 codes: 8 KB
-constexpr int kColsPerRound = 16;      // score columns filtered between two drains
-constexpr int kQueueCap = kTileM * kColsPerRound;
+constexpr int kColsPerRound = 16;      // score columns read from TMEM and filtered at a time
+constexpr int kQueueCap = kTileM * kColsPerRound;   // candidate slots, shared out among the queries
 constexpr int kMaxStages = 8;
 
 // Lists stay in shared memory if this many ring stages still fit beside them.

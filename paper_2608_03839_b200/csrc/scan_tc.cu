@@ -1175,10 +1175,11 @@ static TcPlan tc_plan(int nq, int k, int n_tiles128, int num_sms, size_t smem_li
     p.n_pad = (nq + 31) / 32 * 32;
     p.pair = 1; p.global_lists = 1; p.stages = 0;
     // two tiles per CTA and query tile: with both accumulator sets up to 128 columns, with
-    // one set up to 224 (what the shared query tile saves outweighs the epilogue no longer
+    // one set above (what the shared query tile saves outweighs the epilogue no longer
     // overlapping the MMAs: C5 nq = 160 3.94 -> 3.63 ms, nq = 192 4.20 -> 3.93, nq = 224
-    // 4.46 -> 4.35; at 256 columns it does not: 4.72 -> 4.71)
-    if (p.n_pad <= 224 && n_tiles128 >= 8 * num_sms) {
+    // 4.46 -> 4.35; at 256 columns it did not, 4.72 -> 4.71, until the epilogue folded its
+    // candidates once per tile: 4.66 -> 4.48 ms)
+    if (p.n_pad <= 256 && n_tiles128 >= 8 * num_sms) {
       p.mt = 2;
       p.n_bufs = 2 * 2 * p.n_pad <= 512 ? 2 : 1;
       if (tc_fits(p.n_pad, list_len(k), 2, true, 3, smem_limit, &p.stages, true)) return p;

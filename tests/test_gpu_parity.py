@@ -618,9 +618,10 @@ def test_pairs_of_ctas_on_batches_above_128_queries(nq, k):
     assert pool.stats()["stalled"] == 0
 
 
-@pytest.mark.parametrize("nq,k", [(97, 8), (128, 64), (120, 1), (160, 16), (224, 64), (129, 8)])
-def test_pairs_of_ctas_with_two_tiles_each_from_97_to_224_queries(nq, k):
-    """97 to 224 queries on a pool of at least eight tiles per SM: a pair of CTAs takes macro
+@pytest.mark.parametrize("nq,k", [(97, 8), (128, 64), (120, 1), (160, 16), (224, 64), (129, 8),
+                                  (256, 64), (241, 128)])
+def test_pairs_of_ctas_with_two_tiles_each_from_97_to_256_queries(nq, k):
+    """97 to 256 queries on a pool of at least eight tiles per SM: a pair of CTAs takes macro
     tiles of 512 rows (two MMAs over both CTAs per query tile), with two accumulator sets up
     to 128 queries and one above.  Last macro tile with one, two and three of its four
     sub-tiles (partly) filled."""

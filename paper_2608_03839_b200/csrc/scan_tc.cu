@@ -383,7 +383,7 @@ constexpr int kCrowd = 8;
 template <int E>
 __device__ __forceinline__ void drain_cols(const ListStore& lists, const u64* q_key, int q_cap,
                                            const int* q_cnt, const int (&cols)[kDrainQ], int k,
-                                           float* thr_s, int lane) {
+                                           float* thr_s, int lane, int col0) {
   u64 v[kDrainQ][E];
   u64 kth[kDrainQ];
   int n[kDrainQ];
@@ -414,7 +414,7 @@ __device__ __forceinline__ void drain_cols(const ListStore& lists, const u64* q_
 #pragma unroll
       for (int r = 0; r < E; ++r) {
         const int i = i0 + r * 32 + lane;
-        const u64 key = (n[u] >= kCrowd && i < n[u]) ? q_key[(size_t)cols[u] * q_cap + i] : 0;
+        const u64 key = (n[u] >= kCrowd && i < n[u]) ? q_key[(size_t)(cols[u] - col0) * q_cap + i] : 0;
         b[u][r] = key > kth[u] ? key : 0;
       }
     }
@@ -428,7 +428,7 @@ __device__ __forceinline__ void drain_cols(const ListStore& lists, const u64* q_
     for (int u = 0; u < kDrainQ; ++u) {
       // every queued candidate beat the threshold it was filtered with; kth only settles
       // ties and is refreshed after the round (a worse key just falls off the end)
-      u64 key = (n[u] < kCrowd && i < n[u]) ? q_key[(size_t)cols[u] * q_cap + i] : 0;
+      u64 key = (n[u] < kCrowd && i < n[u]) ? q_key[(size_t)(cols[u] - col0) * q_cap + i] : 0;
       key = key > kth[u] ? key : 0;
       warp_sorted_insert<E>(v[u], key, lane);
     }
@@ -456,7 +456,8 @@ __device__ __forceinline__ void drain_cols(const ListStore& lists, const u64* q_
 template <int E>
 __device__ __forceinline__ void flush_queues(const ListStore& lists, const u64* q_key, int q_cap,
                                              int* q_cnt, int n_pad, int ew, int k, float* thr_s,
-                                             int lane) {
+                                             int lane, int col0 = 0) {
+  // col0: the queue of query q starts at slot (q - col0) * q_cap (the round-wide layout below)
   const int per_warp = n_pad >> 2;
   for (int base = 0; base < per_warp; base += 32) {
     const int i = base + lane;
@@ -469,7 +470,7 @@ __device__ __forceinline__ void flush_queues(const ListStore& lists, const u64* 
         cols[u] = m ? ew + 4 * (base + __ffs(m) - 1) : -1;
         m &= m - 1;
       }
-      drain_cols<E>(lists, q_key, q_cap, q_cnt, cols, k, thr_s, lane);
+      drain_cols<E>(lists, q_key, q_cap, q_cnt, cols, k, thr_s, lane, col0);
       __syncwarp();
       int mine = -1;
 #pragma unroll
@@ -923,6 +924,7 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap key_map,
         }
       }
       epilogue_bar();
+      bool long_way = false;                    // (see the rounds below) per tile, all warps alike
       for (int sub = 0; sub < mt; ++sub) {      // sub-tiles in row order: ties stay exact
       const int row = (kPair ? (tile * mt + sub) * 2 + (int)rank : tile * mt + sub) * kTileM + lane_grp * 32 + lane;
       const bool row_ok = row < pv.n_rows;
@@ -967,10 +969,13 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap key_map,
         const int rot = lane & (kColsPerRound - 1);
         pass = ((pass >> rot) | (pass << (kColsPerRound - rot))) & ((1u << kColsPerRound) - 1u);
         // Passing scores go into their query's queue; the queues are folded into the lists at
-        // the end of the tile, or at once when one is full (the threads it turned away keep
-        // their candidates and queue them again behind the flush).
-        for (;;) {
-          uint32_t retry = 0;
+        // the end of the tile.  When a queue is full (thresholds still loose, or a stretch of
+        // rows each better than the last) the tile goes on the long way: everything queued so
+        // far is folded, and from then on a round's candidates go into queues of a whole
+        // sub-tile's depth, which the queue memory holds for the sixteen columns of one round,
+        // and are folded behind the round (sorted in batches of 32*E).
+        uint32_t retry = 0;
+        if (!long_way) {
           while (pass) {
             const uint32_t low = pass & (0u - pass);
             const int j = (__ffs(pass) - 1 + rot) & (kColsPerRound - 1);
@@ -984,12 +989,31 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap key_map,
             if (pos < q_cap) q_key[(size_t)q * q_cap + pos] = pack_candidate(vj, (uint32_t)row);
             else retry |= low;
           }
-          if (!epilogue_bar_or(retry != 0)) break;                // every candidate found room
+          if (!epilogue_bar_or(retry != 0)) continue;             // every candidate found room
           if (kk == 32) flush_queues<1>(lists, q_key, q_cap, q_cnt, n_pad, ew, k, thr_s, lane);
           else if (kk == 64) flush_queues<2>(lists, q_key, q_cap, q_cnt, n_pad, ew, k, thr_s, lane);
           else flush_queues<4>(lists, q_key, q_cap, q_cnt, n_pad, ew, k, thr_s, lane);
-          epilogue_bar();                                         // the queues are empty again
+          epilogue_bar();                                         // every queue is empty
+          long_way = true;
           pass = retry;
+        }
+        bool pushed = false;
+        while (pass) {
+          const int j = (__ffs(pass) - 1 + rot) & (kColsPerRound - 1);
+          pass &= pass - 1;
+          if (s_ex[c0 + j] != 0 && tag == s_ex[c0 + j]) continue;
+          float vj = v[0];
+#pragma unroll
+          for (int i = 1; i < kColsPerRound; ++i) vj = j == i ? v[i] : vj;
+          const int pos = atomicAdd(&q_cnt[c0 + j], 1);           // < 128: one per row at most
+          q_key[(size_t)j * kTileM + pos] = pack_candidate(vj, (uint32_t)row);
+          pushed = true;
+        }
+        if (epilogue_bar_or(pushed)) {
+          if (kk == 32) flush_queues<1>(lists, q_key, kTileM, q_cnt, n_pad, ew, k, thr_s, lane, c0);
+          else if (kk == 64) flush_queues<2>(lists, q_key, kTileM, q_cnt, n_pad, ew, k, thr_s, lane, c0);
+          else flush_queues<4>(lists, q_key, kTileM, q_cnt, n_pad, ew, k, thr_s, lane, c0);
+          epilogue_bar();
         }
       }
       }

@@ -653,6 +653,37 @@ def test_pairs_of_ctas_with_two_tiles_each_from_97_to_256_queries(nq, k):
     assert pool.stats()["stalled"] == 0
 
 
+@pytest.mark.parametrize("nq,k,n_rows", [(16, 16, 40000), (64, 64, 40000), (256, 64, 148 * 128 * 8 + 77),
+                                         (200, 128, 148 * 128 * 8 + 77)])
+def test_rows_that_keep_getting_better_overflow_the_candidate_queues(nq, k, n_rows):
+    """A pool whose every row is closer to the queries than the rows before it: every score
+    is a candidate, the per-query queues of the tensor scan's epilogue fill up in every round
+    and the tiles go the long way (round-wide queues, sorted batches).  Same answers."""
+    d = 128
+    g = torch.Generator(device="cuda").manual_seed(90 + nq)
+    base = torch.randn(1, d, generator=g, device="cuda")
+    noise = torch.randn(n_rows, d, generator=g, device="cuda")
+    wgt = torch.linspace(3.0, 0.2, n_rows, device="cuda").unsqueeze(1)
+    st = (base + wgt * noise).to(torch.bfloat16)
+    pool = B.Pool(d, n_rows, max_nq=256, max_k=128, max_traces=64)
+    ora = OraclePool(d)
+    per = 8192
+    for i in range(0, n_rows, per):
+        rows = st[i:i + per].contiguous()
+        tk = torch.arange(i, i + rows.shape[0], dtype=torch.int32, device="cuda")
+        pool.append(rows, tk, tag=i // per + 1)
+        ora.append(W.to_bits(rows), tk.cpu().numpy(), tag=i // per + 1)
+    q = (base + 0.05 * torch.randn(nq, d, generator=g, device="cuda")).to(torch.bfloat16)
+    pr = fixed(k, 3, theta=-2.0, path=B.PATH_TENSOR)
+    out = pool.query(q, pr)
+    check_query(out, ora, W.to_bits(q), pr)
+    assert int(out.idx[:, 0].min()) > n_rows - 4000          # the best rows are the last ones
+    a = out.cpu()
+    b = pool.query(q, pr).cpu()
+    assert torch.equal(a.idx, b.idx) and torch.equal(a.score, b.score)
+    assert pool.stats()["stalled"] == 0
+
+
 @pytest.mark.parametrize("d", [8, 72, 200, 1000])
 def test_key_widths_that_are_not_multiples_of_the_k_block(d):
     w = W.C1.scaled(nq=3, k=8, n_rows=1500, d=d, cont_len=4, sigma=0.3)

@@ -453,7 +453,9 @@ const char* oilbird_ring_last_error(void);      /* text of the last failing CUDA
  * cont_tok), by the caller's communication library, into one buffer of n_shards equal
  * slices; (4) oilbird_merge_shards, which selects the global top-k by (score descending,
  * global position ascending), applies theta to the merged best and copies the winners'
- * continuations (zero lengths and -1 tokens when not fired).
+ * continuations (zero lengths and -1 tokens when not fired).  Depths are those the shards
+ * assigned: fixed spans and D(s) are the same on a shard as in the whole pool, depth by rank
+ * (OILBIRD_DEPTH_RANKED) is not, so it cannot be used in step (1).
  * gathered: dev, shard s starts at gathered + s*shard_stride; inside a slice, off_gidx
  * (int64 [nq,k], 8-byte aligned), off_score (float [nq,k]), off_len (int32 [nq,k]),
  * off_tok (int32 [nq,k,L]) are byte offsets.  n_shards * k <= 1024.

@@ -133,6 +133,10 @@ class ShardedPool:
 
     def local_record(self, q: torch.Tensor, params: B.QueryParams):
         """Steps 1 and 2: this rank's record (a uint8 buffer) and its layout."""
+        if params.depth_mode == B.DEPTH_RANKED:
+            # a neighbour's depth would be set by its rank on its own shard, not in the merged
+            # answer, and the merge only carries continuations along
+            raise ValueError("copy depth by rank is not offered on a sharded pool")
         q = q.reshape(-1, self.pool.d)
         lay = RecordLayout(q.shape[0], params.k, params.cont_len)
         buf = self._bufs.get(lay)

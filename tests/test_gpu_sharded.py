@@ -56,6 +56,9 @@ def test_sharded_query_equals_single_pool(n_shards, kind):
     assert torch.equal(a.idx.to(torch.int64), b.gidx.cpu())
     assert torch.equal(a.cont_tok, b.cont_tok.cpu()) and torch.equal(a.fired, b.fired.cpu())
     assert torch.allclose(a.score, b.score.cpu(), atol=1e-6)
+    # depth by rank is a matter of the merged order: a shard cannot assign it
+    with pytest.raises(ValueError):
+        sharded_query(shards, q, B.QueryParams(k=w.k, depth_mode=B.DEPTH_RANKED, cont_len=w.cont_len))
 
 
 def test_exact_ties_across_shards_resolve_to_the_lowest_global_position():
